@@ -1,0 +1,304 @@
+"""Pins for the CPU oracle: everything here runs without a GPU and without the CUDA library.
+
+Each test fixes the oracle to something other than itself: hand-worked numbers, the activation
+table, printed closed-form values, brute force on tiny inputs, a library matmul written with W_2 in
+its own [D, H] orientation, or an invariant of the mathematics.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synthetic_inputs as syn
+
+RNG = np.random.default_rng(1234)
+
+
+# ---------------------------------------------------------------- hand-worked examples (Eq. 1)
+W1_EX = np.array([[1.0, 2.0], [-1.0, 0.5], [0.5, 0.5]], np.float32)
+W3_EX = np.array([[2.0, 0.0], [1.0, 1.0], [0.0, -1.0]], np.float32)
+W2_EX = np.array([[1.0, 10.0, 3.0], [-1.0, 20.0, 0.5]], np.float32)  # [D, H] as in Eq. 1
+X_EX = np.array([1.0, -2.0], np.float32)
+B_EX = np.array([4.0, 0.0, 1.0], np.float32)
+
+
+def test_hand_worked_standard_ffn():
+    # z = W1 x + b = [1-4+4, -1-1+0, 0.5-1+1] = [1, -2, 0.5];  u = W3 x = [2, -1, 2]
+    # RELU: h = [1*2, 0, 0.5*2] = [2, 0, 1];  y = W2 h = [2+0+3, -2+0+0.5] = [5, -1.5]
+    for route in ("dense", "sparse"):
+        out = oracle.ffn(X_EX, W3_EX, np.ascontiguousarray(W2_EX.T), "relu", W_g=W1_EX, b_g=B_EX,
+                         route=route)
+        np.testing.assert_array_equal(out["z"], [1.0, -2.0, 0.5])
+        np.testing.assert_array_equal(out["y"], [5.0, -1.5])
+        assert out["n_act"][0] == 2
+        np.testing.assert_array_equal(out["union_mask"], [True, False, True])
+        # squared RELU: a = [1, 0, .25]; h = [2, 0, .5]; y = [2+1.5, -2+.25]
+        out = oracle.ffn(X_EX, W3_EX, np.ascontiguousarray(W2_EX.T), "sqrelu", W_g=W1_EX, b_g=B_EX,
+                         route=route)
+        np.testing.assert_array_equal(out["y"], [3.5, -1.75])
+    # without the bias (the paper's form): z = [-3, -2, -0.5] -> nothing fires, y = 0
+    out = oracle.ffn(X_EX, W3_EX, np.ascontiguousarray(W2_EX.T), "relu", W_g=W1_EX)
+    np.testing.assert_array_equal(out["y"], [0.0, 0.0])
+    assert out["n_act"][0] == 0
+
+
+def test_hand_worked_lopa_gate():
+    V = np.array([[3.0, 4.0], [1.0, 0.0]], np.float32)        # v = V x = [-5, 1]
+    U = np.array([[1.0, 2.0], [-0.2, 0.0], [0.4, -1.0]], np.float32)
+    g_idx, g_sign = np.array([0, 0, 1], np.int32), np.array([1, -1, 1], np.int8)
+    b = np.array([0.0, 0.0, 5.0], np.float32)
+    # no RMSNorm: U v = [-5+2, 1, -2-1] = [-3, 1, -3];  G x = [1, -1, -2];  z = [-2, 0, 0]
+    z, v, n = oracle.gate_lopa(V, U, X_EX, g_idx, g_sign, None, False, 0.0, b, return_vn=True)
+    np.testing.assert_allclose(v, [-5.0, 1.0], atol=0)
+    np.testing.assert_allclose(z, [-2.0, 0.0, 0.0], atol=1e-6)  # U holds fp32(0.2), fp32(0.4)
+    # RMSNorm: mean(v^2) = 13, eps = 3 -> rms = 4;  gamma = [2, 4] -> n = [-2.5, 1]
+    # U n = [-0.5, 0.5, -2];  z = U n + G x + b = [0.5, -0.5, 1]
+    gamma = np.array([2.0, 4.0], np.float32)
+    z, v, n = oracle.gate_lopa(V, U, X_EX, g_idx, g_sign, gamma, True, 3.0, b, return_vn=True)
+    np.testing.assert_allclose(n, [-2.5, 1.0], atol=1e-15)
+    np.testing.assert_allclose(z, [0.5, -0.5, 1.0], atol=1e-6)
+    # dropping the fixed matrix leaves U n + b
+    z = oracle.gate_lopa(V, U, X_EX, None, None, gamma, True, 3.0, b)
+    np.testing.assert_allclose(z, [-0.5, 0.5, 3.0], atol=1e-6)
+
+
+def test_activation_table(golden):
+    for act, x, want in golden("activation_table.txt"):
+        assert oracle.activation(act, float(x)) == pytest.approx(float(want), abs=1e-15), (act, x)
+    # R-S+ equals SILU on the non-negative side and RELU's zero on the negative side
+    for x in np.linspace(0.0, 6.0, 25):
+        assert oracle.activation("rsplus", x) == pytest.approx(x / (1 + math.exp(-x)), rel=1e-15)
+    for x in (-1e-30, -0.5, -40.0):
+        assert oracle.activation("rsplus", x) == 0.0 and oracle.activation("relu", x) == 0.0
+    assert oracle.activation("relu", -0.0) == 0.0
+    assert oracle.activation("sqrelu", 1e-200) == 0.0   # z*z underflows; activity is decided on z
+
+
+def test_bf16_inputs_decode_exactly():
+    # bf16 bit patterns: 1.0 = 0x3F80, -2.0 = 0xC000, 0.5 = 0x3F00, 3.0 = 0x4040, -1.5 = 0xBFC0
+    W = np.array([[0x3F80, 0xC000], [0x3F00, 0x4040]], np.uint16)   # [[1, -2], [0.5, 3]]
+    x = np.array([0x4040, 0xBFC0], np.uint16)                        # [3, -1.5]
+    np.testing.assert_array_equal(oracle.gate_standard(W, x), [3.0 + 3.0, 1.5 - 4.5])
+    t = torch.tensor([[1.0, -2.0], [0.5, 3.0]], dtype=torch.bfloat16)
+    np.testing.assert_array_equal(oracle.as_oracle_array(t), W)
+
+
+# ---------------------------------------------------------------- library routine, other orientation
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("act", ["relu", "sqrelu", "rsplus"])
+def test_dense_route_matches_matmul_with_w2_as_D_by_H(dtype, act):
+    D, H = 40, 112
+    w = syn.standard_ffn(D, H, dtype, seed=11, sparsity=0.5)
+    x = syn.tokens(3, D, dtype, seed=11)
+    out = oracle.ffn(x, w["W_up"], w["W_down"], act, W_g=w["W_g"], b_g=w["b_g"], route="dense")
+    W1, W3 = w["W_g"].double().numpy(), w["W_up"].double().numpy()
+    W2 = w["W_down"].double().numpy().T.copy()          # [D, H]: Eq. 1's own orientation
+    for b in range(3):
+        xb = x[b].double().numpy()
+        z = W1 @ xb + w["b_g"].double().numpy()
+        a = {"relu": np.maximum(z, 0), "sqrelu": np.maximum(z, 0) ** 2,
+             "rsplus": np.where(z >= 0, z / (1 + np.exp(-z)), 0.0)}[act]
+        y = W2 @ (a * (W3 @ xb))
+        np.testing.assert_allclose(out["z"][b], z, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(out["y"][b], y, rtol=1e-11, atol=1e-12)
+
+
+def test_gate_is_affine_in_x():
+    D, H = 33, 70
+    W = RNG.standard_normal((H, D)).astype(np.float32)
+    x = RNG.standard_normal(D).astype(np.float32)
+    b = RNG.standard_normal(H).astype(np.float32)
+    z1 = oracle.gate_standard(W, x, b) - b.astype(np.float64)
+    z4 = oracle.gate_standard(W, (4.0 * x).astype(np.float32), b) - b.astype(np.float64)
+    np.testing.assert_allclose(z4, 4.0 * z1, rtol=1e-13, atol=1e-13)  # scaling by 4 is exact in fp32
+
+
+# ---------------------------------------------------------------- active set
+def test_active_set_brute_force():
+    z = RNG.standard_normal(500)
+    z[[3, 77, 200]] = [0.0, -0.0, 1e-300]
+    for act in ("relu", "sqrelu", "rsplus"):
+        # brute force: evaluate A(z_j) for every j and keep the nonzeros; squared RELU underflows at
+        # 1e-300, so activity is decided on z (a contributes nothing either way)
+        brute = [j for j in range(500) if oracle.activation(act, z[j]) != 0.0 or z[j] > 0]
+        got = oracle.active_set(z)
+        assert got.tolist() == brute == sorted(brute)
+        assert len(got) + int(np.sum(~(z > 0))) == 500
+    assert 3 not in got and 77 not in got and 200 in got
+
+
+def test_config1_sparsity_statistics():
+    # tiny bring-up config: D=256, H=1024, fp32, RELU, b_g = -Phi^-1(0.9), 64 tokens, seed 0
+    w = syn.standard_ffn(256, 1024, torch.float32, seed=0, sparsity=0.9)
+    assert w["b_g"][0].item() == pytest.approx(-1.2815516, abs=1e-6)
+    x = syn.tokens(64, 256, torch.float32, seed=0)
+    out = oracle.ffn(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=w["b_g"], threads=4)
+    sparsity = 1.0 - out["n_act"].mean() / 1024
+    assert abs(sparsity - 0.9) < 0.01
+    assert np.std(out["z"] - w["b_g"][0].item()) == pytest.approx(1.0, abs=0.03)
+
+
+# ---------------------------------------------------------------- sparse execution is exact
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_sparse_route_is_bit_identical_to_dense_route(dtype):
+    D, H = 48, 130
+    w = syn.standard_ffn(D, H, dtype, seed=5, sparsity=0.8)
+    x = syn.tokens(4, D, dtype, seed=5)
+    for act in ("relu", "sqrelu", "rsplus"):
+        d = oracle.ffn(x, w["W_up"], w["W_down"], act, W_g=w["W_g"], b_g=w["b_g"], route="dense")
+        s = oracle.ffn(x, w["W_up"], w["W_down"], act, W_g=w["W_g"], b_g=w["b_g"], route="sparse")
+        assert np.array_equal(d["y"], s["y"]) and np.array_equal(d["z"], s["z"])
+        assert 0 < s["n_act"].min() and s["n_act"].max() < H
+
+
+def test_zero_and_full_sparsity_and_single_neuron():
+    D, H = 24, 60
+    w = syn.standard_ffn(D, H, torch.float32, seed=6, sparsity=None)
+    x = syn.tokens(1, D, torch.float32, seed=6)[0]
+    hi, lo = torch.full((H,), 1e3), torch.full((H,), -1e3)
+    full = oracle.ffn(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=hi, route="sparse")
+    dense = oracle.ffn(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=hi, route="dense")
+    assert full["n_act"][0] == H and np.array_equal(full["y"], dense["y"])
+    none = oracle.ffn(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=lo, route="sparse")
+    assert none["n_act"][0] == 0 and not none["y"].any()
+    # exactly one active neuron j: y = a_j u_j W_down[j]
+    j = 17
+    one = lo.clone()
+    one[j] = 1e3
+    out = oracle.ffn(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=one)
+    xd = x.double().numpy()
+    a = float(w["W_g"][j].double().numpy() @ xd + 1e3)
+    u = float(w["W_up"][j].double().numpy() @ xd)
+    assert out["n_act"][0] == 1
+    np.testing.assert_allclose(out["y"], a * u * w["W_down"][j].double().numpy(), rtol=1e-12)
+
+
+def test_neuron_permutation_invariance():
+    D, H = 32, 90
+    w = syn.standard_ffn(D, H, torch.float32, seed=7, sparsity=0.7)
+    x = syn.tokens(1, D, torch.float32, seed=7)[0]
+    perm = torch.randperm(H, generator=torch.Generator().manual_seed(1))
+    a = oracle.ffn(x, w["W_up"], w["W_down"], "rsplus", W_g=w["W_g"], b_g=w["b_g"])
+    b = oracle.ffn(x, w["W_up"][perm], w["W_down"][perm], "rsplus", W_g=w["W_g"][perm],
+                   b_g=w["b_g"][perm])
+    np.testing.assert_allclose(a["y"], b["y"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_array_equal(a["z"][perm.numpy()], b["z"])
+
+
+# ---------------------------------------------------------------- LoPA gate (Eq. 3)
+def test_lopa_equals_materialised_gate():
+    D, H, r = 12, 30, 5
+    V, U = RNG.standard_normal((r, D)), RNG.standard_normal((H, r))
+    x = RNG.standard_normal(D)
+    b = RNG.standard_normal(H).astype(np.float32)
+    for gen in (oracle.g_diagonal, oracle.g_tiled):
+        g_idx = gen(H, D)
+        sign = RNG.choice([-1, 1], H).astype(np.int8)
+        W1 = oracle.fixed_matrix_dense(g_idx, D, sign) + U @ V      # W_1 = G + UV, materialised
+        z_mat = oracle.gate_standard(W1, x, b)
+        z_lopa = oracle.gate_lopa(V, U, x, g_idx, sign, None, False, 0.0, b)
+        np.testing.assert_allclose(z_lopa, z_mat, rtol=1e-12, atol=1e-12)
+    z_uv = oracle.gate_lopa(V, U, x, None, None, None, False, 0.0, None)
+    np.testing.assert_allclose(z_uv, oracle.gate_standard(U @ V, x), rtol=1e-12, atol=1e-12)
+    # whole FFN through the LoPA gate == whole FFN through the materialised W_1
+    W3, Wd = RNG.standard_normal((H, D)), RNG.standard_normal((H, D))
+    g_idx = oracle.g_diagonal(H, D)
+    lopa = dict(V=V, U=U, g_idx=g_idx, use_rmsnorm=False)
+    a = oracle.ffn(x, W3, Wd, "relu", lopa=lopa, b_g=b)
+    m = oracle.ffn(x, W3, Wd, "relu", W_g=oracle.fixed_matrix_dense(g_idx, D) + U @ V, b_g=b)
+    np.testing.assert_allclose(a["y"], m["y"], rtol=1e-10, atol=1e-10)
+
+
+def test_rmsnorm_properties():
+    D, H, r = 20, 16, 8
+    V, U = RNG.standard_normal((r, D)), RNG.standard_normal((H, r))
+    x = RNG.standard_normal(D)
+    _, v, n = oracle.gate_lopa(V, U, x, None, None, None, True, 0.0, None, return_vn=True)
+    assert float(n @ n) == pytest.approx(r, rel=1e-12)            # unit RMS at gain 1, eps 0
+    np.testing.assert_allclose(n, v / math.sqrt(float(v @ v) / r), rtol=1e-13)
+    z1 = oracle.gate_lopa(V, U, x, None, None, None, True, 0.0, None)
+    z3 = oracle.gate_lopa(V, U, 3.0 * x, None, None, None, True, 0.0, None)
+    np.testing.assert_allclose(z3, z1, rtol=1e-12, atol=1e-12)     # scale-invariant without G
+    z0 = oracle.gate_lopa(V, U, x, None, None, None, False, 0.0, None)
+    np.testing.assert_allclose(z0, U @ (V @ x), rtol=1e-12)
+
+
+def test_fixed_matrices_picture(golden):
+    rows = {r[0]: np.array(r[1:], np.int32) for r in golden("fixed_matrices_h12_d6.txt")}
+    np.testing.assert_array_equal(oracle.g_diagonal(12, 6), rows["diagonal"])
+    np.testing.assert_array_equal(oracle.g_tiled(12, 6), rows["tiled_identity"])
+    np.testing.assert_array_equal(oracle.g_padded_identity(12, 6), rows["padded_identity"])
+    for gen in (oracle.g_diagonal, oracle.g_tiled):
+        M = oracle.fixed_matrix_dense(gen(12, 6), 6)
+        assert (M.sum(axis=1) == 1).all() and (M.sum(axis=0) == 2).all()   # one per row, all columns hit
+    assert (oracle.fixed_matrix_dense(oracle.g_padded_identity(12, 6), 6).sum(axis=1)[6:] == 0).all()
+    x = np.arange(6, dtype=np.float64) + 1
+    np.testing.assert_array_equal(oracle.fixed_matrix_dense(oracle.g_tiled(12, 6), 6) @ x,
+                                  x[np.arange(12) % 6])
+    # non-integer H/D (the benchmark shape 14336/4096 = 3.5): still one column per row, all used
+    g = oracle.g_diagonal(14336, 4096)
+    assert g.min() == 0 and g.max() == 4095 and (np.diff(g) >= 0).all()
+    assert set(np.bincount(g).tolist()) == {3, 4}
+
+
+# ---------------------------------------------------------------- closed forms (Eq. 2, Eq. 4, H')
+def test_printed_closed_form_values(golden):
+    for row in golden("flop_ratio_values.txt"):
+        kind, *args = row
+        *args, want, tol = [float(a) for a in args]
+        if kind == "standard":
+            got = oracle.flop_ratio_standard(args[0])
+        elif kind == "hprime":
+            got = oracle.adaptive_hidden_dim(*args)
+        else:
+            alpha, h_over_d, s = args
+            D = 1024.0
+            hp = oracle.adaptive_hidden_dim(D, h_over_d * D, alpha * D)
+            got = oracle.flop_ratio_lopa(s, D, hp, alpha * D)
+        assert abs(got - want) <= tol, (row, got)
+    # parameter count is preserved by H'
+    D, H, r = 2560, 7168, 400
+    hp = oracle.adaptive_hidden_dim(D, H, r)
+    assert r * (hp + D) + 2 * hp * D == pytest.approx(3 * H * D, rel=1e-12)
+
+
+def test_casting_table_speedups(golden):
+    D, H, r = 1920.0, 5120.0, 240.0
+    hp = oracle.adaptive_hidden_dim(D, H, r)
+    f = {"base": oracle.flop_ratio_standard,
+         "lopa": lambda s: oracle.flop_ratio_lopa(s, D, hp, r),
+         "archcast": lambda s: oracle.flop_ratio_lopa_fixed_h(s, D, H, r)}
+    for arch, s, printed in golden("casting_table_speedups.txt"):
+        s, printed = float(s), float(printed)
+        lo, hi = f[arch](max(0.0, s - 0.01)), f[arch](min(1.0, s + 0.01))
+        assert lo - 0.006 <= printed <= hi + 0.006, (arch, s, printed, lo, hi)
+
+
+# ---------------------------------------------------------------- batches and the union of masks
+def test_batch_equals_independent_tokens_and_union():
+    D, H, B = 36, 100, 5
+    w = syn.standard_ffn(D, H, torch.bfloat16, seed=9, sparsity=0.85)
+    x = syn.tokens(B, D, torch.bfloat16, seed=9)
+    batch = oracle.ffn(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=w["b_g"], threads=3)
+    union = np.zeros(H, bool)
+    for b in range(B):
+        one = oracle.ffn(x[b], w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=w["b_g"])
+        assert np.array_equal(one["y"], batch["y"][b]) and np.array_equal(one["z"], batch["z"][b])
+        union[oracle.active_set(one["z"])] = True
+    np.testing.assert_array_equal(batch["union_mask"], union)
+    assert batch["union_mask"].sum() >= batch["n_act"].max()
+
+
+def test_zipf_profile_recipe():
+    H = 14336
+    p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
+    assert float(p.mean()) == pytest.approx(0.1, abs=1e-6)
+    assert int((p >= 0.99 - 1e-12).sum()) in range(300, 400) and float(p.min()) == pytest.approx(0.0169, abs=2e-3)
+    for B, want in ((4, 0.24), (16, 0.53), (64, 0.88)):
+        assert syn.expected_union_fraction(p, B) == pytest.approx(want, abs=0.015)
+    b = syn.bias_from_firing_profile(p)
+    # a N(0,1) pre-activation plus b_j is positive with probability p_j
+    fire = 0.5 * torch.erfc(-b.double() / math.sqrt(2.0))
+    np.testing.assert_allclose(fire.numpy(), p.numpy(), atol=1e-6)
