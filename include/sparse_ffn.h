@@ -1,0 +1,148 @@
+/*
+ * sparse_ffn.h -- C ABI of the activation-sparse gated FFN library for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, for B independent tokens x_b in R^D,
+ *
+ *     y_b = W_2 ( A(W_1 x_b + b_g)  .  (W_3 x_b) )                       (paper Eq. 1)
+ *
+ * by the sparse execution scheme of the paper's Sec. 3.1 ("FFN FLOP-ratio"): the gate W_1 x is always
+ * computed in full; a neuron j whose activation A(.)_j is zero is known before W_3 and W_2 are
+ * touched, so row j of W_3 and column j of W_2 are never read.  W_1 is either a full matrix
+ * (standard gating) or the low-parameter gate of Sec. 3.3 (Eq. 3), W_1 = G + U V, evaluated as
+ * G x + U RMSNorm(V x), with the RMSNorm optional (architecture casting, Sec. 3.4, has none).
+ * For B > 1 the rows are read once for the union of the tokens' active sets (Sec. 5.4).
+ *
+ * Storage (all row-major, all DEVICE memory unless a name ends in _host):
+ *     x       [B, D]   element type = the handle's dtype (fp32 or bf16)
+ *     W_g     [H, D]   = W_1                       same dtype
+ *     W_up    [H, D]   = W_3                       same dtype
+ *     W_down  [H, D]   = W_2 transposed (row j is column j of W_2)   same dtype
+ *     V [r, D], U [H, r]                           same dtype
+ *     b_g [H], rms_gain [r]                        fp32
+ *     g_idx [H] int32, g_sign [H] int8 (+1 / -1)
+ *     y       [B, D]   fp32, overwritten
+ * The gate bias b_g is not part of Eq. 1 (pass NULL for the paper's form); it is the knob the
+ * synthetic workloads use to set the sparsity.
+ *
+ * Ownership: every buffer is owned by the caller and only read (y and the workspace are written).
+ * The library never allocates or frees device memory: the caller allocates `workspace`
+ * (sffn_workspace_bytes) and hands it to sffn_create.  Pointers must be 16-byte aligned and rows
+ * must be a multiple of 16 bytes (D and r multiples of 8 for bf16, of 4 for fp32), otherwise
+ * SFFN_ERR_UNSUPPORTED.
+ *
+ * Errors: every entry point returns an sffn_status.  The return value covers host-side validation
+ * and launch errors only; calls are asynchronous on `stream`.  Conditions detected on the device
+ * (a bounded wait that ran out) are recorded in a status word inside the workspace and read back
+ * with sffn_last_device_status; the kernels never trap and never spin without a limit.
+ * The same inputs give bitwise the same y and the same index list on every call.
+ * Inputs are assumed finite (an Inf/NaN in a skipped row would make sparse and dense differ).
+ */
+#ifndef SPARSE_FFN_H_
+#define SPARSE_FFN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SFFN_OK = 0,
+  SFFN_ERR_INVALID_ARG = 1, /* null handle/pointer, B out of range, bad enum                    */
+  SFFN_ERR_UNSUPPORTED = 2, /* misaligned pointer, row size not a multiple of 16 bytes, too big */
+  SFFN_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small                       */
+  SFFN_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch, copy)                        */
+  SFFN_ERR_TIMEOUT = 5      /* device status only: a bounded device-side wait gave up           */
+} sffn_status;
+
+/* Activation A of Eq. 1.  RELU and R-S+ follow the table of Sec. 3.1 (R-S+: 0 for z < 0,
+ * z*sigmoid(z) for z >= 0); SQRELU = max(z,0)^2 is one of the activations of the paper's activation
+ * study.  For all three A(z) != 0 exactly when z > 0, which is the test the library applies. */
+typedef enum { SFFN_ACT_RELU = 0, SFFN_ACT_SQRELU = 1, SFFN_ACT_RSPLUS = 2 } sffn_act;
+
+typedef enum { SFFN_F32 = 0, SFFN_BF16 = 1 } sffn_dtype;
+
+typedef enum { SFFN_GATE_STANDARD = 0, SFFN_GATE_LOPA = 1 } sffn_gate_kind;
+
+/* Which kernels serve a call.  AUTO picks the fused single-launch kernel for B = 1 when the shape
+ * allows it and the general multi-kernel path otherwise; the other two force one of them
+ * (SFFN_ERR_UNSUPPORTED if the forced path cannot serve the call). */
+typedef enum { SFFN_PATH_AUTO = 0, SFFN_PATH_GENERAL = 1, SFFN_PATH_FUSED = 2 } sffn_path;
+
+/* Gate description.  STANDARD uses W_g only.  LOPA (Eq. 3; "LoPA in practice", Sec. 3.3) uses
+ *   z_j = g_sign[j] * x[g_idx[j]] + sum_k U[j,k] n_k + b_g[j],   n = RMSNorm(V x) or V x,
+ *   RMSNorm(v)_k = rms_gain[k] * v_k / sqrt(mean_k v_k^2 + rms_eps).
+ * g_idx NULL drops the fixed matrix G (plain low-rank gate); g_sign NULL means +1 everywhere;
+ * rms_gain NULL means 1. */
+typedef struct {
+  int32_t kind;            /* sffn_gate_kind                                        */
+  int32_t r;               /* LOPA: rank, 1 <= r <= r_max of the handle             */
+  const void* W_g;         /* STANDARD: [H, D]                                      */
+  const void* V;           /* LOPA: [r, D]                                          */
+  const void* U;           /* LOPA: [H, r]                                          */
+  const int32_t* g_idx;    /* LOPA: [H] column of the single nonzero of G, or NULL  */
+  const int8_t* g_sign;    /* LOPA: [H] +1/-1, or NULL                              */
+  const float* rms_gain;   /* LOPA: [r] or NULL                                     */
+  int32_t use_rmsnorm;     /* LOPA: 1 = with RMSNorm (Sec. 3.3), 0 = without (Sec. 3.4) */
+  float rms_eps;           /* LOPA: added to the mean square; the paper gives no value */
+} sffn_gate;
+
+typedef struct sffn_handle sffn_handle;
+
+/* Bytes of device workspace a handle for these limits needs.  r_max may be 0 (no LoPA calls). */
+int sffn_workspace_bytes(int D, int H, int r_max, int B_max, int dtype, size_t* bytes);
+
+/* Creates a handle on the current device.  `workspace` is device memory of at least
+ * sffn_workspace_bytes(...) bytes, 256-byte aligned, owned by the caller and kept alive (and not
+ * shared with another handle) until sffn_destroy.  The call clears the workspace (synchronously).
+ * Calls on one handle must be issued to one stream at a time. */
+int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dtype,
+                void* workspace, size_t workspace_bytes);
+
+/* Frees host state only; the workspace stays the caller's. */
+int sffn_destroy(sffn_handle* handle);
+
+int sffn_set_path(sffn_handle* handle, int path /* sffn_path */);
+
+/* Sparse execution of Eq. 1 (Sec. 3.1): gate in full, then only the active rows of W_up / W_down.
+ * x [B,D] and all weights on the device; y [B,D] fp32 on the device, fully overwritten (zeros when
+ * no neuron fires).  1 <= B <= B_max.  `stream` is a cudaStream_t (NULL = default stream). */
+int sparse_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate* gate,
+                       const float* b_g, const void* W_up, const void* W_down, int act, float* y,
+                       void* stream);
+
+/* Dense comparator: the same function with every one of the H rows of W_up / W_down read
+ * (Eq. 1 as written).  Same arguments; defines the "x1" of every speedup. */
+int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate* gate,
+                      const float* b_g, const void* W_up, const void* W_down, int act, float* y,
+                      void* stream);
+
+/* End-to-end variant of sparse_ffn_forward for callers whose activations live on the host:
+ * x_host [B,D] (handle dtype) and y_host [B,D] fp32 are HOST pointers (pinned memory makes the
+ * copies asynchronous); weights stay on the device.  Copies x in, runs the sparse path, copies y
+ * out, all on `stream`; y_host is valid once the stream has synchronised. */
+int sparse_ffn_forward_host(sffn_handle* handle, const void* x_host, int B, const sffn_gate* gate,
+                            const float* b_g, const void* W_up, const void* W_down, int act,
+                            float* y_host, void* stream);
+
+/* Introspection for tests and benchmarks, valid after the stream of the last sparse call has
+ * synchronised.  *idx_dev points at the ascending list of active neurons of that call (for B > 1:
+ * of the union over the tokens) and *count_dev at its length; both live in the workspace.  The list
+ * is materialised by this call (one small launch on `stream`) and is valid once it synchronises. */
+int sffn_last_active(sffn_handle* handle, const int32_t** idx_dev, const int32_t** count_dev,
+                     void* stream);
+
+/* Reads the device status word (synchronises the device): SFFN_OK or SFFN_ERR_TIMEOUT. */
+int sffn_last_device_status(sffn_handle* handle, int* status);
+
+/* Number of kernels this handle has launched since creation (host-side counter). */
+int sffn_launch_count(sffn_handle* handle, long long* launches);
+
+/* Static string for a status code. */
+const char* sffn_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSE_FFN_H_ */

@@ -1,0 +1,192 @@
+"""ctypes binding of include/sparse_ffn.h.  Marshals torch tensors into plain pointers."""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+ACT = {"relu": 0, "sqrelu": 1, "rsplus": 2}
+PATH = {"auto": 0, "general": 1, "fused": 2}
+_STATUS = {0: "ok", 1: "invalid argument", 2: "unsupported shape, alignment or path",
+           3: "workspace missing, misaligned or too small", 4: "CUDA runtime error",
+           5: "device-side bounded wait ran out"}
+
+
+class SFFNError(RuntimeError):
+    def __init__(self, where: str, code: int):
+        super().__init__(f"{where}: status {code} ({_STATUS.get(code, 'unknown')})")
+        self.code = code
+
+
+class _Gate(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("r", ctypes.c_int32), ("W_g", ctypes.c_void_p),
+                ("V", ctypes.c_void_p), ("U", ctypes.c_void_p), ("g_idx", ctypes.c_void_p),
+                ("g_sign", ctypes.c_void_p), ("rms_gain", ctypes.c_void_p),
+                ("use_rmsnorm", ctypes.c_int32), ("rms_eps", ctypes.c_float)]
+
+
+def lib_path() -> Path:
+    return _PKG / "libsparse_ffn.so"
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        p = lib_path()
+        if not p.exists():
+            raise RuntimeError(f"{p} is missing: build it with `python -m paper_2609_31975_b200.build` "
+                               "(the sparse FFN has no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(str(p))
+        vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        lib.sffn_workspace_bytes.argtypes = [i, i, i, i, i, ctypes.POINTER(sz)]
+        lib.sffn_create.argtypes = [ctypes.POINTER(vp), i, i, i, i, i, vp, sz]
+        lib.sffn_destroy.argtypes = [vp]
+        lib.sffn_set_path.argtypes = [vp, i]
+        fwd = [vp, vp, i, ctypes.POINTER(_Gate), vp, vp, vp, i, vp, vp]
+        lib.sparse_ffn_forward.argtypes = fwd
+        lib.dense_ffn_forward.argtypes = fwd
+        lib.sparse_ffn_forward_host.argtypes = fwd
+        lib.sffn_last_active.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
+        lib.sffn_last_device_status.argtypes = [vp, ctypes.POINTER(i)]
+        lib.sffn_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
+        lib.sffn_status_string.argtypes = [i]
+        lib.sffn_status_string.restype = ctypes.c_char_p
+        _lib = lib
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _check(where: str, rc: int):
+    if rc != 0:
+        raise SFFNError(where, rc)
+
+
+class SparseFFN:
+    """One library handle (fixed D, H, dtype, limits r_max and B_max) plus its torch-owned workspace.
+
+    ``gate`` arguments are dicts: ``{"W_g": t}`` for standard gating, or
+    ``{"V": t, "U": t, "g_idx": t|None, "g_sign": t|None, "rms_gain": t|None,
+    "use_rmsnorm": bool, "rms_eps": float}`` for the LoPA gate.
+    """
+
+    def __init__(self, D: int, H: int, dtype: torch.dtype, r_max: int = 0, B_max: int = 1,
+                 device="cuda:0"):
+        if dtype not in (torch.float32, torch.bfloat16):
+            raise TypeError("dtype must be torch.float32 or torch.bfloat16")
+        self.lib = load_library()
+        self.D, self.H, self.dtype, self.r_max, self.B_max = D, H, dtype, r_max, B_max
+        self.device = torch.device(device)
+        self._dt = 1 if dtype == torch.bfloat16 else 0
+        need = ctypes.c_size_t(0)
+        _check("sffn_workspace_bytes", self.lib.sffn_workspace_bytes(D, H, r_max, B_max, self._dt, ctypes.byref(need)))
+        self.workspace_bytes = need.value
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(need.value + 256, dtype=torch.uint8, device=self.device)
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            h = ctypes.c_void_p()
+            _check("sffn_create", self.lib.sffn_create(ctypes.byref(h), D, H, r_max, B_max, self._dt,
+                                                       ctypes.c_void_p(self._ws_ptr), need.value))
+        self._h = h
+        self._keep = None
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.lib.sffn_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def set_path(self, path: str):
+        _check("sffn_set_path", self.lib.sffn_set_path(self._h, PATH[path]))
+
+    def _gate(self, gate: dict) -> _Gate:
+        g = _Gate()
+        if "W_g" in gate:
+            g.kind, g.W_g = 0, gate["W_g"].data_ptr()
+        else:
+            g.kind, g.r = 1, gate["V"].shape[0]
+            g.V, g.U = gate["V"].data_ptr(), gate["U"].data_ptr()
+            for k in ("g_idx", "g_sign", "rms_gain"):
+                t = gate.get(k)
+                setattr(g, k, None if t is None else t.data_ptr())
+            g.use_rmsnorm = int(gate.get("use_rmsnorm", True))
+            g.rms_eps = float(gate.get("rms_eps", 1e-5))
+        return g
+
+    def _stream(self, stream):
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        return ctypes.c_void_p(s.cuda_stream)
+
+    def _call(self, fn, name, x, gate, b_g, W_up, W_down, act, y, stream):
+        B = 1 if x.dim() == 1 else x.shape[0]
+        g = self._gate(gate)
+        self._keep = (x, gate, b_g, W_up, W_down, y)
+        _check(name, fn(self._h, _ptr(x), B, ctypes.byref(g), _ptr(b_g), _ptr(W_up), _ptr(W_down),
+                        ACT[act] if isinstance(act, str) else int(act), _ptr(y), self._stream(stream)))
+        return y
+
+    def prepared(self, x, gate, b_g, W_up, W_down, act, y, *, dense=False, host=False, stream=None):
+        """Marshals one call once and returns a zero-argument callable that issues it (for launch
+        loops where per-call marshalling would dominate).  The stream is fixed at preparation."""
+        fn = (self.lib.sparse_ffn_forward_host if host else
+              self.lib.dense_ffn_forward if dense else self.lib.sparse_ffn_forward)
+        B = 1 if x.dim() == 1 else x.shape[0]
+        g = self._gate(gate)
+        args = (self._h, _ptr(x), B, ctypes.byref(g), _ptr(b_g), _ptr(W_up), _ptr(W_down),
+                ACT[act] if isinstance(act, str) else int(act), _ptr(y), self._stream(stream))
+        keep = (x, gate, b_g, W_up, W_down, y, g)
+
+        def call(_fn=fn, _args=args, _keep=keep):
+            rc = _fn(*_args)
+            if rc:
+                raise SFFNError("prepared call", rc)
+
+        return call
+
+    def sparse_ffn_forward(self, x, gate, b_g, W_up, W_down, act="relu", y=None, stream=None):
+        """y = W_down^T (A(gate(x) + b_g) * (W_up x)) touching only the rows of fired neurons."""
+        if y is None:
+            y = torch.empty((*x.shape[:-1], self.D), dtype=torch.float32, device=x.device)
+        return self._call(self.lib.sparse_ffn_forward, "sparse_ffn_forward", x, gate, b_g, W_up, W_down, act, y, stream)
+
+    def dense_ffn_forward(self, x, gate, b_g, W_up, W_down, act="relu", y=None, stream=None):
+        """The dense comparator: same function, all H rows read."""
+        if y is None:
+            y = torch.empty((*x.shape[:-1], self.D), dtype=torch.float32, device=x.device)
+        return self._call(self.lib.dense_ffn_forward, "dense_ffn_forward", x, gate, b_g, W_up, W_down, act, y, stream)
+
+    def sparse_ffn_forward_host(self, x_host, gate, b_g, W_up, W_down, act, y_host, stream=None):
+        """End-to-end variant: x_host / y_host are (pinned) host tensors, weights on the device."""
+        assert not x_host.is_cuda and not y_host.is_cuda
+        return self._call(self.lib.sparse_ffn_forward_host, "sparse_ffn_forward_host", x_host, gate, b_g,
+                          W_up, W_down, act, y_host, stream)
+
+    def last_active(self, stream=None) -> torch.Tensor:
+        """Ascending indices of the neurons that fired in the last sparse call (union for B > 1)."""
+        idx, cnt = ctypes.c_void_p(), ctypes.c_void_p()
+        _check("sffn_last_active", self.lib.sffn_last_active(self._h, ctypes.byref(idx), ctypes.byref(cnt),
+                                                             self._stream(stream)))
+        torch.cuda.synchronize(self.device)
+        off_idx, off_cnt = idx.value - self.workspace.data_ptr(), cnt.value - self.workspace.data_ptr()
+        n = int(self.workspace[off_cnt:off_cnt + 4].view(torch.int32).item())
+        return self.workspace[off_idx:off_idx + 4 * n].view(torch.int32).clone()
+
+    def device_status(self) -> int:
+        out = ctypes.c_int(0)
+        _check("sffn_last_device_status", self.lib.sffn_last_device_status(self._h, ctypes.byref(out)))
+        return out.value
+
+    def launch_count(self) -> int:
+        out = ctypes.c_longlong(0)
+        _check("sffn_launch_count", self.lib.sffn_launch_count(self._h, ctypes.byref(out)))
+        return out.value

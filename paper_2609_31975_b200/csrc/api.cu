@@ -1,0 +1,329 @@
+// Host side of the C ABI declared in include/sparse_ffn.h: argument checks, workspace carving and
+// kernel dispatch.  No device memory is allocated or freed here.
+#include "sparse_ffn.h"
+
+#include <cuda_runtime.h>
+
+#include <new>
+
+#include "fused_kernel.cuh"
+#include "general_kernels.cuh"
+
+namespace {
+
+constexpr int kMaxUpDownGrid = 304;  // upper bound of the up/down grid (2 CTAs per SM on 148 SMs)
+constexpr int kMaxChunk = 4;         // tokens per pass of the general kernels
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+  size_t status, act, flag, idx, v, n, partial, xstage, ystage, fused, total;
+};
+
+Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
+  const size_t esz = dtype == SFFN_BF16 ? 2 : 4;
+  Layout L{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  L.status = take(256);  // [0] device status, [1] length of idx
+  L.act = take((size_t)B_max * H * 4);
+  L.flag = take((size_t)H);
+  L.idx = take((size_t)H * 4);
+  L.v = take((size_t)B_max * (r_max > 0 ? r_max : 1) * 4);
+  L.n = take((size_t)B_max * (r_max > 0 ? r_max : 1) * 4);
+  L.partial = take((size_t)kMaxUpDownGrid * kMaxChunk * D * 4);
+  L.xstage = take((size_t)B_max * D * esz);
+  L.ystage = take((size_t)B_max * D * 4);
+  L.fused = take(sffn::fused_workspace_bytes(D, H, r_max));
+  L.total = off;
+  return L;
+}
+
+bool shape_ok(int D, int H, int r_max, int B_max, int dtype) {
+  return D > 0 && H > 0 && r_max >= 0 && B_max > 0 && (dtype == SFFN_F32 || dtype == SFFN_BF16);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+struct sffn_handle {
+  int D, H, r_max, B_max, dtype;
+  char* ws;
+  Layout L;
+  int sm_count;
+  int path;
+  long long launches;
+  int list_state;  // 0: no sparse call yet, 1: idx/count hold the last call's list, 2: flags hold it
+  template <typename T>
+  T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+extern "C" {
+
+const char* sffn_status_string(int s) {
+  switch (s) {
+    case SFFN_OK: return "ok";
+    case SFFN_ERR_INVALID_ARG: return "invalid argument";
+    case SFFN_ERR_UNSUPPORTED: return "unsupported shape, alignment or path";
+    case SFFN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SFFN_ERR_CUDA: return "CUDA runtime error";
+    case SFFN_ERR_TIMEOUT: return "device-side bounded wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int sffn_workspace_bytes(int D, int H, int r_max, int B_max, int dtype, size_t* bytes) {
+  if (!bytes || !shape_ok(D, H, r_max, B_max, dtype)) return SFFN_ERR_INVALID_ARG;
+  const size_t esz = dtype == SFFN_BF16 ? 2 : 4;
+  if ((D * esz) % 16 || (r_max * esz) % 16) return SFFN_ERR_UNSUPPORTED;
+  if (sffn::updown_max_tokens(dtype == SFFN_BF16, D) == 0) return SFFN_ERR_UNSUPPORTED;
+  *bytes = make_layout(D, H, r_max, B_max, dtype).total;
+  return SFFN_OK;
+}
+
+int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dtype, void* workspace,
+                size_t workspace_bytes) {
+  if (!handle) return SFFN_ERR_INVALID_ARG;
+  *handle = nullptr;
+  size_t need = 0;
+  const int rc = sffn_workspace_bytes(D, H, r_max, B_max, dtype, &need);
+  if (rc != SFFN_OK) return rc;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
+    return SFFN_ERR_WORKSPACE;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return SFFN_ERR_CUDA;
+  if (cudaMemset(workspace, 0, need) != cudaSuccess) return SFFN_ERR_CUDA;
+  sffn_handle* h = new (std::nothrow) sffn_handle();
+  if (!h) return SFFN_ERR_INVALID_ARG;
+  h->D = D;
+  h->H = H;
+  h->r_max = r_max;
+  h->B_max = B_max;
+  h->dtype = dtype;
+  h->ws = static_cast<char*>(workspace);
+  h->L = make_layout(D, H, r_max, B_max, dtype);
+  h->sm_count = sms;
+  h->path = SFFN_PATH_AUTO;
+  h->launches = 0;
+  h->list_state = 0;
+  *handle = h;
+  return SFFN_OK;
+}
+
+int sffn_destroy(sffn_handle* h) {
+  if (!h) return SFFN_ERR_INVALID_ARG;
+  delete h;
+  return SFFN_OK;
+}
+
+int sffn_set_path(sffn_handle* h, int path) {
+  if (!h || path < SFFN_PATH_AUTO || path > SFFN_PATH_FUSED) return SFFN_ERR_INVALID_ARG;
+  h->path = path;
+  return SFFN_OK;
+}
+
+int sffn_launch_count(sffn_handle* h, long long* launches) {
+  if (!h || !launches) return SFFN_ERR_INVALID_ARG;
+  *launches = h->launches;
+  return SFFN_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+int check_call(const sffn_handle* h, const void* x, int B, const sffn_gate* g, const void* W_up,
+               const void* W_down, int act, const void* y) {
+  if (!h || !x || !g || !W_up || !W_down || !y) return SFFN_ERR_INVALID_ARG;
+  if (B < 1 || B > h->B_max) return SFFN_ERR_INVALID_ARG;
+  if (act < SFFN_ACT_RELU || act > SFFN_ACT_RSPLUS) return SFFN_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W_up) || !aligned16(W_down) || !aligned16(y)) return SFFN_ERR_UNSUPPORTED;
+  const size_t esz = h->dtype == SFFN_BF16 ? 2 : 4;
+  if (g->kind == SFFN_GATE_STANDARD) {
+    if (!g->W_g) return SFFN_ERR_INVALID_ARG;
+    if (!aligned16(g->W_g)) return SFFN_ERR_UNSUPPORTED;
+  } else if (g->kind == SFFN_GATE_LOPA) {
+    if (!g->V || !g->U || g->r < 1 || g->r > h->r_max) return SFFN_ERR_INVALID_ARG;
+    if (!aligned16(g->V) || !aligned16(g->U) || (g->r * esz) % 16) return SFFN_ERR_UNSUPPORTED;
+  } else {
+    return SFFN_ERR_INVALID_ARG;
+  }
+  return SFFN_OK;
+}
+
+#define SFFN_CUDA(expr)                              \
+  do {                                               \
+    if ((expr) != cudaSuccess) return SFFN_ERR_CUDA; \
+  } while (0)
+
+// General path: gate (all tokens, chunks of <= 4) -> compaction -> up/down + reduce per chunk.
+int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
+                const void* W_up, const void* W_down, int act, float* y, bool dense,
+                cudaStream_t s) {
+  using namespace sffn;
+  const bool bf16 = h->dtype == SFFN_BF16;
+  const size_t esz = bf16 ? 2 : 4;
+  const int D = h->D, H = h->H;
+  float* actbuf = h->at<float>(h->L.act);
+  uint8_t* flag = h->at<uint8_t>(h->L.flag);
+  int32_t* idx = h->at<int32_t>(h->L.idx);
+  int32_t* count = h->at<int32_t>(h->L.status) + 1;
+  const int rs = h->r_max > 0 ? h->r_max : 1;
+  float* vbuf = h->at<float>(h->L.v);
+  float* nbuf = h->at<float>(h->L.n);
+  const char* xb = static_cast<const char*>(x);
+
+  const bool lopa = g->kind == SFFN_GATE_LOPA;
+  if (lopa) {
+    for (int b0 = 0; b0 < B;) {
+      const int nb = B - b0 >= 4 ? 4 : B - b0 >= 2 ? 2 : 1;
+      RowDotParams p{};
+      p.W = g->V; p.R = g->r; p.K = D;
+      p.vec = xb + (size_t)b0 * D * esz; p.vec_stride = D;
+      p.out = vbuf + (size_t)b0 * rs; p.out_stride = rs;
+      SFFN_CUDA(launch_rowdot(bf16, !bf16, nb, false, p, h->sm_count, s));
+      ++h->launches;
+      b0 += nb;
+    }
+    if (g->use_rmsnorm) {
+      SFFN_CUDA(launch_rmsnorm(vbuf, nbuf, g->rms_gain, g->r, rs, g->rms_eps, B, s));
+      ++h->launches;
+    }
+  }
+  for (int b0 = 0; b0 < B;) {
+    const int nb = B - b0 >= 4 ? 4 : B - b0 >= 2 ? 2 : 1;
+    RowDotParams p{};
+    if (lopa) {
+      p.W = g->U; p.R = H; p.K = g->r;
+      p.vec = (g->use_rmsnorm ? nbuf : vbuf) + (size_t)b0 * rs; p.vec_stride = rs;
+      p.g_idx = g->g_idx; p.g_sign = g->g_sign;
+    } else {
+      p.W = g->W_g; p.R = H; p.K = D;
+      p.vec = xb + (size_t)b0 * D * esz; p.vec_stride = D;
+    }
+    p.out = actbuf + (size_t)b0 * H; p.out_stride = H;
+    p.b_g = b_g;
+    p.x = xb + (size_t)b0 * D * esz; p.x_stride = D;
+    p.act = act;
+    p.flag = dense ? nullptr : flag;
+    p.flag_or = b0 > 0;
+    SFFN_CUDA(launch_rowdot(bf16, lopa || !bf16, nb, true, p, h->sm_count, s));
+    ++h->launches;
+    b0 += nb;
+  }
+  if (!dense) {
+    SFFN_CUDA(launch_compact(flag, H, idx, count, s));
+    ++h->launches;
+    h->list_state = 1;
+  }
+  const int nbmax = updown_max_tokens(bf16, D);
+  int grid = 2 * h->sm_count;
+  if (grid > kMaxUpDownGrid) grid = kMaxUpDownGrid;
+  float* partial = h->at<float>(h->L.partial);
+  for (int b0 = 0; b0 < B;) {
+    const int left = B - b0;
+    const int nb = (left >= 4 && nbmax >= 4) ? 4 : left >= 2 ? 2 : 1;
+    UpDownParams p{};
+    p.W_up = W_up; p.W_down = W_down;
+    p.x = xb + (size_t)b0 * D * esz; p.x_stride = D;
+    p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
+    p.idx = dense ? nullptr : idx;
+    p.count = dense ? nullptr : count;
+    p.H = H; p.D = D;
+    p.partial = partial;
+    SFFN_CUDA(launch_updown(bf16, nb, p, grid, s));
+    SFFN_CUDA(launch_reduce(partial, grid, nb, D, y + (size_t)b0 * D, D, s));
+    h->launches += 2;
+    b0 += nb;
+  }
+  return SFFN_OK;
+}
+
+int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g, const void* W_up,
+        const void* W_down, int act, float* y, bool dense, void* stream) {
+  const int rc = check_call(h, x, B, g, W_up, W_down, act, y);
+  if (rc != SFFN_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const bool fused_ok = sffn::fused_supported(h->dtype == SFFN_BF16, h->D, h->H, B, g, h->sm_count);
+  if (h->path == SFFN_PATH_FUSED && !fused_ok) return SFFN_ERR_UNSUPPORTED;
+  if (fused_ok && h->path != SFFN_PATH_GENERAL) {
+    sffn::FusedCall c{};
+    c.bf16 = h->dtype == SFFN_BF16;
+    c.D = h->D; c.H = h->H;
+    c.x = x; c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.y = y;
+    c.dense = dense;
+    c.workspace = h->ws + h->L.fused;
+    c.status = h->at<int32_t>(h->L.status);
+    c.flag = h->at<uint8_t>(h->L.flag);
+    c.sm_count = h->sm_count;
+    int launched = 0;
+    if (sffn::launch_fused(c, s, &launched) != cudaSuccess) return SFFN_ERR_CUDA;
+    h->launches += launched;
+    if (!dense) h->list_state = 2;
+    return SFFN_OK;
+  }
+  return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+int sparse_ffn_forward(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
+                       const void* W_up, const void* W_down, int act, float* y, void* stream) {
+  return run(h, x, B, g, b_g, W_up, W_down, act, y, false, stream);
+}
+
+int dense_ffn_forward(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
+                      const void* W_up, const void* W_down, int act, float* y, void* stream) {
+  return run(h, x, B, g, b_g, W_up, W_down, act, y, true, stream);
+}
+
+int sparse_ffn_forward_host(sffn_handle* h, const void* x_host, int B, const sffn_gate* g,
+                            const float* b_g, const void* W_up, const void* W_down, int act,
+                            float* y_host, void* stream) {
+  if (!h || !x_host || !y_host || B < 1 || B > h->B_max) return SFFN_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t esz = h->dtype == SFFN_BF16 ? 2 : 4;
+  void* xs = h->ws + h->L.xstage;
+  float* ys = h->at<float>(h->L.ystage);
+  SFFN_CUDA(cudaMemcpyAsync(xs, x_host, (size_t)B * h->D * esz, cudaMemcpyHostToDevice, s));
+  const int rc = run(h, xs, B, g, b_g, W_up, W_down, act, ys, false, stream);
+  if (rc != SFFN_OK) return rc;
+  SFFN_CUDA(cudaMemcpyAsync(y_host, ys, (size_t)B * h->D * 4, cudaMemcpyDeviceToHost, s));
+  return SFFN_OK;
+}
+
+int sffn_last_active(sffn_handle* h, const int32_t** idx_dev, const int32_t** count_dev, void* stream) {
+  if (!h || !idx_dev || !count_dev) return SFFN_ERR_INVALID_ARG;
+  if (h->list_state == 0) return SFFN_ERR_INVALID_ARG;
+  int32_t* idx = h->at<int32_t>(h->L.idx);
+  int32_t* count = h->at<int32_t>(h->L.status) + 1;
+  if (h->list_state == 2) {
+    SFFN_CUDA(sffn::launch_compact(h->at<uint8_t>(h->L.flag), h->H, idx, count,
+                                   static_cast<cudaStream_t>(stream)));
+    ++h->launches;
+    h->list_state = 1;
+  }
+  *idx_dev = idx;
+  *count_dev = count;
+  return SFFN_OK;
+}
+
+int sffn_last_device_status(sffn_handle* h, int* status) {
+  if (!h || !status) return SFFN_ERR_INVALID_ARG;
+  int32_t word = 0;
+  SFFN_CUDA(cudaDeviceSynchronize());
+  SFFN_CUDA(cudaMemcpy(&word, h->ws + h->L.status, sizeof word, cudaMemcpyDeviceToHost));
+  *status = word;
+  return SFFN_OK;
+}
+
+}  // extern "C"

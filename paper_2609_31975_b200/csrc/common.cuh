@@ -1,0 +1,71 @@
+// Device helpers shared by the sparse-FFN kernels (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sffn {
+
+constexpr int kActRelu = 0;
+constexpr int kActSqRelu = 1;
+constexpr int kActRsPlus = 2;
+
+// Activation of the gate (activation table of Sec. 3.1; squared RELU from the activation study).
+// For all three, A(z) != 0 exactly when z > 0 in exact arithmetic; callers test z > 0.
+__device__ __forceinline__ float activation(int act, float z) {
+  if (!(z > 0.f)) return 0.f;
+  if (act == kActRelu) return z;
+  if (act == kActSqRelu) return z * z;
+  return z / (1.f + __expf(-z));  // R-S+: z * sigmoid(z) on the non-negative side
+}
+
+// Element traits: 16-byte vectors of the storage type, unpacked to fp32.
+template <typename T>
+struct Elem;
+
+template <>
+struct Elem<float> {
+  static constexpr int kPerVec = 4;  // elements per 16 bytes
+  __device__ __forceinline__ static void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x);
+    f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z);
+    f[3] = __uint_as_float(v.w);
+  }
+  __device__ __forceinline__ static float to_float(float v) { return v; }
+};
+
+template <>
+struct Elem<__nv_bfloat16> {
+  static constexpr int kPerVec = 8;
+  // bf16 -> fp32 is a 16-bit shift: exact.
+  __device__ __forceinline__ static void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x << 16);
+    f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16);
+    f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16);
+    f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16);
+    f[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+  __device__ __forceinline__ static float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+};
+
+// Streaming 16-byte load: weights are read once, so keep them out of L1.
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+}  // namespace sffn

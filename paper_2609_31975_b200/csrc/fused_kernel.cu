@@ -1,0 +1,616 @@
+// Fused single-launch sparse gated FFN for one token on B200 (sm_100a).
+//
+// One persistent CTA per SM owns a contiguous slab of the H neurons and runs the whole of the
+// paper's sparse execution scheme (Sec. 3.1) on it without leaving the SM:
+//
+//   producer warp  one elected thread streams the slab's gate rows (W_1, or U for the LoPA gate)
+//                  into a shared-memory ring with bulk asynchronous copies (TMA, mbarrier
+//                  complete_tx).  As gate results arrive it also queues, in ascending neuron
+//                  order, the W_up / W_down rows of the neurons that fired into a second ring.
+//                  Gate streaming never waits for the up/down work, so HBM stays busy.
+//   gate warps     each takes whole ring slots: z_j = row . vec + b_g[j] (+ fixed-matrix term),
+//                  a_j = A(z_j), and reports "fired" (z_j > 0) to the producer.
+//   act warps      four warps consume the second ring in order: u_j = W_up[j] . x (CTA-level
+//                  reduction), h_j = a_j u_j, y_part += h_j W_down[j]; each thread keeps its own
+//                  column slice of y_part in registers.
+//
+// For the LoPA gate (Eq. 3, Sec. 3.3) the rank-r stage v = V x is spread over the grid, exchanged
+// through a grid barrier, normalised (RMSNorm) into shared memory by every CTA and fed to the U
+// stage of the same launch, while the producer already prefetches U rows.
+// The per-CTA partials of y are summed after a second grid barrier in fixed CTA order, each CTA
+// reducing its own column slice: the result is deterministic, and no float atomics are used.
+// Every wait (mbarrier, flag, grid barrier) is bounded by a cycle budget; when it runs out the
+// kernel records SFFN_ERR_TIMEOUT in the status word and every role winds down.
+#include "fused_kernel.cuh"
+
+#include "common.cuh"
+
+namespace sffn {
+
+namespace {
+
+constexpr int kGateWarps = 8;
+constexpr int kActWarps = 4;
+constexpr int kThreads = 32 * (1 + kGateWarps + kActWarps);  // 416
+constexpr int kActThreads = 32 * kActWarps;
+constexpr int kConsumerThreads = 32 * (kGateWarps + kActWarps);
+constexpr int kMaxGrid = 256;
+constexpr int kSmemBudget = 227 * 1024;
+constexpr long long kWaitCycles = 1LL << 31;  // about one second at B200 clocks
+
+struct FusedParams {
+  int D, H, K;  // K = length of a gate row: D (standard) or r (LoPA)
+  const void* Wgate;  // [H, K]
+  const void* W_up;
+  const void* W_down;
+  const void* x;
+  const float* b_g;
+  const void* V;
+  const int32_t* g_idx;
+  const int8_t* g_sign;
+  const float* gain;
+  int use_rmsnorm;
+  float eps;
+  float* vbuf;  // [r] exchange buffer for V x
+  int act, dense;
+  float* y;
+  float* partial;  // [grid][D]
+  uint8_t* flag;
+  int32_t* status;
+  unsigned int* bar;  // [0] arrival counter, [1] generation
+  int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
+};
+
+// Shared-memory carve-up, identical on host and device.
+struct SmemLayout {
+  int gate_ring, act_ring, sx, sn, aval, pend_a, pend_j, red, ctl, bars, row_done, total;
+  __host__ __device__ SmemLayout(int D, int K, bool lopa, int n_gate_slots, int gate_slot_bytes,
+                                 int n_act_slots, int act_slot_bytes, int slab_max) {
+    int off = 0;
+    auto take = [&](int bytes) {
+      int o = off;
+      off = (off + bytes + 127) / 128 * 128;
+      return o;
+    };
+    gate_ring = take(n_gate_slots * gate_slot_bytes);
+    act_ring = take(n_act_slots * act_slot_bytes);
+    sx = take(D * 4);
+    sn = take(lopa ? K * 4 : 0);
+    aval = take(slab_max * 4);
+    pend_a = take(slab_max * 4);
+    pend_j = take(slab_max * 4);
+    red = take(2 * kActWarps * 4);
+    ctl = take(8 * 4);
+    bars = take(2 * (n_gate_slots + n_act_slots) * 8);
+    row_done = take(slab_max);
+    total = off;
+  }
+};
+
+enum Ctl { kAbort = 0, kActFinal = 1, kActTotal = 2, kDecision = 3 /* [3], [4] */ };
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bulk asynchronous copy global -> shared, completion counted in bytes on an mbarrier.
+// Both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void named_bar(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ unsigned int ld_acquire(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(unsigned int* p, unsigned int v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status) {
+  ctl[kAbort] = 1;
+  atomicExch(status, (int32_t)SFFN_ERR_TIMEOUT);
+}
+
+// Bounded wait on an mbarrier phase.  False when the cycle budget ran out or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status) {
+  if (mbar_test(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_test(bar, parity)) return true;
+    if (ctl[kAbort]) return false;
+    if (clock64() - t0 > kWaitCycles) {
+      raise_timeout(ctl, status);
+      return false;
+    }
+  }
+}
+
+// Sense-reversing grid barrier, called by one thread per CTA (all CTAs are co-resident: the kernel
+// is launched cooperatively).  Bounded like every other wait.
+__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int n_cta, volatile int* ctl,
+                                             int32_t* status) {
+  const unsigned int gen = ld_acquire(bar + 1);
+  __threadfence();
+  const unsigned int old = atomicAdd(bar, 1u);
+  if (old == n_cta - 1) {
+    bar[0] = 0;
+    __threadfence();
+    st_release(bar + 1, gen + 1);
+    return true;
+  }
+  const long long t0 = clock64();
+  while (ld_acquire(bar + 1) == gen) {
+    if (clock64() - t0 > kWaitCycles) {
+      raise_timeout(ctl, status);
+      return false;
+    }
+    __nanosleep(32);
+  }
+  return true;
+}
+
+// Position of element k of a vector inside its shared-memory copy.  For 8-element (bf16) chunks the
+// two halves of every chunk are stored in two planes so that a warp's float4 reads are conflict-free.
+template <int EPV>
+__device__ __forceinline__ int vec_pos(int k, int len) {
+  if (EPV == 4) return k;
+  const int c = k >> 3, q = k & 7;
+  return (q < 4 ? 0 : len / 2) + 4 * c + (q & 3);
+}
+
+// Dot product of one 16-byte chunk of weights with the matching entries of the staged vector.
+template <typename T>
+__device__ __forceinline__ float chunk_dot(const uint4& w, const float* vec, int c, int nvec, float acc) {
+  constexpr int EPV = Elem<T>::kPerVec;
+  float f[EPV];
+  Elem<T>::unpack(w, f);
+  const float4 lo = reinterpret_cast<const float4*>(vec)[c];
+  acc = fmaf(f[0], lo.x, acc);
+  acc = fmaf(f[1], lo.y, acc);
+  acc = fmaf(f[2], lo.z, acc);
+  acc = fmaf(f[3], lo.w, acc);
+  if (EPV == 8) {
+    const float4 hi = reinterpret_cast<const float4*>(vec)[nvec + c];
+    acc = fmaf(f[4], hi.x, acc);
+    acc = fmaf(f[5], hi.y, acc);
+    acc = fmaf(f[6], hi.z, acc);
+    acc = fmaf(f[7], hi.w, acc);
+  }
+  return acc;
+}
+
+template <typename T, int CPT, bool LOPA>
+__global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  constexpr int EPV = Elem<T>::kPerVec;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = gridDim.x, cta = blockIdx.x;
+  const int D = p.D, K = p.K;
+  const int slab_lo = (int)((long long)p.H * cta / G);
+  const int slab_rows = (int)((long long)p.H * (cta + 1) / G) - slab_lo;
+  const int NG = p.n_gate_slots, NA = p.n_act_slots;
+  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NA, p.act_slot_bytes, p.slab_max);
+
+  unsigned char* gate_ring = smem + L.gate_ring;
+  unsigned char* act_ring = smem + L.act_ring;
+  float* sx = reinterpret_cast<float*>(smem + L.sx);
+  float* sn = reinterpret_cast<float*>(smem + L.sn);
+  float* aval = reinterpret_cast<float*>(smem + L.aval);
+  float* pend_a = reinterpret_cast<float*>(smem + L.pend_a);
+  int* pend_j = reinterpret_cast<int*>(smem + L.pend_j);
+  float* red = reinterpret_cast<float*>(smem + L.red);
+  volatile int* ctl = reinterpret_cast<volatile int*>(smem + L.ctl);
+  volatile uint8_t* row_done = smem + L.row_done;
+  const uint32_t bars = smem_u32(smem + L.bars);
+  const uint32_t full_gate = bars, empty_gate = bars + 8 * NG;
+  const uint32_t full_act = bars + 16 * NG, empty_act = bars + 16 * NG + 8 * NA;
+
+  const int nvecD = D / EPV, nvecK = K / EPV;
+  const size_t row_bytes = (size_t)D * sizeof(T);
+  const size_t gate_row_bytes = (size_t)K * sizeof(T);
+
+  // ---- prologue -----------------------------------------------------------------------------
+  if (tid == 0) {
+    for (int s = 0; s < NG; ++s) {
+      mbar_init(full_gate + 8 * s, 1);
+      mbar_init(empty_gate + 8 * s, 1);
+    }
+    for (int s = 0; s < NA; ++s) {
+      mbar_init(full_act + 8 * s, 1);
+      mbar_init(empty_act + 8 * s, kActWarps);
+    }
+    for (int i = 0; i < 8; ++i) ctl[i] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  for (int i = tid; i < slab_rows; i += kThreads) row_done[i] = 0;
+  {
+    const T* xg = static_cast<const T*>(p.x);
+    for (int k = tid; k < D; k += kThreads) sx[vec_pos<EPV>(k, D)] = Elem<T>::to_float(xg[k]);
+  }
+  __syncthreads();
+
+  const float* gvec = LOPA ? sn : sx;  // the vector every gate row is dotted with
+
+  if (warp == 0) {
+    // ======================= producer =========================================================
+    if (lane == 0) {
+      const int nr = p.rows_per_gate_slot;
+      const int n_gslots = (slab_rows + nr - 1) / nr;
+      const char* Wg = static_cast<const char*>(p.Wgate) + (size_t)slab_lo * gate_row_bytes;
+      const char* Wu = static_cast<const char*>(p.W_up);
+      const char* Wd = static_cast<const char*>(p.W_down);
+      int g_issue = 0, scan = 0, pend_head = 0, pend_tail = 0, a_issue = 0;
+      long long t_last = clock64();
+      for (;;) {
+        bool progressed = false;
+        while (scan < slab_rows) {
+          const uint8_t code = row_done[scan];
+          if (code == 0) break;
+          __threadfence_block();
+          if (code == 2 || p.dense) {
+            pend_j[pend_tail] = scan;
+            pend_a[pend_tail] = reinterpret_cast<volatile float*>(aval)[scan];
+            ++pend_tail;
+          }
+          ++scan;
+          progressed = true;
+        }
+        if (pend_head < pend_tail) {
+          const int slot = a_issue % NA;
+          if (mbar_test(empty_act + 8 * slot, ((a_issue / NA) & 1) ^ 1)) {
+            const size_t j = (size_t)(slab_lo + pend_j[pend_head]);
+            const uint32_t dst = smem_u32(act_ring + (size_t)slot * p.act_slot_bytes);
+            __threadfence_block();
+            mbar_expect_tx(full_act + 8 * slot, 2u * (uint32_t)row_bytes);
+            bulk_g2s(dst, Wu + j * row_bytes, (uint32_t)row_bytes, full_act + 8 * slot);
+            bulk_g2s(dst + (uint32_t)row_bytes, Wd + j * row_bytes, (uint32_t)row_bytes, full_act + 8 * slot);
+            ++pend_head;
+            ++a_issue;
+            progressed = true;
+          }
+        }
+        if (g_issue < n_gslots) {
+          const int slot = g_issue % NG;
+          if (mbar_test(empty_gate + 8 * slot, ((g_issue / NG) & 1) ^ 1)) {
+            const int r0 = g_issue * nr;
+            const int rows = min(nr, slab_rows - r0);
+            const uint32_t bytes = (uint32_t)(rows * gate_row_bytes);
+            mbar_expect_tx(full_gate + 8 * slot, bytes);
+            bulk_g2s(smem_u32(gate_ring + (size_t)slot * p.gate_slot_bytes), Wg + (size_t)r0 * gate_row_bytes,
+                     bytes, full_gate + 8 * slot);
+            ++g_issue;
+            progressed = true;
+          }
+        }
+        if (g_issue == n_gslots && scan == slab_rows && pend_head == pend_tail) break;
+        if (progressed) {
+          t_last = clock64();
+        } else {
+          if (ctl[kAbort]) break;
+          if (clock64() - t_last > kWaitCycles) {
+            raise_timeout(ctl, p.status);
+            break;
+          }
+        }
+      }
+      ctl[kActTotal] = a_issue;
+      __threadfence_block();
+      ctl[kActFinal] = 1;
+    }
+    __syncwarp();
+  } else {
+    const int ct = tid - 32;  // consumer thread index 0..383
+    if (LOPA) {
+      // ---- rank-r stage: v = V x spread over the grid, one V row per warp -------------------
+      const int r = K;
+      const int vlo = (int)((long long)r * cta / G), vhi = (int)((long long)r * (cta + 1) / G);
+      for (int k = vlo + (warp - 1); k < vhi; k += kGateWarps + kActWarps) {
+        const uint4* vr = reinterpret_cast<const uint4*>(static_cast<const char*>(p.V) + (size_t)k * row_bytes);
+        float acc = 0.f;
+#pragma unroll 4
+        for (int c = lane; c < nvecD; c += 32) acc = chunk_dot<T>(ld_stream16(vr + c), sx, c, nvecD, acc);
+        acc = warp_sum(acc);
+        if (lane == 0) p.vbuf[k] = acc;
+      }
+      __threadfence();
+      named_bar(1, kConsumerThreads);
+      if (ct == 0) grid_barrier(p.bar, G, ctl, p.status);
+      named_bar(1, kConsumerThreads);
+      for (int k = ct; k < r; k += kConsumerThreads) sn[vec_pos<EPV>(k, r)] = __ldcg(p.vbuf + k);
+      named_bar(1, kConsumerThreads);
+      if (p.use_rmsnorm) {
+        float ss = 0.f;
+        for (int k = lane; k < r; k += 32) {
+          const float v = sn[vec_pos<EPV>(k, r)];
+          ss = fmaf(v, v, ss);
+        }
+        ss = warp_sum(ss);  // every warp computes the same value in the same order
+        const float inv = rsqrtf(ss / (float)r + p.eps);
+        named_bar(1, kConsumerThreads);
+        for (int k = ct; k < r; k += kConsumerThreads)
+          sn[vec_pos<EPV>(k, r)] *= (p.gain ? p.gain[k] : 1.f) * inv;
+        named_bar(1, kConsumerThreads);
+      }
+    }
+
+    if (warp <= kGateWarps) {
+      // ======================= gate warps ====================================================
+      const int gw = warp - 1;
+      const int nr = p.rows_per_gate_slot;
+      const int n_gslots = (slab_rows + nr - 1) / nr;
+      for (int s = gw; s < n_gslots; s += kGateWarps) {
+        const int slot = s % NG;
+        const int r0 = s * nr;
+        const int rows = min(nr, slab_rows - r0);
+        float add = 0.f;  // bias + fixed-matrix term of the row this lane reports
+        if (lane < rows) {
+          const int j = slab_lo + r0 + lane;
+          if (p.b_g) add = p.b_g[j];
+          if (LOPA && p.g_idx) {
+            const float sg = (p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
+            add += sg * sx[vec_pos<EPV>(p.g_idx[j], D)];
+          }
+        }
+        if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status)) break;
+        const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
+        float mine = 0.f;
+        for (int rr = 0; rr < rows; ++rr) {
+          const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr * gate_row_bytes);
+          float a0 = 0.f, a1 = 0.f;
+          int c = lane;
+          for (; c + 32 < nvecK; c += 64) {
+            a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
+            a1 = chunk_dot<T>(w[c + 32], gvec, c + 32, nvecK, a1);
+          }
+          if (c < nvecK) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
+          const float z = warp_sum(a0 + a1);
+          if (lane == rr) mine = z;
+        }
+        if (lane < rows) {
+          const float z = mine + add;
+          const bool fired = z > 0.f;
+          aval[r0 + lane] = activation(p.act, z);
+          if (!p.dense) p.flag[slab_lo + r0 + lane] = fired ? 1 : 0;
+          __threadfence_block();
+          row_done[r0 + lane] = fired ? 2 : 1;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_gate + 8 * slot);
+      }
+    } else {
+      // ======================= act warps =====================================================
+      const int at = tid - 32 * (1 + kGateWarps);  // 0..127
+      const int aw = warp - 1 - kGateWarps;
+      float acc[CPT][EPV];
+#pragma unroll
+      for (int i = 0; i < CPT; ++i)
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) acc[i][e] = 0.f;
+
+      for (int k = 0;; ++k) {
+        const int slot = k % NA;
+        const uint32_t fb = full_act + 8 * slot;
+        const uint32_t par = (k / NA) & 1;
+        if (at == 0) {
+          // one thread decides for the group whether slot k exists, so nobody is left at a barrier
+          int go = 0;
+          const long long t0 = clock64();
+          for (;;) {
+            if (mbar_test(fb, par)) { go = 1; break; }
+            if (ctl[kActFinal] && k >= ctl[kActTotal]) break;
+            if (ctl[kAbort]) break;
+            if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); break; }
+          }
+          ctl[kDecision + (k & 1)] = go;
+        }
+        named_bar(2, kActThreads);
+        if (!ctl[kDecision + (k & 1)]) break;
+        for (int spin = 0; spin < (1 << 20) && !mbar_test(fb, par); ++spin) {}  // complete already: acquire
+
+        const uint4* wu = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes);
+        const uint4* wd = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes + row_bytes);
+        float part = 0.f;
+#pragma unroll
+        for (int i = 0; i < CPT; ++i) {
+          const int c = at + i * kActThreads;
+          if (c < nvecD) part = chunk_dot<T>(wu[c], sx, c, nvecD, part);
+        }
+        part = warp_sum(part);
+        if (lane == 0) red[(k & 1) * kActWarps + aw] = part;
+        named_bar(2, kActThreads);
+        const float* rp = red + (k & 1) * kActWarps;
+        const float u = (rp[0] + rp[1]) + (rp[2] + rp[3]);
+        const float h = pend_a[k] * u;
+#pragma unroll
+        for (int i = 0; i < CPT; ++i) {
+          const int c = at + i * kActThreads;
+          if (c < nvecD) {
+            float f[EPV];
+            Elem<T>::unpack(wd[c], f);
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h, f[e], acc[i][e]);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_act + 8 * slot);
+      }
+      // this CTA's partial of y
+      float* dst = p.partial + (size_t)cta * D;
+#pragma unroll
+      for (int i = 0; i < CPT; ++i) {
+        const int c = at + i * kActThreads;
+        if (c < nvecD) {
+#pragma unroll
+          for (int e = 0; e < EPV; e += 4)
+            __stcg(reinterpret_cast<float4*>(dst + (size_t)c * EPV + e),
+                   make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]));
+        }
+      }
+    }
+  }
+
+  // ---- deterministic cross-CTA reduction ------------------------------------------------------
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) grid_barrier(p.bar, G, ctl, p.status);
+  __syncthreads();
+  if (ctl[kAbort]) return;
+  const int Q = D / 4;
+  const int qlo = (int)((long long)Q * cta / G), qhi = (int)((long long)Q * (cta + 1) / G);
+  const float4* part4 = reinterpret_cast<const float4*>(p.partial);
+  for (int q = qlo + warp; q < qhi; q += kThreads / 32) {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int g = lane; g < G; g += 32) {
+      const float4 v = __ldcg(part4 + (size_t)g * Q + q);
+      s.x += v.x;
+      s.y += v.y;
+      s.z += v.z;
+      s.w += v.w;
+    }
+    s.x = warp_sum(s.x);
+    s.y = warp_sum(s.y);
+    s.z = warp_sum(s.z);
+    s.w = warp_sum(s.w);
+    if (lane == 0) reinterpret_cast<float4*>(p.y)[q] = s;
+  }
+}
+
+// ---- host side --------------------------------------------------------------------------------
+struct Geometry {
+  int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max, smem, cpt;
+  bool ok;
+};
+
+Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
+  Geometry g{};
+  const int esz = bf16 ? 2 : 4, epv = bf16 ? 8 : 4;
+  const int nvecD = D / epv;
+  const int row_bytes = D * esz, gate_row_bytes = K * esz;
+  g.ok = false;
+  if (row_bytes % 16 || gate_row_bytes % 16 || nvecD > kActThreads * 8) return g;
+  g.cpt = nvecD <= kActThreads ? 1 : nvecD <= 2 * kActThreads ? 2 : nvecD <= 4 * kActThreads ? 4 : 8;
+  int nr = 8192 / gate_row_bytes;
+  nr = nr < 1 ? 1 : nr > 32 ? 32 : nr;
+  g.rows_per_gate_slot = nr;
+  g.gate_slot_bytes = (nr * gate_row_bytes + 127) / 128 * 128;
+  g.act_slot_bytes = (2 * row_bytes + 127) / 128 * 128;
+  g.slab_max = (H + grid - 1) / grid;
+  const SmemLayout fixed(D, K, lopa, 0, 0, 0, 0, g.slab_max);
+  const int ring = kSmemBudget - fixed.total - 2048;  // slack for the barrier words
+  if (ring <= 0) return g;
+  int na = (ring / 2) / g.act_slot_bytes;
+  if (na > 16) na = 16;
+  if (na < 2) na = 2;
+  int ng = (ring - na * g.act_slot_bytes) / g.gate_slot_bytes;
+  if (ng > 32) ng = 32;
+  if (ng < 2) return g;
+  g.n_act_slots = na;
+  g.n_gate_slots = ng;
+  const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max);
+  g.smem = full.total;
+  g.ok = g.smem <= kSmemBudget;
+  return g;
+}
+
+template <typename T, bool LOPA>
+cudaError_t launch_t(const FusedParams& p, const Geometry& g, int grid, cudaStream_t s) {
+  void (*k)(const FusedParams) = nullptr;
+  switch (g.cpt) {
+    case 1: k = fused_ffn_kernel<T, 1, LOPA>; break;
+    case 2: k = fused_ffn_kernel<T, 2, LOPA>; break;
+    case 4: k = fused_ffn_kernel<T, 4, LOPA>; break;
+    default: k = fused_ffn_kernel<T, 8, LOPA>; break;
+  }
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = g.smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;  // guarantees co-residency for the grid barriers
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k, p);
+}
+
+}  // namespace
+
+size_t fused_workspace_bytes(int D, int H, int r_max) {
+  (void)H;
+  return 256 + (size_t)kMaxGrid * D * 4 + (size_t)(r_max > 0 ? r_max : 1) * 4 + 256;
+}
+
+static int fused_grid(int sm_count, int H) {
+  int grid = sm_count < kMaxGrid ? sm_count : kMaxGrid;
+  return grid > H ? H : grid;
+}
+
+bool fused_supported(bool bf16, int D, int H, int B, const sffn_gate* gate, int sm_count) {
+  if (B != 1) return false;
+  const bool lopa = gate->kind == SFFN_GATE_LOPA;
+  const int K = lopa ? gate->r : D;
+  return plan(bf16, D, H, K, lopa, fused_grid(sm_count, H)).ok;
+}
+
+cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
+  const bool lopa = c.gate->kind == SFFN_GATE_LOPA;
+  const int K = lopa ? c.gate->r : c.D;
+  const int grid = fused_grid(c.sm_count, c.H);
+  const Geometry g = plan(c.bf16, c.D, c.H, K, lopa, grid);
+  if (!g.ok) return cudaErrorInvalidValue;
+  char* ws = static_cast<char*>(c.workspace);
+  FusedParams p{};
+  p.D = c.D; p.H = c.H; p.K = K;
+  p.Wgate = lopa ? c.gate->U : c.gate->W_g;
+  p.W_up = c.W_up; p.W_down = c.W_down; p.x = c.x; p.b_g = c.b_g;
+  p.V = c.gate->V; p.g_idx = lopa ? c.gate->g_idx : nullptr; p.g_sign = c.gate->g_sign;
+  p.gain = c.gate->rms_gain; p.use_rmsnorm = c.gate->use_rmsnorm; p.eps = c.gate->rms_eps;
+  p.bar = reinterpret_cast<unsigned int*>(ws);
+  p.partial = reinterpret_cast<float*>(ws + 256);
+  p.vbuf = reinterpret_cast<float*>(ws + 256 + (size_t)kMaxGrid * c.D * 4);
+  p.act = c.act; p.dense = c.dense ? 1 : 0;
+  p.y = c.y; p.flag = c.flag; p.status = c.status;
+  p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
+  p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
+  p.slab_max = g.slab_max;
+  cudaError_t e;
+  if (c.bf16)
+    e = lopa ? launch_t<__nv_bfloat16, true>(p, g, grid, s) : launch_t<__nv_bfloat16, false>(p, g, grid, s);
+  else
+    e = lopa ? launch_t<float, true>(p, g, grid, s) : launch_t<float, false>(p, g, grid, s);
+  if (e == cudaSuccess && launched) *launched = 1;
+  return e;
+}
+
+}  // namespace sffn

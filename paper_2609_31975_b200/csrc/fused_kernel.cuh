@@ -1,0 +1,33 @@
+// Fused single-launch sparse FFN for one token (see fused_kernel.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "sparse_ffn.h"
+
+namespace sffn {
+
+struct FusedCall {
+  bool bf16;
+  int D, H;
+  const void* x;
+  const sffn_gate* gate;
+  const float* b_g;
+  const void* W_up;
+  const void* W_down;
+  int act;
+  float* y;
+  bool dense;
+  void* workspace;   // fused_workspace_bytes() bytes, zeroed at handle creation
+  int32_t* status;   // device status word
+  uint8_t* flag;     // [H] "neuron fired" bytes (sparse calls)
+  int sm_count;
+};
+
+size_t fused_workspace_bytes(int D, int H, int r_max);
+bool fused_supported(bool bf16, int D, int H, int B, const sffn_gate* gate, int sm_count);
+cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched);
+
+}  // namespace sffn

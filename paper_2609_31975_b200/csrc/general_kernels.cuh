@@ -1,0 +1,51 @@
+// Launchers of the general multi-kernel path (see general_kernels.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sffn {
+
+struct RowDotParams {
+  const void* W;     // [R, K] storage dtype
+  int R, K;
+  const void* vec;   // [NB][K] with stride vec_stride (elements); storage dtype or fp32
+  int vec_stride;
+  float* out;        // out[b * out_stride + j]
+  int out_stride;
+  // gate epilogue only
+  const float* b_g;       // [R] or null
+  const int32_t* g_idx;   // [R] or null: column of x added to the pre-activation
+  const int8_t* g_sign;   // [R] or null
+  const void* x;          // [NB][.] tokens in storage dtype (fixed-matrix term)
+  int x_stride;
+  int act;
+  uint8_t* flag;          // [R] or null: 1 where any of the NB tokens fires
+  int flag_or;            // 0: overwrite flag, 1: OR into it (later token chunks)
+};
+
+struct UpDownParams {
+  const void* W_up;    // [H, D]
+  const void* W_down;  // [H, D]
+  const void* x;       // [NB][D] storage dtype, stride x_stride
+  int x_stride;
+  const float* a;      // gate values a[b * a_stride + j]
+  int a_stride;
+  const int32_t* idx;  // list of rows, or null = all rows 0..H-1
+  const int32_t* count;  // device length of idx, or null = H
+  int H, D;
+  float* partial;      // [grid][NB][D]
+};
+
+cudaError_t launch_rowdot(bool bf16, bool vec_is_f32, int nb, bool gate, const RowDotParams& p,
+                          int sm_count, cudaStream_t s);
+cudaError_t launch_rmsnorm(const float* v, float* n, const float* gain, int r, int stride, float eps,
+                           int B, cudaStream_t s);
+cudaError_t launch_compact(const uint8_t* flag, int H, int32_t* idx, int32_t* count, cudaStream_t s);
+// Largest token chunk (4, 2 or 0 = unsupported D) the up/down kernel takes at this D.
+int updown_max_tokens(bool bf16, int D);
+cudaError_t launch_updown(bool bf16, int nb, const UpDownParams& p, int grid, cudaStream_t s);
+cudaError_t launch_reduce(const float* partial, int G, int NB, int D, float* y, int y_stride,
+                          cudaStream_t s);
+
+}  // namespace sffn

@@ -1,0 +1,252 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element, on the
+same seeded tensors.  Run with `-m gpu` on a B200."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import synthetic_inputs as syn
+from parity import assert_active_set, assert_y_close, run_oracle
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def mod():
+    import paper_2609_31975_b200 as m
+    m.load_library()
+    return m
+
+
+def make_std(D, H, dtype, seed, s):
+    w = syn.standard_ffn(D, H, dtype, seed, DEV, sparsity=s)
+    return {"W_g": w["W_g"]}, w
+
+
+def make_lopa(mod, D, H, r, dtype, seed, s, fixed="diag", sign=False, gain=False, rms=True):
+    w = syn.lopa_ffn(D, H, r, dtype, seed, DEV, sparsity=s, with_fixed_matrix=fixed is not None)
+    gate = {"V": w["V"], "U": w["U"], "use_rmsnorm": rms, "rms_eps": 1e-5, "g_idx": None}
+    if fixed == "diag":
+        gate["g_idx"] = mod.g_diagonal(H, D, DEV)
+    elif fixed == "tiled":
+        gate["g_idx"] = mod.g_tiled(H, D, DEV)
+    g = torch.Generator().manual_seed(seed)
+    if sign:
+        gate["g_sign"] = (torch.randint(0, 2, (H,), generator=g) * 2 - 1).to(torch.int8).to(DEV)
+    if gain:
+        gate["rms_gain"] = (0.5 + torch.rand(r, generator=g)).to(DEV)
+    return gate, w
+
+
+def run_both_paths(mod, ffn, x, gate, w, act, paths, tol=None, what=""):
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], act)
+    kw = {} if tol is None else dict(rel_l2=tol, max_abs=tol)
+    for path in paths:
+        ffn.set_path(path)
+        y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], act)
+        torch.cuda.synchronize()
+        assert ffn.device_status() == 0
+        assert_y_close(y, ref["y"], what=f"{what} [{path}]", **kw)
+        assert_active_set(ffn.last_active(), ref, what=f"{what} [{path}]")
+    ffn.set_path("auto")
+    return ref
+
+
+# ------------------------------------------------------------------ config 1: tiny fp32 bring-up
+def test_config1_fp32_all_64_tokens(mod):
+    D, H = 256, 1024
+    gate, w = make_std(D, H, torch.float32, 0, 0.9)
+    x = syn.tokens(64, D, torch.float32, 0, DEV)
+    ffn = mod.SparseFFN(D, H, torch.float32, B_max=1)
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    for path in ("general", "fused"):
+        ffn.set_path(path)
+        for t in range(64):
+            y = ffn.sparse_ffn_forward(x[t], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+            one = dict(y=ref["y"][t], z=ref["z"][t])
+            assert_y_close(y, one["y"], rel_l2=1e-5, max_abs=1e-5, what=f"token {t} [{path}]")
+            assert_active_set(ffn.last_active(), one, what=f"token {t} [{path}]")
+    assert ffn.device_status() == 0
+
+
+# ------------------------------------------------------------------ shrunken decode shapes, ragged sizes
+@pytest.mark.parametrize("D,H", [(512, 1000), (264, 777), (1024, 2049), (2048, 300)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_standard_gate_small_shapes(mod, D, H, dtype):
+    ffn = mod.SparseFFN(D, H, dtype, B_max=1)
+    for s, act in ((0.5, "relu"), (0.9, "sqrelu"), (0.95, "rsplus")):
+        gate, w = make_std(D, H, dtype, 21, s)
+        x = syn.tokens(3, D, dtype, 21, DEV)
+        for t in range(3):
+            run_both_paths(mod, ffn, x[t], gate, w, act, ("general", "fused"), what=f"{D}x{H} s={s} {act}")
+
+
+@pytest.mark.parametrize("r,fixed,sign,gain,rms", [
+    (64, "diag", False, False, True), (128, "tiled", True, True, True),
+    (96, None, False, False, False), (256, "diag", True, False, False)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_lopa_gate_small_shapes(mod, r, fixed, sign, gain, rms, dtype):
+    D, H = 512, 1531
+    ffn = mod.SparseFFN(D, H, dtype, r_max=256, B_max=1)
+    gate, w = make_lopa(mod, D, H, r, dtype, 31, 0.9, fixed, sign, gain, rms)
+    x = syn.tokens(2, D, dtype, 31, DEV)
+    for t in range(2):
+        for act in ("relu", "sqrelu"):
+            run_both_paths(mod, ffn, x[t], gate, w, act, ("general", "fused"), what=f"lopa r={r} {fixed}")
+
+
+# ------------------------------------------------------------------ batches: union of active sets
+@pytest.mark.parametrize("B", [2, 3, 4, 7, 16])
+def test_batched_union_general_path(mod, B):
+    D, H = 512, 1200
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=16)
+    gate, w = make_std(D, H, torch.bfloat16, 41, 0.9)
+    p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
+    w["b_g"] = syn.bias_from_firing_profile(p).to(DEV)
+    x = syn.tokens(B, D, torch.bfloat16, 41, DEV)
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert_y_close(y, ref["y"], what=f"B={B}")
+    assert_active_set(ffn.last_active(), ref, what=f"B={B}")
+    # each token of the batch equals its own single-token call
+    for b in (0, B - 1):
+        y1 = ffn.sparse_ffn_forward(x[b], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+        assert_y_close(y1, ref["y"][b], what=f"B={B} token {b} alone")
+
+
+def test_batched_lopa_general_path(mod):
+    D, H, r, B = 512, 1100, 128, 5
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=r, B_max=8)
+    gate, w = make_lopa(mod, D, H, r, torch.bfloat16, 43, 0.9, "diag", True, True, True)
+    x = syn.tokens(B, D, torch.bfloat16, 43, DEV)
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "sqrelu")
+    y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "sqrelu")
+    assert_y_close(y, ref["y"], what="batched lopa")
+    assert_active_set(ffn.last_active(), ref, what="batched lopa")
+
+
+# ------------------------------------------------------------------ degenerate cases
+@pytest.mark.parametrize("path", ["general", "fused"])
+def test_full_and_zero_sparsity(mod, path):
+    D, H = 512, 900
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=1)
+    ffn.set_path(path)
+    gate, w = make_std(D, H, torch.bfloat16, 51, None)
+    x = syn.tokens(1, D, torch.bfloat16, 51, DEV)[0]
+    lo = torch.full((H,), -1e3, device=DEV)
+    y = ffn.sparse_ffn_forward(x, gate, lo, w["W_up"], w["W_down"], "relu")
+    assert not y.any() and ffn.last_active().numel() == 0        # 100 % sparsity: y == 0 exactly
+    hi = torch.full((H,), 1e3, device=DEV)
+    y = ffn.sparse_ffn_forward(x, gate, hi, w["W_up"], w["W_down"], "relu")
+    assert ffn.last_active().tolist() == list(range(H))           # 0 % sparsity: every row
+    yd = ffn.dense_ffn_forward(x, gate, hi, w["W_up"], w["W_down"], "relu")
+    assert torch.equal(y, yd)                                      # same rows, same order, same bits
+    ref = run_oracle(x, gate, hi, w["W_up"], w["W_down"], "relu", route="dense")
+    assert_y_close(y, ref["y"], what="0% sparsity")
+    # no bias at all (the paper's form of Eq. 1)
+    y = ffn.sparse_ffn_forward(x, gate, None, w["W_up"], w["W_down"], "rsplus")
+    ref = run_oracle(x, gate, None, w["W_up"], w["W_down"], "rsplus")
+    assert_y_close(y, ref["y"], what="no bias")
+    assert_active_set(ffn.last_active(), ref, what="no bias")
+
+
+@pytest.mark.parametrize("path", ["general", "fused"])
+def test_dense_comparator_and_determinism(mod, path):
+    D, H = 1024, 3000
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=128, B_max=1)
+    ffn.set_path(path)
+    for gate, w in (make_std(D, H, torch.bfloat16, 61, 0.8),
+                    make_lopa(mod, D, H, 128, torch.bfloat16, 61, 0.8, "diag")):
+        x = syn.tokens(1, D, torch.bfloat16, 61, DEV)[0]
+        ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", route="dense")
+        yd = ffn.dense_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+        ys = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+        assert_y_close(yd, ref["y"], what="dense comparator")
+        assert_y_close(ys, yd.double().cpu().numpy(), rel_l2=1e-5, max_abs=1e-5, what="sparse vs dense (GPU)")
+        idx0 = ffn.last_active()
+        for _ in range(5):                                           # bitwise run-to-run determinism
+            y2 = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+            assert torch.equal(ys, y2) and torch.equal(idx0, ffn.last_active())
+    assert ffn.device_status() == 0
+
+
+def test_host_entry_and_errors(mod):
+    D, H = 512, 640
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=2)
+    gate, w = make_std(D, H, torch.bfloat16, 71, 0.9)
+    x = syn.tokens(2, D, torch.bfloat16, 71, DEV)
+    xh = x.cpu().pin_memory()
+    yh = torch.empty((2, D), dtype=torch.float32).pin_memory()
+    ffn.sparse_ffn_forward_host(xh, gate, w["b_g"], w["W_up"], w["W_down"], "relu", yh)
+    torch.cuda.synchronize()
+    y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert torch.equal(y.cpu(), yh)
+    n0 = ffn.launch_count()
+    ffn.sparse_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert ffn.launch_count() > n0
+    with pytest.raises(mod.SFFNError) as e:                           # B > B_max
+        ffn.sparse_ffn_forward(syn.tokens(3, D, torch.bfloat16, 1, DEV), gate, w["b_g"], w["W_up"], w["W_down"])
+    assert e.value.code == 1
+    with pytest.raises(mod.SFFNError) as e:                           # misaligned weight pointer
+        big = torch.empty(H * D + 8, dtype=torch.bfloat16, device=DEV)
+        ffn.sparse_ffn_forward(x[0], gate, w["b_g"], big[1:1 + H * D].view(H, D), w["W_down"])
+    assert e.value.code == 2
+    ffn.set_path("fused")
+    with pytest.raises(mod.SFFNError) as e:                           # the fused kernel is single-token
+        ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"])
+    assert e.value.code == 2
+    with pytest.raises(mod.SFFNError):                                # rows must be multiples of 16 bytes
+        mod.SparseFFN(260, 64, torch.bfloat16)
+
+
+# ------------------------------------------------------------------ full-size configurations
+def test_config2_full_size_decode(mod):
+    D, H = 4096, 14336
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=1)
+    for s, ntok in ((0.9, 3), (0.5, 1), (0.95, 1)):
+        gate, w = make_std(D, H, torch.bfloat16, 2, s)
+        x = syn.tokens(ntok, D, torch.bfloat16, 2, DEV)
+        for t in range(ntok):
+            ref = run_both_paths(mod, ffn, x[t], gate, w, "relu", ("general", "fused"), what=f"config2 s={s}")
+            assert abs(1 - ref["n_act"][0] / H - s) < 0.03
+        del gate, w
+
+
+def test_config3_full_size_lopa(mod):
+    D, H = 4096, 14336
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=1024, B_max=1)
+    for r, act in ((512, "relu"), (1024, "sqrelu"), (256, "relu")):
+        gate, w = make_lopa(mod, D, H, r, torch.bfloat16, 3, 0.9, "diag")
+        x = syn.tokens(1, D, torch.bfloat16, 3, DEV)[0]
+        ref = run_both_paths(mod, ffn, x, gate, w, act, ("general", "fused"), what=f"config3 r={r}")
+        assert abs(1 - ref["n_act"][0] / H - 0.9) < 0.03
+        del gate, w
+
+
+def test_config4_full_size_batched_zipf(mod):
+    D, H, B = 4096, 14336, 16
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=B)
+    gate, w = make_std(D, H, torch.bfloat16, 4, None)
+    p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
+    w["b_g"] = syn.bias_from_firing_profile(p).to(DEV)
+    x = syn.tokens(B, D, torch.bfloat16, 4, DEV)
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert_y_close(y, ref["y"], what="config4 B=16")
+    assert_active_set(ffn.last_active(), ref, what="config4 B=16")
+    frac = ref["union_mask"].mean()
+    assert abs(frac - syn.expected_union_fraction(p, B)) < 0.05
+
+
+def test_config5_full_size_stress_layer0(mod):
+    D, H = 8192, 28672
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=1024, B_max=1)
+    gate, w = make_std(D, H, torch.bfloat16, 5, 0.9)
+    x = syn.tokens(1, D, torch.bfloat16, 5, DEV)[0]
+    run_both_paths(mod, ffn, x, gate, w, "sqrelu", ("general", "fused"), what="config5 standard")
+    del gate["W_g"], w["W_g"]
+    lg, lw = make_lopa(mod, D, H, 1024, torch.bfloat16, 5, 0.9, "diag")
+    lw["W_up"], lw["W_down"] = w["W_up"], w["W_down"]
+    run_both_paths(mod, ffn, x, lg, lw, "sqrelu", ("general", "fused"), what="config5 lopa")
