@@ -129,6 +129,9 @@ int sffn_set_path(sffn_handle* h, int path) {
   return SFFN_OK;
 }
 
+// Experiment knob (not part of the documented ABI).
+void sffn_debug_set_cooperative(int on) { sffn::debug_set_cooperative(on); }
+
 int sffn_launch_count(sffn_handle* h, long long* launches) {
   if (!h || !launches) return SFFN_ERR_INVALID_ARG;
   *launches = h->launches;

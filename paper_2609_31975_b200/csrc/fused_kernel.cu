@@ -29,9 +29,13 @@ namespace sffn {
 
 namespace {
 
+constexpr int kGateProducerWarp = 0;
+constexpr int kActProducerWarp = 1;
+constexpr int kFirstGateWarp = 2;
 constexpr int kGateWarps = 8;
+constexpr int kFirstActWarp = kFirstGateWarp + kGateWarps;
 constexpr int kActWarps = 4;
-constexpr int kThreads = 32 * (1 + kGateWarps + kActWarps);  // 416
+constexpr int kThreads = 32 * (kFirstActWarp + kActWarps);  // 448
 constexpr int kActThreads = 32 * kActWarps;
 constexpr int kConsumerThreads = 32 * (kGateWarps + kActWarps);
 constexpr int kMaxGrid = 256;
@@ -59,11 +63,13 @@ struct FusedParams {
   int32_t* status;
   unsigned int* bar;  // [0] arrival counter, [1] generation
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
+  int gate_warps;  // gate warps in use; n_gate_slots is a multiple of it, so a ring slot always
+                   // belongs to the same warp and its phases are consumed strictly in order
 };
 
 // Shared-memory carve-up, identical on host and device.
 struct SmemLayout {
-  int gate_ring, act_ring, sx, sn, aval, pend_a, pend_j, red, ctl, bars, row_done, total;
+  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, row_done, total;
   __host__ __device__ SmemLayout(int D, int K, bool lopa, int n_gate_slots, int gate_slot_bytes,
                                  int n_act_slots, int act_slot_bytes, int slab_max) {
     int off = 0;
@@ -77,9 +83,8 @@ struct SmemLayout {
     sx = take(D * 4);
     sn = take(lopa ? K * 4 : 0);
     aval = take(slab_max * 4);
-    pend_a = take(slab_max * 4);
-    pend_j = take(slab_max * 4);
-    red = take(2 * kActWarps * 4);
+    slot_a = take(n_act_slots * 4);
+    red = take(2 * (kActWarps + 1) * 4);
     ctl = take(8 * 4);
     bars = take(2 * (n_gate_slots + n_act_slots) * 8);
     row_done = take(slab_max);
@@ -87,7 +92,7 @@ struct SmemLayout {
   }
 };
 
-enum Ctl { kAbort = 0, kActFinal = 1, kActTotal = 2, kDecision = 3 /* [3], [4] */ };
+enum Ctl { kAbort = 0 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -138,12 +143,27 @@ __device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status
   atomicExch(status, (int32_t)SFFN_ERR_TIMEOUT);
 }
 
-// Bounded wait on an mbarrier phase.  False when the cycle budget ran out or the CTA is aborting.
+// Bounded wait on an mbarrier phase.  try_wait parks the thread in hardware for a short,
+// implementation-defined time, so waiting warps do not steal issue slots from working ones; the
+// cycle budget is checked between attempts.  False when it ran out or the CTA is aborting.
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status) {
-  if (mbar_test(bar, parity)) return true;
+  if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
-    if (mbar_test(bar, parity)) return true;
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try(bar, parity)) return true;
     if (ctl[kAbort]) return false;
     if (clock64() - t0 > kWaitCycles) {
       raise_timeout(ctl, status);
@@ -223,8 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   float* sx = reinterpret_cast<float*>(smem + L.sx);
   float* sn = reinterpret_cast<float*>(smem + L.sn);
   float* aval = reinterpret_cast<float*>(smem + L.aval);
-  float* pend_a = reinterpret_cast<float*>(smem + L.pend_a);
-  int* pend_j = reinterpret_cast<int*>(smem + L.pend_j);
+  float* slot_a = reinterpret_cast<float*>(smem + L.slot_a);  // per act slot: gate value, < 0 = stop
   float* red = reinterpret_cast<float*>(smem + L.red);
   volatile int* ctl = reinterpret_cast<volatile int*>(smem + L.ctl);
   volatile uint8_t* row_done = smem + L.row_done;
@@ -235,6 +254,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const int nvecD = D / EPV, nvecK = K / EPV;
   const size_t row_bytes = (size_t)D * sizeof(T);
   const size_t gate_row_bytes = (size_t)K * sizeof(T);
+  const int nr = p.rows_per_gate_slot;
+  const int n_gslots = (slab_rows + nr - 1) / nr;
 
   // ---- prologue -----------------------------------------------------------------------------
   if (tid == 0) {
@@ -247,92 +268,89 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       mbar_init(empty_act + 8 * s, kActWarps);
     }
     for (int i = 0; i < 8; ++i) ctl[i] = 0;
+    for (int i = 0; i < 2 * (kActWarps + 1); ++i) red[i] = 0.f;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   for (int i = tid; i < slab_rows; i += kThreads) row_done[i] = 0;
-  {
-    const T* xg = static_cast<const T*>(p.x);
-    for (int k = tid; k < D; k += kThreads) sx[vec_pos<EPV>(k, D)] = Elem<T>::to_float(xg[k]);
+  for (int c = tid; c < D / EPV; c += kThreads) {
+    float f[EPV];
+    Elem<T>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + c), f);
+    reinterpret_cast<float4*>(sx)[c] = make_float4(f[0], f[1], f[2], f[3]);
+    if (EPV == 8) reinterpret_cast<float4*>(sx)[D / EPV + c] = make_float4(f[4], f[5], f[6], f[7]);
   }
   __syncthreads();
 
   const float* gvec = LOPA ? sn : sx;  // the vector every gate row is dotted with
 
-  if (warp == 0) {
-    // ======================= producer =========================================================
+  if (warp == kGateProducerWarp) {
+    // ======================= gate producer: stream the slab's gate rows, nothing else =========
     if (lane == 0) {
-      const int nr = p.rows_per_gate_slot;
-      const int n_gslots = (slab_rows + nr - 1) / nr;
       const char* Wg = static_cast<const char*>(p.Wgate) + (size_t)slab_lo * gate_row_bytes;
+      const uint32_t ring = smem_u32(gate_ring);
+      int slot = 0;
+      uint32_t par = 1;
+      for (int s = 0; s < n_gslots; ++s) {
+        if (!mbar_wait(empty_gate + 8 * slot, par, ctl, p.status)) break;
+        const int r0 = s * nr;
+        const uint32_t bytes = (uint32_t)(min(nr, slab_rows - r0) * gate_row_bytes);
+        mbar_expect_tx(full_gate + 8 * slot, bytes);
+        bulk_g2s(ring + (uint32_t)slot * p.gate_slot_bytes, Wg + (size_t)r0 * gate_row_bytes, bytes,
+                 full_gate + 8 * slot);
+        if (++slot == NG) { slot = 0; par ^= 1; }
+      }
+    }
+    __syncwarp();
+  } else if (warp == kActProducerWarp) {
+    // ======================= act producer: rows of fired neurons, ascending ====================
+    if (lane == 0) {
       const char* Wu = static_cast<const char*>(p.W_up);
       const char* Wd = static_cast<const char*>(p.W_down);
-      int g_issue = 0, scan = 0, pend_head = 0, pend_tail = 0, a_issue = 0;
-      long long t_last = clock64();
-      for (;;) {
-        bool progressed = false;
-        while (scan < slab_rows) {
-          const uint8_t code = row_done[scan];
-          if (code == 0) break;
+      const uint32_t ring = smem_u32(act_ring);
+      int slot = 0;
+      uint32_t par = 1;
+      bool ok = true;
+      for (int scan = 0; ok && scan <= slab_rows; ++scan) {
+        float a = -1.f;  // the entry after the last row is the stop marker
+        if (scan < slab_rows) {
+          uint8_t code = row_done[scan];
+          if (code == 0) {
+            const long long t0 = clock64();
+            while ((code = row_done[scan]) == 0) {
+              __nanosleep(20);
+              if (ctl[kAbort]) { ok = false; break; }
+              if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); ok = false; break; }
+            }
+            if (!ok) break;
+          }
+          if (code != 2 && !p.dense) continue;
           __threadfence_block();
-          if (code == 2 || p.dense) {
-            pend_j[pend_tail] = scan;
-            pend_a[pend_tail] = reinterpret_cast<volatile float*>(aval)[scan];
-            ++pend_tail;
-          }
-          ++scan;
-          progressed = true;
+          a = reinterpret_cast<volatile float*>(aval)[scan];
+          a = a < 0.f ? 0.f : a;  // activations are non-negative; keep the sign bit for the marker
         }
-        if (pend_head < pend_tail) {
-          const int slot = a_issue % NA;
-          if (mbar_test(empty_act + 8 * slot, ((a_issue / NA) & 1) ^ 1)) {
-            const size_t j = (size_t)(slab_lo + pend_j[pend_head]);
-            const uint32_t dst = smem_u32(act_ring + (size_t)slot * p.act_slot_bytes);
-            __threadfence_block();
-            mbar_expect_tx(full_act + 8 * slot, 2u * (uint32_t)row_bytes);
-            bulk_g2s(dst, Wu + j * row_bytes, (uint32_t)row_bytes, full_act + 8 * slot);
-            bulk_g2s(dst + (uint32_t)row_bytes, Wd + j * row_bytes, (uint32_t)row_bytes, full_act + 8 * slot);
-            ++pend_head;
-            ++a_issue;
-            progressed = true;
-          }
-        }
-        if (g_issue < n_gslots) {
-          const int slot = g_issue % NG;
-          if (mbar_test(empty_gate + 8 * slot, ((g_issue / NG) & 1) ^ 1)) {
-            const int r0 = g_issue * nr;
-            const int rows = min(nr, slab_rows - r0);
-            const uint32_t bytes = (uint32_t)(rows * gate_row_bytes);
-            mbar_expect_tx(full_gate + 8 * slot, bytes);
-            bulk_g2s(smem_u32(gate_ring + (size_t)slot * p.gate_slot_bytes), Wg + (size_t)r0 * gate_row_bytes,
-                     bytes, full_gate + 8 * slot);
-            ++g_issue;
-            progressed = true;
-          }
-        }
-        if (g_issue == n_gslots && scan == slab_rows && pend_head == pend_tail) break;
-        if (progressed) {
-          t_last = clock64();
+        if (!mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) break;
+        slot_a[slot] = a;
+        if (scan < slab_rows) {
+          const size_t j = (size_t)(slab_lo + scan);
+          mbar_expect_tx(full_act + 8 * slot, 2u * (uint32_t)row_bytes);
+          bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wu + j * row_bytes, (uint32_t)row_bytes,
+                   full_act + 8 * slot);
+          bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes + (uint32_t)row_bytes, Wd + j * row_bytes,
+                   (uint32_t)row_bytes, full_act + 8 * slot);
         } else {
-          if (ctl[kAbort]) break;
-          if (clock64() - t_last > kWaitCycles) {
-            raise_timeout(ctl, p.status);
-            break;
-          }
+          mbar_arrive(full_act + 8 * slot);  // stop marker: completes the phase without data
         }
+        if (++slot == NA) { slot = 0; par ^= 1; }
       }
-      ctl[kActTotal] = a_issue;
-      __threadfence_block();
-      ctl[kActFinal] = 1;
     }
     __syncwarp();
   } else {
-    const int ct = tid - 32;  // consumer thread index 0..383
+    const int ct = tid - 32 * kFirstGateWarp;  // consumer thread index 0..383
     if (LOPA) {
       // ---- rank-r stage: v = V x spread over the grid, one V row per warp -------------------
       const int r = K;
       const int vlo = (int)((long long)r * cta / G), vhi = (int)((long long)r * (cta + 1) / G);
-      for (int k = vlo + (warp - 1); k < vhi; k += kGateWarps + kActWarps) {
+      for (int k = vlo + (warp - kFirstGateWarp); k < vhi; k += kGateWarps + kActWarps) {
         const uint4* vr = reinterpret_cast<const uint4*>(static_cast<const char*>(p.V) + (size_t)k * row_bytes);
         float acc = 0.f;
 #pragma unroll 4
@@ -361,12 +379,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
     }
 
-    if (warp <= kGateWarps) {
+    if (warp < kFirstActWarp) {
       // ======================= gate warps ====================================================
-      const int gw = warp - 1;
-      const int nr = p.rows_per_gate_slot;
-      const int n_gslots = (slab_rows + nr - 1) / nr;
-      for (int s = gw; s < n_gslots; s += kGateWarps) {
+      const int gw = warp - kFirstGateWarp;
+      for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_warps) {
         const int slot = s % NG;
         const int r0 = s * nr;
         const int rows = min(nr, slab_rows - r0);
@@ -384,14 +400,17 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         float mine = 0.f;
         for (int rr = 0; rr < rows; ++rr) {
           const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr * gate_row_bytes);
-          float a0 = 0.f, a1 = 0.f;
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
           int c = lane;
-          for (; c + 32 < nvecK; c += 64) {
-            a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
-            a1 = chunk_dot<T>(w[c + 32], gvec, c + 32, nvecK, a1);
+          for (; c + 96 < nvecK; c += 128) {
+            const uint4 w0 = w[c], w1 = w[c + 32], w2 = w[c + 64], w3 = w[c + 96];
+            a0 = chunk_dot<T>(w0, gvec, c, nvecK, a0);
+            a1 = chunk_dot<T>(w1, gvec, c + 32, nvecK, a1);
+            a2 = chunk_dot<T>(w2, gvec, c + 64, nvecK, a2);
+            a3 = chunk_dot<T>(w3, gvec, c + 96, nvecK, a3);
           }
-          if (c < nvecK) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
-          const float z = warp_sum(a0 + a1);
+          for (; c < nvecK; c += 32) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
+          const float z = warp_sum((a0 + a1) + (a2 + a3));
           if (lane == rr) mine = z;
         }
         if (lane < rows) {
@@ -407,48 +426,40 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
     } else {
       // ======================= act warps =====================================================
-      const int at = tid - 32 * (1 + kGateWarps);  // 0..127
-      const int aw = warp - 1 - kGateWarps;
+      const int at = tid - 32 * kFirstActWarp;  // 0..127
+      const int aw = warp - kFirstActWarp;
       float acc[CPT][EPV];
 #pragma unroll
       for (int i = 0; i < CPT; ++i)
 #pragma unroll
         for (int e = 0; e < EPV; ++e) acc[i][e] = 0.f;
 
+      int slot = 0;
+      uint32_t par = 0;
       for (int k = 0;; ++k) {
-        const int slot = k % NA;
-        const uint32_t fb = full_act + 8 * slot;
-        const uint32_t par = (k / NA) & 1;
-        if (at == 0) {
-          // one thread decides for the group whether slot k exists, so nobody is left at a barrier
-          int go = 0;
-          const long long t0 = clock64();
-          for (;;) {
-            if (mbar_test(fb, par)) { go = 1; break; }
-            if (ctl[kActFinal] && k >= ctl[kActTotal]) break;
-            if (ctl[kAbort]) break;
-            if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); break; }
-          }
-          ctl[kDecision + (k & 1)] = go;
-        }
-        named_bar(2, kActThreads);
-        if (!ctl[kDecision + (k & 1)]) break;
-        for (int spin = 0; spin < (1 << 20) && !mbar_test(fb, par); ++spin) {}  // complete already: acquire
-
+        // Every thread waits for itself; a thread whose wait ran out still joins the barrier below
+        // and raises the group's stop flag, so the four warps always leave the loop together.
+        const bool got = mbar_wait(full_act + 8 * slot, par, ctl, p.status);
+        float* rp = red + (k & 1) * (kActWarps + 1);
+        const float a = got ? slot_a[slot] : -1.f;
+        float part = 0.f;
         const uint4* wu = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes);
         const uint4* wd = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes + row_bytes);
-        float part = 0.f;
+        if (a >= 0.f) {
 #pragma unroll
-        for (int i = 0; i < CPT; ++i) {
-          const int c = at + i * kActThreads;
-          if (c < nvecD) part = chunk_dot<T>(wu[c], sx, c, nvecD, part);
+          for (int i = 0; i < CPT; ++i) {
+            const int c = at + i * kActThreads;
+            if (c < nvecD) part = chunk_dot<T>(wu[c], sx, c, nvecD, part);
+          }
+          part = warp_sum(part);
+          if (lane == 0) rp[aw] = part;
+        } else {
+          rp[kActWarps] = 1.f;  // stop marker or failed wait
         }
-        part = warp_sum(part);
-        if (lane == 0) red[(k & 1) * kActWarps + aw] = part;
         named_bar(2, kActThreads);
-        const float* rp = red + (k & 1) * kActWarps;
+        if (rp[kActWarps] != 0.f) break;
         const float u = (rp[0] + rp[1]) + (rp[2] + rp[3]);
-        const float h = pend_a[k] * u;
+        const float h = a * u;
 #pragma unroll
         for (int i = 0; i < CPT; ++i) {
           const int c = at + i * kActThreads;
@@ -461,6 +472,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_act + 8 * slot);
+        if (++slot == NA) { slot = 0; par ^= 1; }
       }
       // this CTA's partial of y
       float* dst = p.partial + (size_t)cta * D;
@@ -504,8 +516,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
 }
 
 // ---- host side --------------------------------------------------------------------------------
+int g_debug_cooperative = 1;
+
 struct Geometry {
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max, smem, cpt;
+  int gate_warps;
   bool ok;
 };
 
@@ -526,12 +541,22 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   const SmemLayout fixed(D, K, lopa, 0, 0, 0, 0, g.slab_max);
   const int ring = kSmemBudget - fixed.total - 2048;  // slack for the barrier words
   if (ring <= 0) return g;
-  int na = (ring / 2) / g.act_slot_bytes;
-  if (na > 16) na = 16;
-  if (na < 2) na = 2;
+  // Gate ring first: two slots per gate warp hide the release -> refill latency; the act ring takes
+  // what is left (at least two slots).
+  int na = 2;
   int ng = (ring - na * g.act_slot_bytes) / g.gate_slot_bytes;
-  if (ng > 32) ng = 32;
   if (ng < 2) return g;
+  g.gate_warps = ng < kGateWarps ? ng : kGateWarps;
+  if (ng > 3 * g.gate_warps) ng = 3 * g.gate_warps;
+  ng = ng / g.gate_warps * g.gate_warps;
+  na = (ring - ng * g.gate_slot_bytes) / g.act_slot_bytes;
+  if (na > 16) na = 16;
+  if (na < 2) return g;
+  if (ng >= 3 * g.gate_warps && na < 4) {  // rebalance: the act ring matters at low sparsity
+    ng = 2 * g.gate_warps;
+    na = (ring - ng * g.gate_slot_bytes) / g.act_slot_bytes;
+    if (na > 16) na = 16;
+  }
   g.n_act_slots = na;
   g.n_gate_slots = ng;
   const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max);
@@ -549,8 +574,13 @@ cudaError_t launch_t(const FusedParams& p, const Geometry& g, int grid, cudaStre
     case 4: k = fused_ffn_kernel<T, 4, LOPA>; break;
     default: k = fused_ffn_kernel<T, 8, LOPA>; break;
   }
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, g.smem);
-  if (e != cudaSuccess) return e;
+  static bool configured[4] = {false, false, false, false};
+  const int slot = g.cpt == 1 ? 0 : g.cpt == 2 ? 1 : g.cpt == 4 ? 2 : 3;
+  if (!configured[slot]) {
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (e != cudaSuccess) return e;
+    configured[slot] = true;
+  }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kThreads);
@@ -560,11 +590,13 @@ cudaError_t launch_t(const FusedParams& p, const Geometry& g, int grid, cudaStre
   attr[0].id = cudaLaunchAttributeCooperative;  // guarantees co-residency for the grid barriers
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = g_debug_cooperative ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, k, p);
 }
 
 }  // namespace
+
+void debug_set_cooperative(int on) { g_debug_cooperative = on; }
 
 size_t fused_workspace_bytes(int D, int H, int r_max) {
   (void)H;
@@ -604,6 +636,7 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;
+  p.gate_warps = g.gate_warps;
   cudaError_t e;
   if (c.bf16)
     e = lopa ? launch_t<__nv_bfloat16, true>(p, g, grid, s) : launch_t<__nv_bfloat16, false>(p, g, grid, s);
