@@ -1,26 +1,31 @@
-// Fused single-launch sparse gated FFN for one token on B200 (sm_100a).
+// Fused sparse gated FFN for one token on B200 (sm_100a).
 //
-// One persistent CTA per SM owns a contiguous slab of the H neurons and runs the whole of the
-// paper's sparse execution scheme (Sec. 3.1) on it without leaving the SM:
+// Main kernel: one persistent CTA per SM owns a contiguous slab of the H neurons and runs the whole
+// of the paper's sparse execution scheme (Sec. 3.1) on it without leaving the SM:
 //
-//   producer warp  one elected thread streams the slab's gate rows (W_1, or U for the LoPA gate)
-//                  into a shared-memory ring with bulk asynchronous copies (TMA, mbarrier
-//                  complete_tx).  As gate results arrive it also queues, in ascending neuron
-//                  order, the W_up / W_down rows of the neurons that fired into a second ring.
-//                  Gate streaming never waits for the up/down work, so HBM stays busy.
-//   gate warps     each takes whole ring slots: z_j = row . vec + b_g[j] (+ fixed-matrix term),
-//                  a_j = A(z_j), and reports "fired" (z_j > 0) to the producer.
+//   gate producer  one thread streams the slab's gate rows (W_1, or U for the LoPA gate) into a
+//                  shared-memory ring with bulk asynchronous copies (TMA, mbarrier complete_tx).
+//                  It depends on nothing but free ring slots, so HBM stays busy from the first
+//                  cycle of the CTA to the last gate row.
+//   gate warps     each owns ring slots: z_j = row . vec + b_g[j] (+ fixed-matrix term),
+//                  a_j = A(z_j), and publishes "fired" (z_j > 0) per neuron.
+//   act producer   one thread walks the published results in ascending neuron order and queues the
+//                  W_up / W_down rows of the neurons that fired into a second ring.
 //   act warps      four warps consume the second ring in order: u_j = W_up[j] . x (CTA-level
 //                  reduction), h_j = a_j u_j, y_part += h_j W_down[j]; each thread keeps its own
-//                  column slice of y_part in registers.
+//                  column slice of y_part in registers and writes it out once.
 //
-// For the LoPA gate (Eq. 3, Sec. 3.3) the rank-r stage v = V x is spread over the grid, exchanged
-// through a grid barrier, normalised (RMSNorm) into shared memory by every CTA and fed to the U
-// stage of the same launch, while the producer already prefetches U rows.
-// The per-CTA partials of y are summed after a second grid barrier in fixed CTA order, each CTA
-// reducing its own column slice: the result is deterministic, and no float atomics are used.
-// Every wait (mbarrier, flag, grid barrier) is bounded by a cycle budget; when it runs out the
-// kernel records SFFN_ERR_TIMEOUT in the status word and every role winds down.
+// A small second kernel sums the per-CTA partials in CTA order (deterministic, no float atomics).
+// For the LoPA gate (Eq. 3, Sec. 3.3) a small first kernel computes v = V x; the main kernel
+// normalises it (RMSNorm) into shared memory and feeds it to the U stage, with the U rows already
+// being prefetched.
+//
+// The kernels are chained with programmatic dependent launch: each lets its successor start early
+// and waits (griddepcontrol.wait) only before it touches anything a predecessor may write.  Weights
+// are read before that wait -- they are parameters, not results -- so the next call's gate stream
+// starts on an SM the moment the previous call's CTA leaves it.
+// Every mbarrier / flag wait is bounded by a cycle budget; when it runs out the kernel records
+// SFFN_ERR_TIMEOUT in the status word and every role winds down.
 #include "fused_kernel.cuh"
 
 #include "common.cuh"
@@ -29,15 +34,20 @@ namespace sffn {
 
 namespace {
 
-constexpr int kGateProducerWarp = 0;
-constexpr int kActProducerWarp = 1;
-constexpr int kFirstGateWarp = 2;
+// Warp roles.  One thread can issue a bulk copy only every few hundred cycles, which caps a single
+// producer near 4 TB/s over the whole GPU; two gate producers (alternate ring slots) and two act
+// producers (W_up row / W_down row of the same slot) lift that above the HBM rate.
+constexpr int kGateProducers = 2;                          // warps 0, 1
+constexpr int kFirstActProducer = kGateProducers;          // warps 2, 3
+constexpr int kActProducers = 2;
+constexpr int kFirstGateWarp = kFirstActProducer + kActProducers;
 constexpr int kGateWarps = 8;
 constexpr int kFirstActWarp = kFirstGateWarp + kGateWarps;
 constexpr int kActWarps = 4;
-constexpr int kThreads = 32 * (kFirstActWarp + kActWarps);  // 448
+constexpr int kThreads = 32 * (kFirstActWarp + kActWarps);  // 512
 constexpr int kActThreads = 32 * kActWarps;
-constexpr int kConsumerThreads = 32 * (kGateWarps + kActWarps);
+constexpr int kStageBase = 32 * kGateProducers;  // first thread that takes part in staging the token
+constexpr int kStageThreads = kThreads - kStageBase;
 constexpr int kMaxGrid = 256;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr long long kWaitCycles = 1LL << 31;  // about one second at B200 clocks
@@ -49,22 +59,20 @@ struct FusedParams {
   const void* W_down;
   const void* x;
   const float* b_g;
-  const void* V;
   const int32_t* g_idx;
   const int8_t* g_sign;
   const float* gain;
   int use_rmsnorm;
   float eps;
-  float* vbuf;  // [r] exchange buffer for V x
+  const float* vbuf;  // [r] V x from the first kernel (LoPA)
   int act, dense;
-  float* y;
   float* partial;  // [grid][D]
   uint8_t* flag;
   int32_t* status;
-  unsigned int* bar;  // [0] arrival counter, [1] generation
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
-  int gate_warps;  // gate warps in use; n_gate_slots is a multiple of it, so a ring slot always
-                   // belongs to the same warp and its phases are consumed strictly in order
+  int gate_warps;    // gate warps in use; n_gate_slots is a multiple of it, so a ring slot always
+                     // belongs to the same warp and its phases are consumed strictly in order
+  long long* trace;  // diagnostics: [grid][16] cycle stamps, or null
 };
 
 // Shared-memory carve-up, identical on host and device.
@@ -107,11 +115,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -126,17 +134,17 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
       "l"(src), "r"(bytes), "r"(bar)
       : "memory");
 }
-__device__ __forceinline__ void named_bar(int id, int threads) {
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
-__device__ __forceinline__ unsigned int ld_acquire(const unsigned int* p) {
-  unsigned int v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
+__device__ __forceinline__ void named_bar_arrive(int id, int threads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
-__device__ __forceinline__ void st_release(unsigned int* p, unsigned int v) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+// Programmatic dependent launch: let the next kernel in the stream start / wait for the previous one.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status) {
   ctl[kAbort] = 1;
@@ -146,17 +154,6 @@ __device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status
 // Bounded wait on an mbarrier phase.  try_wait parks the thread in hardware for a short,
 // implementation-defined time, so waiting warps do not steal issue slots from working ones; the
 // cycle budget is checked between attempts.  False when it ran out or the CTA is aborting.
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
@@ -170,30 +167,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       return false;
     }
   }
-}
-
-// Sense-reversing grid barrier, called by one thread per CTA (all CTAs are co-resident: the kernel
-// is launched cooperatively).  Bounded like every other wait.
-__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int n_cta, volatile int* ctl,
-                                             int32_t* status) {
-  const unsigned int gen = ld_acquire(bar + 1);
-  __threadfence();
-  const unsigned int old = atomicAdd(bar, 1u);
-  if (old == n_cta - 1) {
-    bar[0] = 0;
-    __threadfence();
-    st_release(bar + 1, gen + 1);
-    return true;
-  }
-  const long long t0 = clock64();
-  while (ld_acquire(bar + 1) == gen) {
-    if (clock64() - t0 > kWaitCycles) {
-      raise_timeout(ctl, status);
-      return false;
-    }
-    __nanosleep(32);
-  }
-  return true;
 }
 
 // Position of element k of a vector inside its shared-memory copy.  For 8-element (bf16) chunks the
@@ -226,9 +199,27 @@ __device__ __forceinline__ float chunk_dot(const uint4& w, const float* vec, int
   return acc;
 }
 
+__device__ __forceinline__ long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return (long long)t;
+}
+#define SFFN_GSTAMP(slot)                                                    \
+  do {                                                                       \
+    if (p.trace) p.trace[(size_t)blockIdx.x * 16 + (slot)] = global_ns();    \
+  } while (0)
+
+#define SFFN_STAMP(slot)                                                          \
+  do {                                                                            \
+    if (p.trace) p.trace[(size_t)blockIdx.x * 16 + (slot)] = clock64() - t_entry; \
+  } while (0)
+
 template <typename T, int CPT, bool LOPA>
 __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
+  const long long t_entry = clock64();
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) SFFN_GSTAMP(10);
   constexpr int EPV = Elem<T>::kPerVec;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x, cta = blockIdx.x;
@@ -257,56 +248,80 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const int nr = p.rows_per_gate_slot;
   const int n_gslots = (slab_rows + nr - 1) / nr;
 
-  // ---- prologue -----------------------------------------------------------------------------
-  if (tid == 0) {
-    for (int s = 0; s < NG; ++s) {
-      mbar_init(full_gate + 8 * s, 1);
-      mbar_init(empty_gate + 8 * s, 1);
+  if (warp < kGateProducers) {
+    // ======================= gate producers ===================================================
+    // Warp 0 sets up the barriers; both producer warps then start streaming at once (alternate
+    // ring slots): the weights do not depend on anything earlier in the stream.
+    if (warp == 0 && lane == 0) {
+      for (int s = 0; s < NG; ++s) {
+        mbar_init(full_gate + 8 * s, 1);
+        mbar_init(empty_gate + 8 * s, 1);
+      }
+      for (int s = 0; s < NA; ++s) {
+        mbar_init(full_act + 8 * s, kActProducers);
+        mbar_init(empty_act + 8 * s, kActWarps);
+      }
+      for (int i = 0; i < 8; ++i) ctl[i] = 0;
+      for (int i = 0; i < 2 * (kActWarps + 1); ++i) red[i] = 0.f;
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (int s = 0; s < NA; ++s) {
-      mbar_init(full_act + 8 * s, 1);
-      mbar_init(empty_act + 8 * s, kActWarps);
-    }
-    for (int i = 0; i < 8; ++i) ctl[i] = 0;
-    for (int i = 0; i < 2 * (kActWarps + 1); ++i) red[i] = 0.f;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  for (int i = tid; i < slab_rows; i += kThreads) row_done[i] = 0;
-  for (int c = tid; c < D / EPV; c += kThreads) {
-    float f[EPV];
-    Elem<T>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + c), f);
-    reinterpret_cast<float4*>(sx)[c] = make_float4(f[0], f[1], f[2], f[3]);
-    if (EPV == 8) reinterpret_cast<float4*>(sx)[D / EPV + c] = make_float4(f[4], f[5], f[6], f[7]);
-  }
-  __syncthreads();
-
-  const float* gvec = LOPA ? sn : sx;  // the vector every gate row is dotted with
-
-  if (warp == kGateProducerWarp) {
-    // ======================= gate producer: stream the slab's gate rows, nothing else =========
+    named_bar_sync(4, 32 * kGateProducers);  // barriers are initialised
+    named_bar_arrive(3, kThreads);           // release the other warps (they block on barrier 3)
     if (lane == 0) {
       const char* Wg = static_cast<const char*>(p.Wgate) + (size_t)slab_lo * gate_row_bytes;
       const uint32_t ring = smem_u32(gate_ring);
-      int slot = 0;
-      uint32_t par = 1;
-      for (int s = 0; s < n_gslots; ++s) {
-        if (!mbar_wait(empty_gate + 8 * slot, par, ctl, p.status)) break;
+      for (int s = warp; s < n_gslots; s += kGateProducers) {
+        const int slot = s % NG;
+        if (!mbar_wait(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status)) break;
         const int r0 = s * nr;
         const uint32_t bytes = (uint32_t)(min(nr, slab_rows - r0) * gate_row_bytes);
         mbar_expect_tx(full_gate + 8 * slot, bytes);
         bulk_g2s(ring + (uint32_t)slot * p.gate_slot_bytes, Wg + (size_t)r0 * gate_row_bytes, bytes,
                  full_gate + 8 * slot);
-        if (++slot == NG) { slot = 0; par ^= 1; }
       }
+      if (warp == 0) SFFN_STAMP(1);
     }
     __syncwarp();
-  } else if (warp == kActProducerWarp) {
-    // ======================= act producer: rows of fired neurons, ascending ====================
+    return;
+  }
+
+  // ---- everyone else: wait for the predecessor in the stream, then stage the token ------------
+  pdl_wait();
+  if (tid == kStageBase) SFFN_GSTAMP(11);
+  for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) row_done[i] = 0;
+  for (int c = tid - kStageBase; c < nvecD; c += kStageThreads) {
+    float f[EPV];
+    Elem<T>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + c), f);
+    reinterpret_cast<float4*>(sx)[c] = make_float4(f[0], f[1], f[2], f[3]);
+    if (EPV == 8) reinterpret_cast<float4*>(sx)[nvecD + c] = make_float4(f[4], f[5], f[6], f[7]);
+  }
+  if (LOPA) {
+    // n = RMSNorm(V x) (or V x) into shared memory; every warp derives the same scale
+    const int r = K;
+    float ss = 0.f;
+    for (int k = lane; k < r; k += 32) {
+      const float v = __ldcg(p.vbuf + k);
+      ss = fmaf(v, v, ss);
+    }
+    ss = warp_sum(ss);
+    const float inv = p.use_rmsnorm ? rsqrtf(ss / (float)r + p.eps) : 1.f;
+    for (int k = tid - kStageBase; k < r; k += kStageThreads)
+      sn[vec_pos<EPV>(k, r)] = __ldcg(p.vbuf + k) * ((p.use_rmsnorm && p.gain) ? p.gain[k] : 1.f) * inv;
+  }
+  named_bar_sync(3, kThreads);
+  if (tid == kStageBase) SFFN_STAMP(0);
+
+  const float* gvec = LOPA ? sn : sx;  // the vector every gate row is dotted with
+
+  if (warp < kFirstGateWarp) {
+    // ======================= act producers: rows of fired neurons, ascending ===================
+    // Both walk the published gate results in the same order; producer 0 copies the W_up row of a
+    // fired neuron, producer 1 its W_down row, into the same ring slot.
+    const int ap = warp - kFirstActProducer;
     if (lane == 0) {
-      const char* Wu = static_cast<const char*>(p.W_up);
-      const char* Wd = static_cast<const char*>(p.W_down);
-      const uint32_t ring = smem_u32(act_ring);
+      const char* Wsrc = static_cast<const char*>(ap == 0 ? p.W_up : p.W_down);
+      const uint32_t ring = smem_u32(act_ring) + (ap == 0 ? 0u : (uint32_t)row_bytes);
       int slot = 0;
       uint32_t par = 1;
       bool ok = true;
@@ -326,197 +341,208 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
           if (code != 2 && !p.dense) continue;
           __threadfence_block();
           a = reinterpret_cast<volatile float*>(aval)[scan];
-          a = a < 0.f ? 0.f : a;  // activations are non-negative; keep the sign bit for the marker
+          a = a < 0.f ? 0.f : a;  // activations are non-negative; the sign is the stop marker
         }
         if (!mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) break;
-        slot_a[slot] = a;
+        if (ap == 0) slot_a[slot] = a;
         if (scan < slab_rows) {
           const size_t j = (size_t)(slab_lo + scan);
-          mbar_expect_tx(full_act + 8 * slot, 2u * (uint32_t)row_bytes);
-          bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wu + j * row_bytes, (uint32_t)row_bytes,
+          mbar_expect_tx(full_act + 8 * slot, (uint32_t)row_bytes);
+          bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
                    full_act + 8 * slot);
-          bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes + (uint32_t)row_bytes, Wd + j * row_bytes,
-                   (uint32_t)row_bytes, full_act + 8 * slot);
         } else {
           mbar_arrive(full_act + 8 * slot);  // stop marker: completes the phase without data
         }
         if (++slot == NA) { slot = 0; par ^= 1; }
       }
+      if (ap == 0) SFFN_STAMP(2);
     }
     __syncwarp();
-  } else {
-    const int ct = tid - 32 * kFirstGateWarp;  // consumer thread index 0..383
-    if (LOPA) {
-      // ---- rank-r stage: v = V x spread over the grid, one V row per warp -------------------
-      const int r = K;
-      const int vlo = (int)((long long)r * cta / G), vhi = (int)((long long)r * (cta + 1) / G);
-      for (int k = vlo + (warp - kFirstGateWarp); k < vhi; k += kGateWarps + kActWarps) {
-        const uint4* vr = reinterpret_cast<const uint4*>(static_cast<const char*>(p.V) + (size_t)k * row_bytes);
-        float acc = 0.f;
-#pragma unroll 4
-        for (int c = lane; c < nvecD; c += 32) acc = chunk_dot<T>(ld_stream16(vr + c), sx, c, nvecD, acc);
-        acc = warp_sum(acc);
-        if (lane == 0) p.vbuf[k] = acc;
-      }
-      __threadfence();
-      named_bar(1, kConsumerThreads);
-      if (ct == 0) grid_barrier(p.bar, G, ctl, p.status);
-      named_bar(1, kConsumerThreads);
-      for (int k = ct; k < r; k += kConsumerThreads) sn[vec_pos<EPV>(k, r)] = __ldcg(p.vbuf + k);
-      named_bar(1, kConsumerThreads);
-      if (p.use_rmsnorm) {
-        float ss = 0.f;
-        for (int k = lane; k < r; k += 32) {
-          const float v = sn[vec_pos<EPV>(k, r)];
-          ss = fmaf(v, v, ss);
+  } else if (warp < kFirstActWarp) {
+    // ======================= gate warps ========================================================
+    const int gw = warp - kFirstGateWarp;
+    for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_warps) {
+      const int slot = s % NG;
+      const int r0 = s * nr;
+      const int rows = min(nr, slab_rows - r0);
+      float add = 0.f;  // bias + fixed-matrix term of the row this lane reports
+      if (lane < rows) {
+        const int j = slab_lo + r0 + lane;
+        if (p.b_g) add = p.b_g[j];
+        if (LOPA && p.g_idx) {
+          const float sg = (p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
+          add += sg * sx[vec_pos<EPV>(p.g_idx[j], D)];
         }
-        ss = warp_sum(ss);  // every warp computes the same value in the same order
-        const float inv = rsqrtf(ss / (float)r + p.eps);
-        named_bar(1, kConsumerThreads);
-        for (int k = ct; k < r; k += kConsumerThreads)
-          sn[vec_pos<EPV>(k, r)] *= (p.gain ? p.gain[k] : 1.f) * inv;
-        named_bar(1, kConsumerThreads);
       }
+      if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status)) break;
+      const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
+      float mine = 0.f;
+      for (int rr = 0; rr < rows; ++rr) {
+        const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr * gate_row_bytes);
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        int c = lane;
+        for (; c + 96 < nvecK; c += 128) {
+          const uint4 w0 = w[c], w1 = w[c + 32], w2 = w[c + 64], w3 = w[c + 96];
+          a0 = chunk_dot<T>(w0, gvec, c, nvecK, a0);
+          a1 = chunk_dot<T>(w1, gvec, c + 32, nvecK, a1);
+          a2 = chunk_dot<T>(w2, gvec, c + 64, nvecK, a2);
+          a3 = chunk_dot<T>(w3, gvec, c + 96, nvecK, a3);
+        }
+        for (; c < nvecK; c += 32) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
+        const float z = warp_sum((a0 + a1) + (a2 + a3));
+        if (lane == rr) mine = z;
+      }
+      if (lane < rows) {
+        const float z = mine + add;
+        const bool fired = z > 0.f;
+        aval[r0 + lane] = activation(p.act, z);
+        if (!p.dense) p.flag[slab_lo + r0 + lane] = fired ? 1 : 0;
+        __threadfence_block();
+        row_done[r0 + lane] = fired ? 2 : 1;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_gate + 8 * slot);
     }
+    if (lane == 0 && gw == (n_gslots - 1) % p.gate_warps) SFFN_STAMP(3);
+  } else {
+    // ======================= act warps =========================================================
+    const int at = tid - 32 * kFirstActWarp;  // 0..127
+    const int aw = warp - kFirstActWarp;
+    float acc[CPT][EPV];
+#pragma unroll
+    for (int i = 0; i < CPT; ++i)
+#pragma unroll
+      for (int e = 0; e < EPV; ++e) acc[i][e] = 0.f;
 
-    if (warp < kFirstActWarp) {
-      // ======================= gate warps ====================================================
-      const int gw = warp - kFirstGateWarp;
-      for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_warps) {
-        const int slot = s % NG;
-        const int r0 = s * nr;
-        const int rows = min(nr, slab_rows - r0);
-        float add = 0.f;  // bias + fixed-matrix term of the row this lane reports
-        if (lane < rows) {
-          const int j = slab_lo + r0 + lane;
-          if (p.b_g) add = p.b_g[j];
-          if (LOPA && p.g_idx) {
-            const float sg = (p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
-            add += sg * sx[vec_pos<EPV>(p.g_idx[j], D)];
-          }
-        }
-        if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status)) break;
-        const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
-        float mine = 0.f;
-        for (int rr = 0; rr < rows; ++rr) {
-          const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr * gate_row_bytes);
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-          int c = lane;
-          for (; c + 96 < nvecK; c += 128) {
-            const uint4 w0 = w[c], w1 = w[c + 32], w2 = w[c + 64], w3 = w[c + 96];
-            a0 = chunk_dot<T>(w0, gvec, c, nvecK, a0);
-            a1 = chunk_dot<T>(w1, gvec, c + 32, nvecK, a1);
-            a2 = chunk_dot<T>(w2, gvec, c + 64, nvecK, a2);
-            a3 = chunk_dot<T>(w3, gvec, c + 96, nvecK, a3);
-          }
-          for (; c < nvecK; c += 32) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
-          const float z = warp_sum((a0 + a1) + (a2 + a3));
-          if (lane == rr) mine = z;
-        }
-        if (lane < rows) {
-          const float z = mine + add;
-          const bool fired = z > 0.f;
-          aval[r0 + lane] = activation(p.act, z);
-          if (!p.dense) p.flag[slab_lo + r0 + lane] = fired ? 1 : 0;
-          __threadfence_block();
-          row_done[r0 + lane] = fired ? 2 : 1;
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_gate + 8 * slot);
-      }
-    } else {
-      // ======================= act warps =====================================================
-      const int at = tid - 32 * kFirstActWarp;  // 0..127
-      const int aw = warp - kFirstActWarp;
-      float acc[CPT][EPV];
-#pragma unroll
-      for (int i = 0; i < CPT; ++i)
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) acc[i][e] = 0.f;
-
-      int slot = 0;
-      uint32_t par = 0;
-      for (int k = 0;; ++k) {
-        // Every thread waits for itself; a thread whose wait ran out still joins the barrier below
-        // and raises the group's stop flag, so the four warps always leave the loop together.
-        const bool got = mbar_wait(full_act + 8 * slot, par, ctl, p.status);
-        float* rp = red + (k & 1) * (kActWarps + 1);
-        const float a = got ? slot_a[slot] : -1.f;
-        float part = 0.f;
-        const uint4* wu = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes);
-        const uint4* wd = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes + row_bytes);
-        if (a >= 0.f) {
-#pragma unroll
-          for (int i = 0; i < CPT; ++i) {
-            const int c = at + i * kActThreads;
-            if (c < nvecD) part = chunk_dot<T>(wu[c], sx, c, nvecD, part);
-          }
-          part = warp_sum(part);
-          if (lane == 0) rp[aw] = part;
-        } else {
-          rp[kActWarps] = 1.f;  // stop marker or failed wait
-        }
-        named_bar(2, kActThreads);
-        if (rp[kActWarps] != 0.f) break;
-        const float u = (rp[0] + rp[1]) + (rp[2] + rp[3]);
-        const float h = a * u;
+    int slot = 0;
+    uint32_t par = 0;
+    for (int k = 0;; ++k) {
+      // Every thread waits for itself; a thread whose wait ran out still joins the barrier below
+      // and raises the group's stop flag, so the four warps always leave the loop together.
+      const bool got = mbar_wait(full_act + 8 * slot, par, ctl, p.status);
+      float* rp = red + (k & 1) * (kActWarps + 1);
+      const float a = got ? slot_a[slot] : -1.f;
+      float part = 0.f;
+      const uint4* wu = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes);
+      const uint4* wd = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes + row_bytes);
+      if (a >= 0.f) {
 #pragma unroll
         for (int i = 0; i < CPT; ++i) {
           const int c = at + i * kActThreads;
-          if (c < nvecD) {
-            float f[EPV];
-            Elem<T>::unpack(wd[c], f);
-#pragma unroll
-            for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h, f[e], acc[i][e]);
-          }
+          if (c < nvecD) part = chunk_dot<T>(wu[c], sx, c, nvecD, part);
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_act + 8 * slot);
-        if (++slot == NA) { slot = 0; par ^= 1; }
+        part = warp_sum(part);
+        if (lane == 0) rp[aw] = part;
+      } else {
+        rp[kActWarps] = 1.f;  // stop marker or failed wait
       }
-      // this CTA's partial of y
-      float* dst = p.partial + (size_t)cta * D;
+      named_bar_sync(2, kActThreads);
+      if (rp[kActWarps] != 0.f) break;
+      const float u = (rp[0] + rp[1]) + (rp[2] + rp[3]);
+      const float h = a * u;
 #pragma unroll
       for (int i = 0; i < CPT; ++i) {
         const int c = at + i * kActThreads;
         if (c < nvecD) {
+          float f[EPV];
+          Elem<T>::unpack(wd[c], f);
 #pragma unroll
-          for (int e = 0; e < EPV; e += 4)
-            __stcg(reinterpret_cast<float4*>(dst + (size_t)c * EPV + e),
-                   make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]));
+          for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h, f[e], acc[i][e]);
         }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_act + 8 * slot);
+      if (++slot == NA) { slot = 0; par ^= 1; }
     }
+    if (at == 0) SFFN_STAMP(4);
+    // this CTA's partial of y
+    float* dst = p.partial + (size_t)cta * D;
+#pragma unroll
+    for (int i = 0; i < CPT; ++i) {
+      const int c = at + i * kActThreads;
+      if (c < nvecD) {
+#pragma unroll
+        for (int e = 0; e < EPV; e += 4)
+          __stcg(reinterpret_cast<float4*>(dst + (size_t)c * EPV + e),
+                 make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]));
+      }
+    }
+    if (at == 0) SFFN_STAMP(5);
+    if (at == 0) SFFN_GSTAMP(12);
   }
+}
 
-  // ---- deterministic cross-CTA reduction ------------------------------------------------------
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) grid_barrier(p.bar, G, ctl, p.status);
-  __syncthreads();
-  if (ctl[kAbort]) return;
+// y[d] = sum over CTAs of partial[cta][d] in a fixed order.  One warp per float4 column: lane l adds
+// the partials l, l+32, ... (every load issued before the first add: one L2 round trip), then a fixed
+// shuffle tree combines the lanes.
+__global__ void __launch_bounds__(256) fused_reduce_kernel(const float* partial, int G, int D, float* y,
+                                                           const int32_t* status, long long* trace) {
+  pdl_launch_dependents();
+  if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)G * 16 + blockIdx.x] = global_ns();
+  pdl_wait();
+  if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)(G + 1) * 16 + blockIdx.x] = global_ns();
   const int Q = D / 4;
-  const int qlo = (int)((long long)Q * cta / G), qhi = (int)((long long)Q * (cta + 1) / G);
-  const float4* part4 = reinterpret_cast<const float4*>(p.partial);
-  for (int q = qlo + warp; q < qhi; q += kThreads / 32) {
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int g = lane; g < G; g += 32) {
-      const float4 v = __ldcg(part4 + (size_t)g * Q + q);
-      s.x += v.x;
-      s.y += v.y;
-      s.z += v.z;
-      s.w += v.w;
+  const int q = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int l = threadIdx.x & 31;
+  if (q < Q) {
+    const float4* src = reinterpret_cast<const float4*>(partial) + q;
+    float4 v[8];  // G <= 256
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int g = l + 32 * i;
+      v[i] = g < G ? __ldcg(src + (size_t)g * Q) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 s = v[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) {
+      s.x += v[i].x;
+      s.y += v[i].y;
+      s.z += v[i].z;
+      s.w += v[i].w;
     }
     s.x = warp_sum(s.x);
     s.y = warp_sum(s.y);
     s.z = warp_sum(s.z);
     s.w = warp_sum(s.w);
-    if (lane == 0) reinterpret_cast<float4*>(p.y)[q] = s;
+    if (l == 0 && *status == 0) reinterpret_cast<float4*>(y)[q] = s;
+  }
+  if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)(G + 2) * 16 + blockIdx.x] = global_ns();
+}
+
+// LoPA rank-r stage: v = V x, one warp per row of V.
+template <typename T>
+__global__ void __launch_bounds__(256) lopa_v_kernel(const void* V, const void* x, int r, int D, float* v) {
+  extern __shared__ __align__(16) float sxv[];
+  constexpr int EPV = Elem<T>::kPerVec;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int nvecD = D / EPV;
+  for (int c = threadIdx.x; c < nvecD; c += blockDim.x) {
+    float f[EPV];
+    Elem<T>::unpack(__ldg(reinterpret_cast<const uint4*>(x) + c), f);
+    reinterpret_cast<float4*>(sxv)[c] = make_float4(f[0], f[1], f[2], f[3]);
+    if (EPV == 8) reinterpret_cast<float4*>(sxv)[nvecD + c] = make_float4(f[4], f[5], f[6], f[7]);
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int k = blockIdx.x * 8 + warp; k < r; k += gridDim.x * 8) {
+    const uint4* vr = reinterpret_cast<const uint4*>(static_cast<const char*>(V) + (size_t)k * D * sizeof(T));
+    float a0 = 0.f, a1 = 0.f;
+    int c = lane;
+    for (; c + 32 < nvecD; c += 64) {
+      const uint4 w0 = ld_stream16(vr + c), w1 = ld_stream16(vr + c + 32);
+      a0 = chunk_dot<T>(w0, sxv, c, nvecD, a0);
+      a1 = chunk_dot<T>(w1, sxv, c + 32, nvecD, a1);
+    }
+    if (c < nvecD) a0 = chunk_dot<T>(ld_stream16(vr + c), sxv, c, nvecD, a0);
+    const float s = warp_sum(a0 + a1);
+    if (lane == 0) v[k] = s;
   }
 }
 
 // ---- host side --------------------------------------------------------------------------------
-int g_debug_cooperative = 1;
+int g_debug_pdl = 1;
+long long* g_debug_trace = nullptr;
 
 struct Geometry {
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max, smem, cpt;
@@ -546,7 +572,7 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   int na = 2;
   int ng = (ring - na * g.act_slot_bytes) / g.gate_slot_bytes;
   if (ng < 2) return g;
-  g.gate_warps = ng < kGateWarps ? ng : kGateWarps;
+  g.gate_warps = (ng < kGateWarps ? ng : kGateWarps) & ~1;  // even: slots alternate between two producers
   if (ng > 3 * g.gate_warps) ng = 3 * g.gate_warps;
   ng = ng / g.gate_warps * g.gate_warps;
   na = (ring - ng * g.gate_slot_bytes) / g.act_slot_bytes;
@@ -565,8 +591,30 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   return g;
 }
 
+int fused_grid(int sm_count, int H) {
+  int grid = sm_count < kMaxGrid ? sm_count : kMaxGrid;
+  return grid > H ? H : grid;
+}
+
+// Launch with the programmatic-stream-serialization attribute: the kernel may begin while its
+// predecessor in the stream is still running; its griddepcontrol.wait restores the ordering.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*k)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_debug_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, k, args...);
+}
+
 template <typename T, bool LOPA>
-cudaError_t launch_t(const FusedParams& p, const Geometry& g, int grid, cudaStream_t s) {
+cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaStream_t s) {
   void (*k)(const FusedParams) = nullptr;
   switch (g.cpt) {
     case 1: k = fused_ffn_kernel<T, 1, LOPA>; break;
@@ -581,37 +629,39 @@ cudaError_t launch_t(const FusedParams& p, const Geometry& g, int grid, cudaStre
     if (e != cudaSuccess) return e;
     configured[slot] = true;
   }
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = g.smem;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeCooperative;  // guarantees co-residency for the grid barriers
-  attr[0].val.cooperative = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = g_debug_cooperative ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, k, p);
+  return launch_pdl(k, dim3(grid), dim3(kThreads), (size_t)g.smem, s, p);
+}
+
+template <typename T>
+cudaError_t launch_v(const FusedCall& c, float* vbuf, cudaStream_t s) {
+  const int r = c.gate->r;
+  const size_t smem = (size_t)c.D * 4;
+  auto k = lopa_v_kernel<T>;
+  static bool configured = false;
+  if (!configured && smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int grid = (r + 7) / 8;
+  return launch_pdl(k, dim3(grid), dim3(256), smem, s, c.gate->V, c.x, r, c.D, vbuf);
 }
 
 }  // namespace
 
-void debug_set_cooperative(int on) { g_debug_cooperative = on; }
+void debug_set_pdl(int on) { g_debug_pdl = on; }
+void debug_set_trace(long long* device_buffer) { g_debug_trace = device_buffer; }
 
 size_t fused_workspace_bytes(int D, int H, int r_max) {
   (void)H;
   return 256 + (size_t)kMaxGrid * D * 4 + (size_t)(r_max > 0 ? r_max : 1) * 4 + 256;
 }
 
-static int fused_grid(int sm_count, int H) {
-  int grid = sm_count < kMaxGrid ? sm_count : kMaxGrid;
-  return grid > H ? H : grid;
-}
-
 bool fused_supported(bool bf16, int D, int H, int B, const sffn_gate* gate, int sm_count) {
   if (B != 1) return false;
   const bool lopa = gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? gate->r : D;
+  if (lopa && (size_t)D * 4 > 128 * 1024) return false;
   return plan(bf16, D, H, K, lopa, fused_grid(sm_count, H)).ok;
 }
 
@@ -622,28 +672,43 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   const Geometry g = plan(c.bf16, c.D, c.H, K, lopa, grid);
   if (!g.ok) return cudaErrorInvalidValue;
   char* ws = static_cast<char*>(c.workspace);
+  float* partial = reinterpret_cast<float*>(ws + 256);
+  float* vbuf = reinterpret_cast<float*>(ws + 256 + (size_t)kMaxGrid * c.D * 4);
+  int n = 0;
+  cudaError_t e;
+  if (lopa) {
+    e = c.bf16 ? launch_v<__nv_bfloat16>(c, vbuf, s) : launch_v<float>(c, vbuf, s);
+    if (e != cudaSuccess) return e;
+    ++n;
+  }
   FusedParams p{};
   p.D = c.D; p.H = c.H; p.K = K;
   p.Wgate = lopa ? c.gate->U : c.gate->W_g;
   p.W_up = c.W_up; p.W_down = c.W_down; p.x = c.x; p.b_g = c.b_g;
-  p.V = c.gate->V; p.g_idx = lopa ? c.gate->g_idx : nullptr; p.g_sign = c.gate->g_sign;
+  p.g_idx = lopa ? c.gate->g_idx : nullptr; p.g_sign = c.gate->g_sign;
   p.gain = c.gate->rms_gain; p.use_rmsnorm = c.gate->use_rmsnorm; p.eps = c.gate->rms_eps;
-  p.bar = reinterpret_cast<unsigned int*>(ws);
-  p.partial = reinterpret_cast<float*>(ws + 256);
-  p.vbuf = reinterpret_cast<float*>(ws + 256 + (size_t)kMaxGrid * c.D * 4);
+  p.vbuf = vbuf;
+  p.partial = partial;
   p.act = c.act; p.dense = c.dense ? 1 : 0;
-  p.y = c.y; p.flag = c.flag; p.status = c.status;
+  p.flag = c.flag; p.status = c.status;
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;
   p.gate_warps = g.gate_warps;
-  cudaError_t e;
+  p.trace = g_debug_trace;
   if (c.bf16)
-    e = lopa ? launch_t<__nv_bfloat16, true>(p, g, grid, s) : launch_t<__nv_bfloat16, false>(p, g, grid, s);
+    e = lopa ? launch_main<__nv_bfloat16, true>(p, g, grid, s) : launch_main<__nv_bfloat16, false>(p, g, grid, s);
   else
-    e = lopa ? launch_t<float, true>(p, g, grid, s) : launch_t<float, false>(p, g, grid, s);
-  if (e == cudaSuccess && launched) *launched = 1;
-  return e;
+    e = lopa ? launch_main<float, true>(p, g, grid, s) : launch_main<float, false>(p, g, grid, s);
+  if (e != cudaSuccess) return e;
+  ++n;
+  const int Q = c.D / 4;
+  e = launch_pdl(fused_reduce_kernel, dim3((Q + 7) / 8), dim3(256), 0, s, (const float*)partial, grid, c.D,
+                 c.y, (const int32_t*)c.status, g_debug_trace);
+  if (e != cudaSuccess) return e;
+  ++n;
+  if (launched) *launched = n;
+  return cudaSuccess;
 }
 
 }  // namespace sffn
