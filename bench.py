@@ -222,7 +222,7 @@ def run_ours(args, rank, world, local):
 
     dev = torch.device(f"cuda:{local}")
     torch.cuda.set_device(dev)
-    wl = Workload(m, dev)
+    wl = Workload(m, dev, tokens=args.calls)
     n_act = wl.count_active()
     mean_rows = statistics.mean(n_act)
     bytes_per_call = statistics.mean(m.touched_bytes(D_MODEL, D_FF, n, 2) for n in n_act)
@@ -234,11 +234,16 @@ def run_ours(args, rank, world, local):
     with ClockSampler(local) as clk:
         ms = time_steps(wl.step, args.steps, args.warmup, world, dev, stream)
     launches = (wl.ffn.launch_count() - l0) * args.steps // (args.steps + args.warmup)
-    calls = args.steps * CALLS_PER_STEP
+    calls = args.steps * args.calls
     us_call = ms * 1e3 / calls
+    if args.skip_extras:
+        if rank == 0:
+            print(json.dumps({"metric": "us_per_ffn_call", "value": us_call / world, "unit": "us/FFN-call",
+                              "note": "sparse path only (profiling run, not a bench line)"}))
+        return
     dsteps = max(1, args.steps // 2)
     ms_dense = time_steps(lambda: wl.step("dense"), dsteps, 1, world, dev, stream)
-    us_dense = ms_dense * 1e3 / (dsteps * CALLS_PER_STEP)
+    us_dense = ms_dense * 1e3 / (dsteps * args.calls)
     ms_e2e = time_steps(lambda: wl.step("host"), args.steps, 1, world, dev, stream)
     us_e2e = ms_e2e * 1e3 / calls
     status = wl.ffn.device_status()
@@ -252,7 +257,7 @@ def run_ours(args, rank, world, local):
         "metric": "us_per_ffn_call", "value": us_call / world, "unit": "us/FFN-call", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "step": f"{CALLS_PER_STEP} single-token FFN calls, one token each",
+        "config": {"workload": WORKLOAD, "step": f"{args.calls} single-token FFN calls, one token each",
                    "l2": f"rotating over {WEIGHT_SETS} independent weight sets ({WEIGHT_SETS * dense_bytes / 1e9:.2f} GB) "
                          "so inputs exceed L2", "storage": "bf16 weights and tokens, fp32 accumulation and output",
                    "measured_sparsity": 1.0 - mean_rows / D_FF, "parallelism": f"{world} independent replicas"},
@@ -263,9 +268,9 @@ def run_ours(args, rank, world, local):
         "speedup_vs_dense": us_dense / us_call,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
-                     "kernel": "fused_ffn_kernel (one launch per FFN call)"},
-        "e2e": {"value": us_e2e / world, "unit": "us/FFN-call", "h2d_bytes_per_step": CALLS_PER_STEP * D_MODEL * 2,
-                "d2h_bytes_per_step": CALLS_PER_STEP * D_MODEL * 4},
+                     "kernel": "fused_ffn_kernel + fused_reduce_kernel (the two launches of one FFN call, chained by programmatic dependent launch)"},
+        "e2e": {"value": us_e2e / world, "unit": "us/FFN-call", "h2d_bytes_per_step": args.calls * D_MODEL * 2,
+                "d2h_bytes_per_step": args.calls * D_MODEL * 4},
         "gpu_launches": launches, "clocks": clk.summary(),
         "cpu_baseline": cpu_baseline() if world == 1 else None,
     }
@@ -279,6 +284,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--report", default=None, help="write the wider measurement matrix to this JSON file")
+    ap.add_argument("--calls", type=int, default=CALLS_PER_STEP, help="FFN calls (tokens) per step")
+    ap.add_argument("--skip-extras", action="store_true",
+                    help="time the sparse path only (no dense comparator, host-buffer or CPU legs): for profiler runs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank, world, local = dist_setup(args.gpus)
