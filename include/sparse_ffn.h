@@ -139,6 +139,35 @@ int sffn_last_device_status(sffn_handle* handle, int* status);
 /* Number of kernels this handle has launched since creation (host-side counter). */
 int sffn_launch_count(sffn_handle* handle, long long* launches);
 
+/* Sparse FFN without a handle, a workspace or any allocation -- the paper has no counterpart; this
+ * entry point exists for callers that cannot obtain device memory at call time: code that runs after
+ * the application has given all of HBM to its own pool (so cudaMalloc fails, or is forbidden by the
+ * host framework), or inside a latency-critical loop where the device-wide synchronisation that
+ * cudaMalloc/cudaFree imply is not acceptable, and that own no buffer they could pass to sffn_create.
+ *
+ * Standard gate, one token (B = 1): y = W_down^T (A(W_g x + b_g) . (W_up x)), sparse execution as
+ * in sparse_ffn_forward, computed by the general-path kernels.  x [D], W_g / W_up / W_down [H, D] in
+ * `dtype` (sffn_dtype), b_g [H] fp32 or NULL, y [D] fp32: all DEVICE pointers owned by the caller,
+ * 16-byte aligned, rows a multiple of 16 bytes.
+ *
+ * Scratch: the gate values, fired flags, index list and per-CTA partial sums live in one array that
+ * is part of this library's device image (about 4.3 MB; every GPU that loads the library keeps it
+ * until the process exits).  That fixes the limits D <= SFFN_STATIC_MAX_D and H <= SFFN_STATIC_MAX_H;
+ * larger shapes return SFFN_ERR_UNSUPPORTED (use a handle with your own workspace instead).
+ * The call makes no cudaMalloc / cudaFree and calls no allocating library routine.
+ *
+ * The first call on each device looks up the array's device address (one cudaGetSymbolAddress with
+ * that device current) and remembers it; make that first call before any stream capture begins.
+ * All calls on a device share the one array, which keeps the previous call's contents: a call
+ * rewrites everything it later reads and clears the list length itself, so back-to-back calls on
+ * one stream are independent -- but two calls that can overlap on the GPU (different streams, or
+ * different host threads on different streams) race on it and must be serialised by the caller. */
+#define SFFN_STATIC_MAX_D 8192
+#define SFFN_STATIC_MAX_H 32768
+int sparse_ffn_forward_static(const void* x, const void* W_g, const float* b_g, const void* W_up,
+                              const void* W_down, int D, int H, int dtype, int act, float* y,
+                              void* stream);
+
 /* Static string for a status code. */
 const char* sffn_status_string(int status);
 

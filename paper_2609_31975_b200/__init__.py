@@ -11,5 +11,6 @@ from .binding import (  # noqa: F401
     SparseFFN,
     lib_path,
     load_library,
+    sparse_ffn_forward_static,
 )
 from .lopa import g_diagonal, g_tiled, touched_bytes, dense_bytes  # noqa: F401

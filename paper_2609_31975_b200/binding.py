@@ -55,6 +55,7 @@ def load_library() -> ctypes.CDLL:
         lib.sffn_last_active.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
         lib.sffn_last_device_status.argtypes = [vp, ctypes.POINTER(i)]
         lib.sffn_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
+        lib.sparse_ffn_forward_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, vp]
         lib.sffn_status_string.argtypes = [i]
         lib.sffn_status_string.restype = ctypes.c_char_p
         _lib = lib
@@ -68,6 +69,25 @@ def _ptr(t):
 def _check(where: str, rc: int):
     if rc != 0:
         raise SFFNError(where, rc)
+
+
+def sparse_ffn_forward_static(x, W_g, b_g, W_up, W_down, act="relu", y=None, stream=None):
+    """Handle-free, allocation-free variant (standard gate, one token): the library's built-in
+    scratch array replaces the workspace.  For callers that cannot allocate device memory at call
+    time; shapes are limited to D <= 8192, H <= 32768, and calls that may overlap on the GPU must be
+    serialised by the caller (they share the scratch).  `y` must be supplied by such a caller; it
+    is created here only as a convenience for tests."""
+    lib = load_library()
+    H, D = W_up.shape
+    if y is None:
+        y = torch.empty(D, dtype=torch.float32, device=x.device)
+    s = torch.cuda.current_stream(x.device) if stream is None else stream
+    _check("sparse_ffn_forward_static",
+           lib.sparse_ffn_forward_static(_ptr(x), _ptr(W_g), _ptr(b_g), _ptr(W_up), _ptr(W_down), D, H,
+                                         1 if W_up.dtype == torch.bfloat16 else 0,
+                                         ACT[act] if isinstance(act, str) else int(act), _ptr(y),
+                                         ctypes.c_void_p(s.cuda_stream)))
+    return y
 
 
 class SparseFFN:
