@@ -6,6 +6,7 @@
 
 #include <new>
 
+#include "batched_kernels.cuh"
 #include "fused_kernel.cuh"
 #include "general_kernels.cuh"
 
@@ -13,11 +14,14 @@ namespace {
 
 constexpr int kMaxUpDownGrid = 304;  // upper bound of the up/down grid (2 CTAs per SM on 148 SMs)
 constexpr int kMaxChunk = 4;         // tokens per pass of the general kernels
+constexpr int kMaxSplits = 16;       // union-row splits of the batched down projection
+constexpr int kMaxMmaTokens = 64;    // tokens per pass of the batched tensor-core kernels
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-  size_t status, act, flag, idx, v, n, partial, xstage, ystage, fused, total;
+  size_t status, act, flag, idx, v, n, partial, xstage, ystage, fused, hmT, x2, total;
+  int hm_stride;
 };
 
 Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
@@ -35,10 +39,15 @@ Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
   L.idx = take((size_t)H * 4);
   L.v = take((size_t)B_max * (r_max > 0 ? r_max : 1) * 4);
   L.n = take((size_t)B_max * (r_max > 0 ? r_max : 1) * 4);
-  L.partial = take((size_t)kMaxUpDownGrid * kMaxChunk * D * 4);
+  const size_t part_general = (size_t)kMaxUpDownGrid * kMaxChunk * D * 4;
+  const size_t part_batched = (size_t)kMaxSplits * (B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * D * 4;
+  L.partial = take(part_general > part_batched ? part_general : part_batched);
   L.xstage = take((size_t)B_max * D * esz);
   L.ystage = take((size_t)B_max * D * 4);
   L.fused = take(sffn::fused_workspace_bytes(D, H, r_max));
+  L.hm_stride = (H + 15) / 16 * 16 + 16;
+  L.hmT = take((size_t)(B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * L.hm_stride * 2);
+  L.x2 = take((size_t)2 * (B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * (r_max > 0 ? r_max : 1) * 2);
   L.total = off;
   return L;
 }
@@ -167,6 +176,94 @@ int check_call(const sffn_handle* h, const void* x, int B, const sffn_gate* g, c
     if ((expr) != cudaSuccess) return SFFN_ERR_CUDA; \
   } while (0)
 
+// Batched tensor-core path (bf16, B >= 2): gate GEMM -> compaction of the union -> up GEMM over the
+// union rows -> down GEMM (split over D-slices and union chunks) -> fixed-order sum of the splits.
+// Tokens are taken kMaxMmaTokens at a time; the union (and the list) is that of the whole batch.
+int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
+                const void* W_up, const void* W_down, int act, float* y, bool dense, cudaStream_t s) {
+  using namespace sffn;
+  const int D = h->D, H = h->H;
+  float* actbuf = h->at<float>(h->L.act);
+  uint8_t* flag = h->at<uint8_t>(h->L.flag);
+  int32_t* idx = h->at<int32_t>(h->L.idx);
+  int32_t* count = h->at<int32_t>(h->L.status) + 1;
+  const int rs = h->r_max > 0 ? h->r_max : 1;
+  float* vbuf = h->at<float>(h->L.v);
+  float* nbuf = h->at<float>(h->L.n);
+  const char* xb = static_cast<const char*>(x);
+  const bool lopa = g->kind == SFFN_GATE_LOPA;
+  const int grid_rows = 2 * h->sm_count;
+
+  if (lopa) {  // v = V x on the CUDA-core row kernel (r rows only), then RMSNorm
+    for (int b0 = 0; b0 < B;) {
+      const int nb = B - b0 >= 4 ? 4 : B - b0 >= 2 ? 2 : 1;
+      RowDotParams p{};
+      p.W = g->V; p.R = g->r; p.K = D;
+      p.vec = xb + (size_t)b0 * D * 2; p.vec_stride = D;
+      p.out = vbuf + (size_t)b0 * rs; p.out_stride = rs;
+      SFFN_CUDA(launch_rowdot(true, false, nb, false, p, h->sm_count, s));
+      ++h->launches;
+      b0 += nb;
+    }
+    if (g->use_rmsnorm) {
+      SFFN_CUDA(launch_rmsnorm(vbuf, nbuf, g->rms_gain, g->r, rs, g->rms_eps, B, s));
+      ++h->launches;
+    }
+  }
+  for (int b0 = 0; b0 < B; b0 += kMaxMmaTokens) {
+    const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
+    RowsMmaParams p{};
+    p.R = H; p.B = nb;
+    p.b_g = b_g; p.act = act;
+    p.xtok = xb + (size_t)b0 * D * 2; p.xtok_stride = D;
+    p.a_out = actbuf + (size_t)b0 * H; p.a_stride = H;
+    p.flag = dense ? nullptr : flag;
+    int cols = nb;
+    if (lopa) {
+      void* x2 = h->ws + h->L.x2;
+      SFFN_CUDA(launch_split_bf16((g->use_rmsnorm ? nbuf : vbuf) + (size_t)b0 * rs, nb, g->r, rs, x2, s));
+      ++h->launches;
+      p.W = g->U; p.K = g->r; p.X = x2; p.x_stride = g->r; p.split_cols = 1;
+      p.g_idx = g->g_idx; p.g_sign = g->g_sign;
+      cols = 2 * nb;
+    } else {
+      p.W = g->W_g; p.K = D; p.X = p.xtok; p.x_stride = D;
+    }
+    p.ncols_valid = cols;
+    if (b0 > 0 && !dense) return SFFN_ERR_UNSUPPORTED;  // flags of later chunks would need OR-ing
+    SFFN_CUDA(launch_rows_mma(false, p, cols, grid_rows, s));
+    ++h->launches;
+  }
+  if (!dense) {
+    SFFN_CUDA(launch_compact(flag, H, idx, count, s));
+    ++h->launches;
+    h->list_state = 1;
+  }
+  int splits = h->sm_count / (D / 256);
+  splits = splits < 1 ? 1 : splits > kMaxSplits ? kMaxSplits : splits;
+  float* partial = h->at<float>(h->L.partial);
+  void* hmT = h->ws + h->L.hmT;
+  for (int b0 = 0; b0 < B; b0 += kMaxMmaTokens) {
+    const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
+    RowsMmaParams p{};
+    p.W = W_up; p.R = H; p.K = D;
+    p.idx = dense ? nullptr : idx; p.count = dense ? nullptr : count;
+    p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
+    p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
+    p.hmT = hmT; p.hm_stride = h->L.hm_stride;
+    SFFN_CUDA(launch_rows_mma(true, p, nb, grid_rows, s));
+    DownMmaParams d{};
+    d.W_down = W_down; d.R = H; d.D = D;
+    d.idx = p.idx; d.count = p.count;
+    d.hmT = hmT; d.hm_stride = h->L.hm_stride; d.B = nb;
+    d.partial = partial;
+    SFFN_CUDA(launch_down_mma(d, splits, s));
+    SFFN_CUDA(launch_reduce(partial, splits, nb, D, y + (size_t)b0 * D, D, s));
+    h->launches += 3;
+  }
+  return SFFN_OK;
+}
+
 // General path: gate (all tokens, chunks of <= 4) -> compaction -> up/down + reduce per chunk.
 int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
                 const void* W_up, const void* W_down, int act, float* y, bool dense,
@@ -273,6 +370,11 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
     if (!dense) h->list_state = 2;
     return SFFN_OK;
   }
+  const int gate_k = g->kind == SFFN_GATE_LOPA ? g->r : h->D;
+  const int gate_cols = g->kind == SFFN_GATE_LOPA ? 2 * (B < kMaxMmaTokens ? B : kMaxMmaTokens) : B;
+  if (h->dtype == SFFN_BF16 && B >= 2 && B <= kMaxMmaTokens && h->path != SFFN_PATH_GENERAL &&
+      sffn::batched_mma_supported(h->D, gate_k, gate_cols))
+    return run_batched(h, x, B, g, b_g, W_up, W_down, act, y, dense, s);
   return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, s);
 }
 

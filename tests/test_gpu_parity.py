@@ -98,33 +98,43 @@ def test_lopa_gate_small_shapes(mod, r, fixed, sign, gain, rms, dtype):
 
 
 # ------------------------------------------------------------------ batches: union of active sets
-@pytest.mark.parametrize("B", [2, 3, 4, 7, 16])
-def test_batched_union_general_path(mod, B):
+@pytest.mark.parametrize("path", ["general", "auto"])     # auto = tensor-core kernels for bf16 batches
+@pytest.mark.parametrize("B", [2, 3, 4, 7, 16, 33, 64])
+def test_batched_union(mod, B, path):
     D, H = 512, 1200
-    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=16)
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=64)
+    ffn.set_path(path)
     gate, w = make_std(D, H, torch.bfloat16, 41, 0.9)
     p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
     w["b_g"] = syn.bias_from_firing_profile(p).to(DEV)
     x = syn.tokens(B, D, torch.bfloat16, 41, DEV)
     ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
     y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
-    assert_y_close(y, ref["y"], what=f"B={B}")
-    assert_active_set(ffn.last_active(), ref, what=f"B={B}")
+    assert_y_close(y, ref["y"], what=f"B={B} [{path}]")
+    assert_active_set(ffn.last_active(), ref, what=f"B={B} [{path}]")
+    y2 = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert torch.equal(y, y2)                                    # run-to-run determinism
+    yd = ffn.dense_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    dref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", route="dense")
+    assert_y_close(yd, dref["y"], what=f"dense B={B} [{path}]")
     # each token of the batch equals its own single-token call
     for b in (0, B - 1):
         y1 = ffn.sparse_ffn_forward(x[b], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
         assert_y_close(y1, ref["y"][b], what=f"B={B} token {b} alone")
 
 
-def test_batched_lopa_general_path(mod):
-    D, H, r, B = 512, 1100, 128, 5
-    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=r, B_max=8)
-    gate, w = make_lopa(mod, D, H, r, torch.bfloat16, 43, 0.9, "diag", True, True, True)
+@pytest.mark.parametrize("path", ["general", "auto"])
+@pytest.mark.parametrize("B,r,rms", [(5, 128, True), (16, 64, True), (24, 96, False)])
+def test_batched_lopa(mod, B, r, rms, path):
+    D, H = 512, 1100
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=128, B_max=32)
+    ffn.set_path(path)
+    gate, w = make_lopa(mod, D, H, r, torch.bfloat16, 43, 0.9, "diag", True, rms, rms)
     x = syn.tokens(B, D, torch.bfloat16, 43, DEV)
     ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "sqrelu")
     y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "sqrelu")
-    assert_y_close(y, ref["y"], what="batched lopa")
-    assert_active_set(ffn.last_active(), ref, what="batched lopa")
+    assert_y_close(y, ref["y"], what=f"batched lopa [{path}]")
+    assert_active_set(ffn.last_active(), ref, what=f"batched lopa [{path}]")
 
 
 # ------------------------------------------------------------------ degenerate cases
@@ -225,17 +235,18 @@ def test_config3_full_size_lopa(mod):
         del gate, w
 
 
-def test_config4_full_size_batched_zipf(mod):
-    D, H, B = 4096, 14336, 16
+@pytest.mark.parametrize("B", [4, 16, 64])
+def test_config4_full_size_batched_zipf(mod, B):
+    D, H = 4096, 14336
     ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=B)
     gate, w = make_std(D, H, torch.bfloat16, 4, None)
     p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
     w["b_g"] = syn.bias_from_firing_profile(p).to(DEV)
     x = syn.tokens(B, D, torch.bfloat16, 4, DEV)
-    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", threads=16)
     y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
-    assert_y_close(y, ref["y"], what="config4 B=16")
-    assert_active_set(ffn.last_active(), ref, what="config4 B=16")
+    assert_y_close(y, ref["y"], what=f"config4 B={B}")
+    assert_active_set(ffn.last_active(), ref, what=f"config4 B={B}")
     frac = ref["union_mask"].mean()
     assert abs(frac - syn.expected_union_fraction(p, B)) < 0.05
 
@@ -250,3 +261,10 @@ def test_config5_full_size_stress_layer0(mod):
     lg, lw = make_lopa(mod, D, H, 1024, torch.bfloat16, 5, 0.9, "diag")
     lw["W_up"], lw["W_down"] = w["W_up"], w["W_down"]
     run_both_paths(mod, ffn, x, lg, lw, "sqrelu", ("general", "fused"), what="config5 lopa")
+    ffn8 = mod.SparseFFN(D, H, torch.bfloat16, r_max=1024, B_max=8)          # config 5, batch 8
+    x8 = syn.tokens(8, D, torch.bfloat16, 5, DEV, extra=1)
+    for gt, ww in ((lg, lw),):
+        ref = run_oracle(x8, gt, ww["b_g"], ww["W_up"], ww["W_down"], "sqrelu", threads=8)
+        y = ffn8.sparse_ffn_forward(x8, gt, ww["b_g"], ww["W_up"], ww["W_down"], "sqrelu")
+        assert_y_close(y, ref["y"], what="config5 lopa B=8")
+        assert_active_set(ffn8.last_active(), ref, what="config5 lopa B=8")
