@@ -284,6 +284,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--report", default=None, help="write the wider measurement matrix to this JSON file")
+    ap.add_argument("--quick", action="store_true", help="with --report: one point per family")
     ap.add_argument("--calls", type=int, default=CALLS_PER_STEP, help="FFN calls (tokens) per step")
     ap.add_argument("--skip-extras", action="store_true",
                     help="time the sparse path only (no dense comparator, host-buffer or CPU legs): for profiler runs")
@@ -296,7 +297,8 @@ def main():
         elif args.report:
             from paper_2609_31975_b200 import report
 
-            report.run(args.report)
+            if rank == 0:
+                report.run(args.report, quick=args.quick)
         else:
             run_ours(args, rank, world, local)
     finally:

@@ -65,10 +65,12 @@ typedef enum { SFFN_F32 = 0, SFFN_BF16 = 1 } sffn_dtype;
 
 typedef enum { SFFN_GATE_STANDARD = 0, SFFN_GATE_LOPA = 1 } sffn_gate_kind;
 
-/* Which kernels serve a call.  AUTO picks the fused single-launch kernel for B = 1 when the shape
- * allows it and the general multi-kernel path otherwise; the other two force one of them
- * (SFFN_ERR_UNSUPPORTED if the forced path cannot serve the call). */
-typedef enum { SFFN_PATH_AUTO = 0, SFFN_PATH_GENERAL = 1, SFFN_PATH_FUSED = 2 } sffn_path;
+/* Which kernels serve a call.  AUTO picks the fused kernels for B = 1 when the shape allows it, the
+ * tcgen05 tensor-core kernels for bf16 batches (B >= 2) and the general CUDA-core kernels otherwise;
+ * the others force one family (SFFN_ERR_UNSUPPORTED if it cannot serve the call): GENERAL = CUDA-core
+ * kernels for any batch, FUSED = single-token fused kernels, MMA_SYNC = batched kernels on the
+ * warp-level mma.sync tensor-core path. */
+typedef enum { SFFN_PATH_AUTO = 0, SFFN_PATH_GENERAL = 1, SFFN_PATH_FUSED = 2, SFFN_PATH_MMA_SYNC = 3 } sffn_path;
 
 /* Gate description.  STANDARD uses W_g only.  LOPA (Eq. 3; "LoPA in practice", Sec. 3.3) uses
  *   z_j = g_sign[j] * x[g_idx[j]] + sum_k U[j,k] n_k + b_g[j],   n = RMSNorm(V x) or V x,

@@ -8,7 +8,7 @@ import torch
 
 _PKG = Path(__file__).resolve().parent
 ACT = {"relu": 0, "sqrelu": 1, "rsplus": 2}
-PATH = {"auto": 0, "general": 1, "fused": 2}
+PATH = {"auto": 0, "general": 1, "fused": 2, "mma_sync": 3}
 _STATUS = {0: "ok", 1: "invalid argument", 2: "unsupported shape, alignment or path",
            3: "workspace missing, misaligned or too small", 4: "CUDA runtime error",
            5: "device-side bounded wait ran out"}

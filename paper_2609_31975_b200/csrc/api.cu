@@ -9,6 +9,7 @@
 #include "batched_kernels.cuh"
 #include "fused_kernel.cuh"
 #include "general_kernels.cuh"
+#include "umma_kernels.cuh"
 
 namespace {
 
@@ -133,7 +134,7 @@ int sffn_destroy(sffn_handle* h) {
 }
 
 int sffn_set_path(sffn_handle* h, int path) {
-  if (!h || path < SFFN_PATH_AUTO || path > SFFN_PATH_FUSED) return SFFN_ERR_INVALID_ARG;
+  if (!h || path < SFFN_PATH_AUTO || path > SFFN_PATH_MMA_SYNC) return SFFN_ERR_INVALID_ARG;
   h->path = path;
   return SFFN_OK;
 }
@@ -180,7 +181,8 @@ int check_call(const sffn_handle* h, const void* x, int B, const sffn_gate* g, c
 // union rows -> down GEMM (split over D-slices and union chunks) -> fixed-order sum of the splits.
 // Tokens are taken kMaxMmaTokens at a time; the union (and the list) is that of the whole batch.
 int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
-                const void* W_up, const void* W_down, int act, float* y, bool dense, cudaStream_t s) {
+                const void* W_up, const void* W_down, int act, float* y, bool dense, bool umma,
+                cudaStream_t s) {
   using namespace sffn;
   const int D = h->D, H = h->H;
   float* actbuf = h->at<float>(h->L.act);
@@ -212,26 +214,47 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
   }
   for (int b0 = 0; b0 < B; b0 += kMaxMmaTokens) {
     const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
-    RowsMmaParams p{};
-    p.R = H; p.B = nb;
-    p.b_g = b_g; p.act = act;
-    p.xtok = xb + (size_t)b0 * D * 2; p.xtok_stride = D;
-    p.a_out = actbuf + (size_t)b0 * H; p.a_stride = H;
-    p.flag = dense ? nullptr : flag;
-    int cols = nb;
-    if (lopa) {
-      void* x2 = h->ws + h->L.x2;
-      SFFN_CUDA(launch_split_bf16((g->use_rmsnorm ? nbuf : vbuf) + (size_t)b0 * rs, nb, g->r, rs, x2, s));
-      ++h->launches;
-      p.W = g->U; p.K = g->r; p.X = x2; p.x_stride = g->r; p.split_cols = 1;
-      p.g_idx = g->g_idx; p.g_sign = g->g_sign;
-      cols = 2 * nb;
-    } else {
-      p.W = g->W_g; p.K = D; p.X = p.xtok; p.x_stride = D;
-    }
-    p.ncols_valid = cols;
+    void* x2 = h->ws + h->L.x2;
+    const float* nsrc = (g->use_rmsnorm ? nbuf : vbuf) + (size_t)b0 * rs;
+    const void* xtok = xb + (size_t)b0 * D * 2;
     if (b0 > 0 && !dense) return SFFN_ERR_UNSUPPORTED;  // flags of later chunks would need OR-ing
-    SFFN_CUDA(launch_rows_mma(false, p, cols, grid_rows, s));
+    if (umma) {
+      UmmaRowsParams p{};
+      p.R = H; p.B = nb; p.b_g = b_g; p.act = act; p.status = h->at<int32_t>(h->L.status);
+      p.xtok = xtok; p.xtok_stride = D;
+      p.a_out = actbuf + (size_t)b0 * H; p.a_stride = H;
+      p.flag = dense ? nullptr : flag;
+      int cols = nb;
+      if (lopa) {
+        SFFN_CUDA(launch_split_interleaved(nsrc, nb, g->r, rs, x2, s));
+        ++h->launches;
+        p.W = g->U; p.K = g->r; p.X = x2; p.x_stride = g->r; p.split_cols = 1;
+        p.g_idx = g->g_idx; p.g_sign = g->g_sign;
+        cols = 2 * nb;
+      } else {
+        p.W = g->W_g; p.K = D; p.X = xtok; p.x_stride = D;
+      }
+      p.ncols_valid = cols;
+      SFFN_CUDA(launch_umma_rows(false, p, cols, h->sm_count, s));
+    } else {
+      RowsMmaParams p{};
+      p.R = H; p.B = nb; p.b_g = b_g; p.act = act;
+      p.xtok = xtok; p.xtok_stride = D;
+      p.a_out = actbuf + (size_t)b0 * H; p.a_stride = H;
+      p.flag = dense ? nullptr : flag;
+      int cols = nb;
+      if (lopa) {
+        SFFN_CUDA(launch_split_bf16(nsrc, nb, g->r, rs, x2, s));
+        ++h->launches;
+        p.W = g->U; p.K = g->r; p.X = x2; p.x_stride = g->r; p.split_cols = 1;
+        p.g_idx = g->g_idx; p.g_sign = g->g_sign;
+        cols = 2 * nb;
+      } else {
+        p.W = g->W_g; p.K = D; p.X = xtok; p.x_stride = D;
+      }
+      p.ncols_valid = cols;
+      SFFN_CUDA(launch_rows_mma(false, p, cols, grid_rows, s));
+    }
     ++h->launches;
   }
   if (!dense) {
@@ -245,16 +268,26 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
   void* hmT = h->ws + h->L.hmT;
   for (int b0 = 0; b0 < B; b0 += kMaxMmaTokens) {
     const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
-    RowsMmaParams p{};
-    p.W = W_up; p.R = H; p.K = D;
-    p.idx = dense ? nullptr : idx; p.count = dense ? nullptr : count;
-    p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
-    p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
-    p.hmT = hmT; p.hm_stride = h->L.hm_stride;
-    SFFN_CUDA(launch_rows_mma(true, p, nb, grid_rows, s));
+    const int32_t* lidx = dense ? nullptr : idx;
+    const int32_t* lcount = dense ? nullptr : count;
+    if (umma) {
+      UmmaRowsParams p{};
+      p.W = W_up; p.R = H; p.K = D; p.idx = lidx; p.count = lcount;
+      p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
+      p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
+      p.hmT = hmT; p.hm_stride = h->L.hm_stride; p.status = h->at<int32_t>(h->L.status);
+      SFFN_CUDA(launch_umma_rows(true, p, nb, h->sm_count, s));
+    } else {
+      RowsMmaParams p{};
+      p.W = W_up; p.R = H; p.K = D; p.idx = lidx; p.count = lcount;
+      p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
+      p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
+      p.hmT = hmT; p.hm_stride = h->L.hm_stride;
+      SFFN_CUDA(launch_rows_mma(true, p, nb, grid_rows, s));
+    }
     DownMmaParams d{};
     d.W_down = W_down; d.R = H; d.D = D;
-    d.idx = p.idx; d.count = p.count;
+    d.idx = lidx; d.count = lcount;
     d.hmT = hmT; d.hm_stride = h->L.hm_stride; d.B = nb;
     d.partial = partial;
     SFFN_CUDA(launch_down_mma(d, splits, s));
@@ -371,10 +404,16 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
     return SFFN_OK;
   }
   const int gate_k = g->kind == SFFN_GATE_LOPA ? g->r : h->D;
-  const int gate_cols = g->kind == SFFN_GATE_LOPA ? 2 * (B < kMaxMmaTokens ? B : kMaxMmaTokens) : B;
-  if (h->dtype == SFFN_BF16 && B >= 2 && B <= kMaxMmaTokens && h->path != SFFN_PATH_GENERAL &&
-      sffn::batched_mma_supported(h->D, gate_k, gate_cols))
-    return run_batched(h, x, B, g, b_g, W_up, W_down, act, y, dense, s);
+  const int gate_cols = g->kind == SFFN_GATE_LOPA ? 2 * B : B;
+  if (h->dtype == SFFN_BF16 && B >= 2 && B <= kMaxMmaTokens && h->path != SFFN_PATH_GENERAL) {
+    const bool mma_ok = sffn::batched_mma_supported(h->D, gate_k, gate_cols);
+    const bool umma_ok = mma_ok && sffn::umma_rows_supported(gate_k, gate_cols) && sffn::umma_rows_supported(h->D, B);
+    if (h->path == SFFN_PATH_MMA_SYNC && !mma_ok) return SFFN_ERR_UNSUPPORTED;
+    if (mma_ok)
+      return run_batched(h, x, B, g, b_g, W_up, W_down, act, y, dense, umma_ok && h->path != SFFN_PATH_MMA_SYNC, s);
+  } else if (h->path == SFFN_PATH_MMA_SYNC) {
+    return SFFN_ERR_UNSUPPORTED;
+  }
   return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, s);
 }
 

@@ -20,8 +20,9 @@ namespace sffn {
 
 namespace {
 
-constexpr int kKC = 256;            // contraction elements staged per step
-constexpr int kXPitch = kKC + 32;   // bf16 elements; 576 bytes = 64 mod 128 -> conflict-free 16-byte reads
+constexpr int kDownStages = 8;      // cp.async stages of the down projection (16 union rows each)
+constexpr int kKC = 128;            // contraction elements staged per step
+constexpr int kXPitch = kKC + 32;   // bf16 elements; 320 bytes = 64 mod 128 -> conflict-free 16-byte reads
 
 __device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
@@ -46,7 +47,7 @@ __device__ __forceinline__ void cp_async_wait() {
 template <int NT, bool UP>
 __global__ void __launch_bounds__(256) rows_mma_kernel(const RowsMmaParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [2][NT*8][kXPitch]
+  __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [3][NT*8][kXPitch]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
   const int K = p.K;
@@ -82,36 +83,51 @@ __global__ void __launch_bounds__(256) rows_mma_kernel(const RowsMmaParams p) {
     };
 
     const int n_steps = (K + kKC - 1) / kKC;
-    __syncthreads();  // previous tile's readers are done with both buffers
-    stage(0, 0);
-    for (int s = 0; s < n_steps; ++s) {
-      const int kc = s * kKC;
+    constexpr int KB = kKC / 32;  // 32-wide blocks per step
+    // Weight fragments are double-buffered in registers (two steps ahead of the tensor cores) and the
+    // token operand is triple-buffered in shared memory, so the loads of steps s+1 and s+2 are in
+    // flight while step s is multiplied.
+    uint4 a0[3][KB], a1[3][KB];
+    auto load_a = [&](int step, int buf) {
+      const int kc = step * kKC;
       const int kblocks = min(kKC, K - kc) / 32;
-      // this step's weight fragments: issue every load before the first use
-      uint4 a0[kKC / 32], a1[kKC / 32];
 #pragma unroll
-      for (int kb = 0; kb < kKC / 32; ++kb) {
+      for (int kb = 0; kb < KB; ++kb) {
         if (kb < kblocks) {
-          a0[kb] = ld_stream16(w0 + (kc / 8) + kb * 4);
-          a1[kb] = ld_stream16(w1 + (kc / 8) + kb * 4);
+          a0[buf][kb] = ld_stream16(w0 + (kc / 8) + kb * 4);
+          a1[buf][kb] = ld_stream16(w1 + (kc / 8) + kb * 4);
         }
       }
-      if (s + 1 < n_steps) stage(kc + kKC, (s + 1) & 1);
-      if (s + 1 < n_steps) cp_async_wait<1>(); else cp_async_wait<0>();
-      __syncthreads();
-      const __nv_bfloat16* xb = xs + (size_t)(s & 1) * ncols * kXPitch;
+    };
+    __syncthreads();  // previous tile's readers are done with the staging buffers
+    stage(0, 0);
+    load_a(0, 0);
+    if (n_steps > 1) { stage(kKC, 1); load_a(1, 1); }
+#pragma unroll 1
+    for (int s3 = 0; s3 < n_steps; s3 += 3) {
 #pragma unroll
-      for (int kb = 0; kb < kKC / 32; ++kb) {
-        if (kb < kblocks) {
+      for (int u = 0; u < 3; ++u) {
+        const int s = s3 + u;
+        if (s < n_steps) {
+          if (s + 2 < n_steps) { stage((s + 2) * kKC, (u + 2) % 3); load_a(s + 2, (u + 2) % 3); }
+          if (s + 2 < n_steps) cp_async_wait<2>(); else if (s + 1 < n_steps) cp_async_wait<1>(); else cp_async_wait<0>();
+          __syncthreads();
+          const int kblocks = min(kKC, K - s * kKC) / 32;
+          const __nv_bfloat16* xb = xs + (size_t)u * ncols * kXPitch;
 #pragma unroll
-          for (int n = 0; n < NT; ++n) {
-            const uint4 b = *reinterpret_cast<const uint4*>(xb + (size_t)(n * 8 + g) * kXPitch + kb * 32 + t * 8);
-            mma_bf16(acc[n], a0[kb].x, a1[kb].x, a0[kb].y, a1[kb].y, b.x, b.y);
-            mma_bf16(acc[n], a0[kb].z, a1[kb].z, a0[kb].w, a1[kb].w, b.z, b.w);
+          for (int kb = 0; kb < KB; ++kb) {
+            if (kb < kblocks) {
+#pragma unroll
+              for (int n = 0; n < NT; ++n) {
+                const uint4 b = *reinterpret_cast<const uint4*>(xb + (size_t)(n * 8 + g) * kXPitch + kb * 32 + t * 8);
+                mma_bf16(acc[n], a0[u][kb].x, a1[u][kb].x, a0[u][kb].y, a1[u][kb].y, b.x, b.y);
+                mma_bf16(acc[n], a0[u][kb].z, a1[u][kb].z, a0[u][kb].w, a1[u][kb].w, b.z, b.w);
+              }
+            }
           }
+          __syncthreads();
         }
       }
-      __syncthreads();
     }
 
     // ---- epilogue: lane (g, t) holds rows i0 (acc[.][0..1]) and i1 (acc[.][2..3]), columns 2t, 2t+1
@@ -192,7 +208,7 @@ __global__ void split_bf16_kernel(const float* n, int B, int r, int n_stride, __
 // HmT; A fragments come from ldmatrix.trans (the staged tile is [u][d], the operand is [d][u]).
 template <int NT>
 __global__ void __launch_bounds__(256) down_mma_kernel(const DownMmaParams p) {
-  constexpr int kStages = 3;
+  constexpr int kStages = kDownStages;
   constexpr int kWPitch = 256 + 8;  // bf16 elements: 528 bytes, odd multiple of 16 -> conflict-free ldmatrix
   constexpr int kHPitch = 16 + 8;   // bf16 elements per token row of the Hm stage (48 bytes)
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -236,17 +252,15 @@ __global__ void __launch_bounds__(256) down_mma_kernel(const DownMmaParams p) {
     cp_async_commit();
   };
 
-  for (int s = s_lo; s < min(s_hi, s_lo + kStages - 1); ++s) stage(s, (s - s_lo) % kStages);
+  // One commit group per step, real or empty, so that "all but the newest kStages-1 groups are
+  // complete" always means "step s has landed".
+  for (int q = 0; q < kStages - 1; ++q) {
+    if (s_lo + q < s_hi) stage(s_lo + q, q); else cp_async_commit();
+  }
   for (int s = s_lo; s < s_hi; ++s) {
     const int buf = (s - s_lo) % kStages;
-    if (s + kStages - 1 < s_hi) {
-      stage(s + kStages - 1, (s - s_lo + kStages - 1) % kStages);
-      cp_async_wait<kStages - 1>();
-    } else if (s + 1 < s_hi) {
-      cp_async_wait<1>();  // conservative near the tail
-    } else {
-      cp_async_wait<0>();
-    }
+    if (s + kStages - 1 < s_hi) stage(s + kStages - 1, (s - s_lo + kStages - 1) % kStages); else cp_async_commit();
+    cp_async_wait<kStages - 1>();
     __syncthreads();
     // B fragments: (k = u: 2t, 2t+1 | 2t+8, 2t+9 ; n = token g of tile n)
     uint32_t bf[NT][2];
@@ -287,7 +301,7 @@ __global__ void __launch_bounds__(256) down_mma_kernel(const DownMmaParams p) {
 
 template <int NT>
 cudaError_t launch_rows_nt(bool up, const RowsMmaParams& p, int grid, cudaStream_t s) {
-  const size_t stage_bytes = (size_t)2 * NT * 8 * kXPitch * sizeof(__nv_bfloat16);
+  const size_t stage_bytes = (size_t)3 * NT * 8 * kXPitch * sizeof(__nv_bfloat16);
   const size_t z_bytes = (size_t)128 * (NT * 8 + 1) * sizeof(float);
   const size_t smem = stage_bytes > z_bytes ? stage_bytes : z_bytes;
   if (up) {
@@ -304,7 +318,7 @@ cudaError_t launch_rows_nt(bool up, const RowsMmaParams& p, int grid, cudaStream
 
 template <int NT>
 cudaError_t launch_down_nt(const DownMmaParams& p, dim3 grid, cudaStream_t s) {
-  const size_t smem = (size_t)3 * (16 * (256 + 8) + NT * 8 * (16 + 8)) * sizeof(__nv_bfloat16);
+  const size_t smem = (size_t)kDownStages * (16 * (256 + 8) + NT * 8 * (16 + 8)) * sizeof(__nv_bfloat16);
   auto k = down_mma_kernel<NT>;
   if (smem > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   k<<<grid, 256, smem, s>>>(p);

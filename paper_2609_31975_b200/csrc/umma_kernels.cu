@@ -1,0 +1,349 @@
+// Batched path on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM), bf16 storage.
+//
+//   umma_rows_kernel<GATE>  Z[H, B] = W[H, K] X[B, K]^T + bias (+ fixed-matrix term), activation, gate values,
+//                           "any token fires" flag per neuron            (Eq. 1 gate / LoPA U stage, batched)
+//   umma_rows_kernel<UP>    over the union list of fired neurons (Sec. 5.4): Up = W_up[idx] X^T, Hm = a . Up,
+//                           stored as bf16 HmT[b][u] for the down projection
+//
+// One CTA owns a tile of 128 weight rows (TMEM lanes) x Npad token columns (Npad = columns rounded up to 16):
+//   warps 0-3  producers: 16-byte cp.async copies gather the 128 (possibly scattered) rows of the current
+//              64-wide K block straight into the 128-byte-swizzled K-major layout the tensor core reads,
+//              several stages ahead of it; a stage is published with fence.proxy.async + mbarrier arrive
+//   warp  8    one thread issues tcgen05.mma (M=128, N=Npad, K=16, four per stage) and commits each stage's
+//              completion to the "slot free" mbarrier; the same warp allocates and frees the TMEM columns
+//   warps 4-7  epilogue: tcgen05.ld the accumulator row of "their" neuron, apply the gate / scale epilogue
+// Every wait is bounded by a cycle budget; on expiry the status word is set, all roles wind down, the
+// producers drain their copies and the TMEM columns are released before the CTA exits.
+#include "umma_kernels.cuh"
+
+#include "common.cuh"
+#include "sparse_ffn.h"
+
+namespace sffn {
+
+namespace {
+
+constexpr int kTileRows = 128;
+constexpr int kKBlock = 64;                          // bf16 elements per stage along K = one 128-byte swizzle row
+constexpr int kATileBytes = kTileRows * 128;         // 16 KB
+constexpr int kProducerThreads = 128;
+constexpr int kThreads = 288;                        // 4 producer warps, 4 epilogue warps, 1 MMA warp
+constexpr int kLag = 4;                              // copy groups a producer thread keeps in flight
+constexpr long long kWaitCycles = 1LL << 31;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) {
+      *abort_flag = 1;
+      atomicExch(status, (int32_t)SFFN_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void cp_async16(uint32_t smem, const void* gmem, bool valid) {
+  const int n = valid ? 16 : 0;  // src-size 0: zero fill
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem), "l"(gmem), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 bytes apart, groups of
+// eight rows 1024 bytes apart (stride byte offset), descriptor version 1 (Blackwell).
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3fff);        // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
+  d |= (uint64_t)1 << 46;                            // version
+  d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t make_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+  uint32_t r[8];
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Byte offset of the 16-byte chunk c (0..7) of row r inside a 128-byte-swizzled K-major tile.
+__device__ __forceinline__ uint32_t swz(int r, int c) {
+  return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4));
+}
+
+template <bool UP>
+__global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsParams p) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  // carve: stages first (1024-byte aligned), then barriers and control words
+  const int npad = p.npad;
+  const int stage_bytes = kATileBytes + npad * 128;
+  const int S = p.stages;
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
+  const uint32_t full = smem_u32(bars), empty = smem_u32(bars + S);
+  const uint32_t acc_full = smem_u32(bars + 2 * S), acc_empty = smem_u32(bars + 2 * S + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int K = p.K;
+  const int n_rows = p.count ? *p.count : p.R;
+  const int n_tiles = (n_rows + kTileRows - 1) / kTileRows;
+  const int kblocks = K / kKBlock;
+  const uint32_t tmem_cols = npad <= 32 ? 32 : npad <= 64 ? 64 : 128;
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full + 8 * s, kProducerThreads);
+      mbar_init(empty + 8 * s, 1);
+    }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 128);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp < 4) {
+    // ======================= producers =========================================================
+    const int pc = tid & 7;    // 16-byte chunk within the 128-byte K block
+    const int pr = tid >> 3;   // first row handled: rows pr, pr+16, ..., pr+112
+    const char* Wb = static_cast<const char*>(p.W);
+    const char* Xb = static_cast<const char*>(p.X);
+    const size_t wpitch = (size_t)K * 2;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+      const char* rowp[8];
+      bool rowok[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int li = tile * kTileRows + pr + 16 * i;
+        rowok[i] = li < n_rows;
+        const int j = rowok[i] ? (p.idx ? p.idx[li] : li) : 0;
+        rowp[i] = Wb + (size_t)j * wpitch + pc * 16;
+      }
+      for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        const int s = it % S;
+        if (!mbar_wait(empty + 8 * s, ((it / S) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+        const uint32_t abase = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t bbase = abase + kATileBytes;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cp_async16(abase + swz(pr + 16 * i, pc), rowp[i] + (size_t)kb * 128, rowok[i]);
+        for (int r = pr; r < npad; r += 16)
+          cp_async16(bbase + swz(r, pc), Xb + ((size_t)(r < p.ncols_valid ? r : 0) * p.x_stride + kb * kKBlock) * 2 + pc * 16,
+                     r < p.ncols_valid);
+        cp_async_commit();
+        if (it >= kLag) {
+          cp_async_wait<kLag>();
+          fence_async_smem();
+          mbar_arrive(full + 8 * ((it - kLag) % S));
+        }
+      }
+    }
+    // drain: publish the stages still in flight
+    cp_async_wait<0>();
+    fence_async_smem();
+    if (ok) {
+      for (int q = (it > kLag ? it - kLag : 0); q < it; ++q) mbar_arrive(full + 8 * (q % S));
+    }
+  } else if (warp == 8) {
+    // ======================= MMA issuer ========================================================
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(npad);
+      int it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++tcount) {
+        if (!mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, p.status)) break;
+        tc_fence_after();
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % S;
+          if (!mbar_wait(full + 8 * s, (it / S) & 1, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t abase = smem_u32(smem + (size_t)s * stage_bytes);
+          const uint64_t adesc = make_desc(abase), bdesc = make_desc(abase + kATileBytes);
+#pragma unroll
+          for (int k = 0; k < kKBlock / 16; ++k)
+            umma(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) ? 1u : 0u);
+          umma_commit(empty + 8 * s);   // slot free once these MMAs have read it
+        }
+        if (ok) umma_commit(acc_full);  // accumulator complete
+      }
+    }
+    __syncwarp();
+  } else {
+    // ======================= epilogue ==========================================================
+    const int ew = warp - 4;                 // TMEM lanes 32*ew .. 32*ew + 31
+    const int row_in_tile = ew * 32 + lane;
+    const int B = p.B;
+    int tcount = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
+      if (!mbar_wait(acc_full, tcount & 1, abort_flag, p.status)) break;
+      __syncwarp();
+      tc_fence_after();
+      const int li = tile * kTileRows + row_in_tile;
+      const bool row_ok = li < n_rows;
+      const int j = row_ok ? (p.idx ? p.idx[li] : li) : 0;
+      const uint32_t taddr = tmem_base + ((uint32_t)(ew * 32) << 16);
+      if (UP) {
+        for (int c0 = 0; c0 < npad; c0 += 8) {
+          float v[8];
+          tmem_ld8(taddr + c0, v);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int b = c0 + q;
+            if (row_ok && b < B)
+              static_cast<__nv_bfloat16*>(p.hmT)[(size_t)b * p.hm_stride + li] =
+                  __float2bfloat16(p.a[(size_t)b * p.a_stride + j] * v[q]);
+          }
+        }
+      } else {
+        const float bias = (row_ok && p.b_g) ? p.b_g[j] : 0.f;
+        const int gi = (row_ok && p.g_idx) ? p.g_idx[j] : -1;
+        const float sg = (row_ok && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
+        bool fired = false;
+        for (int c0 = 0; c0 < npad; c0 += 8) {
+          float v[8];
+          tmem_ld8(taddr + c0, v);
+          const int per = p.split_cols ? 4 : 8;  // tokens covered by these eight columns
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            if (q < per) {
+              const int b = (p.split_cols ? c0 / 2 : c0) + q;
+              if (row_ok && b < B) {
+                float z = p.split_cols ? v[2 * q] + v[2 * q + 1] : v[q];
+                if (gi >= 0)
+                  z += sg * __bfloat162float(static_cast<const __nv_bfloat16*>(p.xtok)[(size_t)b * p.xtok_stride + gi]);
+                z += bias;
+                fired |= z > 0.f;
+                p.a_out[(size_t)b * p.a_stride + j] = activation(p.act, z);
+              }
+            }
+          }
+        }
+        if (row_ok && p.flag) p.flag[j] = fired ? 1 : 0;
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty);
+    }
+  }
+
+  // ---- teardown: everybody meets, then the allocating warp frees the TMEM columns ------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+// n (fp32, [B][r]) -> bf16 pairs: row 2b holds the high parts of token b, row 2b+1 the low parts.
+__global__ void split_interleaved_kernel(const float* n, int r, int n_stride, __nv_bfloat16* x2) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = blockIdx.y;
+  if (k >= r) return;
+  const float v = n[(size_t)b * n_stride + k];
+  const __nv_bfloat16 hi = __float2bfloat16(v);
+  x2[(size_t)(2 * b) * r + k] = hi;
+  x2[(size_t)(2 * b + 1) * r + k] = __float2bfloat16(v - __bfloat162float(hi));
+}
+
+}  // namespace
+
+bool umma_rows_supported(int K, int cols) { return K % kKBlock == 0 && K >= kKBlock && cols >= 1 && cols <= 128; }
+
+cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s) {
+  p.npad = (cols + 15) / 16 * 16;
+  const int stage_bytes = kATileBytes + p.npad * 128;
+  int stages = (220 * 1024 - 1024 - 512) / stage_bytes;
+  if (stages > 10) stages = 10;
+  if (stages < kLag + 2) return cudaErrorInvalidValue;
+  p.stages = stages;
+  const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 64;
+  const int tiles = (p.R + kTileRows - 1) / kTileRows;
+  const int grid = tiles < sm_count ? tiles : sm_count;
+  static bool configured[2] = {false, false};
+  if (up) {
+    auto k = umma_rows_kernel<true>;
+    if (!configured[1]) {
+      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) return e;
+      configured[1] = true;
+    }
+    k<<<grid, kThreads, smem, s>>>(p);
+  } else {
+    auto k = umma_rows_kernel<false>;
+    if (!configured[0]) {
+      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) return e;
+      configured[0] = true;
+    }
+    k<<<grid, kThreads, smem, s>>>(p);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_split_interleaved(const float* n, int B, int r, int n_stride, void* x2, cudaStream_t s) {
+  split_interleaved_kernel<<<dim3((r + 255) / 256, B), 256, 0, s>>>(n, r, n_stride, static_cast<__nv_bfloat16*>(x2));
+  return cudaGetLastError();
+}
+
+}  // namespace sffn

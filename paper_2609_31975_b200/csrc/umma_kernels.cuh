@@ -1,0 +1,39 @@
+// Launchers of the tcgen05 (TMEM accumulator) kernels of the batched path (see umma_kernels.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sffn {
+
+struct UmmaRowsParams {
+  const void* W;         // [*, K] bf16, rows selected by idx (or 0..R-1)
+  int R, K;
+  const int32_t* idx;    // UP: list of rows, or null
+  const int32_t* count;  // UP: device length of the list, or null (= R)
+  const void* X;         // token operand [cols][K] bf16, row stride x_stride (elements)
+  int x_stride;
+  int ncols_valid;
+  int B;                 // tokens
+  int split_cols;        // GATE: 1 = columns 2b, 2b+1 are the high / low bf16 parts of token b's vector
+  const float* b_g;
+  const int32_t* g_idx;
+  const int8_t* g_sign;
+  const void* xtok;      // tokens [B][.] bf16 for the fixed-matrix term
+  int xtok_stride;
+  int act;
+  float* a_out;          // GATE: gate values a_out[b * a_stride + j]
+  uint8_t* flag;         // GATE: [R] any token fires, or null
+  const float* a;        // UP: gate values
+  int a_stride;
+  void* hmT;             // UP: bf16 [B][hm_stride]
+  int hm_stride;
+  int32_t* status;       // device status word
+  int npad, stages;      // filled by the launcher
+};
+
+bool umma_rows_supported(int K, int cols);
+cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s);
+cudaError_t launch_split_interleaved(const float* n, int B, int r, int n_stride, void* x2, cudaStream_t s);
+
+}  // namespace sffn

@@ -1,0 +1,150 @@
+"""Wider measurement matrix behind `bench.py --report`: the sparsity sweep of the decode shape, the LoPA
+gates, batched decode under Zipf firing and the 8192 x 28672 stress shape.  Every row times K back-to-back
+calls with CUDA events on the launching stream, rotating over enough independent weight sets that the
+weights of a call are never L2-resident, and reports microseconds per call, the bytes the call must touch
+(from the measured number of fired rows) and the achieved rate."""
+from __future__ import annotations
+
+import json
+import math
+import statistics
+import sys
+from pathlib import Path
+
+import torch
+
+ROOT = Path(__file__).resolve().parent.parent
+sys.path.insert(0, str(ROOT))
+
+import synthetic_inputs as syn  # noqa: E402
+
+from . import SparseFFN, g_diagonal, touched_bytes, dense_bytes  # noqa: E402
+
+DEV = "cuda:0"
+NOMINAL = 8000.0
+
+
+def _time(calls, stream, reps=3):
+    with torch.cuda.stream(stream):
+        for c in calls[: min(len(calls), 16)]:
+            c()
+        torch.cuda.synchronize()
+        best = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for c in calls:
+                c()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            best.append(e0.elapsed_time(e1) * 1e3 / len(calls))
+    return statistics.median(best), min(best)
+
+
+def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1):
+    """sets: list of weight dicts; gate_of(w) -> gate dict.  Returns one result row."""
+    ffn = SparseFFN(D, H, torch.bfloat16, r_max=r or 0, B_max=B, device=DEV)
+    stream = torch.cuda.Stream(DEV)
+    x = syn.tokens(n_calls * B, D, torch.bfloat16, 99, DEV).view(n_calls, B, D)
+    y = torch.empty((n_calls, B, D), dtype=torch.float32, device=DEV)
+    rows, sparse_calls, dense_calls = [], [], []
+    for t in range(n_calls):
+        w = sets[t % len(sets)]
+        xt = x[t, 0] if B == 1 else x[t]
+        yt = y[t, 0] if B == 1 else y[t]
+        if t < 24:  # fired rows per call (union for B > 1), outside the timed region
+            ffn.sparse_ffn_forward(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt)
+            rows.append(int(ffn.last_active().numel()))
+        sparse_calls.append(ffn.prepared(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt, stream=stream))
+        dense_calls.append(ffn.prepared(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt, dense=True,
+                                        stream=stream))
+    n_rows = statistics.mean(rows)
+    us, us_min = _time(sparse_calls, stream)
+    us_dense, _ = _time(dense_calls[: max(16, n_calls // 4)], stream, reps=2)
+    status = ffn.device_status()
+    nbytes = touched_bytes(D, H, round(n_rows), 2, B, r)
+    row = dict(name=name, D=D, H=H, B=B, r=r, act=act, fired_rows=n_rows, fired_frac=n_rows / H,
+               us_per_call=us, us_min=us_min, tokens_per_s=B * 1e6 / us, touched_mb=nbytes / 1e6,
+               gbs=nbytes / us / 1e3, frac_measured_peak=nbytes / us / 1e3 / peak,
+               frac_nominal=nbytes / us / 1e3 / NOMINAL, dense_us=us_dense,
+               dense_gbs=dense_bytes(D, H, 2, B, r) / us_dense / 1e3, speedup_vs_dense=us_dense / us,
+               device_status=status)
+    del ffn, sparse_calls, dense_calls
+    torch.cuda.empty_cache()
+    return row
+
+
+def run(out_path, quick=False):
+    peak = 6549.1
+    mp = ROOT / "MEASURED_PEAKS.json"
+    if mp.exists():
+        peak = float(json.loads(mp.read_text())["hbm_gbs"])
+    rows = []
+    D, H = 4096, 14336
+    std = lambda w: {"W_g": w["W_g"]}
+    # decode shape: sparsity sweep
+    base = [syn.standard_ffn(D, H, torch.bfloat16, 2, DEV, sparsity=0.9, extra=i) for i in range(4)]
+    for s in ((0.9,) if quick else (0.5, 0.7, 0.8, 0.9, 0.95)):
+        b = syn.gate_bias_for_sparsity(s)
+        sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in base]
+        rows.append(measure(f"decode 4096x14336 s={s}", D, H, 1, sets, std, "relu", peak=peak))
+        print(json.dumps(rows[-1]), flush=True)
+    # batched decode under Zipf firing
+    p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
+    zb = syn.bias_from_firing_profile(p).to(DEV)
+    zsets = [dict(w, b_g=zb) for w in base]
+    for B in ((16,) if quick else (4, 16, 64)):
+        rows.append(measure(f"batched zipf B={B}", D, H, B, zsets, std, "relu", n_calls=100, peak=peak))
+        print(json.dumps(rows[-1]), flush=True)
+    # LoPA gates (up/down weights shared with the standard sets)
+    gi = g_diagonal(H, D, DEV)
+    for r in ((512,) if quick else (256, 512, 1024)):
+        lsets = []
+        for i, w in enumerate(base):
+            lw = syn.lopa_ffn(D, H, r, torch.bfloat16, 3, DEV, sparsity=0.9, extra=i)
+            lw["W_up"], lw["W_down"] = w["W_up"], w["W_down"]
+            lsets.append(lw)
+        lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}
+        for act in ("relu", "sqrelu"):
+            rows.append(measure(f"lopa r={r} {act}", D, H, 1, lsets, lg, act, r=r, peak=peak))
+            print(json.dumps(rows[-1]), flush=True)
+        del lsets
+    del base, zsets
+    torch.cuda.empty_cache()
+    if not quick:
+        # stress shape: 8 independent layers per step
+        D, H = 8192, 28672
+        layers = [syn.standard_ffn(D, H, torch.bfloat16, 5, DEV, sparsity=0.9, extra=i) for i in range(8)]
+        for s in (0.8, 0.9, 0.95):
+            b = syn.gate_bias_for_sparsity(s)
+            sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in layers]
+            for B in (1, 8):
+                rows.append(measure(f"stress 8192x28672 s={s} B={B}", D, H, B, sets, std, "sqrelu", n_calls=64,
+                                    peak=peak))
+                print(json.dumps(rows[-1]), flush=True)
+        gi = g_diagonal(H, D, DEV)
+        lsets = []
+        for i, w in enumerate(layers):
+            lw = {k: syn.normal_tensor(shape, std_, torch.bfloat16, 5, k, DEV, i)
+                  for k, shape, std_ in (("V", (1024, D), 1 / math.sqrt(D)), ("U", (H, 1024), 1 / 32.0))}
+            lw["W_up"], lw["W_down"] = w["W_up"], w["W_down"]
+            lsets.append(lw)
+        lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}
+        for s in (0.8, 0.9, 0.95):
+            b = syn.gate_bias_for_sparsity(s, math.sqrt(2.0))
+            sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in lsets]
+            for B in (1, 8):
+                rows.append(measure(f"stress lopa r=1024 s={s} B={B}", D, H, B, sets, lg, "sqrelu", r=1024,
+                                    n_calls=64, peak=peak))
+                print(json.dumps(rows[-1]), flush=True)
+    Path(out_path).parent.mkdir(parents=True, exist_ok=True)
+    Path(out_path).write_text(json.dumps(rows, indent=1))
+    md = ["| case | B | fired rows | us/call | touched MB | GB/s | % of measured peak | % of 8 TB/s | dense us | speedup |",
+          "|---|---|---|---|---|---|---|---|---|---|"]
+    for r_ in rows:
+        md.append(f"| {r_['name']} | {r_['B']} | {r_['fired_rows']:.0f} ({100 * r_['fired_frac']:.1f} %) | "
+                  f"{r_['us_per_call']:.1f} | {r_['touched_mb']:.1f} | {r_['gbs']:.0f} | "
+                  f"{100 * r_['frac_measured_peak']:.1f} | {100 * r_['frac_nominal']:.1f} | {r_['dense_us']:.1f} | "
+                  f"{r_['speedup_vs_dense']:.2f}x |")
+    Path(out_path).with_suffix(".md").write_text("\n".join(md) + "\n")
+    return rows

@@ -98,7 +98,7 @@ def test_lopa_gate_small_shapes(mod, r, fixed, sign, gain, rms, dtype):
 
 
 # ------------------------------------------------------------------ batches: union of active sets
-@pytest.mark.parametrize("path", ["general", "auto"])     # auto = tensor-core kernels for bf16 batches
+@pytest.mark.parametrize("path", ["general", "mma_sync", "auto"])   # auto = tcgen05 kernels for bf16 batches
 @pytest.mark.parametrize("B", [2, 3, 4, 7, 16, 33, 64])
 def test_batched_union(mod, B, path):
     D, H = 512, 1200
@@ -123,7 +123,7 @@ def test_batched_union(mod, B, path):
         assert_y_close(y1, ref["y"][b], what=f"B={B} token {b} alone")
 
 
-@pytest.mark.parametrize("path", ["general", "auto"])
+@pytest.mark.parametrize("path", ["general", "mma_sync", "auto"])
 @pytest.mark.parametrize("B,r,rms", [(5, 128, True), (16, 64, True), (24, 96, False)])
 def test_batched_lopa(mod, B, r, rms, path):
     D, H = 512, 1100
