@@ -64,7 +64,10 @@ struct FusedParams {
   const float* gain;
   int use_rmsnorm;
   float eps;
-  const float* vbuf;  // [r] V x from the first kernel (LoPA)
+  const void* V;      // LoPA: [r, D]
+  float* vbuf;        // LoPA: [r] exchange buffer for v = V x
+  unsigned long long* v_counter;   // LoPA: CTAs that have published their rows of v (monotonic over calls)
+  unsigned long long v_target;     // LoPA: value of the counter once all CTAs of this call have published
   int act, dense;
   float* partial;  // [grid][D]
   uint8_t* flag;
@@ -92,7 +95,7 @@ struct SmemLayout {
     sn = take(lopa ? K * 4 : 0);
     aval = take(slab_max * 4);
     slot_a = take(n_act_slots * 4);
-    red = take(2 * (kActWarps + 1) * 4);
+    red = take(2 * (2 * kActWarps + 1) * 4);
     ctl = take(8 * 4);
     bars = take(2 * (n_gate_slots + n_act_slots) * 8);
     row_done = take(slab_max);
@@ -215,7 +218,7 @@ __device__ __forceinline__ long long global_ns() {
   } while (0)
 
 template <typename T, int CPT, bool LOPA>
-__global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParams p) {
+__global__ void __maxnreg__(96) fused_ffn_kernel(const FusedParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const long long t_entry = clock64();
   pdl_launch_dependents();
@@ -233,11 +236,14 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   unsigned char* act_ring = smem + L.act_ring;
   float* sx = reinterpret_cast<float*>(smem + L.sx);
   float* sn = reinterpret_cast<float*>(smem + L.sn);
-  float* aval = reinterpret_cast<float*>(smem + L.aval);
+  // One word per neuron of the slab, written once by a gate warp and polled by the act producers:
+  // all ones = gate not computed yet, 0x80000000 = not fired, otherwise the bits of a_j >= 0 (fired).
+  // A single 32-bit store publishes value and state together, so no fence is needed on either side
+  // (a fence in the producers would also wait for their bulk copies in flight).
+  volatile uint32_t* row_state = reinterpret_cast<volatile uint32_t*>(smem + L.aval);
   float* slot_a = reinterpret_cast<float*>(smem + L.slot_a);  // per act slot: gate value, < 0 = stop
   float* red = reinterpret_cast<float*>(smem + L.red);
   volatile int* ctl = reinterpret_cast<volatile int*>(smem + L.ctl);
-  volatile uint8_t* row_done = smem + L.row_done;
   const uint32_t bars = smem_u32(smem + L.bars);
   const uint32_t full_gate = bars, empty_gate = bars + 8 * NG;
   const uint32_t full_act = bars + 16 * NG, empty_act = bars + 16 * NG + 8 * NA;
@@ -262,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         mbar_init(empty_act + 8 * s, kActWarps);
       }
       for (int i = 0; i < 8; ++i) ctl[i] = 0;
-      for (int i = 0; i < 2 * (kActWarps + 1); ++i) red[i] = 0.f;
+      for (int i = 0; i < 2 * (2 * kActWarps + 1); ++i) red[i] = 0.f;
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -286,10 +292,29 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     return;
   }
 
+  // Gate warps fetch the per-neuron parameters (bias, fixed-matrix index and sign) of their first two
+  // ring slots now: like the weights they do not depend on the predecessor in the stream.
+  float pre_bias[2] = {0.f, 0.f}, pre_sg[2] = {1.f, 1.f};
+  int pre_gi[2] = {-1, -1};
+  if (warp >= kFirstGateWarp && warp < kFirstActWarp && warp - kFirstGateWarp < p.gate_warps) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int r0 = (warp - kFirstGateWarp + q * p.gate_warps) * nr;
+      if (r0 + lane < slab_rows && lane < nr) {
+        const int j = slab_lo + r0 + lane;
+        if (p.b_g) pre_bias[q] = p.b_g[j];
+        if (LOPA && p.g_idx) {
+          pre_gi[q] = p.g_idx[j];
+          pre_sg[q] = (p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
+        }
+      }
+    }
+  }
+
   // ---- everyone else: wait for the predecessor in the stream, then stage the token ------------
   pdl_wait();
   if (tid == kStageBase) SFFN_GSTAMP(11);
-  for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) row_done[i] = 0;
+  for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) row_state[i] = 0xffffffffu;
   for (int c = tid - kStageBase; c < nvecD; c += kStageThreads) {
     float f[EPV];
     Elem<T>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + c), f);
@@ -297,8 +322,42 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     if (EPV == 8) reinterpret_cast<float4*>(sx)[nvecD + c] = make_float4(f[4], f[5], f[6], f[7]);
   }
   if (LOPA) {
-    // n = RMSNorm(V x) (or V x) into shared memory; every warp derives the same scale
+    // Rank-r stage of the LoPA gate, v = V x, spread over the grid: this CTA computes its share of
+    // the rows of V (one warp per row, straight from global memory), publishes them, and waits until
+    // every CTA has done so.  All CTAs of the call become resident without waiting for this one
+    // (one CTA per SM, predecessors in the stream never wait on their successors), so the bounded
+    // wait below ends as soon as the slowest CTA has started and published.
     const int r = K;
+    named_bar_sync(5, kStageThreads);  // the token is staged
+    const int vlo = (int)((long long)r * cta / G), vhi = (int)((long long)r * (cta + 1) / G);
+    for (int k = vlo + (warp - kGateProducers); k < vhi; k += kStageThreads / 32) {
+      const uint4* vr = reinterpret_cast<const uint4*>(static_cast<const char*>(p.V) + (size_t)k * row_bytes);
+      float a0 = 0.f, a1 = 0.f;
+      int c = lane;
+      for (; c + 32 < nvecD; c += 64) {
+        const uint4 w0 = ld_stream16(vr + c), w1 = ld_stream16(vr + c + 32);
+        a0 = chunk_dot<T>(w0, sx, c, nvecD, a0);
+        a1 = chunk_dot<T>(w1, sx, c + 32, nvecD, a1);
+      }
+      if (c < nvecD) a0 = chunk_dot<T>(ld_stream16(vr + c), sx, c, nvecD, a0);
+      const float v = warp_sum(a0 + a1);
+      if (lane == 0) __stcg(p.vbuf + k, v);
+    }
+    __threadfence();
+    named_bar_sync(5, kStageThreads);
+    if (tid == kStageBase) {
+      atomicAdd(p.v_counter, 1ULL);
+      const long long t0 = clock64();
+      for (;;) {
+        unsigned long long seen;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.v_counter) : "memory");
+        if (seen >= p.v_target || ctl[kAbort]) break;
+        if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); break; }
+        __nanosleep(40);
+      }
+    }
+    named_bar_sync(5, kStageThreads);
+    // n = RMSNorm(v) (or v) into shared memory; every warp derives the same scale
     float ss = 0.f;
     for (int k = lane; k < r; k += 32) {
       const float v = __ldcg(p.vbuf + k);
@@ -319,44 +378,56 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // Both walk the published gate results in the same order; producer 0 copies the W_up row of a
     // fired neuron, producer 1 its W_down row, into the same ring slot.
     const int ap = warp - kFirstActProducer;
-    if (lane == 0) {
-      const char* Wsrc = static_cast<const char*>(ap == 0 ? p.W_up : p.W_down);
-      const uint32_t ring = smem_u32(act_ring) + (ap == 0 ? 0u : (uint32_t)row_bytes);
-      int slot = 0;
-      uint32_t par = 1;
-      bool ok = true;
-      for (int scan = 0; ok && scan <= slab_rows; ++scan) {
-        float a = -1.f;  // the entry after the last row is the stop marker
-        if (scan < slab_rows) {
-          uint8_t code = row_done[scan];
-          if (code == 0) {
-            const long long t0 = clock64();
-            while ((code = row_done[scan]) == 0) {
-              __nanosleep(20);
-              if (ctl[kAbort]) { ok = false; break; }
-              if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); ok = false; break; }
-            }
-            if (!ok) break;
+    const char* Wsrc = static_cast<const char*>(ap == 0 ? p.W_up : p.W_down);
+    const uint32_t ring = smem_u32(act_ring) + (ap == 0 ? 0u : (uint32_t)row_bytes);
+    int slot = 0;
+    uint32_t par = 1;
+    bool ok = true;
+    // The whole warp classifies 32 rows per step (one shared-memory read + ballots); lane 0 issues
+    // the copies of the fired ones in ascending order.  Only the leading run of finished rows is
+    // consumed, so the order never depends on which gate warp was faster.
+    long long t_idle = 0;
+    for (int base = 0; ok && base < slab_rows;) {
+      const int row = base + lane;
+      const uint32_t st = row < slab_rows ? row_state[row] : 0x80000000u;
+      const unsigned done = __ballot_sync(0xffffffffu, st != 0xffffffffu);
+      const int prefix = done == 0xffffffffu ? 32 : __ffs(~done) - 1;
+      if (prefix == 0) {  // the next row's gate is not computed yet
+        if (t_idle == 0) t_idle = clock64();
+        __nanosleep(20);
+        if (ctl[kAbort]) ok = false;
+        else if (clock64() - t_idle > kWaitCycles) { if (lane == 0) raise_timeout(ctl, p.status); ok = false; }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        continue;
+      }
+      t_idle = 0;
+      const bool take = row < slab_rows && lane < prefix && (p.dense || st != 0x80000000u);
+      unsigned fired = __ballot_sync(0xffffffffu, take);
+      while (fired && ok) {
+        const int l = __ffs(fired) - 1;
+        fired &= fired - 1;
+        const uint32_t sl = __shfl_sync(0xffffffffu, st, l);
+        if (lane == 0) {
+          if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) {
+            if (ap == 0) slot_a[slot] = sl == 0x80000000u ? 0.f : __uint_as_float(sl);
+            const size_t j = (size_t)(slab_lo + base + l);
+            mbar_expect_tx(full_act + 8 * slot, (uint32_t)row_bytes);
+            bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
+                     full_act + 8 * slot);
+          } else {
+            ok = false;
           }
-          if (code != 2 && !p.dense) continue;
-          __threadfence_block();
-          a = reinterpret_cast<volatile float*>(aval)[scan];
-          a = a < 0.f ? 0.f : a;  // activations are non-negative; the sign is the stop marker
         }
-        if (!mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) break;
-        if (ap == 0) slot_a[slot] = a;
-        if (scan < slab_rows) {
-          const size_t j = (size_t)(slab_lo + scan);
-          mbar_expect_tx(full_act + 8 * slot, (uint32_t)row_bytes);
-          bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
-                   full_act + 8 * slot);
-        } else {
-          mbar_arrive(full_act + 8 * slot);  // stop marker: completes the phase without data
-        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (++slot == NA) { slot = 0; par ^= 1; }
       }
-      if (ap == 0) SFFN_STAMP(2);
+      base += prefix;
     }
+    if (lane == 0 && ok && mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) {
+      if (ap == 0) slot_a[slot] = -1.f;      // stop marker: a negative gate value
+      mbar_arrive(full_act + 8 * slot);      // completes the phase without data
+    }
+    if (lane == 0 && ap == 0) SFFN_STAMP(2);
     __syncwarp();
   } else if (warp < kFirstActWarp) {
     // ======================= gate warps ========================================================
@@ -368,11 +439,17 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       float add = 0.f;  // bias + fixed-matrix term of the row this lane reports
       if (lane < rows) {
         const int j = slab_lo + r0 + lane;
-        if (p.b_g) add = p.b_g[j];
-        if (LOPA && p.g_idx) {
-          const float sg = (p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
-          add += sg * sx[vec_pos<EPV>(p.g_idx[j], D)];
+        float bias, sg;
+        int gi;
+        if (s == gw) { bias = pre_bias[0]; gi = pre_gi[0]; sg = pre_sg[0]; }
+        else if (s == gw + p.gate_warps) { bias = pre_bias[1]; gi = pre_gi[1]; sg = pre_sg[1]; }
+        else {
+          bias = p.b_g ? p.b_g[j] : 0.f;
+          gi = (LOPA && p.g_idx) ? p.g_idx[j] : -1;
+          sg = (LOPA && p.g_idx && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
         }
+        add = bias;
+        if (LOPA && gi >= 0) add += sg * sx[vec_pos<EPV>(gi, D)];
       }
       if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status)) break;
       const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
@@ -395,10 +472,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       if (lane < rows) {
         const float z = mine + add;
         const bool fired = z > 0.f;
-        aval[r0 + lane] = activation(p.act, z);
         if (!p.dense) p.flag[slab_lo + r0 + lane] = fired ? 1 : 0;
-        __threadfence_block();
-        row_done[r0 + lane] = fired ? 2 : 1;
+        row_state[r0 + lane] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_gate + 8 * slot);
@@ -414,45 +489,74 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
 #pragma unroll
       for (int e = 0; e < EPV; ++e) acc[i][e] = 0.f;
 
+    // Two ring slots per round when the second one exists: both rows are dotted before the one
+    // four-warp barrier, which halves the serial latency per fired row.  The stop marker always
+    // arrives, so waiting for the second slot of a round cannot block for good.  A thread whose
+    // wait ran out still joins the barrier and raises the group's stop flag, so the four warps
+    // always leave the loop together.
     int slot = 0;
     uint32_t par = 0;
-    for (int k = 0;; ++k) {
-      // Every thread waits for itself; a thread whose wait ran out still joins the barrier below
-      // and raises the group's stop flag, so the four warps always leave the loop together.
-      const bool got = mbar_wait(full_act + 8 * slot, par, ctl, p.status);
-      float* rp = red + (k & 1) * (kActWarps + 1);
-      const float a = got ? slot_a[slot] : -1.f;
-      float part = 0.f;
-      const uint4* wu = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes);
-      const uint4* wd = reinterpret_cast<const uint4*>(act_ring + (size_t)slot * p.act_slot_bytes + row_bytes);
-      if (a >= 0.f) {
+    for (int round = 0;; ++round) {
+      float* rp = red + (round & 1) * (2 * kActWarps + 1);
+      const int slot1 = slot + 1 == NA ? 0 : slot + 1;
+      const uint32_t par1 = slot + 1 == NA ? par ^ 1 : par;
+      const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status);
+      const float a0 = got0 ? slot_a[slot] : -1.f;
+      bool got1 = true;
+      float a1 = -1.f;
+      if (a0 >= 0.f) {
+        got1 = mbar_wait(full_act + 8 * slot1, par1, ctl, p.status);
+        a1 = got1 ? slot_a[slot1] : -1.f;
+      }
+      const unsigned char* s0 = act_ring + (size_t)slot * p.act_slot_bytes;
+      const unsigned char* s1 = act_ring + (size_t)slot1 * p.act_slot_bytes;
+      float part0 = 0.f, part1 = 0.f;
+      if (a0 >= 0.f) {
+        const uint4* wu0 = reinterpret_cast<const uint4*>(s0);
+        const uint4* wu1 = reinterpret_cast<const uint4*>(s1);
 #pragma unroll
         for (int i = 0; i < CPT; ++i) {
           const int c = at + i * kActThreads;
-          if (c < nvecD) part = chunk_dot<T>(wu[c], sx, c, nvecD, part);
+          if (c < nvecD) {
+            part0 = chunk_dot<T>(wu0[c], sx, c, nvecD, part0);
+            if (a1 >= 0.f) part1 = chunk_dot<T>(wu1[c], sx, c, nvecD, part1);
+          }
         }
-        part = warp_sum(part);
-        if (lane == 0) rp[aw] = part;
-      } else {
-        rp[kActWarps] = 1.f;  // stop marker or failed wait
+        part0 = warp_sum(part0);
+        part1 = warp_sum(part1);
+        if (lane == 0) {
+          rp[aw] = part0;
+          rp[kActWarps + aw] = part1;
+        }
       }
+      if (a0 < 0.f || !got1) rp[2 * kActWarps] = 1.f;  // stop marker first in the round, or a failed wait
       named_bar_sync(2, kActThreads);
-      if (rp[kActWarps] != 0.f) break;
-      const float u = (rp[0] + rp[1]) + (rp[2] + rp[3]);
-      const float h = a * u;
+      if (rp[2 * kActWarps] != 0.f) break;
+      const float h0 = a0 * ((rp[0] + rp[1]) + (rp[2] + rp[3]));
+      const float h1 = a1 * ((rp[kActWarps] + rp[kActWarps + 1]) + (rp[kActWarps + 2] + rp[kActWarps + 3]));
+      const uint4* wd0 = reinterpret_cast<const uint4*>(s0 + row_bytes);
+      const uint4* wd1 = reinterpret_cast<const uint4*>(s1 + row_bytes);
 #pragma unroll
       for (int i = 0; i < CPT; ++i) {
         const int c = at + i * kActThreads;
         if (c < nvecD) {
           float f[EPV];
-          Elem<T>::unpack(wd[c], f);
+          Elem<T>::unpack(wd0[c], f);
 #pragma unroll
-          for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h, f[e], acc[i][e]);
+          for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h0, f[e], acc[i][e]);
+          if (a1 >= 0.f) {
+            Elem<T>::unpack(wd1[c], f);
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h1, f[e], acc[i][e]);
+          }
         }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_act + 8 * slot);
-      if (++slot == NA) { slot = 0; par ^= 1; }
+      if (a1 < 0.f) break;  // the second slot was the stop marker
+      if (lane == 0) mbar_arrive(empty_act + 8 * slot1);
+      slot = slot1 + 1 == NA ? 0 : slot1 + 1;
+      par = slot1 + 1 == NA ? par1 ^ 1 : par1;
     }
     if (at == 0) SFFN_STAMP(4);
     // this CTA's partial of y
@@ -472,7 +576,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   }
 }
 
-// y[d] = sum over CTAs of partial[cta][d] in a fixed order.  One warp per float4 column: lane l adds
+// y[d] = sum over CTAs of partial[cta][d] in a fixed order.  Its CTAs (256 threads, ~40 registers) fit on
+// an SM next to a CTA of the main kernel (which is capped at 96 registers per thread for that reason), so
+// they are resident, parked in griddepcontrol.wait, before the main kernel ends.  One warp per float4 column: lane l adds
 // the partials l, l+32, ... (every load issued before the first add: one L2 round trip), then a fixed
 // shuffle tree combines the lanes.
 __global__ void __launch_bounds__(256) fused_reduce_kernel(const float* partial, int G, int D, float* y,
@@ -507,37 +613,6 @@ __global__ void __launch_bounds__(256) fused_reduce_kernel(const float* partial,
     if (l == 0 && *status == 0) reinterpret_cast<float4*>(y)[q] = s;
   }
   if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)(G + 2) * 16 + blockIdx.x] = global_ns();
-}
-
-// LoPA rank-r stage: v = V x, one warp per row of V.
-template <typename T>
-__global__ void __launch_bounds__(256) lopa_v_kernel(const void* V, const void* x, int r, int D, float* v) {
-  extern __shared__ __align__(16) float sxv[];
-  constexpr int EPV = Elem<T>::kPerVec;
-  pdl_launch_dependents();
-  pdl_wait();
-  const int nvecD = D / EPV;
-  for (int c = threadIdx.x; c < nvecD; c += blockDim.x) {
-    float f[EPV];
-    Elem<T>::unpack(__ldg(reinterpret_cast<const uint4*>(x) + c), f);
-    reinterpret_cast<float4*>(sxv)[c] = make_float4(f[0], f[1], f[2], f[3]);
-    if (EPV == 8) reinterpret_cast<float4*>(sxv)[nvecD + c] = make_float4(f[4], f[5], f[6], f[7]);
-  }
-  __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int k = blockIdx.x * 8 + warp; k < r; k += gridDim.x * 8) {
-    const uint4* vr = reinterpret_cast<const uint4*>(static_cast<const char*>(V) + (size_t)k * D * sizeof(T));
-    float a0 = 0.f, a1 = 0.f;
-    int c = lane;
-    for (; c + 32 < nvecD; c += 64) {
-      const uint4 w0 = ld_stream16(vr + c), w1 = ld_stream16(vr + c + 32);
-      a0 = chunk_dot<T>(w0, sxv, c, nvecD, a0);
-      a1 = chunk_dot<T>(w1, sxv, c + 32, nvecD, a1);
-    }
-    if (c < nvecD) a0 = chunk_dot<T>(ld_stream16(vr + c), sxv, c, nvecD, a0);
-    const float s = warp_sum(a0 + a1);
-    if (lane == 0) v[k] = s;
-  }
 }
 
 // ---- host side --------------------------------------------------------------------------------
@@ -632,21 +707,6 @@ cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaS
   return launch_pdl(k, dim3(grid), dim3(kThreads), (size_t)g.smem, s, p);
 }
 
-template <typename T>
-cudaError_t launch_v(const FusedCall& c, float* vbuf, cudaStream_t s) {
-  const int r = c.gate->r;
-  const size_t smem = (size_t)c.D * 4;
-  auto k = lopa_v_kernel<T>;
-  static bool configured = false;
-  if (!configured && smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  const int grid = (r + 7) / 8;
-  return launch_pdl(k, dim3(grid), dim3(256), smem, s, c.gate->V, c.x, r, c.D, vbuf);
-}
-
 }  // namespace
 
 void debug_set_pdl(int on) { g_debug_pdl = on; }
@@ -661,7 +721,6 @@ bool fused_supported(bool bf16, int D, int H, int B, const sffn_gate* gate, int 
   if (B != 1) return false;
   const bool lopa = gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? gate->r : D;
-  if (lopa && (size_t)D * 4 > 128 * 1024) return false;
   return plan(bf16, D, H, K, lopa, fused_grid(sm_count, H)).ok;
 }
 
@@ -676,18 +735,17 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   float* vbuf = reinterpret_cast<float*>(ws + 256 + (size_t)kMaxGrid * c.D * 4);
   int n = 0;
   cudaError_t e;
-  if (lopa) {
-    e = c.bf16 ? launch_v<__nv_bfloat16>(c, vbuf, s) : launch_v<float>(c, vbuf, s);
-    if (e != cudaSuccess) return e;
-    ++n;
-  }
   FusedParams p{};
   p.D = c.D; p.H = c.H; p.K = K;
   p.Wgate = lopa ? c.gate->U : c.gate->W_g;
   p.W_up = c.W_up; p.W_down = c.W_down; p.x = c.x; p.b_g = c.b_g;
   p.g_idx = lopa ? c.gate->g_idx : nullptr; p.g_sign = c.gate->g_sign;
   p.gain = c.gate->rms_gain; p.use_rmsnorm = c.gate->use_rmsnorm; p.eps = c.gate->rms_eps;
+  p.V = c.gate->V;
   p.vbuf = vbuf;
+  p.v_counter = reinterpret_cast<unsigned long long*>(ws);
+  if (lopa) *c.lopa_calls += 1;
+  p.v_target = *c.lopa_calls * (unsigned long long)grid;
   p.partial = partial;
   p.act = c.act; p.dense = c.dense ? 1 : 0;
   p.flag = c.flag; p.status = c.status;
