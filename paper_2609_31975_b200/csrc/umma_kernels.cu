@@ -24,11 +24,11 @@ namespace sffn {
 namespace {
 
 constexpr int kTileRows = 128;
-constexpr int kKBlock = 64;                          // bf16 elements per stage along K = one 128-byte swizzle row
-constexpr int kATileBytes = kTileRows * 128;         // 16 KB
-constexpr int kProducerThreads = 128;
+constexpr int kAtomK = 64;                           // bf16 elements of one 128-byte swizzle row
+constexpr int kAAtomBytes = kTileRows * 128;         // 16 KB: one [128 rows x 64 k] swizzled block
+// A stage holds `atoms` (1, 2 or 4) such blocks side by side along K, i.e. 128 to 512 contiguous bytes of
+// every row.
 constexpr int kThreads = 288;                        // 4 producer warps, 4 epilogue warps, 1 MMA warp
-constexpr int kLag = 4;                              // copy groups a producer thread keeps in flight
 constexpr long long kWaitCycles = 1LL << 31;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -125,7 +125,11 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   // carve: stages first (1024-byte aligned), then barriers and control words
   const int npad = p.npad;
-  const int stage_bytes = kATileBytes + npad * 128;
+  const int kAtoms = p.atoms;
+  const int kKBlock = kAtomK * kAtoms;
+  const int kATileBytes = kAAtomBytes * kAtoms;
+  const int b_atom_bytes = npad * 128;
+  const int stage_bytes = kATileBytes + b_atom_bytes * kAtoms;
   const int S = p.stages;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
@@ -133,17 +137,18 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
   const uint32_t acc_full = smem_u32(bars + 2 * S), acc_empty = smem_u32(bars + 2 * S + 1);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const char** rowptr = reinterpret_cast<const char**>(tmem_slot + 2);  // [4][128] row pointers of the current tile, per producer warp
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int K = p.K;
   const int n_rows = p.count ? *p.count : p.R;
   const int n_tiles = (n_rows + kTileRows - 1) / kTileRows;
-  const int kblocks = K / kKBlock;
+  const int kblocks = (K + kKBlock - 1) / kKBlock;   // the last one may hold fewer atoms
   const uint32_t tmem_cols = npad <= 32 ? 32 : npad <= 64 ? 64 : 128;
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
-      mbar_init(full + 8 * s, kProducerThreads);
+      mbar_init(full + 8 * s, 32);  // the 32 lanes of the producer warp that owns the stage
       mbar_init(empty + 8 * s, 1);
     }
     mbar_init(acc_full, 1);
@@ -164,47 +169,56 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
 
   if (warp < 4) {
     // ======================= producers =========================================================
-    const int pc = tid & 7;    // 16-byte chunk within the 128-byte K block
-    const int pr = tid >> 3;   // first row handled: rows pr, pr+16, ..., pr+112
+    // Each producer warp owns every fourth stage, so four stages are being filled independently and
+    // the wait -> copy -> publish latency of one does not hold up the others.  Lane l copies chunk
+    // l & 7 of rows (l >> 3) + 4 i; its swizzled offset advances by 512 bytes per step because the
+    // row index modulo 8 does not change.
+    const int pc = lane & 7, pq = lane >> 3;
     const char* Wb = static_cast<const char*>(p.W);
     const char* Xb = static_cast<const char*>(p.X);
     const size_t wpitch = (size_t)K * 2;
-    int it = 0;
     bool ok = true;
+    int it = 0;         // global stage counter (all producer warps count the same way)
+    int pending = -1;   // stage copied by this warp but not yet published
     for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-      const char* rowp[8];
-      bool rowok[8];
+      // this warp's own copy of the tile's row pointers (null = beyond the list): no cross-warp barrier
+      const char** myrows = rowptr + warp * kTileRows;
+      __syncwarp();
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int li = tile * kTileRows + pr + 16 * i;
-        rowok[i] = li < n_rows;
-        const int j = rowok[i] ? (p.idx ? p.idx[li] : li) : 0;
-        rowp[i] = Wb + (size_t)j * wpitch + pc * 16;
+      for (int q = 0; q < 4; ++q) {
+        const int li = tile * kTileRows + lane + 32 * q;
+        myrows[lane + 32 * q] = li < n_rows ? Wb + (size_t)(p.idx ? p.idx[li] : li) * wpitch : nullptr;
       }
+      __syncwarp();
       for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        if ((it & 3) != warp) continue;
         const int s = it % S;
         if (!mbar_wait(empty + 8 * s, ((it / S) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
         const uint32_t abase = smem_u32(smem + (size_t)s * stage_bytes);
         const uint32_t bbase = abase + kATileBytes;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) cp_async16(abase + swz(pr + 16 * i, pc), rowp[i] + (size_t)kb * 128, rowok[i]);
-        for (int r = pr; r < npad; r += 16)
-          cp_async16(bbase + swz(r, pc), Xb + ((size_t)(r < p.ncols_valid ? r : 0) * p.x_stride + kb * kKBlock) * 2 + pc * 16,
-                     r < p.ncols_valid);
-        cp_async_commit();
-        if (it >= kLag) {
-          cp_async_wait<kLag>();
-          fence_async_smem();
-          mbar_arrive(full + 8 * ((it - kLag) % S));
+        const size_t koff = (size_t)kb * 128 + pc * 16;
+#pragma unroll 8
+        for (int i = 0; i < 32; ++i) {
+          const int r = pq + 4 * i;
+          const char* rp = myrows[r];
+          cp_async16(abase + swz(r, pc), (rp ? rp : Wb) + koff, rp != nullptr);
         }
+        for (int r = pq; r < npad; r += 4) {
+          const bool v = r < p.ncols_valid;
+          cp_async16(bbase + swz(r, pc), Xb + (size_t)(v ? r : 0) * p.x_stride * 2 + koff, v);
+        }
+        cp_async_commit();
+        if (pending >= 0) {          // publish the previous stage of this warp: its copies are older
+          cp_async_wait<1>();
+          fence_async_smem();
+          mbar_arrive(full + 8 * (pending % S));
+        }
+        pending = it;
       }
     }
-    // drain: publish the stages still in flight
     cp_async_wait<0>();
     fence_async_smem();
-    if (ok) {
-      for (int q = (it > kLag ? it - kLag : 0); q < it; ++q) mbar_arrive(full + 8 * (q % S));
-    }
+    if (ok && pending >= 0) mbar_arrive(full + 8 * (pending % S));
   } else if (warp == 8) {
     // ======================= MMA issuer ========================================================
     if (lane == 0) {
@@ -218,11 +232,15 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
           const int s = it % S;
           if (!mbar_wait(full + 8 * s, (it / S) & 1, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t abase = smem_u32(smem + (size_t)s * stage_bytes);
-          const uint64_t adesc = make_desc(abase), bdesc = make_desc(abase + kATileBytes);
+          const uint32_t sbase = smem_u32(smem + (size_t)s * stage_bytes);
+          const int atoms = min(kAtoms, (K - kb * kKBlock) / kAtomK);
+          for (int a = 0; a < atoms; ++a) {
+            const uint64_t adesc = make_desc(sbase + a * kAAtomBytes);
+            const uint64_t bdesc = make_desc(sbase + kATileBytes + a * b_atom_bytes);
 #pragma unroll
-          for (int k = 0; k < kKBlock / 16; ++k)
-            umma(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) ? 1u : 0u);
+            for (int k = 0; k < kAtomK / 16; ++k)
+              umma(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | a | k) ? 1u : 0u);
+          }
           umma_commit(empty + 8 * s);   // slot free once these MMAs have read it
         }
         if (ok) umma_commit(acc_full);  // accumulator complete
@@ -306,18 +324,24 @@ __global__ void split_interleaved_kernel(const float* n, int r, int n_stride, __
   x2[(size_t)(2 * b + 1) * r + k] = __float2bfloat16(v - __bfloat162float(hi));
 }
 
+int g_umma_atoms = 0;
+
 }  // namespace
 
-bool umma_rows_supported(int K, int cols) { return K % kKBlock == 0 && K >= kKBlock && cols >= 1 && cols <= 128; }
+void debug_set_umma_atoms(int atoms) { g_umma_atoms = atoms; }
+
+bool umma_rows_supported(int K, int cols) { return K % kAtomK == 0 && K >= kAtomK && cols >= 1 && cols <= 128; }
 
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s) {
   p.npad = (cols + 15) / 16 * 16;
-  const int stage_bytes = kATileBytes + p.npad * 128;
-  int stages = (220 * 1024 - 1024 - 512) / stage_bytes;
-  if (stages > 10) stages = 10;
-  if (stages < kLag + 2) return cudaErrorInvalidValue;
+  // Measured on B200 (4096 x 14336, B = 16): 1 atom per stage 153 us per call, 4 atoms 167 us, 2 atoms 183 us.
+  p.atoms = 1;  // the producers copy one 128-byte block per row and stage
+  const int stage_bytes = (kAAtomBytes + p.npad * 128) * p.atoms;
+  int stages = (220 * 1024 - 1024 - 5120) / stage_bytes;
+  if (stages > 12) stages = 12;
+  if (stages < 2) return cudaErrorInvalidValue;
   p.stages = stages;
-  const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 64;
+  const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 16 + 4 * 128 * 8 + 64;
   const int tiles = (p.R + kTileRows - 1) / kTileRows;
   const int grid = tiles < sm_count ? tiles : sm_count;
   static bool configured[2] = {false, false};

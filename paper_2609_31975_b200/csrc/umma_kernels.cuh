@@ -29,9 +29,10 @@ struct UmmaRowsParams {
   void* hmT;             // UP: bf16 [B][hm_stride]
   int hm_stride;
   int32_t* status;       // device status word
-  int npad, stages;      // filled by the launcher
+  int npad, stages, atoms;  // filled by the launcher
 };
 
+void debug_set_umma_atoms(int atoms);
 bool umma_rows_supported(int K, int cols);
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s);
 cudaError_t launch_split_interleaved(const float* n, int B, int r, int n_stride, void* x2, cudaStream_t s);
