@@ -91,7 +91,9 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def dist_setup(n_gpus: int):
+def dist_setup(n_gpus: int, backend: str = "nccl"):
+    """One process per GPU under torchrun; rank 0 alone when launched plainly.  `backend` is "nccl" on
+    GPUs and "gloo" in the CPU tests of this plumbing."""
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -99,12 +101,16 @@ def dist_setup(n_gpus: int):
         import torch.distributed as dist
 
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        if backend == "nccl":
+            torch.cuda.set_device(local)
+            dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        else:
+            dist.init_process_group(backend)
     return rank, world, local
 
 
 def max_over_ranks(ms: float, world: int, dev) -> float:
+    """Slowest rank's time: the job is as fast as its slowest replica."""
     if world == 1:
         return ms
     import torch.distributed as dist
@@ -114,12 +120,19 @@ def max_over_ranks(ms: float, world: int, dev) -> float:
     return float(t.item())
 
 
-def barrier(world: int):
+def barrier(world: int, cuda: bool = True):
     if world > 1:
         import torch.distributed as dist
 
         dist.barrier()
-    torch.cuda.synchronize()
+    if cuda:
+        torch.cuda.synchronize()
+
+
+def whole_job_us_per_call(ms_max: float, steps: int, calls_per_step: int, world: int) -> float:
+    """Microseconds per FFN call of the whole job: `world` replicas each made steps * calls_per_step
+    calls in ms_max milliseconds (weak scaling, no data-path collective)."""
+    return ms_max * 1e3 / (steps * calls_per_step * world)
 
 
 class Workload:
@@ -236,6 +249,7 @@ def run_ours(args, rank, world, local):
     launches = (wl.ffn.launch_count() - l0) * args.steps // (args.steps + args.warmup)
     calls = args.steps * args.calls
     us_call = ms * 1e3 / calls
+    assert abs(us_call / world - whole_job_us_per_call(ms, args.steps, args.calls, world)) < 1e-9
     if args.skip_extras:
         if rank == 0:
             print(json.dumps({"metric": "us_per_ffn_call", "value": us_call / world, "unit": "us/FFN-call",
@@ -285,6 +299,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--report", default=None, help="write the wider measurement matrix to this JSON file")
     ap.add_argument("--quick", action="store_true", help="with --report: one point per family")
+    ap.add_argument("--only", default=None, help="with --report: only the cases whose name contains this")
+    ap.add_argument("--report-calls", type=int, default=None, help="with --report: calls per case")
     ap.add_argument("--calls", type=int, default=CALLS_PER_STEP, help="FFN calls (tokens) per step")
     ap.add_argument("--skip-extras", action="store_true",
                     help="time the sparse path only (no dense comparator, host-buffer or CPU legs): for profiler runs")
@@ -298,7 +314,7 @@ def main():
             from paper_2609_31975_b200 import report
 
             if rank == 0:
-                report.run(args.report, quick=args.quick)
+                report.run(args.report, quick=args.quick, only=args.only, n_calls=args.report_calls)
         else:
             run_ours(args, rank, world, local)
     finally:

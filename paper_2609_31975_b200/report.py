@@ -74,12 +74,25 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1)
     return row
 
 
-def run(out_path, quick=False):
+def run(out_path, quick=False, only=None, n_calls=None):
+    """only: substring filter on the case names (for profiler runs); n_calls: calls per case."""
     peak = 6549.1
     mp = ROOT / "MEASURED_PEAKS.json"
     if mp.exists():
         peak = float(json.loads(mp.read_text())["hbm_gbs"])
     rows = []
+
+    def want(name):
+        return only is None or only in name
+
+    def add(name, *a, **k):
+        if not want(name):
+            return
+        if n_calls:
+            k["n_calls"] = n_calls
+        rows.append(measure(name, *a, **k))
+        print(json.dumps(rows[-1]), flush=True)
+
     D, H = 4096, 14336
     std = lambda w: {"W_g": w["W_g"]}
     # decode shape: sparsity sweep
@@ -87,15 +100,13 @@ def run(out_path, quick=False):
     for s in ((0.9,) if quick else (0.5, 0.7, 0.8, 0.9, 0.95)):
         b = syn.gate_bias_for_sparsity(s)
         sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in base]
-        rows.append(measure(f"decode 4096x14336 s={s}", D, H, 1, sets, std, "relu", peak=peak))
-        print(json.dumps(rows[-1]), flush=True)
+        add(f"decode 4096x14336 s={s}", D, H, 1, sets, std, "relu", peak=peak)
     # batched decode under Zipf firing
     p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
     zb = syn.bias_from_firing_profile(p).to(DEV)
     zsets = [dict(w, b_g=zb) for w in base]
     for B in ((16,) if quick else (4, 16, 64)):
-        rows.append(measure(f"batched zipf B={B}", D, H, B, zsets, std, "relu", n_calls=100, peak=peak))
-        print(json.dumps(rows[-1]), flush=True)
+        add(f"batched zipf B={B}", D, H, B, zsets, std, "relu", n_calls=100, peak=peak)
     # LoPA gates (up/down weights shared with the standard sets)
     gi = g_diagonal(H, D, DEV)
     for r in ((512,) if quick else (256, 512, 1024)):
@@ -106,12 +117,11 @@ def run(out_path, quick=False):
             lsets.append(lw)
         lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}
         for act in ("relu", "sqrelu"):
-            rows.append(measure(f"lopa r={r} {act}", D, H, 1, lsets, lg, act, r=r, peak=peak))
-            print(json.dumps(rows[-1]), flush=True)
+            add(f"lopa r={r} {act}", D, H, 1, lsets, lg, act, r=r, peak=peak)
         del lsets
     del base, zsets
     torch.cuda.empty_cache()
-    if not quick:
+    if not quick and (only is None or "stress" in only):
         # stress shape: 8 independent layers per step
         D, H = 8192, 28672
         layers = [syn.standard_ffn(D, H, torch.bfloat16, 5, DEV, sparsity=0.9, extra=i) for i in range(8)]
@@ -119,9 +129,7 @@ def run(out_path, quick=False):
             b = syn.gate_bias_for_sparsity(s)
             sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in layers]
             for B in (1, 8):
-                rows.append(measure(f"stress 8192x28672 s={s} B={B}", D, H, B, sets, std, "sqrelu", n_calls=64,
-                                    peak=peak))
-                print(json.dumps(rows[-1]), flush=True)
+                add(f"stress 8192x28672 s={s} B={B}", D, H, B, sets, std, "sqrelu", n_calls=64, peak=peak)
         gi = g_diagonal(H, D, DEV)
         lsets = []
         for i, w in enumerate(layers):
@@ -134,9 +142,7 @@ def run(out_path, quick=False):
             b = syn.gate_bias_for_sparsity(s, math.sqrt(2.0))
             sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in lsets]
             for B in (1, 8):
-                rows.append(measure(f"stress lopa r=1024 s={s} B={B}", D, H, B, sets, lg, "sqrelu", r=1024,
-                                    n_calls=64, peak=peak))
-                print(json.dumps(rows[-1]), flush=True)
+                add(f"stress lopa r=1024 s={s} B={B}", D, H, B, sets, lg, "sqrelu", r=1024, n_calls=64, peak=peak)
     Path(out_path).parent.mkdir(parents=True, exist_ok=True)
     Path(out_path).write_text(json.dumps(rows, indent=1))
     md = ["| case | B | fired rows | us/call | touched MB | GB/s | % of measured peak | % of 8 TB/s | dense us | speedup |",
