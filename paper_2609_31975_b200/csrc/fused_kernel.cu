@@ -1,6 +1,6 @@
 // Fused sparse gated FFN for one token on B200 (sm_100a).
 //
-// Main kernel: one persistent CTA per SM owns a contiguous slab of the H neurons and runs the whole
+// Main kernel: one persistent CTA per SM owns a share ("slab") of the H neurons and runs the whole
 // of the paper's sparse execution scheme (Sec. 3.1) on it without leaving the SM:
 //
 //   gate producer  one thread streams the slab's gate rows (W_1, or U for the LoPA gate) into a
@@ -80,7 +80,7 @@ struct FusedParams {
 
 // Shared-memory carve-up, identical on host and device.
 struct SmemLayout {
-  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, row_done, total;
+  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, total;
   __host__ __device__ SmemLayout(int D, int K, bool lopa, int n_gate_slots, int gate_slot_bytes,
                                  int n_act_slots, int act_slot_bytes, int slab_max) {
     int off = 0;
@@ -98,7 +98,6 @@ struct SmemLayout {
     red = take(2 * (2 * kActWarps + 1) * 4);
     ctl = take(8 * 4);
     bars = take(2 * (n_gate_slots + n_act_slots) * 8);
-    row_done = take(slab_max);
     total = off;
   }
 };
@@ -227,8 +226,6 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x, cta = blockIdx.x;
   const int D = p.D, K = p.K;
-  const int slab_lo = (int)((long long)p.H * cta / G);
-  const int slab_rows = (int)((long long)p.H * (cta + 1) / G) - slab_lo;
   const int NG = p.n_gate_slots, NA = p.n_act_slots;
   const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NA, p.act_slot_bytes, p.slab_max);
 
@@ -252,7 +249,16 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
   const size_t row_bytes = (size_t)D * sizeof(T);
   const size_t gate_row_bytes = (size_t)K * sizeof(T);
   const int nr = p.rows_per_gate_slot;
-  const int n_gslots = (slab_rows + nr - 1) / nr;
+  // Neurons are dealt to the CTAs in blocks of nr consecutive rows, round robin: CTA c owns the
+  // blocks c, c + G, c + 2G, ...  One block = one gate ring slot.  Compared with one contiguous slab
+  // per CTA this spreads neighbouring neurons, whose firing can be correlated (LoPA rows that share a
+  // column of the fixed matrix), over different CTAs.  Local row l of this CTA is row l % nr of its
+  // block l / nr; only the globally last block can be short, and it is the last block of its owner.
+  const int n_blocks = (p.H + nr - 1) / nr;
+  const int n_gslots = cta < n_blocks ? (n_blocks - cta + G - 1) / G : 0;
+  const int slab_rows =
+      n_gslots == 0 ? 0 : (n_gslots - 1) * nr + min(nr, p.H - (cta + (n_gslots - 1) * G) * nr);
+  auto slot_first_neuron = [&](int s) { return (cta + s * G) * nr; };
 
   if (warp < kGateProducers) {
     // ======================= gate producers ===================================================
@@ -275,15 +281,15 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
     named_bar_sync(4, 32 * kGateProducers);  // barriers are initialised
     named_bar_arrive(3, kThreads);           // release the other warps (they block on barrier 3)
     if (lane == 0) {
-      const char* Wg = static_cast<const char*>(p.Wgate) + (size_t)slab_lo * gate_row_bytes;
+      const char* Wg = static_cast<const char*>(p.Wgate);
       const uint32_t ring = smem_u32(gate_ring);
       for (int s = warp; s < n_gslots; s += kGateProducers) {
         const int slot = s % NG;
         if (!mbar_wait(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status)) break;
-        const int r0 = s * nr;
-        const uint32_t bytes = (uint32_t)(min(nr, slab_rows - r0) * gate_row_bytes);
+        const int j0 = slot_first_neuron(s);
+        const uint32_t bytes = (uint32_t)(min(nr, p.H - j0) * gate_row_bytes);
         mbar_expect_tx(full_gate + 8 * slot, bytes);
-        bulk_g2s(ring + (uint32_t)slot * p.gate_slot_bytes, Wg + (size_t)r0 * gate_row_bytes, bytes,
+        bulk_g2s(ring + (uint32_t)slot * p.gate_slot_bytes, Wg + (size_t)j0 * gate_row_bytes, bytes,
                  full_gate + 8 * slot);
       }
       if (warp == 0) SFFN_STAMP(1);
@@ -299,9 +305,9 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
   if (warp >= kFirstGateWarp && warp < kFirstActWarp && warp - kFirstGateWarp < p.gate_warps) {
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
-      const int r0 = (warp - kFirstGateWarp + q * p.gate_warps) * nr;
-      if (r0 + lane < slab_rows && lane < nr) {
-        const int j = slab_lo + r0 + lane;
+      const int sq = warp - kFirstGateWarp + q * p.gate_warps;
+      if (sq < n_gslots && lane < nr && slot_first_neuron(sq) + lane < p.H) {
+        const int j = slot_first_neuron(sq) + lane;
         if (p.b_g) pre_bias[q] = p.b_g[j];
         if (LOPA && p.g_idx) {
           pre_gi[q] = p.g_idx[j];
@@ -410,7 +416,8 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         if (lane == 0) {
           if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) {
             if (ap == 0) slot_a[slot] = sl == 0x80000000u ? 0.f : __uint_as_float(sl);
-            const size_t j = (size_t)(slab_lo + base + l);
+            const int lrow = base + l;
+            const size_t j = (size_t)(slot_first_neuron(lrow / nr) + lrow % nr);
             mbar_expect_tx(full_act + 8 * slot, (uint32_t)row_bytes);
             bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
                      full_act + 8 * slot);
@@ -435,10 +442,11 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
     for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_warps) {
       const int slot = s % NG;
       const int r0 = s * nr;
-      const int rows = min(nr, slab_rows - r0);
+      const int j0 = slot_first_neuron(s);
+      const int rows = min(nr, p.H - j0);
       float add = 0.f;  // bias + fixed-matrix term of the row this lane reports
       if (lane < rows) {
-        const int j = slab_lo + r0 + lane;
+        const int j = j0 + lane;
         float bias, sg;
         int gi;
         if (s == gw) { bias = pre_bias[0]; gi = pre_gi[0]; sg = pre_sg[0]; }
@@ -472,7 +480,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
       if (lane < rows) {
         const float z = mine + add;
         const bool fired = z > 0.f;
-        if (!p.dense) p.flag[slab_lo + r0 + lane] = fired ? 1 : 0;
+        if (!p.dense) p.flag[j0 + lane] = fired ? 1 : 0;
         row_state[r0 + lane] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
       }
       __syncwarp();
@@ -643,7 +651,7 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   g.rows_per_gate_slot = nr;
   g.gate_slot_bytes = (nr * gate_row_bytes + 127) / 128 * 128;
   g.act_slot_bytes = (2 * row_bytes + 127) / 128 * 128;
-  g.slab_max = (H + grid - 1) / grid;
+  g.slab_max = (((H + nr - 1) / nr + grid - 1) / grid) * nr;  // most rows one CTA can own
   const SmemLayout fixed(D, K, lopa, 0, 0, 0, 0, g.slab_max);
   const int ring = kSmemBudget - fixed.total - 2048;  // slack for the barrier words
   if (ring <= 0) return g;
