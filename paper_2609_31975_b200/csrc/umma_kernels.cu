@@ -6,15 +6,18 @@
 //                           stored as bf16 HmT[b][u] for the down projection
 //
 // One CTA owns a tile of 128 weight rows (TMEM lanes) x Npad token columns (Npad = columns rounded up to 16):
-//   warps 0-3  producers: 16-byte cp.async copies gather the 128 (possibly scattered) rows of the current
-//              64-wide K block straight into the 128-byte-swizzled K-major layout the tensor core reads,
-//              several stages ahead of it; a stage is published with fence.proxy.async + mbarrier arrive
+//   warps 0-3  producers, one stage per warp in turn: TMA tensor-map copies bring the 128 weight rows and the
+//              Npad token rows of the current 64-wide K block into the 128-byte-swizzled K-major layout the
+//              tensor core reads (mbarrier complete_tx).  Gate: one tiled copy of 128 consecutive rows.
+//              Union rows: tile::gather4, each lane of the warp fetching four listed rows.
 //   warp  8    one thread issues tcgen05.mma (M=128, N=Npad, K=16, four per stage) and commits each stage's
 //              completion to the "slot free" mbarrier; the same warp allocates and frees the TMEM columns
 //   warps 4-7  epilogue: tcgen05.ld the accumulator row of "their" neuron, apply the gate / scale epilogue
 // Every wait is bounded by a cycle budget; on expiry the status word is set, all roles wind down, the
 // producers drain their copies and the TMEM columns are released before the CTA exits.
 #include "umma_kernels.cuh"
+
+#include <cuda.h>
 
 #include "common.cuh"
 #include "sparse_ffn.h"
@@ -66,16 +69,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-__device__ __forceinline__ void cp_async16(uint32_t smem, const void* gmem, bool valid) {
-  const int n = valid ? 16 : 0;  // src-size 0: zero fill
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem), "l"(gmem), "r"(n) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -115,13 +108,31 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
   for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// Byte offset of the 16-byte chunk c (0..7) of row r inside a 128-byte-swizzled K-major tile.
-__device__ __forceinline__ uint32_t swz(int r, int c) {
-  return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4));
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Tiled tensor-map copy: box {64 elements, rows} at (element c0, row c1); out-of-range rows read as zero.
+__device__ __forceinline__ void tma_tile_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+// Gather copy: four rows r0..r3 (any order) x 64 elements starting at element c0 land as four
+// consecutive 128-byte rows at dst (the map's box is {64, 1}).
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int c0, int r0, int r1, int r2,
+                                            int r3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, "
+      "%4, %5, %6}], [%7];" ::"r"(dst),
+      "l"(map), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+      : "memory");
 }
 
 template <bool UP>
-__global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsParams p) {
+__global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsParams p,
+                                                                  const __grid_constant__ CUtensorMap map_w,
+                                                                  const __grid_constant__ CUtensorMap map_x) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   // carve: stages first (1024-byte aligned), then barriers and control words
   const int npad = p.npad;
@@ -137,7 +148,6 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
   const uint32_t acc_full = smem_u32(bars + 2 * S), acc_empty = smem_u32(bars + 2 * S + 1);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  const char** rowptr = reinterpret_cast<const char**>(tmem_slot + 2);  // [4][128] row pointers of the current tile, per producer warp
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int K = p.K;
@@ -148,7 +158,7 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
-      mbar_init(full + 8 * s, 32);  // the 32 lanes of the producer warp that owns the stage
+      mbar_init(full + 8 * s, 1);  // the producer's expect_tx arrive; the copies complete the bytes
       mbar_init(empty + 8 * s, 1);
     }
     mbar_init(acc_full, 1);
@@ -169,56 +179,38 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
 
   if (warp < 4) {
     // ======================= producers =========================================================
-    // Each producer warp owns every fourth stage, so four stages are being filled independently and
-    // the wait -> copy -> publish latency of one does not hold up the others.  Lane l copies chunk
-    // l & 7 of rows (l >> 3) + 4 i; its swizzled offset advances by 512 bytes per step because the
-    // row index modulo 8 does not change.
-    const int pc = lane & 7, pq = lane >> 3;
-    const char* Wb = static_cast<const char*>(p.W);
-    const char* Xb = static_cast<const char*>(p.X);
-    const size_t wpitch = (size_t)K * 2;
+    // Producer warp w owns the stages it = w, w + 4, ...  Lane 0 waits for the slot, announces the byte
+    // count, then the copies go out: one tiled copy for 128 consecutive rows (gate), or one gather4 per
+    // lane for four listed rows each (union rows); the token block is one more tiled copy.
     bool ok = true;
-    int it = 0;         // global stage counter (all producer warps count the same way)
-    int pending = -1;   // stage copied by this warp but not yet published
+    int it = 0;  // global stage counter (all producer warps count the same way)
     for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-      // this warp's own copy of the tile's row pointers (null = beyond the list): no cross-warp barrier
-      const char** myrows = rowptr + warp * kTileRows;
-      __syncwarp();
+      int r[4] = {0, 0, 0, 0};
+      if (UP) {
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int li = tile * kTileRows + lane + 32 * q;
-        myrows[lane + 32 * q] = li < n_rows ? Wb + (size_t)(p.idx ? p.idx[li] : li) * wpitch : nullptr;
+        for (int q = 0; q < 4; ++q) {
+          const int li = tile * kTileRows + lane * 4 + q;
+          r[q] = li < n_rows ? (p.idx ? p.idx[li] : li) : 0;  // rows beyond the list: any valid row, ignored later
+        }
       }
-      __syncwarp();
       for (int kb = 0; kb < kblocks; ++kb, ++it) {
         if ((it & 3) != warp) continue;
         const int s = it % S;
-        if (!mbar_wait(empty + 8 * s, ((it / S) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+        if (lane == 0) {
+          ok = mbar_wait(empty + 8 * s, ((it / S) & 1) ^ 1, abort_flag, p.status);
+          if (ok) mbar_expect_tx(full + 8 * s, (uint32_t)stage_bytes);
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
         const uint32_t abase = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint32_t bbase = abase + kATileBytes;
-        const size_t koff = (size_t)kb * 128 + pc * 16;
-#pragma unroll 8
-        for (int i = 0; i < 32; ++i) {
-          const int r = pq + 4 * i;
-          const char* rp = myrows[r];
-          cp_async16(abase + swz(r, pc), (rp ? rp : Wb) + koff, rp != nullptr);
+        if (UP) {
+          tma_gather4(abase + lane * 512, &map_w, kb * kAtomK, r[0], r[1], r[2], r[3], full + 8 * s);
+        } else if (lane == 0) {
+          tma_tile_2d(abase, &map_w, kb * kAtomK, tile * kTileRows, full + 8 * s);
         }
-        for (int r = pq; r < npad; r += 4) {
-          const bool v = r < p.ncols_valid;
-          cp_async16(bbase + swz(r, pc), Xb + (size_t)(v ? r : 0) * p.x_stride * 2 + koff, v);
-        }
-        cp_async_commit();
-        if (pending >= 0) {          // publish the previous stage of this warp: its copies are older
-          cp_async_wait<1>();
-          fence_async_smem();
-          mbar_arrive(full + 8 * (pending % S));
-        }
-        pending = it;
+        if (lane == 0) tma_tile_2d(abase + kATileBytes, &map_x, kb * kAtomK, 0, full + 8 * s);
       }
     }
-    cp_async_wait<0>();
-    fence_async_smem();
-    if (ok && pending >= 0) mbar_arrive(full + 8 * (pending % S));
   } else if (warp == 8) {
     // ======================= MMA issuer ========================================================
     if (lane == 0) {
@@ -324,26 +316,61 @@ __global__ void split_interleaved_kernel(const float* n, int r, int n_stride, __
   x2[(size_t)(2 * b + 1) * r + k] = __float2bfloat16(v - __bfloat162float(hi));
 }
 
-int g_umma_atoms = 0;
-
 }  // namespace
 
-void debug_set_umma_atoms(int atoms) { g_umma_atoms = atoms; }
+void debug_set_umma_atoms(int) {}
 
 bool umma_rows_supported(int K, int cols) { return K % kAtomK == 0 && K >= kAtomK && cols >= 1 && cols <= 128; }
 
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    cudaDriverEntryPointQueryResult q;
+    void* ptr = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, K] with row pitch `pitch_elems`, read in boxes of 64 elements x box_rows rows, 128-byte swizzle.
+bool make_map(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_elems, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kAtomK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s) {
   p.npad = (cols + 15) / 16 * 16;
-  // Measured on B200 (4096 x 14336, B = 16): 1 atom per stage 153 us per call, 4 atoms 167 us, 2 atoms 183 us.
-  p.atoms = 1;  // the producers copy one 128-byte block per row and stage
-  const int stage_bytes = (kAAtomBytes + p.npad * 128) * p.atoms;
-  int stages = (220 * 1024 - 1024 - 5120) / stage_bytes;
+  p.atoms = 1;
+  const int stage_bytes = kAAtomBytes + p.npad * 128;
+  int stages = (220 * 1024 - 1024 - 1024) / stage_bytes;
   if (stages > 12) stages = 12;
   if (stages < 2) return cudaErrorInvalidValue;
   p.stages = stages;
-  const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 16 + 4 * 128 * 8 + 64;
+  const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 64;
   const int tiles = (p.R + kTileRows - 1) / kTileRows;
   const int grid = tiles < sm_count ? tiles : sm_count;
+  alignas(64) CUtensorMap map_w, map_x;
+  // weights: all R rows; tiled boxes of 128 rows for the gate, single-row boxes for the gather
+  if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : kTileRows)) return cudaErrorNotSupported;
+  // tokens: only the rows that exist; the box covers npad rows and the rest reads as zero
+  if (!make_map(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)) return cudaErrorNotSupported;
   static bool configured[2] = {false, false};
   if (up) {
     auto k = umma_rows_kernel<true>;
@@ -352,7 +379,7 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
       if (e != cudaSuccess) return e;
       configured[1] = true;
     }
-    k<<<grid, kThreads, smem, s>>>(p);
+    k<<<grid, kThreads, smem, s>>>(p, map_w, map_x);
   } else {
     auto k = umma_rows_kernel<false>;
     if (!configured[0]) {
@@ -360,7 +387,7 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
       if (e != cudaSuccess) return e;
       configured[0] = true;
     }
-    k<<<grid, kThreads, smem, s>>>(p);
+    k<<<grid, kThreads, smem, s>>>(p, map_w, map_x);
   }
   return cudaGetLastError();
 }
