@@ -170,6 +170,10 @@ int sparse_ffn_forward_static(const void* x, const void* W_g, const float* b_g, 
                               const void* W_down, int D, int H, int dtype, int act, float* y,
                               void* stream);
 
+/* Name of the CUDA runtime error (cudaGetErrorName, with the library source line that saw it) behind the last SFFN_ERR_CUDA that a handle call
+ * returned on the calling thread; "cudaSuccess" if there was none.  Diagnostics only. */
+const char* sffn_last_cuda_error(void);
+
 /* Static string for a status code. */
 const char* sffn_status_string(int status);
 

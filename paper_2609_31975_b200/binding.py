@@ -16,7 +16,10 @@ _STATUS = {0: "ok", 1: "invalid argument", 2: "unsupported shape, alignment or p
 
 class SFFNError(RuntimeError):
     def __init__(self, where: str, code: int):
-        super().__init__(f"{where}: status {code} ({_STATUS.get(code, 'unknown')})")
+        detail = ""
+        if code == 4 and _lib is not None:
+            detail = ": " + _lib.sffn_last_cuda_error().decode()
+        super().__init__(f"{where}: status {code} ({_STATUS.get(code, 'unknown')}{detail})")
         self.code = code
 
 
@@ -58,6 +61,8 @@ def load_library() -> ctypes.CDLL:
         lib.sparse_ffn_forward_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, vp]
         lib.sffn_status_string.argtypes = [i]
         lib.sffn_status_string.restype = ctypes.c_char_p
+        lib.sffn_last_cuda_error.argtypes = []
+        lib.sffn_last_cuda_error.restype = ctypes.c_char_p
         _lib = lib
     return _lib
 

@@ -2,6 +2,8 @@
 // kernel dispatch.  No device memory is allocated or freed here.
 #include "sparse_ffn.h"
 
+#include <cstdio>
+
 #include <cuda_runtime.h>
 
 #include <new>
@@ -75,6 +77,7 @@ struct sffn_handle {
 };
 
 extern "C" {
+
 
 const char* sffn_status_string(int s) {
   switch (s) {
@@ -175,9 +178,18 @@ int check_call(const sffn_handle* h, const void* x, int B, const sffn_gate* g, c
   return SFFN_OK;
 }
 
-#define SFFN_CUDA(expr)                              \
-  do {                                               \
-    if ((expr) != cudaSuccess) return SFFN_ERR_CUDA; \
+// The CUDA error behind the calling thread's last SFFN_ERR_CUDA (sffn_last_cuda_error).
+thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+thread_local int g_last_cuda_line = 0;
+
+#define SFFN_CUDA(expr)               \
+  do {                                \
+    const cudaError_t e_ = (expr);    \
+    if (e_ != cudaSuccess) {          \
+      g_last_cuda_error = e_;         \
+      g_last_cuda_line = __LINE__;    \
+      return SFFN_ERR_CUDA;           \
+    }                                 \
   } while (0)
 
 // Batched tensor-core path (bf16, B >= 2): gate GEMM -> compaction of the union -> up GEMM over the
@@ -424,6 +436,13 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
 }  // namespace
 
 extern "C" {
+
+const char* sffn_last_cuda_error(void) {
+  static thread_local char text[96];
+  snprintf(text, sizeof(text), "%s (api.cu:%d)", cudaGetErrorName(g_last_cuda_error), g_last_cuda_line);
+  return g_last_cuda_error == cudaSuccess ? "cudaSuccess" : text;
+}
+
 
 int sparse_ffn_forward(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
                        const void* W_up, const void* W_down, int act, float* y, void* stream) {

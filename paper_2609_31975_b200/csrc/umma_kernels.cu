@@ -5,14 +5,18 @@
 //   umma_rows_kernel<UP>    over the union list of fired neurons (Sec. 5.4): Up = W_up[idx] X^T, Hm = a . Up,
 //                           stored as bf16 HmT[b][u] for the down projection
 //
-// One CTA owns a tile of 128 weight rows (TMEM lanes) x Npad token columns (Npad = columns rounded up to 16):
-//   warps 0-3  producers, one stage per warp in turn: TMA tensor-map copies bring the 128 weight rows and the
+// One CTA owns a tile of up to 128 weight rows (TMEM lanes) x Npad token columns (Npad = columns rounded up to 16):
+//   warps 0-3  producers, one stage per warp in turn: TMA tensor-map copies bring the tile's weight rows and the
 //              Npad token rows of the current 64-wide K block into the 128-byte-swizzled K-major layout the
-//              tensor core reads (mbarrier complete_tx).  Gate: one tiled copy of 128 consecutive rows.
+//              tensor core reads (mbarrier complete_tx).  Gate: one tiled copy of the tile's consecutive rows.
 //              Union rows: tile::gather4, each lane of the warp fetching four listed rows.
-//   warp  8    one thread issues tcgen05.mma (M=128, N=Npad, K=16, four per stage) and commits each stage's
-//              completion to the "slot free" mbarrier; the same warp allocates and frees the TMEM columns
-//   warps 4-7  epilogue: tcgen05.ld the accumulator row of "their" neuron, apply the gate / scale epilogue
+//   warps 8-9  one thread each issues tcgen05.mma (M=128, N=Npad, K=16, four per stage) for the even / odd
+//              K blocks into an accumulator of its own and commits each stage's completion to the "slot free"
+//              mbarrier (the serial wait - issue - commit chain of one thread is what limits a single issuer);
+//              warp 8 allocates and frees the TMEM columns
+//   warps 4-7  epilogue: tcgen05.ld the accumulator row of "their" neuron (both accumulators added), apply
+//              the gate / scale epilogue
+// A tile has 128 rows when a CTA owns several tiles; a smaller problem is cut into one tile per SM.
 // Every wait is bounded by a cycle budget; on expiry the status word is set, all roles wind down, the
 // producers drain their copies and the TMEM columns are released before the CTA exits.
 #include "umma_kernels.cuh"
@@ -29,9 +33,8 @@ namespace {
 constexpr int kTileRows = 128;
 constexpr int kAtomK = 64;                           // bf16 elements of one 128-byte swizzle row
 constexpr int kAAtomBytes = kTileRows * 128;         // 16 KB: one [128 rows x 64 k] swizzled block
-// A stage holds `atoms` (1, 2 or 4) such blocks side by side along K, i.e. 128 to 512 contiguous bytes of
-// every row.
-constexpr int kThreads = 288;                        // 4 producer warps, 4 epilogue warps, 1 MMA warp
+constexpr int kThreads = 320;                        // 4 producer warps, 4 epilogue warps, 2 MMA warps
+constexpr int kProducerWarps = 4;
 constexpr long long kWaitCycles = 1LL << 31;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -98,14 +101,20 @@ __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t b
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
-  uint32_t r[8];
+__device__ __forceinline__ void tmem_ld8_raw(uint32_t taddr, uint32_t* r) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                : "r"(taddr));
+}
+// Eight accumulator columns of this thread's TMEM lane, summed over the `nacc` accumulators that lie
+// `stride` columns apart.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int nacc, int stride, float* v) {
+  uint32_t r0[8], r1[8];
+  tmem_ld8_raw(taddr, r0);
+  if (nacc == 2) tmem_ld8_raw(taddr + stride, r1);
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r0[i]) + (nacc == 2 ? __uint_as_float(r1[i]) : 0.f);
 }
 
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
@@ -129,6 +138,14 @@ __device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Rows per tile: 128 when there is more than one tile per CTA, otherwise the row count spread over
+// the whole grid (a multiple of 8, the swizzle period), so that every SM streams a share.
+__host__ __device__ inline int tile_rows_for(int n_rows, int grid) {
+  if (n_rows >= kTileRows * grid) return kTileRows;
+  int t = ((n_rows + grid - 1) / grid + 7) & ~7;
+  return t < 8 ? 8 : t > kTileRows ? kTileRows : t;
+}
+
 template <bool UP>
 __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsParams p,
                                                                   const __grid_constant__ CUtensorMap map_w,
@@ -136,35 +153,39 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   // carve: stages first (1024-byte aligned), then barriers and control words
   const int npad = p.npad;
-  const int kAtoms = p.atoms;
-  const int kKBlock = kAtomK * kAtoms;
-  const int kATileBytes = kAAtomBytes * kAtoms;
-  const int b_atom_bytes = npad * 128;
-  const int stage_bytes = kATileBytes + b_atom_bytes * kAtoms;
+  const int stage_bytes = kAAtomBytes + npad * 128;
   const int S = p.stages;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
+  const uint32_t stage0 = smem_u32(smem);
   const uint32_t full = smem_u32(bars), empty = smem_u32(bars + S);
   const uint32_t acc_full = smem_u32(bars + 2 * S), acc_empty = smem_u32(bars + 2 * S + 1);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int K = p.K;
   const int n_rows = p.count ? *p.count : p.R;
-  const int n_tiles = (n_rows + kTileRows - 1) / kTileRows;
-  const int kblocks = (K + kKBlock - 1) / kKBlock;   // the last one may hold fewer atoms
-  const uint32_t tmem_cols = npad <= 32 ? 32 : npad <= 64 ? 64 : 128;
+  const int tile_rows = tile_rows_for(n_rows, gridDim.x);
+  const int n_tiles = (n_rows + tile_rows - 1) / tile_rows;
+  const int kblocks = p.K / kAtomK;
+  // Two MMA issuers take the even and the odd stages into accumulators of their own (npad TMEM columns
+  // each); the epilogue adds them.  With two or more K blocks per tile each issuer gets at least one of
+  // every tile; a single K block leaves the second issuer idle.
+  const int nacc = kblocks >= 2 ? 2 : 1;
+  const int acc_cols = nacc * npad;
+  const uint32_t tmem_cols = acc_cols <= 32 ? 32 : acc_cols <= 64 ? 64 : acc_cols <= 128 ? 128 : 256;
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(full + 8 * s, 1);  // the producer's expect_tx arrive; the copies complete the bytes
       mbar_init(empty + 8 * s, 1);
     }
-    mbar_init(acc_full, 1);
+    mbar_init(acc_full, nacc);
     mbar_init(acc_empty, 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
   }
   if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -177,65 +198,77 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp < 4) {
+  if (warp < kProducerWarps) {
     // ======================= producers =========================================================
-    // Producer warp w owns the stages it = w, w + 4, ...  Lane 0 waits for the slot, announces the byte
-    // count, then the copies go out: one tiled copy for 128 consecutive rows (gate), or one gather4 per
-    // lane for four listed rows each (union rows); the token block is one more tiled copy.
-    bool ok = true;
-    int it = 0;  // global stage counter (all producer warps count the same way)
-    for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-      int r[4] = {0, 0, 0, 0};
-      if (UP) {
+    // Stages are numbered it = 0, 1, ... over this CTA's (tile, K block) sequence and use ring slot
+    // it mod S.  A slot always belongs to the same producer warp (slot mod 4) and the same MMA issuer
+    // (slot mod 2, S is even): a waiter that owns its slot can never be two barrier phases behind it,
+    // which a parity wait could not tell from "ready".  Lane 0 waits for the slot and announces the byte
+    // count, then the copies go out: one tiled copy for the tile's consecutive rows (gate), or one
+    // gather4 per lane for four listed rows each (union rows); the token block is one more tiled copy.
+    const uint32_t tx_bytes = (uint32_t)(tile_rows + npad) * 128;
+    int s = 0, ph = 0, kb = 0, tile = blockIdx.x;
+    int rows_of = -1;
+    int r[4] = {0, 0, 0, 0};
+    for (; tile < n_tiles; ++s, ++kb) {
+      if (s == S) { s = 0; ph ^= 1; }
+      if (kb == kblocks) {
+        kb = 0;
+        tile += gridDim.x;
+        if (tile >= n_tiles) break;
+      }
+      if ((s & (kProducerWarps - 1)) != warp) continue;
+      if (UP && tile != rows_of) {
+        rows_of = tile;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const int li = tile * kTileRows + lane * 4 + q;
+          const int li = tile * tile_rows + lane * 4 + q;
           r[q] = li < n_rows ? (p.idx ? p.idx[li] : li) : 0;  // rows beyond the list: any valid row, ignored later
         }
       }
-      for (int kb = 0; kb < kblocks; ++kb, ++it) {
-        if ((it & 3) != warp) continue;
-        const int s = it % S;
-        if (lane == 0) {
-          ok = mbar_wait(empty + 8 * s, ((it / S) & 1) ^ 1, abort_flag, p.status);
-          if (ok) mbar_expect_tx(full + 8 * s, (uint32_t)stage_bytes);
-        }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
-        const uint32_t abase = smem_u32(smem + (size_t)s * stage_bytes);
-        if (UP) {
-          tma_gather4(abase + lane * 512, &map_w, kb * kAtomK, r[0], r[1], r[2], r[3], full + 8 * s);
-        } else if (lane == 0) {
-          tma_tile_2d(abase, &map_w, kb * kAtomK, tile * kTileRows, full + 8 * s);
-        }
-        if (lane == 0) tma_tile_2d(abase + kATileBytes, &map_x, kb * kAtomK, 0, full + 8 * s);
+      int ok = 1;
+      if (lane == 0) {
+        ok = mbar_wait(empty + 8 * s, ph ^ 1, abort_flag, p.status) ? 1 : 0;
+        if (ok) mbar_expect_tx(full + 8 * s, tx_bytes);
       }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const uint32_t abase = stage0 + s * stage_bytes;
+      if (UP) {
+        if (lane * 4 < tile_rows)
+          tma_gather4(abase + lane * 512, &map_w, kb * kAtomK, r[0], r[1], r[2], r[3], full + 8 * s);
+      } else if (lane == 0) {
+        tma_tile_2d(abase, &map_w, kb * kAtomK, tile * tile_rows, full + 8 * s);
+      }
+      if (lane == 0) tma_tile_2d(abase + kAAtomBytes, &map_x, kb * kAtomK, 0, full + 8 * s);
     }
-  } else if (warp == 8) {
-    // ======================= MMA issuer ========================================================
-    if (lane == 0) {
+  } else if (warp >= 8) {
+    // ======================= MMA issuers =======================================================
+    const int m = warp - 8;
+    if (lane == 0 && m < nacc) {
       const uint32_t idesc = make_idesc(npad);
-      int it = 0, tcount = 0;
+      const uint32_t acc = tmem_base + m * npad;
+      int tcount = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++tcount) {
         if (!mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, p.status)) break;
         tc_fence_after();
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const int s = it % S;
-          if (!mbar_wait(full + 8 * s, (it / S) & 1, abort_flag, p.status)) { ok = false; break; }
+        const int it0 = tcount * kblocks;
+        int s = it0 % S, ph = (it0 / S) & 1;
+        for (int kb = 0; kb < kblocks; ++kb, ++s) {
+          if (s == S) { s = 0; ph ^= 1; }
+          if (nacc == 2 && (s & 1) != m) continue;   // the other issuer's slot
+          if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sbase = smem_u32(smem + (size_t)s * stage_bytes);
-          const int atoms = min(kAtoms, (K - kb * kKBlock) / kAtomK);
-          for (int a = 0; a < atoms; ++a) {
-            const uint64_t adesc = make_desc(sbase + a * kAAtomBytes);
-            const uint64_t bdesc = make_desc(sbase + kATileBytes + a * b_atom_bytes);
+          const uint32_t sbase = stage0 + s * stage_bytes;
+          const uint64_t adesc = make_desc(sbase);
+          const uint64_t bdesc = make_desc(sbase + kAAtomBytes);
+          umma(acc, adesc, bdesc, idesc, kb >= nacc ? 1u : 0u);
 #pragma unroll
-            for (int k = 0; k < kAtomK / 16; ++k)
-              umma(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | a | k) ? 1u : 0u);
-          }
+          for (int k = 1; k < kAtomK / 16; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
           umma_commit(empty + 8 * s);   // slot free once these MMAs have read it
         }
-        if (ok) umma_commit(acc_full);  // accumulator complete
+        if (ok) umma_commit(acc_full);  // this issuer's accumulator is complete
       }
     }
     __syncwarp();
@@ -244,35 +277,51 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
     const int ew = warp - 4;                 // TMEM lanes 32*ew .. 32*ew + 31
     const int row_in_tile = ew * 32 + lane;
     const int B = p.B;
+    const uint32_t taddr = tmem_base + ((uint32_t)(ew * 32) << 16);
     int tcount = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
-      if (!mbar_wait(acc_full, tcount & 1, abort_flag, p.status)) break;
-      __syncwarp();
-      tc_fence_after();
-      const int li = tile * kTileRows + row_in_tile;
-      const bool row_ok = li < n_rows;
+      const int li = tile * tile_rows + row_in_tile;
+      const bool row_ok = row_in_tile < tile_rows && li < n_rows;
       const int j = row_ok ? (p.idx ? p.idx[li] : li) : 0;
-      const uint32_t taddr = tmem_base + ((uint32_t)(ew * 32) << 16);
+      // everything that does not depend on the accumulator is fetched before the wait
+      float pre[16];
+      float bias = 0.f, sg = 1.f;
+      int gi = -1;
       if (UP) {
+#pragma unroll
+        for (int q = 0; q < 16; ++q) pre[q] = (row_ok && q < B) ? p.a[(size_t)q * p.a_stride + j] : 0.f;
+      } else {
+        bias = (row_ok && p.b_g) ? p.b_g[j] : 0.f;
+        gi = (row_ok && p.g_idx) ? p.g_idx[j] : -1;
+        sg = (row_ok && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
+      }
+      int okw = 1;
+      if (lane == 0) okw = mbar_wait(acc_full, tcount & 1, abort_flag, p.status) ? 1 : 0;
+      okw = __shfl_sync(0xffffffffu, okw, 0);
+      if (!okw) break;
+      tc_fence_after();
+      if (UP) {
+        __nv_bfloat16* hm = static_cast<__nv_bfloat16*>(p.hmT);
         for (int c0 = 0; c0 < npad; c0 += 8) {
-          float v[8];
-          tmem_ld8(taddr + c0, v);
+          float av[8];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             const int b = c0 + q;
-            if (row_ok && b < B)
-              static_cast<__nv_bfloat16*>(p.hmT)[(size_t)b * p.hm_stride + li] =
-                  __float2bfloat16(p.a[(size_t)b * p.a_stride + j] * v[q]);
+            av[q] = c0 == 0 ? pre[q] : c0 == 8 ? pre[8 + q] : ((row_ok && b < B) ? p.a[(size_t)b * p.a_stride + j] : 0.f);
+          }
+          float v[8];
+          tmem_ld8(taddr + c0, nacc, npad, v);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int b = c0 + q;
+            if (row_ok && b < B) hm[(size_t)b * p.hm_stride + li] = __float2bfloat16(av[q] * v[q]);
           }
         }
       } else {
-        const float bias = (row_ok && p.b_g) ? p.b_g[j] : 0.f;
-        const int gi = (row_ok && p.g_idx) ? p.g_idx[j] : -1;
-        const float sg = (row_ok && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
         bool fired = false;
         for (int c0 = 0; c0 < npad; c0 += 8) {
           float v[8];
-          tmem_ld8(taddr + c0, v);
+          tmem_ld8(taddr + c0, nacc, npad, v);
           const int per = p.split_cols ? 4 : 8;  // tokens covered by these eight columns
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
@@ -357,18 +406,17 @@ bool make_map(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_el
 
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s) {
   p.npad = (cols + 15) / 16 * 16;
-  p.atoms = 1;
   const int stage_bytes = kAAtomBytes + p.npad * 128;
   int stages = (220 * 1024 - 1024 - 1024) / stage_bytes;
   if (stages > 12) stages = 12;
+  stages &= ~1;  // even: slot parity = issuer
   if (stages < 2) return cudaErrorInvalidValue;
   p.stages = stages;
   const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 64;
-  const int tiles = (p.R + kTileRows - 1) / kTileRows;
-  const int grid = tiles < sm_count ? tiles : sm_count;
+  const int grid = p.R < 8 * sm_count ? (p.R + 7) / 8 : sm_count;
   alignas(64) CUtensorMap map_w, map_x;
-  // weights: all R rows; tiled boxes of 128 rows for the gate, single-row boxes for the gather
-  if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : kTileRows)) return cudaErrorNotSupported;
+  // weights: all R rows; boxes of one tile's rows for the gate, single-row boxes for the gather
+  if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : tile_rows_for(p.R, grid))) return cudaErrorNotSupported;
   // tokens: only the rows that exist; the box covers npad rows and the rest reads as zero
   if (!make_map(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)) return cudaErrorNotSupported;
   static bool configured[2] = {false, false};
