@@ -39,7 +39,7 @@ Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
   L.status = take(256);  // [0] device status, [1] length of idx
   L.act = take((size_t)B_max * H * 4);
   L.flag = take((size_t)H);
-  L.idx = take((size_t)H * 4);
+  L.idx = take(((size_t)H + 64) * 4);  // readable one 64-row block past the list
   L.v = take((size_t)B_max * (r_max > 0 ? r_max : 1) * 4);
   L.n = take((size_t)B_max * (r_max > 0 ? r_max : 1) * 4);
   const size_t part_general = (size_t)kMaxUpDownGrid * kMaxChunk * D * 4;
@@ -48,7 +48,7 @@ Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
   L.xstage = take((size_t)B_max * D * esz);
   L.ystage = take((size_t)B_max * D * 4);
   L.fused = take(sffn::fused_workspace_bytes(D, H, r_max));
-  L.hm_stride = (H + 15) / 16 * 16 + 16;
+  L.hm_stride = (H + 63) / 64 * 64 + 64;
   L.hmT = take((size_t)(B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * L.hm_stride * 2);
   L.x2 = take((size_t)2 * (B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * (r_max > 0 ? r_max : 1) * 2);
   L.total = off;
@@ -300,13 +300,24 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       p.hmT = hmT; p.hm_stride = h->L.hm_stride;
       SFFN_CUDA(launch_rows_mma(true, p, nb, grid_rows, s));
     }
-    DownMmaParams d{};
-    d.W_down = W_down; d.R = H; d.D = D;
-    d.idx = lidx; d.count = lcount;
-    d.hmT = hmT; d.hm_stride = h->L.hm_stride; d.B = nb;
-    d.partial = partial;
-    SFFN_CUDA(launch_down_mma(d, splits, s));
-    SFFN_CUDA(launch_reduce(partial, splits, nb, D, y + (size_t)b0 * D, D, s));
+    int nsplit = splits;
+    if (umma && umma_down_supported(D, nb)) {
+      UmmaDownParams d{};
+      d.W_down = W_down; d.R = H; d.D = D;
+      d.idx = lidx; d.count = lcount;
+      d.hmT = hmT; d.hm_stride = h->L.hm_stride; d.B = nb;
+      d.splits = nsplit = umma_down_splits(D, h->sm_count, kMaxSplits);
+      d.partial = partial; d.status = h->at<int32_t>(h->L.status);
+      SFFN_CUDA(launch_umma_down(d, s));
+    } else {
+      DownMmaParams d{};
+      d.W_down = W_down; d.R = H; d.D = D;
+      d.idx = lidx; d.count = lcount;
+      d.hmT = hmT; d.hm_stride = h->L.hm_stride; d.B = nb;
+      d.partial = partial;
+      SFFN_CUDA(launch_down_mma(d, splits, s));
+    }
+    SFFN_CUDA(launch_reduce(partial, nsplit, nb, D, y + (size_t)b0 * D, D, s));
     h->launches += 3;
   }
   return SFFN_OK;

@@ -86,6 +86,18 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
   return d;
 }
+// The same for an MN-major operand (here: A[m][k] stored as rows k of 64 contiguous m, 128 bytes each):
+// eight k rows form a 1024-byte swizzle atom; `k_group_bytes` apart lie successive groups of eight k rows
+// (stride byte offset), `mn_atom_bytes` apart successive blocks of 64 m (leading byte offset).
+__device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr, uint32_t mn_atom_bytes, uint32_t k_group_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3fff);
+  d |= (uint64_t)((mn_atom_bytes >> 4) & 0x3fff) << 16;
+  d |= (uint64_t)((k_group_bytes >> 4) & 0x3fff) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
 __device__ __forceinline__ uint32_t make_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
@@ -278,6 +290,13 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
     const int row_in_tile = ew * 32 + lane;
     const int B = p.B;
     const uint32_t taddr = tmem_base + ((uint32_t)(ew * 32) << 16);
+    if (UP && blockIdx.x == 0) {
+      // the down projection walks the list in blocks of 64 rows: entries past its end must read as zero
+      __nv_bfloat16* hm = static_cast<__nv_bfloat16*>(p.hmT);
+      const int end = (n_rows + 63) & ~63;
+      for (int li = n_rows + row_in_tile; li < end; li += 128)
+        for (int b = 0; b < B; ++b) hm[(size_t)b * p.hm_stride + li] = __float2bfloat16(0.f);
+    }
     int tcount = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
       const int li = tile * tile_rows + row_in_tile;
@@ -346,6 +365,158 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
   }
 
   // ---- teardown: everybody meets, then the allocating warp frees the TMEM columns ------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Down projection over the union list (Sec. 5.4): partial[sp][b][d] = sum over the split's listed rows u of
+// Hm[b][u] * W_down[idx[u]][d].  One CTA owns 128 output columns d (TMEM lanes) and one split of the list;
+// the contraction runs over list rows, so the gathered W_down rows are the MN-major A operand (each
+// gathered row delivers 64 contiguous d per swizzle row) and HmT[b][u] is the K-major B operand.
+// Same pipeline as above: 4 producer warps (gather4 per lane: 2 column halves x 16 row quads = one 64-row
+// stage), 2 MMA issuers with their own accumulators, 4 epilogue warps; two CTAs share an SM.
+__global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownParams p,
+                                                                  const __grid_constant__ CUtensorMap map_wg,
+                                                                  const __grid_constant__ CUtensorMap map_wt,
+                                                                  const __grid_constant__ CUtensorMap map_hm) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const int npad = p.npad;
+  const int stage_bytes = kAAtomBytes + npad * 128;
+  const int S = p.stages;
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
+  const uint32_t stage0 = smem_u32(smem);
+  const uint32_t full = smem_u32(bars), empty = smem_u32(bars + S);
+  const uint32_t acc_full = smem_u32(bars + 2 * S);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_rows = p.count ? *p.count : p.R;
+  const int d_tiles = p.D / kTileRows;
+  const int dt = blockIdx.x % d_tiles, sp = blockIdx.x / d_tiles;
+  const int d0 = dt * kTileRows;
+  // the split's share of the list, in blocks of 64 rows
+  const int total_blocks = (n_rows + kAtomK - 1) / kAtomK;
+  const int per_split = (total_blocks + p.splits - 1) / p.splits;
+  const int kb0 = sp * per_split;
+  const int kblocks = min(total_blocks, kb0 + per_split) - kb0;  // <= 0: nothing to add, the partial is zero
+  const int nacc = kblocks >= 2 ? 2 : 1;
+  const int acc_cols = nacc * npad;
+  const uint32_t tmem_cols = acc_cols <= 32 ? 32 : acc_cols <= 64 ? 64 : acc_cols <= 128 ? 128 : 256;
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full + 8 * s, 1);
+      mbar_init(empty + 8 * s, 1);
+    }
+    mbar_init(acc_full, nacc);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(p.idx ? &map_wg : &map_wt) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hm) : "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp < kProducerWarps) {
+    // ======================= producers (slot s belongs to warp s mod 4) =========================
+    const uint32_t tx_bytes = (uint32_t)(kAAtomBytes + npad * 128);
+    const int half = lane >> 4, quad = lane & 15;
+    int s = 0, ph = 0;
+    for (int kb = 0; kb < kblocks; ++kb, ++s) {
+      if (s == S) { s = 0; ph ^= 1; }
+      if ((s & (kProducerWarps - 1)) != warp) continue;
+      const int u0 = (kb0 + kb) * kAtomK;
+      int r[4] = {0, 0, 0, 0};
+      if (p.idx) {
+        // four list entries of this lane (the list buffer is readable past its length; entries there are
+        // replaced by row 0, whose products vanish against the zeroed tail of HmT)
+        const int u = u0 + quad * 4;
+        const int4 v = *reinterpret_cast<const int4*>(p.idx + u);
+        r[0] = u + 0 < n_rows ? v.x : 0;
+        r[1] = u + 1 < n_rows ? v.y : 0;
+        r[2] = u + 2 < n_rows ? v.z : 0;
+        r[3] = u + 3 < n_rows ? v.w : 0;
+      }
+      int ok = 1;
+      if (lane == 0) {
+        ok = mbar_wait(empty + 8 * s, ph ^ 1, abort_flag, p.status) ? 1 : 0;
+        if (ok) mbar_expect_tx(full + 8 * s, tx_bytes);
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const uint32_t abase = stage0 + s * stage_bytes;
+      if (p.idx) {
+        tma_gather4(abase + half * 8192 + quad * 512, &map_wg, d0 + half * kAtomK, r[0], r[1], r[2], r[3], full + 8 * s);
+      } else if (lane < 2) {
+        // every row: 64 consecutive rows per column half; rows past the matrix read as zero
+        tma_tile_2d(abase + lane * 8192, &map_wt, d0 + lane * kAtomK, u0, full + 8 * s);
+      }
+      if (lane == 0) tma_tile_2d(abase + kAAtomBytes, &map_hm, u0, 0, full + 8 * s);
+    }
+  } else if (warp >= 8) {
+    // ======================= MMA issuers (slot s belongs to issuer s mod 2) =====================
+    const int m = warp - 8;
+    if (lane == 0 && m < nacc) {
+      const uint32_t idesc = make_idesc(npad) | (1u << 15);  // A is MN-major
+      const uint32_t acc = tmem_base + m * npad;
+      int s = 0, ph = 0;
+      bool ok = true;
+      for (int kb = 0; kb < kblocks; ++kb, ++s) {
+        if (s == S) { s = 0; ph ^= 1; }
+        if (nacc == 2 && (s & 1) != m) continue;
+        if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sbase = stage0 + s * stage_bytes;
+        const uint64_t bdesc = make_desc(sbase + kAAtomBytes);
+#pragma unroll
+        for (int k = 0; k < kAtomK / 16; ++k)  // 16 list rows = two groups of eight swizzle rows
+          umma(acc, make_desc_mn(sbase + k * 2048, 8192, 1024), bdesc + 2 * k, idesc, (kb >= nacc || k > 0) ? 1u : 0u);
+        umma_commit(empty + 8 * s);
+      }
+      if (ok && kblocks > 0) umma_commit(acc_full);
+    }
+    __syncwarp();
+  } else {
+    // ======================= epilogue: lane = output column d, TMEM columns = tokens ============
+    const int ew = warp - 4;
+    const int d = d0 + ew * 32 + lane;
+    const int B = p.B;
+    float* out = p.partial + (size_t)sp * B * p.D + d;
+    const uint32_t taddr = tmem_base + ((uint32_t)(ew * 32) << 16);
+    if (kblocks <= 0) {
+      for (int b = 0; b < B; ++b) out[(size_t)b * p.D] = 0.f;
+    } else {
+      int okw = 1;
+      if (lane == 0) okw = mbar_wait(acc_full, 0, abort_flag, p.status) ? 1 : 0;
+      okw = __shfl_sync(0xffffffffu, okw, 0);
+      if (okw) {
+        tc_fence_after();
+        for (int c0 = 0; c0 < npad; c0 += 8) {
+          float v[8];
+          tmem_ld8(taddr + c0, nacc, npad, v);
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            if (c0 + q < B) out[(size_t)(c0 + q) * p.D] = v[q];
+        }
+      }
+    }
+  }
+
   tc_fence_before();
   __syncthreads();
   if (warp == 8) {
@@ -437,6 +608,40 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
     }
     k<<<grid, kThreads, smem, s>>>(p, map_w, map_x);
   }
+  return cudaGetLastError();
+}
+
+int umma_down_splits(int D, int sm_count, int max_splits) {
+  const int d_tiles = D / kTileRows;
+  int splits = 2 * sm_count / (d_tiles > 0 ? d_tiles : 1);  // two CTAs per SM
+  return splits < 1 ? 1 : splits > max_splits ? max_splits : splits;
+}
+
+bool umma_down_supported(int D, int cols) { return D % kTileRows == 0 && cols >= 1 && cols <= 64; }
+
+cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s) {
+  p.npad = (p.B + 15) / 16 * 16;
+  const int stage_bytes = kAAtomBytes + p.npad * 128;
+  int stages = (111 * 1024 - 1024 - 1024) / stage_bytes;
+  if (stages > 12) stages = 12;
+  stages &= ~1;
+  if (stages < 2) return cudaErrorInvalidValue;
+  p.stages = stages;
+  const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 64;
+  const int grid = (p.D / kTileRows) * p.splits;
+  alignas(64) CUtensorMap map_wg, map_wt, map_hm;
+  // W_down [H, D]: inner dimension d; single-row boxes for the gather, 64-row boxes for the dense walk
+  if (!make_map(&map_wg, p.W_down, p.D, p.R, (size_t)p.D, 1)) return cudaErrorNotSupported;
+  if (!make_map(&map_wt, p.W_down, p.D, p.R, (size_t)p.D, kAtomK)) return cudaErrorNotSupported;
+  // HmT [B][hm_stride]: inner dimension u; token rows past B read as zero
+  if (!make_map(&map_hm, p.hmT, p.hm_stride, p.B, (size_t)p.hm_stride, p.npad)) return cudaErrorNotSupported;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(umma_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  umma_down_kernel<<<grid, kThreads, smem, s>>>(p, map_wg, map_wt, map_hm);
   return cudaGetLastError();
 }
 

@@ -32,7 +32,24 @@ struct UmmaRowsParams {
   int npad, stages;  // filled by the launcher
 };
 
+struct UmmaDownParams {
+  const void* W_down;    // [R, D] bf16
+  int R, D;
+  const int32_t* idx;    // list of rows (readable up to the next multiple of 64 past its length), or null = all R rows
+  const int32_t* count;  // device length of the list, or null (= R)
+  const void* hmT;       // bf16 [B][hm_stride]; entries from the list's end to the next multiple of 64 are zero
+  int hm_stride;         // multiple of 64
+  int B;
+  int splits;            // the list is cut into this many runs of 64-row blocks
+  float* partial;        // [splits][B][D]
+  int32_t* status;
+  int npad, stages;      // filled by the launcher
+};
+
 void debug_set_umma_atoms(int atoms);
+int umma_down_splits(int D, int sm_count, int max_splits);
+bool umma_down_supported(int D, int cols);
+cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s);
 bool umma_rows_supported(int K, int cols);
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s);
 cudaError_t launch_split_interleaved(const float* n, int B, int r, int n_stride, void* x2, cudaStream_t s);
