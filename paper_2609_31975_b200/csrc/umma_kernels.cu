@@ -10,11 +10,13 @@
 //              Npad token rows of the current 64-wide K block into the 128-byte-swizzled K-major layout the
 //              tensor core reads (mbarrier complete_tx).  Gate: one tiled copy of the tile's consecutive rows.
 //              Union rows: tile::gather4, each lane of the warp fetching four listed rows.
-//   warps 8-9  one thread each issues tcgen05.mma (M=128, N=Npad, K=16, four per stage) for the even / odd
-//              K blocks into an accumulator of its own and commits each stage's completion to the "slot free"
-//              mbarrier (the serial wait - issue - commit chain of one thread is what limits a single issuer);
-//              warp 8 allocates and frees the TMEM columns
-//   warps 4-7  epilogue: tcgen05.ld the accumulator row of "their" neuron (both accumulators added), apply
+//   warps 8-11 one thread each issues tcgen05.mma (M=128, N=Npad, K=16, four per stage) for "its" ring slots
+//              into an accumulator of its own and commits each stage's completion to the "slot free" mbarrier.
+//              The serial wait - issue - commit chain of one thread takes on the order of a thousand cycles
+//              per stage whatever the MMA shape, so several issuers (four when the ring has eight or more
+//              slots, else two) are what lets the copies run at memory speed; warp 8 allocates and frees
+//              the TMEM columns
+//   warps 4-7  epilogue: tcgen05.ld the accumulator row of "their" neuron (all accumulators added), apply
 //              the gate / scale epilogue
 // A tile has 128 rows when a CTA owns several tiles; a smaller problem is cut into one tile per SM.
 // Every wait is bounded by a cycle budget; on expiry the status word is set, all roles wind down, the
@@ -34,6 +36,7 @@ constexpr int kTileRows = 128;
 constexpr int kAtomK = 64;                           // bf16 elements of one 128-byte swizzle row
 constexpr int kAAtomBytes = kTileRows * 128;         // 16 KB: one [128 rows x 64 k] swizzled block
 constexpr int kThreads = 320;                        // 4 producer warps, 4 epilogue warps, 2 MMA warps
+constexpr int kThreadsRows = 384;                    // rows kernels: up to 4 MMA warps
 constexpr int kProducerWarps = 4;
 constexpr long long kWaitCycles = 1LL << 31;
 
@@ -118,15 +121,24 @@ __device__ __forceinline__ void tmem_ld8_raw(uint32_t taddr, uint32_t* r) {
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                : "r"(taddr));
 }
-// Eight accumulator columns of this thread's TMEM lane, summed over the `nacc` accumulators that lie
-// `stride` columns apart.
+// Eight accumulator columns of this thread's TMEM lane, summed over the `nacc` (1, 2 or 4) accumulators
+// that lie `stride` columns apart.
 __device__ __forceinline__ void tmem_ld8(uint32_t taddr, int nacc, int stride, float* v) {
-  uint32_t r0[8], r1[8];
+  uint32_t r0[8], r1[8], r2[8], r3[8];
   tmem_ld8_raw(taddr, r0);
-  if (nacc == 2) tmem_ld8_raw(taddr + stride, r1);
+  if (nacc >= 2) tmem_ld8_raw(taddr + stride, r1);
+  if (nacc == 4) {
+    tmem_ld8_raw(taddr + 2 * stride, r2);
+    tmem_ld8_raw(taddr + 3 * stride, r3);
+  }
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r0[i]) + (nacc == 2 ? __uint_as_float(r1[i]) : 0.f);
+  for (int i = 0; i < 8; ++i) {
+    float a = __uint_as_float(r0[i]);
+    if (nacc >= 2) a += __uint_as_float(r1[i]);
+    if (nacc == 4) a += __uint_as_float(r2[i]) + __uint_as_float(r3[i]);
+    v[i] = a;
+  }
 }
 
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
@@ -159,17 +171,17 @@ __host__ __device__ inline int tile_rows_for(int n_rows, int grid) {
 }
 
 template <bool UP>
-__global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsParams p,
+__global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRowsParams p,
                                                                   const __grid_constant__ CUtensorMap map_w,
                                                                   const __grid_constant__ CUtensorMap map_x) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   // carve: stages first (1024-byte aligned), then barriers and control words
   const int npad = p.npad;
-  const int stage_bytes = kAAtomBytes + npad * 128;
+  const int stage_bytes = kAAtomBytes + p.atoms_max * npad * 128;
   const int S = p.stages;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
-  const uint32_t stage0 = smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem);  // barriers first: the stages end with a read-over pad
+  const uint32_t stage0 = smem_u32(smem) + 1024;
   const uint32_t full = smem_u32(bars), empty = smem_u32(bars + S);
   const uint32_t acc_full = smem_u32(bars + 2 * S), acc_empty = smem_u32(bars + 2 * S + 1);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
@@ -180,12 +192,20 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
   const int tile_rows = tile_rows_for(n_rows, gridDim.x);
   const int n_tiles = (n_rows + tile_rows - 1) / tile_rows;
   const int kblocks = p.K / kAtomK;
-  // Two MMA issuers take the even and the odd stages into accumulators of their own (npad TMEM columns
-  // each); the epilogue adds them.  With two or more K blocks per tile each issuer gets at least one of
-  // every tile; a single K block leaves the second issuer idle.
-  const int nacc = kblocks >= 2 ? 2 : 1;
+  // A stage holds `atoms` successive K blocks of the tile: short tiles (few rows) take several, so that a
+  // stage stays near 16 KB and the bytes in flight do not shrink with the tile.  Block a of a stage sits
+  // tile_rows * 128 bytes after block a - 1; the MMA of a block reads 128 rows from its start, i.e. on
+  // into the following blocks / the token blocks / the pad behind the last stage (rows that are ignored).
+  int atoms = kTileRows / tile_rows;
+  atoms = atoms > p.atoms_max ? p.atoms_max : atoms;
+  const int a_block_bytes = tile_rows * 128, b_block_bytes = npad * 128;
+  const int kstages = (kblocks + atoms - 1) / atoms;
+  // The MMA issuers take the stages of their ring slots (slot mod issuers) into accumulators of their own
+  // (npad TMEM columns each); the epilogue adds them.  A tile with at least as many stages as issuers
+  // gives each issuer a stage; shorter tiles use fewer issuers.
+  const int nacc = kstages >= p.issuers ? p.issuers : kstages >= 2 ? 2 : 1;
   const int acc_cols = nacc * npad;
-  const uint32_t tmem_cols = acc_cols <= 32 ? 32 : acc_cols <= 64 ? 64 : acc_cols <= 128 ? 128 : 256;
+  const uint32_t tmem_cols = acc_cols <= 32 ? 32 : acc_cols <= 64 ? 64 : acc_cols <= 128 ? 128 : acc_cols <= 256 ? 256 : 512;
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
@@ -218,18 +238,19 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
     // which a parity wait could not tell from "ready".  Lane 0 waits for the slot and announces the byte
     // count, then the copies go out: one tiled copy for the tile's consecutive rows (gate), or one
     // gather4 per lane for four listed rows each (union rows); the token block is one more tiled copy.
-    const uint32_t tx_bytes = (uint32_t)(tile_rows + npad) * 128;
-    int s = 0, ph = 0, kb = 0, tile = blockIdx.x;
+    int s = 0, ph = 0, kb = 0, tile = blockIdx.x;   // kb counts stages of the tile here
     int rows_of = -1;
     int r[4] = {0, 0, 0, 0};
     for (; tile < n_tiles; ++s, ++kb) {
       if (s == S) { s = 0; ph ^= 1; }
-      if (kb == kblocks) {
+      if (kb == kstages) {
         kb = 0;
         tile += gridDim.x;
         if (tile >= n_tiles) break;
       }
       if ((s & (kProducerWarps - 1)) != warp) continue;
+      const int na = min(atoms, kblocks - kb * atoms);
+      const uint32_t tx_bytes = (uint32_t)(na * (tile_rows + npad)) * 128;
       if (UP && tile != rows_of) {
         rows_of = tile;
 #pragma unroll
@@ -246,13 +267,16 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       const uint32_t abase = stage0 + s * stage_bytes;
-      if (UP) {
-        if (lane * 4 < tile_rows)
-          tma_gather4(abase + lane * 512, &map_w, kb * kAtomK, r[0], r[1], r[2], r[3], full + 8 * s);
-      } else if (lane == 0) {
-        tma_tile_2d(abase, &map_w, kb * kAtomK, tile * tile_rows, full + 8 * s);
+      for (int a = 0; a < na; ++a) {
+        const int k0 = (kb * atoms + a) * kAtomK;
+        if (UP) {
+          if (lane * 4 < tile_rows)
+            tma_gather4(abase + a * a_block_bytes + lane * 512, &map_w, k0, r[0], r[1], r[2], r[3], full + 8 * s);
+        } else if (lane == 0) {
+          tma_tile_2d(abase + a * a_block_bytes, &map_w, k0, tile * tile_rows, full + 8 * s);
+        }
+        if (lane == 0) tma_tile_2d(abase + kAAtomBytes + a * b_block_bytes, &map_x, k0, 0, full + 8 * s);
       }
-      if (lane == 0) tma_tile_2d(abase + kAAtomBytes, &map_x, kb * kAtomK, 0, full + 8 * s);
     }
   } else if (warp >= 8) {
     // ======================= MMA issuers =======================================================
@@ -265,19 +289,22 @@ __global__ void __launch_bounds__(kThreads, 1) umma_rows_kernel(const UmmaRowsPa
       for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++tcount) {
         if (!mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, p.status)) break;
         tc_fence_after();
-        const int it0 = tcount * kblocks;
+        const int it0 = tcount * kstages;
         int s = it0 % S, ph = (it0 / S) & 1;
-        for (int kb = 0; kb < kblocks; ++kb, ++s) {
+        for (int kb = 0; kb < kstages; ++kb, ++s) {
           if (s == S) { s = 0; ph ^= 1; }
-          if (nacc == 2 && (s & 1) != m) continue;   // the other issuer's slot
+          if ((s & (nacc - 1)) != m) continue;   // another issuer's slot
           if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sbase = stage0 + s * stage_bytes;
-          const uint64_t adesc = make_desc(sbase);
-          const uint64_t bdesc = make_desc(sbase + kAAtomBytes);
-          umma(acc, adesc, bdesc, idesc, kb >= nacc ? 1u : 0u);
+          const int na = min(atoms, kblocks - kb * atoms);
+          for (int a = 0; a < na; ++a) {
+            const uint64_t adesc = make_desc(sbase + a * a_block_bytes);
+            const uint64_t bdesc = make_desc(sbase + kAAtomBytes + a * b_block_bytes);
+            umma(acc, adesc, bdesc, idesc, (kb >= nacc || a > 0) ? 1u : 0u);
 #pragma unroll
-          for (int k = 1; k < kAtomK / 16; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+            for (int k = 1; k < kAtomK / 16; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+          }
           umma_commit(empty + 8 * s);   // slot free once these MMAs have read it
         }
         if (ok) umma_commit(acc_full);  // this issuer's accumulator is complete
@@ -577,14 +604,25 @@ bool make_map(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_el
 
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s) {
   p.npad = (cols + 15) / 16 * 16;
-  const int stage_bytes = kAAtomBytes + p.npad * 128;
-  int stages = (220 * 1024 - 1024 - 1024) / stage_bytes;
+  const int grid = p.R < 8 * sm_count ? (p.R + 7) / 8 : sm_count;
+  // K blocks per stage: up to 8 KB of token rows; the gate knows its tile height, the union rows only a bound
+  p.atoms_max = p.npad <= 16 ? 4 : p.npad <= 32 ? 2 : 1;
+  if (!up) {
+    const int fit = kTileRows / tile_rows_for(p.R, grid);
+    p.atoms_max = fit < p.atoms_max ? fit : p.atoms_max;
+  }
+  const int stage_bytes = kAAtomBytes + p.atoms_max * p.npad * 128;
+  // 1 KB of barriers in front; with several blocks per stage, 16 KB behind the last stage that the MMAs
+  // of the later blocks may read over
+  const int pad = p.atoms_max > 1 ? kAAtomBytes : 0;
+  int stages = (224 * 1024 - 1024 - 1024 - pad) / stage_bytes;
   if (stages > 12) stages = 12;
-  stages &= ~1;  // even: slot parity = issuer
+  // four issuers when each can own two or more slots, otherwise two; slots divide evenly among them
+  p.issuers = stages >= 8 ? 4 : 2;
+  stages &= ~(p.issuers - 1);
   if (stages < 2) return cudaErrorInvalidValue;
   p.stages = stages;
-  const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 64;
-  const int grid = p.R < 8 * sm_count ? (p.R + 7) / 8 : sm_count;
+  const size_t smem = 1024 + 1024 + (size_t)stages * stage_bytes + pad;
   alignas(64) CUtensorMap map_w, map_x;
   // weights: all R rows; boxes of one tile's rows for the gate, single-row boxes for the gather
   if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : tile_rows_for(p.R, grid))) return cudaErrorNotSupported;
@@ -598,7 +636,7 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
       if (e != cudaSuccess) return e;
       configured[1] = true;
     }
-    k<<<grid, kThreads, smem, s>>>(p, map_w, map_x);
+    k<<<grid, kThreadsRows, smem, s>>>(p, map_w, map_x);
   } else {
     auto k = umma_rows_kernel<false>;
     if (!configured[0]) {
@@ -606,7 +644,7 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
       if (e != cudaSuccess) return e;
       configured[0] = true;
     }
-    k<<<grid, kThreads, smem, s>>>(p, map_w, map_x);
+    k<<<grid, kThreadsRows, smem, s>>>(p, map_w, map_x);
   }
   return cudaGetLastError();
 }

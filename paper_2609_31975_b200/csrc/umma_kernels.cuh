@@ -29,7 +29,7 @@ struct UmmaRowsParams {
   void* hmT;             // UP: bf16 [B][hm_stride]
   int hm_stride;
   int32_t* status;       // device status word
-  int npad, stages;  // filled by the launcher
+  int npad, stages, issuers, atoms_max;  // filled by the launcher
 };
 
 struct UmmaDownParams {
