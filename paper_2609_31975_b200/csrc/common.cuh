@@ -68,4 +68,35 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// Programmatic dependent launch.  A kernel lets its successor in the stream start early
+// (launch_dependents) and waits for its predecessor's completion and memory flush (wait) before it
+// reads anything a predecessor may write and before its own first global write.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Host switch (diagnostics): false launches every kernel fully serialised.
+inline bool& pdl_enabled() {
+  static bool on = true;
+  return on;
+}
+
+// Launch with the programmatic-stream-serialisation attribute: the kernel may begin while its
+// predecessor in the stream is still running; its griddepcontrol.wait restores the ordering.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*k)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, k, args...);
+}
+
 }  // namespace sffn

@@ -142,12 +142,6 @@ __device__ __forceinline__ void named_bar_sync(int id, int threads) {
 __device__ __forceinline__ void named_bar_arrive(int id, int threads) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
-// Programmatic dependent launch: let the next kernel in the stream start / wait for the previous one.
-__device__ __forceinline__ void pdl_launch_dependents() {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 __device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status) {
   ctl[kAbort] = 1;
   atomicExch(status, (int32_t)SFFN_ERR_TIMEOUT);
@@ -629,7 +623,6 @@ __global__ void __launch_bounds__(256) fused_reduce_kernel(const float* partial,
 }
 
 // ---- host side --------------------------------------------------------------------------------
-int g_debug_pdl = 1;
 long long* g_debug_trace = nullptr;
 
 struct Geometry {
@@ -690,23 +683,6 @@ int fused_grid(int sm_count, int H) {
   return grid > H ? H : grid;
 }
 
-// Launch with the programmatic-stream-serialization attribute: the kernel may begin while its
-// predecessor in the stream is still running; its griddepcontrol.wait restores the ordering.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*k)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = g_debug_pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, k, args...);
-}
-
 template <typename T, bool LOPA>
 cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaStream_t s) {
   void (*k)(const FusedParams) = nullptr;
@@ -728,7 +704,7 @@ cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaS
 
 }  // namespace
 
-void debug_set_pdl(int on) { g_debug_pdl = on; }
+void debug_set_pdl(int on) { pdl_enabled() = on != 0; }
 void debug_set_trace(long long* device_buffer) { g_debug_trace = device_buffer; }
 
 size_t fused_workspace_bytes(int D, int H, int r_max) {

@@ -3,7 +3,7 @@
 //   rowdot_kernel   z = W vec (+ bias + fixed-matrix term), activation, per-neuron "fires" flag
 //                   (Eq. 1 gate; also the two stages of the LoPA gate, Eq. 3)
 //   rmsnorm_kernel  n = gain * v / sqrt(mean(v^2) + eps)          (LoPA in practice, Sec. 3.3)
-//   compact_kernel  ascending list of the neurons whose flag is set (warp ballot/popc + block scan)
+//   compact_kernel  ascending list of the neurons whose flag is set (16 flags per thread, block scan)
 //   updown_kernel   u_j = W_up[j].x, h_j = a_j u_j, y_part += h_j W_down[j] over the listed rows only
 //                   (sparse execution, Sec. 3.1; union of the batch's active sets, Sec. 5.4)
 //   reduce_kernel   y = sum of the per-CTA partials in CTA order (deterministic)
@@ -137,31 +137,57 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* v, float* n, 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Stream compaction of the flags into an ascending index list.  One CTA of 32 warps; warp w owns
-// the contiguous segment [w*seg, (w+1)*seg).  Pass 1 counts with ballot/popc, a block prefix sum
-// over the 32 warp totals gives each warp its base, pass 2 places the indices.
+// Stream compaction of the flags into an ascending index list.  One CTA of 1024 threads walks the
+// flags in chunks of 16384: a thread reads its 16 consecutive flags with one 16-byte load, a warp scan
+// and a scan over the 32 warp totals give its first position, and it writes its set indices in order.
 __global__ void __launch_bounds__(1024) compact_kernel(const uint8_t* flag, int H, int32_t* idx,
                                                        int32_t* count) {
   __shared__ int warp_total[32];
+  pdl_launch_dependents();
+  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int seg = ((H + 1023) / 1024) * 32;
-  const int lo = warp * seg, hi = min(H, lo + seg);
-  int total = 0;
-  for (int j = lo + lane; j - lane < hi; j += 32) {
-    const bool f = j < hi && flag[j] != 0;
-    total += __popc(__ballot_sync(0xffffffffu, f));
-  }
-  if (lane == 0) warp_total[warp] = total;
-  __syncthreads();
+  const bool vec_ok = (reinterpret_cast<uintptr_t>(flag) & 15u) == 0;
   int base = 0;
-  for (int w = 0; w < warp; ++w) base += warp_total[w];
-  for (int j = lo + lane; j - lane < hi; j += 32) {
-    const bool f = j < hi && flag[j] != 0;
-    const unsigned m = __ballot_sync(0xffffffffu, f);
-    if (f) idx[base + __popc(m & ((1u << lane) - 1u))] = j;
-    base += __popc(m);
+  for (int c0 = 0; c0 < H; c0 += 16384) {
+    const int j0 = c0 + threadIdx.x * 16;
+    uint32_t bits = 0;  // bit q: flag[j0 + q] is set
+    if (vec_ok && j0 + 16 <= H) {
+      const uint4 v = *reinterpret_cast<const uint4*>(flag + j0);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+          if ((w[i] >> (8 * b)) & 0xffu) bits |= 1u << (4 * i + b);
+    } else {
+      for (int q = 0; q < 16; ++q)
+        if (j0 + q < H && flag[j0 + q] != 0) bits |= 1u << q;
+    }
+    const int c = __popc(bits);
+    int incl = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += t;
+    }
+    if (lane == 31) warp_total[warp] = incl;
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < 32; ++w) {
+      const int t = warp_total[w];
+      before += w < warp ? t : 0;
+      total += t;
+    }
+    int pos = base + before + incl - c;
+    while (bits) {
+      const int q = __ffs(bits) - 1;
+      bits &= bits - 1;
+      idx[pos++] = j0 + q;
+    }
+    base += total;
+    __syncthreads();  // warp_total is reused by the next chunk
   }
-  if (threadIdx.x == 1023) *count = base;
+  if (threadIdx.x == 0) *count = base;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -287,6 +313,8 @@ __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
 // y[b][d] = sum_g partial[g][b][d], g ascending.  One thread per four columns.
 __global__ void __launch_bounds__(256) reduce_kernel(const float* partial, int G, int NB, int D,
                                                      float* y, int y_stride) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int q = blockIdx.x * blockDim.x + threadIdx.x;  // float4 index within [NB][D/4]
   const int per = D / 4;
   if (q >= NB * per) return;
@@ -349,8 +377,7 @@ cudaError_t launch_rmsnorm(const float* v, float* n, const float* gain, int r, i
 }
 
 cudaError_t launch_compact(const uint8_t* flag, int H, int32_t* idx, int32_t* count, cudaStream_t s) {
-  compact_kernel<<<1, 1024, 0, s>>>(flag, H, idx, count);
-  return cudaGetLastError();
+  return launch_pdl(compact_kernel, dim3(1), dim3(1024), 0, s, flag, H, idx, count);
 }
 
 template <typename T, int NB, int CPT>
@@ -387,8 +414,7 @@ cudaError_t launch_updown(bool bf16, int nb, const UpDownParams& p, int grid, cu
 cudaError_t launch_reduce(const float* partial, int G, int NB, int D, float* y, int y_stride,
                           cudaStream_t s) {
   const int total = NB * (D / 4);
-  reduce_kernel<<<(total + 255) / 256, 256, 0, s>>>(partial, G, NB, D, y, y_stride);
-  return cudaGetLastError();
+  return launch_pdl(reduce_kernel, dim3((total + 255) / 256), dim3(256), 0, s, partial, G, NB, D, y, y_stride);
 }
 
 }  // namespace sffn

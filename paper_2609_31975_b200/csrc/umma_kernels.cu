@@ -170,6 +170,10 @@ __host__ __device__ inline int tile_rows_for(int n_rows, int grid) {
   return t < 8 ? 8 : t > kTileRows ? kTileRows : t;
 }
 
+__host__ __device__ inline uint32_t tmem_cols_for(int cols) {
+  return cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
+}
+
 template <bool UP>
 __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRowsParams p,
                                                                   const __grid_constant__ CUtensorMap map_w,
@@ -188,10 +192,32 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kblocks = p.K / kAtomK;
+
+  // Set-up that needs nothing from earlier kernels runs while the predecessor in the stream finishes.
+  pdl_launch_dependents();
+  const uint32_t tmem_cols = tmem_cols_for(p.issuers * npad);
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full + 8 * s, 1);  // the producer's expect_tx arrive; the copies complete the bytes
+      mbar_init(empty + 8 * s, 1);
+    }
+    mbar_init(acc_empty, 128);
+    *abort_flag = 0;
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  pdl_wait();
+
   const int n_rows = p.count ? *p.count : p.R;
   const int tile_rows = tile_rows_for(n_rows, gridDim.x);
   const int n_tiles = (n_rows + tile_rows - 1) / tile_rows;
-  const int kblocks = p.K / kAtomK;
   // A stage holds `atoms` successive K blocks of the tile: short tiles (few rows) take several, so that a
   // stage stays near 16 KB and the bytes in flight do not shrink with the tile.  Block a of a stage sits
   // tile_rows * 128 bytes after block a - 1; the MMA of a block reads 128 rows from its start, i.e. on
@@ -204,26 +230,9 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   // (npad TMEM columns each); the epilogue adds them.  A tile with at least as many stages as issuers
   // gives each issuer a stage; shorter tiles use fewer issuers.
   const int nacc = kstages >= p.issuers ? p.issuers : kstages >= 2 ? 2 : 1;
-  const int acc_cols = nacc * npad;
-  const uint32_t tmem_cols = acc_cols <= 32 ? 32 : acc_cols <= 64 ? 64 : acc_cols <= 128 ? 128 : acc_cols <= 256 ? 256 : 512;
-
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(full + 8 * s, 1);  // the producer's expect_tx arrive; the copies complete the bytes
-      mbar_init(empty + 8 * s, 1);
-    }
     mbar_init(acc_full, nacc);
-    mbar_init(acc_empty, 128);
-    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
-  }
-  if (warp == 8) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(tmem_cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -424,27 +433,18 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_rows = p.count ? *p.count : p.R;
   const int d_tiles = p.D / kTileRows;
   const int dt = blockIdx.x % d_tiles, sp = blockIdx.x / d_tiles;
   const int d0 = dt * kTileRows;
-  // the split's share of the list, in blocks of 64 rows
-  const int total_blocks = (n_rows + kAtomK - 1) / kAtomK;
-  const int per_split = (total_blocks + p.splits - 1) / p.splits;
-  const int kb0 = sp * per_split;
-  const int kblocks = min(total_blocks, kb0 + per_split) - kb0;  // <= 0: nothing to add, the partial is zero
-  const int nacc = kblocks >= 2 ? 2 : 1;
-  const int acc_cols = nacc * npad;
-  const uint32_t tmem_cols = acc_cols <= 32 ? 32 : acc_cols <= 64 ? 64 : acc_cols <= 128 ? 128 : 256;
 
+  pdl_launch_dependents();
+  const uint32_t tmem_cols = tmem_cols_for(2 * npad);
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(full + 8 * s, 1);
       mbar_init(empty + 8 * s, 1);
     }
-    mbar_init(acc_full, nacc);
     *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(p.idx ? &map_wg : &map_wt) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hm) : "memory");
   }
@@ -453,6 +453,19 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
                  "r"(tmem_cols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  pdl_wait();
+
+  const int n_rows = p.count ? *p.count : p.R;
+  // the split's share of the list, in blocks of 64 rows
+  const int total_blocks = (n_rows + kAtomK - 1) / kAtomK;
+  const int per_split = (total_blocks + p.splits - 1) / p.splits;
+  const int kb0 = sp * per_split;
+  const int kblocks = min(total_blocks, kb0 + per_split) - kb0;  // <= 0: nothing to add, the partial is zero
+  const int nacc = kblocks >= 2 ? 2 : 1;
+  if (tid == 0) {
+    mbar_init(acc_full, nacc);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -636,7 +649,7 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
       if (e != cudaSuccess) return e;
       configured[1] = true;
     }
-    k<<<grid, kThreadsRows, smem, s>>>(p, map_w, map_x);
+    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x);
   } else {
     auto k = umma_rows_kernel<false>;
     if (!configured[0]) {
@@ -644,9 +657,8 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
       if (e != cudaSuccess) return e;
       configured[0] = true;
     }
-    k<<<grid, kThreadsRows, smem, s>>>(p, map_w, map_x);
+    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x);
   }
-  return cudaGetLastError();
 }
 
 int umma_down_splits(int D, int sm_count, int max_splits) {
@@ -679,8 +691,7 @@ cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  umma_down_kernel<<<grid, kThreads, smem, s>>>(p, map_wg, map_wt, map_hm);
-  return cudaGetLastError();
+  return launch_pdl(umma_down_kernel, dim3(grid), dim3(kThreads), smem, s, p, map_wg, map_wt, map_hm);
 }
 
 cudaError_t launch_split_interleaved(const float* n, int B, int r, int n_stride, void* x2, cudaStream_t s) {
