@@ -272,9 +272,13 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     }
     ++h->launches;
   }
+  // the tcgen05 up-projection compacts the flags itself (and publishes list and length)
+  const bool own_list = umma && !dense && umma_own_list_supported(H, h->sm_count);
   if (!dense) {
-    SFFN_CUDA(launch_compact(flag, H, idx, count, s));
-    ++h->launches;
+    if (!own_list) {
+      SFFN_CUDA(launch_compact(flag, H, idx, count, s));
+      ++h->launches;
+    }
     h->list_state = 1;
   }
   int splits = h->sm_count / (D / 256);
@@ -287,7 +291,12 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     const int32_t* lcount = dense ? nullptr : count;
     if (umma) {
       UmmaRowsParams p{};
-      p.W = W_up; p.R = H; p.K = D; p.idx = lidx; p.count = lcount;
+      p.W = W_up; p.R = H; p.K = D;
+      if (own_list) {
+        p.flag_in = flag; p.idx_out = idx; p.count_out = count;
+      } else {
+        p.idx = lidx; p.count = lcount;
+      }
       p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
       p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
       p.hmT = hmT; p.hm_stride = h->L.hm_stride; p.status = h->at<int32_t>(h->L.status);

@@ -38,6 +38,9 @@ constexpr int kAAtomBytes = kTileRows * 128;         // 16 KB: one [128 rows x 6
 constexpr int kThreads = 320;                        // 4 producer warps, 4 epilogue warps, 2 MMA warps
 constexpr int kThreadsRows = 384;                    // rows kernels: up to 4 MMA warps
 constexpr int kProducerWarps = 4;
+constexpr int kScanChunks = 8;                       // in-kernel compaction: up to 8 * 16 * 384 = 49152 flags
+constexpr int kMaxOwnTiles = 8;                      // tiles of one CTA whose rows are kept in shared memory
+constexpr int kHeaderBytes = 1024 + kMaxOwnTiles * kTileRows * 4;  // barriers + scratch, then the row lists
 constexpr long long kWaitCycles = 1LL << 31;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -184,8 +187,12 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   const int stage_bytes = kAAtomBytes + p.atoms_max * npad * 128;
   const int S = p.stages;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem);  // barriers first: the stages end with a read-over pad
-  const uint32_t stage0 = smem_u32(smem) + 1024;
+  // header: barriers and control words, scan scratch, this CTA's rows of the union list; then the stages
+  // (which end with a read-over pad)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
+  int* scan_wt = reinterpret_cast<int*>(smem + 512);   // [kScanChunks][warps]
+  int* rows_sm = reinterpret_cast<int*>(smem + 1024);  // [kMaxOwnTiles][128]
+  const uint32_t stage0 = smem_u32(smem) + kHeaderBytes;
   const uint32_t full = smem_u32(bars), empty = smem_u32(bars + S);
   const uint32_t acc_full = smem_u32(bars + 2 * S), acc_empty = smem_u32(bars + 2 * S + 1);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
@@ -215,9 +222,97 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   }
   pdl_wait();
 
-  const int n_rows = p.count ? *p.count : p.R;
+  // Union rows: either the list is given (idx, count), or every CTA compacts the "fired" flags of the
+  // gate itself: thread t reads 16 consecutive flags of each chunk of 16 * threads flags with one load,
+  // a warp scan plus the warp totals of all chunks give the position of its first set flag.
+  const bool own_list = UP && p.flag_in != nullptr;
+  uint32_t bits[kScanChunks];
+  int first_pos[kScanChunks];
+  int n_rows;
+  if (own_list) {
+    const int nch = (p.R + 16 * kThreadsRows - 1) / (16 * kThreadsRows);
+#pragma unroll
+    for (int k = 0; k < kScanChunks; ++k) {
+      bits[k] = 0;
+      if (k < nch) {
+        const int j0 = (k * kThreadsRows + tid) * 16;
+        if (j0 + 16 <= p.R) {
+          const uint4 v = *reinterpret_cast<const uint4*>(p.flag_in + j0);
+          const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+              if ((w[i] >> (8 * b)) & 0xffu) bits[k] |= 1u << (4 * i + b);
+        } else {
+          for (int q = 0; q < 16; ++q)
+            if (j0 + q < p.R && p.flag_in[j0 + q] != 0) bits[k] |= 1u << q;
+        }
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < kScanChunks; ++k) {
+      if (k < nch) {
+        int incl = __popc(bits[k]);
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, incl, d);
+          if (lane >= d) incl += t;
+        }
+        first_pos[k] = incl - __popc(bits[k]);
+        if (lane == 31) scan_wt[k * (kThreadsRows / 32) + warp] = incl;
+      }
+    }
+    __syncthreads();
+    int run = 0;
+#pragma unroll
+    for (int k = 0; k < kScanChunks; ++k) {
+      if (k < nch) {
+        int before = 0, total = 0;
+        for (int w = 0; w < kThreadsRows / 32; ++w) {
+          const int t = scan_wt[k * (kThreadsRows / 32) + w];
+          before += w < warp ? t : 0;
+          total += t;
+        }
+        first_pos[k] += run + before;
+        run += total;
+      }
+    }
+    n_rows = run;
+  } else {
+    n_rows = p.count ? *p.count : p.R;
+  }
   const int tile_rows = tile_rows_for(n_rows, gridDim.x);
   const int n_tiles = (n_rows + tile_rows - 1) / tile_rows;
+  if (own_list) {
+    // keep the rows of this CTA's tiles in shared memory and publish them (and the length) for the
+    // down projection and the caller: every list position belongs to exactly one CTA's tile
+    const int nch = (p.R + 16 * kThreadsRows - 1) / (16 * kThreadsRows);
+#pragma unroll
+    for (int k = 0; k < kScanChunks; ++k) {
+      if (k < nch && bits[k]) {
+        const int cnt = __popc(bits[k]);
+        const int j0 = (k * kThreadsRows + tid) * 16;
+        int m = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++m) {
+          const int lo = tile * tile_rows, hi = lo + tile_rows;
+          if (first_pos[k] + cnt <= lo || first_pos[k] >= hi) continue;
+          uint32_t rest = bits[k];
+          int li = first_pos[k];
+          while (rest) {
+            const int q = __ffs(rest) - 1;
+            rest &= rest - 1;
+            if (li >= lo && li < hi) {
+              rows_sm[m * kTileRows + li - lo] = j0 + q;
+              p.idx_out[li] = j0 + q;
+            }
+            ++li;
+          }
+        }
+      }
+    }
+    if (blockIdx.x == 0 && tid == 0) *p.count_out = n_rows;
+  }
   // A stage holds `atoms` successive K blocks of the tile: short tiles (few rows) take several, so that a
   // stage stays near 16 KB and the bytes in flight do not shrink with the tile.  Block a of a stage sits
   // tile_rows * 128 bytes after block a - 1; the MMA of a block reads 128 rows from its start, i.e. on
@@ -248,7 +343,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     // count, then the copies go out: one tiled copy for the tile's consecutive rows (gate), or one
     // gather4 per lane for four listed rows each (union rows); the token block is one more tiled copy.
     int s = 0, ph = 0, kb = 0, tile = blockIdx.x;   // kb counts stages of the tile here
-    int rows_of = -1;
+    int rows_of = -1, own = -1;   // own: index of the current tile among this CTA's tiles
     int r[4] = {0, 0, 0, 0};
     for (; tile < n_tiles; ++s, ++kb) {
       if (s == S) { s = 0; ph ^= 1; }
@@ -262,10 +357,12 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       const uint32_t tx_bytes = (uint32_t)(na * (tile_rows + npad)) * 128;
       if (UP && tile != rows_of) {
         rows_of = tile;
+        ++own;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const int li = tile * tile_rows + lane * 4 + q;
-          r[q] = li < n_rows ? (p.idx ? p.idx[li] : li) : 0;  // rows beyond the list: any valid row, ignored later
+          // rows beyond the list: any valid row, ignored later
+          r[q] = li >= n_rows ? 0 : own_list ? rows_sm[own * kTileRows + lane * 4 + q] : p.idx ? p.idx[li] : li;
         }
       }
       int ok = 1;
@@ -337,7 +434,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
       const int li = tile * tile_rows + row_in_tile;
       const bool row_ok = row_in_tile < tile_rows && li < n_rows;
-      const int j = row_ok ? (p.idx ? p.idx[li] : li) : 0;
+      const int j = !row_ok ? 0 : own_list ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
       // everything that does not depend on the accumulator is fetched before the wait
       float pre[16];
       float bias = 0.f, sg = 1.f;
@@ -580,6 +677,10 @@ __global__ void split_interleaved_kernel(const float* n, int r, int n_stride, __
 
 void debug_set_umma_atoms(int) {}
 
+bool umma_own_list_supported(int R, int sm_count) {
+  return R <= kScanChunks * 16 * kThreadsRows && R <= (long long)kMaxOwnTiles * kTileRows * sm_count;
+}
+
 bool umma_rows_supported(int K, int cols) { return K % kAtomK == 0 && K >= kAtomK && cols >= 1 && cols <= 128; }
 
 namespace {
@@ -628,14 +729,14 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
   // 1 KB of barriers in front; with several blocks per stage, 16 KB behind the last stage that the MMAs
   // of the later blocks may read over
   const int pad = p.atoms_max > 1 ? kAAtomBytes : 0;
-  int stages = (224 * 1024 - 1024 - 1024 - pad) / stage_bytes;
+  int stages = (224 * 1024 - 1024 - kHeaderBytes - pad) / stage_bytes;
   if (stages > 12) stages = 12;
   // four issuers when each can own two or more slots, otherwise two; slots divide evenly among them
   p.issuers = stages >= 8 ? 4 : 2;
   stages &= ~(p.issuers - 1);
   if (stages < 2) return cudaErrorInvalidValue;
   p.stages = stages;
-  const size_t smem = 1024 + 1024 + (size_t)stages * stage_bytes + pad;
+  const size_t smem = 1024 + kHeaderBytes + (size_t)stages * stage_bytes + pad;
   alignas(64) CUtensorMap map_w, map_x;
   // weights: all R rows; boxes of one tile's rows for the gate, single-row boxes for the gather
   if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : tile_rows_for(p.R, grid))) return cudaErrorNotSupported;

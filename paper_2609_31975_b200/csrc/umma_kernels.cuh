@@ -11,6 +11,9 @@ struct UmmaRowsParams {
   int R, K;
   const int32_t* idx;    // UP: list of rows, or null
   const int32_t* count;  // UP: device length of the list, or null (= R)
+  const uint8_t* flag_in;  // UP, instead of idx / count: [R] "fired" flags; the kernel compacts them itself ...
+  int32_t* idx_out;        // ... and writes the ascending list
+  int32_t* count_out;      // ... and its length
   const void* X;         // token operand [cols][K] bf16, row stride x_stride (elements)
   int x_stride;
   int ncols_valid;
@@ -51,6 +54,7 @@ int umma_down_splits(int D, int sm_count, int max_splits);
 bool umma_down_supported(int D, int cols);
 cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s);
 bool umma_rows_supported(int K, int cols);
+bool umma_own_list_supported(int R, int sm_count);
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s);
 cudaError_t launch_split_interleaved(const float* n, int B, int r, int n_stride, void* x2, cudaStream_t s);
 
