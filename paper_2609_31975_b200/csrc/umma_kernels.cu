@@ -78,6 +78,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -334,6 +337,94 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // Epilogue of one tile for the token-column groups c0 = 8 * part, 8 * (part + nparts), ...: waits for the
+  // tile's accumulators, then (gate) adds the fixed-matrix term and the bias, applies the activation and
+  // stores the gate values, reporting whether any token fired; (union rows) scales by the gate values
+  // and stores HmT.  Returns false if the wait was abandoned.
+  const bool share_last = npad >= 32;  // four or more column groups: worth spreading over all warps
+  auto epilogue = [&](int tile, int tcount, int part, int nparts, bool& fired) -> bool {
+    const int row_in_tile = (warp & 3) * 32 + lane;   // TMEM lane of this thread
+    const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const int B = p.B;
+    const int li = tile * tile_rows + row_in_tile;
+    const bool row_ok = row_in_tile < tile_rows && li < n_rows;
+    const int j = !row_ok ? 0 : own_list ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
+    // everything that does not depend on the accumulator is fetched before the wait
+    float bias = 0.f, sg = 1.f;
+    int gi = -1;
+    float pre[16];  // union rows: the gate values of this thread's first two column groups
+    if (UP) {
+#pragma unroll
+      for (int g = 0; g < 2; ++g)
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const int b = 8 * (part + g * nparts) + q;
+          pre[8 * g + q] = (row_ok && b < B) ? p.a[(size_t)b * p.a_stride + j] : 0.f;
+        }
+    } else {
+      bias = (row_ok && p.b_g) ? p.b_g[j] : 0.f;
+      gi = (row_ok && p.g_idx) ? p.g_idx[j] : -1;
+      sg = (row_ok && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
+    }
+    int okw = 1;
+    if (lane == 0) okw = mbar_wait(acc_full, tcount & 1, abort_flag, p.status) ? 1 : 0;
+    okw = __shfl_sync(0xffffffffu, okw, 0);
+    if (!okw) return false;
+    tc_fence_after();
+    if (UP) {
+      __nv_bfloat16* hm = static_cast<__nv_bfloat16*>(p.hmT) + li;
+      const float* arow = p.a + j;
+      int g = 0;
+      for (int c0 = 8 * part; c0 < npad; c0 += 8 * nparts, ++g) {
+        float av[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          av[q] = g == 0 ? pre[q] : g == 1 ? pre[8 + q] : (row_ok && c0 + q < B) ? arow[(size_t)(c0 + q) * p.a_stride] : 0.f;
+        float v[8];
+        tmem_ld8(taddr + c0, nacc, npad, v);
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          if (row_ok && c0 + q < B) hm[(size_t)(c0 + q) * p.hm_stride] = __float2bfloat16(av[q] * v[q]);
+      }
+    } else {
+      const int act = p.act;
+      float* arow = p.a_out + j;
+      const __nv_bfloat16* xg = static_cast<const __nv_bfloat16*>(p.xtok) + (gi >= 0 ? gi : 0);
+      if (p.split_cols) {
+        for (int c0 = 8 * part; c0 < npad; c0 += 8 * nparts) {
+          float v[8];
+          tmem_ld8(taddr + c0, nacc, npad, v);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int b = c0 / 2 + q;
+            if (row_ok && b < B) {
+              float z = v[2 * q] + v[2 * q + 1] + bias;
+              if (gi >= 0) z += sg * __bfloat162float(xg[(size_t)b * p.xtok_stride]);
+              fired |= z > 0.f;
+              arow[(size_t)b * p.a_stride] = activation(act, z);
+            }
+          }
+        }
+      } else {
+        for (int c0 = 8 * part; c0 < npad; c0 += 8 * nparts) {
+          float v[8];
+          tmem_ld8(taddr + c0, nacc, npad, v);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int b = c0 + q;
+            if (row_ok && b < B) {
+              float z = v[q] + bias;
+              if (gi >= 0) z += sg * __bfloat162float(xg[(size_t)b * p.xtok_stride]);
+              fired |= z > 0.f;
+              arow[(size_t)b * p.a_stride] = activation(act, z);
+            }
+          }
+        }
+      }
+    }
+    return true;
+  };
+
   if (warp < kProducerWarps) {
     // ======================= producers =========================================================
     // Stages are numbered it = 0, 1, ... over this CTA's (tile, K block) sequence and use ring slot
@@ -418,82 +509,43 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     }
     __syncwarp();
   } else {
-    // ======================= epilogue ==========================================================
-    const int ew = warp - 4;                 // TMEM lanes 32*ew .. 32*ew + 31
-    const int row_in_tile = ew * 32 + lane;
-    const int B = p.B;
-    const uint32_t taddr = tmem_base + ((uint32_t)(ew * 32) << 16);
+    // ======================= epilogue warps (wide batches: every tile but the CTA's last) =========
     if (UP && blockIdx.x == 0) {
       // the down projection walks the list in blocks of 64 rows: entries past its end must read as zero
       __nv_bfloat16* hm = static_cast<__nv_bfloat16*>(p.hmT);
       const int end = (n_rows + 63) & ~63;
-      for (int li = n_rows + row_in_tile; li < end; li += 128)
-        for (int b = 0; b < B; ++b) hm[(size_t)b * p.hm_stride + li] = __float2bfloat16(0.f);
+      for (int li = n_rows + (warp - 4) * 32 + lane; li < end; li += 128)
+        for (int b = 0; b < p.B; ++b) hm[(size_t)b * p.hm_stride + li] = __float2bfloat16(0.f);
     }
     int tcount = 0;
-    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
+    for (int tile = blockIdx.x; tile + (share_last ? (int)gridDim.x : 0) < n_tiles; tile += gridDim.x, ++tcount) {
+      bool fired = false;
+      if (!epilogue(tile, tcount, 0, 1, fired)) break;
+      const int row_in_tile = (warp - 4) * 32 + lane;
       const int li = tile * tile_rows + row_in_tile;
-      const bool row_ok = row_in_tile < tile_rows && li < n_rows;
-      const int j = !row_ok ? 0 : own_list ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
-      // everything that does not depend on the accumulator is fetched before the wait
-      float pre[16];
-      float bias = 0.f, sg = 1.f;
-      int gi = -1;
-      if (UP) {
-#pragma unroll
-        for (int q = 0; q < 16; ++q) pre[q] = (row_ok && q < B) ? p.a[(size_t)q * p.a_stride + j] : 0.f;
-      } else {
-        bias = (row_ok && p.b_g) ? p.b_g[j] : 0.f;
-        gi = (row_ok && p.g_idx) ? p.g_idx[j] : -1;
-        sg = (row_ok && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
-      }
-      int okw = 1;
-      if (lane == 0) okw = mbar_wait(acc_full, tcount & 1, abort_flag, p.status) ? 1 : 0;
-      okw = __shfl_sync(0xffffffffu, okw, 0);
-      if (!okw) break;
-      tc_fence_after();
-      if (UP) {
-        __nv_bfloat16* hm = static_cast<__nv_bfloat16*>(p.hmT);
-        for (int c0 = 0; c0 < npad; c0 += 8) {
-          float av[8];
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const int b = c0 + q;
-            av[q] = c0 == 0 ? pre[q] : c0 == 8 ? pre[8 + q] : ((row_ok && b < B) ? p.a[(size_t)b * p.a_stride + j] : 0.f);
-          }
-          float v[8];
-          tmem_ld8(taddr + c0, nacc, npad, v);
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const int b = c0 + q;
-            if (row_ok && b < B) hm[(size_t)b * p.hm_stride + li] = __float2bfloat16(av[q] * v[q]);
-          }
-        }
-      } else {
-        bool fired = false;
-        for (int c0 = 0; c0 < npad; c0 += 8) {
-          float v[8];
-          tmem_ld8(taddr + c0, nacc, npad, v);
-          const int per = p.split_cols ? 4 : 8;  // tokens covered by these eight columns
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            if (q < per) {
-              const int b = (p.split_cols ? c0 / 2 : c0) + q;
-              if (row_ok && b < B) {
-                float z = p.split_cols ? v[2 * q] + v[2 * q + 1] : v[q];
-                if (gi >= 0)
-                  z += sg * __bfloat162float(static_cast<const __nv_bfloat16*>(p.xtok)[(size_t)b * p.xtok_stride + gi]);
-                z += bias;
-                fired |= z > 0.f;
-                p.a_out[(size_t)b * p.a_stride + j] = activation(p.act, z);
-              }
-            }
-          }
-        }
-        if (row_ok && p.flag) p.flag[j] = fired ? 1 : 0;
-      }
+      if (!UP && p.flag && row_in_tile < tile_rows && li < n_rows) p.flag[li] = fired ? 1 : 0;
       tc_fence_before();
       mbar_arrive(acc_empty);
+    }
+  }
+
+  // ---- the CTA's last tile (wide batches): by now the producer and issuer warps have nothing left to do, so
+  // all twelve warps share its epilogue.  A warp reads the TMEM lanes of its quarter (warp mod 4); the three warps of
+  // a quarter take every third group of eight token columns.
+  if (share_last && (int)blockIdx.x < n_tiles) {
+    const int my_tiles = (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
+    const int last_tile = blockIdx.x + (my_tiles - 1) * gridDim.x;
+    const int part = warp >= 8 ? 2 : warp >= 4 ? 0 : 1;
+    bool fired = false;
+    const bool done = epilogue(last_tile, my_tiles - 1, part, 3, fired);
+    if (!UP && p.flag) {
+      uint8_t* fired_sm = reinterpret_cast<uint8_t*>(scan_wt);  // [3][128], the scan scratch is free here
+      const int row_in_tile = (warp & 3) * 32 + lane;
+      fired_sm[part * kTileRows + row_in_tile] = fired ? 1 : 0;
+      named_bar_sync(2, kThreadsRows);  // reached by every thread of a CTA that owns a tile, whatever happened
+      const int li = last_tile * tile_rows + row_in_tile;
+      if (part == 0 && done && row_in_tile < tile_rows && li < n_rows)
+        p.flag[li] = fired_sm[row_in_tile] | fired_sm[kTileRows + row_in_tile] | fired_sm[2 * kTileRows + row_in_tile];
     }
   }
 
