@@ -211,7 +211,18 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
   const bool lopa = g->kind == SFFN_GATE_LOPA;
   const int grid_rows = 2 * h->sm_count;
 
-  if (lopa) {  // v = V x on the CUDA-core row kernel (r rows only), then RMSNorm
+  if (lopa && umma) {  // v = V x on the tensor cores: the rows kernel with the identity as its epilogue
+    for (int b0 = 0; b0 < B; b0 += kMaxMmaTokens) {
+      const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
+      UmmaRowsParams p{};
+      p.W = g->V; p.R = g->r; p.K = D;
+      p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
+      p.act = kUmmaActIdentity; p.a_out = vbuf + (size_t)b0 * rs; p.a_stride = rs;
+      p.status = h->at<int32_t>(h->L.status);
+      SFFN_CUDA(launch_umma_rows(false, p, nb, h->sm_count, s));
+      ++h->launches;
+    }
+  } else if (lopa) {  // v = V x on the CUDA-core row kernel (r rows only), then RMSNorm
     for (int b0 = 0; b0 < B;) {
       const int nb = B - b0 >= 4 ? 4 : B - b0 >= 2 ? 2 : 1;
       RowDotParams p{};
@@ -241,7 +252,9 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       p.flag = dense ? nullptr : flag;
       int cols = nb;
       if (lopa) {
-        SFFN_CUDA(launch_split_interleaved(nsrc, nb, g->r, rs, x2, s));
+        // RMSNorm (or none) and the split into bf16 pairs in one launch
+        SFFN_CUDA(launch_rmsnorm_split(vbuf + (size_t)b0 * rs, nb, g->r, rs, g->rms_gain, g->rms_eps,
+                                       g->use_rmsnorm != 0, x2, s));
         ++h->launches;
         p.W = g->U; p.K = g->r; p.X = x2; p.x_stride = g->r; p.split_cols = 1;
         p.g_idx = g->g_idx; p.g_sign = g->g_sign;

@@ -10,10 +10,12 @@ namespace sffn {
 constexpr int kActRelu = 0;
 constexpr int kActSqRelu = 1;
 constexpr int kActRsPlus = 2;
+constexpr int kActNone = 3;  // identity: internal stages that only need the raw products
 
 // Activation of the gate (activation table of Sec. 3.1; squared RELU from the activation study).
 // For all three, A(z) != 0 exactly when z > 0 in exact arithmetic; callers test z > 0.
 __device__ __forceinline__ float activation(int act, float z) {
+  if (act == kActNone) return z;
   if (!(z > 0.f)) return 0.f;
   if (act == kActRelu) return z;
   if (act == kActSqRelu) return z * z;

@@ -30,6 +30,8 @@
 
 namespace sffn {
 
+static_assert(kUmmaActIdentity == kActNone, "identity epilogue code");
+
 namespace {
 
 constexpr int kTileRows = 128;
@@ -714,15 +716,34 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
   }
 }
 
-// n (fp32, [B][r]) -> bf16 pairs: row 2b holds the high parts of token b, row 2b+1 the low parts.
-__global__ void split_interleaved_kernel(const float* n, int r, int n_stride, __nv_bfloat16* x2) {
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  const int b = blockIdx.y;
-  if (k >= r) return;
-  const float v = n[(size_t)b * n_stride + k];
-  const __nv_bfloat16 hi = __float2bfloat16(v);
-  x2[(size_t)(2 * b) * r + k] = hi;
-  x2[(size_t)(2 * b + 1) * r + k] = __float2bfloat16(v - __bfloat162float(hi));
+// LoPA gate, batched: n = RMSNorm(v) (or v itself), written as bf16 pairs for the tensor cores: row 2b of
+// x2 holds the high parts of token b's vector, row 2b+1 the low parts (v - bf16(v)), so that the gate's
+// U n keeps close to fp32 accuracy.  One CTA per token.
+__global__ void __launch_bounds__(256) rmsnorm_split_kernel(const float* v, int r, int v_stride, const float* gain,
+                                                            float eps, int use_rms, __nv_bfloat16* x2) {
+  __shared__ float red[8];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.x;
+  const float* vb = v + (size_t)b * v_stride;
+  float inv = 1.f;
+  if (use_rms) {
+    float ss = 0.f;
+    for (int k = threadIdx.x; k < r; k += blockDim.x) ss = fmaf(vb[k], vb[k], ss);
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    inv = rsqrtf(tot / (float)r + eps);
+  }
+  for (int k = threadIdx.x; k < r; k += blockDim.x) {
+    const float n = use_rms ? (gain ? gain[k] : 1.f) * vb[k] * inv : vb[k];
+    const __nv_bfloat16 hi = __float2bfloat16(n);
+    x2[(size_t)(2 * b) * r + k] = hi;
+    x2[(size_t)(2 * b + 1) * r + k] = __float2bfloat16(n - __bfloat162float(hi));
+  }
 }
 
 }  // namespace
@@ -847,9 +868,10 @@ cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s) {
   return launch_pdl(umma_down_kernel, dim3(grid), dim3(kThreads), smem, s, p, map_wg, map_wt, map_hm);
 }
 
-cudaError_t launch_split_interleaved(const float* n, int B, int r, int n_stride, void* x2, cudaStream_t s) {
-  split_interleaved_kernel<<<dim3((r + 255) / 256, B), 256, 0, s>>>(n, r, n_stride, static_cast<__nv_bfloat16*>(x2));
-  return cudaGetLastError();
+cudaError_t launch_rmsnorm_split(const float* v, int B, int r, int v_stride, const float* gain, float eps,
+                                 bool use_rms, void* x2, cudaStream_t s) {
+  return launch_pdl(rmsnorm_split_kernel, dim3(B), dim3(256), 0, s, v, r, v_stride, gain, eps, use_rms ? 1 : 0,
+                    static_cast<__nv_bfloat16*>(x2));
 }
 
 }  // namespace sffn

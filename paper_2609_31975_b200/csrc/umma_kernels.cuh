@@ -6,6 +6,9 @@
 
 namespace sffn {
 
+// Value of UmmaRowsParams::act that stores the raw products (no bias is usually given, no activation).
+constexpr int kUmmaActIdentity = 3;
+
 struct UmmaRowsParams {
   const void* W;         // [*, K] bf16, rows selected by idx (or 0..R-1)
   int R, K;
@@ -56,6 +59,7 @@ cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s);
 bool umma_rows_supported(int K, int cols);
 bool umma_own_list_supported(int R, int sm_count);
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s);
-cudaError_t launch_split_interleaved(const float* n, int B, int r, int n_stride, void* x2, cudaStream_t s);
+cudaError_t launch_rmsnorm_split(const float* v, int B, int r, int v_stride, const float* gain, float eps,
+                                 bool use_rms, void* x2, cudaStream_t s);
 
 }  // namespace sffn
