@@ -662,6 +662,11 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   if (ng > 3 * gw) ng = 3 * gw;
   ng = ng / gw * gw;
   if (ng < gw) return g;
+  // A short gate (LoPA: a CTA's whole share of U may fit in a few slots) needs no deeper ring than its
+  // slot count; what that frees goes to the act ring.
+  const int slots_of_cta = (g.slab_max + nr - 1) / nr;
+  const int enough = (slots_of_cta + gw - 1) / gw * gw;
+  if (ng > enough) ng = enough;
   na = (ring - ng * g.gate_slot_bytes) / g.act_slot_bytes;
   if (na > 16) na = 16;
   if (na < 2) return g;
