@@ -211,6 +211,47 @@ def test_host_entry_and_errors(mod):
         mod.SparseFFN(260, 64, torch.bfloat16)
 
 
+@pytest.mark.parametrize("D,H,B,s", [
+    (256, 20000, 8, 0.2),    # union = every row: more than 128 rows x 148 CTAs, several tiles per CTA
+    (256, 50048, 4, 0.9),    # more flags than the in-kernel compaction takes: separate compaction launch
+    (256, 777, 3, 0.9),      # H not a multiple of 8: ragged last tile, byte-wise flag reads
+    (512, 1500, 33, 0.95),   # 33 tokens: 48 token columns, three column groups shared by all warps
+    (256, 64, 2, 0.5),       # fewer rows than one tile of eight per CTA
+])
+def test_batched_tcgen05_edge_shapes(mod, D, H, B, s):
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=B)
+    gate, w = make_std(D, H, torch.bfloat16, 43, s)
+    x = syn.tokens(B, D, torch.bfloat16, 43, DEV)
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", threads=16)
+    y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
+    assert_y_close(y, ref["y"], what=f"edge {D}x{H} B={B}")
+    assert_active_set(ffn.last_active(), ref, what=f"edge {D}x{H} B={B}")
+    y2 = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert torch.equal(y, y2)
+    yd = ffn.dense_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    dref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", route="dense", threads=16)
+    assert_y_close(yd, dref["y"], what=f"edge dense {D}x{H} B={B}")
+
+
+def test_batched_empty_and_full_union(mod):
+    D, H, B = 256, 1000, 6
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=B)
+    gate, w = make_std(D, H, torch.bfloat16, 44, None)
+    x = syn.tokens(B, D, torch.bfloat16, 44, DEV)
+    lo = torch.full((H,), -1e3, device=DEV)
+    y = ffn.sparse_ffn_forward(x, gate, lo, w["W_up"], w["W_down"], "relu")
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
+    assert not y.any() and ffn.last_active().numel() == 0        # no neuron fires for any token: y == 0 exactly
+    hi = torch.full((H,), 1e3, device=DEV)
+    y = ffn.sparse_ffn_forward(x, gate, hi, w["W_up"], w["W_down"], "relu")
+    assert ffn.last_active().tolist() == list(range(H))           # every neuron fires: the union is every row
+    ref = run_oracle(x, gate, hi, w["W_up"], w["W_down"], "relu", route="dense")
+    assert_y_close(y, ref["y"], what="batched, full union")
+
+
 # ------------------------------------------------------------------ full-size configurations
 def test_config2_full_size_decode(mod):
     D, H = 4096, 14336
