@@ -456,7 +456,27 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
       if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status)) break;
       const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
       float mine = 0.f;
-      for (int rr = 0; rr < rows; ++rr) {
+      // Short gate rows (LoPA: r elements): a row is a few chunks per lane and its cost is the latency of the
+      // warp reduction, so four rows are dotted and reduced side by side.
+      const int rows_short = nvecK <= 128 ? rows : 0;
+      for (int rr = 0; rr < rows_short; rr += 4) {
+        float a[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int c = lane; c < nvecK; c += 32) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            if (rr + i < rows)
+              a[i] = chunk_dot<T>(reinterpret_cast<const uint4*>(base + (size_t)(rr + i) * gate_row_bytes)[c], gvec, c,
+                                  nvecK, a[i]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) a[i] += __shfl_xor_sync(0xffffffffu, a[i], o);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (lane == rr + i) mine = a[i];
+      }
+      for (int rr = rows_short; rr < rows; ++rr) {
         const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr * gate_row_bytes);
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         int c = lane;
