@@ -38,7 +38,7 @@ Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
   };
   L.status = take(256);  // [0] device status, [1] length of idx
   L.act = take((size_t)B_max * H * 4);
-  L.flag = take((size_t)H);
+  L.flag = take((size_t)2 * H + 256);  // bytes [H], or the tcgen05 gate's bit masks (16 bytes per tile of >= 8 rows)
   L.idx = take(((size_t)H + 64) * 4);  // readable one 64-row block past the list
   L.v = take((size_t)B_max * (r_max > 0 ? r_max : 1) * 4);
   L.n = take((size_t)B_max * (r_max > 0 ? r_max : 1) * 4);
@@ -238,6 +238,12 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       ++h->launches;
     }
   }
+  // The tcgen05 gate kernel can leave its "fired" flags as bit masks, which the up kernel compacts itself
+  // (and publishes list and length): no byte flags, no compaction launch.
+  const bool own_list = umma && !dense && umma_own_list_supported(H, h->sm_count);
+  uint32_t* words = reinterpret_cast<uint32_t*>(flag);  // the flag buffer holds either form
+  int gate_tile_rows = 0, gate_tiles = 0;
+  umma_gate_tiling(H, h->sm_count, &gate_tile_rows, &gate_tiles);
   for (int b0 = 0; b0 < B; b0 += kMaxMmaTokens) {
     const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
     void* x2 = h->ws + h->L.x2;
@@ -249,7 +255,8 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       p.R = H; p.B = nb; p.b_g = b_g; p.act = act; p.status = h->at<int32_t>(h->L.status);
       p.xtok = xtok; p.xtok_stride = D;
       p.a_out = actbuf + (size_t)b0 * H; p.a_stride = H;
-      p.flag = dense ? nullptr : flag;
+      p.flag = (dense || own_list) ? nullptr : flag;
+      p.words_out = own_list ? words : nullptr;
       int cols = nb;
       if (lopa) {
         // RMSNorm (or none) and the split into bf16 pairs in one launch
@@ -285,8 +292,6 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     }
     ++h->launches;
   }
-  // the tcgen05 up-projection compacts the flags itself (and publishes list and length)
-  const bool own_list = umma && !dense && umma_own_list_supported(H, h->sm_count);
   if (!dense) {
     if (!own_list) {
       SFFN_CUDA(launch_compact(flag, H, idx, count, s));
@@ -306,7 +311,8 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       UmmaRowsParams p{};
       p.W = W_up; p.R = H; p.K = D;
       if (own_list) {
-        p.flag_in = flag; p.idx_out = idx; p.count_out = count;
+        p.words_in = words; p.n_words = 4 * gate_tiles; p.gate_tile_rows = gate_tile_rows;
+        p.idx_out = idx; p.count_out = count;
       } else {
         p.idx = lidx; p.count = lcount;
       }

@@ -40,7 +40,7 @@ constexpr int kAAtomBytes = kTileRows * 128;         // 16 KB: one [128 rows x 6
 constexpr int kThreads = 320;                        // 4 producer warps, 4 epilogue warps, 2 MMA warps
 constexpr int kThreadsRows = 384;                    // rows kernels: up to 4 MMA warps
 constexpr int kProducerWarps = 4;
-constexpr int kScanChunks = 8;                       // in-kernel compaction: up to 8 * 16 * 384 = 49152 flags
+constexpr int kScanChunks = 4;                       // in-kernel compaction: up to 4 * 384 mask words = 384 gate tiles
 constexpr int kMaxOwnTiles = 8;                      // tiles of one CTA whose rows are kept in shared memory
 constexpr int kHeaderBytes = 1024 + kMaxOwnTiles * kTileRows * 4;  // barriers + scratch, then the row lists
 constexpr long long kWaitCycles = 1LL << 31;
@@ -227,33 +227,20 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   }
   pdl_wait();
 
-  // Union rows: either the list is given (idx, count), or every CTA compacts the "fired" flags of the
-  // gate itself: thread t reads 16 consecutive flags of each chunk of 16 * threads flags with one load,
-  // a warp scan plus the warp totals of all chunks give the position of its first set flag.
-  const bool own_list = UP && p.flag_in != nullptr;
+  // Union rows: either the list is given (idx, count), or every CTA compacts the gate's "fired" bit masks
+  // itself.  The gate kernel leaves one 32-bit word per epilogue warp and tile (word 4 * tile + warp, bit =
+  // lane = row 32 * warp + lane of the tile); thread t takes word t of each chunk of `threads` words, a
+  // warp scan plus the warp totals of all chunks give the list position of its first set bit.
+  const bool own_list = UP && p.words_in != nullptr;
   uint32_t bits[kScanChunks];
   int first_pos[kScanChunks];
   int n_rows;
+  const int nch = own_list ? (p.n_words + kThreadsRows - 1) / kThreadsRows : 0;
   if (own_list) {
-    const int nch = (p.R + 16 * kThreadsRows - 1) / (16 * kThreadsRows);
 #pragma unroll
     for (int k = 0; k < kScanChunks; ++k) {
-      bits[k] = 0;
-      if (k < nch) {
-        const int j0 = (k * kThreadsRows + tid) * 16;
-        if (j0 + 16 <= p.R) {
-          const uint4 v = *reinterpret_cast<const uint4*>(p.flag_in + j0);
-          const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-              if ((w[i] >> (8 * b)) & 0xffu) bits[k] |= 1u << (4 * i + b);
-        } else {
-          for (int q = 0; q < 16; ++q)
-            if (j0 + q < p.R && p.flag_in[j0 + q] != 0) bits[k] |= 1u << q;
-        }
-      }
+      const int w = k * kThreadsRows + tid;
+      bits[k] = (k < nch && w < p.n_words) ? __ldcg(p.words_in + w) : 0u;
     }
 #pragma unroll
     for (int k = 0; k < kScanChunks; ++k) {
@@ -292,12 +279,12 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   if (own_list) {
     // keep the rows of this CTA's tiles in shared memory and publish them (and the length) for the
     // down projection and the caller: every list position belongs to exactly one CTA's tile
-    const int nch = (p.R + 16 * kThreadsRows - 1) / (16 * kThreadsRows);
 #pragma unroll
     for (int k = 0; k < kScanChunks; ++k) {
       if (k < nch && bits[k]) {
         const int cnt = __popc(bits[k]);
-        const int j0 = (k * kThreadsRows + tid) * 16;
+        const int w = k * kThreadsRows + tid;
+        const int j0 = (w >> 2) * p.gate_tile_rows + (w & 3) * 32;  // row of bit 0
         int m = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++m) {
           const int lo = tile * tile_rows, hi = lo + tile_rows;
@@ -525,7 +512,12 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       if (!epilogue(tile, tcount, 0, 1, fired)) break;
       const int row_in_tile = (warp - 4) * 32 + lane;
       const int li = tile * tile_rows + row_in_tile;
-      if (!UP && p.flag && row_in_tile < tile_rows && li < n_rows) p.flag[li] = fired ? 1 : 0;
+      const bool valid = row_in_tile < tile_rows && li < n_rows;
+      if (!UP && p.flag && valid) p.flag[li] = fired ? 1 : 0;
+      if (!UP && p.words_out) {
+        const unsigned m = __ballot_sync(0xffffffffu, fired && valid);
+        if (lane == 0) p.words_out[4 * tile + (warp & 3)] = m;
+      }
       tc_fence_before();
       mbar_arrive(acc_empty);
     }
@@ -540,14 +532,22 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     const int part = warp >= 8 ? 2 : warp >= 4 ? 0 : 1;
     bool fired = false;
     const bool done = epilogue(last_tile, my_tiles - 1, part, 3, fired);
-    if (!UP && p.flag) {
+    if (!UP && (p.flag || p.words_out)) {
       uint8_t* fired_sm = reinterpret_cast<uint8_t*>(scan_wt);  // [3][128], the scan scratch is free here
       const int row_in_tile = (warp & 3) * 32 + lane;
       fired_sm[part * kTileRows + row_in_tile] = fired ? 1 : 0;
       named_bar_sync(2, kThreadsRows);  // reached by every thread of a CTA that owns a tile, whatever happened
       const int li = last_tile * tile_rows + row_in_tile;
-      if (part == 0 && done && row_in_tile < tile_rows && li < n_rows)
-        p.flag[li] = fired_sm[row_in_tile] | fired_sm[kTileRows + row_in_tile] | fired_sm[2 * kTileRows + row_in_tile];
+      if (part == 0) {  // warps 4-7, all lanes
+        const bool valid = done && row_in_tile < tile_rows && li < n_rows;
+        const bool any =
+            (fired_sm[row_in_tile] | fired_sm[kTileRows + row_in_tile] | fired_sm[2 * kTileRows + row_in_tile]) != 0;
+        if (p.flag && valid) p.flag[li] = any ? 1 : 0;
+        if (p.words_out) {
+          const unsigned m = __ballot_sync(0xffffffffu, any && valid);
+          if (lane == 0) p.words_out[4 * last_tile + (warp & 3)] = m;
+        }
+      }
     }
   }
 
@@ -750,8 +750,17 @@ __global__ void __launch_bounds__(256) rmsnorm_split_kernel(const float* v, int 
 
 void debug_set_umma_atoms(int) {}
 
+// Tiling of the gate GEMM over R rows (the up kernel needs it to read the gate's bit masks).
+void umma_gate_tiling(int R, int sm_count, int* tile_rows, int* n_tiles) {
+  const int grid = R < 8 * sm_count ? (R + 7) / 8 : sm_count;
+  *tile_rows = tile_rows_for(R, grid);
+  *n_tiles = (R + *tile_rows - 1) / *tile_rows;
+}
+
 bool umma_own_list_supported(int R, int sm_count) {
-  return R <= kScanChunks * 16 * kThreadsRows && R <= (long long)kMaxOwnTiles * kTileRows * sm_count;
+  int tr, nt;
+  umma_gate_tiling(R, sm_count, &tr, &nt);
+  return 4 * nt <= kScanChunks * kThreadsRows && R <= (long long)kMaxOwnTiles * kTileRows * sm_count;
 }
 
 bool umma_rows_supported(int K, int cols) { return K % kAtomK == 0 && K >= kAtomK && cols >= 1 && cols <= 128; }

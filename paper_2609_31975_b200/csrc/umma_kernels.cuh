@@ -14,9 +14,11 @@ struct UmmaRowsParams {
   int R, K;
   const int32_t* idx;    // UP: list of rows, or null
   const int32_t* count;  // UP: device length of the list, or null (= R)
-  const uint8_t* flag_in;  // UP, instead of idx / count: [R] "fired" flags; the kernel compacts them itself ...
-  int32_t* idx_out;        // ... and writes the ascending list
-  int32_t* count_out;      // ... and its length
+  const uint32_t* words_in;  // UP, instead of idx / count: the gate kernel's "fired" bit masks (n_words of
+  int n_words;               //   them, 4 per gate tile of gate_tile_rows rows); the kernel compacts them itself
+  int gate_tile_rows;
+  int32_t* idx_out;          //   ... and writes the ascending list
+  int32_t* count_out;        //   ... and its length
   const void* X;         // token operand [cols][K] bf16, row stride x_stride (elements)
   int x_stride;
   int ncols_valid;
@@ -30,6 +32,7 @@ struct UmmaRowsParams {
   int act;
   float* a_out;          // GATE: gate values a_out[b * a_stride + j]
   uint8_t* flag;         // GATE: [R] any token fires, or null
+  uint32_t* words_out;   // GATE: the same as bit masks, word 4 * tile + epilogue warp, or null
   const float* a;        // UP: gate values
   int a_stride;
   void* hmT;             // UP: bf16 [B][hm_stride]
@@ -58,6 +61,7 @@ bool umma_down_supported(int D, int cols);
 cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s);
 bool umma_rows_supported(int K, int cols);
 bool umma_own_list_supported(int R, int sm_count);
+void umma_gate_tiling(int R, int sm_count, int* tile_rows, int* n_tiles);
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s);
 cudaError_t launch_rmsnorm_split(const float* v, int B, int r, int v_stride, const float* gain, float eps,
                                  bool use_rms, void* x2, cudaStream_t s);
