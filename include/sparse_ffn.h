@@ -121,9 +121,13 @@ int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate
                       void* stream);
 
 /* End-to-end variant of sparse_ffn_forward for callers whose activations live on the host:
- * x_host [B,D] (handle dtype) and y_host [B,D] fp32 are HOST pointers (pinned memory makes the
- * copies asynchronous); weights stay on the device.  Copies x in, runs the sparse path, copies y
- * out, all on `stream`; y_host is valid once the stream has synchronised. */
+ * x_host [B,D] (handle dtype) and y_host [B,D] fp32 are HOST pointers; weights stay on the device.
+ * Brings x in, runs the sparse path, puts y out, all on `stream`; y_host is valid once the stream has
+ * synchronised.  Pinned host memory (cudaHostAlloc / cudaHostRegister, 16-byte aligned) is accessed by
+ * the kernels directly -- a small copy kernel reads x, the call's last kernel stores y -- so no
+ * copy-engine operation sits between the kernels; any other host memory goes through cudaMemcpyAsync.
+ * x_host must hold its final contents when the call is made: the library may read it before earlier work
+ * on `stream` has finished (as a copy from pageable memory would). */
 int sparse_ffn_forward_host(sffn_handle* handle, const void* x_host, int B, const sffn_gate* gate,
                             const float* b_g, const void* W_up, const void* W_down, int act,
                             float* y_host, void* stream);

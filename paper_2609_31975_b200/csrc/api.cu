@@ -472,6 +472,17 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
   return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, s);
 }
 
+// Device-side alias of a 16-byte aligned pointer into pinned, mapped host memory; null for anything else.
+const void* mapped_device_pointer(const void* host) {
+  if (!host || (reinterpret_cast<uintptr_t>(host) & 15u)) return nullptr;
+  cudaPointerAttributes attr{};
+  if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
+    cudaGetLastError();  // unregistered memory reports an error on some drivers: not ours to keep
+    return nullptr;
+  }
+  return attr.type == cudaMemoryTypeHost ? attr.devicePointer : nullptr;
+}
+
 }  // namespace
 
 extern "C" {
@@ -499,12 +510,23 @@ int sparse_ffn_forward_host(sffn_handle* h, const void* x_host, int B, const sff
   if (!h || !x_host || !y_host || B < 1 || B > h->B_max) return SFFN_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t esz = h->dtype == SFFN_BF16 ? 2 : 4;
-  void* xs = h->ws + h->L.xstage;
   float* ys = h->at<float>(h->L.ystage);
-  SFFN_CUDA(cudaMemcpyAsync(xs, x_host, (size_t)B * h->D * esz, cudaMemcpyHostToDevice, s));
-  const int rc = run(h, xs, B, g, b_g, W_up, W_down, act, ys, false, stream);
+  const size_t xbytes = (size_t)B * h->D * esz, ybytes = (size_t)B * h->D * 4;
+  // Pinned (mapped) host memory is read and written by the kernels themselves: a small copy kernel brings
+  // the tokens in and the last kernel of the call stores y straight to the host, so the stream carries no
+  // copy-engine operation between kernels.  Pageable memory takes the two asynchronous copies.
+  void* xs = h->ws + h->L.xstage;
+  const void* x_map = mapped_device_pointer(x_host);
+  float* y_map = static_cast<float*>(const_cast<void*>(mapped_device_pointer(y_host)));
+  if (x_map) {
+    SFFN_CUDA(sffn::launch_copy16(x_map, xs, xbytes, s));
+    ++h->launches;
+  } else {
+    SFFN_CUDA(cudaMemcpyAsync(xs, x_host, xbytes, cudaMemcpyHostToDevice, s));
+  }
+  const int rc = run(h, xs, B, g, b_g, W_up, W_down, act, y_map ? y_map : ys, false, stream);
   if (rc != SFFN_OK) return rc;
-  SFFN_CUDA(cudaMemcpyAsync(y_host, ys, (size_t)B * h->D * 4, cudaMemcpyDeviceToHost, s));
+  if (!y_map) SFFN_CUDA(cudaMemcpyAsync(y_host, ys, ybytes, cudaMemcpyDeviceToHost, s));
   return SFFN_OK;
 }
 

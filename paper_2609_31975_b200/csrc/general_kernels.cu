@@ -333,6 +333,25 @@ __global__ void __launch_bounds__(256) reduce_kernel(const float* partial, int G
   *reinterpret_cast<float4*>(y + (size_t)b * y_stride + (size_t)d4 * 4) = s;
 }
 
+// Copy of n16 16-byte units from mapped pinned host memory into a staging buffer of the workspace, without a
+// copy-engine operation between two kernels of the stream.  The source is host data that was complete when
+// the call was made, so its first 4 units per thread are read into registers at once, while the predecessors
+// in the stream still run; nothing is written before they have finished.
+__global__ void __launch_bounds__(256) copy16_kernel(const uint4* src, uint4* dst, size_t n16) {
+  pdl_launch_dependents();
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  uint4 v[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    if (i0 + k * stride < n16) v[k] = src[i0 + k * stride];
+  pdl_wait();
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    if (i0 + k * stride < n16) dst[i0 + k * stride] = v[k];
+  for (size_t i = i0 + 4 * stride; i < n16; i += stride) dst[i] = src[i];
+}
+
 // ------------------------------------------------------------------------------------------------
 // Host-side launchers.
 template <typename T, typename VT, int NB>
@@ -409,6 +428,13 @@ int updown_max_tokens(bool bf16, int D) {
 
 cudaError_t launch_updown(bool bf16, int nb, const UpDownParams& p, int grid, cudaStream_t s) {
   return bf16 ? launch_updown_d<__nv_bfloat16>(p, nb, grid, s) : launch_updown_d<float>(p, nb, grid, s);
+}
+
+cudaError_t launch_copy16(const void* src, void* dst, size_t bytes, cudaStream_t s) {
+  const size_t n16 = bytes / 16;
+  const int grid = (int)((n16 + 255) / 256 < 64 ? (n16 + 255) / 256 : 64);
+  return launch_pdl(copy16_kernel, dim3(grid < 1 ? 1 : grid), dim3(256), 0, s, static_cast<const uint4*>(src),
+                    static_cast<uint4*>(dst), n16);
 }
 
 cudaError_t launch_reduce(const float* partial, int G, int NB, int D, float* y, int y_stride,

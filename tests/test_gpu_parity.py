@@ -193,6 +193,14 @@ def test_host_entry_and_errors(mod):
     torch.cuda.synchronize()
     y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
     assert torch.equal(y.cpu(), yh)
+    xp, yp = x.cpu(), torch.full((2, D), float("nan"), dtype=torch.float32)   # pageable memory: copy-engine route
+    ffn.sparse_ffn_forward_host(xp, gate, w["b_g"], w["W_up"], w["W_down"], "relu", yp)
+    torch.cuda.synchronize()
+    assert torch.equal(y.cpu(), yp)
+    yh1 = torch.empty(D, dtype=torch.float32).pin_memory()                       # one token: fused kernels
+    ffn.sparse_ffn_forward_host(xh[1], gate, w["b_g"], w["W_up"], w["W_down"], "relu", yh1)
+    torch.cuda.synchronize()
+    assert torch.equal(ffn.sparse_ffn_forward(x[1], gate, w["b_g"], w["W_up"], w["W_down"], "relu").cpu(), yh1)
     n0 = ffn.launch_count()
     ffn.sparse_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
     assert ffn.launch_count() > n0
