@@ -146,7 +146,6 @@ int sffn_set_path(sffn_handle* h, int path) {
 
 // Experiment knob (not part of the documented ABI).
 void sffn_debug_set_pdl(int on) { sffn::debug_set_pdl(on); }
-void sffn_debug_set_umma_atoms(int atoms) { sffn::debug_set_umma_atoms(atoms); }
 void sffn_debug_set_trace(void* device_buffer) { sffn::debug_set_trace(static_cast<long long*>(device_buffer)); }
 
 int sffn_launch_count(sffn_handle* h, long long* launches) {

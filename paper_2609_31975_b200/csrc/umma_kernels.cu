@@ -748,7 +748,6 @@ __global__ void __launch_bounds__(256) rmsnorm_split_kernel(const float* v, int 
 
 }  // namespace
 
-void debug_set_umma_atoms(int) {}
 
 // Tiling of the gate GEMM over R rows (the up kernel needs it to read the gate's bit masks).
 void umma_gate_tiling(int R, int sm_count, int* tile_rows, int* n_tiles) {

@@ -55,7 +55,6 @@ struct UmmaDownParams {
   int npad, stages;      // filled by the launcher
 };
 
-void debug_set_umma_atoms(int atoms);
 int umma_down_splits(int D, int sm_count, int max_splits);
 bool umma_down_supported(int D, int cols);
 cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s);
