@@ -311,6 +311,16 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
     }
   }
 
+  // LoPA: this CTA's rows of V are weights too; pull them into L2 now so that the rank-r stage, which sits on the
+  // call's critical path right after the wait, finds them there.
+  if (LOPA && warp == kGateProducers) {
+    const int vlo = (int)((long long)K * cta / G), vhi = (int)((long long)K * (cta + 1) / G);
+    for (int k = vlo + lane; k < vhi; k += 32)
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(static_cast<const char*>(p.V) + (size_t)k * row_bytes),
+                   "r"((uint32_t)row_bytes)
+                   : "memory");
+  }
+
   // ---- everyone else: wait for the predecessor in the stream, then stage the token ------------
   pdl_wait();
   if (tid == kStageBase) SFFN_GSTAMP(11);
