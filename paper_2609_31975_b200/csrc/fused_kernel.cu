@@ -3,22 +3,23 @@
 // Main kernel: one persistent CTA per SM owns a share ("slab") of the H neurons and runs the whole
 // of the paper's sparse execution scheme (Sec. 3.1) on it without leaving the SM:
 //
-//   gate producer  one thread streams the slab's gate rows (W_1, or U for the LoPA gate) into a
+//   gate producers two threads (two warps) stream the slab's gate rows (W_1, or U for the LoPA gate) into a
 //                  shared-memory ring with bulk asynchronous copies (TMA, mbarrier complete_tx).
-//                  It depends on nothing but free ring slots, so HBM stays busy from the first
+//                  They depend on nothing but free ring slots, so HBM stays busy from the first
 //                  cycle of the CTA to the last gate row.
 //   gate warps     each owns ring slots: z_j = row . vec + b_g[j] (+ fixed-matrix term),
 //                  a_j = A(z_j), and publishes "fired" (z_j > 0) per neuron.
-//   act producer   one thread walks the published results in ascending neuron order and queues the
+//   act producers  two warps walk the published results in ascending neuron order and queue the
 //                  W_up / W_down rows of the neurons that fired into a second ring.
-//   act warps      four warps consume the second ring in order: u_j = W_up[j] . x (CTA-level
+//   act warps      four warps (eight for the LoPA gate, which needs only four gate warps) consume the
+//                  second ring in order: u_j = W_up[j] . x (CTA-level
 //                  reduction), h_j = a_j u_j, y_part += h_j W_down[j]; each thread keeps its own
 //                  column slice of y_part in registers and writes it out once.
 //
 // A small second kernel sums the per-CTA partials in CTA order (deterministic, no float atomics).
-// For the LoPA gate (Eq. 3, Sec. 3.3) a small first kernel computes v = V x; the main kernel
-// normalises it (RMSNorm) into shared memory and feeds it to the U stage, with the U rows already
-// being prefetched.
+// For the LoPA gate (Eq. 3, Sec. 3.3) the rank-r stage v = V x is spread over the CTAs of the main
+// kernel, exchanged through global memory (bounded wait on an arrival counter) and normalised (RMSNorm)
+// into shared memory, with the U rows already sitting in the ring.
 //
 // The kernels are chained with programmatic dependent launch: each lets its successor start early
 // and waits (griddepcontrol.wait) only before it touches anything a predecessor may write.  Weights
@@ -45,7 +46,6 @@ constexpr int kGateWarps = 8;
 constexpr int kFirstActWarp = kFirstGateWarp + kGateWarps;
 constexpr int kActWarps = 4;
 constexpr int kThreads = 32 * (kFirstActWarp + kActWarps);  // 512
-constexpr int kActThreads = 32 * kActWarps;
 constexpr int kStageBase = 32 * kGateProducers;  // first thread that takes part in staging the token
 constexpr int kStageThreads = kThreads - kStageBase;
 constexpr int kMaxGrid = 256;
@@ -95,7 +95,7 @@ struct SmemLayout {
     sn = take(lopa ? K * 4 : 0);
     aval = take(slab_max * 4);
     slot_a = take(n_act_slots * 4);
-    red = take(2 * (2 * kActWarps + 1) * 4);
+    red = take(2 * (2 * 8 + 1) * 4);  // up to eight act warps
     ctl = take(8 * 4);
     bars = take(2 * (n_gate_slots + n_act_slots) * 8);
     total = off;
@@ -212,6 +212,15 @@ __device__ __forceinline__ long long global_ns() {
 
 template <typename T, int CPT, bool LOPA>
 __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedParams p) {
+  // Warp roles: 2 gate producers, 2 act producers, then gate warps and act warps.  The standard gate needs its
+  // eight gate warps to keep up with the stream; the LoPA gate is short (r elements per row), the call's time
+  // is then set by the up/down rows, so eight of the twelve workers are act warps there.
+  constexpr int kAW = LOPA ? 8 : 4;                         // act warps
+  constexpr int kGW = kGateWarps + kActWarps - kAW;         // gate warps
+  constexpr int kFAW = kFirstGateWarp + kGW;                // first act warp
+  constexpr int kAT = 32 * kAW;                             // act threads
+  static_assert(kGW >= 2, "gate warps");
+
   extern __shared__ __align__(128) unsigned char smem[];
   const long long t_entry = clock64();
   pdl_launch_dependents();
@@ -265,10 +274,10 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
       }
       for (int s = 0; s < NA; ++s) {
         mbar_init(full_act + 8 * s, kActProducers);
-        mbar_init(empty_act + 8 * s, kActWarps);
+        mbar_init(empty_act + 8 * s, kAW);
       }
       for (int i = 0; i < 8; ++i) ctl[i] = 0;
-      for (int i = 0; i < 2 * (2 * kActWarps + 1); ++i) red[i] = 0.f;
+      for (int i = 0; i < 2 * (2 * kAW + 1); ++i) red[i] = 0.f;
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -296,7 +305,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
   // ring slots now: like the weights they do not depend on the predecessor in the stream.
   float pre_bias[2] = {0.f, 0.f}, pre_sg[2] = {1.f, 1.f};
   int pre_gi[2] = {-1, -1};
-  if (warp >= kFirstGateWarp && warp < kFirstActWarp && warp - kFirstGateWarp < p.gate_warps) {
+  if (warp >= kFirstGateWarp && warp < kFAW && warp - kFirstGateWarp < p.gate_warps) {
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
       const int sq = warp - kFirstGateWarp + q * p.gate_warps;
@@ -440,7 +449,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
     }
     if (lane == 0 && ap == 0) SFFN_STAMP(2);
     __syncwarp();
-  } else if (warp < kFirstActWarp) {
+  } else if (warp < kFAW) {
     // ======================= gate warps ========================================================
     const int gw = warp - kFirstGateWarp;
     for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_warps) {
@@ -513,8 +522,8 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
     if (lane == 0 && gw == (n_gslots - 1) % p.gate_warps) SFFN_STAMP(3);
   } else {
     // ======================= act warps =========================================================
-    const int at = tid - 32 * kFirstActWarp;  // 0..127
-    const int aw = warp - kFirstActWarp;
+    const int at = tid - 32 * kFAW;  // 0..127
+    const int aw = warp - kFAW;
     float acc[CPT][EPV];
 #pragma unroll
     for (int i = 0; i < CPT; ++i)
@@ -529,7 +538,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
     int slot = 0;
     uint32_t par = 0;
     for (int round = 0;; ++round) {
-      float* rp = red + (round & 1) * (2 * kActWarps + 1);
+      float* rp = red + (round & 1) * (2 * kAW + 1);
       const int slot1 = slot + 1 == NA ? 0 : slot + 1;
       const uint32_t par1 = slot + 1 == NA ? par ^ 1 : par;
       const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status);
@@ -549,7 +558,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         const uint4* wu1 = reinterpret_cast<const uint4*>(s1);
 #pragma unroll
         for (int i = 0; i < CPT; ++i) {
-          const int c = at + i * kActThreads;
+          const int c = at + i * kAT;
           if (c < nvecD) {
             part0 = chunk_dot<T>(wu0[c], sx, c, nvecD, part0);
             if (a1 >= 0.f) part1 = chunk_dot<T>(wu1[c], sx, c, nvecD, part1);
@@ -559,19 +568,24 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         part1 = warp_sum(part1);
         if (lane == 0) {
           rp[aw] = part0;
-          rp[kActWarps + aw] = part1;
+          rp[kAW + aw] = part1;
         }
       }
-      if (a0 < 0.f || !got1) rp[2 * kActWarps] = 1.f;  // stop marker first in the round, or a failed wait
-      named_bar_sync(2, kActThreads);
-      if (rp[2 * kActWarps] != 0.f) break;
-      const float h0 = a0 * ((rp[0] + rp[1]) + (rp[2] + rp[3]));
-      const float h1 = a1 * ((rp[kActWarps] + rp[kActWarps + 1]) + (rp[kActWarps + 2] + rp[kActWarps + 3]));
+      if (a0 < 0.f || !got1) rp[2 * kAW] = 1.f;  // stop marker first in the round, or a failed wait
+      named_bar_sync(2, kAT);
+      if (rp[2 * kAW] != 0.f) break;
+      float u0 = (rp[0] + rp[1]) + (rp[2] + rp[3]);
+      float u1 = (rp[kAW] + rp[kAW + 1]) + (rp[kAW + 2] + rp[kAW + 3]);
+      if (kAW == 8) {
+        u0 += (rp[4] + rp[5]) + (rp[6] + rp[7]);
+        u1 += (rp[kAW + 4] + rp[kAW + 5]) + (rp[kAW + 6] + rp[kAW + 7]);
+      }
+      const float h0 = a0 * u0, h1 = a1 * u1;
       const uint4* wd0 = reinterpret_cast<const uint4*>(s0 + row_bytes);
       const uint4* wd1 = reinterpret_cast<const uint4*>(s1 + row_bytes);
 #pragma unroll
       for (int i = 0; i < CPT; ++i) {
-        const int c = at + i * kActThreads;
+        const int c = at + i * kAT;
         if (c < nvecD) {
           float f[EPV];
           Elem<T>::unpack(wd0[c], f);
@@ -600,7 +614,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
     float* dst = p.partial + (size_t)cta * D;
 #pragma unroll
     for (int i = 0; i < CPT; ++i) {
-      const int c = at + i * kActThreads;
+      const int c = at + i * kAT;
       if (c < nvecD) {
 #pragma unroll
         for (int e = 0; e < EPV; e += 4)
@@ -667,8 +681,10 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   const int nvecD = D / epv;
   const int row_bytes = D * esz, gate_row_bytes = K * esz;
   g.ok = false;
-  if (row_bytes % 16 || gate_row_bytes % 16 || nvecD > kActThreads * 8) return g;
-  g.cpt = nvecD <= kActThreads ? 1 : nvecD <= 2 * kActThreads ? 2 : nvecD <= 4 * kActThreads ? 4 : 8;
+  const int act_threads = lopa ? 256 : 128;    // as in the kernel: eight act warps for the LoPA gate
+  const int gate_warps_max = lopa ? 4 : 8;
+  if (row_bytes % 16 || gate_row_bytes % 16 || nvecD > act_threads * 8) return g;
+  g.cpt = nvecD <= act_threads ? 1 : nvecD <= 2 * act_threads ? 2 : nvecD <= 4 * act_threads ? 4 : 8;
   int nr = 8192 / gate_row_bytes;
   nr = nr < 1 ? 1 : nr > 32 ? 32 : nr;
   g.rows_per_gate_slot = nr;
@@ -686,7 +702,7 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   // An even number of gate warps (slots alternate between two producers).  Where memory allows only
   // one slot per warp (16 KB rows), eight warps with one slot each still beat four warps with two
   // (measured at 8192 x 28672: 104 us against 145 us per call).
-  int gw = (ng < kGateWarps ? ng : kGateWarps) & ~1;
+  int gw = (ng < gate_warps_max ? ng : gate_warps_max) & ~1;
   if (gw < 2) gw = 2;
   g.gate_warps = gw;
   if (ng > 3 * gw) ng = 3 * gw;
