@@ -311,6 +311,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       p.W = W_up; p.R = H; p.K = D;
       if (own_list) {
         p.words_in = words; p.n_words = 4 * gate_tiles; p.gate_tile_rows = gate_tile_rows;
+        p.gate_rows_per_word = gate_tile_rows <= 64 ? 16 : 32;
         p.idx_out = idx; p.count_out = count;
       } else {
         p.idx = lidx; p.count = lcount;

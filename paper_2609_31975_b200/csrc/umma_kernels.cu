@@ -40,6 +40,8 @@ constexpr int kAAtomBytes = kTileRows * 128;         // 16 KB: one [128 rows x 6
 constexpr int kThreads = 320;                        // 4 producer warps, 4 epilogue warps, 2 MMA warps
 constexpr int kThreadsRows = 384;                    // rows kernels: up to 4 MMA warps
 constexpr int kProducerWarps = 4;
+constexpr int kMaxStages = 12;
+constexpr int kMaxIssuers = 4;
 constexpr int kScanChunks = 4;                       // in-kernel compaction: up to 4 * 384 mask words = 384 gate tiles
 constexpr int kMaxOwnTiles = 8;                      // tiles of one CTA whose rows are kept in shared memory
 constexpr int kHeaderBytes = 1024 + kMaxOwnTiles * kTileRows * 4;  // barriers + scratch, then the row lists
@@ -109,9 +111,9 @@ __device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr, uint32_t mn
   d |= (uint64_t)2 << 61;
   return d;
 }
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t make_idesc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = m (64 or 128), N = n.
+__device__ __forceinline__ uint32_t make_idesc(int n, int m = kTileRows) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -189,18 +191,16 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   // carve: stages first (1024-byte aligned), then barriers and control words
   const int npad = p.npad;
-  const int stage_bytes = kAAtomBytes + p.atoms_max * npad * 128;
-  const int S = p.stages;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  // header: barriers and control words, scan scratch, this CTA's rows of the union list; then the stages
-  // (which end with a read-over pad)
+  // header: barriers (for the largest ring) and control words, scan scratch, this CTA's rows of the union
+  // list; then the ring of stages, whose geometry is decided below once the tile height is known
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
   int* scan_wt = reinterpret_cast<int*>(smem + 512);   // [kScanChunks][warps]
   int* rows_sm = reinterpret_cast<int*>(smem + 1024);  // [kMaxOwnTiles][128]
   const uint32_t stage0 = smem_u32(smem) + kHeaderBytes;
-  const uint32_t full = smem_u32(bars), empty = smem_u32(bars + S);
-  const uint32_t acc_full = smem_u32(bars + 2 * S), acc_empty = smem_u32(bars + 2 * S + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
+  const uint32_t full = smem_u32(bars), empty = smem_u32(bars + kMaxStages);
+  const uint32_t acc_full = smem_u32(bars + 2 * kMaxStages), acc_empty = smem_u32(bars + 2 * kMaxStages + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -208,9 +208,9 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
 
   // Set-up that needs nothing from earlier kernels runs while the predecessor in the stream finishes.
   pdl_launch_dependents();
-  const uint32_t tmem_cols = tmem_cols_for(p.issuers * npad);
+  const uint32_t tmem_cols = tmem_cols_for(kMaxIssuers * npad);
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(full + 8 * s, 1);  // the producer's expect_tx arrive; the copies complete the bytes
       mbar_init(empty + 8 * s, 1);
     }
@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
 
   // Union rows: either the list is given (idx, count), or every CTA compacts the gate's "fired" bit masks
   // itself.  The gate kernel leaves one 32-bit word per epilogue warp and tile (word 4 * tile + warp, bit =
-  // lane = row 32 * warp + lane of the tile); thread t takes word t of each chunk of `threads` words, a
+  // lane = row rows_per_word * warp + lane of the tile, 32 rows per word for M = 128 tiles, 16 for M = 64); thread t takes word t of each chunk of `threads` words, a
   // warp scan plus the warp totals of all chunks give the list position of its first set bit.
   const bool own_list = UP && p.words_in != nullptr;
   uint32_t bits[kScanChunks];
@@ -284,7 +284,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       if (k < nch && bits[k]) {
         const int cnt = __popc(bits[k]);
         const int w = k * kThreadsRows + tid;
-        const int j0 = (w >> 2) * p.gate_tile_rows + (w & 3) * 32;  // row of bit 0
+        const int j0 = (w >> 2) * p.gate_tile_rows + (w & 3) * p.gate_rows_per_word;  // row of bit 0
         int m = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++m) {
           const int lo = tile * tile_rows, hi = lo + tile_rows;
@@ -305,18 +305,34 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     }
     if (blockIdx.x == 0 && tid == 0) *p.count_out = n_rows;
   }
-  // A stage holds `atoms` successive K blocks of the tile: short tiles (few rows) take several, so that a
-  // stage stays near 16 KB and the bytes in flight do not shrink with the tile.  Block a of a stage sits
-  // tile_rows * 128 bytes after block a - 1; the MMA of a block reads 128 rows from its start, i.e. on
-  // into the following blocks / the token blocks / the pad behind the last stage (rows that are ignored).
+  // Stage geometry.  Tiles of up to 64 rows are multiplied with M = 64 (accumulator row i then sits in TMEM lane
+  // 32 * (i / 16) + i % 16), taller ones with M = 128 (row i in lane i).  A stage holds `atoms` successive K
+  // blocks of the tile -- short tiles take several, so that a stage stays near 16 KB and the bytes in flight do
+  // not shrink with the tile -- followed by the token rows of the same K blocks.  Block a sits tile_rows * 128
+  // bytes after block a - 1; its MMA reads M rows from its start, i.e. on into the following blocks and the
+  // token rows of the same stage (rows that are ignored); the stage is sized so that it never reads past it.
+  const bool m64 = tile_rows <= 64;
+  const int mrows = m64 ? 64 : kTileRows;
   int atoms = kTileRows / tile_rows;
-  atoms = atoms > p.atoms_max ? p.atoms_max : atoms;
+  const int atoms_cap = npad <= 16 ? 4 : npad <= 32 ? 2 : 1;  // at most 8 KB of token rows per stage
+  atoms = atoms > atoms_cap ? atoms_cap : atoms;
   const int a_block_bytes = tile_rows * 128, b_block_bytes = npad * 128;
+  const int b_off = atoms * a_block_bytes;                    // token rows of a stage start here
+  int stage_bytes = atoms * (a_block_bytes + b_block_bytes);
+  stage_bytes = max(stage_bytes, (atoms - 1) * a_block_bytes + mrows * 128);
+  stage_bytes = (stage_bytes + 1023) & ~1023;
+  int S = p.ring_bytes / stage_bytes;
+  S = S > kMaxStages ? kMaxStages : S;
+  // four issuers when the ring divides evenly among them, otherwise two (slot mod issuers = owner)
+  const int issuers = (S >= 8 && S % 4 == 0) ? 4 : 2;
+  S &= ~1;
   const int kstages = (kblocks + atoms - 1) / atoms;
+  // accumulator row that this thread's TMEM lane holds (-1: none); the same for every warp of a lane quarter
+  const int row_thr = m64 ? (lane < 16 ? (warp & 3) * 16 + lane : -1) : (warp & 3) * 32 + lane;
   // The MMA issuers take the stages of their ring slots (slot mod issuers) into accumulators of their own
   // (npad TMEM columns each); the epilogue adds them.  A tile with at least as many stages as issuers
   // gives each issuer a stage; shorter tiles use fewer issuers.
-  const int nacc = kstages >= p.issuers ? p.issuers : kstages >= 2 ? 2 : 1;
+  const int nacc = kstages >= issuers ? issuers : kstages >= 2 ? 2 : 1;
   if (tid == 0) {
     mbar_init(acc_full, nacc);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -332,11 +348,11 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   // and stores HmT.  Returns false if the wait was abandoned.
   const bool share_last = npad >= 32;  // four or more column groups: worth spreading over all warps
   auto epilogue = [&](int tile, int tcount, int part, int nparts, bool& fired) -> bool {
-    const int row_in_tile = (warp & 3) * 32 + lane;   // TMEM lane of this thread
+    const int row_in_tile = row_thr;
     const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     const int B = p.B;
     const int li = tile * tile_rows + row_in_tile;
-    const bool row_ok = row_in_tile < tile_rows && li < n_rows;
+    const bool row_ok = row_in_tile >= 0 && row_in_tile < tile_rows && li < n_rows;
     const int j = !row_ok ? 0 : own_list ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
     // everything that does not depend on the accumulator is fetched before the wait
     float bias = 0.f, sg = 1.f;
@@ -461,14 +477,14 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
         } else if (lane == 0) {
           tma_tile_2d(abase + a * a_block_bytes, &map_w, k0, tile * tile_rows, full + 8 * s);
         }
-        if (lane == 0) tma_tile_2d(abase + kAAtomBytes + a * b_block_bytes, &map_x, k0, 0, full + 8 * s);
+        if (lane == 0) tma_tile_2d(abase + b_off + a * b_block_bytes, &map_x, k0, 0, full + 8 * s);
       }
     }
   } else if (warp >= 8) {
     // ======================= MMA issuers =======================================================
     const int m = warp - 8;
     if (lane == 0 && m < nacc) {
-      const uint32_t idesc = make_idesc(npad);
+      const uint32_t idesc = make_idesc(npad, mrows);
       const uint32_t acc = tmem_base + m * npad;
       int tcount = 0;
       bool ok = true;
@@ -486,7 +502,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
           const int na = min(atoms, kblocks - kb * atoms);
           for (int a = 0; a < na; ++a) {
             const uint64_t adesc = make_desc(sbase + a * a_block_bytes);
-            const uint64_t bdesc = make_desc(sbase + kAAtomBytes + a * b_block_bytes);
+            const uint64_t bdesc = make_desc(sbase + b_off + a * b_block_bytes);
             umma(acc, adesc, bdesc, idesc, (kb >= nacc || a > 0) ? 1u : 0u);
 #pragma unroll
             for (int k = 1; k < kAtomK / 16; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
@@ -510,9 +526,9 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     for (int tile = blockIdx.x; tile + (share_last ? (int)gridDim.x : 0) < n_tiles; tile += gridDim.x, ++tcount) {
       bool fired = false;
       if (!epilogue(tile, tcount, 0, 1, fired)) break;
-      const int row_in_tile = (warp - 4) * 32 + lane;
+      const int row_in_tile = row_thr;
       const int li = tile * tile_rows + row_in_tile;
-      const bool valid = row_in_tile < tile_rows && li < n_rows;
+      const bool valid = row_in_tile >= 0 && row_in_tile < tile_rows && li < n_rows;
       if (!UP && p.flag && valid) p.flag[li] = fired ? 1 : 0;
       if (!UP && p.words_out) {
         const unsigned m = __ballot_sync(0xffffffffu, fired && valid);
@@ -534,14 +550,14 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     const bool done = epilogue(last_tile, my_tiles - 1, part, 3, fired);
     if (!UP && (p.flag || p.words_out)) {
       uint8_t* fired_sm = reinterpret_cast<uint8_t*>(scan_wt);  // [3][128], the scan scratch is free here
-      const int row_in_tile = (warp & 3) * 32 + lane;
-      fired_sm[part * kTileRows + row_in_tile] = fired ? 1 : 0;
+      const int row_in_tile = row_thr;
+      const int me = (warp & 3) * 32 + lane;  // this thread's entry: the same in all three parts
+      fired_sm[part * kTileRows + me] = fired ? 1 : 0;
       named_bar_sync(2, kThreadsRows);  // reached by every thread of a CTA that owns a tile, whatever happened
       const int li = last_tile * tile_rows + row_in_tile;
       if (part == 0) {  // warps 4-7, all lanes
-        const bool valid = done && row_in_tile < tile_rows && li < n_rows;
-        const bool any =
-            (fired_sm[row_in_tile] | fired_sm[kTileRows + row_in_tile] | fired_sm[2 * kTileRows + row_in_tile]) != 0;
+        const bool valid = done && row_in_tile >= 0 && row_in_tile < tile_rows && li < n_rows;
+        const bool any = (fired_sm[me] | fired_sm[kTileRows + me] | fired_sm[2 * kTileRows + me]) != 0;
         if (p.flag && valid) p.flag[li] = any ? 1 : 0;
         if (p.words_out) {
           const unsigned m = __ballot_sync(0xffffffffu, any && valid);
@@ -800,24 +816,9 @@ bool make_map(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_el
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s) {
   p.npad = (cols + 15) / 16 * 16;
   const int grid = p.R < 8 * sm_count ? (p.R + 7) / 8 : sm_count;
-  // K blocks per stage: up to 8 KB of token rows; the gate knows its tile height, the union rows only a bound
-  p.atoms_max = p.npad <= 16 ? 4 : p.npad <= 32 ? 2 : 1;
-  if (!up) {
-    const int fit = kTileRows / tile_rows_for(p.R, grid);
-    p.atoms_max = fit < p.atoms_max ? fit : p.atoms_max;
-  }
-  const int stage_bytes = kAAtomBytes + p.atoms_max * p.npad * 128;
-  // 1 KB of barriers in front; with several blocks per stage, 16 KB behind the last stage that the MMAs
-  // of the later blocks may read over
-  const int pad = p.atoms_max > 1 ? kAAtomBytes : 0;
-  int stages = (224 * 1024 - 1024 - kHeaderBytes - pad) / stage_bytes;
-  if (stages > 12) stages = 12;
-  // four issuers when each can own two or more slots, otherwise two; slots divide evenly among them
-  p.issuers = stages >= 8 ? 4 : 2;
-  stages &= ~(p.issuers - 1);
-  if (stages < 2) return cudaErrorInvalidValue;
-  p.stages = stages;
-  const size_t smem = 1024 + kHeaderBytes + (size_t)stages * stage_bytes + pad;
+  // all the dynamic shared memory a CTA can have; the kernel cuts its ring out of it once it knows its tiles
+  const size_t smem = 226 * 1024;
+  p.ring_bytes = (int)smem - 1024 - kHeaderBytes;
   alignas(64) CUtensorMap map_w, map_x;
   // weights: all R rows; boxes of one tile's rows for the gate, single-row boxes for the gather
   if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : tile_rows_for(p.R, grid))) return cudaErrorNotSupported;

@@ -17,6 +17,7 @@ struct UmmaRowsParams {
   const uint32_t* words_in;  // UP, instead of idx / count: the gate kernel's "fired" bit masks (n_words of
   int n_words;               //   them, 4 per gate tile of gate_tile_rows rows); the kernel compacts them itself
   int gate_tile_rows;
+  int gate_rows_per_word;    //   rows covered by one mask word: 32 for gate tiles of more than 64 rows, else 16
   int32_t* idx_out;          //   ... and writes the ascending list
   int32_t* count_out;        //   ... and its length
   const void* X;         // token operand [cols][K] bf16, row stride x_stride (elements)
@@ -38,7 +39,7 @@ struct UmmaRowsParams {
   void* hmT;             // UP: bf16 [B][hm_stride]
   int hm_stride;
   int32_t* status;       // device status word
-  int npad, stages, issuers, atoms_max;  // filled by the launcher
+  int npad, ring_bytes;  // filled by the launcher
 };
 
 struct UmmaDownParams {
