@@ -136,13 +136,15 @@ def active_set(z) -> np.ndarray:
     return idx[:n].copy()
 
 
-def ffn(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, b_g=None, route="sparse", threads=1):
+def ffn(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, b_g=None, route="sparse", threads=1, act_up=None):
     """Gated FFN for a batch of independent tokens.
 
     x [B,D] (or [D]); W_up, W_down [H,D] (W_down = W_2 transposed); either ``W_g`` [H,D] or
     ``lopa`` = dict(V=[r,D], U=[H,r], g_idx=None|[H], g_sign=None|[H], gamma=None|[r],
     use_rmsnorm=bool, eps=float).  ``route`` is "dense" (all H neurons, Eq. 1) or "sparse"
-    (only z_j > 0).  Returns dict(y [B,D] f64, z [B,H] f64, n_act [B], union_mask [H] bool).
+    (only z_j > 0).  ``act_up`` names the activation A_3 on the output of W_3 (double activation,
+    Sec. 3.3); None is Eq. 1.  Returns dict(y [B,D] f64, z [B,H] f64, n_act [B], n_gated [B] = number
+    of neurons with a nonzero h_j, union_mask [H] bool).
     """
     x = as_oracle_array(x)
     single = x.ndim == 1
@@ -156,6 +158,7 @@ def ffn(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, b_g=None, route="sp
     y = np.zeros((B, D), np.float64)
     z = np.zeros((B, H), np.float64)
     n_act = np.zeros(B, np.int32)
+    n_gated = np.zeros(B, np.int32)
     mask = np.zeros(H, np.uint8)
     W1 = V = U = gi = gs = gm = None
     kind, use_rms, eps, r = 0, 0, 0.0, 0
@@ -173,10 +176,11 @@ def ffn(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, b_g=None, route="sp
     rc = _load().oracle_ffn_batch(
         kind, _p(W1), _p(V), _p(U), _p(gi), _p(gs), _p(gm), use_rms, ctypes.c_double(eps), r, _p(b),
         _p(W_up), _p(W_down), _DT[W_up.dtype], _p(x), _DT[x.dtype], B, H, D, ACT[act],
-        {"dense": 0, "sparse": 1}[route], int(threads), _p(y), _p(z), _p(n_act), _p(mask))
+        -1 if act_up is None else ACT[act_up], {"dense": 0, "sparse": 1}[route], int(threads), _p(y), _p(z),
+        _p(n_act), _p(n_gated), _p(mask))
     if rc != 0:
         raise ValueError("oracle_ffn_batch rejected its arguments")
-    out = dict(y=y, z=z, n_act=n_act, union_mask=mask.astype(bool))
+    out = dict(y=y, z=z, n_act=n_act, n_gated=n_gated, union_mask=mask.astype(bool))
     if single:
         out["y"], out["z"] = y[0], z[0]
     return out

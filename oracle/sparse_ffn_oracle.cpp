@@ -131,26 +131,33 @@ int oracle_active_set(const double* z, int H, int32_t* idx) {
 //   route 0 (dense):  every j in 0..H-1           (Eq. 1 as written)
 //   route 1 (sparse): only j with z_j > 0         (Sec. 3.1 skipping rule)
 // W_down is W_2 transposed, [H, D] row-major.  y is [D] double.  Returns rows of W_3 touched.
-int oracle_updown(const double* z, int act, const void* W3, const void* Wdown, int wdtype,
-                  const void* x, int xdtype, int H, int D, int route, double* y) {
+// Double activation (Sec. 3.3, "Double activation"): with act_up >= 0 the activation A_3 = act_up is
+// applied to the output of W_3 as well, h_j = A(z_j) * A_3(u_j); act_up < 0 is Eq. 1 as written.
+// *n_gated (may be NULL) counts the j with h_j != 0, the "s_gated" site of the sparsity-sites table:
+// rows of W_2 whose contribution is not identically zero.
+int oracle_updown(const double* z, int act, int act_up, const void* W3, const void* Wdown, int wdtype,
+                  const void* x, int xdtype, int H, int D, int route, double* y, int* n_gated) {
   for (int d = 0; d < D; ++d) y[d] = 0.0;
-  int touched = 0;
+  int touched = 0, gated = 0;
   for (int j = 0; j < H; ++j) {
     if (route == 1 && !(z[j] > 0.0)) continue;
     ++touched;
     const double a = activation(act, z[j]);
     double u = 0.0;
     for (int d = 0; d < D; ++d) u += load(W3, wdtype, (size_t)j * D + d) * load(x, xdtype, d);
-    const double h = a * u;
+    const double h = a * (act_up >= 0 ? activation(act_up, u) : u);
+    gated += h != 0.0;
     for (int d = 0; d < D; ++d) y[d] += h * load(Wdown, wdtype, (size_t)j * D + d);
   }
+  if (n_gated) *n_gated = gated;
   return touched;
 }
 
 // Whole FFN for a batch of B independent tokens (a batch is B separate FFNs; Sec. 5.4 only adds
 // that rows must be loaded for the union of the tokens' active sets).
 //   gate_kind 0: standard (W1 used);  1: LoPA (V, U, g_idx, g_sign, gamma, use_rmsnorm, eps, r used)
-//   x [B,D];  y [B,D] double;  z_out [B,H] double or NULL;  n_act_out [B] or NULL;
+//   act_up < 0: Eq. 1; >= 0: double activation with A_3 = act_up (see oracle_updown);
+//   x [B,D];  y [B,D] double;  z_out [B,H] double or NULL;  n_act_out, n_gated_out [B] or NULL;
 //   union_mask [H] bytes or NULL (1 where any token fires).
 // threads > 1 splits the tokens over OpenMP threads; the arithmetic per token is unchanged.
 // Returns 0, or -1 on a bad argument.
@@ -158,14 +165,14 @@ int oracle_ffn_batch(int gate_kind, const void* W1, const void* V, const void* U
                      const int32_t* g_idx, const int8_t* g_sign, const float* gamma,
                      int use_rmsnorm, double eps, int r, const float* b_g, const void* W3,
                      const void* Wdown, int wdtype, const void* x, int xdtype, int B, int H, int D,
-                     int act, int route, int threads, double* y, double* z_out, int32_t* n_act_out,
-                     uint8_t* union_mask) {
+                     int act, int act_up, int route, int threads, double* y, double* z_out,
+                     int32_t* n_act_out, int32_t* n_gated_out, uint8_t* union_mask) {
   if (B < 0 || H <= 0 || D <= 0 || !W3 || !Wdown || !x || !y) return -1;
   if (gate_kind == 0 && !W1) return -1;
   if (gate_kind == 1 && (!V || !U || r <= 0)) return -1;
   if (union_mask) std::memset(union_mask, 0, (size_t)H);
   const size_t xstride = (size_t)D * (xdtype == F32 ? 4 : xdtype == BF16 ? 2 : 8);
-  std::vector<int32_t> n_act(B > 0 ? B : 1);
+  std::vector<int32_t> n_act(B > 0 ? B : 1), n_gated(B > 0 ? B : 1);
   std::vector<std::vector<uint8_t>> masks;
   if (union_mask) masks.assign(B, std::vector<uint8_t>());
 #pragma omp parallel for schedule(dynamic, 1) num_threads(threads > 1 ? threads : 1)
@@ -177,7 +184,9 @@ int oracle_ffn_batch(int gate_kind, const void* W1, const void* V, const void* U
     else
       oracle_gate_lopa(V, U, wdtype, g_idx, g_sign, gamma, use_rmsnorm, eps, r, xb, xdtype, b_g, H,
                        D, z.data(), nullptr, nullptr);
-    oracle_updown(z.data(), act, W3, Wdown, wdtype, xb, xdtype, H, D, route, y + (size_t)b * D);
+    int gated = 0;
+    oracle_updown(z.data(), act, act_up, W3, Wdown, wdtype, xb, xdtype, H, D, route, y + (size_t)b * D, &gated);
+    n_gated[b] = gated;
     int cnt = 0;
     for (int j = 0; j < H; ++j) cnt += z[j] > 0.0;
     n_act[b] = cnt;
@@ -189,6 +198,7 @@ int oracle_ffn_batch(int gate_kind, const void* W1, const void* V, const void* U
   }
   for (int b = 0; b < B; ++b) {
     if (n_act_out) n_act_out[b] = n_act[b];
+    if (n_gated_out) n_gated_out[b] = n_gated[b];
     if (union_mask)
       for (int j = 0; j < H; ++j) union_mask[j] |= masks[b][j];
   }

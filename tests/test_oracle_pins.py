@@ -302,3 +302,56 @@ def test_zipf_profile_recipe():
     # a N(0,1) pre-activation plus b_j is positive with probability p_j
     fire = 0.5 * torch.erfc(-b.double() / math.sqrt(2.0))
     np.testing.assert_allclose(fire.numpy(), p.numpy(), atol=1e-6)
+
+
+# ---------------------------------------------------------------- double activation (Sec. 3.3) and the s_gated site
+def test_hand_worked_double_activation():
+    # x = [1, 2];  z = W1 x = [1, -2, 3] (RELU: a = [1, 0, 3]);  u = W3 x = [3-2, 2+4, -1+0.5] = [1, 6, -0.5]
+    W1 = np.array([[1.0, 0.0], [0.0, -1.0], [1.0, 1.0]], np.float32)
+    W3 = np.array([[3.0, -1.0], [2.0, 2.0], [-1.0, 0.25]], np.float32)
+    Wd = np.array([[1.0, 1.0], [5.0, 5.0], [2.0, -2.0]], np.float32)   # rows = columns of W_2
+    x = np.array([1.0, 2.0], np.float32)
+    for route in ("dense", "sparse"):
+        # Eq. 1: h = a * u = [1, 0, -1.5];  y = 1*[1,1] - 1.5*[2,-2] = [-2, 4];  two neurons with h != 0
+        out = oracle.ffn(x, W3, Wd, "relu", W_g=W1, route=route)
+        np.testing.assert_array_equal(out["y"], [-2.0, 4.0])
+        assert out["n_act"][0] == 2 and out["n_gated"][0] == 2
+        # A_3 = RELU on the W_3 output: A_3(u) = [1, 6, 0];  h = [1, 0, 0];  y = [1, 1];  one gated neuron
+        out = oracle.ffn(x, W3, Wd, "relu", W_g=W1, route=route, act_up="relu")
+        np.testing.assert_array_equal(out["y"], [1.0, 1.0])
+        assert out["n_act"][0] == 2 and out["n_gated"][0] == 1
+        # A_3 = squared RELU: A_3(u) = [1, 36, 0] -> the same h;  A = squared RELU too: a = [1, 0, 9], h = [1, 0, 0]
+        out = oracle.ffn(x, W3, Wd, "sqrelu", W_g=W1, route=route, act_up="sqrelu")
+        np.testing.assert_array_equal(out["y"], [1.0, 1.0])
+        # A_3 = R-S+: A_3(1) = sigmoid(1) = 1 / (1 + e^-1)
+        out = oracle.ffn(x, W3, Wd, "relu", W_g=W1, route=route, act_up="rsplus")
+        np.testing.assert_allclose(out["y"], [1.0 / (1.0 + math.exp(-1.0))] * 2, rtol=1e-15)
+
+
+def test_double_activation_special_cases():
+    D, H, B = 24, 40, 5
+    x = np.abs(RNG.standard_normal((B, D))).astype(np.float32)          # x >= 0
+    W1 = RNG.standard_normal((H, D)).astype(np.float32)
+    Wd = RNG.standard_normal((H, D)).astype(np.float32)
+    Wp = np.abs(RNG.standard_normal((H, D))).astype(np.float32)         # W_3 >= 0  =>  u >= 0
+    single = oracle.ffn(x, Wp, Wd, "relu", W_g=W1)
+    double = oracle.ffn(x, Wp, Wd, "relu", W_g=W1, act_up="relu")
+    np.testing.assert_array_equal(double["y"], single["y"])               # RELU is the identity on u >= 0
+    np.testing.assert_array_equal(double["n_gated"], single["n_act"])
+    neg = oracle.ffn(x, -Wp, Wd, "relu", W_g=W1, act_up="relu")          # u <= 0: A_3(u) = 0 everywhere
+    assert not neg["y"].any() and not neg["n_gated"].any()
+    np.testing.assert_array_equal(neg["n_act"], single["n_act"])          # the gate is untouched
+    # skipping rows never changes y, and the gated set is a subset of the active set
+    W3 = RNG.standard_normal((H, D)).astype(np.float32)
+    for a3 in ("relu", "sqrelu", "rsplus"):
+        dense = oracle.ffn(x, W3, Wd, "sqrelu", W_g=W1, route="dense", act_up=a3)
+        sparse = oracle.ffn(x, W3, Wd, "sqrelu", W_g=W1, route="sparse", act_up=a3)
+        np.testing.assert_array_equal(dense["y"], sparse["y"])
+        assert (sparse["n_gated"] <= sparse["n_act"]).all()
+        # against a library matmul: y = W_2 (A(z) * A_3(u)) with W_2 = Wd^T
+        z = x.astype(np.float64) @ W1.astype(np.float64).T
+        u = x.astype(np.float64) @ W3.astype(np.float64).T
+        a = np.maximum(z, 0.0) ** 2
+        g = {"relu": np.maximum(u, 0.0), "sqrelu": np.maximum(u, 0.0) ** 2,
+             "rsplus": np.where(u >= 0, u / (1.0 + np.exp(-u)), 0.0)}[a3]
+        np.testing.assert_allclose(sparse["y"], (a * g) @ Wd.astype(np.float64), rtol=1e-12, atol=1e-12)
