@@ -59,7 +59,7 @@ typedef enum {
 /* Activation A of Eq. 1.  RELU and R-S+ follow the table of Sec. 3.1 (R-S+: 0 for z < 0,
  * z*sigmoid(z) for z >= 0); SQRELU = max(z,0)^2 is one of the activations of the paper's activation
  * study.  For all three A(z) != 0 exactly when z > 0, which is the test the library applies. */
-typedef enum { SFFN_ACT_RELU = 0, SFFN_ACT_SQRELU = 1, SFFN_ACT_RSPLUS = 2 } sffn_act;
+typedef enum { SFFN_ACT_RELU = 0, SFFN_ACT_SQRELU = 1, SFFN_ACT_RSPLUS = 2, SFFN_ACT_NONE = 3 } sffn_act;
 
 typedef enum { SFFN_F32 = 0, SFFN_BF16 = 1 } sffn_dtype;
 
@@ -106,6 +106,15 @@ int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dt
 int sffn_destroy(sffn_handle* handle);
 
 int sffn_set_path(sffn_handle* handle, int path /* sffn_path */);
+
+/* Double activation (Sec. 3.3, "Double activation"): with act_up = RELU / SQRELU / RSPLUS every later
+ * call on the handle computes y = W_2 ( A(W_1 x + b_g) . A_3(W_3 x) ), A_3 = act_up, in the sparse and
+ * in the dense entry points alike; SFFN_ACT_NONE (the default) is Eq. 1.  A neuron whose product
+ * A(.) A_3(.) is zero for every token of the call contributes nothing (the "s_gated" site of the
+ * paper's sparsity-sites table): the CUDA-core path (SFFN_PATH_GENERAL) then does not read its row of
+ * W_down; the fused and the tensor-core paths fetch the two rows of a fired neuron together and read it.
+ * SFFN_ACT_NONE is not a gate activation: `act` of the forward calls stays one of the other three. */
+int sffn_set_up_activation(sffn_handle* handle, int act_up /* sffn_act */);
 
 /* Sparse execution of Eq. 1 (Sec. 3.1): gate in full, then only the active rows of W_up / W_down.
  * x [B,D] and all weights on the device; y [B,D] fp32 on the device, fully overwritten (zeros when

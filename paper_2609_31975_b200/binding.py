@@ -51,6 +51,7 @@ def load_library() -> ctypes.CDLL:
         lib.sffn_create.argtypes = [ctypes.POINTER(vp), i, i, i, i, i, vp, sz]
         lib.sffn_destroy.argtypes = [vp]
         lib.sffn_set_path.argtypes = [vp, i]
+        lib.sffn_set_up_activation.argtypes = [vp, i]
         fwd = [vp, vp, i, ctypes.POINTER(_Gate), vp, vp, vp, i, vp, vp]
         lib.sparse_ffn_forward.argtypes = fwd
         lib.dense_ffn_forward.argtypes = fwd
@@ -130,6 +131,11 @@ class SparseFFN:
             self._h = None
 
     __del__ = close
+
+    def set_up_activation(self, act_up):
+        """Double activation: ``act_up`` in ACT (or None for Eq. 1) is applied to the up projection."""
+        code = 3 if act_up is None else ACT[act_up]
+        _check("sffn_set_up_activation", self.lib.sffn_set_up_activation(self._h, code))
 
     def set_path(self, path: str):
         _check("sffn_set_path", self.lib.sffn_set_path(self._h, PATH[path]))

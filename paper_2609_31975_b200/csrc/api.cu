@@ -69,6 +69,7 @@ struct sffn_handle {
   Layout L;
   int sm_count;
   int path;
+  int act_up;  // activation on the up projection (double activation), SFFN_ACT_NONE = Eq. 1
   long long launches;
   unsigned long long lopa_calls;
   int list_state;  // 0: no sparse call yet, 1: idx/count hold the last call's list, 2: flags hold it
@@ -125,6 +126,7 @@ int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dt
   h->L = make_layout(D, H, r_max, B_max, dtype);
   h->sm_count = sms;
   h->path = SFFN_PATH_AUTO;
+  h->act_up = SFFN_ACT_NONE;
   h->launches = 0;
   h->list_state = 0;
   h->lopa_calls = 0;
@@ -135,6 +137,12 @@ int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dt
 int sffn_destroy(sffn_handle* h) {
   if (!h) return SFFN_ERR_INVALID_ARG;
   delete h;
+  return SFFN_OK;
+}
+
+int sffn_set_up_activation(sffn_handle* h, int act_up) {
+  if (!h || act_up < SFFN_ACT_RELU || act_up > SFFN_ACT_NONE) return SFFN_ERR_INVALID_ARG;
+  h->act_up = act_up;
   return SFFN_OK;
 }
 
@@ -319,6 +327,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
       p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
       p.hmT = hmT; p.hm_stride = h->L.hm_stride; p.status = h->at<int32_t>(h->L.status);
+      p.act_up = h->act_up;
       SFFN_CUDA(launch_umma_rows(true, p, nb, h->sm_count, s));
     } else {
       RowsMmaParams p{};
@@ -326,6 +335,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
       p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
       p.hmT = hmT; p.hm_stride = h->L.hm_stride;
+      p.act_up = h->act_up;
       SFFN_CUDA(launch_rows_mma(true, p, nb, grid_rows, s));
     }
     int nsplit = splits;
@@ -426,6 +436,7 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     p.count = dense ? nullptr : count;
     p.H = H; p.D = D;
     p.partial = partial;
+    p.act_up = h->act_up;
     SFFN_CUDA(launch_updown(bf16, nb, p, grid, s));
     SFFN_CUDA(launch_reduce(partial, grid, nb, D, y + (size_t)b0 * D, D, s));
     h->launches += 2;
@@ -445,7 +456,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
     sffn::FusedCall c{};
     c.bf16 = h->dtype == SFFN_BF16;
     c.D = h->D; c.H = h->H;
-    c.x = x; c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.y = y;
+    c.x = x; c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up; c.y = y;
     c.dense = dense;
     c.workspace = h->ws + h->L.fused;
     c.status = h->at<int32_t>(h->L.status);

@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(256) rows_mma_kernel(const RowsMmaParams p) {
             for (int q = 0; q < 2; ++q) {
               const int col = n * 8 + 2 * t + q;
               if (col < B) {
-                const float h = p.a[(size_t)col * p.a_stride + j] * acc[n][half * 2 + q];
+                const float h = p.a[(size_t)col * p.a_stride + j] * activation(p.act_up, acc[n][half * 2 + q]);
                 static_cast<__nv_bfloat16*>(p.hmT)[(size_t)col * p.hm_stride + i] = __float2bfloat16(h);
               }
             }

@@ -30,6 +30,7 @@ struct RowsMmaParams {
   int a_stride;
   void* hmT;             // bf16 [B][hm_stride]: h of token b for list position u
   int hm_stride;
+  int act_up;            // activation on the up projection (double activation), kActNone = none
 };
 
 struct DownMmaParams {

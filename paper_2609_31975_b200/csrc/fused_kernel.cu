@@ -69,6 +69,7 @@ struct FusedParams {
   unsigned long long* v_counter;   // LoPA: CTAs that have published their rows of v (monotonic over calls)
   unsigned long long v_target;     // LoPA: value of the counter once all CTAs of this call have published
   int act, dense;
+  int act_up;        // activation on the up projection (double activation, Sec. 3.3); kActNone = Eq. 1
   float* partial;  // [grid][D]
   uint8_t* flag;
   int32_t* status;
@@ -580,7 +581,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         u0 += (rp[4] + rp[5]) + (rp[6] + rp[7]);
         u1 += (rp[kAW + 4] + rp[kAW + 5]) + (rp[kAW + 6] + rp[kAW + 7]);
       }
-      const float h0 = a0 * u0, h1 = a1 * u1;
+      const float h0 = a0 * activation(p.act_up, u0), h1 = a1 * activation(p.act_up, u1);
       const uint4* wd0 = reinterpret_cast<const uint4*>(s0 + row_bytes);
       const uint4* wd1 = reinterpret_cast<const uint4*>(s1 + row_bytes);
 #pragma unroll
@@ -794,6 +795,7 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.v_target = *c.lopa_calls * (unsigned long long)grid;
   p.partial = partial;
   p.act = c.act; p.dense = c.dense ? 1 : 0;
+  p.act_up = c.act_up;
   p.flag = c.flag; p.status = c.status;
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;

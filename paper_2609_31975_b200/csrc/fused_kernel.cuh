@@ -18,6 +18,7 @@ struct FusedCall {
   const void* W_up;
   const void* W_down;
   int act;
+  int act_up;
   float* y;
   bool dense;
   void* workspace;   // fused_workspace_bytes() bytes, zeroed at handle creation

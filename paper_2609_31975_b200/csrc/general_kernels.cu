@@ -199,6 +199,7 @@ template <typename T, int NB, int CPT>
 __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
   extern __shared__ float svec[];  // [NB][D] tokens as fp32
   __shared__ float hbuf[16][NB];
+  __shared__ int lbuf[16];  // row contributes (some token has h != 0): otherwise its W_down row is not read
   __shared__ int jbuf[16];
   constexpr int EPV = Elem<T>::kPerVec;
   const int D = p.D;
@@ -258,9 +259,15 @@ __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
     for (int b = 0; b < NB; ++b) u[b] = warp_sum(u[b]);
     if (lane == 0) {
       jbuf[warp] = j;
+      bool live = false;
 #pragma unroll
-      for (int b = 0; b < NB; ++b)
-        hbuf[warp][b] = valid ? p.a[(size_t)b * p.a_stride + j] * u[b] : 0.f;
+      for (int b = 0; b < NB; ++b) {
+        // h = A(z) * A_3(u): double activation of Sec. 3.3 when act_up names one, Eq. 1 otherwise
+        const float h = valid ? p.a[(size_t)b * p.a_stride + j] * activation(p.act_up, u[b]) : 0.f;
+        hbuf[warp][b] = h;
+        live |= h != 0.f;
+      }
+      lbuf[warp] = live ? 1 : 0;
     }
     __syncthreads();
     const int rows = min(16, hi - base);
@@ -272,12 +279,12 @@ __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
 #pragma unroll
         for (int c = 0; c < CPT; ++c) {
           const int cc = threadIdx.x + c * 512;
-          wv[q][c] = (r0 + q < rows && cc < nvec) ? ld_stream16(w + cc) : make_uint4(0, 0, 0, 0);
+          wv[q][c] = (r0 + q < rows && lbuf[r0 + q] && cc < nvec) ? ld_stream16(w + cc) : make_uint4(0, 0, 0, 0);
         }
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        if (r0 + q < rows) {
+        if (r0 + q < rows && lbuf[r0 + q]) {
 #pragma unroll
           for (int c = 0; c < CPT; ++c) {
             float fw[EPV];

@@ -35,6 +35,7 @@ struct UpDownParams {
   const int32_t* count;  // device length of idx, or null = H
   int H, D;
   float* partial;      // [grid][NB][D]
+  int act_up;          // activation on the up projection (double activation), kActNone = none
 };
 
 cudaError_t launch_rowdot(bool bf16, bool vec_is_f32, int nb, bool gate, const RowDotParams& p,

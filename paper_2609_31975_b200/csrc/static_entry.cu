@@ -102,6 +102,7 @@ extern "C" int sparse_ffn_forward_static(const void* x, const void* W_g, const f
   u.idx = idx; u.count = count;
   u.H = H; u.D = D;
   u.partial = partial;
+  u.act_up = SFFN_ACT_NONE;
   if (launch_updown(bf16, 1, u, kGrid, st) != cudaSuccess) return SFFN_ERR_CUDA;
   if (launch_reduce(partial, kGrid, 1, D, y, D, st) != cudaSuccess) return SFFN_ERR_CUDA;
   return SFFN_OK;

@@ -389,7 +389,8 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
         tmem_ld8(taddr + c0, nacc, npad, v);
 #pragma unroll
         for (int q = 0; q < 8; ++q)
-          if (row_ok && c0 + q < B) hm[(size_t)(c0 + q) * p.hm_stride] = __float2bfloat16(av[q] * v[q]);
+          if (row_ok && c0 + q < B)
+            hm[(size_t)(c0 + q) * p.hm_stride] = __float2bfloat16(av[q] * activation(p.act_up, v[q]));
       }
     } else {
       const int act = p.act;

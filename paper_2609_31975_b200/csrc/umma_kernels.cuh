@@ -38,6 +38,7 @@ struct UmmaRowsParams {
   int a_stride;
   void* hmT;             // UP: bf16 [B][hm_stride]
   int hm_stride;
+  int act_up;            // UP: activation on the up projection (double activation), kUmmaActIdentity = none
   int32_t* status;       // device status word
   int npad, ring_bytes;  // filled by the launcher
 };

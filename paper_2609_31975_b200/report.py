@@ -41,9 +41,11 @@ def _time(calls, stream, reps=3):
     return statistics.median(best), min(best)
 
 
-def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1):
-    """sets: list of weight dicts; gate_of(w) -> gate dict.  Returns one result row."""
+def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1, act_up=None):
+    """sets: list of weight dicts; gate_of(w) -> gate dict; act_up: activation on the up projection (double
+    activation) or None.  Returns one result row."""
     ffn = SparseFFN(D, H, torch.bfloat16, r_max=r or 0, B_max=B, device=DEV)
+    ffn.set_up_activation(act_up)
     stream = torch.cuda.Stream(DEV)
     x = syn.tokens(n_calls * B, D, torch.bfloat16, 99, DEV).view(n_calls, B, D)
     y = torch.empty((n_calls, B, D), dtype=torch.float32, device=DEV)
@@ -101,12 +103,17 @@ def run(out_path, quick=False, only=None, n_calls=None):
         b = syn.gate_bias_for_sparsity(s)
         sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in base]
         add(f"decode 4096x14336 s={s}", D, H, 1, sets, std, "relu", peak=peak)
+        if s == 0.9:  # double activation (RELU on the up projection as well): same rows read, one more epilogue op
+            add(f"decode 4096x14336 s={s} double activation", D, H, 1, sets, std, "relu", peak=peak, act_up="relu")
     # batched decode under Zipf firing
     p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
     zb = syn.bias_from_firing_profile(p).to(DEV)
     zsets = [dict(w, b_g=zb) for w in base]
     for B in ((16,) if quick else (4, 16, 64)):
         add(f"batched zipf B={B}", D, H, B, zsets, std, "relu", n_calls=100, peak=peak)
+        if B == 16:
+            add(f"batched zipf B={B} double activation", D, H, B, zsets, std, "relu", n_calls=100, peak=peak,
+                act_up="relu")
     # LoPA gates (up/down weights shared with the standard sets)
     gi = g_diagonal(H, D, DEV)
     for r in ((512,) if quick else (256, 512, 1024)):

@@ -24,9 +24,9 @@ def gate_dict_to_oracle(gate):
                           use_rmsnorm=gate.get("use_rmsnorm", True), eps=gate.get("rms_eps", 1e-5)))
 
 
-def run_oracle(x, gate, b_g, W_up, W_down, act, route="sparse", threads=8):
+def run_oracle(x, gate, b_g, W_up, W_down, act, route="sparse", threads=8, act_up=None):
     return oracle.ffn(host(x), host(W_up), host(W_down), act, b_g=host(b_g), route=route,
-                      threads=threads, **gate_dict_to_oracle(gate))
+                      threads=threads, act_up=act_up, **gate_dict_to_oracle(gate))
 
 
 def assert_y_close(y_gpu, y_ref, rel_l2=REL_L2, max_abs=MAX_ABS, what=""):

@@ -260,6 +260,43 @@ def test_batched_empty_and_full_union(mod):
     assert_y_close(y, ref["y"], what="batched, full union")
 
 
+# ------------------------------------------------------------------ double activation (Sec. 3.3)
+@pytest.mark.parametrize("act,act_up", [("relu", "relu"), ("sqrelu", "rsplus"), ("rsplus", "sqrelu")])
+def test_double_activation_all_paths(mod, act, act_up):
+    D, H = 512, 1100
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=64, B_max=8)
+    ffn.set_up_activation(act_up)
+    gate, w = make_std(D, H, torch.bfloat16, 61, 0.8)
+    x = syn.tokens(8, D, torch.bfloat16, 61, DEV)
+    ref1 = run_oracle(x[0], gate, w["b_g"], w["W_up"], w["W_down"], act, act_up=act_up)
+    assert 0 < ref1["n_gated"][0] < ref1["n_act"][0]                    # A_3 really removes neurons
+    for path in ("general", "fused"):                                   # one token
+        ffn.set_path(path)
+        y = ffn.sparse_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], act)
+        assert_y_close(y, ref1["y"], what=f"double activation {act}/{act_up} [{path}]")
+        assert_active_set(ffn.last_active(), ref1, what=f"double activation [{path}]")   # the list is the gate's
+        yd = ffn.dense_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], act)
+        assert_y_close(yd, ref1["y"], what=f"double activation dense [{path}]")
+    ref8 = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], act, act_up=act_up)
+    for path in ("general", "mma_sync", "auto"):                        # a batch: CUDA cores, mma.sync, tcgen05
+        ffn.set_path(path)
+        y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], act)
+        assert_y_close(y, ref8["y"], what=f"double activation batch [{path}]")
+    # LoPA gate, one token and a batch
+    lg, lw = make_lopa(mod, D, H, 64, torch.bfloat16, 62, 0.8, "diag")
+    ffn.set_path("auto")
+    for xs in (x[1], x[:5]):
+        ref = run_oracle(xs, lg, lw["b_g"], lw["W_up"], lw["W_down"], act, act_up=act_up)
+        y = ffn.sparse_ffn_forward(xs, lg, lw["b_g"], lw["W_up"], lw["W_down"], act)
+        assert_y_close(y, ref["y"], what="double activation, LoPA gate")
+    # back to Eq. 1
+    ffn.set_up_activation(None)
+    y = ffn.sparse_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], act)
+    assert_y_close(y, run_oracle(x[0], gate, w["b_g"], w["W_up"], w["W_down"], act)["y"], what="act_up reset")
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
+
+
 # ------------------------------------------------------------------ full-size configurations
 def test_config2_full_size_decode(mod):
     D, H = 4096, 14336
