@@ -187,6 +187,14 @@ int sparse_ffn_forward_static(const void* x, const void* W_g, const float* b_g, 
  * returned on the calling thread; "cudaSuccess" if there was none.  Diagnostics only. */
 const char* sffn_last_cuda_error(void);
 
+/* Glue for a layer loop (not a step of the paper's FFN): out[i] = dtype(resid[i] + alpha * y[i]) for the n
+ * elements (a multiple of 4) of an fp32 FFN output y, e.g. the residual stream's update and its cast back to
+ * the token dtype.  Device pointers, 16-byte aligned; out may alias resid.  The kernel takes part in the
+ * programmatic dependent launch chain of the FFN kernels, so a loop FFN -> this -> FFN runs without the
+ * full serialisation a foreign elementwise kernel would put between two calls. */
+int sffn_residual_cast(const float* y, const void* resid, float alpha, void* out, int n, int dtype /* sffn_dtype */,
+                       void* stream);
+
 /* Static string for a status code. */
 const char* sffn_status_string(int status);
 

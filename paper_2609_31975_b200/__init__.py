@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     SparseFFN,
     lib_path,
     load_library,
+    residual_cast,
     sparse_ffn_forward_static,
 )
 from .lopa import g_diagonal, g_tiled, touched_bytes, dense_bytes  # noqa: F401

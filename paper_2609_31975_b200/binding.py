@@ -61,6 +61,7 @@ def load_library() -> ctypes.CDLL:
         lib.sffn_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
         lib.sparse_ffn_forward_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, vp]
         lib.sffn_status_string.argtypes = [i]
+        lib.sffn_residual_cast.argtypes = [vp, vp, ctypes.c_float, vp, i, i, vp]
         lib.sffn_status_string.restype = ctypes.c_char_p
         lib.sffn_last_cuda_error.argtypes = []
         lib.sffn_last_cuda_error.restype = ctypes.c_char_p
@@ -94,6 +95,17 @@ def sparse_ffn_forward_static(x, W_g, b_g, W_up, W_down, act="relu", y=None, str
                                          ACT[act] if isinstance(act, str) else int(act), _ptr(y),
                                          ctypes.c_void_p(s.cuda_stream)))
     return y
+
+
+def residual_cast(y, resid, alpha, out, stream=None):
+    """out = dtype(resid + alpha * y) for an fp32 FFN output ``y`` (glue between the FFN calls of a layer loop)."""
+    lib = load_library()
+    assert y.dtype == torch.float32 and resid.dtype == out.dtype and y.numel() == resid.numel() == out.numel()
+    s = stream if stream is not None else torch.cuda.current_stream(y.device)
+    _check("sffn_residual_cast",
+           lib.sffn_residual_cast(_ptr(y), _ptr(resid), float(alpha), _ptr(out), y.numel(),
+                                  1 if out.dtype == torch.bfloat16 else 0, ctypes.c_void_p(s.cuda_stream)))
+    return out
 
 
 class SparseFFN:

@@ -541,6 +541,13 @@ int sparse_ffn_forward_host(sffn_handle* h, const void* x_host, int B, const sff
   return SFFN_OK;
 }
 
+int sffn_residual_cast(const float* y, const void* resid, float alpha, void* out, int n, int dtype, void* stream) {
+  if (!y || !resid || !out || n < 4 || n % 4 || (dtype != SFFN_F32 && dtype != SFFN_BF16)) return SFFN_ERR_INVALID_ARG;
+  if (!aligned16(y) || !aligned16(resid) || !aligned16(out)) return SFFN_ERR_UNSUPPORTED;
+  SFFN_CUDA(sffn::launch_residual_cast(dtype == SFFN_BF16, y, resid, alpha, out, n, static_cast<cudaStream_t>(stream)));
+  return SFFN_OK;
+}
+
 int sffn_last_active(sffn_handle* h, const int32_t** idx_dev, const int32_t** count_dev, void* stream) {
   if (!h || !idx_dev || !count_dev) return SFFN_ERR_INVALID_ARG;
   if (h->list_state == 0) return SFFN_ERR_INVALID_ARG;

@@ -359,6 +359,35 @@ __global__ void __launch_bounds__(256) copy16_kernel(const uint4* src, uint4* ds
   for (size_t i = i0 + 4 * stride; i < n16; i += stride) dst[i] = src[i];
 }
 
+// Glue between two FFN calls of a layer loop: out = T(resid + alpha * y), four elements per thread.
+template <typename T>
+__global__ void __launch_bounds__(256) residual_cast_kernel(const float* y, const T* resid, float alpha, T* out, int n4) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4 v = reinterpret_cast<const float4*>(y)[i];
+  float r[4];
+  if (sizeof(T) == 4) {
+    const float4 q = reinterpret_cast<const float4*>(resid)[i];
+    r[0] = q.x; r[1] = q.y; r[2] = q.z; r[3] = q.w;
+  } else {
+    const uint2 q = reinterpret_cast<const uint2*>(resid)[i];
+    r[0] = __uint_as_float(q.x << 16); r[1] = __uint_as_float(q.x & 0xffff0000u);
+    r[2] = __uint_as_float(q.y << 16); r[3] = __uint_as_float(q.y & 0xffff0000u);
+  }
+  const float o[4] = {fmaf(alpha, v.x, r[0]), fmaf(alpha, v.y, r[1]), fmaf(alpha, v.z, r[2]), fmaf(alpha, v.w, r[3])};
+  if (sizeof(T) == 4) {
+    reinterpret_cast<float4*>(out)[i] = make_float4(o[0], o[1], o[2], o[3]);
+  } else {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(o[0], o[1]), hi = __floats2bfloat162_rn(o[2], o[3]);
+    uint2 w;
+    w.x = *reinterpret_cast<const uint32_t*>(&lo);
+    w.y = *reinterpret_cast<const uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(out)[i] = w;
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Host-side launchers.
 template <typename T, typename VT, int NB>
@@ -435,6 +464,17 @@ int updown_max_tokens(bool bf16, int D) {
 
 cudaError_t launch_updown(bool bf16, int nb, const UpDownParams& p, int grid, cudaStream_t s) {
   return bf16 ? launch_updown_d<__nv_bfloat16>(p, nb, grid, s) : launch_updown_d<float>(p, nb, grid, s);
+}
+
+cudaError_t launch_residual_cast(bool bf16, const float* y, const void* resid, float alpha, void* out, int n,
+                                 cudaStream_t s) {
+  const int n4 = n / 4;
+  const dim3 grid((n4 + 255) / 256);
+  if (bf16)
+    return launch_pdl(residual_cast_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, y,
+                      static_cast<const __nv_bfloat16*>(resid), alpha, static_cast<__nv_bfloat16*>(out), n4);
+  return launch_pdl(residual_cast_kernel<float>, grid, dim3(256), 0, s, y, static_cast<const float*>(resid), alpha,
+                    static_cast<float*>(out), n4);
 }
 
 cudaError_t launch_copy16(const void* src, void* dst, size_t bytes, cudaStream_t s) {

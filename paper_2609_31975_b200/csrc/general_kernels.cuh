@@ -46,6 +46,8 @@ cudaError_t launch_compact(const uint8_t* flag, int H, int32_t* idx, int32_t* co
 // Largest token chunk (4, 2 or 0 = unsupported D) the up/down kernel takes at this D.
 int updown_max_tokens(bool bf16, int D);
 cudaError_t launch_updown(bool bf16, int nb, const UpDownParams& p, int grid, cudaStream_t s);
+cudaError_t launch_residual_cast(bool bf16, const float* y, const void* resid, float alpha, void* out, int n,
+                                 cudaStream_t s);
 cudaError_t launch_copy16(const void* src, void* dst, size_t bytes, cudaStream_t s);
 cudaError_t launch_reduce(const float* partial, int G, int NB, int D, float* y, int y_stride,
                           cudaStream_t s);
