@@ -84,6 +84,20 @@ inline bool& pdl_enabled() {
   return on;
 }
 
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute belongs to the device's copy of
+// the kernel); `done` holds one bit per device ordinal.
+template <typename K>
+cudaError_t allow_dynamic_smem(K kernel, int bytes, unsigned long long& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (done & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) done |= bit;
+  return e;
+}
+
 // Launch with the programmatic-stream-serialisation attribute: the kernel may begin while its
 // predecessor in the stream is still running; its griddepcontrol.wait restores the ordering.
 template <typename... KArgs, typename... Args>

@@ -639,6 +639,7 @@ __global__ void __launch_bounds__(256) fused_reduce_kernel(const float* partial,
   if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)G * 16 + blockIdx.x] = global_ns();
   pdl_wait();
   if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)(G + 1) * 16 + blockIdx.x] = global_ns();
+  const int32_t failed = __ldcg(status);  // in flight together with the partials, not after them
   const int Q = D / 4;
   const int q = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int l = threadIdx.x & 31;
@@ -662,7 +663,7 @@ __global__ void __launch_bounds__(256) fused_reduce_kernel(const float* partial,
     s.y = warp_sum(s.y);
     s.z = warp_sum(s.z);
     s.w = warp_sum(s.w);
-    if (l == 0 && *status == 0) reinterpret_cast<float4*>(y)[q] = s;
+    if (l == 0 && failed == 0) reinterpret_cast<float4*>(y)[q] = s;
   }
   if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)(G + 2) * 16 + blockIdx.x] = global_ns();
 }
@@ -744,13 +745,10 @@ cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaS
     case 4: k = fused_ffn_kernel<T, 4, LOPA>; break;
     default: k = fused_ffn_kernel<T, 8, LOPA>; break;
   }
-  static bool configured[4] = {false, false, false, false};
+  static unsigned long long configured[4] = {0, 0, 0, 0};  // per instantiation of this template, per row width
   const int slot = g.cpt == 1 ? 0 : g.cpt == 2 ? 1 : g.cpt == 4 ? 2 : 3;
-  if (!configured[slot]) {
-    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-    if (e != cudaSuccess) return e;
-    configured[slot] = true;
-  }
+  const cudaError_t e = allow_dynamic_smem(k, kSmemBudget, configured[slot]);
+  if (e != cudaSuccess) return e;
   return launch_pdl(k, dim3(grid), dim3(kThreads), (size_t)g.smem, s, p);
 }
 

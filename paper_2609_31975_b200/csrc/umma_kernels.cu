@@ -825,22 +825,16 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
   if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : tile_rows_for(p.R, grid))) return cudaErrorNotSupported;
   // tokens: only the rows that exist; the box covers npad rows and the rest reads as zero
   if (!make_map(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)) return cudaErrorNotSupported;
-  static bool configured[2] = {false, false};
+  static unsigned long long configured[2] = {0, 0};
   if (up) {
     auto k = umma_rows_kernel<true>;
-    if (!configured[1]) {
-      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return e;
-      configured[1] = true;
-    }
+    const cudaError_t e = allow_dynamic_smem(k, 227 * 1024, configured[1]);
+    if (e != cudaSuccess) return e;
     return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x);
   } else {
     auto k = umma_rows_kernel<false>;
-    if (!configured[0]) {
-      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return e;
-      configured[0] = true;
-    }
+    const cudaError_t e = allow_dynamic_smem(k, 227 * 1024, configured[0]);
+    if (e != cudaSuccess) return e;
     return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x);
   }
 }
@@ -869,12 +863,9 @@ cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s) {
   if (!make_map(&map_wt, p.W_down, p.D, p.R, (size_t)p.D, kAtomK)) return cudaErrorNotSupported;
   // HmT [B][hm_stride]: inner dimension u; token rows past B read as zero
   if (!make_map(&map_hm, p.hmT, p.hm_stride, p.B, (size_t)p.hm_stride, p.npad)) return cudaErrorNotSupported;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(umma_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static unsigned long long configured = 0;
+  const cudaError_t e = allow_dynamic_smem(umma_down_kernel, 113 * 1024, configured);
+  if (e != cudaSuccess) return e;
   return launch_pdl(umma_down_kernel, dim3(grid), dim3(kThreads), smem, s, p, map_wg, map_wt, map_hm);
 }
 
