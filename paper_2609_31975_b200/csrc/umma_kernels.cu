@@ -1,26 +1,31 @@
 // Batched path on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM), bf16 storage.
 //
 //   umma_rows_kernel<GATE>  Z[H, B] = W[H, K] X[B, K]^T + bias (+ fixed-matrix term), activation, gate values,
-//                           "any token fires" flag per neuron            (Eq. 1 gate / LoPA U stage, batched)
-//   umma_rows_kernel<UP>    over the union list of fired neurons (Sec. 5.4): Up = W_up[idx] X^T, Hm = a . Up,
-//                           stored as bf16 HmT[b][u] for the down projection
+//                           "any token fires" bit per neuron             (Eq. 1 gate / LoPA U and V stages, batched)
+//   umma_rows_kernel<UP>    compacts those bits into the union list of fired neurons (Sec. 5.4), then over that
+//                           list: Up = W_up[idx] X^T, Hm = a . A_3(Up), stored as bf16 HmT[b][u]
+//   umma_down_kernel        partial[split][b][d] = sum over the split's list rows u of HmT[b][u] W_down[idx[u]][d]
+//   rmsnorm_split_kernel    LoPA: n = RMSNorm(v) as bf16 high / low pairs (the B operand of the U stage)
 //
-// One CTA owns a tile of up to 128 weight rows (TMEM lanes) x Npad token columns (Npad = columns rounded up to 16):
-//   warps 0-3  producers, one stage per warp in turn: TMA tensor-map copies bring the tile's weight rows and the
-//              Npad token rows of the current 64-wide K block into the 128-byte-swizzled K-major layout the
-//              tensor core reads (mbarrier complete_tx).  Gate: one tiled copy of the tile's consecutive rows.
-//              Union rows: tile::gather4, each lane of the warp fetching four listed rows.
-//   warps 8-11 one thread each issues tcgen05.mma (M=128, N=Npad, K=16, four per stage) for "its" ring slots
-//              into an accumulator of its own and commits each stage's completion to the "slot free" mbarrier.
-//              The serial wait - issue - commit chain of one thread takes on the order of a thousand cycles
-//              per stage whatever the MMA shape, so several issuers (four when the ring has eight or more
-//              slots, else two) are what lets the copies run at memory speed; warp 8 allocates and frees
-//              the TMEM columns
-//   warps 4-7  epilogue: tcgen05.ld the accumulator row of "their" neuron (all accumulators added), apply
-//              the gate / scale epilogue
-// A tile has 128 rows when a CTA owns several tiles; a smaller problem is cut into one tile per SM.
-// Every wait is bounded by a cycle budget; on expiry the status word is set, all roles wind down, the
-// producers drain their copies and the TMEM columns are released before the CTA exits.
+// Rows kernels: one CTA owns a tile of up to 128 weight rows (TMEM lanes) x Npad token columns (Npad = columns
+// rounded up to 16); tiles of up to 64 rows use M = 64:
+//   warps 0-3  producers: TMA tensor-map copies bring the tile's weight rows and the Npad token rows of a stage's
+//              64-wide K blocks into the 128-byte-swizzled K-major layout the tensor core reads (mbarrier
+//              complete_tx).  Gate: one tiled copy of the tile's consecutive rows per block.  Union rows:
+//              tile::gather4, each lane of the warp fetching four listed rows.
+//   warps 8-11 one thread each issues tcgen05.mma (N=Npad, K=16, four per K block) for "its" ring slots into an
+//              accumulator of its own and commits each stage's completion to the "slot free" mbarrier.  The serial
+//              wait - issue - commit chain of one thread takes on the order of a thousand cycles per stage whatever
+//              the MMA shape, so several issuers (four when the ring divides evenly among them, else two) are what
+//              lets the copies run at memory speed; warp 8 allocates and frees the TMEM columns
+//   warps 4-7  epilogue: tcgen05.ld the accumulator row of "their" neuron (all accumulators added), apply the
+//              gate / scale epilogue; for wide batches all twelve warps share the epilogue of the CTA's last tile
+// A tile has 128 rows when a CTA owns several tiles; a smaller problem is cut into one tile per SM.  The ring of
+// stages (up to 12) is cut out of the dynamic shared memory on the device, once the tile height is known.
+// Every kernel here is launched with programmatic dependent launch: set-up first, griddepcontrol.wait before the
+// first dependent read or global write.
+// Every wait is bounded by a cycle budget; on expiry the status word is set, all roles wind down and the TMEM
+// columns are released before the CTA exits.
 #include "umma_kernels.cuh"
 
 #include <cuda.h>
