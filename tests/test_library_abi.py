@@ -43,6 +43,14 @@ def test_host_side_validation_without_a_gpu():
     assert lib.sffn_create(ctypes.byref(h), 4096, 14336, 0, 1, 1, None, 0) == 3         # no workspace
     assert lib.sffn_status_string(5) == b"device-side bounded wait ran out"
     assert lib.sparse_ffn_forward(None, None, 1, None, None, None, None, 0, None, None) == 1
+    assert lib.sffn_set_up_activation(None, 0) == 1                                      # no handle
+    buf = (ctypes.c_float * 8)()
+    p = ctypes.cast(buf, ctypes.c_void_p)
+    assert lib.sffn_residual_cast(None, p, 1.0, p, 8, 0, None) == 1                      # null y
+    assert lib.sffn_residual_cast(p, p, 1.0, p, 6, 0, None) == 1                         # n not a multiple of 4
+    assert lib.sffn_residual_cast(p, p, 1.0, p, 8, 5, None) == 1                         # bad dtype
+    assert lib.sffn_residual_cast(p, ctypes.c_void_p(p.value + 4), 1.0, p, 4, 0, None) == 2   # misaligned
+    assert lib.sffn_last_cuda_error() == b"cudaSuccess"
 
 
 def test_product_index_generators_match_the_oracle_restatement():
