@@ -36,7 +36,7 @@ Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
     off = align_up(off + bytes, 256);
     return o;
   };
-  L.status = take(256);  // [0] device status, [1] length of idx
+  L.status = take(256);  // [0] device status, [1] length of idx, [2] batched path: every row was walked
   L.act = take((size_t)B_max * H * 4);
   L.flag = take((size_t)2 * H + 256);  // bytes [H], or the tcgen05 gate's bit masks (16 bytes per tile of >= 8 rows)
   L.idx = take(((size_t)H + 64) * 4);  // readable one 64-row block past the list
@@ -320,7 +320,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       if (own_list) {
         p.words_in = words; p.n_words = 4 * gate_tiles; p.gate_tile_rows = gate_tile_rows;
         p.gate_rows_per_word = gate_tile_rows <= 64 ? 16 : 32;
-        p.idx_out = idx; p.count_out = count;
+        p.idx_out = idx; p.count_out = count; p.walk_all = umma_may_walk(nb) ? count + 1 : nullptr;
       } else {
         p.idx = lidx; p.count = lcount;
       }
@@ -345,6 +345,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       d.idx = lidx; d.count = lcount;
       d.hmT = hmT; d.hm_stride = h->L.hm_stride; d.B = nb;
       d.splits = nsplit = umma_down_splits(D, h->sm_count, kMaxSplits);
+      d.walk_all = (own_list && umma_may_walk(nb)) ? count + 1 : nullptr;
       d.partial = partial; d.status = h->at<int32_t>(h->L.status);
       SFFN_CUDA(launch_umma_down(d, s));
     } else {

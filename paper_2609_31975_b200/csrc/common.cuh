@@ -14,12 +14,16 @@ constexpr int kActNone = 3;  // identity: internal stages that only need the raw
 
 // Activation of the gate (activation table of Sec. 3.1; squared RELU from the activation study).
 // For all three, A(z) != 0 exactly when z > 0 in exact arithmetic; callers test z > 0.
+// The R-S+ branch is kept out of line: `act` is the same for every thread, so the cheap activations then cost a
+// compare and a max per element instead of a speculated exponential and division.
+static __device__ __noinline__ float rsplus_of_nonnegative(float p) { return p / (1.f + __expf(-p)); }
+
 __device__ __forceinline__ float activation(int act, float z) {
   if (act == kActNone) return z;
-  if (!(z > 0.f)) return 0.f;
-  if (act == kActRelu) return z;
-  if (act == kActSqRelu) return z * z;
-  return z / (1.f + __expf(-z));  // R-S+: z * sigmoid(z) on the non-negative side
+  const float p = fmaxf(z, 0.f);                 // 0 for z <= 0
+  if (act == kActRelu) return p;
+  if (act == kActSqRelu) return p * p;
+  return rsplus_of_nonnegative(p);               // R-S+: z * sigmoid(z) on the non-negative side, 0 at 0
 }
 
 // Element traits: 16-byte vectors of the storage type, unpacked to fp32.

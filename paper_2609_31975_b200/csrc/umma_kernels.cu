@@ -46,6 +46,8 @@ constexpr int kThreads = 320;                        // 4 producer warps, 4 epil
 constexpr int kThreadsRows = 384;                    // rows kernels: up to 4 MMA warps
 constexpr int kProducerWarps = 4;
 constexpr int kMaxStages = 12;
+constexpr int kWalkMinTokens = 32;                   // batches from which the up kernel may walk every row
+constexpr int kWalkAllPercent = 70;                  // union share of the rows from which "every row" is walked
 constexpr int kMaxIssuers = 4;
 constexpr int kScanChunks = 4;                       // in-kernel compaction: up to 4 * 384 mask words = 384 gate tiles
 constexpr int kMaxOwnTiles = 8;                      // tiles of one CTA whose rows are kept in shared memory
@@ -189,10 +191,26 @@ __host__ __device__ inline uint32_t tmem_cols_for(int cols) {
   return cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
 }
 
-template <bool UP>
+// Third tensor map of the up kernel that may walk every row (tiled boxes over all rows); empty otherwise, so
+// that the other instantiations keep their two-map signature.
+template <bool HAS>
+struct WalkMap {
+  CUtensorMap m;
+  __device__ const CUtensorMap* get() const { return &m; }
+};
+template <>
+struct WalkMap<false> {
+  __device__ const CUtensorMap* get() const { return nullptr; }
+};
+
+enum RowsMode { kGate = 0, kUp = 1, kUpMayWalk = 2 };  // kUpMayWalk: wide batches, see walk_all below
+
+template <int MODE>
 __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRowsParams p,
                                                                   const __grid_constant__ CUtensorMap map_w,
-                                                                  const __grid_constant__ CUtensorMap map_x) {
+                                                                  const __grid_constant__ CUtensorMap map_x,
+                                                                  const __grid_constant__ WalkMap<MODE == kUpMayWalk> map_t) {
+  constexpr bool UP = MODE != kGate;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   // carve: stages first (1024-byte aligned), then barriers and control words
   const int npad = p.npad;
@@ -279,9 +297,37 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   } else {
     n_rows = p.count ? *p.count : p.R;
   }
+  // A union that covers most of the rows is cheaper to walk as "every row" with tiled copies (which stream about
+  // 1.5x faster than gathered rows) than as a list: unfired rows have a = 0 for every token, so their h is 0.
+  // The list and its length are still published; the down kernel is told through *walk_all to do the same.
+  const int n_listed = n_rows;
+  const bool walk_all = MODE == kUpMayWalk && own_list && p.walk_all &&
+                        (long long)n_listed * 100 >= (long long)p.R * kWalkAllPercent;
+  if (walk_all) n_rows = p.R;
   const int tile_rows = tile_rows_for(n_rows, gridDim.x);
   const int n_tiles = (n_rows + tile_rows - 1) / tile_rows;
-  if (own_list) {
+  if (own_list && walk_all) {
+    // publish the list only: word w is written out by CTA w mod grid
+#pragma unroll
+    for (int k = 0; k < kScanChunks; ++k) {
+      const int w = k * kThreadsRows + tid;
+      if (k < nch && bits[k] && w % (int)gridDim.x == (int)blockIdx.x) {
+        const int j0 = (w >> 2) * p.gate_tile_rows + (w & 3) * p.gate_rows_per_word;
+        uint32_t rest = bits[k];
+        int li = first_pos[k];
+        while (rest) {
+          const int q = __ffs(rest) - 1;
+          rest &= rest - 1;
+          p.idx_out[li++] = j0 + q;
+        }
+      }
+    }
+    if (blockIdx.x == 0 && tid == 0) {
+      *p.count_out = n_listed;
+      *p.walk_all = 1;
+    }
+  } else if (own_list) {
+    if (blockIdx.x == 0 && tid == 0 && p.walk_all) *p.walk_all = 0;
     // keep the rows of this CTA's tiles in shared memory and publish them (and the length) for the
     // down projection and the caller: every list position belongs to exactly one CTA's tile
 #pragma unroll
@@ -358,7 +404,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     const int B = p.B;
     const int li = tile * tile_rows + row_in_tile;
     const bool row_ok = row_in_tile >= 0 && row_in_tile < tile_rows && li < n_rows;
-    const int j = !row_ok ? 0 : own_list ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
+    const int j = !row_ok ? 0 : (own_list && !walk_all) ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
     // everything that does not depend on the accumulator is fetched before the wait
     float bias = 0.f, sg = 1.f;
     int gi = -1;
@@ -384,6 +430,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     if (UP) {
       __nv_bfloat16* hm = static_cast<__nv_bfloat16*>(p.hmT) + li;
       const float* arow = p.a + j;
+      const int act_up = p.act_up;
       int g = 0;
       for (int c0 = 8 * part; c0 < npad; c0 += 8 * nparts, ++g) {
         float av[8];
@@ -395,7 +442,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
 #pragma unroll
         for (int q = 0; q < 8; ++q)
           if (row_ok && c0 + q < B)
-            hm[(size_t)(c0 + q) * p.hm_stride] = __float2bfloat16(av[q] * activation(p.act_up, v[q]));
+            hm[(size_t)(c0 + q) * p.hm_stride] = __float2bfloat16(av[q] * activation(act_up, v[q]));
       }
     } else {
       const int act = p.act;
@@ -457,14 +504,14 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       if ((s & (kProducerWarps - 1)) != warp) continue;
       const int na = min(atoms, kblocks - kb * atoms);
       const uint32_t tx_bytes = (uint32_t)(na * (tile_rows + npad)) * 128;
-      if (UP && tile != rows_of) {
+      if (UP && !walk_all && tile != rows_of) {
         rows_of = tile;
         ++own;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const int li = tile * tile_rows + lane * 4 + q;
           // rows beyond the list: any valid row, ignored later
-          r[q] = li >= n_rows ? 0 : own_list ? rows_sm[own * kTileRows + lane * 4 + q] : p.idx ? p.idx[li] : li;
+          r[q] = li >= n_rows ? 0 : (own_list && !walk_all) ? rows_sm[own * kTileRows + lane * 4 + q] : p.idx ? p.idx[li] : li;
         }
       }
       int ok = 1;
@@ -477,9 +524,11 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       const uint32_t abase = stage0 + s * stage_bytes;
       for (int a = 0; a < na; ++a) {
         const int k0 = (kb * atoms + a) * kAtomK;
-        if (UP) {
+        if (UP && !walk_all) {
           if (lane * 4 < tile_rows)
             tma_gather4(abase + a * a_block_bytes + lane * 512, &map_w, k0, r[0], r[1], r[2], r[3], full + 8 * s);
+        } else if (UP) {
+          if (lane == 0) tma_tile_2d(abase + a * a_block_bytes, map_t.get(), k0, tile * tile_rows, full + 8 * s);
         } else if (lane == 0) {
           tma_tile_2d(abase + a * a_block_bytes, &map_w, k0, tile * tile_rows, full + 8 * s);
         }
@@ -618,7 +667,8 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
       mbar_init(empty + 8 * s, 1);
     }
     *abort_flag = 0;
-    asm volatile("prefetch.tensormap [%0];" ::"l"(p.idx ? &map_wg : &map_wt) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_wg) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_wt) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hm) : "memory");
   }
   if (warp == 8) {
@@ -629,7 +679,11 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
   }
   pdl_wait();
 
-  const int n_rows = p.count ? *p.count : p.R;
+  // both words are fetched at once (one round trip), then combined
+  const int listed = p.count ? __ldcg(p.count) : p.R;
+  const int walk_word = p.walk_all ? __ldcg(p.walk_all) : 0;
+  const bool walk_all = p.idx == nullptr || walk_word != 0;  // every row, not the list
+  const int n_rows = walk_all ? p.R : listed;
   // the split's share of the list, in blocks of 64 rows
   const int total_blocks = (n_rows + kAtomK - 1) / kAtomK;
   const int per_split = (total_blocks + p.splits - 1) / p.splits;
@@ -655,7 +709,7 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
       if ((s & (kProducerWarps - 1)) != warp) continue;
       const int u0 = (kb0 + kb) * kAtomK;
       int r[4] = {0, 0, 0, 0};
-      if (p.idx) {
+      if (!walk_all) {
         // four list entries of this lane (the list buffer is readable past its length; entries there are
         // replaced by row 0, whose products vanish against the zeroed tail of HmT)
         const int u = u0 + quad * 4;
@@ -673,7 +727,7 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       const uint32_t abase = stage0 + s * stage_bytes;
-      if (p.idx) {
+      if (!walk_all) {
         tma_gather4(abase + half * 8192 + quad * 512, &map_wg, d0 + half * kAtomK, r[0], r[1], r[2], r[3], full + 8 * s);
       } else if (lane < 2) {
         // every row: 64 consecutive rows per column half; rows past the matrix read as zero
@@ -784,6 +838,8 @@ bool umma_own_list_supported(int R, int sm_count) {
   return 4 * nt <= kScanChunks * kThreadsRows && R <= (long long)kMaxOwnTiles * kTileRows * sm_count;
 }
 
+bool umma_may_walk(int B) { return B >= kWalkMinTokens; }
+
 bool umma_rows_supported(int K, int cols) { return K % kAtomK == 0 && K >= kAtomK && cols >= 1 && cols <= 128; }
 
 namespace {
@@ -830,18 +886,25 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
   if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : tile_rows_for(p.R, grid))) return cudaErrorNotSupported;
   // tokens: only the rows that exist; the box covers npad rows and the rest reads as zero
   if (!make_map(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)) return cudaErrorNotSupported;
-  static unsigned long long configured[2] = {0, 0};
-  if (up) {
-    auto k = umma_rows_kernel<true>;
-    const cudaError_t e = allow_dynamic_smem(k, 227 * 1024, configured[1]);
-    if (e != cudaSuccess) return e;
-    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x);
-  } else {
-    auto k = umma_rows_kernel<false>;
-    const cudaError_t e = allow_dynamic_smem(k, 227 * 1024, configured[0]);
-    if (e != cudaSuccess) return e;
-    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x);
+  static unsigned long long configured[3] = {0, 0, 0};
+  cudaError_t e;
+  if (!up) {
+    auto k = umma_rows_kernel<kGate>;
+    if ((e = allow_dynamic_smem(k, 227 * 1024, configured[0])) != cudaSuccess) return e;
+    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, WalkMap<false>{});
   }
+  if (p.walk_all && umma_may_walk(p.B)) {
+    // wide batches: the union may cover most rows; the kernel then walks every row with tiled boxes of the tile
+    // height of R rows (decided on the device from the union's size, so it depends on this call's inputs only)
+    WalkMap<true> map_t;
+    if (!make_map(&map_t.m, p.W, p.K, p.R, (size_t)p.K, tile_rows_for(p.R, grid))) return cudaErrorNotSupported;
+    auto k = umma_rows_kernel<kUpMayWalk>;
+    if ((e = allow_dynamic_smem(k, 227 * 1024, configured[2])) != cudaSuccess) return e;
+    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, map_t);
+  }
+  auto k = umma_rows_kernel<kUp>;
+  if ((e = allow_dynamic_smem(k, 227 * 1024, configured[1])) != cudaSuccess) return e;
+  return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, WalkMap<false>{});
 }
 
 int umma_down_splits(int D, int sm_count, int max_splits) {

@@ -20,6 +20,7 @@ struct UmmaRowsParams {
   int gate_rows_per_word;    //   rows covered by one mask word: 32 for gate tiles of more than 64 rows, else 16
   int32_t* idx_out;          //   ... and writes the ascending list
   int32_t* count_out;        //   ... and its length
+  int32_t* walk_all;         //   ... and 1 here when it walked every row instead of the list (the down kernel must too), else 0
   const void* X;         // token operand [cols][K] bf16, row stride x_stride (elements)
   int x_stride;
   int ncols_valid;
@@ -52,6 +53,7 @@ struct UmmaDownParams {
   int hm_stride;         // multiple of 64
   int B;
   int splits;            // the list is cut into this many runs of 64-row blocks
+  const int32_t* walk_all;  // device word: nonzero = walk every row of W_down instead of the list (set by the up kernel), or null
   float* partial;        // [splits][B][D]
   int32_t* status;
   int npad, stages;      // filled by the launcher
@@ -61,6 +63,8 @@ int umma_down_splits(int D, int sm_count, int max_splits);
 bool umma_down_supported(int D, int cols);
 cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s);
 bool umma_rows_supported(int K, int cols);
+// Batches wide enough for the up kernel to consider walking every row instead of the union list.
+bool umma_may_walk(int B);
 bool umma_own_list_supported(int R, int sm_count);
 void umma_gate_tiling(int R, int sm_count, int* tile_rows, int* n_tiles);
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s);
