@@ -23,6 +23,8 @@ __global__ void __launch_bounds__(256) rowdot_kernel(const RowDotParams p) {
   extern __shared__ float svec[];  // [NB][K]
   constexpr int EPV = Elem<T>::kPerVec;
   const int K = p.K;
+  pdl_launch_dependents();
+  pdl_wait();  // the vectors (and, for the gate, the flag / value buffers) belong to earlier kernels until here
   for (int b = 0; b < NB; ++b) {
     const VT* v = static_cast<const VT*>(p.vec) + (size_t)b * p.vec_stride;
     for (int k = threadIdx.x; k < K; k += blockDim.x) svec[b * K + k] = Elem<VT>::to_float(v[k]);
@@ -122,6 +124,8 @@ __global__ void __launch_bounds__(256) rowdot_kernel(const RowDotParams p) {
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* v, float* n, const float* gain,
                                                       int r, int stride, float eps) {
   __shared__ float red[8];
+  pdl_launch_dependents();
+  pdl_wait();
   const float* vb = v + (size_t)blockIdx.x * stride;
   float* nb = n + (size_t)blockIdx.x * stride;
   float ss = 0.f;
@@ -203,6 +207,8 @@ __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
   __shared__ int jbuf[16];
   constexpr int EPV = Elem<T>::kPerVec;
   const int D = p.D;
+  pdl_launch_dependents();
+  pdl_wait();
   for (int b = 0; b < NB; ++b) {
     const T* xb = static_cast<const T*>(p.x) + (size_t)b * p.x_stride;
     for (int k = threadIdx.x; k < D; k += blockDim.x) svec[b * D + k] = Elem<T>::to_float(xb[k]);
@@ -396,13 +402,12 @@ static cudaError_t launch_rowdot_t(const RowDotParams& p, bool gate, int grid, c
   if (gate) {
     auto k = rowdot_kernel<T, VT, NB, true>;
     if (smem > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    k<<<grid, 256, smem, s>>>(p);
+    return launch_pdl(k, dim3(grid), dim3(256), smem, s, p);
   } else {
     auto k = rowdot_kernel<T, VT, NB, false>;
     if (smem > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    k<<<grid, 256, smem, s>>>(p);
+    return launch_pdl(k, dim3(grid), dim3(256), smem, s, p);
   }
-  return cudaGetLastError();
 }
 
 template <typename T, typename VT>
@@ -427,8 +432,7 @@ cudaError_t launch_rowdot(bool bf16, bool vec_is_f32, int nb, bool gate, const R
 
 cudaError_t launch_rmsnorm(const float* v, float* n, const float* gain, int r, int stride, float eps,
                            int B, cudaStream_t s) {
-  rmsnorm_kernel<<<B, 256, 0, s>>>(v, n, gain, r, stride, eps);
-  return cudaGetLastError();
+  return launch_pdl(rmsnorm_kernel, dim3(B), dim3(256), 0, s, v, n, gain, r, stride, eps);
 }
 
 cudaError_t launch_compact(const uint8_t* flag, int H, int32_t* idx, int32_t* count, cudaStream_t s) {
@@ -440,8 +444,7 @@ static cudaError_t launch_updown_t(const UpDownParams& p, int grid, cudaStream_t
   const size_t smem = (size_t)NB * p.D * sizeof(float);
   auto k = updown_kernel<T, NB, CPT>;
   if (smem > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  k<<<grid, 512, smem, s>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(k, dim3(grid), dim3(512), smem, s, p);
 }
 
 template <typename T>
