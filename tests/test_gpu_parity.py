@@ -260,6 +260,31 @@ def test_batched_empty_and_full_union(mod):
     assert_y_close(y, ref["y"], what="batched, full union")
 
 
+def test_batched_calls_repeat_bit_for_bit(mod):
+    """Back-to-back calls chained by dependent launch, interleaved with other work on the same handle, must
+    give the same bits every time (ring phases, bit masks, list and partial buffers are reused across calls)."""
+    D, H = 512, 2500
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=64, B_max=33)
+    gate, w = make_std(D, H, torch.bfloat16, 45, 0.9)
+    gate2, w2 = make_std(D, H, torch.bfloat16, 46, 0.5)
+    lg, lw = make_lopa(mod, D, H, 64, torch.bfloat16, 47, 0.9, "diag")
+    for B in (33, 5, 1):
+        x = syn.tokens(B, D, torch.bfloat16, 45, DEV)
+        xs = x if B > 1 else x[0]
+        for g_, w_ in ((gate, w), (lg, lw)):
+            ref = ffn.sparse_ffn_forward(xs, g_, w_["b_g"], w_["W_up"], w_["W_down"], "relu").clone()
+            idx = ffn.last_active().clone()
+            for it in range(30):
+                if it % 3 == 0:
+                    ffn.dense_ffn_forward(xs, gate2, w2["b_g"], w2["W_up"], w2["W_down"], "sqrelu")
+                if it % 5 == 0:
+                    ffn.sparse_ffn_forward(x[0], gate2, w2["b_g"], w2["W_up"], w2["W_down"], "relu")
+                y = ffn.sparse_ffn_forward(xs, g_, w_["b_g"], w_["W_up"], w_["W_down"], "relu")
+                assert torch.equal(y, ref), f"B={B} repeat {it}"
+            assert torch.equal(ffn.last_active(), idx)
+    assert ffn.device_status() == 0
+
+
 # ------------------------------------------------------------------ double activation (Sec. 3.3)
 @pytest.mark.parametrize("act,act_up", [("relu", "relu"), ("sqrelu", "rsplus"), ("rsplus", "sqrelu")])
 def test_double_activation_all_paths(mod, act, act_up):
