@@ -30,6 +30,13 @@
  * must be a multiple of 16 bytes (D and r multiples of 8 for bf16, of 4 for fp32), otherwise
  * SFFN_ERR_UNSUPPORTED.
  *
+ * Stream order: a call is ordered after everything queued before it on `stream` as far as x, the workspace
+ * and y are concerned.  The weights and per-neuron gate parameters (W_g, W_up, W_down, V, U, b_g, g_idx,
+ * g_sign, rms_gain) are treated as parameters: the kernels may start reading them while the work queued
+ * just before the call is still running (that is how back-to-back calls overlap), so they must not be
+ * written by device work queued immediately before a call on the same stream -- put a stream or event
+ * synchronisation between an update of the weights and the next call.
+ *
  * Errors: every entry point returns an sffn_status.  The return value covers host-side validation
  * and launch errors only; calls are asynchronous on `stream`.  Conditions detected on the device
  * (a bounded wait that ran out) are recorded in a status word inside the workspace and read back

@@ -248,7 +248,10 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  pdl_wait();
+  // The up kernel needs the gate's results from here on.  The gate kernel's tiles depend on nothing but its
+  // own arguments, and its weights are parameters: its producers fill the ring before they wait (see below),
+  // every other role of it waits just before its first dependent access.
+  if (MODE != kGate) pdl_wait();
 
   // Union rows: either the list is given (idx, count), or every CTA compacts the gate's "fired" bit masks
   // itself.  The gate kernel leaves one 32-bit word per epilogue warp and tile (word 4 * tile + warp, bit =
@@ -406,6 +409,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     const bool row_ok = row_in_tile >= 0 && row_in_tile < tile_rows && li < n_rows;
     const int j = !row_ok ? 0 : (own_list && !walk_all) ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
     // everything that does not depend on the accumulator is fetched before the wait
+    if (MODE == kGate) pdl_wait();  // before the first read of a buffer an earlier kernel may write, and the first store
     float bias = 0.f, sg = 1.f;
     int gi = -1;
     float pre[16];  // union rows: the gate values of this thread's first two column groups
@@ -491,49 +495,66 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     // which a parity wait could not tell from "ready".  Lane 0 waits for the slot and announces the byte
     // count, then the copies go out: one tiled copy for the tile's consecutive rows (gate), or one
     // gather4 per lane for four listed rows each (union rows); the token block is one more tiled copy.
-    int s = 0, ph = 0, kb = 0, tile = blockIdx.x;   // kb counts stages of the tile here
-    int rows_of = -1, own = -1;   // own: index of the current tile among this CTA's tiles
-    int r[4] = {0, 0, 0, 0};
-    for (; tile < n_tiles; ++s, ++kb) {
-      if (s == S) { s = 0; ph ^= 1; }
-      if (kb == kstages) {
-        kb = 0;
-        tile += gridDim.x;
-        if (tile >= n_tiles) break;
-      }
-      if ((s & (kProducerWarps - 1)) != warp) continue;
-      const int na = min(atoms, kblocks - kb * atoms);
-      const uint32_t tx_bytes = (uint32_t)(na * (tile_rows + npad)) * 128;
-      if (UP && !walk_all && tile != rows_of) {
-        rows_of = tile;
-        ++own;
+    const int my_tiles = (int)blockIdx.x < n_tiles ? (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int total = my_tiles * kstages;
+    // Stages [it0, it1) of this CTA's sequence; with_w / with_x say which of the two operands are copied.  A
+    // stage is armed (slot waited for, byte count announced) together with its weight copy.
+    auto produce = [&](int it0, int it1, bool with_w, bool with_x) -> bool {
+      int s = it0 % S, ph = (it0 / S) & 1, kb = it0 % kstages, tl = it0 / kstages;
+      int rows_of = -1;
+      int r[4] = {0, 0, 0, 0};
+      for (int it = it0; it < it1; ++it, ++s, ++kb) {
+        if (s == S) { s = 0; ph ^= 1; }
+        if (kb == kstages) { kb = 0; ++tl; }
+        if ((s & (kProducerWarps - 1)) != warp) continue;
+        const int tile = blockIdx.x + tl * gridDim.x;
+        const int na = min(atoms, kblocks - kb * atoms);
+        const uint32_t tx_bytes = (uint32_t)(na * (tile_rows + npad)) * 128;
+        if (UP && !walk_all && tl != rows_of) {
+          rows_of = tl;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int li = tile * tile_rows + lane * 4 + q;
-          // rows beyond the list: any valid row, ignored later
-          r[q] = li >= n_rows ? 0 : (own_list && !walk_all) ? rows_sm[own * kTileRows + lane * 4 + q] : p.idx ? p.idx[li] : li;
+          for (int q = 0; q < 4; ++q) {
+            const int li = tile * tile_rows + lane * 4 + q;
+            // rows beyond the list: any valid row, ignored later
+            r[q] = li >= n_rows ? 0 : own_list ? rows_sm[tl * kTileRows + lane * 4 + q] : p.idx ? p.idx[li] : li;
+          }
+        }
+        if (with_w) {
+          int ok = 1;
+          if (lane == 0) {
+            ok = mbar_wait(empty + 8 * s, ph ^ 1, abort_flag, p.status) ? 1 : 0;
+            if (ok) mbar_expect_tx(full + 8 * s, tx_bytes);
+          }
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) return false;
+        }
+        const uint32_t abase = stage0 + s * stage_bytes;
+        for (int a = 0; a < na; ++a) {
+          const int k0 = (kb * atoms + a) * kAtomK;
+          if (with_w) {
+            if (UP && !walk_all) {
+              if (lane * 4 < tile_rows)
+                tma_gather4(abase + a * a_block_bytes + lane * 512, &map_w, k0, r[0], r[1], r[2], r[3], full + 8 * s);
+            } else if (UP) {
+              if (lane == 0) tma_tile_2d(abase + a * a_block_bytes, map_t.get(), k0, tile * tile_rows, full + 8 * s);
+            } else if (lane == 0) {
+              tma_tile_2d(abase + a * a_block_bytes, &map_w, k0, tile * tile_rows, full + 8 * s);
+            }
+          }
+          if (with_x && lane == 0) tma_tile_2d(abase + b_off + a * b_block_bytes, &map_x, k0, 0, full + 8 * s);
         }
       }
-      int ok = 1;
-      if (lane == 0) {
-        ok = mbar_wait(empty + 8 * s, ph ^ 1, abort_flag, p.status) ? 1 : 0;
-        if (ok) mbar_expect_tx(full + 8 * s, tx_bytes);
-      }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      const uint32_t abase = stage0 + s * stage_bytes;
-      for (int a = 0; a < na; ++a) {
-        const int k0 = (kb * atoms + a) * kAtomK;
-        if (UP && !walk_all) {
-          if (lane * 4 < tile_rows)
-            tma_gather4(abase + a * a_block_bytes + lane * 512, &map_w, k0, r[0], r[1], r[2], r[3], full + 8 * s);
-        } else if (UP) {
-          if (lane == 0) tma_tile_2d(abase + a * a_block_bytes, map_t.get(), k0, tile * tile_rows, full + 8 * s);
-        } else if (lane == 0) {
-          tma_tile_2d(abase + a * a_block_bytes, &map_w, k0, tile * tile_rows, full + 8 * s);
-        }
-        if (lane == 0) tma_tile_2d(abase + b_off + a * b_block_bytes, &map_x, k0, 0, full + 8 * s);
-      }
+      return true;
+    };
+    if (MODE == kGate) {
+      // the first ring-full of weight tiles goes out while the predecessor in the stream still runs; the token
+      // rows of those stages follow once it has finished
+      const int ahead = total < S ? total : S;
+      const bool ok = produce(0, ahead, true, false);
+      pdl_wait();
+      if (ok && produce(0, ahead, false, true)) produce(ahead, total, true, true);
+    } else {
+      produce(0, total, true, true);
     }
   } else if (warp >= 8) {
     // ======================= MMA issuers =======================================================
