@@ -154,6 +154,14 @@ int sffn_set_path(sffn_handle* h, int path) {
 
 // Experiment knob (not part of the documented ABI).
 void sffn_debug_set_pdl(int on) { sffn::debug_set_pdl(on); }
+// Host-side geometry of the kernels for a shape (no GPU needed): see debug_fused_plan / umma_gate_tiling.
+void sffn_debug_fused_plan(int bf16, int D, int H, int K, int lopa, int sm_count, int* out9) {
+  sffn::debug_fused_plan(bf16 != 0, D, H, K, lopa != 0, sm_count, out9);
+}
+void sffn_debug_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list) {
+  sffn::umma_gate_tiling(R, sm_count, tile_rows, n_tiles);
+  *own_list = sffn::umma_own_list_supported(R, sm_count) ? 1 : 0;
+}
 void sffn_debug_set_trace(void* device_buffer) { sffn::debug_set_trace(static_cast<long long*>(device_buffer)); }
 
 int sffn_launch_count(sffn_handle* h, long long* launches) {

@@ -762,6 +762,15 @@ size_t fused_workspace_bytes(int D, int H, int r_max) {
   return 256 + (size_t)kMaxGrid * D * 4 + (size_t)(r_max > 0 ? r_max : 1) * 4 + 256;
 }
 
+// Geometry of the fused kernel for a shape, as nine integers (for host-side checks): ok, rows per gate slot, gate
+// slot bytes, gate slots, gate warps, act slot bytes, act slots, chunks per act thread, shared memory bytes.
+void debug_fused_plan(bool bf16, int D, int H, int K, bool lopa, int sm_count, int* out) {
+  const Geometry g = plan(bf16, D, H, K, lopa, fused_grid(sm_count, H));
+  const int v[9] = {g.ok ? 1 : 0, g.rows_per_gate_slot, g.gate_slot_bytes, g.n_gate_slots, g.gate_warps,
+                    g.act_slot_bytes, g.n_act_slots, g.cpt, g.smem};
+  for (int i = 0; i < 9; ++i) out[i] = v[i];
+}
+
 bool fused_supported(bool bf16, int D, int H, int B, const sffn_gate* gate, int sm_count) {
   if (B != 1) return false;
   const bool lopa = gate->kind == SFFN_GATE_LOPA;

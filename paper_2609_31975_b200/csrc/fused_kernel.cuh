@@ -32,6 +32,7 @@ size_t fused_workspace_bytes(int D, int H, int r_max);
 bool fused_supported(bool bf16, int D, int H, int B, const sffn_gate* gate, int sm_count);
 void debug_set_pdl(int on);
 void debug_set_trace(long long* device_buffer);
+void debug_fused_plan(bool bf16, int D, int H, int K, bool lopa, int sm_count, int* out);
 cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched);
 
 }  // namespace sffn
