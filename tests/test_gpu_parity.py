@@ -83,6 +83,29 @@ def test_standard_gate_small_shapes(mod, D, H, dtype):
             run_both_paths(mod, ffn, x[t], gate, w, act, ("general", "fused"), what=f"{D}x{H} s={s} {act}")
 
 
+@pytest.mark.parametrize("D,H", [(3840, 300), (5120, 200), (8192, 160), (16384, 96)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_wide_rows(mod, D, H, dtype):
+    """Rows of 7.5 to 64 KB: one row per gate slot, few ring slots, up to eight chunks per act thread; whatever
+    `auto` picks for the shape (the fused kernels where their geometry fits, else the general ones)."""
+    if D * (2 if dtype == torch.bfloat16 else 4) > 32768:               # rows above 32 KB are refused, not mangled
+        with pytest.raises(mod.SFFNError) as e:
+            mod.SparseFFN(D, H, dtype, r_max=64, B_max=2)
+        assert e.value.code == 2
+        return
+    ffn = mod.SparseFFN(D, H, dtype, r_max=64, B_max=2)
+    gate, w = make_std(D, H, dtype, 23, 0.8)
+    x = syn.tokens(2, D, dtype, 23, DEV)
+    run_both_paths(mod, ffn, x[0], gate, w, "relu", ("general", "auto"), what=f"wide {D}x{H}")
+    lg, lw = make_lopa(mod, D, H, 64, dtype, 24, 0.8, "tiled")
+    run_both_paths(mod, ffn, x[1], lg, lw, "sqrelu", ("general", "auto"), what=f"wide lopa {D}x{H}")
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")      # two tokens
+    assert_y_close(y, ref["y"], what=f"wide {D}x{H} B=2")
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
+
+
 @pytest.mark.parametrize("r,fixed,sign,gain,rms", [
     (64, "diag", False, False, True), (128, "tiled", True, True, True),
     (96, None, False, False, False), (256, "diag", True, False, False)])
