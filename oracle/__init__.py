@@ -184,3 +184,24 @@ def ffn(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, b_g=None, route="sp
     if single:
         out["y"], out["z"] = y[0], z[0]
     return out
+
+
+def dequantize_rows(q, scale) -> np.ndarray:
+    """The matrix int8 codes stand for under weight-only quantisation with one scale per row (appendix on
+    quantisation-aware training: "weights are converted to int8 at inference"; the paper does not fix the
+    granularity, one fp32 scale per output row is the reading taken here): W[j, k] = scale[j] * q[j, k], as float64."""
+    if not isinstance(q, np.ndarray):
+        q = q.detach().cpu().numpy()
+    if not isinstance(scale, np.ndarray):
+        scale = scale.detach().cpu().numpy()
+    assert q.dtype == np.int8 and q.ndim == 2 and scale.shape == (q.shape[0],)
+    return scale.astype(np.float64)[:, None] * q.astype(np.float64)
+
+
+def ffn_q8(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, **kw):
+    """:func:`ffn` on int8 weights: every matrix is a dict(q=int8 [rows, cols], s=fp32 [rows]) and enters Eq. 1 as
+    its float64 dequantisation (:func:`dequantize_rows`); tokens stay in their own dtype (weight-only)."""
+    dq = lambda m: dequantize_rows(m["q"], m["s"])  # noqa: E731
+    if lopa is not None:
+        lopa = dict(lopa, V=dq(lopa["V"]), U=dq(lopa["U"]))
+    return ffn(x, dq(W_up), dq(W_down), act, W_g=None if W_g is None else dq(W_g), lopa=lopa, **kw)

@@ -11,6 +11,10 @@ Recipe (all configurable):
            nearest even by ``Tensor.to``);  tokens x ~ N(0, 1), same rounding;
   gate bias b_g = -Phi^-1(s) * sigma_z, the constant that makes a N(0, sigma_z^2) pre-activation
            negative with probability s;  or a per-neuron bias from a Zipf firing profile.
+  int8 weights (weight-only quantisation): codes drawn directly, q = clip(round(N(0, 32^2)), +-127), which is
+           what an abs-max quantiser leaves of a Gaussian row of a few thousand entries (max ~ 4 sigma), and
+           one fp32 scale per row, s_j = std / 32 * (1 + 0.1 u_j), u_j ~ U(-1, 1); the matrix the codes stand
+           for is s_j * q[j, :].  Nothing is quantised here, so no rounding rule is shared with either side.
 """
 from __future__ import annotations
 
@@ -18,7 +22,7 @@ import math
 
 import torch
 
-_TAGS = {"W_g": 1, "W_up": 2, "W_down": 3, "V": 4, "U": 5, "x": 6, "perm": 7}
+_TAGS = {"W_g": 1, "W_up": 2, "W_down": 3, "V": 4, "U": 5, "x": 6, "perm": 7, "scale": 8}
 
 
 def _gen(seed: int, tag: str, device, extra: int = 0) -> torch.Generator:
@@ -78,6 +82,48 @@ def lopa_ffn(D: int, H: int, r: int, dtype, seed: int, device="cpu", sparsity: f
         "U": normal_tensor((H, r), 1.0 / math.sqrt(r), dtype, seed, "U", device, extra),
         "W_up": normal_tensor((H, D), 1.0 / math.sqrt(D), dtype, seed, "W_up", device, extra),
         "W_down": normal_tensor((H, D), 1.0 / math.sqrt(D), dtype, seed, "W_down", device, extra),
+    }
+    sigma = math.sqrt(2.0) if with_fixed_matrix else 1.0
+    w["b_g"] = None if sparsity is None else torch.full(
+        (H,), gate_bias_for_sparsity(sparsity, sigma), dtype=torch.float32, device=device)
+    return w
+
+
+def q8_matrix(shape, std: float, seed: int, tag: str, device="cpu", extra: int = 0, chunk_rows: int = 4096) -> dict:
+    """int8 codes q [rows, cols] and fp32 row scales s [rows] of a matrix whose entries s_j q[j,k] have
+    standard deviation ~ std (see the module recipe).  Returns dict(q=int8 tensor, s=float32 tensor)."""
+    rows, cols = shape
+    q = torch.empty((rows, cols), dtype=torch.int8, device=device)
+    g = _gen(seed, tag, device, extra)
+    for r0 in range(0, rows, chunk_rows):
+        r1 = min(rows, r0 + chunk_rows)
+        blk = torch.randn((r1 - r0, cols), generator=g, device=device, dtype=torch.float32)
+        q[r0:r1] = (blk * 32.0).round().clamp(-127, 127).to(torch.int8)
+    u = torch.rand((rows,), generator=_gen(seed, "scale", device, extra * 16 + _TAGS[tag]), device=device,
+                   dtype=torch.float32)
+    s = (std / 32.0) * (1.0 + 0.1 * (2.0 * u - 1.0))
+    return {"q": q, "s": s.float()}
+
+
+def standard_ffn_q8(D: int, H: int, seed: int, device="cpu", sparsity: float | None = 0.9, extra: int = 0) -> dict:
+    """Standard-gated FFN in int8 codes + row scales: W_g, W_up, W_down each dict(q [H,D], s [H]); b_g as in
+    :func:`standard_ffn`."""
+    std = 1.0 / math.sqrt(D)
+    w = {k: q8_matrix((H, D), std, seed, k, device, extra) for k in ("W_g", "W_up", "W_down")}
+    w["b_g"] = None if sparsity is None else torch.full(
+        (H,), gate_bias_for_sparsity(sparsity), dtype=torch.float32, device=device)
+    return w
+
+
+def lopa_ffn_q8(D: int, H: int, r: int, seed: int, device="cpu", sparsity: float | None = 0.9,
+                with_fixed_matrix: bool = True, extra: int = 0) -> dict:
+    """LoPA-gated FFN in int8 codes + row scales (V [r,D], U [H,r], W_up, W_down [H,D]); b_g as in
+    :func:`lopa_ffn`."""
+    w = {
+        "V": q8_matrix((r, D), 1.0 / math.sqrt(D), seed, "V", device, extra),
+        "U": q8_matrix((H, r), 1.0 / math.sqrt(r), seed, "U", device, extra),
+        "W_up": q8_matrix((H, D), 1.0 / math.sqrt(D), seed, "W_up", device, extra),
+        "W_down": q8_matrix((H, D), 1.0 / math.sqrt(D), seed, "W_down", device, extra),
     }
     sigma = math.sqrt(2.0) if with_fixed_matrix else 1.0
     w["b_g"] = None if sparsity is None else torch.full(

@@ -355,3 +355,67 @@ def test_double_activation_special_cases():
         g = {"relu": np.maximum(u, 0.0), "sqrelu": np.maximum(u, 0.0) ** 2,
              "rsplus": np.where(u >= 0, u / (1.0 + np.exp(-u)), 0.0)}[a3]
         np.testing.assert_allclose(sparse["y"], (a * g) @ Wd.astype(np.float64), rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------- weight-only int8 (appendix on quantisation-aware training)
+def test_hand_worked_int8_rows():
+    # codes with one scale per ROW: W = [[0.5*1, 0.5*-2], [0.25*3, 0.25*4]] = [[0.5, -1], [0.75, 1]]
+    q = np.array([[1, -2], [3, 4]], np.int8)
+    s = np.array([0.5, 0.25], np.float32)
+    np.testing.assert_array_equal(oracle.dequantize_rows(q, s), [[0.5, -1.0], [0.75, 1.0]])
+    # x = [2, 1];  z = W1 x = [0, 2.5]: only neuron 1 fires (z > 0);  u = W3 x with W3 = 2*[[1,1],[1,-1]] = [6, 2]
+    # y = a_1 u_1 Wd[1] = 2.5 * 2 * (0.5*[4, -6]) = [10, -15]
+    W1 = dict(q=q, s=s)
+    W3 = dict(q=np.array([[1, 1], [1, -1]], np.int8), s=np.array([2.0, 2.0], np.float32))
+    Wd = dict(q=np.array([[100, 100], [4, -6]], np.int8), s=np.array([1.0, 0.5], np.float32))
+    x = np.array([2.0, 1.0], np.float32)
+    for route in ("dense", "sparse"):
+        out = oracle.ffn_q8(x, W3, Wd, "relu", W_g=W1, route=route)
+        np.testing.assert_array_equal(out["z"], [0.0, 2.5])
+        np.testing.assert_array_equal(out["y"], [10.0, -15.0])
+        assert out["n_act"][0] == 1
+
+
+def test_int8_with_power_of_two_scales_equals_fp32_weights():
+    # s_j q_jk is exactly an fp32 number when s_j is a power of two, so the int8 route and the fp32 route see the
+    # same real matrices and must agree to the last bit (both accumulate the same products in the same order)
+    D, H, r, B = 32, 48, 16, 3
+    x = syn.tokens(B, D, torch.bfloat16, 5)
+
+    def mat(rows, cols, tag):
+        q = RNG.integers(-127, 128, (rows, cols)).astype(np.int8)
+        s = (2.0 ** RNG.integers(-9, -3, rows)).astype(np.float32)
+        return dict(q=q, s=s), (s[:, None] * q.astype(np.float32)).astype(np.float32)
+
+    (W1q, W1), (W3q, W3), (Wdq, Wd) = mat(H, D, "g"), mat(H, D, "u"), mat(H, D, "d")
+    (Vq, V), (Uq, U) = mat(r, D, "V"), mat(H, r, "U")
+    b = np.full(H, -0.3, np.float32)
+    a = oracle.ffn_q8(x, W3q, Wdq, "relu", W_g=W1q, b_g=b)
+    f = oracle.ffn(x, W3, Wd, "relu", W_g=W1, b_g=b)
+    np.testing.assert_array_equal(a["y"], f["y"])
+    np.testing.assert_array_equal(a["z"], f["z"])
+    gi = RNG.integers(0, D, H).astype(np.int32)
+    lq = dict(V=Vq, U=Uq, g_idx=gi, use_rmsnorm=True, eps=1e-5)
+    lf = dict(V=V, U=U, g_idx=gi, use_rmsnorm=True, eps=1e-5)
+    a = oracle.ffn_q8(x, W3q, Wdq, "rsplus", lopa=lq, b_g=b, act_up="relu")
+    f = oracle.ffn(x, W3, Wd, "rsplus", lopa=lf, b_g=b, act_up="relu")
+    np.testing.assert_array_equal(a["y"], f["y"])
+    assert a["y"].any()
+
+
+def test_int8_inputs_recipe():
+    w = syn.standard_ffn_q8(256, 512, 3)
+    for k in ("W_g", "W_up", "W_down"):
+        q, s = w[k]["q"], w[k]["s"]
+        assert q.dtype == torch.int8 and s.dtype == torch.float32 and q.shape == (512, 256) and s.shape == (512,)
+        assert int(q.min()) >= -127 and int(q.max()) <= 127
+        assert float(q.float().std()) == pytest.approx(32.0, rel=0.02)
+        # dequantised entries have the standard deviation of the bf16 recipe, 1/sqrt(D), within the +-10 % row spread
+        W = oracle.dequantize_rows(q, s)
+        assert float(W.std()) * 16.0 == pytest.approx(1.0, rel=0.02)
+        assert len(torch.unique(s)) > 500                                  # the scales really differ by row
+    assert not torch.equal(w["W_g"]["q"], w["W_up"]["q"]) and not torch.equal(w["W_g"]["s"], w["W_up"]["s"])
+    # 90 % target sparsity holds on the dequantised gate
+    x = syn.tokens(16, 256, torch.bfloat16, 3)
+    out = oracle.ffn_q8(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=w["b_g"])
+    assert out["n_act"].mean() / 512 == pytest.approx(0.1, abs=0.03)
