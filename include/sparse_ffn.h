@@ -136,6 +136,31 @@ int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate
                       const float* b_g, const void* W_up, const void* W_down, int act, float* y,
                       void* stream);
 
+/* Weight-only int8 (the paper's appendix on quantisation-aware training: "weights are converted to int8 at
+ * inference", tokens and all arithmetic stay in floating point).  The paper does not fix the format; here every
+ * weight matrix is stored as int8 codes, row-major, with one fp32 scale per row:
+ *     W[j, k] = s[j] * q[j, k],   q in [-127, 127].
+ * In these two calls the pointers W_up, W_down and, inside `gate`, W_g (STANDARD) or V and U (LOPA) address the
+ * int8 codes ([H,D], [H,D], [H,D], [r,D], [H,r]); `scales` carries the row scales.  Tokens x are bf16: the handle
+ * must have been created with SFFN_BF16.  Rows must be a multiple of 16 bytes (D and r multiples of 16).
+ * Everything else (b_g, g_idx, g_sign, RMSNorm, act, y, the active list, double activation) is as in
+ * sparse_ffn_forward / dense_ffn_forward.  One token runs in the fused kernels, batches in the CUDA-core
+ * kernels (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is an offline
+ * step outside this library. */
+typedef struct {
+  const float* s_gate; /* [H]  row scales of W_g (STANDARD) or of U (LOPA) */
+  const float* s_V;    /* [r]  row scales of V (LOPA only; may be NULL otherwise) */
+  const float* s_up;   /* [H]  row scales of W_up */
+  const float* s_down; /* [H]  row scales of W_down (row j = column j of W_2) */
+} sffn_q8_scales;
+
+int sparse_ffn_forward_q8(sffn_handle* handle, const void* x, int B, const sffn_gate* gate, const float* b_g,
+                          const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
+                          void* stream);
+int dense_ffn_forward_q8(sffn_handle* handle, const void* x, int B, const sffn_gate* gate, const float* b_g,
+                         const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
+                         void* stream);
+
 /* End-to-end variant of sparse_ffn_forward for callers whose activations live on the host:
  * x_host [B,D] (handle dtype) and y_host [B,D] fp32 are HOST pointers; weights stay on the device.
  * Brings x in, runs the sparse path, puts y out, all on `stream`; y_host is valid once the stream has

@@ -30,6 +30,11 @@ class _Gate(ctypes.Structure):
                 ("use_rmsnorm", ctypes.c_int32), ("rms_eps", ctypes.c_float)]
 
 
+class _Q8Scales(ctypes.Structure):
+    _fields_ = [("s_gate", ctypes.c_void_p), ("s_V", ctypes.c_void_p), ("s_up", ctypes.c_void_p),
+                ("s_down", ctypes.c_void_p)]
+
+
 def lib_path() -> Path:
     return _PKG / "libsparse_ffn.so"
 
@@ -56,6 +61,9 @@ def load_library() -> ctypes.CDLL:
         lib.sparse_ffn_forward.argtypes = fwd
         lib.dense_ffn_forward.argtypes = fwd
         lib.sparse_ffn_forward_host.argtypes = fwd
+        fwd_q8 = [vp, vp, i, ctypes.POINTER(_Gate), vp, vp, vp, ctypes.POINTER(_Q8Scales), i, vp, vp]
+        lib.sparse_ffn_forward_q8.argtypes = fwd_q8
+        lib.dense_ffn_forward_q8.argtypes = fwd_q8
         lib.sffn_last_active.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
         lib.sffn_last_device_status.argtypes = [vp, ctypes.POINTER(i)]
         lib.sffn_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
@@ -71,6 +79,16 @@ def load_library() -> ctypes.CDLL:
 
 def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _codes(m):
+    """The tensor whose address goes to the library: an int8 matrix given as dict(q=codes, s=row scales), or a tensor."""
+    if isinstance(m, dict):
+        q, s = m["q"], m["s"]
+        if q.dtype != torch.int8 or s.dtype != torch.float32 or s.shape != (q.shape[0],):
+            raise TypeError("an int8 matrix is dict(q=int8 [rows, cols], s=float32 [rows])")
+        return q
+    return m
 
 
 def _check(where: str, rc: int):
@@ -114,6 +132,10 @@ class SparseFFN:
     ``gate`` arguments are dicts: ``{"W_g": t}`` for standard gating, or
     ``{"V": t, "U": t, "g_idx": t|None, "g_sign": t|None, "rms_gain": t|None,
     "use_rmsnorm": bool, "rms_eps": float}`` for the LoPA gate.
+
+    Weight-only int8: hand every weight matrix (W_up, W_down and W_g, or V and U inside ``gate``) as
+    ``dict(q=int8 codes [rows, cols], s=float32 row scales [rows])`` to the ``*_q8`` methods (or to
+    :meth:`prepared`); the handle's dtype, the tokens', must then be bfloat16.
     """
 
     def __init__(self, D: int, H: int, dtype: torch.dtype, r_max: int = 0, B_max: int = 1,
@@ -155,16 +177,26 @@ class SparseFFN:
     def _gate(self, gate: dict) -> _Gate:
         g = _Gate()
         if "W_g" in gate:
-            g.kind, g.W_g = 0, gate["W_g"].data_ptr()
+            g.kind, g.W_g = 0, _codes(gate["W_g"]).data_ptr()
         else:
-            g.kind, g.r = 1, gate["V"].shape[0]
-            g.V, g.U = gate["V"].data_ptr(), gate["U"].data_ptr()
+            g.kind, g.r = 1, _codes(gate["V"]).shape[0]
+            g.V, g.U = _codes(gate["V"]).data_ptr(), _codes(gate["U"]).data_ptr()
             for k in ("g_idx", "g_sign", "rms_gain"):
                 t = gate.get(k)
                 setattr(g, k, None if t is None else t.data_ptr())
             g.use_rmsnorm = int(gate.get("use_rmsnorm", True))
             g.rms_eps = float(gate.get("rms_eps", 1e-5))
         return g
+
+    @staticmethod
+    def _scales(gate: dict, W_up, W_down) -> _Q8Scales:
+        sc = _Q8Scales()
+        if "W_g" in gate:
+            sc.s_gate = gate["W_g"]["s"].data_ptr()
+        else:
+            sc.s_gate, sc.s_V = gate["U"]["s"].data_ptr(), gate["V"]["s"].data_ptr()
+        sc.s_up, sc.s_down = W_up["s"].data_ptr(), W_down["s"].data_ptr()
+        return sc
 
     def _stream(self, stream):
         s = torch.cuda.current_stream(self.device) if stream is None else stream
@@ -178,16 +210,35 @@ class SparseFFN:
                         ACT[act] if isinstance(act, str) else int(act), _ptr(y), self._stream(stream)))
         return y
 
+    def _call_q8(self, fn, name, x, gate, b_g, W_up, W_down, act, y, stream):
+        B = 1 if x.dim() == 1 else x.shape[0]
+        g, sc = self._gate(gate), self._scales(gate, W_up, W_down)
+        self._keep = (x, gate, b_g, W_up, W_down, y)
+        _check(name, fn(self._h, _ptr(x), B, ctypes.byref(g), _ptr(b_g), _ptr(_codes(W_up)), _ptr(_codes(W_down)),
+                        ctypes.byref(sc), ACT[act] if isinstance(act, str) else int(act), _ptr(y),
+                        self._stream(stream)))
+        return y
+
     def prepared(self, x, gate, b_g, W_up, W_down, act, y, *, dense=False, host=False, stream=None):
         """Marshals one call once and returns a zero-argument callable that issues it (for launch
         loops where per-call marshalling would dominate).  The stream is fixed at preparation."""
-        fn = (self.lib.sparse_ffn_forward_host if host else
-              self.lib.dense_ffn_forward if dense else self.lib.sparse_ffn_forward)
         B = 1 if x.dim() == 1 else x.shape[0]
         g = self._gate(gate)
-        args = (self._h, _ptr(x), B, ctypes.byref(g), _ptr(b_g), _ptr(W_up), _ptr(W_down),
-                ACT[act] if isinstance(act, str) else int(act), _ptr(y), self._stream(stream))
-        keep = (x, gate, b_g, W_up, W_down, y, g)
+        a = ACT[act] if isinstance(act, str) else int(act)
+        if isinstance(W_up, dict):  # weight-only int8
+            if host:
+                raise ValueError("the host entry point takes fp32 / bf16 weights")
+            fn = self.lib.dense_ffn_forward_q8 if dense else self.lib.sparse_ffn_forward_q8
+            sc = self._scales(gate, W_up, W_down)
+            args = (self._h, _ptr(x), B, ctypes.byref(g), _ptr(b_g), _ptr(_codes(W_up)), _ptr(_codes(W_down)),
+                    ctypes.byref(sc), a, _ptr(y), self._stream(stream))
+            keep = (x, gate, b_g, W_up, W_down, y, g, sc)
+        else:
+            fn = (self.lib.sparse_ffn_forward_host if host else
+                  self.lib.dense_ffn_forward if dense else self.lib.sparse_ffn_forward)
+            args = (self._h, _ptr(x), B, ctypes.byref(g), _ptr(b_g), _ptr(W_up), _ptr(W_down), a, _ptr(y),
+                    self._stream(stream))
+            keep = (x, gate, b_g, W_up, W_down, y, g)
 
         def call(_fn=fn, _args=args, _keep=keep):
             rc = _fn(*_args)
@@ -207,6 +258,20 @@ class SparseFFN:
         if y is None:
             y = torch.empty((*x.shape[:-1], self.D), dtype=torch.float32, device=x.device)
         return self._call(self.lib.dense_ffn_forward, "dense_ffn_forward", x, gate, b_g, W_up, W_down, act, y, stream)
+
+    def sparse_ffn_forward_q8(self, x, gate, b_g, W_up, W_down, act="relu", y=None, stream=None):
+        """:meth:`sparse_ffn_forward` on int8 weights with one fp32 scale per row (see the class docstring)."""
+        if y is None:
+            y = torch.empty((*x.shape[:-1], self.D), dtype=torch.float32, device=x.device)
+        return self._call_q8(self.lib.sparse_ffn_forward_q8, "sparse_ffn_forward_q8", x, gate, b_g, W_up, W_down,
+                             act, y, stream)
+
+    def dense_ffn_forward_q8(self, x, gate, b_g, W_up, W_down, act="relu", y=None, stream=None):
+        """The dense comparator on int8 weights."""
+        if y is None:
+            y = torch.empty((*x.shape[:-1], self.D), dtype=torch.float32, device=x.device)
+        return self._call_q8(self.lib.dense_ffn_forward_q8, "dense_ffn_forward_q8", x, gate, b_g, W_up, W_down,
+                             act, y, stream)
 
     def sparse_ffn_forward_host(self, x_host, gate, b_g, W_up, W_down, act, y_host, stream=None):
         """End-to-end variant: x_host / y_host are (pinned) host tensors, weights on the device."""

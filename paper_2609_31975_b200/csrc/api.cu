@@ -9,6 +9,7 @@
 #include <new>
 
 #include "batched_kernels.cuh"
+#include "common.cuh"
 #include "fused_kernel.cuh"
 #include "general_kernels.cuh"
 #include "umma_kernels.cuh"
@@ -155,8 +156,8 @@ int sffn_set_path(sffn_handle* h, int path) {
 // Experiment knob (not part of the documented ABI).
 void sffn_debug_set_pdl(int on) { sffn::debug_set_pdl(on); }
 // Host-side geometry of the kernels for a shape (no GPU needed): see debug_fused_plan / umma_gate_tiling.
-void sffn_debug_fused_plan(int bf16, int D, int H, int K, int lopa, int sm_count, int* out9) {
-  sffn::debug_fused_plan(bf16 != 0, D, H, K, lopa != 0, sm_count, out9);
+void sffn_debug_fused_plan(int wkind, int D, int H, int K, int lopa, int sm_count, int* out9) {
+  sffn::debug_fused_plan(wkind, D, H, K, lopa != 0, sm_count, out9);  // wkind: 0 fp32, 1 bf16, 2 int8 rows
 }
 void sffn_debug_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list) {
   sffn::umma_gate_tiling(R, sm_count, tile_rows, n_tiles);
@@ -175,12 +176,20 @@ int sffn_launch_count(sffn_handle* h, long long* launches) {
 namespace {
 
 int check_call(const sffn_handle* h, const void* x, int B, const sffn_gate* g, const void* W_up,
-               const void* W_down, int act, const void* y) {
+               const void* W_down, int act, const void* y, const sffn_q8_scales* q8) {
   if (!h || !x || !g || !W_up || !W_down || !y) return SFFN_ERR_INVALID_ARG;
   if (B < 1 || B > h->B_max) return SFFN_ERR_INVALID_ARG;
   if (act < SFFN_ACT_RELU || act > SFFN_ACT_RSPLUS) return SFFN_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(W_up) || !aligned16(W_down) || !aligned16(y)) return SFFN_ERR_UNSUPPORTED;
-  const size_t esz = h->dtype == SFFN_BF16 ? 2 : 4;
+  const size_t esz = q8 ? 1 : h->dtype == SFFN_BF16 ? 2 : 4;  // bytes of a weight element
+  if (q8) {
+    if (h->dtype != SFFN_BF16) return SFFN_ERR_UNSUPPORTED;  // int8 weights meet bf16 tokens
+    if (!q8->s_gate || !q8->s_up || !q8->s_down) return SFFN_ERR_INVALID_ARG;
+    if (g->kind == SFFN_GATE_LOPA && !q8->s_V) return SFFN_ERR_INVALID_ARG;
+    if (h->D % 16) return SFFN_ERR_UNSUPPORTED;
+    if (sffn::updown_max_tokens(sffn::kWQ8, h->D) == 0) return SFFN_ERR_UNSUPPORTED;
+    if (h->path == SFFN_PATH_MMA_SYNC) return SFFN_ERR_UNSUPPORTED;
+  }
   if (g->kind == SFFN_GATE_STANDARD) {
     if (!g->W_g) return SFFN_ERR_INVALID_ARG;
     if (!aligned16(g->W_g)) return SFFN_ERR_UNSUPPORTED;
@@ -373,10 +382,11 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
 // General path: gate (all tokens, chunks of <= 4) -> compaction -> up/down + reduce per chunk.
 int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
                 const void* W_up, const void* W_down, int act, float* y, bool dense,
-                cudaStream_t s) {
+                const sffn_q8_scales* q8, cudaStream_t s) {
   using namespace sffn;
   const bool bf16 = h->dtype == SFFN_BF16;
-  const size_t esz = bf16 ? 2 : 4;
+  const int wkind = q8 ? kWQ8 : bf16 ? kWBF16 : kWF32;
+  const size_t esz = bf16 ? 2 : 4;  // bytes of a token element
   const int D = h->D, H = h->H;
   float* actbuf = h->at<float>(h->L.act);
   uint8_t* flag = h->at<uint8_t>(h->L.flag);
@@ -395,7 +405,8 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       p.W = g->V; p.R = g->r; p.K = D;
       p.vec = xb + (size_t)b0 * D * esz; p.vec_stride = D;
       p.out = vbuf + (size_t)b0 * rs; p.out_stride = rs;
-      SFFN_CUDA(launch_rowdot(bf16, !bf16, nb, false, p, h->sm_count, s));
+      p.row_scale = q8 ? q8->s_V : nullptr;
+      SFFN_CUDA(launch_rowdot(wkind, !bf16, nb, false, p, h->sm_count, s));
       ++h->launches;
       b0 += nb;
     }
@@ -421,7 +432,8 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     p.act = act;
     p.flag = dense ? nullptr : flag;
     p.flag_or = b0 > 0;
-    SFFN_CUDA(launch_rowdot(bf16, lopa || !bf16, nb, true, p, h->sm_count, s));
+    p.row_scale = q8 ? q8->s_gate : nullptr;
+    SFFN_CUDA(launch_rowdot(wkind, lopa || !bf16, nb, true, p, h->sm_count, s));
     ++h->launches;
     b0 += nb;
   }
@@ -430,7 +442,7 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     ++h->launches;
     h->list_state = 1;
   }
-  const int nbmax = updown_max_tokens(bf16, D);
+  const int nbmax = updown_max_tokens(wkind, D);
   int grid = 2 * h->sm_count;
   if (grid > kMaxUpDownGrid) grid = kMaxUpDownGrid;
   float* partial = h->at<float>(h->L.partial);
@@ -446,7 +458,8 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     p.H = H; p.D = D;
     p.partial = partial;
     p.act_up = h->act_up;
-    SFFN_CUDA(launch_updown(bf16, nb, p, grid, s));
+    p.s_up = q8 ? q8->s_up : nullptr; p.s_down = q8 ? q8->s_down : nullptr;
+    SFFN_CUDA(launch_updown(wkind, nb, p, grid, s));
     SFFN_CUDA(launch_reduce(partial, grid, nb, D, y + (size_t)b0 * D, D, s));
     h->launches += 2;
     b0 += nb;
@@ -455,15 +468,17 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
 }
 
 int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g, const void* W_up,
-        const void* W_down, int act, float* y, bool dense, void* stream) {
-  const int rc = check_call(h, x, B, g, W_up, W_down, act, y);
+        const void* W_down, int act, float* y, bool dense, void* stream, const sffn_q8_scales* q8 = nullptr) {
+  const int rc = check_call(h, x, B, g, W_up, W_down, act, y, q8);
   if (rc != SFFN_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const bool fused_ok = sffn::fused_supported(h->dtype == SFFN_BF16, h->D, h->H, B, g, h->sm_count);
+  const int wkind = q8 ? sffn::kWQ8 : h->dtype == SFFN_BF16 ? sffn::kWBF16 : sffn::kWF32;
+  const bool fused_ok = sffn::fused_supported(wkind, h->D, h->H, B, g, h->sm_count);
   if (h->path == SFFN_PATH_FUSED && !fused_ok) return SFFN_ERR_UNSUPPORTED;
   if (fused_ok && h->path != SFFN_PATH_GENERAL) {
     sffn::FusedCall c{};
-    c.bf16 = h->dtype == SFFN_BF16;
+    c.wkind = wkind;
+    if (q8) { c.s_gate = q8->s_gate; c.s_V = q8->s_V; c.s_up = q8->s_up; c.s_down = q8->s_down; }
     c.D = h->D; c.H = h->H;
     c.x = x; c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up; c.y = y;
     c.dense = dense;
@@ -480,7 +495,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
   }
   const int gate_k = g->kind == SFFN_GATE_LOPA ? g->r : h->D;
   const int gate_cols = g->kind == SFFN_GATE_LOPA ? 2 * B : B;
-  if (h->dtype == SFFN_BF16 && B >= 2 && B <= kMaxMmaTokens && h->path != SFFN_PATH_GENERAL) {
+  if (!q8 && h->dtype == SFFN_BF16 && B >= 2 && B <= kMaxMmaTokens && h->path != SFFN_PATH_GENERAL) {
     const bool mma_ok = sffn::batched_mma_supported(h->D, gate_k, gate_cols);
     const bool umma_ok = mma_ok && sffn::umma_rows_supported(gate_k, gate_cols) && sffn::umma_rows_supported(h->D, B);
     if (h->path == SFFN_PATH_MMA_SYNC && !mma_ok) return SFFN_ERR_UNSUPPORTED;
@@ -489,7 +504,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
   } else if (h->path == SFFN_PATH_MMA_SYNC) {
     return SFFN_ERR_UNSUPPORTED;
   }
-  return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, s);
+  return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, q8, s);
 }
 
 // Device-side alias of a 16-byte aligned pointer into pinned, mapped host memory; null for anything else.
@@ -522,6 +537,20 @@ int sparse_ffn_forward(sffn_handle* h, const void* x, int B, const sffn_gate* g,
 int dense_ffn_forward(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
                       const void* W_up, const void* W_down, int act, float* y, void* stream) {
   return run(h, x, B, g, b_g, W_up, W_down, act, y, true, stream);
+}
+
+int sparse_ffn_forward_q8(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
+                          const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
+                          void* stream) {
+  if (!scales) return SFFN_ERR_INVALID_ARG;
+  return run(h, x, B, g, b_g, W_up, W_down, act, y, false, stream, scales);
+}
+
+int dense_ffn_forward_q8(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
+                         const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
+                         void* stream) {
+  if (!scales) return SFFN_ERR_INVALID_ARG;
+  return run(h, x, B, g, b_g, W_up, W_down, act, y, true, stream, scales);
 }
 
 int sparse_ffn_forward_host(sffn_handle* h, const void* x_host, int B, const sffn_gate* g,

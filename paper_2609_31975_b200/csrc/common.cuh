@@ -59,6 +59,64 @@ struct Elem<__nv_bfloat16> {
   __device__ __forceinline__ static float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 };
 
+// Two fp32 operations in one instruction (sm_100 packed fp32): d = a * b + c and d = a + b, element-wise on pairs.
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+
+// int8 codes of weight-only quantisation (one fp32 scale per row, applied by the caller of unpack to the
+// finished dot product or to the row's coefficient).  Tokens that meet such weights are bf16.
+// code -> fp32 without an integer conversion: with the sign bit flipped the byte is u = code + 128 in 0..255;
+// placed in the low mantissa byte of 2^23 it reads 2^23 + u exactly, and one subtraction of 2^23 + 128 leaves
+// the code.
+template <>
+struct Elem<int8_t> {
+  static constexpr int kPerVec = 16;
+  // four codes of one 32-bit word as two pairs (codes 0, 1 and codes 2, 3)
+  __device__ __forceinline__ static void unpack4(uint32_t w, float2& lo, float2& hi) {
+    w ^= 0x80808080u;
+    const float2 bias = make_float2(-8388736.f, -8388736.f);
+    lo = add2(make_float2(__uint_as_float(__byte_perm(w, 0x4b000000u, 0x7650)),
+                          __uint_as_float(__byte_perm(w, 0x4b000000u, 0x7651))), bias);
+    hi = add2(make_float2(__uint_as_float(__byte_perm(w, 0x4b000000u, 0x7652)),
+                          __uint_as_float(__byte_perm(w, 0x4b000000u, 0x7653))), bias);
+  }
+  __device__ __forceinline__ static void unpack4(uint32_t w, float* f) {
+    float2 lo, hi;
+    unpack4(w, lo, hi);
+    f[0] = lo.x; f[1] = lo.y; f[2] = hi.x; f[3] = hi.y;
+  }
+  __device__ __forceinline__ static void unpack(const uint4& v, float* f) {
+    unpack4(v.x, f);
+    unpack4(v.y, f + 4);
+    unpack4(v.z, f + 8);
+    unpack4(v.w, f + 12);
+  }
+};
+
+// Storage type of the tokens that go with weights of type T, and whether rows of T carry a scale.
+template <typename T>
+struct TokenOf { using type = T; static constexpr bool kScaled = false; };
+template <>
+struct TokenOf<int8_t> { using type = __nv_bfloat16; static constexpr bool kScaled = true; };
+
+// Weight storage kinds as the launchers take them (0 and 1 coincide with "is bf16" of older call sites).
+constexpr int kWF32 = 0, kWBF16 = 1, kWQ8 = 2;
+__host__ __device__ constexpr int weight_bytes(int wkind) { return wkind == kWF32 ? 4 : wkind == kWBF16 ? 2 : 1; }
+
 // Streaming 16-byte load: weights are read once, so keep them out of L1.
 __device__ __forceinline__ uint4 ld_stream16(const void* p) {
   uint4 v;

@@ -70,6 +70,10 @@ struct FusedParams {
   unsigned long long v_target;     // LoPA: value of the counter once all CTAs of this call have published
   int act, dense;
   int act_up;        // activation on the up projection (double activation, Sec. 3.3); kActNone = Eq. 1
+  const float* s_gate;  // int8 rows only: one scale per row of the gate matrix [H], of V [r], of W_up and W_down [H]
+  const float* s_V;
+  const float* s_up;
+  const float* s_down;
   float* partial;  // [grid][D]
   uint8_t* flag;
   int32_t* status;
@@ -81,9 +85,9 @@ struct FusedParams {
 
 // Shared-memory carve-up, identical on host and device.
 struct SmemLayout {
-  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, total;
+  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, row_scales, slot_scales, total;
   __host__ __device__ SmemLayout(int D, int K, bool lopa, int n_gate_slots, int gate_slot_bytes,
-                                 int n_act_slots, int act_slot_bytes, int slab_max) {
+                                 int n_act_slots, int act_slot_bytes, int slab_max, bool scaled) {
     int off = 0;
     auto take = [&](int bytes) {
       int o = off;
@@ -99,6 +103,8 @@ struct SmemLayout {
     red = take(2 * (2 * 8 + 1) * 4);  // up to eight act warps
     ctl = take(8 * 4);
     bars = take(2 * (n_gate_slots + n_act_slots) * 8);
+    row_scales = take(scaled ? 2 * slab_max * 4 : 0);     // int8 rows: scales of the slab's W_up / W_down rows
+    slot_scales = take(scaled ? 2 * n_act_slots * 4 : 0);  // the same two for the row in each act slot
     total = off;
   }
 };
@@ -166,13 +172,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-// Position of element k of a vector inside its shared-memory copy.  For 8-element (bf16) chunks the
-// two halves of every chunk are stored in two planes so that a warp's float4 reads are conflict-free.
+// Position of element k of a vector inside its shared-memory copy.  For 8-element (bf16) and 16-element (int8)
+// chunks the quarters of every chunk are stored in two / four planes so that a warp's float4 reads are conflict-free.
 template <int EPV>
 __device__ __forceinline__ int vec_pos(int k, int len) {
   if (EPV == 4) return k;
-  const int c = k >> 3, q = k & 7;
-  return (q < 4 ? 0 : len / 2) + 4 * c + (q & 3);
+  const int c = k / EPV, q = k % EPV;
+  return (q >> 2) * (len / (EPV / 4)) + 4 * c + (q & 3);
 }
 
 // Dot product of one 16-byte chunk of weights with the matching entries of the staged vector.
@@ -186,12 +192,44 @@ __device__ __forceinline__ float chunk_dot(const uint4& w, const float* vec, int
   acc = fmaf(f[1], lo.y, acc);
   acc = fmaf(f[2], lo.z, acc);
   acc = fmaf(f[3], lo.w, acc);
-  if (EPV == 8) {
-    const float4 hi = reinterpret_cast<const float4*>(vec)[nvec + c];
-    acc = fmaf(f[4], hi.x, acc);
-    acc = fmaf(f[5], hi.y, acc);
-    acc = fmaf(f[6], hi.z, acc);
-    acc = fmaf(f[7], hi.w, acc);
+#pragma unroll
+  for (int q = 1; q < EPV / 4; ++q) {
+    const float4 hi = reinterpret_cast<const float4*>(vec)[q * nvec + c];
+    acc = fmaf(f[4 * q + 0], hi.x, acc);
+    acc = fmaf(f[4 * q + 1], hi.y, acc);
+    acc = fmaf(f[4 * q + 2], hi.z, acc);
+    acc = fmaf(f[4 * q + 3], hi.w, acc);
+  }
+  return acc;
+}
+
+// Two int8 rows' chunks against the same entries of the staged vector (read once), packed fp32 arithmetic: the
+// sums are kept as pairs (even / odd elements).
+__device__ __forceinline__ void chunk_dot2_q8(const uint4& wa, const uint4& wb, const float* vec, int c, int nvec,
+                                              float2& acc_a, float2& acc_b) {
+  const uint32_t a[4] = {wa.x, wa.y, wa.z, wa.w}, b[4] = {wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 v = reinterpret_cast<const float4*>(vec)[q * nvec + c];
+    float2 lo, hi;
+    Elem<int8_t>::unpack4(a[q], lo, hi);
+    acc_a = fma2(lo, make_float2(v.x, v.y), acc_a);
+    acc_a = fma2(hi, make_float2(v.z, v.w), acc_a);
+    Elem<int8_t>::unpack4(b[q], lo, hi);
+    acc_b = fma2(lo, make_float2(v.x, v.y), acc_b);
+    acc_b = fma2(hi, make_float2(v.z, v.w), acc_b);
+  }
+}
+// One int8 chunk against the staged vector, packed.
+__device__ __forceinline__ float2 chunk_dot_q8(const uint4& w, const float* vec, int c, int nvec, float2 acc) {
+  const uint32_t a[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 v = reinterpret_cast<const float4*>(vec)[q * nvec + c];
+    float2 lo, hi;
+    Elem<int8_t>::unpack4(a[q], lo, hi);
+    acc = fma2(lo, make_float2(v.x, v.y), acc);
+    acc = fma2(hi, make_float2(v.z, v.w), acc);
   }
   return acc;
 }
@@ -212,7 +250,7 @@ __device__ __forceinline__ long long global_ns() {
   } while (0)
 
 template <typename T, int CPT, bool LOPA>
-__global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedParams p) {
+__global__ void __maxnreg__((CPT == 8 || CPT * Elem<T>::kPerVec >= 64) ? 128 : 96) fused_ffn_kernel(const FusedParams p) {
   // Warp roles: 2 gate producers, 2 act producers, then gate warps and act warps.  The standard gate needs its
   // eight gate warps to keep up with the stream; the LoPA gate is short (r elements per row), the call's time
   // is then set by the up/down rows, so eight of the twelve workers are act warps there.
@@ -227,11 +265,13 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
   pdl_launch_dependents();
   if (threadIdx.x == 0) SFFN_GSTAMP(10);
   constexpr int EPV = Elem<T>::kPerVec;
+  using X = typename TokenOf<T>::type;             // storage type of the token
+  constexpr bool kScaled = TokenOf<T>::kScaled;    // int8 rows: every row comes with an fp32 scale
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x, cta = blockIdx.x;
   const int D = p.D, K = p.K;
   const int NG = p.n_gate_slots, NA = p.n_act_slots;
-  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NA, p.act_slot_bytes, p.slab_max);
+  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NA, p.act_slot_bytes, p.slab_max, kScaled);
 
   unsigned char* gate_ring = smem + L.gate_ring;
   unsigned char* act_ring = smem + L.act_ring;
@@ -243,6 +283,10 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
   // (a fence in the producers would also wait for their bulk copies in flight).
   volatile uint32_t* row_state = reinterpret_cast<volatile uint32_t*>(smem + L.aval);
   float* slot_a = reinterpret_cast<float*>(smem + L.slot_a);  // per act slot: gate value, < 0 = stop
+  float* row_su = reinterpret_cast<float*>(smem + L.row_scales);  // [slab_max] scale of the W_up row, then
+  float* row_sd = row_su + p.slab_max;                            // [slab_max] of the W_down row (int8 only)
+  float* slot_su = reinterpret_cast<float*>(smem + L.slot_scales);
+  float* slot_sd = slot_su + NA;
   float* red = reinterpret_cast<float*>(smem + L.red);
   volatile int* ctl = reinterpret_cast<volatile int*>(smem + L.ctl);
   const uint32_t bars = smem_u32(smem + L.bars);
@@ -304,7 +348,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
 
   // Gate warps fetch the per-neuron parameters (bias, fixed-matrix index and sign) of their first two
   // ring slots now: like the weights they do not depend on the predecessor in the stream.
-  float pre_bias[2] = {0.f, 0.f}, pre_sg[2] = {1.f, 1.f};
+  float pre_bias[2] = {0.f, 0.f}, pre_sg[2] = {1.f, 1.f}, pre_scale[2] = {1.f, 1.f};
   int pre_gi[2] = {-1, -1};
   if (warp >= kFirstGateWarp && warp < kFAW && warp - kFirstGateWarp < p.gate_warps) {
 #pragma unroll
@@ -313,6 +357,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
       if (sq < n_gslots && lane < nr && slot_first_neuron(sq) + lane < p.H) {
         const int j = slot_first_neuron(sq) + lane;
         if (p.b_g) pre_bias[q] = p.b_g[j];
+        if (kScaled) pre_scale[q] = p.s_gate[j];
         if (LOPA && p.g_idx) {
           pre_gi[q] = p.g_idx[j];
           pre_sg[q] = (p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
@@ -331,15 +376,30 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
                    : "memory");
   }
 
+  // int8 rows: the scales of this CTA's W_up / W_down rows (parameters, like the weights) go into shared memory
+  // now; the act producers hand the two of a fired row to the act warps together with the row.
+  if (kScaled) {
+    for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) {
+      const int j = slot_first_neuron(i / nr) + i % nr;
+      row_su[i] = __ldg(p.s_up + j);
+      row_sd[i] = __ldg(p.s_down + j);
+    }
+  }
+
   // ---- everyone else: wait for the predecessor in the stream, then stage the token ------------
   pdl_wait();
   if (tid == kStageBase) SFFN_GSTAMP(11);
   for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) row_state[i] = 0xffffffffu;
-  for (int c = tid - kStageBase; c < nvecD; c += kStageThreads) {
-    float f[EPV];
-    Elem<T>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + c), f);
-    reinterpret_cast<float4*>(sx)[c] = make_float4(f[0], f[1], f[2], f[3]);
-    if (EPV == 8) reinterpret_cast<float4*>(sx)[nvecD + c] = make_float4(f[4], f[5], f[6], f[7]);
+  constexpr int XEPV = Elem<X>::kPerVec;  // token elements per 16 bytes (the weights' EPV unless those are int8)
+  for (int cx = tid - kStageBase; cx < D / XEPV; cx += kStageThreads) {
+    float f[XEPV];
+    Elem<X>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + cx), f);
+#pragma unroll
+    for (int g4 = 0; g4 < XEPV / 4; ++g4) {
+      const int k0 = cx * XEPV + 4 * g4;  // first of four consecutive elements: quarter (k0 % EPV) / 4 of chunk k0 / EPV
+      reinterpret_cast<float4*>(sx)[((k0 % EPV) >> 2) * nvecD + k0 / EPV] =
+          make_float4(f[4 * g4], f[4 * g4 + 1], f[4 * g4 + 2], f[4 * g4 + 3]);
+    }
   }
   if (LOPA) {
     // Rank-r stage of the LoPA gate, v = V x, spread over the grid: this CTA computes its share of
@@ -360,7 +420,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         a1 = chunk_dot<T>(w1, sx, c + 32, nvecD, a1);
       }
       if (c < nvecD) a0 = chunk_dot<T>(ld_stream16(vr + c), sx, c, nvecD, a0);
-      const float v = warp_sum(a0 + a1);
+      const float v = warp_sum(a0 + a1) * (kScaled ? __ldg(p.s_V + k) : 1.f);
       if (lane == 0) __stcg(p.vbuf + k, v);
     }
     __threadfence();
@@ -431,6 +491,10 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
           if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) {
             if (ap == 0) slot_a[slot] = sl == 0x80000000u ? 0.f : __uint_as_float(sl);
             const int lrow = base + l;
+            if (kScaled && ap == 0) {
+              slot_su[slot] = row_su[lrow];
+              slot_sd[slot] = row_sd[lrow];
+            }
             const size_t j = (size_t)(slot_first_neuron(lrow / nr) + lrow % nr);
             mbar_expect_tx(full_act + 8 * slot, (uint32_t)row_bytes);
             bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
@@ -459,13 +523,15 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
       const int j0 = slot_first_neuron(s);
       const int rows = min(nr, p.H - j0);
       float add = 0.f;  // bias + fixed-matrix term of the row this lane reports
+      float scale = 1.f;  // int8 rows: scale of that row
       if (lane < rows) {
         const int j = j0 + lane;
         float bias, sg;
         int gi;
-        if (s == gw) { bias = pre_bias[0]; gi = pre_gi[0]; sg = pre_sg[0]; }
-        else if (s == gw + p.gate_warps) { bias = pre_bias[1]; gi = pre_gi[1]; sg = pre_sg[1]; }
+        if (s == gw) { bias = pre_bias[0]; gi = pre_gi[0]; sg = pre_sg[0]; scale = pre_scale[0]; }
+        else if (s == gw + p.gate_warps) { bias = pre_bias[1]; gi = pre_gi[1]; sg = pre_sg[1]; scale = pre_scale[1]; }
         else {
+          if (kScaled) scale = p.s_gate[j];
           bias = p.b_g ? p.b_g[j] : 0.f;
           gi = (LOPA && p.g_idx) ? p.g_idx[j] : -1;
           sg = (LOPA && p.g_idx && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
@@ -496,7 +562,25 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         for (int i = 0; i < 4; ++i)
           if (lane == rr + i) mine = a[i];
       }
-      for (int rr = rows_short; rr < rows; ++rr) {
+      int rr_single = rows_short;
+      if (EPV == 16) {
+        // int8 rows: the staged vector is four times the bytes of a row, so two rows share every read of it
+        for (; rr_single + 1 < rows; rr_single += 2) {
+          const uint4* w0 = reinterpret_cast<const uint4*>(base + (size_t)rr_single * gate_row_bytes);
+          const uint4* w1 = reinterpret_cast<const uint4*>(base + (size_t)(rr_single + 1) * gate_row_bytes);
+          float2 a0 = make_float2(0.f, 0.f), a1 = a0, b0 = a0, b1 = a0;
+          int c = lane;
+          for (; c + 32 < nvecK; c += 64) {
+            chunk_dot2_q8(w0[c], w1[c], gvec, c, nvecK, a0, b0);
+            chunk_dot2_q8(w0[c + 32], w1[c + 32], gvec, c + 32, nvecK, a1, b1);
+          }
+          if (c < nvecK) chunk_dot2_q8(w0[c], w1[c], gvec, c, nvecK, a0, b0);
+          const float z0 = warp_sum((a0.x + a0.y) + (a1.x + a1.y)), z1 = warp_sum((b0.x + b0.y) + (b1.x + b1.y));
+          if (lane == rr_single) mine = z0;
+          if (lane == rr_single + 1) mine = z1;
+        }
+      }
+      for (int rr = rr_single; rr < rows; ++rr) {
         const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr * gate_row_bytes);
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         int c = lane;
@@ -512,7 +596,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         if (lane == rr) mine = z;
       }
       if (lane < rows) {
-        const float z = mine + add;
+        const float z = kScaled ? fmaf(mine, scale, add) : mine + add;
         const bool fired = z > 0.f;
         if (!p.dense) p.flag[j0 + lane] = fired ? 1 : 0;
         row_state[r0 + lane] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
@@ -554,6 +638,7 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
       const unsigned char* s0 = act_ring + (size_t)slot * p.act_slot_bytes;
       const unsigned char* s1 = act_ring + (size_t)slot1 * p.act_slot_bytes;
       float part0 = 0.f, part1 = 0.f;
+      float2 pk0 = make_float2(0.f, 0.f), pk1 = pk0;  // int8 rows: packed partial sums
       if (a0 >= 0.f) {
         const uint4* wu0 = reinterpret_cast<const uint4*>(s0);
         const uint4* wu1 = reinterpret_cast<const uint4*>(s1);
@@ -561,9 +646,18 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         for (int i = 0; i < CPT; ++i) {
           const int c = at + i * kAT;
           if (c < nvecD) {
-            part0 = chunk_dot<T>(wu0[c], sx, c, nvecD, part0);
-            if (a1 >= 0.f) part1 = chunk_dot<T>(wu1[c], sx, c, nvecD, part1);
+            if constexpr (EPV == 16) {
+              pk0 = chunk_dot_q8(wu0[c], sx, c, nvecD, pk0);
+              if (a1 >= 0.f) pk1 = chunk_dot_q8(wu1[c], sx, c, nvecD, pk1);
+            } else {
+              part0 = chunk_dot<T>(wu0[c], sx, c, nvecD, part0);
+              if (a1 >= 0.f) part1 = chunk_dot<T>(wu1[c], sx, c, nvecD, part1);
+            }
           }
+        }
+        if constexpr (EPV == 16) {
+          part0 = pk0.x + pk0.y;
+          part1 = pk1.x + pk1.y;
         }
         part0 = warp_sum(part0);
         part1 = warp_sum(part1);
@@ -581,7 +675,15 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         u0 += (rp[4] + rp[5]) + (rp[6] + rp[7]);
         u1 += (rp[kAW + 4] + rp[kAW + 5]) + (rp[kAW + 6] + rp[kAW + 7]);
       }
-      const float h0 = a0 * activation(p.act_up, u0), h1 = a1 * activation(p.act_up, u1);
+      if (kScaled) {  // int8 rows: u = s_up (codes . x); the W_down row's scale rides on h
+        u0 *= slot_su[slot];
+        u1 *= slot_su[slot1];
+      }
+      float h0 = a0 * activation(p.act_up, u0), h1 = a1 * activation(p.act_up, u1);
+      if (kScaled) {
+        h0 *= slot_sd[slot];
+        h1 *= slot_sd[slot1];
+      }
       const uint4* wd0 = reinterpret_cast<const uint4*>(s0 + row_bytes);
       const uint4* wd1 = reinterpret_cast<const uint4*>(s1 + row_bytes);
 #pragma unroll
@@ -590,12 +692,30 @@ __global__ void __maxnreg__(CPT == 8 ? 128 : 96) fused_ffn_kernel(const FusedPar
         if (c < nvecD) {
           float f[EPV];
           Elem<T>::unpack(wd0[c], f);
+          if constexpr (EPV == 16) {
 #pragma unroll
-          for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h0, f[e], acc[i][e]);
+            for (int e = 0; e < EPV; e += 2) {
+              const float2 t = fma2(make_float2(h0, h0), make_float2(f[e], f[e + 1]), make_float2(acc[i][e], acc[i][e + 1]));
+              acc[i][e] = t.x;
+              acc[i][e + 1] = t.y;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h0, f[e], acc[i][e]);
+          }
           if (a1 >= 0.f) {
             Elem<T>::unpack(wd1[c], f);
+            if constexpr (EPV == 16) {
 #pragma unroll
-            for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h1, f[e], acc[i][e]);
+              for (int e = 0; e < EPV; e += 2) {
+                const float2 t = fma2(make_float2(h1, h1), make_float2(f[e], f[e + 1]), make_float2(acc[i][e], acc[i][e + 1]));
+                acc[i][e] = t.x;
+                acc[i][e + 1] = t.y;
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h1, f[e], acc[i][e]);
+            }
           }
         }
       }
@@ -677,9 +797,10 @@ struct Geometry {
   bool ok;
 };
 
-Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
+Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   Geometry g{};
-  const int esz = bf16 ? 2 : 4, epv = bf16 ? 8 : 4;
+  const int esz = weight_bytes(wkind), epv = 16 / esz;
+  const bool scaled = wkind == kWQ8;
   const int nvecD = D / epv;
   const int row_bytes = D * esz, gate_row_bytes = K * esz;
   g.ok = false;
@@ -687,13 +808,14 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   const int gate_warps_max = lopa ? 4 : 8;
   if (row_bytes % 16 || gate_row_bytes % 16 || nvecD > act_threads * 8) return g;
   g.cpt = nvecD <= act_threads ? 1 : nvecD <= 2 * act_threads ? 2 : nvecD <= 4 * act_threads ? 4 : 8;
+  if (scaled && g.cpt == 8) return g;  // 128 accumulators per act thread: the CUDA-core path takes such rows
   int nr = 8192 / gate_row_bytes;
   nr = nr < 1 ? 1 : nr > 32 ? 32 : nr;
   g.rows_per_gate_slot = nr;
   g.gate_slot_bytes = (nr * gate_row_bytes + 127) / 128 * 128;
   g.act_slot_bytes = (2 * row_bytes + 127) / 128 * 128;
   g.slab_max = (((H + nr - 1) / nr + grid - 1) / grid) * nr;  // most rows one CTA can own
-  const SmemLayout fixed(D, K, lopa, 0, 0, 0, 0, g.slab_max);
+  const SmemLayout fixed(D, K, lopa, 0, 0, 0, 0, g.slab_max, scaled);
   const int ring = kSmemBudget - fixed.total - 2048;  // slack for the barrier words
   if (ring <= 0) return g;
   // Gate ring first: two slots per gate warp hide the release -> refill latency; the act ring takes
@@ -725,7 +847,7 @@ Geometry plan(bool bf16, int D, int H, int K, bool lopa, int grid) {
   }
   g.n_act_slots = na;
   g.n_gate_slots = ng;
-  const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max);
+  const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max, scaled);
   g.smem = full.total;
   g.ok = g.smem <= kSmemBudget;
   return g;
@@ -743,7 +865,7 @@ cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaS
     case 1: k = fused_ffn_kernel<T, 1, LOPA>; break;
     case 2: k = fused_ffn_kernel<T, 2, LOPA>; break;
     case 4: k = fused_ffn_kernel<T, 4, LOPA>; break;
-    default: k = fused_ffn_kernel<T, 8, LOPA>; break;
+    default: k = fused_ffn_kernel<T, (TokenOf<T>::kScaled ? 4 : 8), LOPA>; break;  // int8 rows: plan() never asks for 8
   }
   static unsigned long long configured[4] = {0, 0, 0, 0};  // per instantiation of this template, per row width
   const int slot = g.cpt == 1 ? 0 : g.cpt == 2 ? 1 : g.cpt == 4 ? 2 : 3;
@@ -764,25 +886,25 @@ size_t fused_workspace_bytes(int D, int H, int r_max) {
 
 // Geometry of the fused kernel for a shape, as nine integers (for host-side checks): ok, rows per gate slot, gate
 // slot bytes, gate slots, gate warps, act slot bytes, act slots, chunks per act thread, shared memory bytes.
-void debug_fused_plan(bool bf16, int D, int H, int K, bool lopa, int sm_count, int* out) {
-  const Geometry g = plan(bf16, D, H, K, lopa, fused_grid(sm_count, H));
+void debug_fused_plan(int wkind, int D, int H, int K, bool lopa, int sm_count, int* out) {
+  const Geometry g = plan(wkind, D, H, K, lopa, fused_grid(sm_count, H));
   const int v[9] = {g.ok ? 1 : 0, g.rows_per_gate_slot, g.gate_slot_bytes, g.n_gate_slots, g.gate_warps,
                     g.act_slot_bytes, g.n_act_slots, g.cpt, g.smem};
   for (int i = 0; i < 9; ++i) out[i] = v[i];
 }
 
-bool fused_supported(bool bf16, int D, int H, int B, const sffn_gate* gate, int sm_count) {
+bool fused_supported(int wkind, int D, int H, int B, const sffn_gate* gate, int sm_count) {
   if (B != 1) return false;
   const bool lopa = gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? gate->r : D;
-  return plan(bf16, D, H, K, lopa, fused_grid(sm_count, H)).ok;
+  return plan(wkind, D, H, K, lopa, fused_grid(sm_count, H)).ok;
 }
 
 cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   const bool lopa = c.gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? c.gate->r : c.D;
   const int grid = fused_grid(c.sm_count, c.H);
-  const Geometry g = plan(c.bf16, c.D, c.H, K, lopa, grid);
+  const Geometry g = plan(c.wkind, c.D, c.H, K, lopa, grid);
   if (!g.ok) return cudaErrorInvalidValue;
   char* ws = static_cast<char*>(c.workspace);
   float* partial = reinterpret_cast<float*>(ws + 256);
@@ -803,13 +925,16 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.partial = partial;
   p.act = c.act; p.dense = c.dense ? 1 : 0;
   p.act_up = c.act_up;
+  p.s_gate = c.s_gate; p.s_V = c.s_V; p.s_up = c.s_up; p.s_down = c.s_down;
   p.flag = c.flag; p.status = c.status;
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;
   p.gate_warps = g.gate_warps;
   p.trace = g_debug_trace;
-  if (c.bf16)
+  if (c.wkind == kWQ8)
+    e = lopa ? launch_main<int8_t, true>(p, g, grid, s) : launch_main<int8_t, false>(p, g, grid, s);
+  else if (c.wkind == kWBF16)
     e = lopa ? launch_main<__nv_bfloat16, true>(p, g, grid, s) : launch_main<__nv_bfloat16, false>(p, g, grid, s);
   else
     e = lopa ? launch_main<float, true>(p, g, grid, s) : launch_main<float, false>(p, g, grid, s);

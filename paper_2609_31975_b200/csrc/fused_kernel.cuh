@@ -10,7 +10,11 @@
 namespace sffn {
 
 struct FusedCall {
-  bool bf16;
+  int wkind;  // kWF32 / kWBF16 / kWQ8: storage of the weights (tokens: fp32, bf16, bf16)
+  const float* s_gate;  // kWQ8: row scales of the gate matrix (W_g or U), of V, of W_up and of W_down
+  const float* s_V;
+  const float* s_up;
+  const float* s_down;
   int D, H;
   const void* x;
   const sffn_gate* gate;
@@ -29,10 +33,10 @@ struct FusedCall {
 };
 
 size_t fused_workspace_bytes(int D, int H, int r_max);
-bool fused_supported(bool bf16, int D, int H, int B, const sffn_gate* gate, int sm_count);
+bool fused_supported(int wkind, int D, int H, int B, const sffn_gate* gate, int sm_count);
 void debug_set_pdl(int on);
 void debug_set_trace(long long* device_buffer);
-void debug_fused_plan(bool bf16, int D, int H, int K, bool lopa, int sm_count, int* out);
+void debug_fused_plan(int wkind, int D, int H, int K, bool lopa, int sm_count, int* out);
 cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched);
 
 }  // namespace sffn

@@ -22,6 +22,7 @@ template <typename T, typename VT, int NB, bool GATE>
 __global__ void __launch_bounds__(256) rowdot_kernel(const RowDotParams p) {
   extern __shared__ float svec[];  // [NB][K]
   constexpr int EPV = Elem<T>::kPerVec;
+  using X = typename TokenOf<T>::type;  // storage type of the tokens
   const int K = p.K;
   pdl_launch_dependents();
   pdl_wait();  // the vectors (and, for the gate, the flag / value buffers) belong to earlier kernels until here
@@ -95,9 +96,11 @@ __global__ void __launch_bounds__(256) rowdot_kernel(const RowDotParams p) {
       for (int rr = 0; rr < 2; ++rr) {
         const int j = j0 + rr;
         if (j >= p.R) break;
+        // int8 rows: the dot product of the codes times the row's scale
+        const float sc = (TokenOf<T>::kScaled && p.row_scale) ? p.row_scale[j] : 1.f;
         if (!GATE) {
 #pragma unroll
-          for (int b = 0; b < NB; ++b) p.out[(size_t)b * p.out_stride + j] = rr ? acc1[b] : acc0[b];
+          for (int b = 0; b < NB; ++b) p.out[(size_t)b * p.out_stride + j] = (rr ? acc1[b] : acc0[b]) * sc;
         } else {
           const float bias = p.b_g ? p.b_g[j] : 0.f;
           const int gi = p.g_idx ? p.g_idx[j] : -1;
@@ -105,9 +108,9 @@ __global__ void __launch_bounds__(256) rowdot_kernel(const RowDotParams p) {
           bool any = false;
 #pragma unroll
           for (int b = 0; b < NB; ++b) {
-            float z = (rr ? acc1[b] : acc0[b]);
+            float z = (rr ? acc1[b] : acc0[b]) * sc;
             if (gi >= 0)
-              z += sg * Elem<T>::to_float(static_cast<const T*>(p.x)[(size_t)b * p.x_stride + gi]);
+              z += sg * Elem<X>::to_float(static_cast<const X*>(p.x)[(size_t)b * p.x_stride + gi]);
             z += bias;
             any |= z > 0.f;
             p.out[(size_t)b * p.out_stride + j] = activation(p.act, z);
@@ -209,9 +212,10 @@ __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
   const int D = p.D;
   pdl_launch_dependents();
   pdl_wait();
+  using X = typename TokenOf<T>::type;
   for (int b = 0; b < NB; ++b) {
-    const T* xb = static_cast<const T*>(p.x) + (size_t)b * p.x_stride;
-    for (int k = threadIdx.x; k < D; k += blockDim.x) svec[b * D + k] = Elem<T>::to_float(xb[k]);
+    const X* xb = static_cast<const X*>(p.x) + (size_t)b * p.x_stride;
+    for (int k = threadIdx.x; k < D; k += blockDim.x) svec[b * D + k] = Elem<X>::to_float(xb[k]);
   }
   const int n = p.count ? *p.count : p.H;
   const int lo = (int)((long long)n * blockIdx.x / gridDim.x);
@@ -266,10 +270,13 @@ __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
     if (lane == 0) {
       jbuf[warp] = j;
       bool live = false;
+      // int8 rows: u = s_up[j] (codes . x); the scale of the W_down row rides on the coefficient h
+      const float su = (TokenOf<T>::kScaled && valid) ? p.s_up[j] : 1.f;
+      const float sd = (TokenOf<T>::kScaled && valid) ? p.s_down[j] : 1.f;
 #pragma unroll
       for (int b = 0; b < NB; ++b) {
         // h = A(z) * A_3(u): double activation of Sec. 3.3 when act_up names one, Eq. 1 otherwise
-        const float h = valid ? p.a[(size_t)b * p.a_stride + j] * activation(p.act_up, u[b]) : 0.f;
+        const float h = valid ? p.a[(size_t)b * p.a_stride + j] * activation(p.act_up, u[b] * su) * sd : 0.f;
         hbuf[warp][b] = h;
         live |= h != 0.f;
       }
@@ -419,11 +426,15 @@ static cudaError_t launch_rowdot_nb(const RowDotParams& p, int nb, bool gate, in
   }
 }
 
-cudaError_t launch_rowdot(bool bf16, bool vec_is_f32, int nb, bool gate, const RowDotParams& p,
+cudaError_t launch_rowdot(int wkind, bool vec_is_f32, int nb, bool gate, const RowDotParams& p,
                           int sm_count, cudaStream_t s) {
   const int blocks_needed = (p.R + 15) / 16;  // 8 warps x 2 rows per pass
   const int grid = blocks_needed < sm_count * 4 ? (blocks_needed > 0 ? blocks_needed : 1) : sm_count * 4;
-  if (bf16) {
+  if (wkind == kWQ8) {
+    return vec_is_f32 ? launch_rowdot_nb<int8_t, float>(p, nb, gate, grid, s)
+                      : launch_rowdot_nb<int8_t, __nv_bfloat16>(p, nb, gate, grid, s);
+  }
+  if (wkind == kWBF16) {
     return vec_is_f32 ? launch_rowdot_nb<__nv_bfloat16, float>(p, nb, gate, grid, s)
                       : launch_rowdot_nb<__nv_bfloat16, __nv_bfloat16>(p, nb, gate, grid, s);
   }
@@ -459,14 +470,27 @@ static cudaError_t launch_updown_d(const UpDownParams& p, int nb, int grid, cuda
   return cudaErrorInvalidValue;
 }
 
-int updown_max_tokens(bool bf16, int D) {
-  const int nvec = D / (bf16 ? 8 : 4);
+int updown_max_tokens(int wkind, int D) {
+  const int nvec = D / (16 / weight_bytes(wkind));
+  if (wkind == kWQ8) return nvec > 1024 ? 0 : nvec > 512 ? 2 : 4;  // 16 accumulators per chunk and token
   if (nvec > 2048) return 0;
   return nvec > 1024 ? 2 : 4;
 }
 
-cudaError_t launch_updown(bool bf16, int nb, const UpDownParams& p, int grid, cudaStream_t s) {
-  return bf16 ? launch_updown_d<__nv_bfloat16>(p, nb, grid, s) : launch_updown_d<float>(p, nb, grid, s);
+cudaError_t launch_updown(int wkind, int nb, const UpDownParams& p, int grid, cudaStream_t s) {
+  if (wkind == kWQ8) {
+    const int nvec = p.D / 16;
+    if (nvec <= 512) {
+      if (nb == 1) return launch_updown_t<int8_t, 1, 1>(p, grid, s);
+      if (nb == 2) return launch_updown_t<int8_t, 2, 1>(p, grid, s);
+      if (nb == 4) return launch_updown_t<int8_t, 4, 1>(p, grid, s);
+    } else if (nvec <= 1024) {
+      if (nb == 1) return launch_updown_t<int8_t, 1, 2>(p, grid, s);
+      if (nb == 2) return launch_updown_t<int8_t, 2, 2>(p, grid, s);
+    }
+    return cudaErrorInvalidValue;
+  }
+  return wkind == kWBF16 ? launch_updown_d<__nv_bfloat16>(p, nb, grid, s) : launch_updown_d<float>(p, nb, grid, s);
 }
 
 cudaError_t launch_residual_cast(bool bf16, const float* y, const void* resid, float alpha, void* out, int n,

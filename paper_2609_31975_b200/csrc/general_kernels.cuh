@@ -22,6 +22,7 @@ struct RowDotParams {
   int act;
   uint8_t* flag;          // [R] or null: 1 where any of the NB tokens fires
   int flag_or;            // 0: overwrite flag, 1: OR into it (later token chunks)
+  const float* row_scale; // int8 rows: [R] scale of each row; null = 1
 };
 
 struct UpDownParams {
@@ -36,16 +37,19 @@ struct UpDownParams {
   int H, D;
   float* partial;      // [grid][NB][D]
   int act_up;          // activation on the up projection (double activation), kActNone = none
+  const float* s_up;   // int8 rows: [H] row scales of W_up and W_down
+  const float* s_down;
 };
 
-cudaError_t launch_rowdot(bool bf16, bool vec_is_f32, int nb, bool gate, const RowDotParams& p,
+// wkind: kWF32 / kWBF16 / kWQ8 (common.cuh); tokens are fp32, bf16, bf16 respectively.
+cudaError_t launch_rowdot(int wkind, bool vec_is_f32, int nb, bool gate, const RowDotParams& p,
                           int sm_count, cudaStream_t s);
 cudaError_t launch_rmsnorm(const float* v, float* n, const float* gain, int r, int stride, float eps,
                            int B, cudaStream_t s);
 cudaError_t launch_compact(const uint8_t* flag, int H, int32_t* idx, int32_t* count, cudaStream_t s);
 // Largest token chunk (4, 2 or 0 = unsupported D) the up/down kernel takes at this D.
-int updown_max_tokens(bool bf16, int D);
-cudaError_t launch_updown(bool bf16, int nb, const UpDownParams& p, int grid, cudaStream_t s);
+int updown_max_tokens(int wkind, int D);
+cudaError_t launch_updown(int wkind, int nb, const UpDownParams& p, int grid, cudaStream_t s);
 cudaError_t launch_residual_cast(bool bf16, const float* y, const void* resid, float alpha, void* out, int n,
                                  cudaStream_t s);
 cudaError_t launch_copy16(const void* src, void* dst, size_t bytes, cudaStream_t s);

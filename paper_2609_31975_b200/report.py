@@ -41,6 +41,18 @@ def _time(calls, stream, reps=3):
     return statistics.median(best), min(best)
 
 
+def _is_q8(w):
+    return isinstance(w["W_up"], dict)
+
+
+def _bytes(D, H, n_rows, esz, B, r, q8):
+    """Algorithmic bytes of one call; int8 weights: one byte per weight, bf16 tokens, and the fp32 row scales of
+    the gate matrix and of the fired W_up / W_down rows."""
+    if not q8:
+        return touched_bytes(D, H, n_rows, esz, B, r)
+    return touched_bytes(D, H, n_rows, 1, B, r) + B * D + 4 * (H + 2 * n_rows + (r or 0))
+
+
 def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1, act_up=None):
     """sets: list of weight dicts; gate_of(w) -> gate dict; act_up: activation on the up projection (double
     activation) or None.  Returns one result row."""
@@ -55,7 +67,8 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1,
         xt = x[t, 0] if B == 1 else x[t]
         yt = y[t, 0] if B == 1 else y[t]
         if t < 24:  # fired rows per call (union for B > 1), outside the timed region
-            ffn.sparse_ffn_forward(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt)
+            fwd = ffn.sparse_ffn_forward_q8 if _is_q8(w) else ffn.sparse_ffn_forward
+            fwd(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt)
             rows.append(int(ffn.last_active().numel()))
         sparse_calls.append(ffn.prepared(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt, stream=stream))
         dense_calls.append(ffn.prepared(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt, dense=True,
@@ -64,12 +77,13 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1,
     us, us_min = _time(sparse_calls, stream)
     us_dense, _ = _time(dense_calls[: max(16, n_calls // 4)], stream, reps=2)
     status = ffn.device_status()
-    nbytes = touched_bytes(D, H, round(n_rows), 2, B, r)
+    q8 = _is_q8(sets[0])
+    nbytes = _bytes(D, H, round(n_rows), 2, B, r, q8)
     row = dict(name=name, D=D, H=H, B=B, r=r, act=act, fired_rows=n_rows, fired_frac=n_rows / H,
                us_per_call=us, us_min=us_min, tokens_per_s=B * 1e6 / us, touched_mb=nbytes / 1e6,
                gbs=nbytes / us / 1e3, frac_measured_peak=nbytes / us / 1e3 / peak,
                frac_nominal=nbytes / us / 1e3 / NOMINAL, dense_us=us_dense,
-               dense_gbs=dense_bytes(D, H, 2, B, r) / us_dense / 1e3, speedup_vs_dense=us_dense / us,
+               dense_gbs=_bytes(D, H, H, 2, B, r, q8) / us_dense / 1e3, speedup_vs_dense=us_dense / us,
                device_status=status)
     del ffn, sparse_calls, dense_calls
     torch.cuda.empty_cache()
@@ -89,11 +103,14 @@ def measure_chain(name, D, H, layers, gate_of, act, r=None, dtype=torch.bfloat16
     ys = torch.empty((L, D), dtype=torch.float32, device=DEV)
     out = {}
     esz = 2 if dtype == torch.bfloat16 else 4
+    q8 = _is_q8(layers[0])
+    sparse_fwd = ffn.sparse_ffn_forward_q8 if q8 else ffn.sparse_ffn_forward
+    dense_fwd = ffn.dense_ffn_forward_q8 if q8 else ffn.dense_ffn_forward
     for route in ("sparse", "dense"):
         def body():
             xs[0].copy_(x_pre[0])
             for l, w in enumerate(layers):
-                fwd = ffn.dense_ffn_forward if route == "dense" else ffn.sparse_ffn_forward
+                fwd = dense_fwd if route == "dense" else sparse_fwd
                 fwd(xs[l], gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, ys[l], stream=stream)
                 residual_cast(ys[l], x_pre[l + 1], 0.0, xs[l + 1], stream=stream)
         with torch.cuda.stream(stream):
@@ -114,17 +131,17 @@ def measure_chain(name, D, H, layers, gate_of, act, r=None, dtype=torch.bfloat16
         del graph
     rows = []
     for l, w in enumerate(layers[:8]):
-        ffn.sparse_ffn_forward(xs[l], gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, ys[l])
+        sparse_fwd(xs[l], gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, ys[l])
         rows.append(int(ffn.last_active().numel()))
     n_rows = statistics.mean(rows)
     status = ffn.device_status()
-    nbytes = touched_bytes(D, H, round(n_rows), esz, 1, r)
+    nbytes = _bytes(D, H, round(n_rows), esz, 1, r, q8)
     us = out["sparse"]
     row = dict(name=name, D=D, H=H, B=1, r=r, act=act, fired_rows=n_rows, fired_frac=n_rows / H,
                us_per_call=us, us_min=us, tokens_per_s=1e6 / (us * L), touched_mb=nbytes / 1e6,
                gbs=nbytes / us / 1e3, frac_measured_peak=nbytes / us / 1e3 / peak,
                frac_nominal=nbytes / us / 1e3 / NOMINAL, dense_us=out["dense"],
-               dense_gbs=dense_bytes(D, H, esz, 1, r) / out["dense"] / 1e3, speedup_vs_dense=out["dense"] / us,
+               dense_gbs=_bytes(D, H, H, esz, 1, r, q8) / out["dense"] / 1e3, speedup_vs_dense=out["dense"] / us,
                device_status=status, layers=L)
     del ffn
     torch.cuda.empty_cache()
@@ -183,6 +200,22 @@ def run(out_path, quick=False, only=None, n_calls=None):
         del lsets
     del base, zsets
     torch.cuda.empty_cache()
+    # weight-only int8 (codes + one fp32 scale per row): the decode shape and one LoPA gate
+    if only is None or "int8" in only:
+        qsets = [syn.standard_ffn_q8(D, H, 6, DEV, sparsity=0.9, extra=i) for i in range(8)]
+        for s in ((0.9,) if quick else (0.8, 0.9, 0.95)):
+            b = syn.gate_bias_for_sparsity(s)
+            sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in qsets]
+            add(f"decode 4096x14336 s={s} int8", D, H, 1, sets, std, "relu", peak=peak)
+        lsets = []
+        for i, w in enumerate(qsets):
+            lw = syn.lopa_ffn_q8(D, H, 512, 7, DEV, sparsity=0.9, extra=i)
+            lw["W_up"], lw["W_down"] = w["W_up"], w["W_down"]
+            lsets.append(lw)
+        lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}
+        add("lopa r=512 relu int8", D, H, 1, lsets, lg, "relu", r=512, peak=peak)
+        del qsets, lsets
+        torch.cuda.empty_cache()
     if not quick and (only is None or "stress" in only):
         # stress shape: 8 independent layers per step
         D, H = 8192, 28672
@@ -232,6 +265,23 @@ def run(out_path, quick=False, only=None, n_calls=None):
                     print(json.dumps(rows[-1]), flush=True)
                 del layers
                 torch.cuda.empty_cache()
+        # the same two chains on int8 weights (bf16 tokens)
+        layers = [syn.standard_ffn_q8(D, H, 15, DEV, sparsity=0.9, extra=i) for i in range(L)]
+        name = f"paper shape 3840x10240 x{L} layers int8 s=0.9 standard (graph)"
+        if want(name):
+            rows.append(measure_chain(name, D, H, layers, std, "relu", peak=peak))
+            print(json.dumps(rows[-1]), flush=True)
+        del layers
+        torch.cuda.empty_cache()
+        gi = g_diagonal(Hp, D, DEV)
+        layers = [syn.lopa_ffn_q8(D, Hp, r, 16, DEV, sparsity=0.9, extra=i) for i in range(L)]
+        lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}
+        name = f"paper shape 3840x{Hp} x{L} layers int8 s=0.9 LoPA r={r} (graph)"
+        if want(name):
+            rows.append(measure_chain(name, D, Hp, layers, lg, "relu", r=r, peak=peak))
+            print(json.dumps(rows[-1]), flush=True)
+        del layers
+        torch.cuda.empty_cache()
     Path(out_path).parent.mkdir(parents=True, exist_ok=True)
     Path(out_path).write_text(json.dumps(rows, indent=1))
     md = ["| case | B | fired rows | us/call | touched MB | GB/s | % of measured peak | % of 8 TB/s | dense us | speedup |",
