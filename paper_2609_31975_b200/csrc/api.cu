@@ -72,7 +72,6 @@ struct sffn_handle {
   int path;
   int act_up;  // activation on the up projection (double activation), SFFN_ACT_NONE = Eq. 1
   long long launches;
-  unsigned long long lopa_calls;
   int list_state;  // 0: no sparse call yet, 1: idx/count hold the last call's list, 2: flags hold it
   template <typename T>
   T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
@@ -130,7 +129,6 @@ int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dt
   h->act_up = SFFN_ACT_NONE;
   h->launches = 0;
   h->list_state = 0;
-  h->lopa_calls = 0;
   *handle = h;
   return SFFN_OK;
 }
@@ -486,7 +484,6 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
     c.status = h->at<int32_t>(h->L.status);
     c.flag = h->at<uint8_t>(h->L.flag);
     c.sm_count = h->sm_count;
-    c.lopa_calls = &h->lopa_calls;
     int launched = 0;
     if (sffn::launch_fused(c, s, &launched) != cudaSuccess) return SFFN_ERR_CUDA;
     h->launches += launched;

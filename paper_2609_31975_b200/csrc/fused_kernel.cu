@@ -66,8 +66,12 @@ struct FusedParams {
   float eps;
   const void* V;      // LoPA: [r, D]
   float* vbuf;        // LoPA: [r] exchange buffer for v = V x
-  unsigned long long* v_counter;   // LoPA: CTAs that have published their rows of v (monotonic over calls)
-  unsigned long long v_target;     // LoPA: value of the counter once all CTAs of this call have published
+  // Two arrival counters in the workspace, monotonic over calls.  Every call adds exactly gridDim.x to each and
+  // calls on one workspace are serialised, so a CTA derives its call's first and last value from what its own
+  // atomicAdd returned: nothing depends on a host-side count, and a captured launch can be replayed.
+  unsigned long long* v_counter;     // LoPA: CTAs that have published their rows of v = V x
+  unsigned long long* done_counter;  // CTAs that have written their partial of y
+  float* y;                          // [D] result, written by the last CTAs to finish
   int act, dense;
   int act_up;        // activation on the up projection (double activation, Sec. 3.3); kActNone = Eq. 1
   const float* s_gate;  // int8 rows only: one scale per row of the gate matrix [H], of V [r], of W_up and W_down [H]
@@ -100,7 +104,7 @@ struct SmemLayout {
     sn = take(lopa ? K * 4 : 0);
     aval = take(slab_max * 4);
     slot_a = take(n_act_slots * 4);
-    red = take(2 * (2 * 8 + 1) * 4);  // up to eight act warps
+    red = take(3 * 16 * 16);  // act warps: 2 x (2 x 8 + 1) floats; afterwards the scratch of the cross-CTA sum
     ctl = take(8 * 4);
     bars = take(2 * (n_gate_slots + n_act_slots) * 8);
     row_params = take((lopa || scaled) ? (1 + (lopa ? 2 : 0) + (scaled ? 1 : 0)) * slab_max * 4 : 0);  // per-neuron gate parameters
@@ -110,7 +114,7 @@ struct SmemLayout {
   }
 };
 
-enum Ctl { kAbort = 0 };
+enum Ctl { kAbort = 0, kRank = 1 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -251,7 +255,7 @@ __device__ __forceinline__ long long global_ns() {
   } while (0)
 
 template <typename T, int CPT, bool LOPA>
-__global__ void __maxnreg__((CPT == 8 || CPT * Elem<T>::kPerVec >= 64) ? 128 : 96) fused_ffn_kernel(const FusedParams p) {
+__global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParams p) {
   // Warp roles: 2 gate producers, 2 act producers, then gate warps and act warps.  The standard gate needs its
   // eight gate warps to keep up with the stream; the LoPA gate is short (r elements per row), the call's time
   // is then set by the up/down rows, so eight of the twelve workers are act warps there.
@@ -431,12 +435,12 @@ __global__ void __maxnreg__((CPT == 8 || CPT * Elem<T>::kPerVec >= 64) ? 128 : 9
     __threadfence();
     named_bar_sync(5, kStageThreads);
     if (tid == kStageBase) {
-      atomicAdd(p.v_counter, 1ULL);
+      const unsigned long long v_target = (atomicAdd(p.v_counter, 1ULL) / G + 1) * G;
       const long long t0 = clock64();
       for (;;) {
         unsigned long long seen;
         asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.v_counter) : "memory");
-        if (seen >= p.v_target || ctl[kAbort]) break;
+        if (seen >= v_target || ctl[kAbort]) break;
         if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); break; }
         __nanosleep(40);
       }
@@ -747,46 +751,87 @@ __global__ void __maxnreg__((CPT == 8 || CPT * Elem<T>::kPerVec >= 64) ? 128 : 9
     if (at == 0) SFFN_STAMP(5);
     if (at == 0) SFFN_GSTAMP(12);
   }
-}
 
-// y[d] = sum over CTAs of partial[cta][d] in a fixed order.  Its CTAs (256 threads, ~40 registers) fit on
-// an SM next to a CTA of the main kernel (which is capped at 96 registers per thread for that reason), so
-// they are resident, parked in griddepcontrol.wait, before the main kernel ends.  One warp per float4 column: lane l adds
-// the partials l, l+32, ... (every load issued before the first add: one L2 round trip), then a fixed
-// shuffle tree combines the lanes.
-__global__ void __launch_bounds__(256) fused_reduce_kernel(const float* partial, int G, int D, float* y,
-                                                           const int32_t* status, long long* trace) {
-  pdl_launch_dependents();
-  if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)G * 16 + blockIdx.x] = global_ns();
-  pdl_wait();
-  if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)(G + 1) * 16 + blockIdx.x] = global_ns();
-  const int32_t failed = __ldcg(status);  // in flight together with the partials, not after them
+  // ---- y = sum over CTAs of their partials, by the last CTAs to finish -------------------------------------------
+  // A CTA that finishes among the last R of its call stays, waits (bounded) until every CTA has arrived and sums one
+  // slice of the columns over all partials in CTA order: which CTA does a slice depends on timing, what it computes
+  // does not, so y is bitwise the same on every run.  Earlier CTAs leave at once and their SMs take the next kernel
+  // of the stream.
+  if (warp < kFirstGateWarp) return;  // act producers (the gate producers left long ago)
+  constexpr int kTail = 32 * (kGW + kAW);
+  const int tw = warp - kFirstGateWarp;
   const int Q = D / 4;
-  const int q = blockIdx.x * 8 + (threadIdx.x >> 5);
-  const int l = threadIdx.x & 31;
-  if (q < Q) {
-    const float4* src = reinterpret_cast<const float4*>(partial) + q;
-    float4 v[8];  // G <= 256
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int g = l + 32 * i;
-      v[i] = g < G ? __ldcg(src + (size_t)g * Q) : make_float4(0.f, 0.f, 0.f, 0.f);
+  const int R = min(G, max(1, Q / 16));  // reducers: 16 columns each where the grid allows
+  named_bar_sync(6, kTail);
+  if (tid == 32 * kFirstGateWarp) {
+    SFFN_GSTAMP(6);
+    // Release at device scope after the CTA barrier: the act threads' partial stores happen before it, so a CTA that
+    // acquires the counter's final value sees every partial.
+    unsigned long long old;
+    asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(p.done_counter) : "memory");
+    const unsigned long long first = old / G * G;
+    const int rank = (int)(old - first);
+    ctl[kRank] = rank;
+    SFFN_GSTAMP(7);
+    if (rank >= G - R) {
+      const long long t0 = clock64();
+      for (;;) {
+        unsigned long long seen;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.done_counter) : "memory");
+        if (seen >= first + G || ctl[kAbort]) break;
+        if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); break; }
+        __nanosleep(20);
+      }
+      SFFN_GSTAMP(8);
     }
-    float4 s = v[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i) {
-      s.x += v[i].x;
-      s.y += v[i].y;
-      s.z += v[i].z;
-      s.w += v[i].w;
-    }
-    s.x = warp_sum(s.x);
-    s.y = warp_sum(s.y);
-    s.z = warp_sum(s.z);
-    s.w = warp_sum(s.w);
-    if (l == 0 && failed == 0) reinterpret_cast<float4*>(y)[q] = s;
   }
-  if (trace && threadIdx.x == 0 && blockIdx.x < 16) trace[(size_t)(G + 2) * 16 + blockIdx.x] = global_ns();
+  named_bar_sync(6, kTail);
+  const int slice = ctl[kRank] - (G - R);
+  if (slice < 0 || ctl[kAbort]) return;
+  const int32_t failed = __ldcg(p.status);  // in flight together with the partials, not after them
+  const int cols = (Q + R - 1) / R;
+  const int q_hi = min(Q, (slice + 1) * cols);
+  // Twelve warps = 4 groups of four columns x 3 row parts.  Lane (r8, c4) reads column c4 of its group in the rows
+  // 8 (3 i + part) + r8: one warp load covers eight rows x 64 contiguous bytes (whole 32-byte sectors).
+  static_assert(kGW + kAW == 12, "reduction tail is laid out for twelve warps");
+  const int part = tw % 3, cgw = tw / 3, r8 = lane >> 2, c4 = lane & 3;
+  float4* scratch = reinterpret_cast<float4*>(red);  // [3 parts][16 columns]; the act warps are done with it
+  const int tt = tid - 32 * kFirstGateWarp;
+  for (int c0 = slice * cols; c0 < q_hi; c0 += 16) {
+    const int q = c0 + 4 * cgw + c4;
+    float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (q < q_hi) {
+      const float4* src = reinterpret_cast<const float4*>(p.partial) + q;
+      for (int i0 = 0; 8 * (3 * i0 + part) < G; i0 += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int g = 8 * (3 * (i0 + i) + part) + r8;
+          v[i] = g < G ? __ldcg(src + (size_t)g * Q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          s4.x += v[i].x; s4.y += v[i].y; s4.z += v[i].z; s4.w += v[i].w;
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {  // the eight row residues of a column sit in lanes c4 + 4 r8
+      s4.x += __shfl_xor_sync(0xffffffffu, s4.x, o);
+      s4.y += __shfl_xor_sync(0xffffffffu, s4.y, o);
+      s4.z += __shfl_xor_sync(0xffffffffu, s4.z, o);
+      s4.w += __shfl_xor_sync(0xffffffffu, s4.w, o);
+    }
+    if (r8 == 0) scratch[part * 16 + 4 * cgw + c4] = s4;
+    named_bar_sync(6, kTail);
+    if (tt < 16 && c0 + tt < q_hi && failed == 0) {
+      const float4 a = scratch[tt], b = scratch[16 + tt], c = scratch[32 + tt];
+      reinterpret_cast<float4*>(p.y)[c0 + tt] =
+          make_float4((a.x + b.x) + c.x, (a.y + b.y) + c.y, (a.z + b.z) + c.z, (a.w + b.w) + c.w);
+    }
+    if (c0 + 16 < q_hi) named_bar_sync(6, kTail);  // the scratch is reused by the next pass
+  }
+  if (tid == 32 * kFirstGateWarp) SFFN_GSTAMP(13);
 }
 
 // ---- host side --------------------------------------------------------------------------------
@@ -923,8 +968,8 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.V = c.gate->V;
   p.vbuf = vbuf;
   p.v_counter = reinterpret_cast<unsigned long long*>(ws);
-  if (lopa) *c.lopa_calls += 1;
-  p.v_target = *c.lopa_calls * (unsigned long long)grid;
+  p.done_counter = p.v_counter + 1;
+  p.y = c.y;
   p.partial = partial;
   p.act = c.act; p.dense = c.dense ? 1 : 0;
   p.act_up = c.act_up;
@@ -941,11 +986,6 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
     e = lopa ? launch_main<__nv_bfloat16, true>(p, g, grid, s) : launch_main<__nv_bfloat16, false>(p, g, grid, s);
   else
     e = lopa ? launch_main<float, true>(p, g, grid, s) : launch_main<float, false>(p, g, grid, s);
-  if (e != cudaSuccess) return e;
-  ++n;
-  const int Q = c.D / 4;
-  e = launch_pdl(fused_reduce_kernel, dim3((Q + 7) / 8), dim3(256), 0, s, (const float*)partial, grid, c.D,
-                 c.y, (const int32_t*)c.status, g_debug_trace);
   if (e != cudaSuccess) return e;
   ++n;
   if (launched) *launched = n;

@@ -29,7 +29,6 @@ struct FusedCall {
   int32_t* status;   // device status word
   uint8_t* flag;     // [H] "neuron fired" bytes (sparse calls)
   int sm_count;
-  unsigned long long* lopa_calls;  // host counter of fused LoPA calls issued on this workspace
 };
 
 size_t fused_workspace_bytes(int D, int H, int r_max);

@@ -346,11 +346,17 @@ def test_double_activation_all_paths(mod, act, act_up):
 
 
 # ------------------------------------------------------------------ layer loop under a CUDA graph
+@pytest.mark.parametrize("kind", ["standard", "lopa"])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_layer_chain_in_cuda_graph(mod, dtype):
-    D, H, L = 512, 900, 3
-    ffn = mod.SparseFFN(D, H, dtype, B_max=1)
-    layers = [syn.standard_ffn(D, H, dtype, 81, DEV, sparsity=0.8, extra=i) for i in range(L)]
+def test_layer_chain_in_cuda_graph(mod, dtype, kind):
+    D, H, L, r = 512, 900, 3, 64
+    ffn = mod.SparseFFN(D, H, dtype, r_max=r, B_max=1)
+    if kind == "standard":
+        layers = [syn.standard_ffn(D, H, dtype, 81, DEV, sparsity=0.8, extra=i) for i in range(L)]
+        gates = [{"W_g": w["W_g"]} for w in layers]
+    else:
+        made = [make_lopa(mod, D, H, r, dtype, 81 + i, 0.8, sign=True, gain=True) for i in range(L)]
+        gates, layers = [g for g, _ in made], [w for _, w in made]
     resid = syn.tokens(L + 1, D, dtype, 81, DEV)
     xs = torch.zeros((L + 1, D), dtype=dtype, device=DEV)
     ys = torch.zeros((L, D), dtype=torch.float32, device=DEV)
@@ -359,8 +365,7 @@ def test_layer_chain_in_cuda_graph(mod, dtype):
     def body():
         xs[0].copy_(resid[0])
         for l, w in enumerate(layers):
-            ffn.sparse_ffn_forward(xs[l], {"W_g": w["W_g"]}, w["b_g"], w["W_up"], w["W_down"], "relu", ys[l],
-                                   stream=stream)
+            ffn.sparse_ffn_forward(xs[l], gates[l], w["b_g"], w["W_up"], w["W_down"], "relu", ys[l], stream=stream)
             mod.residual_cast(ys[l], resid[l + 1], 0.25, xs[l + 1], stream=stream)
 
     with torch.cuda.stream(stream):
@@ -371,16 +376,20 @@ def test_layer_chain_in_cuda_graph(mod, dtype):
         for l in range(L):
             want = (resid[l + 1].float() + 0.25 * eager_y[l]).to(dtype)
             assert torch.equal(eager_x[l + 1], want)
-            ref = run_oracle(eager_x[l], {"W_g": layers[l]["W_g"]}, layers[l]["b_g"], layers[l]["W_up"],
-                             layers[l]["W_down"], "relu")
+            ref = run_oracle(eager_x[l], gates[l], layers[l]["b_g"], layers[l]["W_up"], layers[l]["W_down"], "relu")
             assert_y_close(eager_y[l], ref["y"], what=f"chain layer {l}")
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=stream):
             body()
-        xs.zero_(); ys.zero_()
-        graph.replay()
+        # a captured launch is replayed with the arguments of its capture: nothing in them may count calls
+        for _ in range(4):
+            xs.zero_(); ys.zero_()
+            graph.replay()
+            stream.synchronize()
+            assert torch.equal(xs, eager_x) and torch.equal(ys, eager_y)   # bit for bit the eager run, every replay
+        body()                                                             # and eager calls after the replays
         stream.synchronize()
-    assert torch.equal(xs, eager_x) and torch.equal(ys, eager_y)      # the replayed graph repeats the eager run bit for bit
+        assert torch.equal(ys, eager_y)
     assert ffn.device_status() == 0
 
 
