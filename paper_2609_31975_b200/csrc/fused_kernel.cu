@@ -361,6 +361,15 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     return;
   }
 
+  // The token itself may still be written by the predecessor, so it is not read before the wait -- but its lines can
+  // be asked into L2 (a hint: whatever is written later lands in the same L2), which turns the staging loads right
+  // after the wait into L2 hits when the token comes from HBM.
+  if (warp == kGateProducers + 1) {
+    const int lines = (int)(((size_t)D * sizeof(X) + 127) / 128);
+    for (int i = lane; i < lines; i += 32)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const char*>(p.x) + (size_t)i * 128) : "memory");
+  }
+
   // LoPA: this CTA's rows of V are weights too; pull them into L2 now so that the rank-r stage, which sits on the
   // call's critical path right after the wait, finds them there.
   if (LOPA && warp == kGateProducers) {
