@@ -28,6 +28,8 @@ from .cost_model import (  # noqa: F401  (re-exported)
     g_tiled,
 )
 
+from . import lopa_cast  # noqa: F401,E402  (the LoPA approximation of Sec. 3.4)
+
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "sparse_ffn_oracle.cpp"
 _LIB = _HERE / "build" / "libsparse_ffn_oracle.so"

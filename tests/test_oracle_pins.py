@@ -419,3 +419,71 @@ def test_int8_inputs_recipe():
     x = syn.tokens(16, 256, torch.bfloat16, 3)
     out = oracle.ffn_q8(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=w["b_g"])
     assert out["n_act"].mean() / 512 == pytest.approx(0.1, abs=0.03)
+
+
+# ---------------------------------------------------------------- LoPA approximation of a full gate (Sec. 3.4)
+def test_lopa_approximation_m_step_is_the_row_optimum_by_brute_force():
+    cast = oracle.lopa_cast
+    H, D, r = 7, 5, 2
+    W = RNG.standard_normal((H, D))
+    U, V = RNG.standard_normal((H, r)) * 0.3, RNG.standard_normal((r, D)) * 0.3
+    g_idx, g_sign = cast.m_step(W, U, V)
+    R = W - U @ V
+    for i in range(H):
+        # every admissible row of M: one entry, +1 or -1
+        costs = {(j, sg): ((R[i] - sg * np.eye(D)[j]) ** 2).sum() for j in range(D) for sg in (-1, 1)}
+        best = min(costs, key=costs.get)
+        assert (int(g_idx[i]), int(g_sign[i])) == best
+    # hand-worked: R = [[0.2, -3, 1], [0.5, 0.4, -0.1]] -> row 0: column 1, sign -1; row 1: column 0, sign +1
+    gi, gs = cast.m_step(np.array([[0.2, -3.0, 1.0], [0.5, 0.4, -0.1]]), np.zeros((2, 1)), np.zeros((1, 3)))
+    assert gi.tolist() == [1, 0] and gs.tolist() == [-1, 1]
+    # objective of that choice: (0.04 + 4 + 1) + (0.25 + 0.16 + 0.01) = 5.46
+    assert cast.objective(np.array([[0.2, -3.0, 1.0], [0.5, 0.4, -0.1]]), gi, gs, np.zeros((2, 1)), np.zeros((1, 3))) \
+        == pytest.approx(5.46, abs=1e-12)
+
+
+def test_lopa_approximation_uv_step_is_the_best_rank_r_matrix():
+    cast = oracle.lopa_cast
+    H, D, r = 12, 9, 3
+    W = RNG.standard_normal((H, D))
+    g_idx, g_sign = cast.m_step(W, np.zeros((H, r)), np.zeros((r, D)))
+    U, V = cast.uv_step(W, g_idx, g_sign, r)
+    A = W.copy()
+    A[np.arange(H), g_idx] -= g_sign
+    sv = np.linalg.svd(A, compute_uv=False)
+    # Eckart-Young: the error of the best rank-r approximation is the energy of the dropped singular values
+    assert cast.objective(W, g_idx, g_sign, U, V) == pytest.approx((sv[r:] ** 2).sum(), rel=1e-12)
+    assert np.linalg.matrix_rank(U @ V) == r
+    # no other rank-r matrix does better (random perturbations of the factors)
+    for _ in range(20):
+        U2, V2 = U + 0.05 * RNG.standard_normal(U.shape), V + 0.05 * RNG.standard_normal(V.shape)
+        assert cast.objective(W, g_idx, g_sign, U2, V2) >= cast.objective(W, g_idx, g_sign, U, V)
+    # full rank: nothing is left
+    Uf, Vf = cast.uv_step(W, g_idx, g_sign, min(H, D))
+    assert cast.objective(W, g_idx, g_sign, Uf, Vf) < 1e-20
+
+
+def test_lopa_approximation_descends_and_recovers_a_planted_gate():
+    cast = oracle.lopa_cast
+    H, D, r = 40, 24, 4
+    # the objective never increases, half-step by half-step (the guarantee stated with the algorithm)
+    W = RNG.standard_normal((H, D)) / np.sqrt(D)
+    out = cast.lopa_approximation(W, r, n_iter=5)
+    tr = np.array(out["trace"])
+    assert (np.diff(tr) <= 1e-12).all() and tr[-1] < tr[0]
+    assert tr[0] == pytest.approx(cast.objective(W, out["g_idx"] * 0 + np.argmax(np.abs(W), 1), np.sign(
+        W[np.arange(H), np.argmax(np.abs(W), 1)]), np.zeros((H, r)), np.zeros((r, D))))   # first M-step: U = V = 0
+    # a matrix that is exactly M0 + U0 V0 with small low-rank part is recovered: first M-step finds M0, the SVD the rest
+    gi0 = RNG.integers(0, D, H)
+    gs0 = RNG.choice([-1, 1], H)
+    U0, V0 = 0.1 * RNG.standard_normal((H, r)), 0.1 * RNG.standard_normal((r, D))
+    Wp = U0 @ V0
+    Wp[np.arange(H), gi0] += gs0
+    rec = cast.lopa_approximation(Wp, r, n_iter=2)
+    assert rec["g_idx"].tolist() == gi0.tolist() and rec["g_sign"].tolist() == gs0.tolist()
+    assert rec["trace"][-1] < 1e-20
+    np.testing.assert_allclose(rec["U"] @ rec["V"], U0 @ V0, atol=1e-12)
+    # the result drives the gate of Eq. 3 without RMSNorm: z = M x + U V x equals the materialised matrix times x
+    x = RNG.standard_normal(D).astype(np.float32)
+    z = oracle.gate_lopa(rec["V"], rec["U"], x, g_idx=rec["g_idx"], g_sign=rec["g_sign"], use_rmsnorm=False)
+    np.testing.assert_allclose(z, Wp @ x.astype(np.float64), atol=1e-10)
