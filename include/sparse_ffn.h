@@ -227,6 +227,20 @@ const char* sffn_last_cuda_error(void);
 int sffn_residual_cast(const float* y, const void* resid, float alpha, void* out, int n, int dtype /* sffn_dtype */,
                        void* stream);
 
+/* Offline conversion of a full gate matrix W [H,D] (fp32) into a LoPA gate M + U V (architecture casting, Sec. 3.4,
+ * "LoPA approximation": minimise ||W - M - U V||_F^2 by alternating two exact half-steps, M first, from U = V = 0).
+ * These two calls are the half-steps' element-wise parts; the truncated SVD of the UV-step and the product U V are
+ * left to a library (the Python package drives the loop, `lopa_approximation`).  All pointers are DEVICE memory.
+ *
+ * sffn_lopa_m_step: R = W - P (P [H,D] = U V, or NULL for the first step).  For every row i: g_idx[i] = column of the
+ *   largest |R_ij| (the first one on ties), g_sign[i] = sign of that entry (+1 for an exact zero), row_best[i] =
+ *   |R_ij| there, row_energy[i] = sum_j R_ij^2 (either may be NULL).  The objective after the step is
+ *   sum_i (row_energy[i] - 2 row_best[i] + 1); called with W := W - M it also yields the objective after a UV-step.
+ * sffn_lopa_residual: A = W - M, M[i, g_idx[i]] = g_sign[i]: the matrix whose truncated SVD at rank r is the best U V. */
+int sffn_lopa_m_step(const float* W, const float* P, int H, int D, int32_t* g_idx, int8_t* g_sign, double* row_energy,
+                     float* row_best, void* stream);
+int sffn_lopa_residual(const float* W, const int32_t* g_idx, const int8_t* g_sign, int H, int D, float* A, void* stream);
+
 /* Static string for a status code. */
 const char* sffn_status_string(int status);
 

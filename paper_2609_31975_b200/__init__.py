@@ -14,4 +14,4 @@ from .binding import (  # noqa: F401
     residual_cast,
     sparse_ffn_forward_static,
 )
-from .lopa import g_diagonal, g_tiled, touched_bytes, dense_bytes  # noqa: F401
+from .lopa import g_diagonal, g_tiled, touched_bytes, dense_bytes, lopa_approximation  # noqa: F401

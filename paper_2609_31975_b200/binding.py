@@ -71,6 +71,8 @@ def load_library() -> ctypes.CDLL:
         lib.sffn_status_string.argtypes = [i]
         lib.sffn_residual_cast.argtypes = [vp, vp, ctypes.c_float, vp, i, i, vp]
         lib.sffn_status_string.restype = ctypes.c_char_p
+        lib.sffn_lopa_m_step.argtypes = [vp, vp, i, i, vp, vp, vp, vp, vp]
+        lib.sffn_lopa_residual.argtypes = [vp, vp, vp, i, i, vp, vp]
         lib.sffn_last_cuda_error.argtypes = []
         lib.sffn_last_cuda_error.restype = ctypes.c_char_p
         _lib = lib
@@ -124,6 +126,36 @@ def residual_cast(y, resid, alpha, out, stream=None):
            lib.sffn_residual_cast(_ptr(y), _ptr(resid), float(alpha), _ptr(out), y.numel(),
                                   1 if out.dtype == torch.bfloat16 else 0, ctypes.c_void_p(s.cuda_stream)))
     return out
+
+
+def lopa_m_step(W, P=None, stream=None):
+    """M-step of the LoPA approximation (Sec. 3.4) on fp32 device tensors: per row of R = W - P the column of the
+    largest |R_ij| and its sign.  Returns (g_idx int32 [H], g_sign int8 [H], row_energy float64 [H], row_best fp32 [H])."""
+    lib = load_library()
+    if W.dtype != torch.float32 or not W.is_cuda or not W.is_contiguous() or W.dim() != 2:
+        raise TypeError("W must be a contiguous fp32 CUDA matrix")
+    if P is not None and (P.dtype != torch.float32 or P.shape != W.shape or not P.is_contiguous()):
+        raise TypeError("P must match W")
+    H, D = W.shape
+    g_idx = torch.empty(H, dtype=torch.int32, device=W.device)
+    g_sign = torch.empty(H, dtype=torch.int8, device=W.device)
+    energy = torch.empty(H, dtype=torch.float64, device=W.device)
+    best = torch.empty(H, dtype=torch.float32, device=W.device)
+    s = torch.cuda.current_stream(W.device) if stream is None else stream
+    _check("sffn_lopa_m_step", lib.sffn_lopa_m_step(_ptr(W), _ptr(P), H, D, _ptr(g_idx), _ptr(g_sign), _ptr(energy),
+                                                    _ptr(best), ctypes.c_void_p(s.cuda_stream)))
+    return g_idx, g_sign, energy, best
+
+
+def lopa_residual(W, g_idx, g_sign, stream=None):
+    """A = W - M for the one-nonzero-per-row matrix M described by (g_idx, g_sign); fp32 device tensors."""
+    lib = load_library()
+    H, D = W.shape
+    A = torch.empty_like(W)
+    s = torch.cuda.current_stream(W.device) if stream is None else stream
+    _check("sffn_lopa_residual", lib.sffn_lopa_residual(_ptr(W), _ptr(g_idx), _ptr(g_sign), H, D, _ptr(A),
+                                                        ctypes.c_void_p(s.cuda_stream)))
+    return A
 
 
 class SparseFFN:

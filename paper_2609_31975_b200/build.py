@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libsparse_ffn.so"
-SOURCES = ["api.cu", "general_kernels.cu", "fused_kernel.cu", "static_entry.cu", "batched_kernels.cu", "umma_kernels.cu"]
+SOURCES = ["api.cu", "general_kernels.cu", "fused_kernel.cu", "static_entry.cu", "batched_kernels.cu", "umma_kernels.cu", "cast_kernels.cu"]
 
 
 def _stale() -> bool:

@@ -9,6 +9,7 @@
 #include <new>
 
 #include "batched_kernels.cuh"
+#include "cast_kernels.cuh"
 #include "common.cuh"
 #include "fused_kernel.cuh"
 #include "general_kernels.cuh"
@@ -580,6 +581,19 @@ int sffn_residual_cast(const float* y, const void* resid, float alpha, void* out
   if (!y || !resid || !out || n < 4 || n % 4 || (dtype != SFFN_F32 && dtype != SFFN_BF16)) return SFFN_ERR_INVALID_ARG;
   if (!aligned16(y) || !aligned16(resid) || !aligned16(out)) return SFFN_ERR_UNSUPPORTED;
   SFFN_CUDA(sffn::launch_residual_cast(dtype == SFFN_BF16, y, resid, alpha, out, n, static_cast<cudaStream_t>(stream)));
+  return SFFN_OK;
+}
+
+int sffn_lopa_m_step(const float* W, const float* P, int H, int D, int32_t* g_idx, int8_t* g_sign, double* row_energy,
+                     float* row_best, void* stream) {
+  if (!W || !g_idx || !g_sign || H < 1 || D < 1) return SFFN_ERR_INVALID_ARG;
+  SFFN_CUDA(sffn::launch_lopa_m_step(W, P, H, D, g_idx, g_sign, row_energy, row_best, static_cast<cudaStream_t>(stream)));
+  return SFFN_OK;
+}
+
+int sffn_lopa_residual(const float* W, const int32_t* g_idx, const int8_t* g_sign, int H, int D, float* A, void* stream) {
+  if (!W || !g_idx || !g_sign || !A || H < 1 || D < 1) return SFFN_ERR_INVALID_ARG;
+  SFFN_CUDA(sffn::launch_lopa_residual(W, g_idx, g_sign, H, D, A, static_cast<cudaStream_t>(stream)));
   return SFFN_OK;
 }
 

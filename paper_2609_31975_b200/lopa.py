@@ -32,3 +32,33 @@ def touched_bytes(D: int, H: int, n_rows: int, esz: int, B: int = 1, r: int | No
 def dense_bytes(D: int, H: int, esz: int, B: int = 1, r: int | None = None) -> int:
     """Bytes of the dense comparator: as touched_bytes with all H rows."""
     return touched_bytes(D, H, H, esz, B, r)
+
+
+def lopa_approximation(W: torch.Tensor, r: int, n_iter: int = 4) -> dict:
+    """Architecture casting (Sec. 3.4, "LoPA approximation"): replaces a full gate matrix W [H, D] (fp32, on the GPU)
+    by M + U V with one +-1 per row of M, minimising ||W - M - U V||_F^2 by alternating minimisation from U = V = 0,
+    M-step first.  The row-wise and element-wise parts run in this library's kernels (``sffn_lopa_m_step``,
+    ``sffn_lopa_residual``); the truncated SVD and the product U V are torch's (cuSOLVER / cuBLAS).
+
+    Returns dict(g_idx int32 [H], g_sign int8 [H], U [H, r], V [r, D], trace): ``trace`` lists the objective after every
+    half-step (M, UV, M, UV, ...).  Feed the result to ``sparse_ffn_forward`` as a LoPA gate with ``use_rmsnorm=False``
+    (architecture casting has no RMSNorm between U and V), cast to the handle's dtype.
+    """
+    from .binding import lopa_m_step, lopa_residual
+
+    W = W.contiguous().float()
+    H, D = W.shape
+    U = torch.zeros((H, r), dtype=torch.float32, device=W.device)
+    V = torch.zeros((r, D), dtype=torch.float32, device=W.device)
+    P = None
+    trace = []
+    for _ in range(n_iter):
+        g_idx, g_sign, energy, best = lopa_m_step(W, P)
+        trace.append(float((energy - 2.0 * best.double() + 1.0).sum()))
+        A = lopa_residual(W, g_idx, g_sign)
+        Pm, sv, Qt = torch.linalg.svd(A, full_matrices=False)
+        U, V = (Pm[:, :r] * sv[:r]).contiguous(), Qt[:r].contiguous()
+        P = U @ V
+        _, _, energy, _ = lopa_m_step(A, P)      # || (W - M) - U V ||^2 row by row
+        trace.append(float(energy.sum()))
+    return dict(g_idx=g_idx, g_sign=g_sign, U=U, V=V, trace=trace)
