@@ -1,6 +1,6 @@
 // Fused sparse gated FFN for one token on B200 (sm_100a).
 //
-// Main kernel: one persistent CTA per SM owns a share ("slab") of the H neurons and runs the whole
+// One kernel per call: one persistent CTA per SM owns a share ("slab") of the H neurons and runs the whole
 // of the paper's sparse execution scheme (Sec. 3.1) on it without leaving the SM:
 //
 //   gate producers two threads (two warps) stream the slab's gate rows (W_1, or U for the LoPA gate) into a
@@ -16,12 +16,13 @@
 //                  reduction), h_j = a_j u_j, y_part += h_j W_down[j]; each thread keeps its own
 //                  column slice of y_part in registers and writes it out once.
 //
-// A small second kernel sums the per-CTA partials in CTA order (deterministic, no float atomics).
+// The last CTAs to finish sum the per-CTA partials in CTA order (deterministic, no float atomics).
+// Weights are fp32, bf16 or int8 codes with one fp32 scale per row (bf16 token).
 // For the LoPA gate (Eq. 3, Sec. 3.3) the rank-r stage v = V x is spread over the CTAs of the main
 // kernel, exchanged through global memory (bounded wait on an arrival counter) and normalised (RMSNorm)
 // into shared memory, with the U rows already sitting in the ring.
 //
-// The kernels are chained with programmatic dependent launch: each lets its successor start early
+// Calls are chained with programmatic dependent launch: a kernel lets its successor start early
 // and waits (griddepcontrol.wait) only before it touches anything a predecessor may write.  Weights
 // are read before that wait -- they are parameters, not results -- so the next call's gate stream
 // starts on an SM the moment the previous call's CTA leaves it.
