@@ -41,6 +41,30 @@ def _time(calls, stream, reps=3):
     return statistics.median(best), min(best)
 
 
+def _time_graph(calls, stream, replays=5):
+    """The same sequence of calls captured once in a CUDA graph and replayed: no host work between the calls."""
+    with torch.cuda.stream(stream):
+        for c in calls[: min(len(calls), 16)]:
+            c()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for c in calls:
+                c()
+        graph.replay()
+        stream.synchronize()
+        times = []
+        for _ in range(replays):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e3 / len(calls))
+        del graph
+    return statistics.median(times), min(times)
+
+
 def _is_q8(w):
     return isinstance(w["W_up"], dict)
 
@@ -53,7 +77,7 @@ def _bytes(D, H, n_rows, esz, B, r, q8):
     return touched_bytes(D, H, n_rows, 1, B, r) + B * D + 4 * (H + 2 * n_rows + (r or 0))
 
 
-def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1, act_up=None):
+def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1, act_up=None, graph=False):
     """sets: list of weight dicts; gate_of(w) -> gate dict; act_up: activation on the up projection (double
     activation) or None.  Returns one result row."""
     ffn = SparseFFN(D, H, torch.bfloat16, r_max=r or 0, B_max=B, device=DEV)
@@ -74,7 +98,7 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=6549.1,
         dense_calls.append(ffn.prepared(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt, dense=True,
                                         stream=stream))
     n_rows = statistics.mean(rows)
-    us, us_min = _time(sparse_calls, stream)
+    us, us_min = _time_graph(sparse_calls, stream) if graph else _time(sparse_calls, stream)
     us_dense, _ = _time(dense_calls[: max(16, n_calls // 4)], stream, reps=2)
     status = ffn.device_status()
     q8 = _is_q8(sets[0])
@@ -177,6 +201,10 @@ def run(out_path, quick=False, only=None, n_calls=None):
         add(f"decode 4096x14336 s={s}", D, H, 1, sets, std, "relu", peak=peak)
         if s == 0.9:  # double activation (RELU on the up projection as well): same rows read, one more epilogue op
             add(f"decode 4096x14336 s={s} double activation", D, H, 1, sets, std, "relu", peak=peak, act_up="relu")
+            # the same 200 calls captured in one CUDA graph and replayed (no host work between calls), and the warm
+            # figure: one weight set only, so part of every call's bytes comes from L2 (not a roofline number)
+            add(f"decode 4096x14336 s={s} (one CUDA graph of the calls)", D, H, 1, sets, std, "relu", peak=peak, graph=True)
+            add(f"decode 4096x14336 s={s} warm (a single weight set, L2 hits)", D, H, 1, sets[:1], std, "relu", peak=peak)
     # batched decode under Zipf firing
     p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
     zb = syn.bias_from_firing_profile(p).to(DEV)
