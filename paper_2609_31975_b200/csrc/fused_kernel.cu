@@ -557,25 +557,59 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status)) break;
       const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
       float mine = 0.f;
-      // Short gate rows (LoPA: r elements): a row is a few chunks per lane and its cost is the latency of the
-      // warp reduction, so four rows are dotted and reduced side by side.
+      // Short gate rows (LoPA: r elements): a row is a few chunks per lane, and with one warp per scheduler the cost is
+      // instruction latency, not throughput.  Eight rows are dotted side by side (eight independent chains, the vector
+      // read once for all of them, every load requested before the first multiply) and reduced together: each
+      // exchange halves the number of sums a lane carries, so eight rows cost 4 + 2 + 1 + 1 + 1 shuffles instead of 40.
       const int rows_short = nvecK <= 128 ? rows : 0;
-      for (int rr = 0; rr < rows_short; rr += 4) {
-        float a[4] = {0.f, 0.f, 0.f, 0.f};
+      int rr_short = 0;
+      for (; rows_short - rr_short > 2; rr_short += 8) {  // one or two left-over rows are cheaper one by one (below)
+        const int rr = rr_short;
+        float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int c = lane; c < nvecK; c += 32) {
+          uint4 w[8];
+          float4 v[EPV / 4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            if (rr + i < rows)
-              a[i] = chunk_dot<T>(reinterpret_cast<const uint4*>(base + (size_t)(rr + i) * gate_row_bytes)[c], gvec, c,
-                                  nvecK, a[i]);
+          for (int i = 0; i < 8; ++i)
+            w[i] = rr + i < rows ? reinterpret_cast<const uint4*>(base + (size_t)(rr + i) * gate_row_bytes)[c]
+                                 : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+          for (int q = 0; q < EPV / 4; ++q) v[q] = reinterpret_cast<const float4*>(gvec)[q * nvecK + c];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float f[EPV];
+            Elem<T>::unpack(w[i], f);
+#pragma unroll
+            for (int q = 0; q < EPV / 4; ++q) {
+              a[i] = fmaf(f[4 * q + 0], v[q].x, a[i]);
+              a[i] = fmaf(f[4 * q + 1], v[q].y, a[i]);
+              a[i] = fmaf(f[4 * q + 2], v[q].z, a[i]);
+              a[i] = fmaf(f[4 * q + 3], v[q].w, a[i]);
+            }
+          }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) a[i] += __shfl_xor_sync(0xffffffffu, a[i], o);
+        // lanes with bit 4 set keep rows 4..7, the others rows 0..3; then bit 3 picks two of the four, bit 2 one of
+        // the two; bits 1 and 0 are plain sums.  Afterwards lanes 4 k .. 4 k + 3 hold the dot product of row rr + k.
+        float b4[4], b2[2];
+        const bool up16 = lane & 16, up8 = lane & 8, up4 = lane & 4;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          if (lane == rr + i) mine = a[i];
+          b4[i] = (up16 ? a[4 + i] : a[i]) + __shfl_xor_sync(0xffffffffu, up16 ? a[i] : a[4 + i], 16);
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+          b2[i] = (up8 ? b4[2 + i] : b4[i]) + __shfl_xor_sync(0xffffffffu, up8 ? b4[i] : b4[2 + i], 8);
+        float z = (up4 ? b2[1] : b2[0]) + __shfl_xor_sync(0xffffffffu, up4 ? b2[0] : b2[1], 4);
+        z += __shfl_xor_sync(0xffffffffu, z, 2);
+        z += __shfl_xor_sync(0xffffffffu, z, 1);
+        const float got = __shfl_sync(0xffffffffu, z, 4 * ((lane - rr) & 7));
+        if (lane >= rr && lane < rr + 8) mine = got;
+      }
+      for (; rr_short < rows_short; ++rr_short) {
+        const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr_short * gate_row_bytes);
+        float a0 = 0.f;
+        for (int c = lane; c < nvecK; c += 32) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
+        const float z = warp_sum(a0);
+        if (lane == rr_short) mine = z;
       }
       int rr_single = rows_short;
       if (EPV == 16) {
@@ -867,6 +901,19 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   if (scaled && g.cpt == 8) return g;  // 128 accumulators per act thread: the CUDA-core path takes such rows
   int nr = 8192 / gate_row_bytes;
   nr = nr < 1 ? 1 : nr > 32 ? 32 : nr;
+  if (lopa) {
+    // Short gate (LoPA): when the CTA's whole share of U fits in three slots per gate warp with a few more rows per
+    // slot, take them: every row is then on its way before the token arrives and none waits for a slot to come free
+    // (r = 512 at 14336 neurons: 11 slots of 9 rows instead of 13 of 8, whose last arrived 2 us into the gate phase).
+    const int share = (H + grid - 1) / grid;
+    for (int cand = nr; cand <= 32; ++cand) {
+      const int slots = (share + cand - 1) / cand + 1;  // + 1: block-cyclic dealing can give one CTA an extra block
+      if (slots <= 3 * gate_warps_max && slots * cand * gate_row_bytes <= 112 * 1024) {
+        nr = cand;
+        break;
+      }
+    }
+  }
   g.rows_per_gate_slot = nr;
   g.gate_slot_bytes = (nr * gate_row_bytes + 127) / 128 * 128;
   g.act_slot_bytes = (2 * row_bytes + 127) / 128 * 128;
