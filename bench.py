@@ -206,9 +206,17 @@ def cpu_baseline(sample_tokens=96, sparsity=SPARSITY, seed=2):
     t0 = time.perf_counter()
     oracle.ffn(x, w["W_up"], w["W_down"], ACT, W_g=w["W_g"], b_g=w["b_g"], route="sparse", threads=cores)
     dt = time.perf_counter() - t0
+    # one thread, sparse and dense route, on a few tokens: what one host core does per call
+    n1 = min(4, sample_tokens)
+    t1 = time.perf_counter()
+    oracle.ffn(x[:n1], w["W_up"], w["W_down"], ACT, W_g=w["W_g"], b_g=w["b_g"], route="sparse", threads=1)
+    t2 = time.perf_counter()
+    oracle.ffn(x[:n1], w["W_up"], w["W_down"], ACT, W_g=w["W_g"], b_g=w["b_g"], route="dense", threads=1)
+    t3 = time.perf_counter()
     return {"value": dt / sample_tokens * 1e6, "unit": "us/FFN-call", "cores": min(cores, sample_tokens),
             "kind": "oracle", "sample": f"{sample_tokens} tokens of the same workload, one weight set, sparse route, "
-                                        f"OpenMP over tokens ({dt:.1f} s wall)"}
+                                        f"OpenMP over tokens ({dt:.1f} s wall)",
+            "single_thread_us": {"sparse": (t2 - t1) / n1 * 1e6, "dense": (t3 - t2) / n1 * 1e6, "tokens": n1}}
 
 
 def run_reference(args, rank):
