@@ -450,3 +450,29 @@ def test_config5_full_size_stress_layer0(mod):
         y = ffn8.sparse_ffn_forward(x8, gt, ww["b_g"], ww["W_up"], ww["W_down"], "sqrelu")
         assert_y_close(y, ref["y"], what="config5 lopa B=8")
         assert_active_set(ffn8.last_active(), ref, what="config5 lopa B=8")
+
+
+def test_two_handles_on_two_streams_overlap_and_agree(mod):
+    # Two standard-gate single-token calls in flight at once (different handles, different streams): each wants every SM
+    # and its last CTAs wait for the rest, but at most 63 + 63 CTAs sit waiting, so both complete -- and bit for bit with
+    # what they give one after the other.
+    D, H = 4096, 14336
+    sets = [syn.standard_ffn(D, H, torch.bfloat16, 90 + i, DEV, sparsity=0.9) for i in range(2)]
+    x = syn.tokens(40, D, torch.bfloat16, 90, DEV)
+    ffns = [mod.SparseFFN(D, H, torch.bfloat16, B_max=1) for _ in range(2)]
+    streams = [torch.cuda.Stream(DEV) for _ in range(2)]
+    want = [torch.empty((40, D), device=DEV) for _ in range(2)]
+    for i in range(2):
+        for t in range(40):
+            ffns[i].sparse_ffn_forward(x[t], {"W_g": sets[i]["W_g"]}, sets[i]["b_g"], sets[i]["W_up"], sets[i]["W_down"],
+                                       "relu", want[i][t])
+        torch.cuda.synchronize()
+    got = [torch.zeros((40, D), device=DEV) for _ in range(2)]
+    for t in range(40):
+        for i in range(2):
+            ffns[i].sparse_ffn_forward(x[t], {"W_g": sets[i]["W_g"]}, sets[i]["b_g"], sets[i]["W_up"], sets[i]["W_down"],
+                                       "relu", got[i][t], stream=streams[i])
+    torch.cuda.synchronize()
+    for i in range(2):
+        assert ffns[i].device_status() == 0
+        assert torch.equal(got[i], want[i])
