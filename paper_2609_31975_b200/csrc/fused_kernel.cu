@@ -105,7 +105,7 @@ struct SmemLayout {
     sn = take(lopa ? K * 4 : 0);
     aval = take(slab_max * 4);
     slot_a = take(n_act_slots * 4);
-    red = take(3 * 16 * 16);  // act warps: 2 x (2 x 8 + 1) floats; afterwards the scratch of the cross-CTA sum
+    red = take(2 * (2 * 8 + 1) * 4);  // up to eight act warps
     ctl = take(8 * 4);
     bars = take(2 * (n_gate_slots + n_act_slots) * 8);
     row_params = take((lopa || scaled) ? (1 + (lopa ? 2 : 0) + (scaled ? 1 : 0)) * slab_max * 4 : 0);  // per-neuron gate parameters
@@ -835,26 +835,25 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const int32_t failed = __ldcg(p.status);  // in flight together with the partials, not after them
   const int cols = (Q + R - 1) / R;
   const int q_hi = min(Q, (slice + 1) * cols);
-  // Twelve warps = 4 groups of four columns x 3 row parts.  Lane (r8, c4) reads column c4 of its group in the rows
-  // 8 (3 i + part) + r8: one warp load covers eight rows x 64 contiguous bytes (whole 32-byte sectors).
-  static_assert(kGW + kAW == 12, "reduction tail is laid out for twelve warps");
-  const int part = tw % 3, cgw = tw / 3, r8 = lane >> 2, c4 = lane & 3;
-  float4* scratch = reinterpret_cast<float4*>(red);  // [3 parts][16 columns]; the act warps are done with it
-  const int tt = tid - 32 * kFirstGateWarp;
+  // Four warps, one group of four columns each.  Lane (r8, c4) reads column c4 of its group in the rows r8, r8 + 8,
+  // ...: one warp load covers eight rows x 64 contiguous bytes (whole 32-byte sectors), twenty loads are in flight per
+  // lane (160 CTAs; more take another pass), the eight row residues are combined by shuffles in a fixed order.
+  const int r8 = lane >> 2, c4 = lane & 3;
+  if (tw >= 4) return;
   for (int c0 = slice * cols; c0 < q_hi; c0 += 16) {
-    const int q = c0 + 4 * cgw + c4;
+    const int q = c0 + 4 * tw + c4;
     float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
     if (q < q_hi) {
       const float4* src = reinterpret_cast<const float4*>(p.partial) + q;
-      for (int i0 = 0; 8 * (3 * i0 + part) < G; i0 += 8) {
-        float4 v[8];
+      for (int i0 = 0; 8 * i0 < G; i0 += 20) {
+        float4 v[20];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int g = 8 * (3 * (i0 + i) + part) + r8;
+        for (int i = 0; i < 20; ++i) {
+          const int g = 8 * (i0 + i) + r8;
           v[i] = g < G ? __ldcg(src + (size_t)g * Q) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 20; ++i) {
           s4.x += v[i].x; s4.y += v[i].y; s4.z += v[i].z; s4.w += v[i].w;
         }
       }
@@ -866,14 +865,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       s4.z += __shfl_xor_sync(0xffffffffu, s4.z, o);
       s4.w += __shfl_xor_sync(0xffffffffu, s4.w, o);
     }
-    if (r8 == 0) scratch[part * 16 + 4 * cgw + c4] = s4;
-    named_bar_sync(6, kTail);
-    if (tt < 16 && c0 + tt < q_hi && failed == 0) {
-      const float4 a = scratch[tt], b = scratch[16 + tt], c = scratch[32 + tt];
-      reinterpret_cast<float4*>(p.y)[c0 + tt] =
-          make_float4((a.x + b.x) + c.x, (a.y + b.y) + c.y, (a.z + b.z) + c.z, (a.w + b.w) + c.w);
-    }
-    if (c0 + 16 < q_hi) named_bar_sync(6, kTail);  // the scratch is reused by the next pass
+    if (r8 == 0 && q < q_hi && failed == 0) reinterpret_cast<float4*>(p.y)[q] = s4;
   }
   if (tid == 32 * kFirstGateWarp) SFFN_GSTAMP(13);
 }
