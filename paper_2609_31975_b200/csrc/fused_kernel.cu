@@ -442,10 +442,12 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       const float v = warp_sum(a0 + a1) * (kScaled ? __ldg(p.s_V + k) : 1.f);
       if (lane == 0) __stcg(p.vbuf + k, v);
     }
-    __threadfence();
     named_bar_sync(5, kStageThreads);
     if (tid == kStageBase) {
-      const unsigned long long v_target = (atomicAdd(p.v_counter, 1ULL) / G + 1) * G;
+      // release at device scope after the barrier: this CTA's rows of v happen before it
+      unsigned long long arrived;
+      asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(arrived) : "l"(p.v_counter) : "memory");
+      const unsigned long long v_target = (arrived / G + 1) * G;
       const long long t0 = clock64();
       for (;;) {
         unsigned long long seen;
