@@ -185,8 +185,15 @@ int sparse_ffn_forward_host(sffn_handle* handle, const void* x_host, int B, cons
 int sffn_last_active(sffn_handle* handle, const int32_t** idx_dev, const int32_t** count_dev,
                      void* stream);
 
-/* Reads the device status word (synchronises the device): SFFN_OK or SFFN_ERR_TIMEOUT. */
+/* Reads the device status word (synchronises the device): SFFN_OK or SFFN_ERR_TIMEOUT.  The word is sticky: once a
+ * bounded wait has run out, the single-token kernels' arrival counters are out of step and every later call on the
+ * handle leaves y unwritten until sffn_reset. */
 int sffn_last_device_status(sffn_handle* handle, int* status);
+
+/* Puts a handle back into its initial state after SFFN_ERR_TIMEOUT: clears the status word and the arrival counters
+ * (two small asynchronous memsets on `stream`, ordered like a call).  The handle's stream must hold no unfinished
+ * call of this handle that could still time out.  Weights, settings and the workspace's other contents are kept. */
+int sffn_reset(sffn_handle* handle, void* stream);
 
 /* Number of kernels this handle has launched since creation (host-side counter). */
 int sffn_launch_count(sffn_handle* handle, long long* launches);
@@ -248,6 +255,29 @@ int sffn_lopa_residual(const float* W, const int32_t* g_idx, const int8_t* g_sig
 
 /* Static string for a status code. */
 const char* sffn_status_string(int status);
+
+/* ---- test hooks ----------------------------------------------------------------------------------------------
+ * Not steps of the paper's method: they let the tests look at launch geometry without a GPU and exercise the
+ * device-side failure handling without ever hanging or faulting a GPU.  Process-wide, not thread-safe.
+ *
+ * sffn_test_fused_plan: geometry of the single-token CUDA-core kernel for a shape, as nine integers: ok, rows per
+ *   gate slot, gate slot bytes, gate slots, gate warps, act slot bytes, act slots, chunks per act thread, shared
+ *   memory bytes (wkind: 0 fp32, 1 bf16, 2 int8 rows).  sffn_test_umma_tiling: tiling of the batched gate GEMM.
+ * sffn_test_set_knob: PDL = programmatic dependent launch between calls (default 1); TENSOR_GATE = take the
+ *   tensor-core gate in single-token bf16 calls where it applies (default 1); WAIT_CYCLES = budget of every
+ *   device-side wait in clock cycles (default 2^31, about a second; 0 restores it); SKIP_ARRIVAL_CTA = index of a CTA
+ *   of the single-token kernels that does not report itself finished, so that the CTAs which sum the partial
+ *   results see their (bounded) wait run out and record SFFN_ERR_TIMEOUT (-1 = none, the default; use it with a
+ *   small WAIT_CYCLES); RING_GATE_SLOTS / RING_ACT_SLOTS = split of the tensor-core kernel's shared-memory rings
+ *   (0 = planned); TRACE_BUFFER = device address of [grid][16] int64 time stamps, written only by libraries built
+ *   with -DSFFN_TRACE. */
+typedef enum {
+  SFFN_KNOB_PDL = 0, SFFN_KNOB_TENSOR_GATE = 1, SFFN_KNOB_WAIT_CYCLES = 2, SFFN_KNOB_SKIP_ARRIVAL_CTA = 3,
+  SFFN_KNOB_RING_GATE_SLOTS = 4, SFFN_KNOB_RING_ACT_SLOTS = 5, SFFN_KNOB_TRACE_BUFFER = 6
+} sffn_test_knob;
+void sffn_test_fused_plan(int wkind, int D, int H, int K, int lopa, int sm_count, int* out9);
+void sffn_test_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list);
+int sffn_test_set_knob(int knob, long long value);
 
 #ifdef __cplusplus
 }

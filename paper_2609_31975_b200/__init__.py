@@ -13,5 +13,6 @@ from .binding import (  # noqa: F401
     load_library,
     residual_cast,
     sparse_ffn_forward_static,
+    test_set_knob,
 )
 from .lopa import g_diagonal, g_tiled, touched_bytes, dense_bytes, lopa_approximation  # noqa: F401

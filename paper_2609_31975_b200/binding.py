@@ -36,7 +36,11 @@ class _Q8Scales(ctypes.Structure):
 
 
 def lib_path() -> Path:
-    return _PKG / "libsparse_ffn.so"
+    """The library this process loads: libsparse_ffn.so, or the build named by SFFN_LIBRARY (e.g. the time-stamp
+    build libsparse_ffn_trace.so)."""
+    import os
+
+    return _PKG / os.environ.get("SFFN_LIBRARY", "libsparse_ffn.so")
 
 
 _lib = None
@@ -75,8 +79,19 @@ def load_library() -> ctypes.CDLL:
         lib.sffn_lopa_residual.argtypes = [vp, vp, vp, i, i, vp, vp]
         lib.sffn_last_cuda_error.argtypes = []
         lib.sffn_last_cuda_error.restype = ctypes.c_char_p
+        lib.sffn_test_set_knob.argtypes = [i, ctypes.c_longlong]
+        lib.sffn_reset.argtypes = [vp, vp]
         _lib = lib
     return _lib
+
+
+KNOB = {"pdl": 0, "tensor_gate": 1, "wait_cycles": 2, "skip_arrival_cta": 3, "ring_gate_slots": 4,
+        "ring_act_slots": 5, "trace_buffer": 6}
+
+
+def test_set_knob(name: str, value: int):
+    """Process-wide test hook of the library (see the "test hooks" section of sparse_ffn.h)."""
+    _check("sffn_test_set_knob", load_library().sffn_test_set_knob(KNOB[name], int(value)))
 
 
 def _ptr(t):
@@ -325,6 +340,10 @@ class SparseFFN:
         out = ctypes.c_int(0)
         _check("sffn_last_device_status", self.lib.sffn_last_device_status(self._h, ctypes.byref(out)))
         return out.value
+
+    def reset(self, stream=None):
+        """Clears the device status word and the arrival counters after a device-side timeout."""
+        _check("sffn_reset", self.lib.sffn_reset(self._h, self._stream(stream)))
 
     def launch_count(self) -> int:
         out = ctypes.c_longlong(0)

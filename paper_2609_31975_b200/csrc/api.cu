@@ -152,17 +152,27 @@ int sffn_set_path(sffn_handle* h, int path) {
   return SFFN_OK;
 }
 
-// Experiment knob (not part of the documented ABI).
-void sffn_debug_set_pdl(int on) { sffn::debug_set_pdl(on); }
-// Host-side geometry of the kernels for a shape (no GPU needed): see debug_fused_plan / umma_gate_tiling.
-void sffn_debug_fused_plan(int wkind, int D, int H, int K, int lopa, int sm_count, int* out9) {
+// ---- test hooks (declared in the last section of sparse_ffn.h) ------------------------------------------------
+void sffn_test_fused_plan(int wkind, int D, int H, int K, int lopa, int sm_count, int* out9) {
   sffn::debug_fused_plan(wkind, D, H, K, lopa != 0, sm_count, out9);  // wkind: 0 fp32, 1 bf16, 2 int8 rows
 }
-void sffn_debug_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list) {
+void sffn_test_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list) {
   sffn::umma_gate_tiling(R, sm_count, tile_rows, n_tiles);
   *own_list = sffn::umma_own_list_supported(R, sm_count) ? 1 : 0;
 }
-void sffn_debug_set_trace(void* device_buffer) { sffn::debug_set_trace(static_cast<long long*>(device_buffer)); }
+int sffn_test_set_knob(int knob, long long value) {
+  sffn::FusedTestKnobs& k = sffn::fused_test_knobs();
+  switch (knob) {
+    case SFFN_KNOB_PDL: k.pdl = value != 0; return SFFN_OK;
+    case SFFN_KNOB_TENSOR_GATE: k.tensor_gate = value != 0; return SFFN_OK;
+    case SFFN_KNOB_WAIT_CYCLES: k.wait_cycles = value > 0 ? value : (1LL << 31); return SFFN_OK;
+    case SFFN_KNOB_SKIP_ARRIVAL_CTA: k.skip_arrival_cta = (int)value; return SFFN_OK;
+    case SFFN_KNOB_RING_GATE_SLOTS: k.ring_S = (int)value; return SFFN_OK;
+    case SFFN_KNOB_RING_ACT_SLOTS: k.ring_NA = (int)value; return SFFN_OK;
+    case SFFN_KNOB_TRACE_BUFFER: k.trace = reinterpret_cast<long long*>(static_cast<uintptr_t>(value)); return SFFN_OK;
+    default: return SFFN_ERR_INVALID_ARG;
+  }
+}
 
 int sffn_launch_count(sffn_handle* h, long long* launches) {
   if (!h || !launches) return SFFN_ERR_INVALID_ARG;
@@ -610,6 +620,15 @@ int sffn_last_active(sffn_handle* h, const int32_t** idx_dev, const int32_t** co
   }
   *idx_dev = idx;
   *count_dev = count;
+  return SFFN_OK;
+}
+
+int sffn_reset(sffn_handle* h, void* stream) {
+  if (!h) return SFFN_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  SFFN_CUDA(cudaMemsetAsync(h->ws + h->L.status, 0, 256, s));
+  SFFN_CUDA(cudaMemsetAsync(h->ws + h->L.fused, 0, 256, s));  // the single-token kernels' arrival counters
+  h->list_state = 0;
   return SFFN_OK;
 }
 

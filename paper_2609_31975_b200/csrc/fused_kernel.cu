@@ -51,7 +51,6 @@ constexpr int kStageBase = 32 * kGateProducers;  // first thread that takes part
 constexpr int kStageThreads = kThreads - kStageBase;
 constexpr int kMaxGrid = 256;
 constexpr int kSmemBudget = 227 * 1024;
-constexpr long long kWaitCycles = 1LL << 31;  // about one second at B200 clocks
 
 struct FusedParams {
   int D, H, K;  // K = length of a gate row: D (standard) or r (LoPA)
@@ -85,7 +84,9 @@ struct FusedParams {
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
   int gate_warps;    // gate warps in use; n_gate_slots is a multiple of it, so a ring slot always
                      // belongs to the same warp and its phases are consumed strictly in order
-  long long* trace;  // diagnostics: [grid][16] cycle stamps, or null
+  long long wait_cycles;  // budget of every wait below (about one second unless a test shortens it)
+  int skip_arrival_cta;   // test hook: this CTA does not count itself as finished (-1: none)
+  long long* trace;       // SFFN_TRACE builds: [grid][16] time stamps, or null
 };
 
 // Shared-memory carve-up, identical on host and device.
@@ -163,7 +164,8 @@ __device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status
 // Bounded wait on an mbarrier phase.  try_wait parks the thread in hardware for a short,
 // implementation-defined time, so waiting warps do not steal issue slots from working ones; the
 // cycle budget is checked between attempts.  False when it ran out or the CTA is aborting.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status,
+                                          long long budget) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
@@ -171,7 +173,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 64; ++i)
       if (mbar_try(bar, parity)) return true;
     if (ctl[kAbort]) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > budget) {
       raise_timeout(ctl, status);
       return false;
     }
@@ -240,6 +242,7 @@ __device__ __forceinline__ float2 chunk_dot_q8(const uint4& w, const float* vec,
   return acc;
 }
 
+#ifdef SFFN_TRACE
 __device__ __forceinline__ long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -254,6 +257,10 @@ __device__ __forceinline__ long long global_ns() {
   do {                                                                            \
     if (p.trace) p.trace[(size_t)blockIdx.x * 16 + (slot)] = clock64() - t_entry; \
   } while (0)
+#else
+#define SFFN_GSTAMP(slot) do { } while (0)
+#define SFFN_STAMP(slot) do { } while (0)
+#endif
 
 template <typename T, int CPT, bool LOPA>
 __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParams p) {
@@ -267,7 +274,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   static_assert(kGW >= 2, "gate warps");
 
   extern __shared__ __align__(128) unsigned char smem[];
+#ifdef SFFN_TRACE
   const long long t_entry = clock64();
+#endif
   pdl_launch_dependents();
   if (threadIdx.x == 0) SFFN_GSTAMP(10);
   constexpr int EPV = Elem<T>::kPerVec;
@@ -349,7 +358,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       const uint32_t ring = smem_u32(gate_ring);
       for (int s = warp; s < n_gslots; s += kGateProducers) {
         const int slot = s % NG;
-        if (!mbar_wait(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status)) break;
+        if (!mbar_wait(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status, p.wait_cycles)) break;
         const int j0 = slot_first_neuron(s);
         const uint32_t bytes = (uint32_t)(min(nr, p.H - j0) * gate_row_bytes);
         mbar_expect_tx(full_gate + 8 * slot, bytes);
@@ -453,7 +462,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         unsigned long long seen;
         asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.v_counter) : "memory");
         if (seen >= v_target || ctl[kAbort]) break;
-        if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); break; }
+        if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status); break; }
         __nanosleep(40);
       }
     }
@@ -497,7 +506,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         if (t_idle == 0) t_idle = clock64();
         __nanosleep(20);
         if (ctl[kAbort]) ok = false;
-        else if (clock64() - t_idle > kWaitCycles) { if (lane == 0) raise_timeout(ctl, p.status); ok = false; }
+        else if (clock64() - t_idle > p.wait_cycles) { if (lane == 0) raise_timeout(ctl, p.status); ok = false; }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         continue;
       }
@@ -509,7 +518,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         fired &= fired - 1;
         const uint32_t sl = __shfl_sync(0xffffffffu, st, l);
         if (lane == 0) {
-          if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) {
+          if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles)) {
             if (ap == 0) slot_a[slot] = sl == 0x80000000u ? 0.f : __uint_as_float(sl);
             const int lrow = base + l;
             if (kScaled && ap == 0) {
@@ -529,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
       base += prefix;
     }
-    if (lane == 0 && ok && mbar_wait(empty_act + 8 * slot, par, ctl, p.status)) {
+    if (lane == 0 && ok && mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles)) {
       if (ap == 0) slot_a[slot] = -1.f;      // stop marker: a negative gate value
       mbar_arrive(full_act + 8 * slot);      // completes the phase without data
     }
@@ -556,7 +565,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
           if (gi >= 0) add += row_sg[r0 + lane] * sx[vec_pos<EPV>(gi, D)];
         }
       }
-      if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status)) break;
+      if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status, p.wait_cycles)) break;
       const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
       float mine = 0.f;
       // Short gate rows (LoPA: r elements): a row is a few chunks per lane, and with one warp per scheduler the cost is
@@ -677,13 +686,13 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       float* rp = red + (round & 1) * (2 * kAW + 1);
       const int slot1 = slot + 1 == NA ? 0 : slot + 1;
       const uint32_t par1 = slot + 1 == NA ? par ^ 1 : par;
-      const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status);
+      const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status, p.wait_cycles);
       const float a0 = got0 ? slot_a[slot] : -1.f;
       bool got1 = true;
       float a1 = -1.f;
       const bool pair = NA >= 4;  // with fewer slots, holding two at a time would stall the act producers
       if (pair && a0 >= 0.f) {
-        got1 = mbar_wait(full_act + 8 * slot1, par1, ctl, p.status);
+        got1 = mbar_wait(full_act + 8 * slot1, par1, ctl, p.status, p.wait_cycles);
         a1 = got1 ? slot_a[slot1] : -1.f;
       }
       const unsigned char* s0 = act_ring + (size_t)slot * p.act_slot_bytes;
@@ -807,14 +816,19 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   constexpr int kTail = 32 * (kGW + kAW);
   const int tw = warp - kFirstGateWarp;
   const int Q = D / 4;
-  const int R = min(G, max(1, Q / 16));  // reducers: 16 columns each where the grid allows
+  // reducers: 16 float4 columns each where the grid allows, but never more than half the grid, so that the waiting
+  // CTAs of two calls that overlap (two handles on two streams) cannot hold every SM between them
+  const int R = min(max(1, (G - 1) / 2), max(1, Q / 16));
   named_bar_sync(6, kTail);
   if (tid == 32 * kFirstGateWarp) {
     SFFN_GSTAMP(6);
     // Release at device scope after the CTA barrier: the act threads' partial stores happen before it, so a CTA that
     // acquires the counter's final value sees every partial.
     unsigned long long old;
-    asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(p.done_counter) : "memory");
+    if (cta == p.skip_arrival_cta)  // test hook: the count never completes and the summing CTAs give up
+      asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(old) : "l"(p.done_counter) : "memory");
+    else
+      asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(p.done_counter) : "memory");
     const unsigned long long first = old / G * G;
     const int rank = (int)(old - first);
     ctl[kRank] = rank;
@@ -825,7 +839,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         unsigned long long seen;
         asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.done_counter) : "memory");
         if (seen >= first + G || ctl[kAbort]) break;
-        if (clock64() - t0 > kWaitCycles) { raise_timeout(ctl, p.status); break; }
+        if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status); break; }
         __nanosleep(20);
       }
       SFFN_GSTAMP(8);
@@ -873,8 +887,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
 }
 
 // ---- host side --------------------------------------------------------------------------------
-long long* g_debug_trace = nullptr;
-
 struct Geometry {
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max, smem, cpt;
   int gate_warps;
@@ -975,8 +987,10 @@ cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaS
 
 }  // namespace
 
-void debug_set_pdl(int on) { pdl_enabled() = on != 0; }
-void debug_set_trace(long long* device_buffer) { g_debug_trace = device_buffer; }
+FusedTestKnobs& fused_test_knobs() {
+  static FusedTestKnobs k;
+  return k;
+}
 
 size_t fused_workspace_bytes(int D, int H, int r_max) {
   (void)H;
@@ -994,12 +1008,16 @@ void debug_fused_plan(int wkind, int D, int H, int K, bool lopa, int sm_count, i
 
 bool fused_supported(int wkind, int D, int H, int B, const sffn_gate* gate, int sm_count) {
   if (B != 1) return false;
+  if (fused_test_knobs().tensor_gate && fused_tc_supported(wkind, D, H, B, gate, sm_count)) return true;
   const bool lopa = gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? gate->r : D;
   return plan(wkind, D, H, K, lopa, fused_grid(sm_count, H)).ok;
 }
 
 cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
+  pdl_enabled() = fused_test_knobs().pdl;
+  if (fused_test_knobs().tensor_gate && fused_tc_supported(c.wkind, c.D, c.H, 1, c.gate, c.sm_count))
+    return launch_fused_tc(c, s, launched);
   const bool lopa = c.gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? c.gate->r : c.D;
   const int grid = fused_grid(c.sm_count, c.H);
@@ -1030,7 +1048,9 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;
   p.gate_warps = g.gate_warps;
-  p.trace = g_debug_trace;
+  p.wait_cycles = fused_test_knobs().wait_cycles;
+  p.skip_arrival_cta = fused_test_knobs().skip_arrival_cta;
+  p.trace = fused_test_knobs().trace;
   if (c.wkind == kWQ8)
     e = lopa ? launch_main<int8_t, true>(p, g, grid, s) : launch_main<int8_t, false>(p, g, grid, s);
   else if (c.wkind == kWBF16)

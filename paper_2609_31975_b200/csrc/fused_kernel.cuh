@@ -33,9 +33,23 @@ struct FusedCall {
 
 size_t fused_workspace_bytes(int D, int H, int r_max);
 bool fused_supported(int wkind, int D, int H, int B, const sffn_gate* gate, int sm_count);
-void debug_set_pdl(int on);
-void debug_set_trace(long long* device_buffer);
 void debug_fused_plan(int wkind, int D, int H, int K, bool lopa, int sm_count, int* out);
 cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched);
+
+// The same call with the gate on the tensor cores (fused_tc_kernel.cu): bf16 rows, standard gate, D a multiple of
+// 64 and at least 1024.  launch_fused takes this route by itself when it applies.
+bool fused_tc_supported(int wkind, int D, int H, int B, const sffn_gate* gate, int sm_count);
+cudaError_t launch_fused_tc(const FusedCall& c, cudaStream_t s, int* launched);
+
+// Test hooks (see the "test hooks" section of sparse_ffn.h).
+struct FusedTestKnobs {
+  bool pdl = true;               // programmatic dependent launch between calls
+  bool tensor_gate = true;       // take the tensor-core gate where it applies
+  long long wait_cycles = 1LL << 31;  // budget of every device-side wait (about one second)
+  int skip_arrival_cta = -1;     // this CTA does not count itself as finished: the summing CTAs' wait runs out
+  int ring_S = 0, ring_NA = 0;   // tensor-core gate: ring split override (0 = planned)
+  long long* trace = nullptr;    // SFFN_TRACE builds: [grid][16] time stamps
+};
+FusedTestKnobs& fused_test_knobs();
 
 }  // namespace sffn

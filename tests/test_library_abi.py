@@ -65,7 +65,7 @@ def test_kernel_geometry_invariants_on_the_host():
         for D in (256, 512, 1024, 2048, 3840, 4096, 5120, 8192, 16384):
             for H in (64, 777, 1024, 10240, 14336, 28672, 53248):
                 for lopa, K in ((0, D), (1, 64), (1, 256), (1, 480), (1, 1024)):
-                    lib.sffn_debug_fused_plan(bf16, D, H, K, lopa, 148, out)
+                    lib.sffn_test_fused_plan(bf16, D, H, K, lopa, 148, out)
                     ok, nr, gsb, ng, gw, asb, na, cpt, smem = list(out)
                     if not ok:
                         continue
@@ -78,17 +78,17 @@ def test_kernel_geometry_invariants_on_the_host():
                     act_threads = 256 if lopa else 128
                     assert cpt in (1, 2, 4, 8) and cpt * act_threads * (16 // esz) >= D
     assert n_ok > 300                                          # the benchmark shapes and most others are served
-    lib.sffn_debug_fused_plan(1, 4096, 14336, 4096, 0, 148, out)
+    lib.sffn_test_fused_plan(1, 4096, 14336, 4096, 0, 148, out)
     assert list(out)[0] == 1 and list(out)[3] == 16            # the graded shape: 16 gate slots of one 8 KB row
     tr, nt, own = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
     for R in (8, 64, 100, 777, 1184, 1200, 14336, 18944, 18945, 28672, 53248, 200000):
-        lib.sffn_debug_umma_tiling(R, 148, ctypes.byref(tr), ctypes.byref(nt), ctypes.byref(own))
+        lib.sffn_test_umma_tiling(R, 148, ctypes.byref(tr), ctypes.byref(nt), ctypes.byref(own))
         assert tr.value % 8 == 0 and 8 <= tr.value <= 128
         assert (nt.value - 1) * tr.value < R <= nt.value * tr.value          # the tiles cover the rows exactly
         assert nt.value <= 148 or tr.value == 128                             # one tile per SM until tiles are full
         if own.value:
             assert 4 * nt.value <= 4 * 384                                    # mask words fit the in-kernel scan
-    lib.sffn_debug_umma_tiling(14336, 148, ctypes.byref(tr), ctypes.byref(nt), ctypes.byref(own))
+    lib.sffn_test_umma_tiling(14336, 148, ctypes.byref(tr), ctypes.byref(nt), ctypes.byref(own))
     assert (tr.value, nt.value, own.value) == (104, 138, 1)
 
 
