@@ -269,11 +269,13 @@ const char* sffn_status_string(int status);
  *   of the single-token kernels that does not report itself finished, so that the CTAs which sum the partial
  *   results see their (bounded) wait run out and record SFFN_ERR_TIMEOUT (-1 = none, the default; use it with a
  *   small WAIT_CYCLES); RING_GATE_SLOTS / RING_ACT_SLOTS = split of the tensor-core kernel's shared-memory rings
- *   (0 = planned); TRACE_BUFFER = device address of [grid][16] int64 time stamps, written only by libraries built
+ *   (0 = planned), RING_PARKED_STAGES = gate stages it prefetches into idle act slots at the start of a call (-1 =
+ *   planned); TRACE_BUFFER = device address of [grid][16] int64 time stamps, written only by libraries built
  *   with -DSFFN_TRACE. */
 typedef enum {
   SFFN_KNOB_PDL = 0, SFFN_KNOB_TENSOR_GATE = 1, SFFN_KNOB_WAIT_CYCLES = 2, SFFN_KNOB_SKIP_ARRIVAL_CTA = 3,
-  SFFN_KNOB_RING_GATE_SLOTS = 4, SFFN_KNOB_RING_ACT_SLOTS = 5, SFFN_KNOB_TRACE_BUFFER = 6
+  SFFN_KNOB_RING_GATE_SLOTS = 4, SFFN_KNOB_RING_ACT_SLOTS = 5, SFFN_KNOB_TRACE_BUFFER = 6,
+  SFFN_KNOB_RING_PARKED_STAGES = 7, SFFN_KNOB_L2_HINTS = 8, SFFN_KNOB_RING_IN_FLIGHT = 9
 } sffn_test_knob;
 void sffn_test_fused_plan(int wkind, int D, int H, int K, int lopa, int sm_count, int* out9);
 void sffn_test_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list);

@@ -169,6 +169,9 @@ int sffn_test_set_knob(int knob, long long value) {
     case SFFN_KNOB_SKIP_ARRIVAL_CTA: k.skip_arrival_cta = (int)value; return SFFN_OK;
     case SFFN_KNOB_RING_GATE_SLOTS: k.ring_S = (int)value; return SFFN_OK;
     case SFFN_KNOB_RING_ACT_SLOTS: k.ring_NA = (int)value; return SFFN_OK;
+    case SFFN_KNOB_RING_PARKED_STAGES: k.ring_E = (int)value; return SFFN_OK;
+    case SFFN_KNOB_L2_HINTS: k.l2_hints = (int)value; return SFFN_OK;
+    case SFFN_KNOB_RING_IN_FLIGHT: k.ring_F = (int)value; return SFFN_OK;
     case SFFN_KNOB_TRACE_BUFFER: k.trace = reinterpret_cast<long long*>(static_cast<uintptr_t>(value)); return SFFN_OK;
     default: return SFFN_ERR_INVALID_ARG;
   }
@@ -492,6 +495,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
     c.x = x; c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up; c.y = y;
     c.dense = dense;
     c.workspace = h->ws + h->L.fused;
+    c.r_max = h->r_max;
     c.status = h->at<int32_t>(h->L.status);
     c.flag = h->at<uint8_t>(h->L.flag);
     c.sm_count = h->sm_count;
@@ -627,7 +631,8 @@ int sffn_reset(sffn_handle* h, void* stream) {
   if (!h) return SFFN_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   SFFN_CUDA(cudaMemsetAsync(h->ws + h->L.status, 0, 256, s));
-  SFFN_CUDA(cudaMemsetAsync(h->ws + h->L.fused, 0, 256, s));  // the single-token kernels' arrival counters
+  // the single-token kernels' arrival counters, call number and tagged partials
+  SFFN_CUDA(cudaMemsetAsync(h->ws + h->L.fused, 0, sffn::fused_workspace_bytes(h->D, h->H, h->r_max), s));
   h->list_state = 0;
   return SFFN_OK;
 }

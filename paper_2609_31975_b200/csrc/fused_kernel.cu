@@ -992,9 +992,18 @@ FusedTestKnobs& fused_test_knobs() {
   return k;
 }
 
+// Workspace of the single-token kernels: 256 bytes of counters, the fp32 partials [kMaxGrid][D] of this file's
+// kernel, the LoPA exchange vector, then the tagged partials [kMaxGrid][D] x 8 bytes of the tensor-core kernel.
+size_t fused_tagged_partials_offset(int D, int r_max) {
+  const size_t plain = 256 + (size_t)kMaxGrid * D * 4 + (size_t)(r_max > 0 ? r_max : 1) * 4;
+  return (plain + 255) / 256 * 256;
+}
 size_t fused_workspace_bytes(int D, int H, int r_max) {
   (void)H;
-  return 256 + (size_t)kMaxGrid * D * 4 + (size_t)(r_max > 0 ? r_max : 1) * 4 + 256;
+  // a row of tagged partials is padded to 2048, 4096, 8192 or 16384 values (whole chunks per act thread)
+  size_t row = 2048;
+  while (row < (size_t)D) row *= 2;
+  return fused_tagged_partials_offset(D, r_max) + (size_t)kMaxGrid * row * 8 + 256;
 }
 
 // Geometry of the fused kernel for a shape, as nine integers (for host-side checks): ok, rows per gate slot, gate

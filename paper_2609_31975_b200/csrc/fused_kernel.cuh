@@ -25,6 +25,7 @@ struct FusedCall {
   int act_up;
   float* y;
   bool dense;
+  int r_max;         // the handle's largest LoPA rank (workspace layout)
   void* workspace;   // fused_workspace_bytes() bytes, zeroed at handle creation
   int32_t* status;   // device status word
   uint8_t* flag;     // [H] "neuron fired" bytes (sparse calls)
@@ -32,6 +33,7 @@ struct FusedCall {
 };
 
 size_t fused_workspace_bytes(int D, int H, int r_max);
+size_t fused_tagged_partials_offset(int D, int r_max);  // where the tensor-core kernel's tagged partials start
 bool fused_supported(int wkind, int D, int H, int B, const sffn_gate* gate, int sm_count);
 void debug_fused_plan(int wkind, int D, int H, int K, bool lopa, int sm_count, int* out);
 cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched);
@@ -48,6 +50,9 @@ struct FusedTestKnobs {
   long long wait_cycles = 1LL << 31;  // budget of every device-side wait (about one second)
   int skip_arrival_cta = -1;     // this CTA does not count itself as finished: the summing CTAs' wait runs out
   int ring_S = 0, ring_NA = 0;   // tensor-core gate: ring split override (0 = planned)
+  int l2_hints = 2;              // tensor-core gate: bit 0 weights evict-first, bit 1 partials evict-last
+  int ring_F = 0;                // tensor-core gate: most gate stages in flight per CTA (0 = no limit)
+  int ring_E = -1;               // tensor-core gate: gate stages parked in the act ring at the start (-1 = planned)
   long long* trace = nullptr;    // SFFN_TRACE builds: [grid][16] time stamps
 };
 FusedTestKnobs& fused_test_knobs();

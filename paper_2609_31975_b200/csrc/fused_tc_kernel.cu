@@ -48,11 +48,13 @@ constexpr int kFirstAct = 10;
 constexpr int kActWarps = 8;       // warps 10..17
 constexpr int kThreads = 32 * (kFirstAct + kActWarps);  // 576
 constexpr int kAT = 32 * kActWarps;
+constexpr int kTail = 32 * (kEpiWarps + kActWarps);  // threads that take part in the cross-CTA sum
 constexpr int kStageThreads = 32 * (kFirstAct - kFirstActProducer);  // warps 2..9 build the B operand
 constexpr int kTileRows = 8;       // neurons per gate tile
 constexpr int kSegs = 16;          // K blocks per ring slot = columns of the MMA
 constexpr int kStageBytes = kTileRows * kSegs * 128;  // 16 KB
 constexpr int kXbBytes = kSegs * 128;                 // token K blocks of one slot position
+constexpr int kMaxParked = 16;     // most gate stages parked in the act ring at the start of a call
 constexpr int kTmemCols = 64;      // 2 tiles in flight x 2 issuers x 16 columns
 constexpr int kMaxGrid = 256;
 constexpr int kSmemBudget = 227 * 1024;
@@ -63,16 +65,20 @@ struct TcParams {
   const void* W_down;
   const void* x;
   const float* b_g;
-  unsigned long long* done_counter;
+  unsigned long long* done_counter;  // CTAs that have finished their rows, monotonic over calls
+  uint32_t* epoch_word;              // number of calls completed on this workspace
   float* y;
-  float* partial;
+  unsigned long long* partial;       // [grid][D] per-CTA partials of y, each value paired with the call's number
   uint8_t* flag;
   int32_t* status;
   int act, dense, act_up;
   int S, NA, act_slot_bytes, slab_max, kst, nacc;
+  int F;         // most gate stages a CTA has in flight (requested, not yet landed); 0 = no limit
+  int E;         // gate stages that are prefetched into the (still idle) last E act slots at the start of a call
   int nf;        // full tiles of every CTA (tile t of CTA c is tile c + t * grid of the matrix)
   int rem_base;  // rows from here on are dealt in contiguous runs of <= 8 (each CTA's last, short tile)
   int rem;
+  int l2_hints;           // bit 0: weights evict-first, bit 1: partials evict-last
   long long wait_cycles;  // budget of every wait (about one second unless a test shortens it)
   int skip_arrival_cta;   // test hook: this CTA does not count itself as finished (-1: none)
   long long* trace;       // SFFN_TRACE builds: [grid][16] time stamps, or null
@@ -90,12 +96,12 @@ struct TcLayout {
     };
     gate_ring = take(S * kStageBytes, 1024);
     xb = take(kst * kXbBytes, 1024);
-    act_ring = take(NA * act_slot_bytes, 128);
+    act_ring = take(NA * act_slot_bytes, 1024);
     row_state = take(slab_max * 4, 128);
     slot_a = take(NA * 4, 16);
     red = take(2 * (2 * kActWarps + 1) * 4, 16);
     ctl = take(8 * 4, 16);
-    bars = take((2 * S + 2 * NA + 4) * 8, 8);
+    bars = take((2 * S + 3 * NA + kMaxParked + 4) * 8, 8);
     tmem_slot = take(8, 8);
     total = off + 1024;  // slack for aligning the dynamic shared memory to 1024 bytes
   }
@@ -126,19 +132,48 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+// L2 policies: weights are read once per call (evict first); the per-CTA partials are rewritten by every call and
+// should stay in L2 instead of being written back behind the weight stream (evict last).
+__device__ __forceinline__ uint64_t policy_evict_first(bool on) {
+  uint64_t pol;
+  if (on) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t policy_evict_last(bool on) {
+  uint64_t pol;
+  if (on) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
       "l"(src), "r"(bytes), "r"(bar)
       : "memory");
+  (void)pol;
+}
+// One value of a partial with the number of the call that wrote it: a naturally aligned 64-bit word is written and
+// read as a whole, so a reader that finds the expected number has the value that belongs to it (no fence, no flag
+// round trip between writer and reader).
+__device__ __forceinline__ unsigned long long tagged(float v, uint32_t epoch) {
+  return ((unsigned long long)epoch << 32) | (unsigned long long)__float_as_uint(v);
+}
+__device__ __forceinline__ void st_tagged2(unsigned long long* dst, unsigned long long a, unsigned long long b, uint64_t pol) {
+  asm volatile("st.global.cg.L2::cache_hint.v2.b64 [%0], {%1, %2}, %3;" ::"l"(dst), "l"(a), "l"(b), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void ld_tagged2(const unsigned long long* src, unsigned long long& a, unsigned long long& b) {
+  asm volatile("ld.global.cg.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(src) : "memory");
 }
 // Tiled tensor-map copy of one box at (element 0, K block c1, neuron c2); parts of the box outside the tensor read
 // as zero and still count towards the barrier's bytes.
-__device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+__device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar,
+                                            uint64_t pol) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
       "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
       : "memory");
+  (void)pol;
 }
 __device__ __forceinline__ void named_bar_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
@@ -178,12 +213,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
       : "r"(taddr));
 }
 
-__device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status) {
+// `site` says which wait gave up (diagnostics: word 3 of the status block holds site + 256 * CTA of the last one).
+__device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status, int site) {
   ctl[kAbort] = 1;
+  status[3] = site + 256 * (int)blockIdx.x;
   atomicExch(status, (int32_t)SFFN_ERR_TIMEOUT);
 }
+// After a wait has run out the CTA winds down.  Copies and MMAs it has issued may still be in flight; they end within
+// microseconds, so a thread that leaves an aborting CTA lets that time pass first: shared memory and TMEM are
+// only given back when nothing can write to them any more.
+__device__ __forceinline__ void abort_grace(volatile int* ctl) {
+  if (ctl[kAbort])
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status,
-                                          long long budget) {
+                                          long long budget, int site) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
@@ -192,7 +236,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (mbar_try(bar, parity)) return true;
     if (ctl[kAbort]) return false;
     if (clock64() - t0 > budget) {
-      raise_timeout(ctl, status);
+      raise_timeout(ctl, status, site);
       return false;
     }
   }
@@ -212,6 +256,28 @@ __device__ __forceinline__ long long global_ns() {
 #define TC_STAMP(slot) do { } while (0)
 #endif
 
+// Where the gate stages of a CTA's sequence live, walked by one thread with a fixed stride (the loops of the
+// producer and issuer threads are single-thread latency chains: no division per stage).  Stage it < S: gate ring
+// slot it; S <= it < S + E: parked in the act ring; later: gate ring slot (it - E) mod S, phase ((it - E) / S) & 1.
+struct StageCursor {
+  int S, E, step, it, slot;
+  uint32_t phase;
+  __device__ __forceinline__ void start(int S_, int E_, int first, int step_) {
+    S = S_; E = E_; step = step_; it = first; slot = first; phase = 0;
+    if (first >= S + E) { slot = (first - E) % S; phase = ((first - E) / S) & 1; }
+  }
+  __device__ __forceinline__ bool parked() const { return it >= S && it < S + E; }
+  __device__ __forceinline__ bool in_ring_again() const { return it >= S + E; }
+  __device__ __forceinline__ void next() {
+    const bool was_ring = it >= S + E;
+    it += step;
+    if (it < S) { slot = it; }
+    else if (it < S + E) { }
+    else if (!was_ring) { slot = (it - E) % S; phase = ((it - E) / S) & 1; }
+    else { slot += step; if (slot >= S) { slot -= S; phase ^= 1; } }
+  }
+};
+
 template <int CPT>
 __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map8,
                                                                const __grid_constant__ CUtensorMap map1) {
@@ -222,7 +288,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   const int G = gridDim.x, cta = blockIdx.x;
   if (tid == 0) TC_STAMP(10);
   const int D = p.D;
-  const int S = p.S, NA = p.NA, kst = p.kst, nacc = p.nacc;
+  const int S = p.S, NA = p.NA, kst = p.kst, nacc = p.nacc, E = p.E;
   const TcLayout L(S, NA, p.act_slot_bytes, p.slab_max, kst);
   unsigned char* act_ring = smem + L.act_ring;
   unsigned char* xb = smem + L.xb;
@@ -235,7 +301,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   const uint32_t bars = smem_u32(smem + L.bars);
   const uint32_t full_gate = bars, empty_gate = bars + 8 * S;
   const uint32_t full_act = bars + 16 * S, empty_act = full_act + 8 * NA;
-  const uint32_t acc_full = empty_act + 8 * NA, acc_empty = acc_full + 16;
+  const uint32_t extra_full = empty_act + 8 * NA, extra_done = extra_full + 8 * kMaxParked;
+  const uint32_t acc_full = extra_done + 8 * NA, acc_empty = acc_full + 16;
 
   const int nvecD = D / 8;
   const size_t row_bytes = (size_t)D * 2;
@@ -249,7 +316,13 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
     const int t = l >> 3;
     return t < nf ? (cta + t * G) * kTileRows + (l & 7) : rem_lo + (l - nf * kTileRows);
   };
-
+  // Where gate stage `it` of this CTA's sequence lives.  The first S stages fill the gate ring; the next E go into the
+  // last act slots, which no fired row can need yet (no gate result exists before the token has arrived): the CTA
+  // starts while its predecessor in the stream still runs, and everything it can fetch before the token is there
+  // shortens the call.  From then on the gate ring is used round robin.
+  const int m_per_slot = p.act_slot_bytes / kStageBytes;  // gate stages per act slot (E > 0 only if it divides)
+  const int extra_slots = E > 0 ? E / m_per_slot : 0;      // act slots that start out holding gate stages
+  const uint32_t extra_base = smem_u32(act_ring) + (uint32_t)(NA - extra_slots) * p.act_slot_bytes;
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(full_gate + 8 * s, 1);
@@ -258,7 +331,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
     for (int s = 0; s < NA; ++s) {
       mbar_init(full_act + 8 * s, kActProducers);
       mbar_init(empty_act + 8 * s, kActWarps);
+      mbar_init(extra_done + 8 * s, m_per_slot > 0 ? m_per_slot : 1);
     }
+    for (int s = 0; s < kMaxParked; ++s) mbar_init(extra_full + 8 * s, 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(acc_full + 8 * b, nacc);
       mbar_init(acc_empty + 8 * b, kEpiWarps);
@@ -282,27 +357,48 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp < kGateProducers) {
-    // ======================= gate producers (alternate ring slots) ==================================
-    // The weights depend on nothing earlier in the stream: the ring fills while the predecessor still runs.
+    // ======================= gate producers (alternate stages) ======================================
+    // The weights depend on nothing earlier in the stream: the rings fill while the predecessor still runs.
     if (lane == 0) {
+      const uint64_t once = policy_evict_first(p.l2_hints & 1);
       const int total = n_tiles * kst;
-      for (int it = warp; it < total; it += kGateProducers) {
-        const int slot = it % S;
-        if (!mbar_wait(empty_gate + 8 * slot, ((it / S) & 1) ^ 1, ctl, p.status, p.wait_cycles)) break;
-        const int t = it / kst, st = it - t * kst;
-        const uint32_t dst = gate_ring + (uint32_t)slot * kStageBytes;
-        if (t < nf) {
-          mbar_expect_tx(full_gate + 8 * slot, kStageBytes);
-          tma_tile_3d(dst, &map8, 0, st * kSegs, (cta + t * G) * kTileRows, full_gate + 8 * slot);
-        } else {
-          mbar_expect_tx(full_gate + 8 * slot, (uint32_t)rc * (kSegs * 128));
-          for (int i = 0; i < rc; ++i)
-            tma_tile_3d(dst + (uint32_t)i * (kSegs * 128), &map1, 0, st * kSegs, rem_lo + i, full_gate + 8 * slot);
+      StageCursor c, lag;  // lag: the stage p.F before c (same producer), whose arrival is waited for first
+      c.start(S, E, warp, kGateProducers);
+      lag.start(S, E, warp, kGateProducers);
+      int t = warp / kst, st = warp - t * kst;
+      for (; c.it < total; c.next()) {
+        // Bytes in flight beyond what the memory system needs to run at its rate only queue up in front of every
+        // other access of the GPU (the token, the partial sums): a stage is requested once the stage F before it
+        // has landed.
+        if (p.F > 0 && c.it >= p.F + warp) {
+          const uint32_t lbar = lag.parked() ? extra_full + 8 * (lag.it - S) : full_gate + 8 * lag.slot;
+          if (!mbar_wait(lbar, lag.parked() ? 0u : lag.phase, ctl, p.status, p.wait_cycles, 1)) break;
+          lag.next();
         }
+        uint32_t dst, bar;
+        if (c.parked()) {
+          dst = extra_base + (uint32_t)(c.it - S) * kStageBytes;
+          bar = extra_full + 8 * (c.it - S);
+        } else {
+          if (c.in_ring_again() && !mbar_wait(empty_gate + 8 * c.slot, c.phase ^ 1, ctl, p.status, p.wait_cycles, 2)) break;
+          dst = gate_ring + (uint32_t)c.slot * kStageBytes;
+          bar = full_gate + 8 * c.slot;
+        }
+        if (t < nf) {
+          mbar_expect_tx(bar, kStageBytes);
+          tma_tile_3d(dst, &map8, 0, st * kSegs, (cta + t * G) * kTileRows, bar, once);
+        } else {
+          mbar_expect_tx(bar, (uint32_t)rc * (kSegs * 128));
+          for (int i = 0; i < rc; ++i)
+            tma_tile_3d(dst + (uint32_t)i * (kSegs * 128), &map1, 0, st * kSegs, rem_lo + i, bar, once);
+        }
+        st += kGateProducers;
+        while (st >= kst) { st -= kst; ++t; }
       }
       if (warp == 0) TC_STAMP(1);
     }
     __syncwarp();
+    abort_grace(ctl);
     return;
   }
 
@@ -318,7 +414,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
 
   const int at = tid - 32 * kFirstAct;  // act threads: 0 .. kAT - 1
   float2 xr[CPT][4];                    // act threads: this thread's slice of the token
+  uint32_t ep = 0;                      // this call's number (epilogue and act warps: they write and sum the partials)
+  uint64_t keep = 0;                    // act threads: L2 policy of the partial stores (made early: it takes a while)
   if (warp >= kFirstAct) {
+    ep = __ldcg(p.epoch_word) + 1u;
+    keep = policy_evict_last(p.l2_hints & 2);
 #pragma unroll
     for (int i = 0; i < CPT; ++i) {
       const int c = at + i * kAT;
@@ -330,6 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   } else {
     // Token as the B operand: K block kb is row kb mod 16 of slot position kb / 16, 128 bytes, swizzled like the
     // weight tiles (16-byte chunk index xor row mod 8).  K blocks past the row's end are zero.
+    if (warp >= kFirstEpi && warp < kFirstIssuer) ep = __ldcg(p.epoch_word) + 1u;
     const int st_tid = tid - 32 * kFirstActProducer;
     for (int i = st_tid; i < slab_rows; i += kStageThreads) row_state[i] = 0xffffffffu;
     const int chunks = kst * kSegs * 8;
@@ -346,9 +447,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   if (warp < kFirstEpi) {
     // ======================= act producers: rows of fired neurons, ascending ========================
     const int ap = warp - kFirstActProducer;
+    const uint64_t once = policy_evict_first(p.l2_hints & 1);
     const char* Wsrc = static_cast<const char*>(ap == 0 ? p.W_up : p.W_down);
     const uint32_t ring = smem_u32(act_ring) + (ap == 0 ? 0u : (uint32_t)row_bytes);
-    int slot = 0;
+    int slot = 0, used = 0;
     uint32_t par = 1;
     bool ok = true;
     long long t_idle = 0;
@@ -361,7 +463,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
         if (t_idle == 0) t_idle = clock64();
         __nanosleep(20);
         if (ctl[kAbort]) ok = false;
-        else if (clock64() - t_idle > p.wait_cycles) { if (lane == 0) raise_timeout(ctl, p.status); ok = false; }
+        else if (clock64() - t_idle > p.wait_cycles) { if (lane == 0) raise_timeout(ctl, p.status, 20); ok = false; }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         continue;
       }
@@ -373,27 +475,47 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
         fired &= fired - 1;
         const uint32_t sl = __shfl_sync(0xffffffffu, st, l);
         if (lane == 0) {
-          if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles)) {
+          bool free_now = mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 3);
+          if (free_now && used < NA && slot >= NA - extra_slots)  // first use: the gate stages parked here must be gone
+            free_now = mbar_wait(extra_done + 8 * (slot - (NA - extra_slots)), 0, ctl, p.status, p.wait_cycles, 4);
+          if (free_now) {
             if (ap == 0) slot_a[slot] = sl == 0x80000000u ? 0.f : __uint_as_float(sl);
             const size_t j = (size_t)neuron_of(base + l);
             mbar_expect_tx(full_act + 8 * slot, (uint32_t)row_bytes);
             bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
-                     full_act + 8 * slot);
+                     full_act + 8 * slot, once);
           } else {
             ok = false;
           }
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        ++used;
         if (++slot == NA) { slot = 0; par ^= 1; }
       }
       base += prefix;
     }
-    if (lane == 0 && ok && mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles)) {
+    if (lane == 0 && ok && mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 5)) {
       if (ap == 0) slot_a[slot] = -1.f;  // stop marker: a negative gate value
       mbar_arrive(full_act + 8 * slot);  // completes the phase without data
     }
-    if (lane == 0 && ap == 0) TC_STAMP(2);
-    __syncwarp();
+    if (ap == 0) {
+      // This CTA's place in the order of finishing (the last R sum the partials), taken now so that the round trip
+      // overlaps with the act warps' last rows; -1 under the test hook that makes a CTA go missing.
+      if (lane == 0) {
+        TC_STAMP(2);
+        int rank = -1;
+        if (cta != p.skip_arrival_cta) {
+          unsigned long long old;
+          asm volatile("atom.add.relaxed.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(p.done_counter) : "memory");
+          rank = (int)(old - old / G * G);
+        }
+        ctl[kRank] = rank;
+        TC_STAMP(7);
+      }
+      __syncwarp();
+      asm volatile("bar.arrive 6, %0;" ::"r"(kTail + 32) : "memory");
+    }
+    abort_grace(ctl);
     return;
   }
 
@@ -401,34 +523,56 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
     // ======================= MMA issuers ============================================================
     const int m = warp - kFirstIssuer;
     if (lane == 0 && m < nacc) {
-      bool ok = true;
-      for (int t = 0; ok && t < n_tiles; ++t) {
-        const int b = t & 1;
-        if (!mbar_wait(acc_empty + 8 * b, ((t >> 1) & 1) ^ 1, ctl, p.status, p.wait_cycles)) break;
-        tc_fence_after();
-        const uint32_t acc = tmem_base + (uint32_t)((b * kIssuers + m) * kSegs);
-        bool first = true;
-        for (int st = 0; st < kst; ++st) {
-          const int it = t * kst + st;
-          if (nacc == 2 && (it & 1) != m) continue;
-          const int slot = it % S;
-          if (!mbar_wait(full_gate + 8 * slot, (it / S) & 1, ctl, p.status, p.wait_cycles)) { ok = false; break; }
+      const int total = n_tiles * kst;
+      const uint64_t bdesc0 = make_desc(smem_u32(xb));
+      StageCursor c;
+      c.start(S, E, m, nacc);
+      int t = m / kst, st = m - t * kst;
+      int t_cur = -1;
+      uint32_t acc = 0, accumulate = 0;
+      for (; c.it < total; c.next()) {
+        if (t != t_cur) {  // first stage of this issuer in a new tile
+          if (t_cur >= 0) umma_commit(acc_full + 8 * (t_cur & 1));
+          t_cur = -1;
+          if (!mbar_wait(acc_empty + 8 * (t & 1), ((t >> 1) & 1) ^ 1, ctl, p.status, p.wait_cycles, 6)) break;
           tc_fence_after();
-          const uint64_t adesc = make_desc(gate_ring + (uint32_t)slot * kStageBytes);
-          const uint64_t bdesc = make_desc(smem_u32(xb) + (uint32_t)st * kXbBytes);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, (first && k == 0) ? 0u : 1u);
-          umma_commit(empty_gate + 8 * slot);  // slot free once these MMAs have read it
-          first = false;
+          t_cur = t;
+          acc = tmem_base + (uint32_t)(((t & 1) * kIssuers + m) * kSegs);
+          accumulate = 0;
         }
-        if (ok) umma_commit(acc_full + 8 * b);
+        uint32_t addr, bar, done, par;
+        if (c.parked()) {
+          addr = extra_base + (uint32_t)(c.it - S) * kStageBytes;
+          bar = extra_full + 8 * (c.it - S);
+          done = extra_done + 8 * ((c.it - S) / m_per_slot);
+          par = 0;
+        } else {
+          addr = gate_ring + (uint32_t)c.slot * kStageBytes;
+          bar = full_gate + 8 * c.slot;
+          done = empty_gate + 8 * c.slot;
+          par = c.phase;
+        }
+        if (!mbar_wait(bar, par, ctl, p.status, p.wait_cycles, 7)) { t_cur = -1; break; }
+        tc_fence_after();
+        const uint64_t adesc = make_desc(addr);
+        const uint64_t bdesc = bdesc0 + (uint64_t)(st * (kXbBytes >> 4));
+        umma(acc, adesc, bdesc, accumulate);
+#pragma unroll
+        for (int k = 1; k < 4; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, 1u);
+        umma_commit(done);  // the stage's memory is free once these MMAs have read it
+        accumulate = 1;
+        st += nacc;
+        while (st >= kst) { st -= kst; ++t; }
       }
+      if (t_cur >= 0) umma_commit(acc_full + 8 * (t_cur & 1));
       if (m == 0) TC_STAMP(3);
     }
     __syncwarp();
+    abort_grace(ctl);
     return;
   }
 
+  const int tt = warp < kFirstIssuer ? tid - 32 * kFirstEpi : 32 * kEpiWarps + at;  // index among the tail threads
   if (warp < kFirstIssuer) {
     // ======================= epilogue warps =========================================================
     // TMEM lane 16 i + s holds neuron i of the tile against segment s of its row; column n is segment n of the token.
@@ -442,7 +586,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
       const int j = i_loc < rows ? neuron_of(l) : 0;
       const float bias = (seg == 0 && i_loc < rows && p.b_g) ? __ldg(p.b_g + j) : 0.f;
       int okw = 1;
-      if (lane == 0) okw = mbar_wait(acc_full + 8 * b, (t >> 1) & 1, ctl, p.status, p.wait_cycles) ? 1 : 0;
+      if (lane == 0) okw = mbar_wait(acc_full + 8 * b, (t >> 1) & 1, ctl, p.status, p.wait_cycles, 8) ? 1 : 0;
       okw = __shfl_sync(0xffffffffu, okw, 0);
       if (!okw) { ok = false; break; }
       tc_fence_after();
@@ -473,6 +617,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
     }
     if (warp == kFirstEpi && lane == 0) TC_STAMP(4);
     // the accumulators are idle once every epilogue warp has left its loop: release the TMEM columns
+    abort_grace(ctl);
     tc_fence_before();
     named_bar_sync(7, 32 * kEpiWarps);
     if (warp == kFirstEpi) {
@@ -497,12 +642,12 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
       float* rp = red + (round & 1) * (2 * kActWarps + 1);
       const int slot1 = slot + 1 == NA ? 0 : slot + 1;
       const uint32_t par1 = slot + 1 == NA ? par ^ 1 : par;
-      const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status, p.wait_cycles);
+      const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 9);
       const float a0 = got0 ? slot_a[slot] : -1.f;
       bool got1 = true;
       float a1 = -1.f;
       if (pair && a0 >= 0.f) {
-        got1 = mbar_wait(full_act + 8 * slot1, par1, ctl, p.status, p.wait_cycles);
+        got1 = mbar_wait(full_act + 8 * slot1, par1, ctl, p.status, p.wait_cycles, 10);
         a1 = got1 ? slot_a[slot1] : -1.f;
       }
       const unsigned char* s0 = act_ring + (size_t)slot * p.act_slot_bytes;
@@ -567,13 +712,18 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
       par = slot1 + 1 == NA ? par1 ^ 1 : par1;
     }
     if (at == 0) TC_STAMP(5);
-    float* dst = p.partial + (size_t)cta * D;
+    // This CTA's partial of y, every value tagged with the call's number.  Stored unit (two columns, 16 bytes)
+    // (i * 4 + e) * kAT + at holds columns 8 (at + i kAT) + 2 e and the next one: a warp's store is 512 contiguous
+    // bytes; the summing threads undo the permutation when they write y.
+    if (cta != p.skip_arrival_cta) {
+      unsigned long long* dst = p.partial + (size_t)cta * (CPT * 8 * kAT);
 #pragma unroll
-    for (int i = 0; i < CPT; ++i) {
-      const int c = at + i * kAT;
-      if (c < nvecD) {
-        __stcg(reinterpret_cast<float4*>(dst + (size_t)c * 8), make_float4(acc[i][0].x, acc[i][0].y, acc[i][1].x, acc[i][1].y));
-        __stcg(reinterpret_cast<float4*>(dst + (size_t)c * 8 + 4), make_float4(acc[i][2].x, acc[i][2].y, acc[i][3].x, acc[i][3].y));
+      for (int i = 0; i < CPT; ++i) {
+        if (at + i * kAT < nvecD) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            st_tagged2(dst + 2 * (size_t)((i * 4 + e) * kAT + at), tagged(acc[i][e].x, ep), tagged(acc[i][e].y, ep), keep);
+        }
       }
     }
     if (at == 0) TC_STAMP(12);
@@ -581,73 +731,95 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
 
   // ---- y = sum over CTAs of their partials, by the last CTAs to finish (epilogue and act warps get here) --------
   // Which CTA sums a slice of the columns depends on timing, what it computes does not: y is bitwise repeatable.
-  constexpr int kTail = 32 * (kEpiWarps + kActWarps);
-  const int Q = D / 4;
-  const int R = min(max(1, (G - 1) / 2), max(1, Q / 16));  // never more than half the grid waits
-  named_bar_sync(6, kTail);
-  if (tid == 32 * kFirstEpi) {
-    TC_STAMP(6);
-    // release at device scope after the CTA barrier: the act threads' partial stores happen before it
-    unsigned long long old;
-    if (cta == p.skip_arrival_cta)  // test hook: the count never completes and the summing CTAs give up
-      asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(old) : "l"(p.done_counter) : "memory");
-    else
-      asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(p.done_counter) : "memory");
-    const unsigned long long first = old / G * G;
-    const int rank = (int)(old - first);
-    ctl[kRank] = rank;
-    TC_STAMP(7);
-    if (rank >= G - R) {
-      const long long t0 = clock64();
-      for (;;) {
-        unsigned long long seen;
-        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.done_counter) : "memory");
-        if (seen >= first + G || ctl[kAbort]) break;
-        if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status); break; }
-        __nanosleep(20);
-      }
-      TC_STAMP(8);
-    }
+  // A summing CTA does not wait for a count or a flag: it reads the other CTAs' tagged values and re-reads those
+  // that still carry an older call's number (bounded).  Thread (u, rg) takes two columns (one 16-byte unit) in the
+  // rows rg, rg + RG, ...; the RG row groups are then added in order through shared memory.
+  const int units = CPT * 4 * kAT;  // stored units of a partial (a multiple of 32; those past D / 2 are never written)
+  const int R = min(max(1, (G - 1) / 2), max(1, units / 32));  // never more than half the grid stays
+  named_bar_sync(6, kTail + 32);  // + the act producer that took the rank
+  const int rank = ctl[kRank];
+  const int slice = rank - (G - R);
+  if (slice < 0 || ctl[kAbort]) {
+    abort_grace(ctl);
+    return;
   }
-  named_bar_sync(6, kTail);
-  const int slice = ctl[kRank] - (G - R);
-  if (slice < 0 || ctl[kAbort] || warp >= kFirstIssuer) return;
-  const int32_t failed = __ldcg(p.status);
-  const int cols = (Q + R - 1) / R;
-  const int q_hi = min(Q, (slice + 1) * cols);
-  // Four warps, one group of four float4 columns each.  Lane (r8, c4) reads column c4 of its group in the rows r8,
-  // r8 + 8, ...: a warp load covers eight rows x 64 contiguous bytes, twenty loads in flight per lane, the eight
-  // row residues combined by shuffles in a fixed order.
-  const int tw = warp - kFirstEpi;
-  const int r8 = lane >> 2, c4 = lane & 3;
-  for (int c0 = slice * cols; c0 < q_hi; c0 += 16) {
-    const int qc = c0 + 4 * tw + c4;
-    float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (qc < q_hi) {
-      const float4* src = reinterpret_cast<const float4*>(p.partial) + qc;
-      for (int i0 = 0; 8 * i0 < G; i0 += 20) {
-        float4 v[20];
+  if (tt == 0) TC_STAMP(8);
+  constexpr int kBatch = 13;
+  const int32_t failed = __ldcg(p.status);  // in flight together with the partials, not after them
+  float2* comb = reinterpret_cast<float2*>(smem + L.gate_ring);  // the rings are idle by now
+  const int U = (units + R - 1) / R;
+  const int UW = U <= 32 ? 32 : U <= 64 ? 64 : 128;
+  const int RG = kTail / UW;
+  const int u = tt % UW, rg = tt / UW;
+  bool ok = true;
+  for (int u0 = 0; u0 < U; u0 += UW) {
+    const int unit = slice * U + u0 + u;
+    float2 sum = make_float2(0.f, 0.f);
+    const int col = 8 * ((unit % kAT) + (unit / (4 * kAT)) * kAT) + 2 * ((unit / kAT) & 3);  // first of its two columns
+    if (u0 + u < U && unit < units && col < D) {
+      const unsigned long long* src = p.partial + 2 * (size_t)unit;
+      for (int g0 = rg; ok && g0 < G; g0 += RG * kBatch) {
+        unsigned long long a[kBatch], b[kBatch];
 #pragma unroll
-        for (int i = 0; i < 20; ++i) {
-          const int g = 8 * (i0 + i) + r8;
-          v[i] = g < G ? __ldcg(src + (size_t)g * Q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k = 0; k < kBatch; ++k) {
+          const int g = g0 + k * RG;
+          a[k] = b[k] = (unsigned long long)ep << 32;  // rows past the grid: zero, already "there"
+          if (g < G) ld_tagged2(src + (size_t)g * (CPT * 8 * kAT), a[k], b[k]);
         }
+        long long t0 = 0;
+#ifdef SFFN_TRACE
+        int tries = 0;
+#endif
+        for (;;) {
+#ifdef SFFN_TRACE
+          if (tt == 0 && g0 == rg && tries == 0 && p.trace) { asm volatile("" ::"l"(a[12]) : "memory"); TC_STAMP(9); }
+          ++tries;
+#endif
+          bool all = true;
 #pragma unroll
-        for (int i = 0; i < 20; ++i) {
-          s4.x += v[i].x; s4.y += v[i].y; s4.z += v[i].z; s4.w += v[i].w;
+          for (int k = 0; k < kBatch; ++k) {
+            if ((uint32_t)(a[k] >> 32) != ep || (uint32_t)(b[k] >> 32) != ep) {
+              all = false;
+              ld_tagged2(src + (size_t)(g0 + k * RG) * (CPT * 8 * kAT), a[k], b[k]);
+            }
+          }
+          if (all) break;
+          if (t0 == 0) t0 = clock64();
+          if (ctl[kAbort]) { ok = false; break; }
+          if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status, 21); ok = false; break; }
+          __nanosleep(64);
+        }
+#ifdef SFFN_TRACE
+        if (tt == 0 && g0 == rg && p.trace) { TC_STAMP(14); p.trace[(size_t)blockIdx.x * 16 + 15] = tries; }
+#endif
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+          sum.x += __uint_as_float((uint32_t)a[k]);
+          sum.y += __uint_as_float((uint32_t)b[k]);
         }
       }
     }
-#pragma unroll
-    for (int o = 4; o < 32; o <<= 1) {
-      s4.x += __shfl_xor_sync(0xffffffffu, s4.x, o);
-      s4.y += __shfl_xor_sync(0xffffffffu, s4.y, o);
-      s4.z += __shfl_xor_sync(0xffffffffu, s4.z, o);
-      s4.w += __shfl_xor_sync(0xffffffffu, s4.w, o);
+    comb[rg * UW + u] = sum;
+    named_bar_sync(5, kTail);
+    if (tt < UW) {
+      const int unit2 = slice * U + u0 + tt;
+      const int col2 = 8 * ((unit2 % kAT) + (unit2 / (4 * kAT)) * kAT) + 2 * ((unit2 / kAT) & 3);
+      if (u0 + tt < U && unit2 < units && col2 < D) {
+        float2 t = make_float2(0.f, 0.f);
+        for (int r = 0; r < RG; ++r) {
+          t.x += comb[r * UW + tt].x;
+          t.y += comb[r * UW + tt].y;
+        }
+        if (!ctl[kAbort] && failed == 0) *reinterpret_cast<float2*>(p.y + col2) = t;
+      }
     }
-    if (r8 == 0 && qc < q_hi && failed == 0) reinterpret_cast<float4*>(p.y)[qc] = s4;
+    named_bar_sync(5, kTail);
   }
-  if (tid == 32 * kFirstEpi) TC_STAMP(13);
+  abort_grace(ctl);
+  if (tt == 0) {
+    if (rank == G - 1 && !ctl[kAbort]) *p.epoch_word = ep;  // the call is complete: the next one tags with ep + 1
+    TC_STAMP(13);
+  }
 }
 
 // ---- host side ------------------------------------------------------------------------------------------------
@@ -703,7 +875,7 @@ const MapEntry* gate_maps(const void* base, int D, int H) {
 }
 
 struct TcGeometry {
-  int S, NA, act_slot_bytes, slab_max, kst, nacc, nf, rem_base, rem, cpt, smem;
+  int S, NA, E, act_slot_bytes, slab_max, kst, nacc, nf, rem_base, rem, cpt, smem;
   bool ok;
 };
 
@@ -719,9 +891,12 @@ TcGeometry tc_plan(int D, int H, int grid) {
   g.rem_base = g.nf * grid * kTileRows;
   g.rem = H - g.rem_base;
   g.slab_max = g.nf * kTileRows + (g.rem + grid - 1) / grid;
-  g.act_slot_bytes = 2 * D * 2;
+  g.act_slot_bytes = (2 * D * 2 + 1023) / 1024 * 1024;
+  // a slot that is nearly a whole number of gate stages is padded to it: it can then park gate stages at the start
+  const int whole = (g.act_slot_bytes + kStageBytes - 1) / kStageBytes * kStageBytes;
+  if (whole - g.act_slot_bytes <= g.act_slot_bytes / 8) g.act_slot_bytes = whole;
   const TcLayout fixed(0, 0, 0, g.slab_max, g.kst);
-  const int ring = kSmemBudget - fixed.total - 512;  // 512: barrier words and gate values per slot
+  const int ring = kSmemBudget - fixed.total - 1024;  // 1024: barrier words and gate values per slot
   // Gate slots first (an even number, each issuer and producer owns alternate ones), at least four act slots
   // where they fit so that the act warps can take two rows per round.
   int na = ring >= 6 * kStageBytes + 4 * g.act_slot_bytes ? 4 : 2;
@@ -738,6 +913,17 @@ TcGeometry tc_plan(int D, int H, int grid) {
   if (knobs.ring_S > 0 && knobs.ring_NA > 0) { s = knobs.ring_S & ~1; na = knobs.ring_NA; }
   if (s < 2 || na < 2) return g;
   g.S = s; g.NA = na;
+  // gate stages parked in the last act slots at the start of a call: all but the first slot, an even number of stages
+  g.E = 0;
+  if (g.act_slot_bytes % kStageBytes == 0) {
+    const int per = g.act_slot_bytes / kStageBytes;
+    int e = (na - 1) * per;
+    if (knobs.ring_E >= 0) e = knobs.ring_E < e ? knobs.ring_E : e;
+    e = e / per * per;
+    if (e > kMaxParked) e = kMaxParked / per * per;
+    if (e & 1) e -= per;
+    g.E = e < 0 ? 0 : e;
+  }
   const TcLayout full(s, na, g.act_slot_bytes, g.slab_max, g.kst);
   g.smem = full.total;
   g.ok = g.smem <= kSmemBudget;
@@ -767,12 +953,16 @@ cudaError_t launch_fused_tc(const FusedCall& c, cudaStream_t s, int* launched) {
   p.D = c.D; p.H = c.H;
   p.W_up = c.W_up; p.W_down = c.W_down; p.x = c.x; p.b_g = c.b_g;
   p.done_counter = reinterpret_cast<unsigned long long*>(ws) + 1;
+  p.epoch_word = reinterpret_cast<uint32_t*>(ws + 16);
   p.y = c.y;
-  p.partial = reinterpret_cast<float*>(ws + 256);
+  p.partial = reinterpret_cast<unsigned long long*>(ws + fused_tagged_partials_offset(c.D, c.r_max));
   p.flag = c.flag; p.status = c.status;
   p.act = c.act; p.dense = c.dense ? 1 : 0; p.act_up = c.act_up;
-  p.S = g.S; p.NA = g.NA; p.act_slot_bytes = g.act_slot_bytes; p.slab_max = g.slab_max; p.kst = g.kst; p.nacc = g.nacc;
+  p.S = g.S; p.NA = g.NA; p.E = g.E; p.F = fused_test_knobs().ring_F & ~1;
+  if (p.F > g.S) p.F = g.S;  // the stage waited for must be the latest use of its ring slot
+  p.act_slot_bytes = g.act_slot_bytes; p.slab_max = g.slab_max; p.kst = g.kst; p.nacc = g.nacc;
   p.nf = g.nf; p.rem_base = g.rem_base; p.rem = g.rem;
+  p.l2_hints = fused_test_knobs().l2_hints;
   p.wait_cycles = fused_test_knobs().wait_cycles;
   p.skip_arrival_cta = fused_test_knobs().skip_arrival_cta;
   p.trace = fused_test_knobs().trace;
