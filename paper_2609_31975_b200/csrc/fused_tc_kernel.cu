@@ -31,6 +31,8 @@
 
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace sffn {
@@ -75,7 +77,9 @@ struct TcParams {
   int S, NA, act_slot_bytes, slab_max, kst, nacc;
   int F;         // most gate stages a CTA has in flight (requested, not yet landed); 0 = no limit
   int E;         // gate stages that are prefetched into the (still idle) last E act slots at the start of a call
-  int nf;        // full tiles of every CTA (tile t of CTA c is tile c + t * grid of the matrix)
+  int R;         // CTAs that stay to sum the partials (the last R to finish)
+  int lead;      // extra tiles of the first grid - R CTAs (see tile_of)
+  int nf;        // full tiles of every CTA beyond those
   int rem_base;  // rows from here on are dealt in contiguous runs of <= 8 (each CTA's last, short tile)
   int rem;
   int l2_hints;           // bit 0: weights evict-first, bit 1: partials evict-last
@@ -307,14 +311,20 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   const int nvecD = D / 8;
   const size_t row_bytes = (size_t)D * 2;
   // This CTA's neurons: nf full tiles dealt round robin over the CTAs, then a contiguous run of the left-over rows.
-  const int nf = p.nf;
+  // Tiles are dealt round robin, with a head start for the CTAs that can use one: in a run of back-to-back calls
+  // the R CTAs that summed the previous call's partials start last (their SMs come free last, and the hardware
+  // hands out CTAs in index order), with nothing prefetched; the other G - R get `lead` more tiles each.
+  const int early = G - p.R;
+  const int lead = cta < early ? p.lead : 0;
+  const int nf = p.nf + lead;
+  auto tile_of = [&](int t) { return t < lead ? cta + t * early : p.lead * early + cta + (t - lead) * G; };
   const int rem_lo = p.rem_base + (int)((long long)p.rem * cta / G);
   const int rc = p.rem_base + (int)((long long)p.rem * (cta + 1) / G) - rem_lo;
   const int n_tiles = nf + (rc > 0 ? 1 : 0);
   const int slab_rows = nf * kTileRows + rc;
   auto neuron_of = [&](int l) {
     const int t = l >> 3;
-    return t < nf ? (cta + t * G) * kTileRows + (l & 7) : rem_lo + (l - nf * kTileRows);
+    return t < nf ? tile_of(t) * kTileRows + (l & 7) : rem_lo + (l - nf * kTileRows);
   };
   // Where gate stage `it` of this CTA's sequence lives.  The first S stages fill the gate ring; the next E go into the
   // last act slots, which no fired row can need yet (no gate result exists before the token has arrived): the CTA
@@ -386,7 +396,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
         }
         if (t < nf) {
           mbar_expect_tx(bar, kStageBytes);
-          tma_tile_3d(dst, &map8, 0, st * kSegs, (cta + t * G) * kTileRows, bar, once);
+          tma_tile_3d(dst, &map8, 0, st * kSegs, tile_of(t) * kTileRows, bar, once);
         } else {
           mbar_expect_tx(bar, (uint32_t)rc * (kSegs * 128));
           for (int i = 0; i < rc; ++i)
@@ -735,10 +745,15 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   // that still carry an older call's number (bounded).  Thread (u, rg) takes two columns (one 16-byte unit) in the
   // rows rg, rg + RG, ...; the RG row groups are then added in order through shared memory.
   const int units = CPT * 4 * kAT;  // stored units of a partial (a multiple of 32; those past D / 2 are never written)
-  const int R = min(max(1, (G - 1) / 2), max(1, units / 32));  // never more than half the grid stays
+  const int R = p.R;
   named_bar_sync(6, kTail + 32);  // + the act producer that took the rank
+  // The first R CTAs to finish do the sum: they have time to spare until the slowest CTA is done, fetch the
+  // partials that are already there meanwhile and only have the late ones left to fetch at the end.  Their SMs come
+  // free last, so the next call starts with nothing prefetched there -- which costs little: the CTAs of a call
+  // share the memory system's rate whatever their head start.
   const int rank = ctl[kRank];
-  const int slice = rank - (G - R);
+  const int slice = rank >= 0 && rank < R ? rank : -1;
+  if (rank == G - 1 && tt == 0 && !ctl[kAbort]) *p.epoch_word = ep;  // every CTA has its number: the next call tags with ep + 1
   if (slice < 0 || ctl[kAbort]) {
     abort_grace(ctl);
     return;
@@ -787,7 +802,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
           if (t0 == 0) t0 = clock64();
           if (ctl[kAbort]) { ok = false; break; }
           if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status, 21); ok = false; break; }
-          __nanosleep(64);
+          __nanosleep(100);
         }
 #ifdef SFFN_TRACE
         if (tt == 0 && g0 == rg && p.trace) { TC_STAMP(14); p.trace[(size_t)blockIdx.x * 16 + 15] = tries; }
@@ -816,10 +831,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
     named_bar_sync(5, kTail);
   }
   abort_grace(ctl);
-  if (tt == 0) {
-    if (rank == G - 1 && !ctl[kAbort]) *p.epoch_word = ep;  // the call is complete: the next one tags with ep + 1
-    TC_STAMP(13);
-  }
+  if (tt == 0) TC_STAMP(13);
 }
 
 // ---- host side ------------------------------------------------------------------------------------------------
@@ -875,7 +887,7 @@ const MapEntry* gate_maps(const void* base, int D, int H) {
 }
 
 struct TcGeometry {
-  int S, NA, E, act_slot_bytes, slab_max, kst, nacc, nf, rem_base, rem, cpt, smem;
+  int S, NA, E, act_slot_bytes, slab_max, kst, nacc, nf, rem_base, rem, cpt, smem, R, lead;
   bool ok;
 };
 
@@ -887,10 +899,18 @@ TcGeometry tc_plan(int D, int H, int grid) {
   g.cpt = nvecD <= kAT ? 1 : nvecD <= 2 * kAT ? 2 : nvecD <= 4 * kAT ? 4 : 8;
   g.kst = (D / 64 + kSegs - 1) / kSegs;
   g.nacc = g.kst >= 2 ? 2 : 1;
-  g.nf = (H / kTileRows) / grid;
-  g.rem_base = g.nf * grid * kTileRows;
+  // CTAs that stay for the cross-CTA sum: one per 32 stored units of a partial, never more than half the grid (the
+  // waiting CTAs of two calls that overlap must not hold every SM between them)
+  const int units = g.cpt * 4 * kAT;
+  g.R = std::min(std::max(1, (grid - 1) / 2), std::max(1, units / 32));
+  const int tiles = H / kTileRows, early = grid - g.R;
+  g.lead = fused_test_knobs().lead_tiles;
+  if (g.lead < 0) g.lead = 0;
+  while (g.lead > 0 && (g.lead + 1) * early > tiles) --g.lead;
+  g.nf = (tiles - g.lead * early) / grid;
+  g.rem_base = (g.lead * early + g.nf * grid) * kTileRows;
   g.rem = H - g.rem_base;
-  g.slab_max = g.nf * kTileRows + (g.rem + grid - 1) / grid;
+  g.slab_max = (g.nf + g.lead) * kTileRows + (g.rem + grid - 1) / grid;
   g.act_slot_bytes = (2 * D * 2 + 1023) / 1024 * 1024;
   // a slot that is nearly a whole number of gate stages is padded to it: it can then park gate stages at the start
   const int whole = (g.act_slot_bytes + kStageBytes - 1) / kStageBytes * kStageBytes;
@@ -961,7 +981,7 @@ cudaError_t launch_fused_tc(const FusedCall& c, cudaStream_t s, int* launched) {
   p.S = g.S; p.NA = g.NA; p.E = g.E; p.F = fused_test_knobs().ring_F & ~1;
   if (p.F > g.S) p.F = g.S;  // the stage waited for must be the latest use of its ring slot
   p.act_slot_bytes = g.act_slot_bytes; p.slab_max = g.slab_max; p.kst = g.kst; p.nacc = g.nacc;
-  p.nf = g.nf; p.rem_base = g.rem_base; p.rem = g.rem;
+  p.nf = g.nf; p.rem_base = g.rem_base; p.rem = g.rem; p.R = g.R; p.lead = g.lead;
   p.l2_hints = fused_test_knobs().l2_hints;
   p.wait_cycles = fused_test_knobs().wait_cycles;
   p.skip_arrival_cta = fused_test_knobs().skip_arrival_cta;
