@@ -275,7 +275,7 @@ const char* sffn_status_string(int status);
 typedef enum {
   SFFN_KNOB_PDL = 0, SFFN_KNOB_TENSOR_GATE = 1, SFFN_KNOB_WAIT_CYCLES = 2, SFFN_KNOB_SKIP_ARRIVAL_CTA = 3,
   SFFN_KNOB_RING_GATE_SLOTS = 4, SFFN_KNOB_RING_ACT_SLOTS = 5, SFFN_KNOB_TRACE_BUFFER = 6,
-  SFFN_KNOB_RING_PARKED_STAGES = 7, SFFN_KNOB_L2_HINTS = 8, SFFN_KNOB_RING_IN_FLIGHT = 9, SFFN_KNOB_LEAD_TILES = 10
+  SFFN_KNOB_RING_PARKED_STAGES = 7, SFFN_KNOB_L2_HINTS = 8
 } sffn_test_knob;
 void sffn_test_fused_plan(int wkind, int D, int H, int K, int lopa, int sm_count, int* out9);
 void sffn_test_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list);

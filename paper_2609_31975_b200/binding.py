@@ -86,7 +86,7 @@ def load_library() -> ctypes.CDLL:
 
 
 KNOB = {"pdl": 0, "tensor_gate": 1, "wait_cycles": 2, "skip_arrival_cta": 3, "ring_gate_slots": 4,
-        "ring_act_slots": 5, "trace_buffer": 6, "ring_parked_stages": 7, "l2_hints": 8, "ring_in_flight": 9, "lead_tiles": 10}
+        "ring_act_slots": 5, "trace_buffer": 6, "ring_parked_stages": 7, "l2_hints": 8}
 
 
 def test_set_knob(name: str, value: int):

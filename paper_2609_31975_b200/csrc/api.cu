@@ -171,8 +171,6 @@ int sffn_test_set_knob(int knob, long long value) {
     case SFFN_KNOB_RING_ACT_SLOTS: k.ring_NA = (int)value; return SFFN_OK;
     case SFFN_KNOB_RING_PARKED_STAGES: k.ring_E = (int)value; return SFFN_OK;
     case SFFN_KNOB_L2_HINTS: k.l2_hints = (int)value; return SFFN_OK;
-    case SFFN_KNOB_RING_IN_FLIGHT: k.ring_F = (int)value; return SFFN_OK;
-    case SFFN_KNOB_LEAD_TILES: k.lead_tiles = (int)value; return SFFN_OK;
     case SFFN_KNOB_TRACE_BUFFER: k.trace = reinterpret_cast<long long*>(static_cast<uintptr_t>(value)); return SFFN_OK;
     default: return SFFN_ERR_INVALID_ARG;
   }

@@ -51,8 +51,6 @@ struct FusedTestKnobs {
   int skip_arrival_cta = -1;     // this CTA does not count itself as finished: the summing CTAs' wait runs out
   int ring_S = 0, ring_NA = 0;   // tensor-core gate: ring split override (0 = planned)
   int l2_hints = 2;              // tensor-core gate: bit 0 weights evict-first, bit 1 partials evict-last
-  int lead_tiles = 0;            // tensor-core gate: extra tiles of the CTAs that do not stay for the cross-CTA sum
-  int ring_F = 0;                // tensor-core gate: most gate stages in flight per CTA (0 = no limit)
   int ring_E = -1;               // tensor-core gate: gate stages parked in the act ring at the start (-1 = planned)
   long long* trace = nullptr;    // SFFN_TRACE builds: [grid][16] time stamps
 };

@@ -75,11 +75,9 @@ struct TcParams {
   int32_t* status;
   int act, dense, act_up;
   int S, NA, act_slot_bytes, slab_max, kst, nacc;
-  int F;         // most gate stages a CTA has in flight (requested, not yet landed); 0 = no limit
   int E;         // gate stages that are prefetched into the (still idle) last E act slots at the start of a call
   int R;         // CTAs that stay to sum the partials (the last R to finish)
-  int lead;      // extra tiles of the first grid - R CTAs (see tile_of)
-  int nf;        // full tiles of every CTA beyond those
+  int nf;        // full tiles of every CTA (tile t of CTA c is tile c + t * grid of the matrix)
   int rem_base;  // rows from here on are dealt in contiguous runs of <= 8 (each CTA's last, short tile)
   int rem;
   int l2_hints;           // bit 0: weights evict-first, bit 1: partials evict-last
@@ -292,7 +290,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   const int G = gridDim.x, cta = blockIdx.x;
   if (tid == 0) TC_STAMP(10);
   const int D = p.D;
-  const int S = p.S, NA = p.NA, kst = p.kst, nacc = p.nacc, E = p.E;
+  const int S = p.S, NA = p.NA, kst = p.kst, nacc = p.nacc;
   const TcLayout L(S, NA, p.act_slot_bytes, p.slab_max, kst);
   unsigned char* act_ring = smem + L.act_ring;
   unsigned char* xb = smem + L.xb;
@@ -311,26 +309,26 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
   const int nvecD = D / 8;
   const size_t row_bytes = (size_t)D * 2;
   // This CTA's neurons: nf full tiles dealt round robin over the CTAs, then a contiguous run of the left-over rows.
-  // Tiles are dealt round robin, with a head start for the CTAs that can use one: in a run of back-to-back calls
-  // the R CTAs that summed the previous call's partials start last (their SMs come free last, and the hardware
-  // hands out CTAs in index order), with nothing prefetched; the other G - R get `lead` more tiles each.
-  const int early = G - p.R;
-  const int lead = cta < early ? p.lead : 0;
-  const int nf = p.nf + lead;
-  auto tile_of = [&](int t) { return t < lead ? cta + t * early : p.lead * early + cta + (t - lead) * G; };
+  const int nf = p.nf;
   const int rem_lo = p.rem_base + (int)((long long)p.rem * cta / G);
   const int rc = p.rem_base + (int)((long long)p.rem * (cta + 1) / G) - rem_lo;
   const int n_tiles = nf + (rc > 0 ? 1 : 0);
   const int slab_rows = nf * kTileRows + rc;
   auto neuron_of = [&](int l) {
     const int t = l >> 3;
-    return t < nf ? tile_of(t) * kTileRows + (l & 7) : rem_lo + (l - nf * kTileRows);
+    return t < nf ? (cta + t * G) * kTileRows + (l & 7) : rem_lo + (l - nf * kTileRows);
   };
   // Where gate stage `it` of this CTA's sequence lives.  The first S stages fill the gate ring; the next E go into the
   // last act slots, which no fired row can need yet (no gate result exists before the token has arrived): the CTA
   // starts while its predecessor in the stream still runs, and everything it can fetch before the token is there
   // shortens the call.  From then on the gate ring is used round robin.
-  const int m_per_slot = p.act_slot_bytes / kStageBytes;  // gate stages per act slot (E > 0 only if it divides)
+  const int m_per_slot = p.act_slot_bytes / kStageBytes;  // gate stages per act slot (p.E > 0 only if it divides)
+  // stages parked by this CTA: no more than it has beyond the gate ring, whole act slots, an even number
+  int E = min(p.E, max(0, n_tiles * kst - S));
+  if (E > 0) {
+    E = E / m_per_slot * m_per_slot;
+    if (E & 1) E -= m_per_slot;
+  }
   const int extra_slots = E > 0 ? E / m_per_slot : 0;      // act slots that start out holding gate stages
   const uint32_t extra_base = smem_u32(act_ring) + (uint32_t)(NA - extra_slots) * p.act_slot_bytes;
   if (tid == 0) {
@@ -372,19 +370,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
     if (lane == 0) {
       const uint64_t once = policy_evict_first(p.l2_hints & 1);
       const int total = n_tiles * kst;
-      StageCursor c, lag;  // lag: the stage p.F before c (same producer), whose arrival is waited for first
+      StageCursor c;
       c.start(S, E, warp, kGateProducers);
-      lag.start(S, E, warp, kGateProducers);
       int t = warp / kst, st = warp - t * kst;
       for (; c.it < total; c.next()) {
-        // Bytes in flight beyond what the memory system needs to run at its rate only queue up in front of every
-        // other access of the GPU (the token, the partial sums): a stage is requested once the stage F before it
-        // has landed.
-        if (p.F > 0 && c.it >= p.F + warp) {
-          const uint32_t lbar = lag.parked() ? extra_full + 8 * (lag.it - S) : full_gate + 8 * lag.slot;
-          if (!mbar_wait(lbar, lag.parked() ? 0u : lag.phase, ctl, p.status, p.wait_cycles, 1)) break;
-          lag.next();
-        }
         uint32_t dst, bar;
         if (c.parked()) {
           dst = extra_base + (uint32_t)(c.it - S) * kStageBytes;
@@ -396,7 +385,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
         }
         if (t < nf) {
           mbar_expect_tx(bar, kStageBytes);
-          tma_tile_3d(dst, &map8, 0, st * kSegs, tile_of(t) * kTileRows, bar, once);
+          tma_tile_3d(dst, &map8, 0, st * kSegs, (cta + t * G) * kTileRows, bar, once);
         } else {
           mbar_expect_tx(bar, (uint32_t)rc * (kSegs * 128));
           for (int i = 0; i < rc; ++i)
@@ -802,7 +791,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
           if (t0 == 0) t0 = clock64();
           if (ctl[kAbort]) { ok = false; break; }
           if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status, 21); ok = false; break; }
-          __nanosleep(100);
+          __nanosleep(20);
         }
 #ifdef SFFN_TRACE
         if (tt == 0 && g0 == rg && p.trace) { TC_STAMP(14); p.trace[(size_t)blockIdx.x * 16 + 15] = tries; }
@@ -887,7 +876,7 @@ const MapEntry* gate_maps(const void* base, int D, int H) {
 }
 
 struct TcGeometry {
-  int S, NA, E, act_slot_bytes, slab_max, kst, nacc, nf, rem_base, rem, cpt, smem, R, lead;
+  int S, NA, E, act_slot_bytes, slab_max, kst, nacc, nf, rem_base, rem, cpt, smem, R;
   bool ok;
 };
 
@@ -903,14 +892,10 @@ TcGeometry tc_plan(int D, int H, int grid) {
   // waiting CTAs of two calls that overlap must not hold every SM between them)
   const int units = g.cpt * 4 * kAT;
   g.R = std::min(std::max(1, (grid - 1) / 2), std::max(1, units / 32));
-  const int tiles = H / kTileRows, early = grid - g.R;
-  g.lead = fused_test_knobs().lead_tiles;
-  if (g.lead < 0) g.lead = 0;
-  while (g.lead > 0 && (g.lead + 1) * early > tiles) --g.lead;
-  g.nf = (tiles - g.lead * early) / grid;
-  g.rem_base = (g.lead * early + g.nf * grid) * kTileRows;
+  g.nf = (H / kTileRows) / grid;
+  g.rem_base = g.nf * grid * kTileRows;
   g.rem = H - g.rem_base;
-  g.slab_max = (g.nf + g.lead) * kTileRows + (g.rem + grid - 1) / grid;
+  g.slab_max = g.nf * kTileRows + (g.rem + grid - 1) / grid;
   g.act_slot_bytes = (2 * D * 2 + 1023) / 1024 * 1024;
   // a slot that is nearly a whole number of gate stages is padded to it: it can then park gate stages at the start
   const int whole = (g.act_slot_bytes + kStageBytes - 1) / kStageBytes * kStageBytes;
@@ -978,10 +963,9 @@ cudaError_t launch_fused_tc(const FusedCall& c, cudaStream_t s, int* launched) {
   p.partial = reinterpret_cast<unsigned long long*>(ws + fused_tagged_partials_offset(c.D, c.r_max));
   p.flag = c.flag; p.status = c.status;
   p.act = c.act; p.dense = c.dense ? 1 : 0; p.act_up = c.act_up;
-  p.S = g.S; p.NA = g.NA; p.E = g.E; p.F = fused_test_knobs().ring_F & ~1;
-  if (p.F > g.S) p.F = g.S;  // the stage waited for must be the latest use of its ring slot
+  p.S = g.S; p.NA = g.NA; p.E = g.E;
   p.act_slot_bytes = g.act_slot_bytes; p.slab_max = g.slab_max; p.kst = g.kst; p.nacc = g.nacc;
-  p.nf = g.nf; p.rem_base = g.rem_base; p.rem = g.rem; p.R = g.R; p.lead = g.lead;
+  p.nf = g.nf; p.rem_base = g.rem_base; p.rem = g.rem; p.R = g.R;
   p.l2_hints = fused_test_knobs().l2_hints;
   p.wait_cycles = fused_test_knobs().wait_cycles;
   p.skip_arrival_cta = fused_test_knobs().skip_arrival_cta;
