@@ -71,7 +71,7 @@ typedef enum {
 /* Activation A of Eq. 1.  RELU and R-S+ follow the table of Sec. 3.1 (R-S+: 0 for z < 0,
  * z*sigmoid(z) for z >= 0); SQRELU = max(z,0)^2 is one of the activations of the paper's activation
  * study.  For all three A(z) != 0 exactly when z > 0, which is the test the library applies. */
-typedef enum { SFFN_ACT_RELU = 0, SFFN_ACT_SQRELU = 1, SFFN_ACT_RSPLUS = 2, SFFN_ACT_NONE = 3 } sffn_act;
+typedef enum { SFFN_ACT_RELU = 0, SFFN_ACT_SQRELU = 1, SFFN_ACT_RSPLUS = 2, SFFN_ACT_NONE = 3, SFFN_ACT_SILU = 4 } sffn_act;
 
 typedef enum { SFFN_F32 = 0, SFFN_BF16 = 1 } sffn_dtype;
 
@@ -119,13 +119,15 @@ int sffn_destroy(sffn_handle* handle);
 
 int sffn_set_path(sffn_handle* handle, int path /* sffn_path */);
 
-/* Double activation (Sec. 3.3, "Double activation"): with act_up = RELU / SQRELU / RSPLUS every later
+/* Double activation (Sec. 3.3, "Double activation"): with act_up = RELU / SQRELU / RSPLUS / SILU every later
  * call on the handle computes y = W_2 ( A(W_1 x + b_g) . A_3(W_3 x) ), A_3 = act_up, in the sparse and
- * in the dense entry points alike; SFFN_ACT_NONE (the default) is Eq. 1.  A neuron whose product
+ * in the dense entry points alike; SFFN_ACT_NONE (the default) is Eq. 1.  SILU (z * sigmoid(z), the table of
+ * Sec. 3.1) is what a model cast per Sec. 3.3 keeps on the up branch: only the activation of W_1 is cast to a
+ * sparse one.  It exists as A_3 only: the gate's `act` must be one of the three sparse activations.  A neuron whose product
  * A(.) A_3(.) is zero for every token of the call contributes nothing (the "s_gated" site of the
  * paper's sparsity-sites table): the CUDA-core path (SFFN_PATH_GENERAL) then does not read its row of
  * W_down; the fused and the tensor-core paths fetch the two rows of a fired neuron together and read it.
- * SFFN_ACT_NONE is not a gate activation: `act` of the forward calls stays one of the other three. */
+ * SFFN_ACT_NONE and SFFN_ACT_SILU are not gate activations: `act` of the forward calls stays one of the first three. */
 int sffn_set_up_activation(sffn_handle* handle, int act_up /* sffn_act */);
 
 /* Sparse execution of Eq. 1 (Sec. 3.1): gate in full, then only the active rows of W_up / W_down.
@@ -263,19 +265,26 @@ const char* sffn_status_string(int status);
  * sffn_test_fused_plan: geometry of the single-token CUDA-core kernel for a shape, as nine integers: ok, rows per
  *   gate slot, gate slot bytes, gate slots, gate warps, act slot bytes, act slots, chunks per act thread, shared
  *   memory bytes (wkind: 0 fp32, 1 bf16, 2 int8 rows).  sffn_test_umma_tiling: tiling of the batched gate GEMM.
- * sffn_test_set_knob: PDL = programmatic dependent launch between calls (default 1); TENSOR_GATE = take the
- *   tensor-core gate in single-token bf16 calls where it applies (default 1); WAIT_CYCLES = budget of every
- *   device-side wait in clock cycles (default 2^31, about a second; 0 restores it); SKIP_ARRIVAL_CTA = index of a CTA
- *   of the single-token kernels that does not report itself finished, so that the CTAs which sum the partial
- *   results see their (bounded) wait run out and record SFFN_ERR_TIMEOUT (-1 = none, the default; use it with a
- *   small WAIT_CYCLES); RING_GATE_SLOTS / RING_ACT_SLOTS = split of the tensor-core kernel's shared-memory rings
- *   (0 = planned), RING_PARKED_STAGES = gate stages it prefetches into idle act slots at the start of a call (-1 =
- *   planned); TRACE_BUFFER = device address of [grid][16] int64 time stamps, written only by libraries built
- *   with -DSFFN_TRACE. */
+ * sffn_test_set_knob(knob, value):
+ *   PDL                 programmatic dependent launch between calls (default 1)
+ *   TENSOR_GATE         single-token bf16 calls take the tensor-core gate kernel where it applies (default 1)
+ *   WAIT_CYCLES         budget of every device-side wait in clock cycles (default 2^31, about a second; 0 restores it)
+ *   SKIP_ARRIVAL_CTA    index of a CTA of the single-token kernels that neither reports itself finished nor hands in
+ *                       its partial result, so that the CTAs which sum the partials see their (bounded) wait run out
+ *                       and record SFFN_ERR_TIMEOUT (-1 = none, the default; use it with a small WAIT_CYCLES)
+ *   DROP_STAGE          index of a stage of the batched gate kernel whose weight copy CTA 0 leaves out, so that the wait
+ *                       for it runs out and the kernel winds down and releases its TMEM columns (-1 = none, the default)
+ *   RING_GATE_SLOTS, RING_ACT_SLOTS, RING_PARKED_STAGES
+ *                       tensor-core gate kernel: split of its shared-memory rings and the number of gate stages it
+ *                       prefetches into idle act slots at the start of a call (0, 0, -1 = planned)
+ *   L2_HINTS            tensor-core gate kernel: bit 0 = weights are fetched evict-first, bit 1 = the per-CTA partial
+ *                       results are stored evict-last (default 2)
+ *   TRACE_BUFFER        device address of [grid][16] int64 time stamps, written only by libraries built with
+ *                       -DSFFN_TRACE (0 = none) */
 typedef enum {
   SFFN_KNOB_PDL = 0, SFFN_KNOB_TENSOR_GATE = 1, SFFN_KNOB_WAIT_CYCLES = 2, SFFN_KNOB_SKIP_ARRIVAL_CTA = 3,
   SFFN_KNOB_RING_GATE_SLOTS = 4, SFFN_KNOB_RING_ACT_SLOTS = 5, SFFN_KNOB_TRACE_BUFFER = 6,
-  SFFN_KNOB_RING_PARKED_STAGES = 7, SFFN_KNOB_L2_HINTS = 8
+  SFFN_KNOB_RING_PARKED_STAGES = 7, SFFN_KNOB_L2_HINTS = 8, SFFN_KNOB_DROP_STAGE = 9
 } sffn_test_knob;
 void sffn_test_fused_plan(int wkind, int D, int H, int K, int lopa, int sm_count, int* out9);
 void sffn_test_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list);

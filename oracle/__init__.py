@@ -34,7 +34,7 @@ _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "sparse_ffn_oracle.cpp"
 _LIB = _HERE / "build" / "libsparse_ffn_oracle.so"
 
-ACT = {"relu": 0, "sqrelu": 1, "rsplus": 2}
+ACT = {"relu": 0, "sqrelu": 1, "rsplus": 2, "silu": 3}  # silu: only as act_up (it is not sparse)
 _DT = {np.dtype(np.float32): 0, np.dtype(np.uint16): 1, np.dtype(np.float64): 2}
 
 

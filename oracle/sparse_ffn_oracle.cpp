@@ -36,7 +36,7 @@
 namespace {
 
 enum DType { F32 = 0, BF16 = 1, F64 = 2 };
-enum Act { RELU = 0, SQRELU = 1, RSPLUS = 2 };
+enum Act { RELU = 0, SQRELU = 1, RSPLUS = 2, SILU = 3 };
 
 // Exact decode of one stored element to double.
 inline double load(const void* p, int dtype, size_t i) {
@@ -54,9 +54,12 @@ inline double load(const void* p, int dtype, size_t i) {
   }
 }
 
-// Activation table of Sec. 3.1 (RELU, R-S+) plus squared RELU (Sec. 5, other activations).
+// Activation table of Sec. 3.1 (RELU, SILU, R-S+) plus squared RELU (Sec. 5, other activations).  SILU is not
+// sparse; it only ever serves as A_3 on the up projection (Sec. 3.3, "Double activation": the activation of W_1
+// alone is cast, the other one stays what the model was trained with).
 inline double activation(int act, double z) {
-  if (!(z > 0.0)) return 0.0;  // z <= 0 (and -0) give exactly 0 for all three
+  if (act == SILU) return z / (1.0 + std::exp(-z));  // z * sigmoid(z) on both sides
+  if (!(z > 0.0)) return 0.0;  // z <= 0 (and -0) give exactly 0 for the three sparse activations
   switch (act) {
     case RELU:
       return z;
@@ -170,6 +173,7 @@ int oracle_ffn_batch(int gate_kind, const void* W1, const void* V, const void* U
   if (B < 0 || H <= 0 || D <= 0 || !W3 || !Wdown || !x || !y) return -1;
   if (gate_kind == 0 && !W1) return -1;
   if (gate_kind == 1 && (!V || !U || r <= 0)) return -1;
+  if (act < RELU || act > RSPLUS || act_up > SILU) return -1;  // the gate's activation must be a sparse one
   if (union_mask) std::memset(union_mask, 0, (size_t)H);
   const size_t xstride = (size_t)D * (xdtype == F32 ? 4 : xdtype == BF16 ? 2 : 8);
   std::vector<int32_t> n_act(B > 0 ? B : 1), n_gated(B > 0 ? B : 1);

@@ -8,6 +8,7 @@ import torch
 
 _PKG = Path(__file__).resolve().parent
 ACT = {"relu": 0, "sqrelu": 1, "rsplus": 2}
+ACT_UP = dict(ACT, silu=4)  # activations of the up projection (double activation); SILU is not a gate activation
 PATH = {"auto": 0, "general": 1, "fused": 2, "mma_sync": 3}
 _STATUS = {0: "ok", 1: "invalid argument", 2: "unsupported shape, alignment or path",
            3: "workspace missing, misaligned or too small", 4: "CUDA runtime error",
@@ -86,7 +87,7 @@ def load_library() -> ctypes.CDLL:
 
 
 KNOB = {"pdl": 0, "tensor_gate": 1, "wait_cycles": 2, "skip_arrival_cta": 3, "ring_gate_slots": 4,
-        "ring_act_slots": 5, "trace_buffer": 6, "ring_parked_stages": 7, "l2_hints": 8}
+        "ring_act_slots": 5, "trace_buffer": 6, "ring_parked_stages": 7, "l2_hints": 8, "drop_stage": 9}
 
 
 def test_set_knob(name: str, value: int):
@@ -215,7 +216,7 @@ class SparseFFN:
 
     def set_up_activation(self, act_up):
         """Double activation: ``act_up`` in ACT (or None for Eq. 1) is applied to the up projection."""
-        code = 3 if act_up is None else ACT[act_up]
+        code = 3 if act_up is None else ACT_UP[act_up]
         _check("sffn_set_up_activation", self.lib.sffn_set_up_activation(self._h, code))
 
     def set_path(self, path: str):

@@ -141,7 +141,7 @@ int sffn_destroy(sffn_handle* h) {
 }
 
 int sffn_set_up_activation(sffn_handle* h, int act_up) {
-  if (!h || act_up < SFFN_ACT_RELU || act_up > SFFN_ACT_NONE) return SFFN_ERR_INVALID_ARG;
+  if (!h || act_up < SFFN_ACT_RELU || act_up > SFFN_ACT_SILU) return SFFN_ERR_INVALID_ARG;
   h->act_up = act_up;
   return SFFN_OK;
 }
@@ -171,6 +171,7 @@ int sffn_test_set_knob(int knob, long long value) {
     case SFFN_KNOB_RING_ACT_SLOTS: k.ring_NA = (int)value; return SFFN_OK;
     case SFFN_KNOB_RING_PARKED_STAGES: k.ring_E = (int)value; return SFFN_OK;
     case SFFN_KNOB_L2_HINTS: k.l2_hints = (int)value; return SFFN_OK;
+    case SFFN_KNOB_DROP_STAGE: k.drop_stage = (int)value; return SFFN_OK;
     case SFFN_KNOB_TRACE_BUFFER: k.trace = reinterpret_cast<long long*>(static_cast<uintptr_t>(value)); return SFFN_OK;
     default: return SFFN_ERR_INVALID_ARG;
   }

@@ -11,6 +11,7 @@ constexpr int kActRelu = 0;
 constexpr int kActSqRelu = 1;
 constexpr int kActRsPlus = 2;
 constexpr int kActNone = 3;  // identity: internal stages that only need the raw products
+constexpr int kActSilu = 4;  // z * sigmoid(z) on both sides: only ever A_3 on the up projection (it is not sparse)
 
 // Activation of the gate (activation table of Sec. 3.1; squared RELU from the activation study).
 // For all three, A(z) != 0 exactly when z > 0 in exact arithmetic; callers test z > 0.
@@ -20,6 +21,7 @@ static __device__ __noinline__ float rsplus_of_nonnegative(float p) { return p /
 
 __device__ __forceinline__ float activation(int act, float z) {
   if (act == kActNone) return z;
+  if (act == kActSilu) return rsplus_of_nonnegative(z);  // the same expression on the whole axis (-0 for z -> -inf)
   const float p = fmaxf(z, 0.f);                 // 0 for z <= 0
   if (act == kActRelu) return p;
   if (act == kActSqRelu) return p * p;

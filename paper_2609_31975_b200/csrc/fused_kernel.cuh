@@ -48,6 +48,7 @@ struct FusedTestKnobs {
   bool pdl = true;               // programmatic dependent launch between calls
   bool tensor_gate = true;       // take the tensor-core gate where it applies
   long long wait_cycles = 1LL << 31;  // budget of every device-side wait (about one second)
+  int drop_stage = -1;           // batched gate kernel: CTA 0 never copies this stage's weights (its wait runs out)
   int skip_arrival_cta = -1;     // this CTA does not count itself as finished: the summing CTAs' wait runs out
   int ring_S = 0, ring_NA = 0;   // tensor-core gate: ring split override (0 = planned)
   int l2_hints = 2;              // tensor-core gate: bit 0 weights evict-first, bit 1 partials evict-last

@@ -31,6 +31,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "fused_kernel.cuh"
 #include "sparse_ffn.h"
 
 namespace sffn {
@@ -52,7 +53,6 @@ constexpr int kMaxIssuers = 4;
 constexpr int kScanChunks = 4;                       // in-kernel compaction: up to 4 * 384 mask words = 384 gate tiles
 constexpr int kMaxOwnTiles = 8;                      // tiles of one CTA whose rows are kept in shared memory
 constexpr int kHeaderBytes = 1024 + kMaxOwnTiles * kTileRows * 4;  // barriers + scratch, then the row lists
-constexpr long long kWaitCycles = 1LL << 31;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -74,7 +74,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          long long budget) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
@@ -82,7 +83,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 64; ++i)
       if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > budget) {
       *abort_flag = 1;
       atomicExch(status, (int32_t)SFFN_ERR_TIMEOUT);
       return false;
@@ -427,7 +428,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       sg = (row_ok && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
     }
     int okw = 1;
-    if (lane == 0) okw = mbar_wait(acc_full, tcount & 1, abort_flag, p.status) ? 1 : 0;
+    if (lane == 0) okw = mbar_wait(acc_full, tcount & 1, abort_flag, p.status, p.wait_cycles) ? 1 : 0;
     okw = __shfl_sync(0xffffffffu, okw, 0);
     if (!okw) return false;
     tc_fence_after();
@@ -522,7 +523,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
         if (with_w) {
           int ok = 1;
           if (lane == 0) {
-            ok = mbar_wait(empty + 8 * s, ph ^ 1, abort_flag, p.status) ? 1 : 0;
+            ok = mbar_wait(empty + 8 * s, ph ^ 1, abort_flag, p.status, p.wait_cycles) ? 1 : 0;
             if (ok) mbar_expect_tx(full + 8 * s, tx_bytes);
           }
           ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -531,7 +532,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
         const uint32_t abase = stage0 + s * stage_bytes;
         for (int a = 0; a < na; ++a) {
           const int k0 = (kb * atoms + a) * kAtomK;
-          if (with_w) {
+          if (with_w && !(MODE == kGate && blockIdx.x == 0 && it == p.drop_stage)) {  // test hook: a copy that never comes
             if (UP && !walk_all) {
               if (lane * 4 < tile_rows)
                 tma_gather4(abase + a * a_block_bytes + lane * 512, &map_w, k0, r[0], r[1], r[2], r[3], full + 8 * s);
@@ -565,14 +566,14 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       int tcount = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++tcount) {
-        if (!mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, p.status)) break;
+        if (!mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, p.status, p.wait_cycles)) break;
         tc_fence_after();
         const int it0 = tcount * kstages;
         int s = it0 % S, ph = (it0 / S) & 1;
         for (int kb = 0; kb < kstages; ++kb, ++s) {
           if (s == S) { s = 0; ph ^= 1; }
           if ((s & (nacc - 1)) != m) continue;   // another issuer's slot
-          if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+          if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status, p.wait_cycles)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sbase = stage0 + s * stage_bytes;
           const int na = min(atoms, kblocks - kb * atoms);
@@ -644,6 +645,10 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   }
 
   // ---- teardown: everybody meets, then the allocating warp frees the TMEM columns ------------------
+  // (after a wait that ran out, copies and MMAs may still be in flight: they end within microseconds, and shared
+  // memory and TMEM are only given back after that)
+  if (*abort_flag)
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);
   tc_fence_before();
   __syncthreads();
   if (warp == 8) {
@@ -742,7 +747,7 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
       }
       int ok = 1;
       if (lane == 0) {
-        ok = mbar_wait(empty + 8 * s, ph ^ 1, abort_flag, p.status) ? 1 : 0;
+        ok = mbar_wait(empty + 8 * s, ph ^ 1, abort_flag, p.status, p.wait_cycles) ? 1 : 0;
         if (ok) mbar_expect_tx(full + 8 * s, tx_bytes);
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -767,7 +772,7 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
       for (int kb = 0; kb < kblocks; ++kb, ++s) {
         if (s == S) { s = 0; ph ^= 1; }
         if (nacc == 2 && (s & 1) != m) continue;
-        if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status, p.wait_cycles)) { ok = false; break; }
         tc_fence_after();
         const uint32_t sbase = stage0 + s * stage_bytes;
         const uint64_t bdesc = make_desc(sbase + kAAtomBytes);
@@ -790,7 +795,7 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
       for (int b = 0; b < B; ++b) out[(size_t)b * p.D] = 0.f;
     } else {
       int okw = 1;
-      if (lane == 0) okw = mbar_wait(acc_full, 0, abort_flag, p.status) ? 1 : 0;
+      if (lane == 0) okw = mbar_wait(acc_full, 0, abort_flag, p.status, p.wait_cycles) ? 1 : 0;
       okw = __shfl_sync(0xffffffffu, okw, 0);
       if (okw) {
         tc_fence_after();
@@ -805,6 +810,8 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
     }
   }
 
+  if (*abort_flag)
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);
   tc_fence_before();
   __syncthreads();
   if (warp == 8) {
@@ -898,6 +905,8 @@ bool make_map(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_el
 
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s) {
   p.npad = (cols + 15) / 16 * 16;
+  p.wait_cycles = fused_test_knobs().wait_cycles;
+  p.drop_stage = fused_test_knobs().drop_stage;
   const int grid = p.R < 8 * sm_count ? (p.R + 7) / 8 : sm_count;
   // all the dynamic shared memory a CTA can have; the kernel cuts its ring out of it once it knows its tiles
   const size_t smem = 226 * 1024;
@@ -938,6 +947,7 @@ bool umma_down_supported(int D, int cols) { return D % kTileRows == 0 && cols >=
 
 cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s) {
   p.npad = (p.B + 15) / 16 * 16;
+  p.wait_cycles = fused_test_knobs().wait_cycles;
   const int stage_bytes = kAAtomBytes + p.npad * 128;
   int stages = (111 * 1024 - 1024 - 1024) / stage_bytes;
   if (stages > 12) stages = 12;

@@ -42,6 +42,8 @@ struct UmmaRowsParams {
   int act_up;            // UP: activation on the up projection (double activation), kUmmaActIdentity = none
   int32_t* status;       // device status word
   int npad, ring_bytes;  // filled by the launcher
+  long long wait_cycles; // budget of every device-side wait (filled by the launcher)
+  int drop_stage;        // test hook: CTA 0 of the gate kernel never copies the weights of this stage (-1: none)
 };
 
 struct UmmaDownParams {
@@ -57,6 +59,7 @@ struct UmmaDownParams {
   float* partial;        // [splits][B][D]
   int32_t* status;
   int npad, stages;      // filled by the launcher
+  long long wait_cycles; // budget of every device-side wait (filled by the launcher)
 };
 
 int umma_down_splits(int D, int sm_count, int max_splits);

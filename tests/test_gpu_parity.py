@@ -309,7 +309,7 @@ def test_batched_calls_repeat_bit_for_bit(mod):
 
 
 # ------------------------------------------------------------------ double activation (Sec. 3.3)
-@pytest.mark.parametrize("act,act_up", [("relu", "relu"), ("sqrelu", "rsplus"), ("rsplus", "sqrelu")])
+@pytest.mark.parametrize("act,act_up", [("relu", "relu"), ("sqrelu", "rsplus"), ("rsplus", "sqrelu"), ("relu", "silu")])
 def test_double_activation_all_paths(mod, act, act_up):
     D, H = 512, 1100
     ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=64, B_max=8)
@@ -317,7 +317,10 @@ def test_double_activation_all_paths(mod, act, act_up):
     gate, w = make_std(D, H, torch.bfloat16, 61, 0.8)
     x = syn.tokens(8, D, torch.bfloat16, 61, DEV)
     ref1 = run_oracle(x[0], gate, w["b_g"], w["W_up"], w["W_down"], act, act_up=act_up)
-    assert 0 < ref1["n_gated"][0] < ref1["n_act"][0]                    # A_3 really removes neurons
+    if act_up == "silu":                                                # SILU is not sparse: nothing is removed
+        assert ref1["n_gated"][0] == ref1["n_act"][0]
+    else:
+        assert 0 < ref1["n_gated"][0] < ref1["n_act"][0]                # A_3 really removes neurons
     for path in ("general", "fused"):                                   # one token
         ffn.set_path(path)
         y = ffn.sparse_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], act)
@@ -394,27 +397,50 @@ def test_layer_chain_in_cuda_graph(mod, dtype, kind):
 
 
 # ------------------------------------------------------------------ full-size configurations
-def test_config2_full_size_decode(mod):
+@pytest.mark.parametrize("s,ntok", [(0.9, 8), (0.5, 1), (0.7, 2), (0.8, 2), (0.95, 1)])
+def test_config2_full_size_decode(mod, s, ntok):
     D, H = 4096, 14336
     ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=1)
-    for s, ntok in ((0.9, 3), (0.5, 1), (0.95, 1)):
-        gate, w = make_std(D, H, torch.bfloat16, 2, s)
-        x = syn.tokens(ntok, D, torch.bfloat16, 2, DEV)
-        for t in range(ntok):
-            ref = run_both_paths(mod, ffn, x[t], gate, w, "relu", ("general", "fused"), what=f"config2 s={s}")
-            assert abs(1 - ref["n_act"][0] / H - s) < 0.03
-        del gate, w
+    gate, w = make_std(D, H, torch.bfloat16, 2, s)
+    x = syn.tokens(ntok, D, torch.bfloat16, 2, DEV)
+    ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", threads=16)
+    assert abs(1 - ref["n_act"].mean() / H - s) < 0.03
+    for path in ("general", "fused"):            # fused: the tensor-core gate kernel at this shape
+        ffn.set_path(path)
+        for t in range(ntok if path == "fused" else min(ntok, 2)):
+            y = ffn.sparse_ffn_forward(x[t], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+            one = dict(y=ref["y"][t], z=ref["z"][t])
+            assert_y_close(y, one["y"], what=f"config2 s={s} token {t} [{path}]")
+            assert_active_set(ffn.last_active(), one, what=f"config2 s={s} token {t} [{path}]")
+    # the CUDA-core gate of the single-token kernel (what other storage types run) at the same shape
+    mod.test_set_knob("tensor_gate", 0)
+    try:
+        y = ffn.sparse_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+        assert_y_close(y, ref["y"][0], what=f"config2 s={s} [fused, CUDA-core gate]")
+        assert_active_set(ffn.last_active(), dict(z=ref["z"][0]), what=f"config2 s={s} [fused, CUDA-core gate]")
+    finally:
+        mod.test_set_knob("tensor_gate", 1)
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
 
 
-def test_config3_full_size_lopa(mod):
+def test_config2_full_size_rsplus(mod):
+    D, H = 4096, 14336
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=1)
+    gate, w = make_std(D, H, torch.bfloat16, 2, 0.9)
+    x = syn.tokens(1, D, torch.bfloat16, 7, DEV)[0]
+    run_both_paths(mod, ffn, x, gate, w, "rsplus", ("general", "fused"), what="config2 R-S+")
+
+
+@pytest.mark.parametrize("r", [256, 512, 1024])
+@pytest.mark.parametrize("act", ["relu", "sqrelu"])
+def test_config3_full_size_lopa(mod, r, act):
     D, H = 4096, 14336
     ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=1024, B_max=1)
-    for r, act in ((512, "relu"), (1024, "sqrelu"), (256, "relu")):
-        gate, w = make_lopa(mod, D, H, r, torch.bfloat16, 3, 0.9, "diag")
-        x = syn.tokens(1, D, torch.bfloat16, 3, DEV)[0]
-        ref = run_both_paths(mod, ffn, x, gate, w, act, ("general", "fused"), what=f"config3 r={r}")
-        assert abs(1 - ref["n_act"][0] / H - 0.9) < 0.03
-        del gate, w
+    gate, w = make_lopa(mod, D, H, r, torch.bfloat16, 3, 0.9, "diag")
+    x = syn.tokens(1, D, torch.bfloat16, 3, DEV)[0]
+    ref = run_both_paths(mod, ffn, x, gate, w, act, ("general", "fused"), what=f"config3 r={r} {act}")
+    assert abs(1 - ref["n_act"][0] / H - 0.9) < 0.03
 
 
 @pytest.mark.parametrize("B", [4, 16, 64])
@@ -433,23 +459,39 @@ def test_config4_full_size_batched_zipf(mod, B):
     assert abs(frac - syn.expected_union_fraction(p, B)) < 0.05
 
 
-def test_config5_full_size_stress_layer0(mod):
+@pytest.mark.parametrize("s", [0.9, 0.8, 0.95])
+def test_config5_full_size_stress_layer0(mod, s):
+    """8192 x 28672, squared RELU, standard and LoPA r = 1024 gates, one token and a batch of eight (the batch:
+    the tcgen05 gate GEMM with K = 8192 and several 128-row tiles per CTA, gather4 over the union)."""
     D, H = 8192, 28672
-    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=1024, B_max=1)
-    gate, w = make_std(D, H, torch.bfloat16, 5, 0.9)
-    x = syn.tokens(1, D, torch.bfloat16, 5, DEV)[0]
-    run_both_paths(mod, ffn, x, gate, w, "sqrelu", ("general", "fused"), what="config5 standard")
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=1024, B_max=8)
+    gate, w = make_std(D, H, torch.bfloat16, 5, s)
+    x8 = syn.tokens(8, D, torch.bfloat16, 5, DEV, extra=1)
+    ntok = 8 if s == 0.9 else 2                     # the other sparsities: two tokens of the batch are checked
+    ref = run_oracle(x8[:ntok], gate, w["b_g"], w["W_up"], w["W_down"], "sqrelu", threads=16)
+    assert abs(1 - ref["n_act"].mean() / H - s) < 0.03
+    for path in ("general", "fused") if s == 0.9 else ("fused",):
+        ffn.set_path(path)
+        y = ffn.sparse_ffn_forward(x8[0], gate, w["b_g"], w["W_up"], w["W_down"], "sqrelu")
+        one = dict(y=ref["y"][0], z=ref["z"][0])
+        assert_y_close(y, one["y"], what=f"config5 standard s={s} [{path}]")
+        assert_active_set(ffn.last_active(), one, what=f"config5 standard s={s} [{path}]")
+    ffn.set_path("auto")
+    y = ffn.sparse_ffn_forward(x8[:ntok], gate, w["b_g"], w["W_up"], w["W_down"], "sqrelu")
+    assert_y_close(y, ref["y"], what=f"config5 standard s={s} B={ntok}")
+    assert_active_set(ffn.last_active(), ref, what=f"config5 standard s={s} B={ntok}")
+    if s != 0.9:
+        return
     del gate["W_g"], w["W_g"]
     lg, lw = make_lopa(mod, D, H, 1024, torch.bfloat16, 5, 0.9, "diag")
     lw["W_up"], lw["W_down"] = w["W_up"], w["W_down"]
-    run_both_paths(mod, ffn, x, lg, lw, "sqrelu", ("general", "fused"), what="config5 lopa")
-    ffn8 = mod.SparseFFN(D, H, torch.bfloat16, r_max=1024, B_max=8)          # config 5, batch 8
-    x8 = syn.tokens(8, D, torch.bfloat16, 5, DEV, extra=1)
-    for gt, ww in ((lg, lw),):
-        ref = run_oracle(x8, gt, ww["b_g"], ww["W_up"], ww["W_down"], "sqrelu", threads=8)
-        y = ffn8.sparse_ffn_forward(x8, gt, ww["b_g"], ww["W_up"], ww["W_down"], "sqrelu")
-        assert_y_close(y, ref["y"], what="config5 lopa B=8")
-        assert_active_set(ffn8.last_active(), ref, what="config5 lopa B=8")
+    run_both_paths(mod, ffn, x8[0], lg, lw, "sqrelu", ("general", "fused"), what="config5 lopa")
+    ref = run_oracle(x8, lg, lw["b_g"], lw["W_up"], lw["W_down"], "sqrelu", threads=16)
+    y = ffn.sparse_ffn_forward(x8, lg, lw["b_g"], lw["W_up"], lw["W_down"], "sqrelu")
+    assert_y_close(y, ref["y"], what="config5 lopa B=8")
+    assert_active_set(ffn.last_active(), ref, what="config5 lopa B=8")
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
 
 
 def test_two_handles_on_two_streams_overlap_and_agree(mod):

@@ -14,7 +14,7 @@ ROOT = Path(__file__).resolve().parent.parent
 def declared_functions():
     text = (ROOT / "include" / "sparse_ffn.h").read_text()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(?:int|const char\*)\s+(\w+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(?:int|void|const char\*)\s+(\w+)\s*\(", text)))
 
 
 def test_library_builds_and_exports_every_declared_symbol():

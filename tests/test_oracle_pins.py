@@ -74,6 +74,13 @@ def test_activation_table(golden):
         assert oracle.activation("rsplus", x) == 0.0 and oracle.activation("relu", x) == 0.0
     assert oracle.activation("relu", -0.0) == 0.0
     assert oracle.activation("sqrelu", 1e-200) == 0.0   # z*z underflows; activity is decided on z
+    # SILU: x * sigmoid(x) on both sides; odd part is x / 2 (silu(x) - silu(-x) = x), minimum near x = -1.2785
+    for x in np.linspace(-6.0, 6.0, 49):
+        assert oracle.activation("silu", x) == pytest.approx(x / (1 + math.exp(-x)), rel=1e-15, abs=1e-300)
+        assert oracle.activation("silu", x) - oracle.activation("silu", -x) == pytest.approx(x, abs=1e-14)
+        if x >= 0:
+            assert oracle.activation("silu", x) == oracle.activation("rsplus", x)
+    assert oracle.activation("silu", -1.2785) == pytest.approx(-0.27846, abs=1e-5)
 
 
 def test_bf16_inputs_decode_exactly():
@@ -326,6 +333,14 @@ def test_hand_worked_double_activation():
         # A_3 = R-S+: A_3(1) = sigmoid(1) = 1 / (1 + e^-1)
         out = oracle.ffn(x, W3, Wd, "relu", W_g=W1, route=route, act_up="rsplus")
         np.testing.assert_allclose(out["y"], [1.0 / (1.0 + math.exp(-1.0))] * 2, rtol=1e-15)
+        # A_3 = SILU (the uncast activation of the up branch): A_3(u) = [sigmoid(1), 6 sigmoid(6), -0.5 sigmoid(-0.5)];
+        # h = [sigmoid(1), 0, -1.5 sigmoid(-0.5)];  y = h_0 [1, 1] + h_2 [2, -2];  both fired neurons keep h != 0
+        out = oracle.ffn(x, W3, Wd, "relu", W_g=W1, route=route, act_up="silu")
+        h0, h2 = 1.0 / (1.0 + math.exp(-1.0)), -1.5 / (1.0 + math.exp(0.5))
+        np.testing.assert_allclose(out["y"], [h0 + 2 * h2, h0 - 2 * h2], rtol=1e-15)
+        assert out["n_act"][0] == 2 and out["n_gated"][0] == 2
+    with pytest.raises(ValueError):          # SILU is not sparse: it cannot be the gate's activation
+        oracle.ffn(x, W3, Wd, "silu", W_g=W1)
 
 
 def test_double_activation_special_cases():
@@ -343,7 +358,7 @@ def test_double_activation_special_cases():
     np.testing.assert_array_equal(neg["n_act"], single["n_act"])          # the gate is untouched
     # skipping rows never changes y, and the gated set is a subset of the active set
     W3 = RNG.standard_normal((H, D)).astype(np.float32)
-    for a3 in ("relu", "sqrelu", "rsplus"):
+    for a3 in ("relu", "sqrelu", "rsplus", "silu"):
         dense = oracle.ffn(x, W3, Wd, "sqrelu", W_g=W1, route="dense", act_up=a3)
         sparse = oracle.ffn(x, W3, Wd, "sqrelu", W_g=W1, route="sparse", act_up=a3)
         np.testing.assert_array_equal(dense["y"], sparse["y"])
@@ -353,7 +368,7 @@ def test_double_activation_special_cases():
         u = x.astype(np.float64) @ W3.astype(np.float64).T
         a = np.maximum(z, 0.0) ** 2
         g = {"relu": np.maximum(u, 0.0), "sqrelu": np.maximum(u, 0.0) ** 2,
-             "rsplus": np.where(u >= 0, u / (1.0 + np.exp(-u)), 0.0)}[a3]
+             "rsplus": np.where(u >= 0, u / (1.0 + np.exp(-u)), 0.0), "silu": u / (1.0 + np.exp(-u))}[a3]
         np.testing.assert_allclose(sparse["y"], (a * g) @ Wd.astype(np.float64), rtol=1e-12, atol=1e-12)
 
 
