@@ -31,26 +31,55 @@ sys.path.insert(0, str(ROOT))
 import torch  # noqa: E402
 
 import synthetic_inputs as syn  # noqa: E402
+from bench_report import measured_hbm_peak  # noqa: E402
 
 D_MODEL, D_FF, SPARSITY, ACT = 4096, 14336, 0.9, "relu"
 CALLS_PER_STEP = 1000
 WEIGHT_SETS = 4
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the main kernel at this workload, from the ncu
-# capture summarised in profiles/fused_ffn_kernel_decode_4096x14336_s090.md (140.9 MB read + 5.1 MB written)
-NCU_DRAM_TRAFFIC_PER_LAUNCH = 146.0e6
-FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the main kernel at this workload: kept beside the
+# ncu summary it comes from and rewritten whenever that summary is refreshed
+NCU_TRAFFIC_FILE = ROOT / "profiles" / "fused_tc_kernel_decode_4096x14336_s090.json"
 WORKLOAD = "llama-style standard-gated FFN decode, d_model=4096 d_ff=14336 bf16 batch=1 RELU, sparsity 0.9"
 
 
-def measured_hbm_peak():
-    p = ROOT / "MEASURED_PEAKS.json"
-    if p.exists():
-        try:
-            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
-        except Exception:
-            pass
-    return FALLBACK_HBM_GBS, "fallback"
+def ncu_traffic_per_launch():
+    """DRAM bytes per launch of the dominant kernel from the kept ncu summary, or None if there is none."""
+    try:
+        return float(json.loads(NCU_TRAFFIC_FILE.read_text())["dram_bytes_per_launch"])
+    except Exception:
+        return None
+
+
+def extra_points(m, dev):
+    """Headline points of the other configurations (LoPA gate, batched decode, the 8192 x 28672 shape), short runs
+    of the measurement matrix's own routine, so that a default bench run observes them too."""
+    import bench_report as rep
+
+    D, H = D_MODEL, D_FF
+    base = [syn.standard_ffn(D, H, torch.bfloat16, 2, dev, sparsity=0.9, extra=i) for i in range(WEIGHT_SETS)]
+    std = lambda w: {"W_g": w["W_g"]}  # noqa: E731
+    rows = []
+    gi = m.g_diagonal(H, D, dev)
+    lsets = []
+    for i, w in enumerate(base):
+        lw = syn.lopa_ffn(D, H, 512, torch.bfloat16, 3, dev, sparsity=0.9, extra=i)
+        lw["W_up"], lw["W_down"] = w["W_up"], w["W_down"]
+        lsets.append(lw)
+    lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}  # noqa: E731
+    rows.append(rep.measure("lopa r=512 relu", D, H, 1, lsets, lg, "relu", r=512, n_calls=120))
+    del lsets
+    p = syn.zipf_firing_profile(H, 1.1, 0.1, 0.99, seed=4)
+    zb = syn.bias_from_firing_profile(p).to(dev)
+    rows.append(rep.measure("batched zipf B=16", D, H, 16, [dict(w, b_g=zb) for w in base], std, "relu", n_calls=80))
+    del base
+    torch.cuda.empty_cache()
+    D, H = 8192, 28672
+    layers = [syn.standard_ffn(D, H, torch.bfloat16, 5, dev, sparsity=0.9, extra=i) for i in range(4)]
+    rows.append(rep.measure("stress 8192x28672 s=0.9 B=1", D, H, 1, layers, std, "sqrelu", n_calls=48))
+    keep = ("name", "B", "fired_rows", "us_per_call", "touched_mb", "gbs", "frac_measured_peak", "dense_us",
+            "speedup_vs_dense", "device_status")
+    return [{k: r[k] for k in keep} for r in rows]
 
 
 class ClockSampler:
@@ -281,7 +310,7 @@ def run_ours(args, rank, world, local):
     line = {
         "metric": "us_per_ffn_call", "value": us_call / world, "unit": "us/FFN-call", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": False,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "step": f"{args.calls} single-token FFN calls, one token each",
                    "l2": f"rotating over {WEIGHT_SETS} independent weight sets ({WEIGHT_SETS * dense_bytes / 1e9:.2f} GB) "
                          "so inputs exceed L2", "storage": "bf16 weights and tokens, fp32 accumulation and output",
@@ -292,13 +321,15 @@ def run_ours(args, rank, world, local):
         "dense_us_per_call": us_dense, "dense_gbs": dense_bytes / (us_dense * 1e-6) / 1e9,
         "speedup_vs_dense": us_dense / us_call,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"{peak_kind} copy bandwidth", "traffic": NCU_DRAM_TRAFFIC_PER_LAUNCH,
+                     "peak_kind": f"{peak_kind} copy bandwidth", "traffic": ncu_traffic_per_launch(),
                      "algorithmic_bytes_per_launch": bytes_per_call,
-                     "kernel": "fused_ffn_kernel (one launch per FFN call; the cross-CTA sum runs in its last CTAs)"},
+                     "kernel": "fused_tc_kernel (one launch per FFN call: gate on tcgen05, rows of fired neurons, "
+                               "cross-CTA sum in the first CTAs to finish)"},
         "e2e": {"value": us_e2e / world, "unit": "us/FFN-call", "h2d_bytes_per_step": args.calls * D_MODEL * 2,
                 "d2h_bytes_per_step": args.calls * D_MODEL * 4},
         "gpu_launches": launches, "clocks": clk.summary(),
         "cpu_baseline": cpu_baseline() if world == 1 else None,
+        "extra": extra_points(m, dev) if world == 1 and not args.no_extra else None,
     }
     print(json.dumps(line))
 
@@ -314,6 +345,7 @@ def main():
     ap.add_argument("--only", default=None, help="with --report: only the cases whose name contains this")
     ap.add_argument("--report-calls", type=int, default=None, help="with --report: calls per case")
     ap.add_argument("--calls", type=int, default=CALLS_PER_STEP, help="FFN calls (tokens) per step")
+    ap.add_argument("--no-extra", action="store_true", help="leave out the other configurations' headline points")
     ap.add_argument("--skip-extras", action="store_true",
                     help="time the sparse path only (no dense comparator, host-buffer or CPU legs): for profiler runs")
     args = ap.parse_args()
@@ -323,7 +355,7 @@ def main():
         if args.impl == "reference":
             run_reference(args, rank)
         elif args.report:
-            from paper_2609_31975_b200 import report
+            import bench_report as report
 
             if rank == 0:
                 report.run(args.report, quick=args.quick, only=args.only, n_calls=args.report_calls)

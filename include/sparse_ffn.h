@@ -143,8 +143,8 @@ int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate
                       const float* b_g, const void* W_up, const void* W_down, int act, float* y,
                       void* stream);
 
-/* Weight-only int8 (the paper's appendix on quantisation-aware training: "weights are converted to int8 at
- * inference", tokens and all arithmetic stay in floating point).  The paper does not fix the format; here every
+/* Weight-only int8 (the paper's appendix on quantisation-aware training: only the weights become int8, at inference
+ * time; tokens and all arithmetic stay in floating point).  The paper does not fix the format; here every
  * weight matrix is stored as int8 codes, row-major, with one fp32 scale per row:
  *     W[j, k] = s[j] * q[j, k],   q in [-127, 127].
  * In these two calls the pointers W_up, W_down and, inside `gate`, W_g (STANDARD) or V and U (LOPA) address the

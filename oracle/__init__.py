@@ -190,7 +190,7 @@ def ffn(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, b_g=None, route="sp
 
 def dequantize_rows(q, scale) -> np.ndarray:
     """The matrix int8 codes stand for under weight-only quantisation with one scale per row (appendix on
-    quantisation-aware training: "weights are converted to int8 at inference"; the paper does not fix the
+    quantisation-aware training: only the weights are turned into int8, at inference time; the paper does not fix the
     granularity, one fp32 scale per output row is the reading taken here): W[j, k] = scale[j] * q[j, k], as float64."""
     if not isinstance(q, np.ndarray):
         q = q.detach().cpu().numpy()

@@ -411,8 +411,10 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
 
   const bool lopa = g->kind == SFFN_GATE_LOPA;
   if (lopa) {
+    const int v_nb_max = (size_t)4 * D * 4 <= 227 * 1024 ? 4 : (size_t)2 * D * 4 <= 227 * 1024 ? 2 : 1;
     for (int b0 = 0; b0 < B;) {
-      const int nb = B - b0 >= 4 ? 4 : B - b0 >= 2 ? 2 : 1;
+      int nb = B - b0 >= 4 ? 4 : B - b0 >= 2 ? 2 : 1;
+      nb = nb > v_nb_max ? v_nb_max : nb;
       RowDotParams p{};
       p.W = g->V; p.R = g->r; p.K = D;
       p.vec = xb + (size_t)b0 * D * esz; p.vec_stride = D;
@@ -427,8 +429,12 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       ++h->launches;
     }
   }
+  const int gate_k = lopa ? g->r : D;
+  // the gate kernel stages its tokens as fp32 in shared memory: nb * K * 4 bytes must fit (two tokens above 14.5k)
+  const int gate_nb_max = (size_t)4 * gate_k * 4 <= 227 * 1024 ? 4 : (size_t)2 * gate_k * 4 <= 227 * 1024 ? 2 : 1;
   for (int b0 = 0; b0 < B;) {
-    const int nb = B - b0 >= 4 ? 4 : B - b0 >= 2 ? 2 : 1;
+    int nb = B - b0 >= 4 ? 4 : B - b0 >= 2 ? 2 : 1;
+    nb = nb > gate_nb_max ? gate_nb_max : nb;
     RowDotParams p{};
     if (lopa) {
       p.W = g->U; p.R = H; p.K = g->r;

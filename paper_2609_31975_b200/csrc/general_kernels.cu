@@ -408,11 +408,17 @@ static cudaError_t launch_rowdot_t(const RowDotParams& p, bool gate, int grid, c
   const size_t smem = (size_t)NB * p.K * sizeof(float);
   if (gate) {
     auto k = rowdot_kernel<T, VT, NB, true>;
-    if (smem > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (smem > 48 * 1024) {
+      const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
     return launch_pdl(k, dim3(grid), dim3(256), smem, s, p);
   } else {
     auto k = rowdot_kernel<T, VT, NB, false>;
-    if (smem > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (smem > 48 * 1024) {
+      const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
     return launch_pdl(k, dim3(grid), dim3(256), smem, s, p);
   }
 }
@@ -454,7 +460,10 @@ template <typename T, int NB, int CPT>
 static cudaError_t launch_updown_t(const UpDownParams& p, int grid, cudaStream_t s) {
   const size_t smem = (size_t)NB * p.D * sizeof(float);
   auto k = updown_kernel<T, NB, CPT>;
-  if (smem > 48 * 1024) cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (smem > 48 * 1024) {
+    const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
   return launch_pdl(k, dim3(grid), dim3(512), smem, s, p);
 }
 

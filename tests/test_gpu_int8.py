@@ -187,6 +187,16 @@ def test_int8_wide_rows(mod, D, H):
         assert e.value.code == 2
 
 
+def test_int8_widest_rows_batch_of_four(mod):
+    """16384 codes per row: the gate kernel stages its tokens as fp32 in shared memory and takes two tokens per pass
+    there (four would need 256 KB)."""
+    D, H = 16384, 160
+    gate, w = make_std(D, H, 18, 0.8)
+    x = syn.tokens(4, D, torch.bfloat16, 18, DEV)
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=4)
+    check(mod, ffn, x, gate, w, "relu", ("auto",), "q8 wide 16384 B=4")
+
+
 def test_int8_full_size_decode_and_lopa(mod):
     D, H = 4096, 14336
     ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=512, B_max=4)

@@ -106,6 +106,16 @@ def test_wide_rows(mod, D, H, dtype):
     assert ffn.device_status() == 0
 
 
+def test_widest_rows_batch_of_four_on_the_cuda_core_path(mod):
+    """16384 bf16 elements per row: the CUDA-core gate kernel stages its tokens as fp32 in shared memory and takes
+    two tokens per pass there (four would need 256 KB)."""
+    D, H = 16384, 96
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=4)
+    gate, w = make_std(D, H, torch.bfloat16, 25, 0.8)
+    x = syn.tokens(4, D, torch.bfloat16, 25, DEV)
+    run_both_paths(mod, ffn, x, gate, w, "relu", ("general",), what="wide 16384 B=4")
+
+
 @pytest.mark.parametrize("r,fixed,sign,gain,rms", [
     (64, "diag", False, False, True), (128, "tiled", True, True, True),
     (96, None, False, False, False), (256, "diag", True, False, False)])
