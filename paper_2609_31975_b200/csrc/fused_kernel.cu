@@ -78,7 +78,8 @@ struct FusedParams {
   const float* s_V;
   const float* s_up;
   const float* s_down;
-  float* partial;  // [grid][D]
+  unsigned long long* partial;  // [grid][row] per-CTA partials of y, each value paired with the call's number
+  uint32_t* epoch_word;         // number of calls completed on this workspace
   uint8_t* flag;
   int32_t* status;
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
@@ -240,6 +241,24 @@ __device__ __forceinline__ float2 chunk_dot_q8(const uint4& w, const float* vec,
     acc = fma2(hi, make_float2(v.z, v.w), acc);
   }
   return acc;
+}
+
+// One value of a partial with the number of the call that wrote it: a naturally aligned 64-bit word is written and
+// read as a whole, so a reader that finds the expected number has the value that belongs to it (no fence, no flag
+// round trip between writer and reader).
+__device__ __forceinline__ unsigned long long tagged(float v, uint32_t epoch) {
+  return ((unsigned long long)epoch << 32) | (unsigned long long)__float_as_uint(v);
+}
+__device__ __forceinline__ void st_tagged2(unsigned long long* dst, unsigned long long a, unsigned long long b, uint64_t pol) {
+  asm volatile("st.global.cg.L2::cache_hint.v2.b64 [%0], {%1, %2}, %3;" ::"l"(dst), "l"(a), "l"(b), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void ld_tagged2(const unsigned long long* src, unsigned long long& a, unsigned long long& b) {
+  asm volatile("ld.global.cg.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(src) : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
 }
 
 #ifdef SFFN_TRACE
@@ -417,6 +436,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   // ---- everyone else: wait for the predecessor in the stream, then stage the token ------------
   pdl_wait();
   if (tid == kStageBase) SFFN_GSTAMP(11);
+  const uint32_t ep = warp >= kFirstGateWarp ? __ldcg(p.epoch_word) + 1u : 0u;  // this call's number (tags of the partials)
   for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) row_state[i] = 0xffffffffu;
   constexpr int XEPV = Elem<X>::kPerVec;  // token elements per 16 bytes (the weights' EPV unless those are int8)
   for (int cx = tid - kStageBase; cx < D / XEPV; cx += kStageThreads) {
@@ -542,7 +562,22 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       if (ap == 0) slot_a[slot] = -1.f;      // stop marker: a negative gate value
       mbar_arrive(full_act + 8 * slot);      // completes the phase without data
     }
-    if (lane == 0 && ap == 0) SFFN_STAMP(2);
+    if (ap == 0) {
+      // This CTA's place in the order of finishing (the first R sum the partials), taken now so that the round trip
+      // overlaps with the act warps' last rows; -1 under the test hook that makes a CTA go missing.
+      if (lane == 0) {
+        SFFN_STAMP(2);
+        int rank = -1;
+        if (cta != p.skip_arrival_cta) {
+          unsigned long long old;
+          asm volatile("atom.add.relaxed.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(p.done_counter) : "memory");
+          rank = (int)(old - old / G * G);
+        }
+        ctl[kRank] = rank;
+      }
+      __syncwarp();
+      asm volatile("bar.arrive 6, %0;" ::"r"(32 * (kGW + kAW) + 32) : "memory");
+    }
     __syncwarp();
   } else if (warp < kFAW) {
     // ======================= gate warps ========================================================
@@ -791,99 +826,112 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       par = slot1 + 1 == NA ? par1 ^ 1 : par1;
     }
     if (at == 0) SFFN_STAMP(4);
-    // this CTA's partial of y
-    float* dst = p.partial + (size_t)cta * D;
+    // This CTA's partial of y, every value tagged with the call's number.  Stored unit (two columns, 16 bytes)
+    // (i * EPV / 2 + e) * kAT + at holds columns EPV (at + i kAT) + 2 e and the next one: a warp's store is 512
+    // contiguous bytes; the summing threads undo the permutation when they write y.
+    if (cta != p.skip_arrival_cta) {
+      const uint64_t keep = policy_evict_last();  // the partials are rewritten by every call: they should stay in L2
+      unsigned long long* dst = p.partial + (size_t)cta * (CPT * EPV * kAT);
 #pragma unroll
-    for (int i = 0; i < CPT; ++i) {
-      const int c = at + i * kAT;
-      if (c < nvecD) {
+      for (int i = 0; i < CPT; ++i) {
+        if (at + i * kAT < nvecD) {
 #pragma unroll
-        for (int e = 0; e < EPV; e += 4)
-          __stcg(reinterpret_cast<float4*>(dst + (size_t)c * EPV + e),
-                 make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]));
+          for (int e = 0; e < EPV / 2; ++e)
+            st_tagged2(dst + 2 * (size_t)((i * (EPV / 2) + e) * kAT + at), tagged(acc[i][2 * e], ep),
+                       tagged(acc[i][2 * e + 1], ep), keep);
+        }
       }
     }
     if (at == 0) SFFN_STAMP(5);
     if (at == 0) SFFN_GSTAMP(12);
   }
 
-  // ---- y = sum over CTAs of their partials, by the last CTAs to finish -------------------------------------------
-  // A CTA that finishes among the last R of its call stays, waits (bounded) until every CTA has arrived and sums one
-  // slice of the columns over all partials in CTA order: which CTA does a slice depends on timing, what it computes
-  // does not, so y is bitwise the same on every run.  Earlier CTAs leave at once and their SMs take the next kernel
-  // of the stream.
+  // ---- y = sum over CTAs of their partials, by the first CTAs to finish ------------------------------------------
+  // The first R CTAs of a call to finish stay and each sums one slice of the columns over all partials in a fixed order
+  // (which CTA does a slice depends on timing, what it computes does not: y is bitwise the same on every run).  They
+  // have time to spare until the slowest CTA is done and fetch the partials that are already there meanwhile.  A
+  // summing CTA does not wait for a count or a flag: it reads the other CTAs' tagged values and re-reads those that
+  // still carry an older call's number (bounded).  Thread (u, rg) takes two columns (one 16-byte unit) in the rows
+  // rg, rg + RG, ...; the RG row groups are then added in order through shared memory.  The other CTAs leave at once
+  // and their SMs take the next kernel of the stream.
   if (warp < kFirstGateWarp) return;  // act producers (the gate producers left long ago)
   constexpr int kTail = 32 * (kGW + kAW);
-  const int tw = warp - kFirstGateWarp;
-  const int Q = D / 4;
-  // reducers: 16 float4 columns each where the grid allows, but never more than half the grid, so that the waiting
-  // CTAs of two calls that overlap (two handles on two streams) cannot hold every SM between them
-  const int R = min(max(1, (G - 1) / 2), max(1, Q / 16));
-  named_bar_sync(6, kTail);
-  if (tid == 32 * kFirstGateWarp) {
-    SFFN_GSTAMP(6);
-    // Release at device scope after the CTA barrier: the act threads' partial stores happen before it, so a CTA that
-    // acquires the counter's final value sees every partial.
-    unsigned long long old;
-    if (cta == p.skip_arrival_cta)  // test hook: the count never completes and the summing CTAs give up
-      asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(old) : "l"(p.done_counter) : "memory");
-    else
-      asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(p.done_counter) : "memory");
-    const unsigned long long first = old / G * G;
-    const int rank = (int)(old - first);
-    ctl[kRank] = rank;
-    SFFN_GSTAMP(7);
-    if (rank >= G - R) {
-      const long long t0 = clock64();
-      for (;;) {
-        unsigned long long seen;
-        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.done_counter) : "memory");
-        if (seen >= first + G || ctl[kAbort]) break;
-        if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status); break; }
-        __nanosleep(20);
-      }
-      SFFN_GSTAMP(8);
-    }
-  }
-  named_bar_sync(6, kTail);
-  const int slice = ctl[kRank] - (G - R);
+  constexpr int kRow = CPT * EPV * kAT;        // values of a stored partial
+  constexpr int kUnits = kRow / 2;             // two columns each (a multiple of 32; those past D are never written)
+  const int tt = tid - 32 * kFirstGateWarp;    // index among the tail threads
+  // never more than half the grid stays, so that the waiting CTAs of two calls that overlap (two handles on two
+  // streams) cannot hold every SM between them
+  const int R = min(max(1, (G - 1) / 2), max(1, kUnits / 32));
+  named_bar_sync(6, kTail + 32);  // + the act producer that took the rank
+  const int rank = ctl[kRank];
+  const int slice = rank >= 0 && rank < R ? rank : -1;
+  if (rank == G - 1 && tt == 0 && !ctl[kAbort]) *p.epoch_word = ep;  // every CTA has its number: the next call tags with ep + 1
   if (slice < 0 || ctl[kAbort]) return;
+  if (tt == 0) SFFN_GSTAMP(8);
+  constexpr int kBatch = 13;
   const int32_t failed = __ldcg(p.status);  // in flight together with the partials, not after them
-  const int cols = (Q + R - 1) / R;
-  const int q_hi = min(Q, (slice + 1) * cols);
-  // Four warps, one group of four columns each.  Lane (r8, c4) reads column c4 of its group in the rows r8, r8 + 8,
-  // ...: one warp load covers eight rows x 64 contiguous bytes (whole 32-byte sectors), twenty loads are in flight per
-  // lane (160 CTAs; more take another pass), the eight row residues are combined by shuffles in a fixed order.
-  const int r8 = lane >> 2, c4 = lane & 3;
-  if (tw >= 4) return;
-  for (int c0 = slice * cols; c0 < q_hi; c0 += 16) {
-    const int q = c0 + 4 * tw + c4;
-    float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (q < q_hi) {
-      const float4* src = reinterpret_cast<const float4*>(p.partial) + q;
-      for (int i0 = 0; 8 * i0 < G; i0 += 20) {
-        float4 v[20];
+  float2* comb = reinterpret_cast<float2*>(gate_ring);  // the rings are idle by now
+  const int U = (kUnits + R - 1) / R;
+  const int UW = U <= 32 ? 32 : U <= 64 ? 64 : 128;
+  const int RG = kTail / UW;
+  const int u = tt % UW, rg = tt / UW;
+  auto first_column = [&](int unit) {  // undoes the permutation of the stored units
+    return EPV * ((unit % kAT) + (unit / ((EPV / 2) * kAT)) * kAT) + 2 * ((unit / kAT) % (EPV / 2));
+  };
+  bool ok = true;
+  for (int u0 = 0; u0 < U; u0 += UW) {
+    const int unit = slice * U + u0 + u;
+    float2 sum = make_float2(0.f, 0.f);
+    if (u0 + u < U && unit < kUnits && first_column(unit) < D) {
+      const unsigned long long* src = p.partial + 2 * (size_t)unit;
+      for (int g0 = rg; ok && g0 < G; g0 += RG * kBatch) {
+        unsigned long long a[kBatch], b[kBatch];
 #pragma unroll
-        for (int i = 0; i < 20; ++i) {
-          const int g = 8 * (i0 + i) + r8;
-          v[i] = g < G ? __ldcg(src + (size_t)g * Q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k = 0; k < kBatch; ++k) {
+          const int g = g0 + k * RG;
+          a[k] = b[k] = (unsigned long long)ep << 32;  // rows past the grid: zero, already "there"
+          if (g < G) ld_tagged2(src + (size_t)g * kRow, a[k], b[k]);
+        }
+        long long t0 = 0;
+        for (;;) {
+          bool all = true;
+#pragma unroll
+          for (int k = 0; k < kBatch; ++k) {
+            if ((uint32_t)(a[k] >> 32) != ep || (uint32_t)(b[k] >> 32) != ep) {
+              all = false;
+              ld_tagged2(src + (size_t)(g0 + k * RG) * kRow, a[k], b[k]);
+            }
+          }
+          if (all) break;
+          if (t0 == 0) t0 = clock64();
+          if (ctl[kAbort]) { ok = false; break; }
+          if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status); ok = false; break; }
+          __nanosleep(20);
         }
 #pragma unroll
-        for (int i = 0; i < 20; ++i) {
-          s4.x += v[i].x; s4.y += v[i].y; s4.z += v[i].z; s4.w += v[i].w;
+        for (int k = 0; k < kBatch; ++k) {
+          sum.x += __uint_as_float((uint32_t)a[k]);
+          sum.y += __uint_as_float((uint32_t)b[k]);
         }
       }
     }
-#pragma unroll
-    for (int o = 4; o < 32; o <<= 1) {  // the eight row residues of a column sit in lanes c4 + 4 r8
-      s4.x += __shfl_xor_sync(0xffffffffu, s4.x, o);
-      s4.y += __shfl_xor_sync(0xffffffffu, s4.y, o);
-      s4.z += __shfl_xor_sync(0xffffffffu, s4.z, o);
-      s4.w += __shfl_xor_sync(0xffffffffu, s4.w, o);
+    comb[rg * UW + u] = sum;
+    named_bar_sync(7, kTail);
+    if (tt < UW) {
+      const int unit2 = slice * U + u0 + tt;
+      const int col2 = first_column(unit2);
+      if (u0 + tt < U && unit2 < kUnits && col2 < D) {
+        float2 t = make_float2(0.f, 0.f);
+        for (int r = 0; r < RG; ++r) {
+          t.x += comb[r * UW + tt].x;
+          t.y += comb[r * UW + tt].y;
+        }
+        if (!ctl[kAbort] && failed == 0) *reinterpret_cast<float2*>(p.y + col2) = t;
+      }
     }
-    if (r8 == 0 && q < q_hi && failed == 0) reinterpret_cast<float4*>(p.y)[q] = s4;
+    named_bar_sync(7, kTail);
   }
-  if (tid == 32 * kFirstGateWarp) SFFN_GSTAMP(13);
+  if (tt == 0) SFFN_GSTAMP(13);
 }
 
 // ---- host side --------------------------------------------------------------------------------
@@ -1000,8 +1048,8 @@ size_t fused_tagged_partials_offset(int D, int r_max) {
 }
 size_t fused_workspace_bytes(int D, int H, int r_max) {
   (void)H;
-  // a row of tagged partials is padded to 2048, 4096, 8192 or 16384 values (whole chunks per act thread)
-  size_t row = 2048;
+  // a row of tagged partials is padded to 4096, 8192 or 16384 values (whole chunks per act thread of either kernel)
+  size_t row = 4096;
   while (row < (size_t)D) row *= 2;
   return fused_tagged_partials_offset(D, r_max) + (size_t)kMaxGrid * row * 8 + 256;
 }
@@ -1033,7 +1081,6 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   const Geometry g = plan(c.wkind, c.D, c.H, K, lopa, grid);
   if (!g.ok) return cudaErrorInvalidValue;
   char* ws = static_cast<char*>(c.workspace);
-  float* partial = reinterpret_cast<float*>(ws + 256);
   float* vbuf = reinterpret_cast<float*>(ws + 256 + (size_t)kMaxGrid * c.D * 4);
   int n = 0;
   cudaError_t e;
@@ -1048,7 +1095,8 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.v_counter = reinterpret_cast<unsigned long long*>(ws);
   p.done_counter = p.v_counter + 1;
   p.y = c.y;
-  p.partial = partial;
+  p.partial = reinterpret_cast<unsigned long long*>(ws + fused_tagged_partials_offset(c.D, c.r_max));
+  p.epoch_word = reinterpret_cast<uint32_t*>(ws + 16);
   p.act = c.act; p.dense = c.dense ? 1 : 0;
   p.act_up = c.act_up;
   p.s_gate = c.s_gate; p.s_V = c.s_V; p.s_up = c.s_up; p.s_down = c.s_down;
