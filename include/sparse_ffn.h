@@ -109,7 +109,7 @@ int sffn_workspace_bytes(int D, int H, int r_max, int B_max, int dtype, size_t* 
 
 /* Creates a handle on the current device.  `workspace` is device memory of at least
  * sffn_workspace_bytes(...) bytes, 256-byte aligned, owned by the caller and kept alive (and not
- * shared with another handle) until sffn_destroy.  The call clears the workspace (synchronously).
+ * shared with another handle) until sffn_destroy.  The call clears the workspace and returns when that is done.
  * Calls on one handle must be issued to one stream at a time. */
 int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dtype,
                 void* workspace, size_t workspace_bytes);
@@ -118,6 +118,16 @@ int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dt
 int sffn_destroy(sffn_handle* handle);
 
 int sffn_set_path(sffn_handle* handle, int path /* sffn_path */);
+
+/* Where a single-token call (B = 1, fused path) computes the gate.  Both engines give the result of Eq. 1 and stream
+ * the same bytes; they differ in what the SMs' issue slots are spent on.  CUDA_CORE: fp32 FMAs on bf16 / fp32 / int8
+ * rows, any gate.  TENSOR_CORE: tcgen05 MMAs, which leaves the issue slots to the up / down stage -- bf16 rows,
+ * standard gate, D a multiple of 64 and at least 1024; a call it does not cover runs on the CUDA cores.  AUTO (the
+ * default) takes the CUDA cores for sparse calls, where at the paper's sparsity levels (0.8 and up) the gate stream
+ * alone sets the time, and the tensor cores for dense calls; a caller whose models fire more than about a fifth of
+ * their neurons sets TENSOR_CORE. */
+typedef enum { SFFN_GATE_ENGINE_AUTO = 0, SFFN_GATE_ENGINE_CUDA_CORE = 1, SFFN_GATE_ENGINE_TENSOR_CORE = 2 } sffn_gate_engine;
+int sffn_set_gate_engine(sffn_handle* handle, int engine /* sffn_gate_engine */);
 
 /* Double activation (Sec. 3.3, "Double activation"): with act_up = RELU / SQRELU / RSPLUS / SILU every later
  * call on the handle computes y = W_2 ( A(W_1 x + b_g) . A_3(W_3 x) ), A_3 = act_up, in the sparse and
@@ -267,7 +277,8 @@ const char* sffn_status_string(int status);
  *   memory bytes (wkind: 0 fp32, 1 bf16, 2 int8 rows).  sffn_test_umma_tiling: tiling of the batched gate GEMM.
  * sffn_test_set_knob(knob, value):
  *   PDL                 programmatic dependent launch between calls (default 1)
- *   TENSOR_GATE         single-token bf16 calls take the tensor-core gate kernel where it applies (default 1)
+ *   TENSOR_GATE         1 / 0: single-token calls take the tensor-core gate kernel wherever it applies / nowhere,
+ *                       whatever sffn_set_gate_engine said; -1 (the default): the handle's engine decides
  *   WAIT_CYCLES         budget of every device-side wait in clock cycles (default 2^31, about a second; 0 restores it)
  *   SKIP_ARRIVAL_CTA    index of a CTA of the single-token kernels that neither reports itself finished nor hands in
  *                       its partial result, so that the CTAs which sum the partials see their (bounded) wait run out

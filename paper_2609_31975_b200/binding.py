@@ -62,6 +62,7 @@ def load_library() -> ctypes.CDLL:
         lib.sffn_destroy.argtypes = [vp]
         lib.sffn_set_path.argtypes = [vp, i]
         lib.sffn_set_up_activation.argtypes = [vp, i]
+        lib.sffn_set_gate_engine.argtypes = [vp, i]
         fwd = [vp, vp, i, ctypes.POINTER(_Gate), vp, vp, vp, i, vp, vp]
         lib.sparse_ffn_forward.argtypes = fwd
         lib.dense_ffn_forward.argtypes = fwd
@@ -86,6 +87,7 @@ def load_library() -> ctypes.CDLL:
     return _lib
 
 
+GATE_ENGINE = {"auto": 0, "cuda_core": 1, "tensor_core": 2}
 KNOB = {"pdl": 0, "tensor_gate": 1, "wait_cycles": 2, "skip_arrival_cta": 3, "ring_gate_slots": 4,
         "ring_act_slots": 5, "trace_buffer": 6, "ring_parked_stages": 7, "l2_hints": 8, "drop_stage": 9}
 
@@ -221,6 +223,10 @@ class SparseFFN:
 
     def set_path(self, path: str):
         _check("sffn_set_path", self.lib.sffn_set_path(self._h, PATH[path]))
+
+    def set_gate_engine(self, engine: str):
+        """Where single-token calls compute the gate: "auto", "cuda_core" or "tensor_core" (sffn_set_gate_engine)."""
+        _check("sffn_set_gate_engine", self.lib.sffn_set_gate_engine(self._h, GATE_ENGINE[engine]))
 
     def _gate(self, gate: dict) -> _Gate:
         g = _Gate()

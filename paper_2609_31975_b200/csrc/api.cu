@@ -72,6 +72,7 @@ struct sffn_handle {
   int sm_count;
   int path;
   int act_up;  // activation on the up projection (double activation), SFFN_ACT_NONE = Eq. 1
+  int gate_engine = SFFN_GATE_ENGINE_AUTO;
   long long launches;
   int list_state;  // 0: no sparse call yet, 1: idx/count hold the last call's list, 2: flags hold it
   template <typename T>
@@ -115,7 +116,7 @@ int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dt
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return SFFN_ERR_CUDA;
-  if (cudaMemset(workspace, 0, need) != cudaSuccess) return SFFN_ERR_CUDA;
+  if (cudaMemset(workspace, 0, need) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return SFFN_ERR_CUDA;
   sffn_handle* h = new (std::nothrow) sffn_handle();
   if (!h) return SFFN_ERR_INVALID_ARG;
   h->D = D;
@@ -137,6 +138,12 @@ int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dt
 int sffn_destroy(sffn_handle* h) {
   if (!h) return SFFN_ERR_INVALID_ARG;
   delete h;
+  return SFFN_OK;
+}
+
+int sffn_set_gate_engine(sffn_handle* h, int engine) {
+  if (!h || engine < SFFN_GATE_ENGINE_AUTO || engine > SFFN_GATE_ENGINE_TENSOR_CORE) return SFFN_ERR_INVALID_ARG;
+  h->gate_engine = engine;
   return SFFN_OK;
 }
 
@@ -164,7 +171,7 @@ int sffn_test_set_knob(int knob, long long value) {
   sffn::FusedTestKnobs& k = sffn::fused_test_knobs();
   switch (knob) {
     case SFFN_KNOB_PDL: k.pdl = value != 0; return SFFN_OK;
-    case SFFN_KNOB_TENSOR_GATE: k.tensor_gate = value != 0; return SFFN_OK;
+    case SFFN_KNOB_TENSOR_GATE: k.tensor_gate = value < 0 ? -1 : (value != 0); return SFFN_OK;
     case SFFN_KNOB_WAIT_CYCLES: k.wait_cycles = value > 0 ? value : (1LL << 31); return SFFN_OK;
     case SFFN_KNOB_SKIP_ARRIVAL_CTA: k.skip_arrival_cta = (int)value; return SFFN_OK;
     case SFFN_KNOB_RING_GATE_SLOTS: k.ring_S = (int)value; return SFFN_OK;
@@ -498,7 +505,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
     c.wkind = wkind;
     if (q8) { c.s_gate = q8->s_gate; c.s_V = q8->s_V; c.s_up = q8->s_up; c.s_down = q8->s_down; }
     c.D = h->D; c.H = h->H;
-    c.x = x; c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up; c.y = y;
+    c.x = x; c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up; c.engine = h->gate_engine; c.y = y;
     c.dense = dense;
     c.workspace = h->ws + h->L.fused;
     c.r_max = h->r_max;

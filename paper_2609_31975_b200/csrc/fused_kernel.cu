@@ -157,8 +157,10 @@ __device__ __forceinline__ void named_bar_sync(int id, int threads) {
 __device__ __forceinline__ void named_bar_arrive(int id, int threads) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
-__device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status) {
+// `site` says which wait gave up (diagnostics: word 3 of the status block holds site + 256 * CTA of the last one).
+__device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status, int site) {
   ctl[kAbort] = 1;
+  status[3] = site + 256 * (int)blockIdx.x;
   atomicExch(status, (int32_t)SFFN_ERR_TIMEOUT);
 }
 
@@ -166,7 +168,7 @@ __device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status
 // implementation-defined time, so waiting warps do not steal issue slots from working ones; the
 // cycle budget is checked between attempts.  False when it ran out or the CTA is aborting.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status,
-                                          long long budget) {
+                                          long long budget, int site) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
@@ -175,7 +177,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (mbar_try(bar, parity)) return true;
     if (ctl[kAbort]) return false;
     if (clock64() - t0 > budget) {
-      raise_timeout(ctl, status);
+      raise_timeout(ctl, status, site);
       return false;
     }
   }
@@ -377,7 +379,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       const uint32_t ring = smem_u32(gate_ring);
       for (int s = warp; s < n_gslots; s += kGateProducers) {
         const int slot = s % NG;
-        if (!mbar_wait(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status, p.wait_cycles)) break;
+        if (!mbar_wait(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status, p.wait_cycles, 41)) break;
         const int j0 = slot_first_neuron(s);
         const uint32_t bytes = (uint32_t)(min(nr, p.H - j0) * gate_row_bytes);
         mbar_expect_tx(full_gate + 8 * slot, bytes);
@@ -482,7 +484,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         unsigned long long seen;
         asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.v_counter) : "memory");
         if (seen >= v_target || ctl[kAbort]) break;
-        if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status); break; }
+        if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status, 47); break; }
         __nanosleep(40);
       }
     }
@@ -526,7 +528,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         if (t_idle == 0) t_idle = clock64();
         __nanosleep(20);
         if (ctl[kAbort]) ok = false;
-        else if (clock64() - t_idle > p.wait_cycles) { if (lane == 0) raise_timeout(ctl, p.status); ok = false; }
+        else if (clock64() - t_idle > p.wait_cycles) { if (lane == 0) raise_timeout(ctl, p.status, 48); ok = false; }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         continue;
       }
@@ -538,7 +540,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         fired &= fired - 1;
         const uint32_t sl = __shfl_sync(0xffffffffu, st, l);
         if (lane == 0) {
-          if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles)) {
+          if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 42)) {
             if (ap == 0) slot_a[slot] = sl == 0x80000000u ? 0.f : __uint_as_float(sl);
             const int lrow = base + l;
             if (kScaled && ap == 0) {
@@ -558,7 +560,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
       base += prefix;
     }
-    if (lane == 0 && ok && mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles)) {
+    if (lane == 0 && ok && mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 43)) {
       if (ap == 0) slot_a[slot] = -1.f;      // stop marker: a negative gate value
       mbar_arrive(full_act + 8 * slot);      // completes the phase without data
     }
@@ -600,7 +602,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
           if (gi >= 0) add += row_sg[r0 + lane] * sx[vec_pos<EPV>(gi, D)];
         }
       }
-      if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status, p.wait_cycles)) break;
+      if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status, p.wait_cycles, 44)) break;
       const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
       float mine = 0.f;
       // Short gate rows (LoPA: r elements): a row is a few chunks per lane, and with one warp per scheduler the cost is
@@ -721,13 +723,13 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       float* rp = red + (round & 1) * (2 * kAW + 1);
       const int slot1 = slot + 1 == NA ? 0 : slot + 1;
       const uint32_t par1 = slot + 1 == NA ? par ^ 1 : par;
-      const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status, p.wait_cycles);
+      const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 45);
       const float a0 = got0 ? slot_a[slot] : -1.f;
       bool got1 = true;
       float a1 = -1.f;
       const bool pair = NA >= 4;  // with fewer slots, holding two at a time would stall the act producers
       if (pair && a0 >= 0.f) {
-        got1 = mbar_wait(full_act + 8 * slot1, par1, ctl, p.status, p.wait_cycles);
+        got1 = mbar_wait(full_act + 8 * slot1, par1, ctl, p.status, p.wait_cycles, 46);
         a1 = got1 ? slot_a[slot1] : -1.f;
       }
       const unsigned char* s0 = act_ring + (size_t)slot * p.act_slot_bytes;
@@ -905,7 +907,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
           if (all) break;
           if (t0 == 0) t0 = clock64();
           if (ctl[kAbort]) { ok = false; break; }
-          if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status); ok = false; break; }
+          if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status, 49); ok = false; break; }
           __nanosleep(20);
         }
 #pragma unroll
@@ -1063,9 +1065,17 @@ void debug_fused_plan(int wkind, int D, int H, int K, bool lopa, int sm_count, i
   for (int i = 0; i < 9; ++i) out[i] = v[i];
 }
 
+// Whether this call's gate goes to the tensor cores (see sffn_set_gate_engine).
+static bool wants_tensor_gate(const FusedCall& c) {
+  const int knob = fused_test_knobs().tensor_gate;
+  if (knob >= 0) return knob != 0;
+  if (c.engine == SFFN_GATE_ENGINE_AUTO) return c.dense;
+  return c.engine == SFFN_GATE_ENGINE_TENSOR_CORE;
+}
+
 bool fused_supported(int wkind, int D, int H, int B, const sffn_gate* gate, int sm_count) {
   if (B != 1) return false;
-  if (fused_test_knobs().tensor_gate && fused_tc_supported(wkind, D, H, B, gate, sm_count)) return true;
+  if (fused_test_knobs().tensor_gate != 0 && fused_tc_supported(wkind, D, H, B, gate, sm_count)) return true;
   const bool lopa = gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? gate->r : D;
   return plan(wkind, D, H, K, lopa, fused_grid(sm_count, H)).ok;
@@ -1073,7 +1083,7 @@ bool fused_supported(int wkind, int D, int H, int B, const sffn_gate* gate, int 
 
 cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   pdl_enabled() = fused_test_knobs().pdl;
-  if (fused_test_knobs().tensor_gate && fused_tc_supported(c.wkind, c.D, c.H, 1, c.gate, c.sm_count))
+  if (wants_tensor_gate(c) && fused_tc_supported(c.wkind, c.D, c.H, 1, c.gate, c.sm_count))
     return launch_fused_tc(c, s, launched);
   const bool lopa = c.gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? c.gate->r : c.D;

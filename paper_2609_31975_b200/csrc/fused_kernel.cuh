@@ -25,6 +25,7 @@ struct FusedCall {
   int act_up;
   float* y;
   bool dense;
+  int engine;        // sffn_gate_engine of the handle
   int r_max;         // the handle's largest LoPA rank (workspace layout)
   void* workspace;   // fused_workspace_bytes() bytes, zeroed at handle creation
   int32_t* status;   // device status word
@@ -46,7 +47,7 @@ cudaError_t launch_fused_tc(const FusedCall& c, cudaStream_t s, int* launched);
 // Test hooks (see the "test hooks" section of sparse_ffn.h).
 struct FusedTestKnobs {
   bool pdl = true;               // programmatic dependent launch between calls
-  bool tensor_gate = true;       // take the tensor-core gate where it applies
+  int tensor_gate = -1;          // 1 / 0: tensor-core gate wherever it applies / nowhere; -1: the handle's engine decides
   long long wait_cycles = 1LL << 31;  // budget of every device-side wait (about one second)
   int drop_stage = -1;           // batched gate kernel: CTA 0 never copies this stage's weights (its wait runs out)
   int skip_arrival_cta = -1;     // this CTA does not count itself as finished: the summing CTAs' wait runs out

@@ -18,7 +18,7 @@ def mod():
     import paper_2609_31975_b200 as m
     m.load_library()
     yield m
-    for knob, value in (("wait_cycles", 0), ("skip_arrival_cta", -1), ("drop_stage", -1), ("tensor_gate", 1)):
+    for knob, value in (("wait_cycles", 0), ("skip_arrival_cta", -1), ("drop_stage", -1), ("tensor_gate", -1)):
         m.test_set_knob(knob, value)
 
 

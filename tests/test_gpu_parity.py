@@ -20,6 +20,15 @@ def mod():
     return m
 
 
+@pytest.fixture(params=["cuda_core_gate", "tensor_core_gate"])
+def gate_engine(request, mod):
+    """Single-token calls on the fused path with the gate forced onto one engine (where the tensor-core kernel does
+    not cover the call, both values run the CUDA-core kernel)."""
+    mod.test_set_knob("tensor_gate", 1 if request.param == "tensor_core_gate" else 0)
+    yield request.param
+    mod.test_set_knob("tensor_gate", -1)
+
+
 def make_std(D, H, dtype, seed, s):
     w = syn.standard_ffn(D, H, dtype, seed, DEV, sparsity=s)
     return {"W_g": w["W_g"]}, w
@@ -74,7 +83,7 @@ def test_config1_fp32_all_64_tokens(mod):
 # ------------------------------------------------------------------ shrunken decode shapes, ragged sizes
 @pytest.mark.parametrize("D,H", [(512, 1000), (264, 777), (1024, 2049), (2048, 300)])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_standard_gate_small_shapes(mod, D, H, dtype):
+def test_standard_gate_small_shapes(mod, gate_engine, D, H, dtype):
     ffn = mod.SparseFFN(D, H, dtype, B_max=1)
     for s, act in ((0.5, "relu"), (0.9, "sqrelu"), (0.95, "rsplus")):
         gate, w = make_std(D, H, dtype, 21, s)
@@ -85,7 +94,7 @@ def test_standard_gate_small_shapes(mod, D, H, dtype):
 
 @pytest.mark.parametrize("D,H", [(3840, 300), (5120, 200), (8192, 160), (16384, 96)])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_wide_rows(mod, D, H, dtype):
+def test_wide_rows(mod, gate_engine, D, H, dtype):
     """Rows of 7.5 to 64 KB: one row per gate slot, few ring slots, up to eight chunks per act thread; whatever
     `auto` picks for the shape (the fused kernels where their geometry fits, else the general ones)."""
     if D * (2 if dtype == torch.bfloat16 else 4) > 32768:               # rows above 32 KB are refused, not mangled
@@ -172,7 +181,7 @@ def test_batched_lopa(mod, B, r, rms, path):
 
 # ------------------------------------------------------------------ degenerate cases
 @pytest.mark.parametrize("path", ["general", "fused"])
-def test_full_and_zero_sparsity(mod, path):
+def test_full_and_zero_sparsity(mod, gate_engine, path):
     D, H = 512, 900
     ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=1)
     ffn.set_path(path)
@@ -196,7 +205,7 @@ def test_full_and_zero_sparsity(mod, path):
 
 
 @pytest.mark.parametrize("path", ["general", "fused"])
-def test_dense_comparator_and_determinism(mod, path):
+def test_dense_comparator_and_determinism(mod, gate_engine, path):
     D, H = 1024, 3000
     ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=128, B_max=1)
     ffn.set_path(path)
@@ -320,7 +329,7 @@ def test_batched_calls_repeat_bit_for_bit(mod):
 
 # ------------------------------------------------------------------ double activation (Sec. 3.3)
 @pytest.mark.parametrize("act,act_up", [("relu", "relu"), ("sqrelu", "rsplus"), ("rsplus", "sqrelu"), ("relu", "silu")])
-def test_double_activation_all_paths(mod, act, act_up):
+def test_double_activation_all_paths(mod, gate_engine, act, act_up):
     D, H = 512, 1100
     ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=64, B_max=8)
     ffn.set_up_activation(act_up)
@@ -361,7 +370,7 @@ def test_double_activation_all_paths(mod, act, act_up):
 # ------------------------------------------------------------------ layer loop under a CUDA graph
 @pytest.mark.parametrize("kind", ["standard", "lopa"])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_layer_chain_in_cuda_graph(mod, dtype, kind):
+def test_layer_chain_in_cuda_graph(mod, gate_engine, dtype, kind):
     D, H, L, r = 512, 900, 3, 64
     ffn = mod.SparseFFN(D, H, dtype, r_max=r, B_max=1)
     if kind == "standard":
@@ -408,33 +417,25 @@ def test_layer_chain_in_cuda_graph(mod, dtype, kind):
 
 # ------------------------------------------------------------------ full-size configurations
 @pytest.mark.parametrize("s,ntok", [(0.9, 8), (0.5, 1), (0.7, 2), (0.8, 2), (0.95, 1)])
-def test_config2_full_size_decode(mod, s, ntok):
+def test_config2_full_size_decode(mod, gate_engine, s, ntok):
     D, H = 4096, 14336
     ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=1)
     gate, w = make_std(D, H, torch.bfloat16, 2, s)
     x = syn.tokens(ntok, D, torch.bfloat16, 2, DEV)
     ref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", threads=16)
     assert abs(1 - ref["n_act"].mean() / H - s) < 0.03
-    for path in ("general", "fused"):            # fused: the tensor-core gate kernel at this shape
+    for path in ("general", "fused"):
         ffn.set_path(path)
         for t in range(ntok if path == "fused" else min(ntok, 2)):
             y = ffn.sparse_ffn_forward(x[t], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
             one = dict(y=ref["y"][t], z=ref["z"][t])
             assert_y_close(y, one["y"], what=f"config2 s={s} token {t} [{path}]")
             assert_active_set(ffn.last_active(), one, what=f"config2 s={s} token {t} [{path}]")
-    # the CUDA-core gate of the single-token kernel (what other storage types run) at the same shape
-    mod.test_set_knob("tensor_gate", 0)
-    try:
-        y = ffn.sparse_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
-        assert_y_close(y, ref["y"][0], what=f"config2 s={s} [fused, CUDA-core gate]")
-        assert_active_set(ffn.last_active(), dict(z=ref["z"][0]), what=f"config2 s={s} [fused, CUDA-core gate]")
-    finally:
-        mod.test_set_knob("tensor_gate", 1)
     torch.cuda.synchronize()
     assert ffn.device_status() == 0
 
 
-def test_config2_full_size_rsplus(mod):
+def test_config2_full_size_rsplus(mod, gate_engine):
     D, H = 4096, 14336
     ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=1)
     gate, w = make_std(D, H, torch.bfloat16, 2, 0.9)
@@ -470,7 +471,7 @@ def test_config4_full_size_batched_zipf(mod, B):
 
 
 @pytest.mark.parametrize("s", [0.9, 0.8, 0.95])
-def test_config5_full_size_stress_layer0(mod, s):
+def test_config5_full_size_stress_layer0(mod, gate_engine, s):
     """8192 x 28672, squared RELU, standard and LoPA r = 1024 gates, one token and a batch of eight (the batch:
     the tcgen05 gate GEMM with K = 8192 and several 128-row tiles per CTA, gather4 over the union)."""
     D, H = 8192, 28672
@@ -506,7 +507,7 @@ def test_config5_full_size_stress_layer0(mod, s):
 
 def test_two_handles_on_two_streams_overlap_and_agree(mod):
     # Two standard-gate single-token calls in flight at once (different handles, different streams): each wants every SM
-    # and its last CTAs wait for the rest, but at most 63 + 63 CTAs sit waiting, so both complete -- and bit for bit with
+    # and its last CTAs wait for the rest, but at most 64 + 64 CTAs sit waiting for partial results, so both complete -- and bit for bit with
     # what they give one after the other.
     D, H = 4096, 14336
     sets = [syn.standard_ffn(D, H, torch.bfloat16, 90 + i, DEV, sparsity=0.9) for i in range(2)]
@@ -528,3 +529,35 @@ def test_two_handles_on_two_streams_overlap_and_agree(mod):
     for i in range(2):
         assert ffns[i].device_status() == 0
         assert torch.equal(got[i], want[i])
+
+
+def test_gate_engine_setting_and_a_long_chain_of_mixed_calls(mod):
+    # The public engine setting (parity under each value), then 6000 calls back to back on one stream that switch
+    # engine, weights and sparse / dense every few calls: no wait runs out, and every call repeats its first result
+    # bit for bit (the calls of a chain overlap at their edges; nothing of one call may leak into the next).
+    D, H = 4096, 14336
+    sets = [syn.standard_ffn(D, H, torch.bfloat16, 70 + i, DEV, sparsity=sp) for i, sp in enumerate((0.9, 0.6, 0.97))]
+    x = syn.tokens(6, D, torch.bfloat16, 70, DEV)
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=1)
+    assert ffn.lib.sffn_set_gate_engine(ffn._h, 3) == 1          # no such engine: SFFN_ERR_INVALID_ARG
+    ref = run_oracle(x[0], {"W_g": sets[0]["W_g"]}, sets[0]["b_g"], sets[0]["W_up"], sets[0]["W_down"], "relu", threads=16)
+    for engine in ("cuda_core", "tensor_core", "auto"):
+        ffn.set_gate_engine(engine)
+        for dense in (False, True):
+            fn = ffn.dense_ffn_forward if dense else ffn.sparse_ffn_forward
+            y = fn(x[0], {"W_g": sets[0]["W_g"]}, sets[0]["b_g"], sets[0]["W_up"], sets[0]["W_down"], "relu")
+            assert_y_close(y, ref["y"], what=f"engine {engine}, dense {dense}")
+    engines = ("cuda_core", "tensor_core", "auto")
+    kinds = [(e, w, dense) for e in range(3) for w in range(3) for dense in (False, True)]
+    first = torch.empty((len(kinds), 6, D), device=DEV)
+    out = torch.empty((len(kinds), 6, D), device=DEV)
+    for rounds, dst in ((1, first), (55, out)):
+        for rnd in range(rounds):
+            for k, (e, w, dense) in enumerate(kinds):
+                ffn.set_gate_engine(engines[e])
+                fn = ffn.dense_ffn_forward if dense else ffn.sparse_ffn_forward
+                for t in range(6):
+                    fn(x[t], {"W_g": sets[w]["W_g"]}, sets[w]["b_g"], sets[w]["W_up"], sets[w]["W_down"], "relu", dst[k, t])
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
+    assert torch.equal(first, out)
