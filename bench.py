@@ -39,7 +39,7 @@ WEIGHT_SETS = 4
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the main kernel at this workload: kept beside the
 # ncu summary it comes from and rewritten whenever that summary is refreshed
-NCU_TRAFFIC_FILE = ROOT / "profiles" / "fused_tc_kernel_decode_4096x14336_s090.json"
+NCU_TRAFFIC_FILE = ROOT / "profiles" / "fused_ffn_kernel_decode_4096x14336_s090.json"
 WORKLOAD = "llama-style standard-gated FFN decode, d_model=4096 d_ff=14336 bf16 batch=1 RELU, sparsity 0.9"
 
 
@@ -323,8 +323,8 @@ def run_ours(args, rank, world, local):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"{peak_kind} copy bandwidth", "traffic": ncu_traffic_per_launch(),
                      "algorithmic_bytes_per_launch": bytes_per_call,
-                     "kernel": "fused_tc_kernel (one launch per FFN call: gate on tcgen05, rows of fired neurons, "
-                               "cross-CTA sum in the first CTAs to finish)"},
+                     "kernel": "fused_ffn_kernel (one launch per FFN call: gate stream on the CUDA cores, rows of fired "
+                               "neurons, cross-CTA sum in the first CTAs to finish)"},
         "e2e": {"value": us_e2e / world, "unit": "us/FFN-call", "h2d_bytes_per_step": args.calls * D_MODEL * 2,
                 "d2h_bytes_per_step": args.calls * D_MODEL * 4},
         "gpu_launches": launches, "clocks": clk.summary(),

@@ -65,11 +65,10 @@ struct FusedParams {
   int use_rmsnorm;
   float eps;
   const void* V;      // LoPA: [r, D]
-  float* vbuf;        // LoPA: [r] exchange buffer for v = V x
+  unsigned long long* vtag;  // LoPA: [r] exchange buffer for v = V x, every value tagged with the call's number
   // Two arrival counters in the workspace, monotonic over calls.  Every call adds exactly gridDim.x to each and
   // calls on one workspace are serialised, so a CTA derives its call's first and last value from what its own
   // atomicAdd returned: nothing depends on a host-side count, and a captured launch can be replayed.
-  unsigned long long* v_counter;     // LoPA: CTAs that have published their rows of v = V x
   unsigned long long* done_counter;  // CTAs that have written their partial of y
   float* y;                          // [D] result, written by the last CTAs to finish
   int act, dense;
@@ -83,6 +82,9 @@ struct FusedParams {
   uint8_t* flag;
   int32_t* status;
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
+  int v_in_smem;     // LoPA: this CTA's rows of V are copied into the (idle) act ring at the start of the call
+  int gate_workers;  // warps that take gate slots, slot s going to worker s % gate_workers: the gate warps, and for
+                     // the LoPA gate also act warps (a ring slot that is reused always belongs to the same worker)
   int gate_warps;    // gate warps in use; n_gate_slots is a multiple of it, so a ring slot always
                      // belongs to the same warp and its phases are consumed strictly in order
   long long wait_cycles;  // budget of every wait below (about one second unless a test shortens it)
@@ -109,7 +111,7 @@ struct SmemLayout {
     slot_a = take(n_act_slots * 4);
     red = take(2 * (2 * 8 + 1) * 4);  // up to eight act warps
     ctl = take(8 * 4);
-    bars = take(2 * (n_gate_slots + n_act_slots) * 8);
+    bars = take(2 * (n_gate_slots + n_act_slots) * 8 + 8);  // + one for the CTA's rows of V (LoPA)
     row_params = take((lopa || scaled) ? (1 + (lopa ? 2 : 0) + (scaled ? 1 : 0)) * slab_max * 4 : 0);  // per-neuron gate parameters
     row_scales = take(scaled ? 2 * slab_max * 4 : 0);     // int8 rows: scales of the slab's W_up / W_down rows
     slot_scales = take(scaled ? 2 * n_act_slots * 4 : 0);  // the same two for the row in each act slot
@@ -167,14 +169,17 @@ __device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status
 // Bounded wait on an mbarrier phase.  try_wait parks the thread in hardware for a short,
 // implementation-defined time, so waiting warps do not steal issue slots from working ones; the
 // cycle budget is checked between attempts.  False when it ran out or the CTA is aborting.
+template <bool kBackoff = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl, int32_t* status,
                                           long long budget, int site) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < 64; ++i) {
       if (mbar_try(bar, parity)) return true;
+      if (kBackoff) __nanosleep(100);  // a producer waiting for a free slot: keep out of the working warps' way
+    }
     if (ctl[kAbort]) return false;
     if (clock64() - t0 > budget) {
       raise_timeout(ctl, status, site);
@@ -338,6 +343,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const uint32_t bars = smem_u32(smem + L.bars);
   const uint32_t full_gate = bars, empty_gate = bars + 8 * NG;
   const uint32_t full_act = bars + 16 * NG, empty_act = bars + 16 * NG + 8 * NA;
+  const uint32_t v_bar = bars + 16 * (NG + NA);
 
   const int nvecD = D / EPV, nvecK = K / EPV;
   const size_t row_bytes = (size_t)D * sizeof(T);
@@ -367,6 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         mbar_init(full_act + 8 * s, kActProducers);
         mbar_init(empty_act + 8 * s, kAW);
       }
+      mbar_init(v_bar, 1);
       for (int i = 0; i < 8; ++i) ctl[i] = 0;
       for (int i = 0; i < 2 * (2 * kAW + 1); ++i) red[i] = 0.f;
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -374,19 +381,30 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     }
     named_bar_sync(4, 32 * kGateProducers);  // barriers are initialised
     named_bar_arrive(3, kThreads);           // release the other warps (they block on barrier 3)
+    if (LOPA && warp == 1 && lane == 0) {
+      // This CTA's rows of V (consecutive rows: one copy) go into the act ring, which is idle until the gate vector
+      // is complete; they are weights, so they travel while the CTA still waits for its predecessor.
+      const int vlo = (int)((long long)K * cta / G), vhi = (int)((long long)K * (cta + 1) / G);
+      if (vhi > vlo && p.v_in_smem) {
+        mbar_expect_tx(v_bar, (uint32_t)((vhi - vlo) * row_bytes));
+        bulk_g2s(smem_u32(act_ring), static_cast<const char*>(p.V) + (size_t)vlo * row_bytes,
+                 (uint32_t)((vhi - vlo) * row_bytes), v_bar);
+      } else {
+        mbar_arrive(v_bar);
+      }
+    }
     if (lane == 0) {
       const char* Wg = static_cast<const char*>(p.Wgate);
       const uint32_t ring = smem_u32(gate_ring);
       for (int s = warp; s < n_gslots; s += kGateProducers) {
         const int slot = s % NG;
-        if (!mbar_wait(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status, p.wait_cycles, 41)) break;
+        if (!mbar_wait<true>(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status, p.wait_cycles, 41)) break;
         const int j0 = slot_first_neuron(s);
         const uint32_t bytes = (uint32_t)(min(nr, p.H - j0) * gate_row_bytes);
         mbar_expect_tx(full_gate + 8 * slot, bytes);
         bulk_g2s(ring + (uint32_t)slot * p.gate_slot_bytes, Wg + (size_t)j0 * gate_row_bytes, bytes,
                  full_gate + 8 * slot);
       }
-      if (warp == 0) SFFN_STAMP(1);
     }
     __syncwarp();
     return;
@@ -399,16 +417,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     const int lines = (int)(((size_t)D * sizeof(X) + 127) / 128);
     for (int i = lane; i < lines; i += 32)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const char*>(p.x) + (size_t)i * 128) : "memory");
-  }
-
-  // LoPA: this CTA's rows of V are weights too; pull them into L2 now so that the rank-r stage, which sits on the
-  // call's critical path right after the wait, finds them there.
-  if (LOPA && warp == kGateProducers) {
-    const int vlo = (int)((long long)K * cta / G), vhi = (int)((long long)K * (cta + 1) / G);
-    for (int k = vlo + lane; k < vhi; k += 32)
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(static_cast<const char*>(p.V) + (size_t)k * row_bytes),
-                   "r"((uint32_t)row_bytes)
-                   : "memory");
   }
 
   // Per-neuron parameters of the slab go into shared memory now; for int8 rows also the scales of its W_up / W_down
@@ -438,7 +446,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   // ---- everyone else: wait for the predecessor in the stream, then stage the token ------------
   pdl_wait();
   if (tid == kStageBase) SFFN_GSTAMP(11);
-  const uint32_t ep = warp >= kFirstGateWarp ? __ldcg(p.epoch_word) + 1u : 0u;  // this call's number (tags of the partials)
+  // this call's number: the tag of the partials and of the LoPA exchange values
+  const uint32_t ep = (LOPA || warp >= kFirstGateWarp) ? __ldcg(p.epoch_word) + 1u : 0u;
   for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) row_state[i] = 0xffffffffu;
   constexpr int XEPV = Elem<X>::kPerVec;  // token elements per 16 bytes (the weights' EPV unless those are int8)
   for (int cx = tid - kStageBase; cx < D / XEPV; cx += kStageThreads) {
@@ -452,58 +461,203 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     }
   }
   if (LOPA) {
-    // Rank-r stage of the LoPA gate, v = V x, spread over the grid: this CTA computes its share of
-    // the rows of V (one warp per row, straight from global memory), publishes them, and waits until
-    // every CTA has done so.  All CTAs of the call become resident without waiting for this one
-    // (one CTA per SM, predecessors in the stream never wait on their successors), so the bounded
-    // wait below ends as soon as the slowest CTA has started and published.
+    // Rank-r stage of the LoPA gate, v = V x, spread over the grid: this CTA computes its share of the rows of V,
+    // publishes them, and collects everybody's.  All CTAs of the call become resident without waiting for this one
+    // (one CTA per SM, predecessors in the stream never wait on their successors), so the bounded wait below ends as
+    // soon as the slowest CTA has started and published.  The stage sits on the call's critical path, so it is made of
+    // as few dependent memory round trips as it can be: every warp takes 32-chunk segments of the CTA's rows (all
+    // loads of a warp in flight together), the segment sums are added per row in a fixed order, and the values are
+    // published with the call's number in the same 64-bit word -- a reader that finds the number has the value, no
+    // counter and no fence in between.
     const int r = K;
-    named_bar_sync(5, kStageThreads);  // the token is staged
+    const int st = tid - kStageBase, sw = warp - kGateProducers;
+    constexpr int kSW = kStageThreads / 32;
     const int vlo = (int)((long long)r * cta / G), vhi = (int)((long long)r * (cta + 1) / G);
-    for (int k = vlo + (warp - kGateProducers); k < vhi; k += kStageThreads / 32) {
-      const uint4* vr = reinterpret_cast<const uint4*>(static_cast<const char*>(p.V) + (size_t)k * row_bytes);
-      float a0 = 0.f, a1 = 0.f;
-      int c = lane;
-      for (; c + 32 < nvecD; c += 64) {
-        const uint4 w0 = ld_stream16(vr + c), w1 = ld_stream16(vr + c + 32);
-        a0 = chunk_dot<T>(w0, sx, c, nvecD, a0);
-        a1 = chunk_dot<T>(w1, sx, c + 32, nvecD, a1);
-      }
-      if (c < nvecD) a0 = chunk_dot<T>(ld_stream16(vr + c), sx, c, nvecD, a0);
-      const float v = warp_sum(a0 + a1) * (kScaled ? __ldg(p.s_V + k) : 1.f);
-      if (lane == 0) __stcg(p.vbuf + k, v);
+    const int v_max = (r + G - 1) / G;                  // most rows of V a CTA has
+    // where they do not fit beside the sums (wide rows, high rank) they are read from global memory instead
+    const uint4* vsm = p.v_in_smem ? reinterpret_cast<const uint4*>(act_ring)
+                                   : reinterpret_cast<const uint4*>(static_cast<const char*>(p.V) + (size_t)vlo * row_bytes);
+    float* wss = reinterpret_cast<float*>(act_ring + (p.v_in_smem ? (size_t)v_max * row_bytes : 0));
+    float* vpart = wss + 32;
+    named_bar_sync(5, kStageThreads);  // the token is staged
+    if (st == 0) SFFN_STAMP(15);
+    mbar_wait(v_bar, 0, ctl, p.status, p.wait_cycles, 50);
+    const int nseg = (nvecD + 31) / 32, items = (vhi - vlo) * nseg;  // fits the act ring: checked on the host
+    for (int it = sw; it < items; it += kSW) {
+      const int row = it / nseg, c = (it - row * nseg) * 32 + lane;
+      const float a = warp_sum(c < nvecD ? chunk_dot<T>(vsm[(size_t)row * nvecD + c], sx, c, nvecD, 0.f) : 0.f);
+      if (lane == 0) vpart[it] = a;
     }
     named_bar_sync(5, kStageThreads);
-    if (tid == kStageBase) {
-      // release at device scope after the barrier: this CTA's rows of v happen before it
-      unsigned long long arrived;
-      asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(arrived) : "l"(p.v_counter) : "memory");
-      const unsigned long long v_target = (arrived / G + 1) * G;
-      const long long t0 = clock64();
-      for (;;) {
-        unsigned long long seen;
-        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(p.v_counter) : "memory");
-        if (seen >= v_target || ctl[kAbort]) break;
-        if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status, 47); break; }
-        __nanosleep(40);
-      }
+    if (st == 0) SFFN_STAMP(9);
+    for (int k = vlo + st; k < vhi; k += kStageThreads) {
+      float v = 0.f;
+      for (int g = 0; g < nseg; ++g) v += vpart[(k - vlo) * nseg + g];
+      if (kScaled) v *= __ldg(p.s_V + k);
+      asm volatile("st.global.cg.b64 [%0], %1;" ::"l"(p.vtag + k), "l"(tagged(v, ep)) : "memory");
     }
-    named_bar_sync(5, kStageThreads);
-    // n = RMSNorm(v) (or v) into shared memory; every warp derives the same scale
+    // collect: two values per thread and pass, both loads in flight; a value still carrying an older number is
+    // read again (bounded)
     float ss = 0.f;
-    for (int k = lane; k < r; k += 32) {
-      const float v = __ldcg(p.vbuf + k);
-      ss = fmaf(v, v, ss);
+    const long long t0 = clock64();
+    for (int k = st; k < r; k += 2 * kStageThreads) {
+      const int k1 = k + kStageThreads;
+      unsigned long long w0 = 0, w1 = 0;
+      bool have0 = false, have1 = k1 >= r;
+      for (;;) {
+        if (!have0) asm volatile("ld.global.cg.b64 %0, [%1];" : "=l"(w0) : "l"(p.vtag + k) : "memory");
+        if (!have1) asm volatile("ld.global.cg.b64 %0, [%1];" : "=l"(w1) : "l"(p.vtag + k1) : "memory");
+        have0 = (uint32_t)(w0 >> 32) == ep;
+        have1 = have1 || (uint32_t)(w1 >> 32) == ep;
+        if ((have0 && have1) || ctl[kAbort]) break;
+        if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status, 47); break; }
+      }
+      const float v0 = __uint_as_float((uint32_t)w0), v1 = k1 < r ? __uint_as_float((uint32_t)w1) : 0.f;
+      ss = fmaf(v0, v0, ss);
+      ss = fmaf(v1, v1, ss);
+      sn[vec_pos<EPV>(k, r)] = v0;
+      if (k1 < r) sn[vec_pos<EPV>(k1, r)] = v1;
     }
+    // n = RMSNorm(v) (or v): the warps' sums of squares are added in a fixed order by everyone
+    if (st == 0) SFFN_STAMP(14);
     ss = warp_sum(ss);
-    const float inv = p.use_rmsnorm ? rsqrtf(ss / (float)r + p.eps) : 1.f;
-    for (int k = tid - kStageBase; k < r; k += kStageThreads)
-      sn[vec_pos<EPV>(k, r)] = __ldcg(p.vbuf + k) * ((p.use_rmsnorm && p.gain) ? p.gain[k] : 1.f) * inv;
+    if (lane == 0) wss[sw] = ss;
+    named_bar_sync(5, kStageThreads);
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < kSW; ++i) tot += wss[i];
+    const float inv = p.use_rmsnorm ? rsqrtf(tot / (float)r + p.eps) : 1.f;
+    for (int k = st; k < r; k += kStageThreads)
+      sn[vec_pos<EPV>(k, r)] *= ((p.use_rmsnorm && p.gain) ? p.gain[k] : 1.f) * inv;
   }
   named_bar_sync(3, kThreads);
   if (tid == kStageBase) SFFN_STAMP(0);
 
   const float* gvec = LOPA ? sn : sx;  // the vector every gate row is dotted with
+
+  // One ring slot of gate rows: dot every row with the gate vector, publish the results, give the slot back.  False
+  // when the wait for the slot's rows ran out.
+  const int gw = warp - kFirstGateWarp;
+  auto gate_slot = [&](int s) -> bool {
+    const int slot = s % NG;
+    const int r0 = s * nr;
+    const int j0 = slot_first_neuron(s);
+    const int rows = min(nr, p.H - j0);
+    float add = 0.f;  // bias + fixed-matrix term of the row this lane reports
+    float scale = 1.f;  // int8 rows: scale of that row
+    if (lane < rows) {
+      if (kTables) add = row_bias[r0 + lane];
+      else if (s == gw) add = pre_bias[0];
+      else if (s == gw + p.gate_warps) add = pre_bias[1];
+      else add = p.b_g ? p.b_g[j0 + lane] : 0.f;
+      if (kScaled) scale = row_gscale[r0 + lane];
+      if (LOPA) {
+        const int gi = row_gi[r0 + lane];
+        if (gi >= 0) add += row_sg[r0 + lane] * sx[vec_pos<EPV>(gi, D)];
+      }
+    }
+    if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status, p.wait_cycles, 44)) return false;
+    if (lane == 0 && s == 0) SFFN_STAMP(7);
+    const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
+    float mine = 0.f;
+    // Short gate rows (LoPA: r elements): a row is a few chunks per lane, and with one warp per scheduler the cost is
+    // instruction latency, not throughput.  Eight rows are dotted side by side (eight independent chains, the vector
+    // read once for all of them, every load requested before the first multiply) and reduced together: each
+    // exchange halves the number of sums a lane carries, so eight rows cost 4 + 2 + 1 + 1 + 1 shuffles instead of 40.
+    const int rows_short = nvecK <= 128 ? rows : 0;
+    int rr_short = 0;
+    for (; rows_short - rr_short > 2; rr_short += 8) {  // one or two left-over rows are cheaper one by one (below)
+      const int rr = rr_short;
+      float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      for (int c = lane; c < nvecK; c += 32) {
+        uint4 w[8];
+        float4 v[EPV / 4];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          w[i] = rr + i < rows ? reinterpret_cast<const uint4*>(base + (size_t)(rr + i) * gate_row_bytes)[c]
+                               : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int q = 0; q < EPV / 4; ++q) v[q] = reinterpret_cast<const float4*>(gvec)[q * nvecK + c];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float f[EPV];
+          Elem<T>::unpack(w[i], f);
+#pragma unroll
+          for (int q = 0; q < EPV / 4; ++q) {
+            a[i] = fmaf(f[4 * q + 0], v[q].x, a[i]);
+            a[i] = fmaf(f[4 * q + 1], v[q].y, a[i]);
+            a[i] = fmaf(f[4 * q + 2], v[q].z, a[i]);
+            a[i] = fmaf(f[4 * q + 3], v[q].w, a[i]);
+          }
+        }
+      }
+      // lanes with bit 4 set keep rows 4..7, the others rows 0..3; then bit 3 picks two of the four, bit 2 one of
+      // the two; bits 1 and 0 are plain sums.  Afterwards lanes 4 k .. 4 k + 3 hold the dot product of row rr + k.
+      float b4[4], b2[2];
+      const bool up16 = lane & 16, up8 = lane & 8, up4 = lane & 4;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        b4[i] = (up16 ? a[4 + i] : a[i]) + __shfl_xor_sync(0xffffffffu, up16 ? a[i] : a[4 + i], 16);
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+        b2[i] = (up8 ? b4[2 + i] : b4[i]) + __shfl_xor_sync(0xffffffffu, up8 ? b4[i] : b4[2 + i], 8);
+      float z = (up4 ? b2[1] : b2[0]) + __shfl_xor_sync(0xffffffffu, up4 ? b2[0] : b2[1], 4);
+      z += __shfl_xor_sync(0xffffffffu, z, 2);
+      z += __shfl_xor_sync(0xffffffffu, z, 1);
+      const float got = __shfl_sync(0xffffffffu, z, 4 * ((lane - rr) & 7));
+      if (lane >= rr && lane < rr + 8) mine = got;
+    }
+    for (; rr_short < rows_short; ++rr_short) {
+      const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr_short * gate_row_bytes);
+      float a0 = 0.f;
+      for (int c = lane; c < nvecK; c += 32) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
+      const float z = warp_sum(a0);
+      if (lane == rr_short) mine = z;
+    }
+    int rr_single = rows_short;
+    if (EPV == 16) {
+      // int8 rows: the staged vector is four times the bytes of a row, so two rows share every read of it
+      for (; rr_single + 1 < rows; rr_single += 2) {
+        const uint4* w0 = reinterpret_cast<const uint4*>(base + (size_t)rr_single * gate_row_bytes);
+        const uint4* w1 = reinterpret_cast<const uint4*>(base + (size_t)(rr_single + 1) * gate_row_bytes);
+        float2 a0 = make_float2(0.f, 0.f), a1 = a0, b0 = a0, b1 = a0;
+        int c = lane;
+        for (; c + 32 < nvecK; c += 64) {
+          chunk_dot2_q8(w0[c], w1[c], gvec, c, nvecK, a0, b0);
+          chunk_dot2_q8(w0[c + 32], w1[c + 32], gvec, c + 32, nvecK, a1, b1);
+        }
+        if (c < nvecK) chunk_dot2_q8(w0[c], w1[c], gvec, c, nvecK, a0, b0);
+        const float z0 = warp_sum((a0.x + a0.y) + (a1.x + a1.y)), z1 = warp_sum((b0.x + b0.y) + (b1.x + b1.y));
+        if (lane == rr_single) mine = z0;
+        if (lane == rr_single + 1) mine = z1;
+      }
+    }
+    for (int rr = rr_single; rr < rows; ++rr) {
+      const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr * gate_row_bytes);
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      int c = lane;
+      for (; c + 96 < nvecK; c += 128) {
+        const uint4 w0 = w[c], w1 = w[c + 32], w2 = w[c + 64], w3 = w[c + 96];
+        a0 = chunk_dot<T>(w0, gvec, c, nvecK, a0);
+        a1 = chunk_dot<T>(w1, gvec, c + 32, nvecK, a1);
+        a2 = chunk_dot<T>(w2, gvec, c + 64, nvecK, a2);
+        a3 = chunk_dot<T>(w3, gvec, c + 96, nvecK, a3);
+      }
+      for (; c < nvecK; c += 32) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
+      const float z = warp_sum((a0 + a1) + (a2 + a3));
+      if (lane == rr) mine = z;
+    }
+    if (lane < rows) {
+      const float z = kScaled ? fmaf(mine, scale, add) : mine + add;
+      const bool fired = z > 0.f;
+      if (!p.dense) p.flag[j0 + lane] = fired ? 1 : 0;
+      row_state[r0 + lane] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty_gate + 8 * slot);
+    if (lane == 0 && s == 0) SFFN_STAMP(6);
+    return true;
+  };
 
   if (warp < kFirstGateWarp) {
     // ======================= act producers: rows of fired neurons, ascending ===================
@@ -518,6 +672,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // The whole warp classifies 32 rows per step (one shared-memory read + ballots); lane 0 issues
     // the copies of the fired ones in ascending order.  Only the leading run of finished rows is
     // consumed, so the order never depends on which gate warp was faster.
+#ifdef SFFN_TRACE
+    int n_issued = 0;
+#endif
     long long t_idle = 0;
     for (int base = 0; ok && base < slab_rows;) {
       const int row = base + lane;
@@ -535,32 +692,43 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       t_idle = 0;
       const bool take = row < slab_rows && lane < prefix && (p.dense || st != 0x80000000u);
       unsigned fired = __ballot_sync(0xffffffffu, take);
+      // Every lane issues the copy of its own row: up to NA rows go out per step, each into the ring slot of its
+      // place among the fired rows (one lane issuing them one after the other manages a row every ~500 cycles, which
+      // is what bounds a call with a short gate).
       while (fired && ok) {
-        const int l = __ffs(fired) - 1;
-        fired &= fired - 1;
-        const uint32_t sl = __shfl_sync(0xffffffffu, st, l);
-        if (lane == 0) {
-          if (mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 42)) {
-            if (ap == 0) slot_a[slot] = sl == 0x80000000u ? 0.f : __uint_as_float(sl);
-            const int lrow = base + l;
+        const int place = __popc(fired & ((1u << lane) - 1u));
+        const int nb = min(__popc(fired), NA);
+        const bool mine = ((fired >> lane) & 1u) != 0 && place < nb;
+        bool good = true;
+        if (mine) {
+          int ms = slot + place;
+          uint32_t mp = par;
+          if (ms >= NA) { ms -= NA; mp ^= 1; }
+          if (mbar_wait<true>(empty_act + 8 * ms, mp, ctl, p.status, p.wait_cycles, 42)) {
+            if (ap == 0) slot_a[ms] = st == 0x80000000u ? 0.f : __uint_as_float(st);
             if (kScaled && ap == 0) {
-              slot_su[slot] = row_su[lrow];
-              slot_sd[slot] = row_sd[lrow];
+              slot_su[ms] = row_su[row];
+              slot_sd[ms] = row_sd[row];
             }
-            const size_t j = (size_t)(slot_first_neuron(lrow / nr) + lrow % nr);
-            mbar_expect_tx(full_act + 8 * slot, (uint32_t)row_bytes);
-            bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
-                     full_act + 8 * slot);
+            const size_t j = (size_t)(slot_first_neuron(row / nr) + row % nr);
+            mbar_expect_tx(full_act + 8 * ms, (uint32_t)row_bytes);
+            bulk_g2s(ring + (uint32_t)ms * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
+                     full_act + 8 * ms);
           } else {
-            ok = false;
+            good = false;
           }
         }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (++slot == NA) { slot = 0; par ^= 1; }
+        ok = __all_sync(0xffffffffu, good);
+        fired &= ~__ballot_sync(0xffffffffu, mine);
+#ifdef SFFN_TRACE
+        n_issued += nb;
+#endif
+        slot += nb;
+        if (slot >= NA) { slot -= NA; par ^= 1; }
       }
       base += prefix;
     }
-    if (lane == 0 && ok && mbar_wait(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 43)) {
+    if (lane == 0 && ok && mbar_wait<true>(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 43)) {
       if (ap == 0) slot_a[slot] = -1.f;      // stop marker: a negative gate value
       mbar_arrive(full_act + 8 * slot);      // completes the phase without data
     }
@@ -569,6 +737,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       // overlaps with the act warps' last rows; -1 under the test hook that makes a CTA go missing.
       if (lane == 0) {
         SFFN_STAMP(2);
+#ifdef SFFN_TRACE
+        if (p.trace) p.trace[(size_t)blockIdx.x * 16 + 1] = n_issued;
+#endif
         int rank = -1;
         if (cta != p.skip_arrival_cta) {
           unsigned long long old;
@@ -583,134 +754,41 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     __syncwarp();
   } else if (warp < kFAW) {
     // ======================= gate warps ========================================================
-    const int gw = warp - kFirstGateWarp;
-    for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_warps) {
-      const int slot = s % NG;
-      const int r0 = s * nr;
-      const int j0 = slot_first_neuron(s);
-      const int rows = min(nr, p.H - j0);
-      float add = 0.f;  // bias + fixed-matrix term of the row this lane reports
-      float scale = 1.f;  // int8 rows: scale of that row
-      if (lane < rows) {
-        if (kTables) add = row_bias[r0 + lane];
-        else if (s == gw) add = pre_bias[0];
-        else if (s == gw + p.gate_warps) add = pre_bias[1];
-        else add = p.b_g ? p.b_g[j0 + lane] : 0.f;
-        if (kScaled) scale = row_gscale[r0 + lane];
-        if (LOPA) {
-          const int gi = row_gi[r0 + lane];
-          if (gi >= 0) add += row_sg[r0 + lane] * sx[vec_pos<EPV>(gi, D)];
-        }
-      }
-      if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status, p.wait_cycles, 44)) break;
-      const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
-      float mine = 0.f;
-      // Short gate rows (LoPA: r elements): a row is a few chunks per lane, and with one warp per scheduler the cost is
-      // instruction latency, not throughput.  Eight rows are dotted side by side (eight independent chains, the vector
-      // read once for all of them, every load requested before the first multiply) and reduced together: each
-      // exchange halves the number of sums a lane carries, so eight rows cost 4 + 2 + 1 + 1 + 1 shuffles instead of 40.
-      const int rows_short = nvecK <= 128 ? rows : 0;
-      int rr_short = 0;
-      for (; rows_short - rr_short > 2; rr_short += 8) {  // one or two left-over rows are cheaper one by one (below)
-        const int rr = rr_short;
-        float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int c = lane; c < nvecK; c += 32) {
-          uint4 w[8];
-          float4 v[EPV / 4];
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            w[i] = rr + i < rows ? reinterpret_cast<const uint4*>(base + (size_t)(rr + i) * gate_row_bytes)[c]
-                                 : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-          for (int q = 0; q < EPV / 4; ++q) v[q] = reinterpret_cast<const float4*>(gvec)[q * nvecK + c];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            float f[EPV];
-            Elem<T>::unpack(w[i], f);
-#pragma unroll
-            for (int q = 0; q < EPV / 4; ++q) {
-              a[i] = fmaf(f[4 * q + 0], v[q].x, a[i]);
-              a[i] = fmaf(f[4 * q + 1], v[q].y, a[i]);
-              a[i] = fmaf(f[4 * q + 2], v[q].z, a[i]);
-              a[i] = fmaf(f[4 * q + 3], v[q].w, a[i]);
-            }
-          }
-        }
-        // lanes with bit 4 set keep rows 4..7, the others rows 0..3; then bit 3 picks two of the four, bit 2 one of
-        // the two; bits 1 and 0 are plain sums.  Afterwards lanes 4 k .. 4 k + 3 hold the dot product of row rr + k.
-        float b4[4], b2[2];
-        const bool up16 = lane & 16, up8 = lane & 8, up4 = lane & 4;
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          b4[i] = (up16 ? a[4 + i] : a[i]) + __shfl_xor_sync(0xffffffffu, up16 ? a[i] : a[4 + i], 16);
-#pragma unroll
-        for (int i = 0; i < 2; ++i)
-          b2[i] = (up8 ? b4[2 + i] : b4[i]) + __shfl_xor_sync(0xffffffffu, up8 ? b4[i] : b4[2 + i], 8);
-        float z = (up4 ? b2[1] : b2[0]) + __shfl_xor_sync(0xffffffffu, up4 ? b2[0] : b2[1], 4);
-        z += __shfl_xor_sync(0xffffffffu, z, 2);
-        z += __shfl_xor_sync(0xffffffffu, z, 1);
-        const float got = __shfl_sync(0xffffffffu, z, 4 * ((lane - rr) & 7));
-        if (lane >= rr && lane < rr + 8) mine = got;
-      }
-      for (; rr_short < rows_short; ++rr_short) {
-        const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr_short * gate_row_bytes);
-        float a0 = 0.f;
-        for (int c = lane; c < nvecK; c += 32) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
-        const float z = warp_sum(a0);
-        if (lane == rr_short) mine = z;
-      }
-      int rr_single = rows_short;
-      if (EPV == 16) {
-        // int8 rows: the staged vector is four times the bytes of a row, so two rows share every read of it
-        for (; rr_single + 1 < rows; rr_single += 2) {
-          const uint4* w0 = reinterpret_cast<const uint4*>(base + (size_t)rr_single * gate_row_bytes);
-          const uint4* w1 = reinterpret_cast<const uint4*>(base + (size_t)(rr_single + 1) * gate_row_bytes);
-          float2 a0 = make_float2(0.f, 0.f), a1 = a0, b0 = a0, b1 = a0;
-          int c = lane;
-          for (; c + 32 < nvecK; c += 64) {
-            chunk_dot2_q8(w0[c], w1[c], gvec, c, nvecK, a0, b0);
-            chunk_dot2_q8(w0[c + 32], w1[c + 32], gvec, c + 32, nvecK, a1, b1);
-          }
-          if (c < nvecK) chunk_dot2_q8(w0[c], w1[c], gvec, c, nvecK, a0, b0);
-          const float z0 = warp_sum((a0.x + a0.y) + (a1.x + a1.y)), z1 = warp_sum((b0.x + b0.y) + (b1.x + b1.y));
-          if (lane == rr_single) mine = z0;
-          if (lane == rr_single + 1) mine = z1;
-        }
-      }
-      for (int rr = rr_single; rr < rows; ++rr) {
-        const uint4* w = reinterpret_cast<const uint4*>(base + (size_t)rr * gate_row_bytes);
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        int c = lane;
-        for (; c + 96 < nvecK; c += 128) {
-          const uint4 w0 = w[c], w1 = w[c + 32], w2 = w[c + 64], w3 = w[c + 96];
-          a0 = chunk_dot<T>(w0, gvec, c, nvecK, a0);
-          a1 = chunk_dot<T>(w1, gvec, c + 32, nvecK, a1);
-          a2 = chunk_dot<T>(w2, gvec, c + 64, nvecK, a2);
-          a3 = chunk_dot<T>(w3, gvec, c + 96, nvecK, a3);
-        }
-        for (; c < nvecK; c += 32) a0 = chunk_dot<T>(w[c], gvec, c, nvecK, a0);
-        const float z = warp_sum((a0 + a1) + (a2 + a3));
-        if (lane == rr) mine = z;
-      }
-      if (lane < rows) {
-        const float z = kScaled ? fmaf(mine, scale, add) : mine + add;
-        const bool fired = z > 0.f;
-        if (!p.dense) p.flag[j0 + lane] = fired ? 1 : 0;
-        row_state[r0 + lane] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty_gate + 8 * slot);
-    }
-    if (lane == 0 && gw == (n_gslots - 1) % p.gate_warps) SFFN_STAMP(3);
+    for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_workers)
+      if (!gate_slot(s)) break;
+    if (lane == 0 && gw == (n_gslots - 1) % p.gate_workers) SFFN_STAMP(3);
   } else {
     // ======================= act warps =========================================================
     const int at = tid - 32 * kFAW;  // 0..127
     const int aw = warp - kFAW;
+    // Short gate (LoPA): the act warps have nothing to do until the first fired rows arrive, so they take gate slots
+    // too -- with a dozen warps on it the whole gate is one or two slots per warp.
+    if (LOPA) {
+      for (int s = p.gate_warps + aw; s < n_gslots; s += p.gate_workers)
+        if (p.gate_warps + aw >= p.gate_workers || !gate_slot(s)) break;
+      if (lane == 0 && p.gate_warps + aw == (n_gslots - 1) % p.gate_workers) SFFN_STAMP(3);
+    }
     float acc[CPT][EPV];
 #pragma unroll
     for (int i = 0; i < CPT; ++i)
 #pragma unroll
       for (int e = 0; e < EPV; ++e) acc[i][e] = 0.f;
+    // The entries of the token that this thread's chunks of a W_up row meet, in registers where they fit: the staged
+    // fp32 token is twice the bytes of a bf16 row, and reading it from shared memory for every fired row made the
+    // act warps' round (measured: 0.74 us for two rows at 4096 columns) a matter of shared-memory bandwidth.
+    constexpr bool kXReg = CPT * EPV <= 32;
+    float xr[kXReg ? CPT : 1][EPV];
+    if (kXReg) {
+#pragma unroll
+      for (int i = 0; i < CPT; ++i) {
+        const int c = at + i * kAT;
+#pragma unroll
+        for (int q = 0; q < EPV / 4; ++q) {
+          const float4 v = c < nvecD ? reinterpret_cast<const float4*>(sx)[q * nvecD + c] : make_float4(0.f, 0.f, 0.f, 0.f);
+          xr[i][4 * q] = v.x; xr[i][4 * q + 1] = v.y; xr[i][4 * q + 2] = v.z; xr[i][4 * q + 3] = v.w;
+        }
+      }
+    }
 
     // Two ring slots per round when the second one exists: both rows are dotted before the one
     // four-warp barrier, which halves the serial latency per fired row.  The stop marker always
@@ -735,7 +813,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       const unsigned char* s0 = act_ring + (size_t)slot * p.act_slot_bytes;
       const unsigned char* s1 = act_ring + (size_t)slot1 * p.act_slot_bytes;
       float part0 = 0.f, part1 = 0.f;
-      float2 pk0 = make_float2(0.f, 0.f), pk1 = pk0;  // int8 rows: packed partial sums
+      float2 pk0 = make_float2(0.f, 0.f), pk1 = pk0, pk0b = pk0, pk1b = pk0;  // packed partial sums
       if (a0 >= 0.f) {
         const uint4* wu0 = reinterpret_cast<const uint4*>(s0);
         const uint4* wu1 = reinterpret_cast<const uint4*>(s1);
@@ -746,6 +824,23 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
             if constexpr (EPV == 16) {
               pk0 = chunk_dot_q8(wu0[c], sx, c, nvecD, pk0);
               if (a1 >= 0.f) pk1 = chunk_dot_q8(wu1[c], sx, c, nvecD, pk1);
+            } else if constexpr (kXReg) {
+              // packed FMAs on two pairs of running sums per row: half the instructions, chains a quarter as long
+              float f[EPV];
+              Elem<T>::unpack(wu0[c], f);
+#pragma unroll
+              for (int e = 0; e < EPV; e += 4) {
+                pk0 = fma2(make_float2(f[e], f[e + 1]), make_float2(xr[i][e], xr[i][e + 1]), pk0);
+                pk0b = fma2(make_float2(f[e + 2], f[e + 3]), make_float2(xr[i][e + 2], xr[i][e + 3]), pk0b);
+              }
+              if (a1 >= 0.f) {
+                Elem<T>::unpack(wu1[c], f);
+#pragma unroll
+                for (int e = 0; e < EPV; e += 4) {
+                  pk1 = fma2(make_float2(f[e], f[e + 1]), make_float2(xr[i][e], xr[i][e + 1]), pk1);
+                  pk1b = fma2(make_float2(f[e + 2], f[e + 3]), make_float2(xr[i][e + 2], xr[i][e + 3]), pk1b);
+                }
+              }
             } else {
               part0 = chunk_dot<T>(wu0[c], sx, c, nvecD, part0);
               if (a1 >= 0.f) part1 = chunk_dot<T>(wu1[c], sx, c, nvecD, part1);
@@ -755,6 +850,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         if constexpr (EPV == 16) {
           part0 = pk0.x + pk0.y;
           part1 = pk1.x + pk1.y;
+        } else if constexpr (kXReg) {
+          part0 = (pk0.x + pk0.y) + (pk0b.x + pk0b.y);
+          part1 = (pk1.x + pk1.y) + (pk1b.x + pk1b.y);
         }
         part0 = warp_sum(part0);
         part1 = warp_sum(part1);
@@ -789,29 +887,19 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         if (c < nvecD) {
           float f[EPV];
           Elem<T>::unpack(wd0[c], f);
-          if constexpr (EPV == 16) {
 #pragma unroll
-            for (int e = 0; e < EPV; e += 2) {
-              const float2 t = fma2(make_float2(h0, h0), make_float2(f[e], f[e + 1]), make_float2(acc[i][e], acc[i][e + 1]));
-              acc[i][e] = t.x;
-              acc[i][e + 1] = t.y;
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h0, f[e], acc[i][e]);
+          for (int e = 0; e < EPV; e += 2) {
+            const float2 t = fma2(make_float2(h0, h0), make_float2(f[e], f[e + 1]), make_float2(acc[i][e], acc[i][e + 1]));
+            acc[i][e] = t.x;
+            acc[i][e + 1] = t.y;
           }
           if (a1 >= 0.f) {
             Elem<T>::unpack(wd1[c], f);
-            if constexpr (EPV == 16) {
 #pragma unroll
-              for (int e = 0; e < EPV; e += 2) {
-                const float2 t = fma2(make_float2(h1, h1), make_float2(f[e], f[e + 1]), make_float2(acc[i][e], acc[i][e + 1]));
-                acc[i][e] = t.x;
-                acc[i][e + 1] = t.y;
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < EPV; ++e) acc[i][e] = fmaf(h1, f[e], acc[i][e]);
+            for (int e = 0; e < EPV; e += 2) {
+              const float2 t = fma2(make_float2(h1, h1), make_float2(f[e], f[e + 1]), make_float2(acc[i][e], acc[i][e + 1]));
+              acc[i][e] = t.x;
+              acc[i][e + 1] = t.y;
             }
           }
         }
@@ -939,7 +1027,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
 // ---- host side --------------------------------------------------------------------------------
 struct Geometry {
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max, smem, cpt;
-  int gate_warps;
+  int gate_warps, gate_workers;
+  bool v_in_smem;  // LoPA: the CTA's rows of V are copied into the idle act ring ahead of the rank-r stage
   bool ok;
 };
 
@@ -1008,6 +1097,21 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   }
   g.n_act_slots = na;
   g.n_gate_slots = ng;
+  // the rank-r stage keeps the CTA's rows of V and one sum per 32-chunk segment of them in the (then idle) act ring
+  g.v_in_smem = false;
+  if (lopa) {
+    const size_t v_max = (size_t)(K + grid - 1) / grid, sums = (v_max * ((nvecD + 31) / 32) + 32) * 4;
+    if (sums > (size_t)na * g.act_slot_bytes) return g;
+    g.v_in_smem = v_max * row_bytes + sums <= (size_t)na * g.act_slot_bytes;
+  }
+  // Warps that take gate slots.  When the CTA's whole share of the gate rows sits in the ring at once (a short gate), the
+  // act warps take slots too: they would idle until the first fired rows arrive.  A longer gate stays with the gate
+  // warps (measured at r = 1024: act warps that are busy with gate slots drain the act ring too late).
+  g.gate_workers = gw;
+  if (lopa) {
+    const int most = gw + 8;  // the eight act warps of the LoPA kernel
+    if (slots_of_cta <= ng) g.gate_workers = slots_of_cta < gw ? gw : slots_of_cta > most ? most : slots_of_cta;
+  }
   const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max, scaled);
   g.smem = full.total;
   g.ok = g.smem <= kSmemBudget;
@@ -1091,7 +1195,6 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   const Geometry g = plan(c.wkind, c.D, c.H, K, lopa, grid);
   if (!g.ok) return cudaErrorInvalidValue;
   char* ws = static_cast<char*>(c.workspace);
-  float* vbuf = reinterpret_cast<float*>(ws + 256 + (size_t)kMaxGrid * c.D * 4);
   int n = 0;
   cudaError_t e;
   FusedParams p{};
@@ -1101,9 +1204,8 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.g_idx = lopa ? c.gate->g_idx : nullptr; p.g_sign = c.gate->g_sign;
   p.gain = c.gate->rms_gain; p.use_rmsnorm = c.gate->use_rmsnorm; p.eps = c.gate->rms_eps;
   p.V = c.gate->V;
-  p.vbuf = vbuf;
-  p.v_counter = reinterpret_cast<unsigned long long*>(ws);
-  p.done_counter = p.v_counter + 1;
+  p.vtag = reinterpret_cast<unsigned long long*>(ws + 256);
+  p.done_counter = reinterpret_cast<unsigned long long*>(ws) + 1;
   p.y = c.y;
   p.partial = reinterpret_cast<unsigned long long*>(ws + fused_tagged_partials_offset(c.D, c.r_max));
   p.epoch_word = reinterpret_cast<uint32_t*>(ws + 16);
@@ -1114,7 +1216,7 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;
-  p.gate_warps = g.gate_warps;
+  p.gate_warps = g.gate_warps; p.gate_workers = g.gate_workers; p.v_in_smem = g.v_in_smem ? 1 : 0;
   p.wait_cycles = fused_test_knobs().wait_cycles;
   p.skip_arrival_cta = fused_test_knobs().skip_arrival_cta;
   p.trace = fused_test_knobs().trace;
