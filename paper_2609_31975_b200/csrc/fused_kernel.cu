@@ -82,6 +82,7 @@ struct FusedParams {
   uint8_t* flag;
   int32_t* status;
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
+  int act_extra;     // LoPA: act slots inside the gate ring, used once the gate is done (0 = none)
   int v_in_smem;     // LoPA: this CTA's rows of V are copied into the (idle) act ring at the start of the call
   int gate_workers;  // warps that take gate slots, slot s going to worker s % gate_workers: the gate warps, and for
                      // the LoPA gate also act warps (a ring slot that is reused always belongs to the same worker)
@@ -96,7 +97,7 @@ struct FusedParams {
 struct SmemLayout {
   int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, row_params, row_scales, slot_scales, total;
   __host__ __device__ SmemLayout(int D, int K, bool lopa, int n_gate_slots, int gate_slot_bytes,
-                                 int n_act_slots, int act_slot_bytes, int slab_max, bool scaled) {
+                                 int n_act_slots, int act_slot_bytes, int slab_max, bool scaled, int act_extra = 0) {
     int off = 0;
     auto take = [&](int bytes) {
       int o = off;
@@ -108,18 +109,18 @@ struct SmemLayout {
     sx = take(D * 4);
     sn = take(lopa ? K * 4 : 0);
     aval = take(slab_max * 4);
-    slot_a = take(n_act_slots * 4);
-    red = take(2 * (2 * 8 + 1) * 4);  // up to eight act warps
+    slot_a = take((n_act_slots + act_extra) * 4);
+    red = take(4 * (2 * 4 + 1) * 4);  // two buffers per act group (four warps each), up to two groups
     ctl = take(8 * 4);
-    bars = take(2 * (n_gate_slots + n_act_slots) * 8 + 8);  // + one for the CTA's rows of V (LoPA)
+    bars = take(2 * (n_gate_slots + n_act_slots + act_extra) * 8 + 8);  // + one for the CTA's rows of V (LoPA)
     row_params = take((lopa || scaled) ? (1 + (lopa ? 2 : 0) + (scaled ? 1 : 0)) * slab_max * 4 : 0);  // per-neuron gate parameters
     row_scales = take(scaled ? 2 * slab_max * 4 : 0);     // int8 rows: scales of the slab's W_up / W_down rows
-    slot_scales = take(scaled ? 2 * n_act_slots * 4 : 0);  // the same two for the row in each act slot
+    slot_scales = take(scaled ? 2 * (n_act_slots + act_extra) * 4 : 0);  // the same two for the row in each act slot
     total = off;
   }
 };
 
-enum Ctl { kAbort = 0, kRank = 1 };
+enum Ctl { kAbort = 0, kRank = 1, kGateDone = 2 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -297,6 +298,14 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   constexpr int kGW = kGateWarps + kActWarps - kAW;         // gate warps
   constexpr int kFAW = kFirstGateWarp + kGW;                // first act warp
   constexpr int kAT = 32 * kAW;                             // act threads
+  // The act warps work in groups of four; a group takes whole rounds (two ring slots) by itself.  With the short LoPA
+  // gate the act stage is what a call waits for, and one round is a chain of latencies (shared-memory loads, shuffles,
+  // a barrier, loads again: 0.7 us for two rows however many warps share it), so two groups on alternate rounds double
+  // the rows per microsecond; each keeps its own sums, added through shared memory at the end.
+  constexpr int kGroups = LOPA ? 2 : 1;
+  constexpr int kGAW = kAW / kGroups;                       // warps of a group
+  constexpr int kGT = 32 * kGAW;                            // threads of a group
+  static_assert(kGAW == 4, "the up projection's sum over a group's warps is written out for four");
   static_assert(kGW >= 2, "gate warps");
 
   extern __shared__ __align__(128) unsigned char smem[];
@@ -311,11 +320,17 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x, cta = blockIdx.x;
   const int D = p.D, K = p.K;
-  const int NG = p.n_gate_slots, NA = p.n_act_slots;
-  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NA, p.act_slot_bytes, p.slab_max, kScaled);
+  // Act slots: NAown in the act ring, plus (short LoPA gate) p.act_extra more that lie in the gate ring and come into
+  // use once every gate row has been consumed -- from then on the rows of fired neurons are all that is left to
+  // fetch, and how many of them are in flight sets how fast they come.
+  const int NG = p.n_gate_slots, NAown = p.n_act_slots, NA = NAown + p.act_extra;
+  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra);
 
   unsigned char* gate_ring = smem + L.gate_ring;
   unsigned char* act_ring = smem + L.act_ring;
+  auto act_slot = [&](int sl) -> unsigned char* {
+    return sl < NAown ? act_ring + (size_t)sl * p.act_slot_bytes : gate_ring + (size_t)(sl - NAown) * p.act_slot_bytes;
+  };
   float* sx = reinterpret_cast<float*>(smem + L.sx);
   float* sn = reinterpret_cast<float*>(smem + L.sn);
   // One word per neuron of the slab, written once by a gate warp and polled by the act producers:
@@ -371,11 +386,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
       for (int s = 0; s < NA; ++s) {
         mbar_init(full_act + 8 * s, kActProducers);
-        mbar_init(empty_act + 8 * s, kAW);
+        mbar_init(empty_act + 8 * s, kGAW);
       }
       mbar_init(v_bar, 1);
       for (int i = 0; i < 8; ++i) ctl[i] = 0;
-      for (int i = 0; i < 2 * (2 * kAW + 1); ++i) red[i] = 0.f;
+      for (int i = 0; i < 4 * (2 * 4 + 1); ++i) red[i] = 0.f;
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -480,7 +495,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     float* wss = reinterpret_cast<float*>(act_ring + (p.v_in_smem ? (size_t)v_max * row_bytes : 0));
     float* vpart = wss + 32;
     named_bar_sync(5, kStageThreads);  // the token is staged
-    if (st == 0) SFFN_STAMP(15);
     mbar_wait(v_bar, 0, ctl, p.status, p.wait_cycles, 50);
     const int nseg = (nvecD + 31) / 32, items = (vhi - vlo) * nseg;  // fits the act ring: checked on the host
     for (int it = sw; it < items; it += kSW) {
@@ -489,7 +503,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       if (lane == 0) vpart[it] = a;
     }
     named_bar_sync(5, kStageThreads);
-    if (st == 0) SFFN_STAMP(9);
     for (int k = vlo + st; k < vhi; k += kStageThreads) {
       float v = 0.f;
       for (int g = 0; g < nseg; ++g) v += vpart[(k - vlo) * nseg + g];
@@ -519,7 +532,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       if (k1 < r) sn[vec_pos<EPV>(k1, r)] = v1;
     }
     // n = RMSNorm(v) (or v): the warps' sums of squares are added in a fixed order by everyone
-    if (st == 0) SFFN_STAMP(14);
     ss = warp_sum(ss);
     if (lane == 0) wss[sw] = ss;
     named_bar_sync(5, kStageThreads);
@@ -557,7 +569,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
     }
     if (!mbar_wait(full_gate + 8 * slot, (s / NG) & 1, ctl, p.status, p.wait_cycles, 44)) return false;
-    if (lane == 0 && s == 0) SFFN_STAMP(7);
     const unsigned char* base = gate_ring + (size_t)slot * p.gate_slot_bytes;
     float mine = 0.f;
     // Short gate rows (LoPA: r elements): a row is a few chunks per lane, and with one warp per scheduler the cost is
@@ -654,8 +665,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       row_state[r0 + lane] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(empty_gate + 8 * slot);
-    if (lane == 0 && s == 0) SFFN_STAMP(6);
+    if (lane == 0) {
+      mbar_arrive(empty_gate + 8 * slot);
+      if (p.act_extra) atomicAdd(const_cast<int*>(ctl) + kGateDone, 1);  // this slot's rows have been read
+    }
     return true;
   };
 
@@ -665,10 +678,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // fired neuron, producer 1 its W_down row, into the same ring slot.
     const int ap = warp - kFirstActProducer;
     const char* Wsrc = static_cast<const char*>(ap == 0 ? p.W_up : p.W_down);
-    const uint32_t ring = smem_u32(act_ring) + (ap == 0 ? 0u : (uint32_t)row_bytes);
     int slot = 0;
     uint32_t par = 1;
     bool ok = true;
+    int n_seq = 0;  // ring slots handed out so far
     // The whole warp classifies 32 rows per step (one shared-memory read + ballots); lane 0 issues
     // the copies of the fired ones in ascending order.  Only the leading run of finished rows is
     // consumed, so the order never depends on which gate warp was faster.
@@ -704,7 +717,17 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
           int ms = slot + place;
           uint32_t mp = par;
           if (ms >= NA) { ms -= NA; mp ^= 1; }
-          if (mbar_wait<true>(empty_act + 8 * ms, mp, ctl, p.status, p.wait_cycles, 42)) {
+          bool free_slot = mbar_wait<true>(empty_act + 8 * ms, mp, ctl, p.status, p.wait_cycles, 42);
+          if (free_slot && ms >= NAown && n_seq + place < NA) {
+            // first use of a slot inside the gate ring: not before the gate warps have read every gate row
+            const long long t0 = clock64();
+            while (ctl[kGateDone] < n_gslots) {
+              if (ctl[kAbort]) { free_slot = false; break; }
+              if (clock64() - t0 > p.wait_cycles) { raise_timeout(ctl, p.status, 51); free_slot = false; break; }
+              __nanosleep(40);
+            }
+          }
+          if (free_slot) {
             if (ap == 0) slot_a[ms] = st == 0x80000000u ? 0.f : __uint_as_float(st);
             if (kScaled && ap == 0) {
               slot_su[ms] = row_su[row];
@@ -712,8 +735,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
             }
             const size_t j = (size_t)(slot_first_neuron(row / nr) + row % nr);
             mbar_expect_tx(full_act + 8 * ms, (uint32_t)row_bytes);
-            bulk_g2s(ring + (uint32_t)ms * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
-                     full_act + 8 * ms);
+            bulk_g2s(smem_u32(act_slot(ms)) + (ap == 0 ? 0u : (uint32_t)row_bytes), Wsrc + j * row_bytes,
+                     (uint32_t)row_bytes, full_act + 8 * ms);
           } else {
             good = false;
           }
@@ -724,13 +747,26 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         n_issued += nb;
 #endif
         slot += nb;
+        n_seq += nb;
         if (slot >= NA) { slot -= NA; par ^= 1; }
       }
       base += prefix;
     }
-    if (lane == 0 && ok && mbar_wait<true>(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 43)) {
-      if (ap == 0) slot_a[slot] = -1.f;      // stop marker: a negative gate value
-      mbar_arrive(full_act + 8 * slot);      // completes the phase without data
+    // Stop markers (a negative gate value, the phase completed without data): every act group meets one in the first
+    // slot of the round it would take next.
+    if (lane == 0 && ap == 0) SFFN_STAMP(7);
+    if (lane == 0) {
+      const int per_round = NA >= 4 ? 2 : 1;
+      const int n_end = kGroups == 1 ? n_seq + 1 : (n_seq / per_round + kGroups) * per_round;
+      for (; ok && n_seq < n_end; ++n_seq) {
+        if (mbar_wait<true>(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 43)) {
+          if (ap == 0) slot_a[slot] = -1.f;
+          mbar_arrive(full_act + 8 * slot);
+        } else {
+          ok = false;
+        }
+        if (++slot == NA) { slot = 0; par ^= 1; }
+      }
     }
     if (ap == 0) {
       // This CTA's place in the order of finishing (the first R sum the partials), taken now so that the round trip
@@ -759,8 +795,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     if (lane == 0 && gw == (n_gslots - 1) % p.gate_workers) SFFN_STAMP(3);
   } else {
     // ======================= act warps =========================================================
-    const int at = tid - 32 * kFAW;  // 0..127
+    const int at = tid - 32 * kFAW;
     const int aw = warp - kFAW;
+    const int grp = aw / kGAW, gaw = aw % kGAW, gat = at % kGT;  // act group, warp and thread within it
     // Short gate (LoPA): the act warps have nothing to do until the first fired rows arrive, so they take gate slots
     // too -- with a dozen warps on it the whole gate is one or two slots per warp.
     if (LOPA) {
@@ -781,7 +818,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     if (kXReg) {
 #pragma unroll
       for (int i = 0; i < CPT; ++i) {
-        const int c = at + i * kAT;
+        const int c = gat + i * kGT;
 #pragma unroll
         for (int q = 0; q < EPV / 4; ++q) {
           const float4 v = c < nvecD ? reinterpret_cast<const float4*>(sx)[q * nvecD + c] : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -795,23 +832,25 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // arrives, so waiting for the second slot of a round cannot block for good.  A thread whose
     // wait ran out still joins the barrier and raises the group's stop flag, so the four warps
     // always leave the loop together.
-    int slot = 0;
+    const bool pair = NA >= 4;  // with fewer slots, holding two at a time would stall the act producers
+    const int stride = (pair ? 2 : 1) * kGroups;  // ring slots from one round of a group to its next
+    int slot = (pair ? 2 : 1) * grp;
     uint32_t par = 0;
+    while (slot >= NA) { slot -= NA; par ^= 1; }
     for (int round = 0;; ++round) {
-      float* rp = red + (round & 1) * (2 * kAW + 1);
+      float* rp = red + (2 * grp + (round & 1)) * (2 * kGAW + 1);
       const int slot1 = slot + 1 == NA ? 0 : slot + 1;
       const uint32_t par1 = slot + 1 == NA ? par ^ 1 : par;
       const bool got0 = mbar_wait(full_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 45);
       const float a0 = got0 ? slot_a[slot] : -1.f;
       bool got1 = true;
       float a1 = -1.f;
-      const bool pair = NA >= 4;  // with fewer slots, holding two at a time would stall the act producers
       if (pair && a0 >= 0.f) {
         got1 = mbar_wait(full_act + 8 * slot1, par1, ctl, p.status, p.wait_cycles, 46);
         a1 = got1 ? slot_a[slot1] : -1.f;
       }
-      const unsigned char* s0 = act_ring + (size_t)slot * p.act_slot_bytes;
-      const unsigned char* s1 = act_ring + (size_t)slot1 * p.act_slot_bytes;
+      const unsigned char* s0 = act_slot(slot);
+      const unsigned char* s1 = act_slot(slot1);
       float part0 = 0.f, part1 = 0.f;
       float2 pk0 = make_float2(0.f, 0.f), pk1 = pk0, pk0b = pk0, pk1b = pk0;  // packed partial sums
       if (a0 >= 0.f) {
@@ -819,7 +858,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         const uint4* wu1 = reinterpret_cast<const uint4*>(s1);
 #pragma unroll
         for (int i = 0; i < CPT; ++i) {
-          const int c = at + i * kAT;
+          const int c = gat + i * kGT;
           if (c < nvecD) {
             if constexpr (EPV == 16) {
               pk0 = chunk_dot_q8(wu0[c], sx, c, nvecD, pk0);
@@ -857,19 +896,15 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         part0 = warp_sum(part0);
         part1 = warp_sum(part1);
         if (lane == 0) {
-          rp[aw] = part0;
-          rp[kAW + aw] = part1;
+          rp[gaw] = part0;
+          rp[kGAW + gaw] = part1;
         }
       }
-      if (a0 < 0.f || !got1) rp[2 * kAW] = 1.f;  // stop marker first in the round, or a failed wait
-      named_bar_sync(2, kAT);
-      if (rp[2 * kAW] != 0.f) break;
+      if (a0 < 0.f || !got1) rp[2 * kGAW] = 1.f;  // stop marker first in the round, or a failed wait
+      named_bar_sync(2 + 6 * grp, kGT);
+      if (rp[2 * kGAW] != 0.f) break;
       float u0 = (rp[0] + rp[1]) + (rp[2] + rp[3]);
-      float u1 = (rp[kAW] + rp[kAW + 1]) + (rp[kAW + 2] + rp[kAW + 3]);
-      if (kAW == 8) {
-        u0 += (rp[4] + rp[5]) + (rp[6] + rp[7]);
-        u1 += (rp[kAW + 4] + rp[kAW + 5]) + (rp[kAW + 6] + rp[kAW + 7]);
-      }
+      float u1 = (rp[kGAW] + rp[kGAW + 1]) + (rp[kGAW + 2] + rp[kGAW + 3]);
       if (kScaled) {  // int8 rows: u = s_up (codes . x); the W_down row's scale rides on h
         u0 *= slot_su[slot];
         u1 *= slot_su[slot1];
@@ -883,7 +918,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       const uint4* wd1 = reinterpret_cast<const uint4*>(s1 + row_bytes);
 #pragma unroll
       for (int i = 0; i < CPT; ++i) {
-        const int c = at + i * kAT;
+        const int c = gat + i * kGT;
         if (c < nvecD) {
           float f[EPV];
           Elem<T>::unpack(wd0[c], f);
@@ -906,28 +941,44 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_act + 8 * slot);
-      if (!pair) {
-        if (++slot == NA) { slot = 0; par ^= 1; }
-        continue;
+      if (pair) {
+        if (a1 < 0.f) break;  // the second slot was the stop marker
+        if (lane == 0) mbar_arrive(empty_act + 8 * slot1);
       }
-      if (a1 < 0.f) break;  // the second slot was the stop marker
-      if (lane == 0) mbar_arrive(empty_act + 8 * slot1);
-      slot = slot1 + 1 == NA ? 0 : slot1 + 1;
-      par = slot1 + 1 == NA ? par1 ^ 1 : par1;
+      slot += stride;
+      while (slot >= NA) { slot -= NA; par ^= 1; }
     }
     if (at == 0) SFFN_STAMP(4);
+    if (kGroups == 2) {
+      // the second group's sums go to the first through the act ring, once both groups have left it
+      float* xch = reinterpret_cast<float*>(act_ring);
+      named_bar_sync(9, kAT);
+      if (grp == 1) {
+#pragma unroll
+        for (int i = 0; i < CPT; ++i)
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) xch[(i * EPV + e) * kGT + gat] = acc[i][e];
+      }
+      named_bar_sync(9, kAT);
+      if (grp == 0) {
+#pragma unroll
+        for (int i = 0; i < CPT; ++i)
+#pragma unroll
+          for (int e = 0; e < EPV; ++e) acc[i][e] += xch[(i * EPV + e) * kGT + gat];
+      }
+    }
     // This CTA's partial of y, every value tagged with the call's number.  Stored unit (two columns, 16 bytes)
-    // (i * EPV / 2 + e) * kAT + at holds columns EPV (at + i kAT) + 2 e and the next one: a warp's store is 512
+    // (i * EPV / 2 + e) * kGT + gat holds columns EPV (gat + i kGT) + 2 e and the next one: a warp's store is 512
     // contiguous bytes; the summing threads undo the permutation when they write y.
-    if (cta != p.skip_arrival_cta) {
+    if (cta != p.skip_arrival_cta && grp == 0) {
       const uint64_t keep = policy_evict_last();  // the partials are rewritten by every call: they should stay in L2
-      unsigned long long* dst = p.partial + (size_t)cta * (CPT * EPV * kAT);
+      unsigned long long* dst = p.partial + (size_t)cta * (CPT * EPV * kGT);
 #pragma unroll
       for (int i = 0; i < CPT; ++i) {
-        if (at + i * kAT < nvecD) {
+        if (gat + i * kGT < nvecD) {
 #pragma unroll
           for (int e = 0; e < EPV / 2; ++e)
-            st_tagged2(dst + 2 * (size_t)((i * (EPV / 2) + e) * kAT + at), tagged(acc[i][2 * e], ep),
+            st_tagged2(dst + 2 * (size_t)((i * (EPV / 2) + e) * kGT + gat), tagged(acc[i][2 * e], ep),
                        tagged(acc[i][2 * e + 1], ep), keep);
         }
       }
@@ -946,7 +997,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   // and their SMs take the next kernel of the stream.
   if (warp < kFirstGateWarp) return;  // act producers (the gate producers left long ago)
   constexpr int kTail = 32 * (kGW + kAW);
-  constexpr int kRow = CPT * EPV * kAT;        // values of a stored partial
+  constexpr int kRow = CPT * EPV * kGT;        // values of a stored partial
   constexpr int kUnits = kRow / 2;             // two columns each (a multiple of 32; those past D are never written)
   const int tt = tid - 32 * kFirstGateWarp;    // index among the tail threads
   // never more than half the grid stays, so that the waiting CTAs of two calls that overlap (two handles on two
@@ -966,7 +1017,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const int RG = kTail / UW;
   const int u = tt % UW, rg = tt / UW;
   auto first_column = [&](int unit) {  // undoes the permutation of the stored units
-    return EPV * ((unit % kAT) + (unit / ((EPV / 2) * kAT)) * kAT) + 2 * ((unit / kAT) % (EPV / 2));
+    return EPV * ((unit % kGT) + (unit / ((EPV / 2) * kGT)) * kGT) + 2 * ((unit / kGT) % (EPV / 2));
   };
   bool ok = true;
   for (int u0 = 0; u0 < U; u0 += UW) {
@@ -1028,6 +1079,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
 struct Geometry {
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max, smem, cpt;
   int gate_warps, gate_workers;
+  int act_extra;   // LoPA: act slots inside the gate ring (used once the gate is done)
   bool v_in_smem;  // LoPA: the CTA's rows of V are copied into the idle act ring ahead of the rank-r stage
   bool ok;
 };
@@ -1039,7 +1091,7 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   const int nvecD = D / epv;
   const int row_bytes = D * esz, gate_row_bytes = K * esz;
   g.ok = false;
-  const int act_threads = lopa ? 256 : 128;    // as in the kernel: eight act warps for the LoPA gate
+  const int act_threads = 128;                 // as in the kernel: the threads of one act group
   const int gate_warps_max = lopa ? 4 : 8;
   if (row_bytes % 16 || gate_row_bytes % 16 || nvecD > act_threads * 8) return g;
   g.cpt = nvecD <= act_threads ? 1 : nvecD <= 2 * act_threads ? 2 : nvecD <= 4 * act_threads ? 4 : 8;
@@ -1099,6 +1151,14 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   g.n_gate_slots = ng;
   // the rank-r stage keeps the CTA's rows of V and one sum per 32-chunk segment of them in the (then idle) act ring
   g.v_in_smem = false;
+  // the two act groups of the LoPA kernel add their sums through the act ring
+  if (lopa && (size_t)na * g.act_slot_bytes < (size_t)g.cpt * epv * act_threads * 4) return g;
+  // a short gate leaves the gate ring idle early: it then holds more act slots
+  g.act_extra = 0;
+  if (lopa && slots_of_cta <= ng) {
+    g.act_extra = (int)((size_t)ng * g.gate_slot_bytes / g.act_slot_bytes);
+    if (na + g.act_extra > 16) g.act_extra = 16 - na;
+  }
   if (lopa) {
     const size_t v_max = (size_t)(K + grid - 1) / grid, sums = (v_max * ((nvecD + 31) / 32) + 32) * 4;
     if (sums > (size_t)na * g.act_slot_bytes) return g;
@@ -1112,7 +1172,7 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
     const int most = gw + 8;  // the eight act warps of the LoPA kernel
     if (slots_of_cta <= ng) g.gate_workers = slots_of_cta < gw ? gw : slots_of_cta > most ? most : slots_of_cta;
   }
-  const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max, scaled);
+  const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max, scaled, g.act_extra);
   g.smem = full.total;
   g.ok = g.smem <= kSmemBudget;
   return g;
@@ -1216,7 +1276,7 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;
-  p.gate_warps = g.gate_warps; p.gate_workers = g.gate_workers; p.v_in_smem = g.v_in_smem ? 1 : 0;
+  p.gate_warps = g.gate_warps; p.gate_workers = g.gate_workers; p.v_in_smem = g.v_in_smem ? 1 : 0; p.act_extra = g.act_extra;
   p.wait_cycles = fused_test_knobs().wait_cycles;
   p.skip_arrival_cta = fused_test_knobs().skip_arrival_cta;
   p.trace = fused_test_knobs().trace;
