@@ -65,7 +65,9 @@ typedef enum {
   SFFN_ERR_UNSUPPORTED = 2, /* misaligned pointer, row size not a multiple of 16 bytes, too big */
   SFFN_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small                       */
   SFFN_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch, copy)                        */
-  SFFN_ERR_TIMEOUT = 5      /* device status only: a bounded device-side wait gave up           */
+  SFFN_ERR_TIMEOUT = 5,     /* device status only: a bounded device-side wait gave up           */
+  SFFN_ERR_BOUNDS = 6       /* device status only, debug builds (-DSFFN_DEBUG): an index that was about to address
+                               global memory lay outside its array; the access was skipped or clamped */
 } sffn_status;
 
 /* Activation A of Eq. 1.  RELU and R-S+ follow the table of Sec. 3.1 (R-S+: 0 for z < 0,
@@ -290,12 +292,16 @@ const char* sffn_status_string(int status);
  *                       prefetches into idle act slots at the start of a call (0, 0, -1 = planned)
  *   L2_HINTS            tensor-core gate kernel: bit 0 = weights are fetched evict-first, bit 1 = the per-CTA partial
  *                       results are stored evict-last (default 2)
+ *   POISON_LIST         debug builds (-DSFFN_DEBUG) only, SFFN_ERR_UNSUPPORTED otherwise: 1 = the CUDA-core path
+ *                       overwrites the first entry of its list of fired neurons with a number far beyond H before
+ *                       the up / down kernel reads it, so that the kernel's index check has something to find (it
+ *                       records SFFN_ERR_BOUNDS and takes row 0 instead; the bad index is never used as an address)
  *   TRACE_BUFFER        device address of [grid][16] int64 time stamps, written only by libraries built with
  *                       -DSFFN_TRACE (0 = none) */
 typedef enum {
   SFFN_KNOB_PDL = 0, SFFN_KNOB_TENSOR_GATE = 1, SFFN_KNOB_WAIT_CYCLES = 2, SFFN_KNOB_SKIP_ARRIVAL_CTA = 3,
   SFFN_KNOB_RING_GATE_SLOTS = 4, SFFN_KNOB_RING_ACT_SLOTS = 5, SFFN_KNOB_TRACE_BUFFER = 6,
-  SFFN_KNOB_RING_PARKED_STAGES = 7, SFFN_KNOB_L2_HINTS = 8, SFFN_KNOB_DROP_STAGE = 9
+  SFFN_KNOB_RING_PARKED_STAGES = 7, SFFN_KNOB_L2_HINTS = 8, SFFN_KNOB_DROP_STAGE = 9, SFFN_KNOB_POISON_LIST = 10
 } sffn_test_knob;
 void sffn_test_fused_plan(int wkind, int D, int H, int K, int lopa, int sm_count, int* out9);
 void sffn_test_umma_tiling(int R, int sm_count, int* tile_rows, int* n_tiles, int* own_list);

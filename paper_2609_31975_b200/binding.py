@@ -12,7 +12,7 @@ ACT_UP = dict(ACT, silu=4)  # activations of the up projection (double activatio
 PATH = {"auto": 0, "general": 1, "fused": 2, "mma_sync": 3}
 _STATUS = {0: "ok", 1: "invalid argument", 2: "unsupported shape, alignment or path",
            3: "workspace missing, misaligned or too small", 4: "CUDA runtime error",
-           5: "device-side bounded wait ran out"}
+           5: "device-side bounded wait ran out", 6: "debug build: index outside its array"}
 
 
 class SFFNError(RuntimeError):
@@ -89,7 +89,8 @@ def load_library() -> ctypes.CDLL:
 
 GATE_ENGINE = {"auto": 0, "cuda_core": 1, "tensor_core": 2}
 KNOB = {"pdl": 0, "tensor_gate": 1, "wait_cycles": 2, "skip_arrival_cta": 3, "ring_gate_slots": 4,
-        "ring_act_slots": 5, "trace_buffer": 6, "ring_parked_stages": 7, "l2_hints": 8, "drop_stage": 9}
+        "ring_act_slots": 5, "trace_buffer": 6, "ring_parked_stages": 7, "l2_hints": 8, "drop_stage": 9,
+        "poison_list": 10}
 
 
 def test_set_knob(name: str, value: int):

@@ -2,7 +2,10 @@
 
 Every source file is compiled to an object of its own (in parallel, only when it or a header changed) and the
 objects are linked into the shared library.  `python -m paper_2609_31975_b200.build --trace` builds a second
-library, libsparse_ffn_trace.so, whose single-token kernels write time stamps (see SFFN_KNOB_TRACE_BUFFER)."""
+library, libsparse_ffn_trace.so, whose single-token kernels write time stamps (see SFFN_KNOB_TRACE_BUFFER);
+`--debug` builds libsparse_ffn_debug.so (-DSFFN_DEBUG), whose kernels check the indices they address global memory
+with and report SFFN_ERR_BOUNDS in the device status instead of making the access.  Either is selected at run time
+with the environment variable SFFN_LIBRARY."""
 from __future__ import annotations
 
 import os
@@ -25,18 +28,20 @@ def _headers_mtime() -> float:
     return max(d.stat().st_mtime for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, trace: bool = False) -> Path:
-    lib = PKG / "libsparse_ffn_trace.so" if trace else LIB
+def build(force: bool = False, verbose: bool = False, trace: bool = False, debug: bool = False) -> Path:
+    lib = PKG / "libsparse_ffn_trace.so" if trace else PKG / "libsparse_ffn_debug.so" if debug else LIB
     newest = max(_headers_mtime(), max((CSRC / s).stat().st_mtime for s in SOURCES))
     if not force and lib.exists() and lib.stat().st_mtime >= newest:
         return lib
-    objdir = OBJ / ("trace" if trace else "plain")
+    objdir = OBJ / ("trace" if trace else "debug" if debug else "plain")
     objdir.mkdir(parents=True, exist_ok=True)
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
              "-I", str(ROOT / "include"), "-I", str(CSRC)]
     if trace:
         flags += ["-DSFFN_TRACE"]
+    if debug:
+        flags += ["-DSFFN_DEBUG"]
     if verbose:
         flags += ["-Xptxas", "-v"]
     hdr = _headers_mtime()
@@ -69,4 +74,4 @@ def build(force: bool = False, verbose: bool = False, trace: bool = False) -> Pa
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv, debug="--debug" in sys.argv))

@@ -90,6 +90,7 @@ const char* sffn_status_string(int s) {
     case SFFN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case SFFN_ERR_CUDA: return "CUDA runtime error";
     case SFFN_ERR_TIMEOUT: return "device-side bounded wait ran out";
+    case SFFN_ERR_BOUNDS: return "debug build: index outside its array";
     default: return "unknown status";
   }
 }
@@ -179,6 +180,13 @@ int sffn_test_set_knob(int knob, long long value) {
     case SFFN_KNOB_RING_PARKED_STAGES: k.ring_E = (int)value; return SFFN_OK;
     case SFFN_KNOB_L2_HINTS: k.l2_hints = (int)value; return SFFN_OK;
     case SFFN_KNOB_DROP_STAGE: k.drop_stage = (int)value; return SFFN_OK;
+    case SFFN_KNOB_POISON_LIST:
+#ifdef SFFN_DEBUG
+      k.poison_list = value != 0;
+      return SFFN_OK;
+#else
+      return value ? SFFN_ERR_UNSUPPORTED : SFFN_OK;
+#endif
     case SFFN_KNOB_TRACE_BUFFER: k.trace = reinterpret_cast<long long*>(static_cast<uintptr_t>(value)); return SFFN_OK;
     default: return SFFN_ERR_INVALID_ARG;
   }
@@ -316,6 +324,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       SFFN_CUDA(launch_umma_rows(false, p, cols, h->sm_count, s));
     } else {
       RowsMmaParams p{};
+      p.status = h->at<int32_t>(h->L.status);
       p.R = H; p.B = nb; p.b_g = b_g; p.act = act;
       p.xtok = xtok; p.xtok_stride = D;
       p.a_out = actbuf + (size_t)b0 * H; p.a_stride = H;
@@ -367,6 +376,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       SFFN_CUDA(launch_umma_rows(true, p, nb, h->sm_count, s));
     } else {
       RowsMmaParams p{};
+      p.status = h->at<int32_t>(h->L.status);
       p.W = W_up; p.R = H; p.K = D; p.idx = lidx; p.count = lcount;
       p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
       p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
@@ -386,6 +396,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       SFFN_CUDA(launch_umma_down(d, s));
     } else {
       DownMmaParams d{};
+      d.status = h->at<int32_t>(h->L.status);
       d.W_down = W_down; d.R = H; d.D = D;
       d.idx = lidx; d.count = lcount;
       d.hmT = hmT; d.hm_stride = h->L.hm_stride; d.B = nb;
@@ -466,6 +477,9 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     SFFN_CUDA(launch_compact(flag, H, idx, count, s));
     ++h->launches;
     h->list_state = 1;
+#ifdef SFFN_DEBUG
+    if (sffn::fused_test_knobs().poison_list) SFFN_CUDA(cudaMemsetAsync(idx, 0x7f, 4, s));  // entry 0 := 2139062143
+#endif
   }
   const int nbmax = updown_max_tokens(wkind, D);
   int grid = 2 * h->sm_count;
@@ -475,6 +489,7 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     const int left = B - b0;
     const int nb = (left >= 4 && nbmax >= 4) ? 4 : left >= 2 ? 2 : 1;
     UpDownParams p{};
+    p.status = h->at<int32_t>(h->L.status);
     p.W_up = W_up; p.W_down = W_down;
     p.x = xb + (size_t)b0 * D * esz; p.x_stride = D;
     p.a = actbuf + (size_t)b0 * H; p.a_stride = H;

@@ -59,8 +59,9 @@ __global__ void __launch_bounds__(256) rows_mma_kernel(const RowsMmaParams p) {
   for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
     const int i0 = tile * 128 + warp * 16 + g;  // list positions of this lane's two rows
     const int i1 = i0 + 8;
-    const int j0 = p.idx ? p.idx[min(i0, n_rows - 1)] : min(i0, n_rows - 1);
-    const int j1 = p.idx ? p.idx[min(i1, n_rows - 1)] : min(i1, n_rows - 1);
+    int j0 = p.idx ? p.idx[min(i0, n_rows - 1)] : min(i0, n_rows - 1);
+    int j1 = p.idx ? p.idx[min(i1, n_rows - 1)] : min(i1, n_rows - 1);
+    if (!SFFN_IN_BOUNDS(j0 >= 0 && j0 < p.R && j1 >= 0 && j1 < p.R, p.status, 30)) j0 = j1 = 0;
     const uint4* w0 = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.W) + (size_t)j0 * K) + t;
     const uint4* w1 = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.W) + (size_t)j1 * K) + t;
 
@@ -238,7 +239,8 @@ __global__ void __launch_bounds__(256) down_mma_kernel(const DownMmaParams p) {
       const int r = c >> 5, cc = c & 31;
       const int u = u0 + r;
       const bool valid = u < n_rows;
-      const int j = valid ? (p.idx ? p.idx[u] : u) : 0;
+      int j = valid ? (p.idx ? p.idx[u] : u) : 0;
+      if (!SFFN_IN_BOUNDS(j >= 0 && j < p.R, p.status, 31)) j = 0;
       cp_async16(ws + ((size_t)buf * 16 + r) * kWPitch + cc * 8,
                  static_cast<const __nv_bfloat16*>(p.W_down) + (size_t)j * p.D + d0 + cc * 8, valid);
     }

@@ -31,6 +31,7 @@ struct RowsMmaParams {
   void* hmT;             // bf16 [B][hm_stride]: h of token b for list position u
   int hm_stride;
   int act_up;            // activation on the up projection (double activation), kActNone = none
+  int32_t* status;       // device status block (debug builds record a list entry outside [0, R) here), or null
 };
 
 struct DownMmaParams {
@@ -42,6 +43,7 @@ struct DownMmaParams {
   int hm_stride;
   int B;
   float* partial;        // [splits][B][D]
+  int32_t* status;       // device status block (debug builds), or null
 };
 
 bool batched_mma_supported(int D, int K, int cols);

@@ -7,6 +7,23 @@
 
 namespace sffn {
 
+// Debug builds (-DSFFN_DEBUG, `python -m paper_2609_31975_b200.build --debug`): an index that is about to address
+// global memory through a list or a computed row number is checked first.  A violation puts SFFN_ERR_BOUNDS into the
+// device status word and the number of the check into word 4 of the status block, and the caller skips or clamps the
+// access; nothing traps.  In release builds the macro is the constant true and the checks compile away.
+#ifdef SFFN_DEBUG
+__device__ __forceinline__ bool in_bounds_or_record(bool ok, int32_t* status, int site) {
+  if (!ok && status) {
+    status[4] = site;
+    atomicCAS(status, 0, 6 /* SFFN_ERR_BOUNDS */);
+  }
+  return ok;
+}
+#define SFFN_IN_BOUNDS(cond, status, site) ::sffn::in_bounds_or_record((cond), (status), (site))
+#else
+#define SFFN_IN_BOUNDS(cond, status, site) true
+#endif
+
 constexpr int kActRelu = 0;
 constexpr int kActSqRelu = 1;
 constexpr int kActRsPlus = 2;

@@ -416,6 +416,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         if (!mbar_wait<true>(empty_gate + 8 * slot, ((s / NG) & 1) ^ 1, ctl, p.status, p.wait_cycles, 41)) break;
         const int j0 = slot_first_neuron(s);
         const uint32_t bytes = (uint32_t)(min(nr, p.H - j0) * gate_row_bytes);
+        if (!SFFN_IN_BOUNDS(j0 >= 0 && j0 < p.H && (uint32_t)slot * p.gate_slot_bytes + bytes <= (uint32_t)NG * p.gate_slot_bytes,
+                            p.status, 1))
+          break;
         mbar_expect_tx(full_gate + 8 * slot, bytes);
         bulk_g2s(ring + (uint32_t)slot * p.gate_slot_bytes, Wg + (size_t)j0 * gate_row_bytes, bytes,
                  full_gate + 8 * slot);
@@ -661,7 +664,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     if (lane < rows) {
       const float z = kScaled ? fmaf(mine, scale, add) : mine + add;
       const bool fired = z > 0.f;
-      if (!p.dense) p.flag[j0 + lane] = fired ? 1 : 0;
+      if (!p.dense && SFFN_IN_BOUNDS(j0 + lane < p.H && r0 + lane < p.slab_max, p.status, 3)) p.flag[j0 + lane] = fired ? 1 : 0;
       row_state[r0 + lane] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
     }
     __syncwarp();
@@ -733,7 +736,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
               slot_su[ms] = row_su[row];
               slot_sd[ms] = row_sd[row];
             }
-            const size_t j = (size_t)(slot_first_neuron(row / nr) + row % nr);
+            size_t j = (size_t)(slot_first_neuron(row / nr) + row % nr);
+            if (!SFFN_IN_BOUNDS(j < (size_t)p.H && ms >= 0 && ms < NA, p.status, 2)) j = 0;
             mbar_expect_tx(full_act + 8 * ms, (uint32_t)row_bytes);
             bulk_g2s(smem_u32(act_slot(ms)) + (ap == 0 ? 0u : (uint32_t)row_bytes), Wsrc + j * row_bytes,
                      (uint32_t)row_bytes, full_act + 8 * ms);
@@ -970,7 +974,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // This CTA's partial of y, every value tagged with the call's number.  Stored unit (two columns, 16 bytes)
     // (i * EPV / 2 + e) * kGT + gat holds columns EPV (gat + i kGT) + 2 e and the next one: a warp's store is 512
     // contiguous bytes; the summing threads undo the permutation when they write y.
-    if (cta != p.skip_arrival_cta && grp == 0) {
+    if (cta != p.skip_arrival_cta && grp == 0 && SFFN_IN_BOUNDS(cta < kMaxGrid, p.status, 4)) {
       const uint64_t keep = policy_evict_last();  // the partials are rewritten by every call: they should stay in L2
       unsigned long long* dst = p.partial + (size_t)cta * (CPT * EPV * kGT);
 #pragma unroll

@@ -49,6 +49,7 @@ struct FusedTestKnobs {
   bool pdl = true;               // programmatic dependent launch between calls
   int tensor_gate = -1;          // 1 / 0: tensor-core gate wherever it applies / nowhere; -1: the handle's engine decides
   long long wait_cycles = 1LL << 31;  // budget of every device-side wait (about one second)
+  bool poison_list = false;      // debug builds: the CUDA-core path corrupts its list's first entry (bounds-check test)
   int drop_stage = -1;           // batched gate kernel: CTA 0 never copies this stage's weights (its wait runs out)
   int skip_arrival_cta = -1;     // this CTA does not count itself as finished: the summing CTAs' wait runs out
   int ring_S = 0, ring_NA = 0;   // tensor-core gate: ring split override (0 = planned)

@@ -479,7 +479,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
             free_now = mbar_wait(extra_done + 8 * (slot - (NA - extra_slots)), 0, ctl, p.status, p.wait_cycles, 4);
           if (free_now) {
             if (ap == 0) slot_a[slot] = sl == 0x80000000u ? 0.f : __uint_as_float(sl);
-            const size_t j = (size_t)neuron_of(base + l);
+            size_t j = (size_t)neuron_of(base + l);
+            if (!SFFN_IN_BOUNDS(j < (size_t)p.H, p.status, 20)) j = 0;
             mbar_expect_tx(full_act + 8 * slot, (uint32_t)row_bytes);
             bulk_g2s(ring + (uint32_t)slot * p.act_slot_bytes, Wsrc + j * row_bytes, (uint32_t)row_bytes,
                      full_act + 8 * slot, once);
@@ -610,7 +611,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_tc_kernel(const TcParams p,
       if (seg == 0 && i_loc < rows) {
         const float z = v + bias;
         const bool fired = z > 0.f;
-        if (!p.dense) p.flag[j] = fired ? 1 : 0;
+        if (!p.dense && SFFN_IN_BOUNDS(j >= 0 && j < p.H, p.status, 21)) p.flag[j] = fired ? 1 : 0;
         row_state[l] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
       }
     }

@@ -238,7 +238,8 @@ __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
   for (int base = lo; base < hi; base += 16) {
     const int i = base + warp;
     const bool valid = i < hi;
-    const int j = valid ? (p.idx ? p.idx[i] : i) : 0;
+    int j = valid ? (p.idx ? p.idx[i] : i) : 0;
+    if (!SFFN_IN_BOUNDS(j >= 0 && j < p.H, p.status, 10)) j = 0;
     float u[NB];
 #pragma unroll
     for (int b = 0; b < NB; ++b) u[b] = 0.f;

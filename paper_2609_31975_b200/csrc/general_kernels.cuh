@@ -39,6 +39,7 @@ struct UpDownParams {
   int act_up;          // activation on the up projection (double activation), kActNone = none
   const float* s_up;   // int8 rows: [H] row scales of W_up and W_down
   const float* s_down;
+  int32_t* status;     // device status block (debug builds record a row index outside [0, H) here), or null
 };
 
 // wkind: kWF32 / kWBF16 / kWQ8 (common.cuh); tokens are fp32, bf16, bf16 respectively.

@@ -408,7 +408,8 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     const int B = p.B;
     const int li = tile * tile_rows + row_in_tile;
     const bool row_ok = row_in_tile >= 0 && row_in_tile < tile_rows && li < n_rows;
-    const int j = !row_ok ? 0 : (own_list && !walk_all) ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
+    int j = !row_ok ? 0 : (own_list && !walk_all) ? rows_sm[tcount * kTileRows + row_in_tile] : p.idx ? p.idx[li] : li;
+    if (!SFFN_IN_BOUNDS(j >= 0 && j < p.R, p.status, 40)) j = 0;
     // everything that does not depend on the accumulator is fetched before the wait
     if (MODE == kGate) pdl_wait();  // before the first read of a buffer an earlier kernel may write, and the first store
     float bias = 0.f, sg = 1.f;
@@ -516,8 +517,10 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const int li = tile * tile_rows + lane * 4 + q;
-            // rows beyond the list: any valid row, ignored later
-            r[q] = li >= n_rows ? 0 : own_list ? rows_sm[tl * kTileRows + lane * 4 + q] : p.idx ? p.idx[li] : li;
+            // rows beyond the list or the tile: row 0, ignored later
+            r[q] = (li >= n_rows || lane * 4 + q >= tile_rows) ? 0
+                   : own_list ? rows_sm[tl * kTileRows + lane * 4 + q] : p.idx ? p.idx[li] : li;
+            if (!SFFN_IN_BOUNDS(r[q] >= 0 && r[q] < p.R, p.status, 41)) r[q] = 0;
           }
         }
         if (with_w) {
@@ -744,6 +747,9 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
         r[1] = u + 1 < n_rows ? v.y : 0;
         r[2] = u + 2 < n_rows ? v.z : 0;
         r[3] = u + 3 < n_rows ? v.w : 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (!SFFN_IN_BOUNDS(r[q] >= 0 && r[q] < p.R, p.status, 42)) r[q] = 0;
       }
       int ok = 1;
       if (lane == 0) {
