@@ -276,6 +276,7 @@ def run_ours(args, rank, world, local):
     dev = torch.device(f"cuda:{local}")
     torch.cuda.set_device(dev)
     wl = Workload(m, dev, tokens=args.calls)
+    wl.ffn.set_gate_engine(args.engine)
     n_act = wl.count_active()
     mean_rows = statistics.mean(n_act)
     bytes_per_call = statistics.mean(m.touched_bytes(D_MODEL, D_FF, n, 2) for n in n_act)
@@ -314,7 +315,7 @@ def run_ours(args, rank, world, local):
         "config": {"workload": WORKLOAD, "step": f"{args.calls} single-token FFN calls, one token each",
                    "l2": f"rotating over {WEIGHT_SETS} independent weight sets ({WEIGHT_SETS * dense_bytes / 1e9:.2f} GB) "
                          "so inputs exceed L2", "storage": "bf16 weights and tokens, fp32 accumulation and output",
-                   "measured_sparsity": 1.0 - mean_rows / D_FF, "parallelism": f"{world} independent replicas"},
+                   "measured_sparsity": 1.0 - mean_rows / D_FF, "gate_engine": args.engine, "parallelism": f"{world} independent replicas"},
         "tokens_per_s": world * 1e6 / us_call,
         "touched_bytes_per_call": bytes_per_call,
         "achieved_gbs": achieved, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
@@ -345,6 +346,8 @@ def main():
     ap.add_argument("--only", default=None, help="with --report: only the cases whose name contains this")
     ap.add_argument("--report-calls", type=int, default=None, help="with --report: calls per case")
     ap.add_argument("--calls", type=int, default=CALLS_PER_STEP, help="FFN calls (tokens) per step")
+    ap.add_argument("--engine", default="auto", choices=["auto", "cuda_core", "tensor_core"],
+                    help="gate engine of the single-token calls (the handle's default is auto)")
     ap.add_argument("--no-extra", action="store_true", help="leave out the other configurations' headline points")
     ap.add_argument("--skip-extras", action="store_true",
                     help="time the sparse path only (no dense comparator, host-buffer or CPU legs): for profiler runs")
