@@ -78,7 +78,7 @@ def extra_points(m, dev):
     layers = [syn.standard_ffn(D, H, torch.bfloat16, 5, dev, sparsity=0.9, extra=i) for i in range(4)]
     rows.append(rep.measure("stress 8192x28672 s=0.9 B=1", D, H, 1, layers, std, "sqrelu", n_calls=48))
     keep = ("name", "B", "fired_rows", "us_per_call", "touched_mb", "gbs", "frac_measured_peak", "dense_us",
-            "speedup_vs_dense", "device_status")
+            "speedup_vs_dense", "dense_library_us", "speedup_vs_best_dense", "device_status")
     return [{k: r[k] for k in keep} for r in rows]
 
 

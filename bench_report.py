@@ -80,6 +80,31 @@ def _is_q8(w):
     return isinstance(w["W_up"], dict)
 
 
+def _library_dense_calls(sets, x, act, n):
+    """A second dense comparator: the same FFN as three library matrix products (cuBLAS through torch, bf16 in and out)
+    and two elementwise kernels per call, outputs preallocated.  Only its time is used; standard gate on bf16 weights."""
+    H, D = sets[0]["W_up"].shape
+    B = 1 if x.dim() == 2 else x.shape[1]
+    z = torch.empty((B, H), dtype=torch.bfloat16, device=DEV)
+    u = torch.empty((B, H), dtype=torch.bfloat16, device=DEV)
+    yb = torch.empty((B, D), dtype=torch.bfloat16, device=DEV)
+    biases = [w["b_g"].to(torch.bfloat16) for w in sets]
+    fn = {"relu": torch.relu_, "sqrelu": lambda t: torch.relu_(t).square_(), "rsplus": torch.nn.functional.silu}[act]
+
+    def one(t):
+        w, b = sets[t % len(sets)], biases[t % len(sets)]
+        xt = x[t].view(B, D)
+
+        def call():
+            torch.addmm(b, xt, w["W_g"].t(), out=z)
+            fn(z)
+            torch.matmul(xt, w["W_up"].t(), out=u)
+            z.mul_(u)
+            torch.matmul(z, w["W_down"], out=yb)
+        return call
+    return [one(t) for t in range(n)]
+
+
 def _bytes(D, H, n_rows, esz, B, r, q8):
     """Algorithmic bytes of one call; int8 weights: one byte per weight, bf16 tokens, and the fp32 row scales of
     the gate matrix and of the fired W_up / W_down rows."""
@@ -112,6 +137,9 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=None, a
     n_rows = statistics.mean(rows)
     us, us_min = _time_graph(sparse_calls, stream) if graph else _time(sparse_calls, stream)
     us_dense, _ = _time(dense_calls[: max(16, n_calls // 4)], stream, reps=2)
+    us_lib = None
+    if not _is_q8(sets[0]) and "W_g" in gate_of(sets[0]):
+        us_lib, _ = _time(_library_dense_calls(sets, x, act, max(16, n_calls // 4)), stream, reps=2)
     status = ffn.device_status()
     q8 = _is_q8(sets[0])
     nbytes = _bytes(D, H, round(n_rows), 2, B, r, q8)
@@ -120,6 +148,7 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=None, a
                gbs=nbytes / us / 1e3, frac_measured_peak=nbytes / us / 1e3 / peak,
                frac_nominal=nbytes / us / 1e3 / NOMINAL, dense_us=us_dense,
                dense_gbs=_bytes(D, H, H, 2, B, r, q8) / us_dense / 1e3, speedup_vs_dense=us_dense / us,
+               dense_library_us=us_lib, speedup_vs_best_dense=min(us_dense, us_lib or us_dense) / us,
                device_status=status)
     del ffn, sparse_calls, dense_calls
     torch.cuda.empty_cache()
@@ -322,12 +351,14 @@ def run(out_path, quick=False, only=None, n_calls=None):
         torch.cuda.empty_cache()
     Path(out_path).parent.mkdir(parents=True, exist_ok=True)
     Path(out_path).write_text(json.dumps(rows, indent=1))
-    md = ["| case | B | fired rows | us/call | touched MB | GB/s | % of measured peak | % of 8 TB/s | dense us | speedup |",
-          "|---|---|---|---|---|---|---|---|---|---|"]
+    md = ["| case | B | fired rows | us/call | touched MB | GB/s | % of measured peak | % of 8 TB/s | dense us | speedup | "
+          "library dense us |",
+          "|---|---|---|---|---|---|---|---|---|---|---|"]
     for r_ in rows:
         md.append(f"| {r_['name']} | {r_['B']} | {r_['fired_rows']:.0f} ({100 * r_['fired_frac']:.1f} %) | "
                   f"{r_['us_per_call']:.1f} | {r_['touched_mb']:.1f} | {r_['gbs']:.0f} | "
                   f"{100 * r_['frac_measured_peak']:.1f} | {100 * r_['frac_nominal']:.1f} | {r_['dense_us']:.1f} | "
-                  f"{r_['speedup_vs_dense']:.2f}x |")
+                  f"{r_['speedup_vs_dense']:.2f}x | "
+                  + (f"{r_['dense_library_us']:.1f} |" if r_.get("dense_library_us") else "- |"))
     Path(out_path).with_suffix(".md").write_text("\n".join(md) + "\n")
     return rows
