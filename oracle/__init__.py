@@ -200,6 +200,33 @@ def dequantize_rows(q, scale) -> np.ndarray:
     return scale.astype(np.float64)[:, None] * q.astype(np.float64)
 
 
+def dequantize_rows_q4(packed, scale) -> np.ndarray:
+    """The matrix that 4-bit codes stand for (the same appendix converts the weights "to int8 or int4 at inference" and
+    fixes no format; reading taken: symmetric two's-complement codes in [-8, 7], two per byte with the even column in
+    the low nibble, one fp32 scale per row): W[j, 2b] = scale[j] * low(packed[j, b]), W[j, 2b + 1] = scale[j] *
+    high(packed[j, b]), as float64.  ``packed`` is uint8 [rows, cols / 2]."""
+    if not isinstance(packed, np.ndarray):
+        packed = packed.detach().cpu().numpy()
+    if not isinstance(scale, np.ndarray):
+        scale = scale.detach().cpu().numpy()
+    assert packed.dtype == np.uint8 and packed.ndim == 2 and scale.shape == (packed.shape[0],)
+    rows, half = packed.shape
+    q = np.empty((rows, 2 * half), np.float64)
+    for part, nib in ((0, packed & 0x0F), (1, packed >> 4)):
+        nib = nib.astype(np.int16)
+        q[:, part::2] = np.where(nib >= 8, nib - 16, nib)   # two's complement on four bits
+    return scale.astype(np.float64)[:, None] * q
+
+
+def ffn_q4(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, **kw):
+    """:func:`ffn` on 4-bit weights: every matrix is a dict(q=uint8 [rows, cols / 2], s=fp32 [rows]) and enters Eq. 1
+    as its float64 dequantisation (:func:`dequantize_rows_q4`); tokens stay in their own dtype (weight-only)."""
+    dq = lambda m: dequantize_rows_q4(m["q"], m["s"])  # noqa: E731
+    if lopa is not None:
+        lopa = dict(lopa, V=dq(lopa["V"]), U=dq(lopa["U"]))
+    return ffn(x, dq(W_up), dq(W_down), act, W_g=None if W_g is None else dq(W_g), lopa=lopa, **kw)
+
+
 def ffn_q8(x, W_up, W_down, act="relu", *, W_g=None, lopa=None, **kw):
     """:func:`ffn` on int8 weights: every matrix is a dict(q=int8 [rows, cols], s=fp32 [rows]) and enters Eq. 1 as
     its float64 dequantisation (:func:`dequantize_rows`); tokens stay in their own dtype (weight-only)."""

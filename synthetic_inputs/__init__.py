@@ -105,6 +105,50 @@ def q8_matrix(shape, std: float, seed: int, tag: str, device="cpu", extra: int =
     return {"q": q, "s": s.float()}
 
 
+def q4_matrix(shape, std: float, seed: int, tag: str, device="cpu", extra: int = 0, chunk_rows: int = 4096) -> dict:
+    """4-bit codes and fp32 row scales of a matrix whose entries s_j q[j,k] have standard deviation ~ std: codes
+    clip(round(N(0, 2.5^2)), -7, 7) (what an abs-max quantiser leaves of a Gaussian row on 4 bits), packed two per byte
+    with the even column in the low nibble, two's complement; scales (std / 2.5) (1 +- 0.1 u).  Returns
+    dict(q=uint8 [rows, cols / 2], s=float32 [rows]).  cols must be even."""
+    rows, cols = shape
+    assert cols % 2 == 0
+    q = torch.empty((rows, cols // 2), dtype=torch.uint8, device=device)
+    g = _gen(seed, tag, device, extra)
+    for r0 in range(0, rows, chunk_rows):
+        r1 = min(rows, r0 + chunk_rows)
+        blk = torch.randn((r1 - r0, cols), generator=g, device=device, dtype=torch.float32)
+        c = (blk * 2.5).round().clamp(-7, 7).to(torch.int16) & 0xF
+        q[r0:r1] = (c[:, 0::2] | (c[:, 1::2] << 4)).to(torch.uint8)
+    u = torch.rand((rows,), generator=_gen(seed, "scale", device, extra * 16 + _TAGS[tag]), device=device,
+                   dtype=torch.float32)
+    s = (std / 2.5) * (1.0 + 0.1 * (2.0 * u - 1.0))
+    return {"q": q, "s": s.float()}
+
+
+def standard_ffn_q4(D: int, H: int, seed: int, device="cpu", sparsity: float | None = 0.9, extra: int = 0) -> dict:
+    """Standard-gated FFN in 4-bit codes + row scales (see :func:`q4_matrix`); b_g as in :func:`standard_ffn`."""
+    std = 1.0 / math.sqrt(D)
+    w = {k: q4_matrix((H, D), std, seed, k, device, extra) for k in ("W_g", "W_up", "W_down")}
+    w["b_g"] = None if sparsity is None else torch.full(
+        (H,), gate_bias_for_sparsity(sparsity), dtype=torch.float32, device=device)
+    return w
+
+
+def lopa_ffn_q4(D: int, H: int, r: int, seed: int, device="cpu", sparsity: float | None = 0.9,
+                with_fixed_matrix: bool = True, extra: int = 0) -> dict:
+    """LoPA-gated FFN in 4-bit codes + row scales (V [r,D], U [H,r], W_up, W_down [H,D]); b_g as in :func:`lopa_ffn`."""
+    w = {
+        "V": q4_matrix((r, D), 1.0 / math.sqrt(D), seed, "V", device, extra),
+        "U": q4_matrix((H, r), 1.0 / math.sqrt(r), seed, "U", device, extra),
+        "W_up": q4_matrix((H, D), 1.0 / math.sqrt(D), seed, "W_up", device, extra),
+        "W_down": q4_matrix((H, D), 1.0 / math.sqrt(D), seed, "W_down", device, extra),
+    }
+    sigma = math.sqrt(2.0) if with_fixed_matrix else 1.0
+    w["b_g"] = None if sparsity is None else torch.full(
+        (H,), gate_bias_for_sparsity(sparsity, sigma), dtype=torch.float32, device=device)
+    return w
+
+
 def standard_ffn_q8(D: int, H: int, seed: int, device="cpu", sparsity: float | None = 0.9, extra: int = 0) -> dict:
     """Standard-gated FFN in int8 codes + row scales: W_g, W_up, W_down each dict(q [H,D], s [H]); b_g as in
     :func:`standard_ffn`."""

@@ -436,6 +436,66 @@ def test_int8_inputs_recipe():
     assert out["n_act"].mean() / 512 == pytest.approx(0.1, abs=0.03)
 
 
+# ---------------------------------------------------------------- weight-only int4 (same appendix)
+def test_hand_worked_int4_nibbles():
+    # byte 0x2F: low nibble F = -1 (even column), high nibble 2 = +2 (odd column); byte 0x78: low 8 = -8, high 7 = +7
+    packed = np.array([[0x2F, 0x78], [0x10, 0xF9]], np.uint8)
+    s = np.array([0.5, 2.0], np.float32)
+    np.testing.assert_array_equal(oracle.dequantize_rows_q4(packed, s),
+                                  [[-0.5, 1.0, -4.0, 3.5], [0.0, 2.0, -14.0, -2.0]])
+    # the same hand-worked FFN as for int8 rows, written in nibbles: W1 = [[0.5,-1],[0.75,1]], W3 = 2*[[1,1],[1,-1]],
+    # Wd = [[7,7],[2,-3]];  x = [2,1]: z = [0, 2.5], u = [6, 2], y = 2.5 * 2 * [2,-3] = [10,-15]
+    W1 = dict(q=np.array([[0xE1], [0x43]], np.uint8), s=np.array([0.5, 0.25], np.float32))
+    W3 = dict(q=np.array([[0x11], [0xF1]], np.uint8), s=np.array([2.0, 2.0], np.float32))
+    Wd = dict(q=np.array([[0x77], [0xA4]], np.uint8), s=np.array([1.0, 0.5], np.float32))
+    x = np.array([2.0, 1.0], np.float32)
+    for route in ("dense", "sparse"):
+        out = oracle.ffn_q4(x, W3, Wd, "relu", W_g=W1, route=route)
+        np.testing.assert_array_equal(out["z"], [0.0, 2.5])
+        np.testing.assert_array_equal(out["y"], [10.0, -15.0])
+
+
+def test_int4_codes_equal_the_same_codes_stored_as_int8():
+    # packing is the only thing the 4-bit route adds: the same integer codes given as int8 go through the pinned int8
+    # route and must give the same bits
+    D, H, r, B = 32, 40, 16, 3
+    x = syn.tokens(B, D, torch.bfloat16, 6)
+
+    def mat(rows, cols):
+        q = RNG.integers(-8, 8, (rows, cols)).astype(np.int8)
+        s = RNG.uniform(0.01, 0.1, rows).astype(np.float32)
+        nib = (q.astype(np.int16) & 0xF).astype(np.uint8)
+        return dict(q=(nib[:, 0::2] | (nib[:, 1::2] << 4)).astype(np.uint8), s=s), dict(q=q, s=s)
+
+    (g4, g8), (u4, u8), (d4, d8), (V4, V8), (U4, U8) = mat(H, D), mat(H, D), mat(H, D), mat(r, D), mat(H, r)
+    b = np.full(H, -0.2, np.float32)
+    a, f = oracle.ffn_q4(x, u4, d4, "relu", W_g=g4, b_g=b), oracle.ffn_q8(x, u8, d8, "relu", W_g=g8, b_g=b)
+    np.testing.assert_array_equal(a["y"], f["y"])
+    np.testing.assert_array_equal(a["z"], f["z"])
+    assert a["y"].any() and 0 < a["n_act"].mean() < H
+    gi = RNG.integers(0, D, H).astype(np.int32)
+    l4 = dict(V=V4, U=U4, g_idx=gi, use_rmsnorm=True, eps=1e-5)
+    l8 = dict(V=V8, U=U8, g_idx=gi, use_rmsnorm=True, eps=1e-5)
+    a = oracle.ffn_q4(x, u4, d4, "sqrelu", lopa=l4, b_g=b, act_up="relu")
+    f = oracle.ffn_q8(x, u8, d8, "sqrelu", lopa=l8, b_g=b, act_up="relu")
+    np.testing.assert_array_equal(a["y"], f["y"])
+
+
+def test_int4_inputs_recipe():
+    w = syn.standard_ffn_q4(256, 512, 3)
+    for k in ("W_g", "W_up", "W_down"):
+        q, s = w[k]["q"], w[k]["s"]
+        assert q.dtype == torch.uint8 and s.dtype == torch.float32 and q.shape == (512, 128) and s.shape == (512,)
+        W = oracle.dequantize_rows_q4(q, s)
+        codes = W / s.numpy().astype(np.float64)[:, None]
+        assert codes.min() >= -7 and codes.max() <= 7 and np.all(codes == np.round(codes))
+        assert float(codes.std()) == pytest.approx(2.5, rel=0.05)
+        assert float(W.std()) * 16.0 == pytest.approx(1.0, rel=0.05)
+    x = syn.tokens(16, 256, torch.bfloat16, 3)
+    out = oracle.ffn_q4(x, w["W_up"], w["W_down"], "relu", W_g=w["W_g"], b_g=w["b_g"])
+    assert out["n_act"].mean() / 512 == pytest.approx(0.1, abs=0.03)
+
+
 # ---------------------------------------------------------------- LoPA approximation of a full gate (Sec. 3.4)
 def test_lopa_approximation_m_step_is_the_row_optimum_by_brute_force():
     cast = oracle.lopa_cast
