@@ -77,7 +77,10 @@ def _time_graph(calls, stream, replays=5):
 
 
 def _is_q8(w):
-    return isinstance(w["W_up"], dict)
+    """0 for fp32 / bf16 weights, 8 for int8 codes, 4 for packed 4-bit codes."""
+    if not isinstance(w["W_up"], dict):
+        return 0
+    return 4 if w["W_up"]["q"].dtype == torch.uint8 else 8
 
 
 def _library_dense_calls(sets, x, act, n):
@@ -110,6 +113,9 @@ def _bytes(D, H, n_rows, esz, B, r, q8):
     the gate matrix and of the fired W_up / W_down rows."""
     if not q8:
         return touched_bytes(D, H, n_rows, esz, B, r)
+    if q8 == 4:  # 4-bit codes: half a byte per weight
+        weights = touched_bytes(D, H, n_rows, 1, 0, r) - H * 4
+        return weights // 2 + H * 4 + B * D * 2 + B * D * 4 + 4 * (H + 2 * n_rows + (r or 0))
     return touched_bytes(D, H, n_rows, 1, B, r) + B * D + 4 * (H + 2 * n_rows + (r or 0))
 
 
@@ -128,7 +134,7 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=None, a
         xt = x[t, 0] if B == 1 else x[t]
         yt = y[t, 0] if B == 1 else y[t]
         if t < 24:  # fired rows per call (union for B > 1), outside the timed region
-            fwd = ffn.sparse_ffn_forward_q8 if _is_q8(w) else ffn.sparse_ffn_forward
+            fwd = {0: ffn.sparse_ffn_forward, 8: ffn.sparse_ffn_forward_q8, 4: ffn.sparse_ffn_forward_q4}[_is_q8(w)]
             fwd(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt)
             rows.append(int(ffn.last_active().numel()))
         sparse_calls.append(ffn.prepared(xt, gate_of(w), w["b_g"], w["W_up"], w["W_down"], act, yt, stream=stream))
@@ -282,6 +288,15 @@ def run(out_path, quick=False, only=None, n_calls=None):
         lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}
         add("lopa r=512 relu int8", D, H, 1, lsets, lg, "relu", r=512, peak=peak)
         del qsets, lsets
+        torch.cuda.empty_cache()
+    # weight-only int4 (packed 4-bit codes + one fp32 scale per row)
+    if only is None or "int4" in only:
+        qsets = [syn.standard_ffn_q4(D, H, 8, DEV, sparsity=0.9, extra=i) for i in range(8)]
+        for s in ((0.9,) if quick else (0.8, 0.9, 0.95)):
+            b = syn.gate_bias_for_sparsity(s)
+            sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in qsets]
+            add(f"decode 4096x14336 s={s} int4", D, H, 1, sets, std, "relu", peak=peak)
+        del qsets
         torch.cuda.empty_cache()
     if not quick and (only is None or "stress" in only):
         # stress shape: 8 independent layers per step

@@ -180,6 +180,19 @@ int dense_ffn_forward_q8(sffn_handle* handle, const void* x, int B, const sffn_g
                          const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
                          void* stream);
 
+/* Weight-only int4 (the same appendix names int4 beside int8 and fixes no format either).  Here: two's-complement
+ * codes in [-8, 7], two per byte with the even column in the low nibble, row-major, one fp32 scale per row:
+ *     W[j, 2b] = s[j] * low_nibble(p[j, b]),   W[j, 2b + 1] = s[j] * high_nibble(p[j, b]).
+ * The weight pointers address the packed bytes ([H, D/2], [r, D/2], [H, r/2]); `scales` as for int8.  Rows must be a
+ * multiple of 16 bytes (D and r multiples of 32).  Otherwise exactly like the _q8 calls: bf16 tokens, fp32 arithmetic,
+ * one token in the fused kernel (rows of up to 8192 codes there), batches and wider rows in the CUDA-core kernels. */
+int sparse_ffn_forward_q4(sffn_handle* handle, const void* x, int B, const sffn_gate* gate, const float* b_g,
+                          const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
+                          void* stream);
+int dense_ffn_forward_q4(sffn_handle* handle, const void* x, int B, const sffn_gate* gate, const float* b_g,
+                         const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
+                         void* stream);
+
 /* End-to-end variant of sparse_ffn_forward for callers whose activations live on the host:
  * x_host [B,D] (handle dtype) and y_host [B,D] fp32 are HOST pointers; weights stay on the device.
  * Brings x in, runs the sparse path, puts y out, all on `stream`; y_host is valid once the stream has

@@ -70,6 +70,8 @@ def load_library() -> ctypes.CDLL:
         fwd_q8 = [vp, vp, i, ctypes.POINTER(_Gate), vp, vp, vp, ctypes.POINTER(_Q8Scales), i, vp, vp]
         lib.sparse_ffn_forward_q8.argtypes = fwd_q8
         lib.dense_ffn_forward_q8.argtypes = fwd_q8
+        lib.sparse_ffn_forward_q4.argtypes = fwd_q8
+        lib.dense_ffn_forward_q4.argtypes = fwd_q8
         lib.sffn_last_active.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
         lib.sffn_last_device_status.argtypes = [vp, ctypes.POINTER(i)]
         lib.sffn_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
@@ -103,11 +105,12 @@ def _ptr(t):
 
 
 def _codes(m):
-    """The tensor whose address goes to the library: an int8 matrix given as dict(q=codes, s=row scales), or a tensor."""
+    """The tensor whose address goes to the library: a quantised matrix given as dict(q=codes, s=row scales), or a tensor."""
     if isinstance(m, dict):
         q, s = m["q"], m["s"]
-        if q.dtype != torch.int8 or s.dtype != torch.float32 or s.shape != (q.shape[0],):
-            raise TypeError("an int8 matrix is dict(q=int8 [rows, cols], s=float32 [rows])")
+        if q.dtype not in (torch.int8, torch.uint8) or s.dtype != torch.float32 or s.shape != (q.shape[0],):
+            raise TypeError("a quantised matrix is dict(q=int8 [rows, cols] or packed 4-bit uint8 [rows, cols / 2], "
+                            "s=float32 [rows])")
         return q
     return m
 
@@ -283,7 +286,10 @@ class SparseFFN:
         if isinstance(W_up, dict):  # weight-only int8
             if host:
                 raise ValueError("the host entry point takes fp32 / bf16 weights")
-            fn = self.lib.dense_ffn_forward_q8 if dense else self.lib.sparse_ffn_forward_q8
+            if W_up["q"].dtype == torch.uint8:  # packed 4-bit codes
+                fn = self.lib.dense_ffn_forward_q4 if dense else self.lib.sparse_ffn_forward_q4
+            else:
+                fn = self.lib.dense_ffn_forward_q8 if dense else self.lib.sparse_ffn_forward_q8
             sc = self._scales(gate, W_up, W_down)
             args = (self._h, _ptr(x), B, ctypes.byref(g), _ptr(b_g), _ptr(_codes(W_up)), _ptr(_codes(W_down)),
                     ctypes.byref(sc), a, _ptr(y), self._stream(stream))
@@ -326,6 +332,21 @@ class SparseFFN:
         if y is None:
             y = torch.empty((*x.shape[:-1], self.D), dtype=torch.float32, device=x.device)
         return self._call_q8(self.lib.dense_ffn_forward_q8, "dense_ffn_forward_q8", x, gate, b_g, W_up, W_down,
+                             act, y, stream)
+
+    def sparse_ffn_forward_q4(self, x, gate, b_g, W_up, W_down, act="relu", y=None, stream=None):
+        """:meth:`sparse_ffn_forward` on 4-bit weights: every matrix is ``dict(q=uint8 [rows, cols / 2], s=float32
+        [rows])``, two's-complement codes, even column in the low nibble (sparse_ffn_forward_q4 of the header)."""
+        if y is None:
+            y = torch.empty((*x.shape[:-1], self.D), dtype=torch.float32, device=x.device)
+        return self._call_q8(self.lib.sparse_ffn_forward_q4, "sparse_ffn_forward_q4", x, gate, b_g, W_up, W_down,
+                             act, y, stream)
+
+    def dense_ffn_forward_q4(self, x, gate, b_g, W_up, W_down, act="relu", y=None, stream=None):
+        """The dense comparator on 4-bit weights."""
+        if y is None:
+            y = torch.empty((*x.shape[:-1], self.D), dtype=torch.float32, device=x.device)
+        return self._call_q8(self.lib.dense_ffn_forward_q4, "dense_ffn_forward_q4", x, gate, b_g, W_up, W_down,
                              act, y, stream)
 
     def sparse_ffn_forward_host(self, x_host, gate, b_g, W_up, W_down, act, y_host, stream=None):

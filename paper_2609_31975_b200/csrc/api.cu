@@ -203,18 +203,19 @@ int sffn_launch_count(sffn_handle* h, long long* launches) {
 namespace {
 
 int check_call(const sffn_handle* h, const void* x, int B, const sffn_gate* g, const void* W_up,
-               const void* W_down, int act, const void* y, const sffn_q8_scales* q8) {
+               const void* W_down, int act, const void* y, const sffn_q8_scales* q8, int qbits) {
   if (!h || !x || !g || !W_up || !W_down || !y) return SFFN_ERR_INVALID_ARG;
   if (B < 1 || B > h->B_max) return SFFN_ERR_INVALID_ARG;
   if (act < SFFN_ACT_RELU || act > SFFN_ACT_RSPLUS) return SFFN_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(W_up) || !aligned16(W_down) || !aligned16(y)) return SFFN_ERR_UNSUPPORTED;
-  const size_t esz = q8 ? 1 : h->dtype == SFFN_BF16 ? 2 : 4;  // bytes of a weight element
+  // elements of a weight row per 16 bytes
+  const int epv = q8 ? (qbits == 4 ? 32 : 16) : h->dtype == SFFN_BF16 ? 8 : 4;
   if (q8) {
-    if (h->dtype != SFFN_BF16) return SFFN_ERR_UNSUPPORTED;  // int8 weights meet bf16 tokens
+    if (h->dtype != SFFN_BF16) return SFFN_ERR_UNSUPPORTED;  // int8 / int4 weights meet bf16 tokens
     if (!q8->s_gate || !q8->s_up || !q8->s_down) return SFFN_ERR_INVALID_ARG;
     if (g->kind == SFFN_GATE_LOPA && !q8->s_V) return SFFN_ERR_INVALID_ARG;
-    if (h->D % 16) return SFFN_ERR_UNSUPPORTED;
-    if (sffn::updown_max_tokens(sffn::kWQ8, h->D) == 0) return SFFN_ERR_UNSUPPORTED;
+    if (h->D % epv) return SFFN_ERR_UNSUPPORTED;
+    if (sffn::updown_max_tokens(qbits == 4 ? sffn::kWQ4 : sffn::kWQ8, h->D) == 0) return SFFN_ERR_UNSUPPORTED;
     if (h->path == SFFN_PATH_MMA_SYNC) return SFFN_ERR_UNSUPPORTED;
   }
   if (g->kind == SFFN_GATE_STANDARD) {
@@ -222,7 +223,7 @@ int check_call(const sffn_handle* h, const void* x, int B, const sffn_gate* g, c
     if (!aligned16(g->W_g)) return SFFN_ERR_UNSUPPORTED;
   } else if (g->kind == SFFN_GATE_LOPA) {
     if (!g->V || !g->U || g->r < 1 || g->r > h->r_max) return SFFN_ERR_INVALID_ARG;
-    if (!aligned16(g->V) || !aligned16(g->U) || (g->r * esz) % 16) return SFFN_ERR_UNSUPPORTED;
+    if (!aligned16(g->V) || !aligned16(g->U) || g->r % epv) return SFFN_ERR_UNSUPPORTED;
   } else {
     return SFFN_ERR_INVALID_ARG;
   }
@@ -412,10 +413,10 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
 // General path: gate (all tokens, chunks of <= 4) -> compaction -> up/down + reduce per chunk.
 int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
                 const void* W_up, const void* W_down, int act, float* y, bool dense,
-                const sffn_q8_scales* q8, cudaStream_t s) {
+                const sffn_q8_scales* q8, int qbits, cudaStream_t s) {
   using namespace sffn;
   const bool bf16 = h->dtype == SFFN_BF16;
-  const int wkind = q8 ? kWQ8 : bf16 ? kWBF16 : kWF32;
+  const int wkind = q8 ? (qbits == 4 ? kWQ4 : kWQ8) : bf16 ? kWBF16 : kWF32;
   const size_t esz = bf16 ? 2 : 4;  // bytes of a token element
   const int D = h->D, H = h->H;
   float* actbuf = h->at<float>(h->L.act);
@@ -508,11 +509,12 @@ int run_general(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
 }
 
 int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g, const void* W_up,
-        const void* W_down, int act, float* y, bool dense, void* stream, const sffn_q8_scales* q8 = nullptr) {
-  const int rc = check_call(h, x, B, g, W_up, W_down, act, y, q8);
+        const void* W_down, int act, float* y, bool dense, void* stream, const sffn_q8_scales* q8 = nullptr,
+        int qbits = 8) {
+  const int rc = check_call(h, x, B, g, W_up, W_down, act, y, q8, qbits);
   if (rc != SFFN_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int wkind = q8 ? sffn::kWQ8 : h->dtype == SFFN_BF16 ? sffn::kWBF16 : sffn::kWF32;
+  const int wkind = q8 ? (qbits == 4 ? sffn::kWQ4 : sffn::kWQ8) : h->dtype == SFFN_BF16 ? sffn::kWBF16 : sffn::kWF32;
   const bool fused_ok = sffn::fused_supported(wkind, h->D, h->H, B, g, h->sm_count);
   if (h->path == SFFN_PATH_FUSED && !fused_ok) return SFFN_ERR_UNSUPPORTED;
   if (fused_ok && h->path != SFFN_PATH_GENERAL) {
@@ -544,7 +546,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
   } else if (h->path == SFFN_PATH_MMA_SYNC) {
     return SFFN_ERR_UNSUPPORTED;
   }
-  return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, q8, s);
+  return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, q8, qbits, s);
 }
 
 // Device-side alias of a 16-byte aligned pointer into pinned, mapped host memory; null for anything else.
@@ -591,6 +593,20 @@ int dense_ffn_forward_q8(sffn_handle* h, const void* x, int B, const sffn_gate* 
                          void* stream) {
   if (!scales) return SFFN_ERR_INVALID_ARG;
   return run(h, x, B, g, b_g, W_up, W_down, act, y, true, stream, scales);
+}
+
+int sparse_ffn_forward_q4(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
+                          const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
+                          void* stream) {
+  if (!scales) return SFFN_ERR_INVALID_ARG;
+  return run(h, x, B, g, b_g, W_up, W_down, act, y, false, stream, scales, 4);
+}
+
+int dense_ffn_forward_q4(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
+                         const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
+                         void* stream) {
+  if (!scales) return SFFN_ERR_INVALID_ARG;
+  return run(h, x, B, g, b_g, W_up, W_down, act, y, true, stream, scales, 4);
 }
 
 int sparse_ffn_forward_host(sffn_handle* h, const void* x_host, int B, const sffn_gate* g,

@@ -126,15 +126,53 @@ struct Elem<int8_t> {
   }
 };
 
+// 4-bit codes of weight-only quantisation: two's complement in [-8, 7], two per byte, the even column in the low
+// nibble, one fp32 scale per row (applied by the caller, as for int8).  A tag type: rows are addressed in bytes.
+// With the sign bits of all eight nibbles of a word flipped each nibble is u = code + 8 in 0..15; the even and the odd
+// nibbles are separated into bytes, a byte goes into the low mantissa byte of 2^23 and one subtraction of 2^23 + 8
+// leaves the code.
+struct q4_t {};
+template <>
+struct Elem<q4_t> {
+  static constexpr int kPerVec = 32;
+  // eight codes of one 32-bit word, in column order
+  __device__ __forceinline__ static void unpack8(uint32_t w, float* f) {
+    w ^= 0x88888888u;
+    const uint32_t even = w & 0x0f0f0f0fu, odd = (w >> 4) & 0x0f0f0f0fu;  // columns 0,2,4,6 and 1,3,5,7 as bytes
+    const float2 bias = make_float2(-8388616.f, -8388616.f);
+#pragma unroll
+    for (int b = 0; b < 4; b += 2) {
+      const float2 e = add2(make_float2(__uint_as_float(__byte_perm(even, 0x4b000000u, 0x7650 + b)),
+                                        __uint_as_float(__byte_perm(even, 0x4b000000u, 0x7651 + b))), bias);
+      const float2 o = add2(make_float2(__uint_as_float(__byte_perm(odd, 0x4b000000u, 0x7650 + b)),
+                                        __uint_as_float(__byte_perm(odd, 0x4b000000u, 0x7651 + b))), bias);
+      f[2 * b] = e.x; f[2 * b + 1] = o.x; f[2 * b + 2] = e.y; f[2 * b + 3] = o.y;
+    }
+  }
+  __device__ __forceinline__ static void unpack(const uint4& v, float* f) {
+    unpack8(v.x, f);
+    unpack8(v.y, f + 8);
+    unpack8(v.z, f + 16);
+    unpack8(v.w, f + 24);
+  }
+};
+
+// Bytes of a row of n elements of storage type T (16 / kPerVec bytes per element: half a byte for 4-bit codes).
+template <typename T>
+__host__ __device__ constexpr size_t row_bytes_of(size_t n) { return n * 16 / Elem<T>::kPerVec; }
+
 // Storage type of the tokens that go with weights of type T, and whether rows of T carry a scale.
 template <typename T>
 struct TokenOf { using type = T; static constexpr bool kScaled = false; };
 template <>
 struct TokenOf<int8_t> { using type = __nv_bfloat16; static constexpr bool kScaled = true; };
+template <>
+struct TokenOf<q4_t> { using type = __nv_bfloat16; static constexpr bool kScaled = true; };
 
 // Weight storage kinds as the launchers take them (0 and 1 coincide with "is bf16" of older call sites).
-constexpr int kWF32 = 0, kWBF16 = 1, kWQ8 = 2;
-__host__ __device__ constexpr int weight_bytes(int wkind) { return wkind == kWF32 ? 4 : wkind == kWBF16 ? 2 : 1; }
+constexpr int kWF32 = 0, kWBF16 = 1, kWQ8 = 2, kWQ4 = 3;
+// elements per 16 bytes of a weight row
+__host__ __device__ constexpr int weight_epv(int wkind) { return wkind == kWF32 ? 4 : wkind == kWBF16 ? 8 : wkind == kWQ8 ? 16 : 32; }
 
 // Streaming 16-byte load: weights are read once, so keep them out of L1.
 __device__ __forceinline__ uint4 ld_stream16(const void* p) {

@@ -361,8 +361,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const uint32_t v_bar = bars + 16 * (NG + NA);
 
   const int nvecD = D / EPV, nvecK = K / EPV;
-  const size_t row_bytes = (size_t)D * sizeof(T);
-  const size_t gate_row_bytes = (size_t)K * sizeof(T);
+  const size_t row_bytes = row_bytes_of<T>(D);
+  const size_t gate_row_bytes = row_bytes_of<T>(K);
   const int nr = p.rows_per_gate_slot;
   // Neurons are dealt to the CTAs in blocks of nr consecutive rows, round robin: CTA c owns the
   // blocks c, c + G, c + 2G, ...  One block = one gate ring slot.  Compared with one contiguous slab
@@ -578,7 +578,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // instruction latency, not throughput.  Eight rows are dotted side by side (eight independent chains, the vector
     // read once for all of them, every load requested before the first multiply) and reduced together: each
     // exchange halves the number of sums a lane carries, so eight rows cost 4 + 2 + 1 + 1 + 1 shuffles instead of 40.
-    const int rows_short = nvecK <= 128 ? rows : 0;
+    const int rows_short = (nvecK <= 128 && EPV < 32) ? rows : 0;
     int rr_short = 0;
     for (; rows_short - rr_short > 2; rr_short += 8) {  // one or two left-over rows are cheaper one by one (below)
       const int rr = rr_short;
@@ -629,6 +629,37 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       if (lane == rr_short) mine = z;
     }
     int rr_single = rows_short;
+    if constexpr (EPV == 32) {
+      // 4-bit rows: the staged vector is eight times the bytes of a row.  Up to four rows are dotted side by side so
+      // that every 128-byte read of it serves all of them; codes are unpacked in pairs and multiplied with packed FMAs.
+      for (; rr_single < rows; rr_single += 4) {
+        float2 acc4[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc4[i] = make_float2(0.f, 0.f);
+        for (int c = lane; c < nvecK; c += 32) {
+          float4 xv[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) xv[q] = reinterpret_cast<const float4*>(gvec)[q * nvecK + c];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (rr_single + i < rows) {
+              float f[32];
+              Elem<T>::unpack(reinterpret_cast<const uint4*>(base + (size_t)(rr_single + i) * gate_row_bytes)[c], f);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                acc4[i] = fma2(make_float2(f[4 * q], f[4 * q + 1]), make_float2(xv[q].x, xv[q].y), acc4[i]);
+                acc4[i] = fma2(make_float2(f[4 * q + 2], f[4 * q + 3]), make_float2(xv[q].z, xv[q].w), acc4[i]);
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float z = warp_sum(acc4[i].x + acc4[i].y);
+          if (lane == rr_single + i) mine = z;
+        }
+      }
+    }
     if (EPV == 16) {
       // int8 rows: the staged vector is four times the bytes of a row, so two rows share every read of it
       for (; rr_single + 1 < rows; rr_single += 2) {
@@ -1090,16 +1121,18 @@ struct Geometry {
 
 Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   Geometry g{};
-  const int esz = weight_bytes(wkind), epv = 16 / esz;
-  const bool scaled = wkind == kWQ8;
+  const int epv = weight_epv(wkind);
+  const bool scaled = wkind == kWQ8 || wkind == kWQ4;
   const int nvecD = D / epv;
-  const int row_bytes = D * esz, gate_row_bytes = K * esz;
+  const int row_bytes = D * 16 / epv, gate_row_bytes = K * 16 / epv;
+  if (D % epv || K % epv) return g;
   g.ok = false;
   const int act_threads = 128;                 // as in the kernel: the threads of one act group
   const int gate_warps_max = lopa ? 4 : 8;
   if (row_bytes % 16 || gate_row_bytes % 16 || nvecD > act_threads * 8) return g;
   g.cpt = nvecD <= act_threads ? 1 : nvecD <= 2 * act_threads ? 2 : nvecD <= 4 * act_threads ? 4 : 8;
-  if (scaled && g.cpt == 8) return g;  // 128 accumulators per act thread: the CUDA-core path takes such rows
+  // at most 64 accumulators per act thread: the CUDA-core path takes wider rows of int8 / int4 codes
+  if (scaled && g.cpt * epv > 64) return g;
   int nr = 8192 / gate_row_bytes;
   nr = nr < 1 ? 1 : nr > 32 ? 32 : nr;
   if (lopa) {
@@ -1190,12 +1223,14 @@ int fused_grid(int sm_count, int H) {
 template <typename T, bool LOPA>
 cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaStream_t s) {
   void (*k)(const FusedParams) = nullptr;
+  constexpr int kMaxCpt = 64 / Elem<T>::kPerVec < 8 && TokenOf<T>::kScaled ? 64 / Elem<T>::kPerVec : 8;  // what plan() allows
   switch (g.cpt) {
     case 1: k = fused_ffn_kernel<T, 1, LOPA>; break;
     case 2: k = fused_ffn_kernel<T, 2, LOPA>; break;
-    case 4: k = fused_ffn_kernel<T, 4, LOPA>; break;
-    default: k = fused_ffn_kernel<T, (TokenOf<T>::kScaled ? 4 : 8), LOPA>; break;  // int8 rows: plan() never asks for 8
+    case 4: k = fused_ffn_kernel<T, (kMaxCpt >= 4 ? 4 : kMaxCpt), LOPA>; break;
+    default: k = fused_ffn_kernel<T, kMaxCpt, LOPA>; break;
   }
+  if (g.cpt > kMaxCpt) return cudaErrorInvalidValue;
   static unsigned long long configured[4] = {0, 0, 0, 0};  // per instantiation of this template, per row width
   const int slot = g.cpt == 1 ? 0 : g.cpt == 2 ? 1 : g.cpt == 4 ? 2 : 3;
   const cudaError_t e = allow_dynamic_smem(k, kSmemBudget, configured[slot]);
@@ -1286,6 +1321,8 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.trace = fused_test_knobs().trace;
   if (c.wkind == kWQ8)
     e = lopa ? launch_main<int8_t, true>(p, g, grid, s) : launch_main<int8_t, false>(p, g, grid, s);
+  else if (c.wkind == kWQ4)
+    e = lopa ? launch_main<q4_t, true>(p, g, grid, s) : launch_main<q4_t, false>(p, g, grid, s);
   else if (c.wkind == kWBF16)
     e = lopa ? launch_main<__nv_bfloat16, true>(p, g, grid, s) : launch_main<__nv_bfloat16, false>(p, g, grid, s);
   else

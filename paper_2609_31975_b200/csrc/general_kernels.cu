@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(256) rowdot_kernel(const RowDotParams p) {
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nvec = K / EPV;
-  const size_t row_bytes = (size_t)K * sizeof(T);
+  const size_t row_bytes = row_bytes_of<T>(K);
   const char* Wb = static_cast<const char*>(p.W);
   constexpr int UNROLL = 4;
 
@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(512) updown_kernel(const UpDownParams p) {
   const int hi = (int)((long long)n * (blockIdx.x + 1) / gridDim.x);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nvec = D / EPV;
-  const size_t row_bytes = (size_t)D * sizeof(T);
+  const size_t row_bytes = row_bytes_of<T>(D);
   const char* Wu = static_cast<const char*>(p.W_up);
   const char* Wd = static_cast<const char*>(p.W_down);
 
@@ -441,6 +441,10 @@ cudaError_t launch_rowdot(int wkind, bool vec_is_f32, int nb, bool gate, const R
     return vec_is_f32 ? launch_rowdot_nb<int8_t, float>(p, nb, gate, grid, s)
                       : launch_rowdot_nb<int8_t, __nv_bfloat16>(p, nb, gate, grid, s);
   }
+  if (wkind == kWQ4) {
+    return vec_is_f32 ? launch_rowdot_nb<q4_t, float>(p, nb, gate, grid, s)
+                      : launch_rowdot_nb<q4_t, __nv_bfloat16>(p, nb, gate, grid, s);
+  }
   if (wkind == kWBF16) {
     return vec_is_f32 ? launch_rowdot_nb<__nv_bfloat16, float>(p, nb, gate, grid, s)
                       : launch_rowdot_nb<__nv_bfloat16, __nv_bfloat16>(p, nb, gate, grid, s);
@@ -481,8 +485,9 @@ static cudaError_t launch_updown_d(const UpDownParams& p, int nb, int grid, cuda
 }
 
 int updown_max_tokens(int wkind, int D) {
-  const int nvec = D / (16 / weight_bytes(wkind));
+  const int nvec = D / weight_epv(wkind);
   if (wkind == kWQ8) return nvec > 1024 ? 0 : nvec > 512 ? 2 : 4;  // 16 accumulators per chunk and token
+  if (wkind == kWQ4) return nvec > 512 ? 0 : 2;                    // 32 accumulators per chunk and token
   if (nvec > 2048) return 0;
   return nvec > 1024 ? 2 : 4;
 }
@@ -497,6 +502,13 @@ cudaError_t launch_updown(int wkind, int nb, const UpDownParams& p, int grid, cu
     } else if (nvec <= 1024) {
       if (nb == 1) return launch_updown_t<int8_t, 1, 2>(p, grid, s);
       if (nb == 2) return launch_updown_t<int8_t, 2, 2>(p, grid, s);
+    }
+    return cudaErrorInvalidValue;
+  }
+  if (wkind == kWQ4) {
+    if (p.D / 32 <= 512) {
+      if (nb == 1) return launch_updown_t<q4_t, 1, 1>(p, grid, s);
+      if (nb == 2) return launch_updown_t<q4_t, 2, 1>(p, grid, s);
     }
     return cudaErrorInvalidValue;
   }
