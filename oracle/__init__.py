@@ -201,7 +201,7 @@ def dequantize_rows(q, scale) -> np.ndarray:
 
 
 def dequantize_rows_q4(packed, scale) -> np.ndarray:
-    """The matrix that 4-bit codes stand for (the same appendix converts the weights "to int8 or int4 at inference" and
+    """The matrix that 4-bit codes stand for (the same appendix also stores the weights on four bits and
     fixes no format; reading taken: symmetric two's-complement codes in [-8, 7], two per byte with the even column in
     the low nibble, one fp32 scale per row): W[j, 2b] = scale[j] * low(packed[j, b]), W[j, 2b + 1] = scale[j] *
     high(packed[j, b]), as float64.  ``packed`` is uint8 [rows, cols / 2]."""
