@@ -157,6 +157,43 @@ struct Elem<q4_t> {
   }
 };
 
+// Packed fp32 pairs kept in 64-bit registers from unpacking to the final sum, so that no instruction is spent on moving
+// halves in and out of pairs between the packed operations.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ unsigned long long fma2_b64(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2_b64(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float sum_halves(unsigned long long v) {
+  float lo, hi;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+  return lo + hi;
+}
+// Eight 4-bit codes of one word times eight entries of a vector given as four packed pairs (x0,x1) .. (x6,x7), added
+// onto a packed running sum.
+__device__ __forceinline__ unsigned long long dot8_q4(uint32_t w, const unsigned long long* xp, unsigned long long acc) {
+  w ^= 0x88888888u;
+  const uint32_t even = w & 0x0f0f0f0fu, odd = (w >> 4) & 0x0f0f0f0fu;
+  const unsigned long long bias = pack2(-8388616.f, -8388616.f);
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    const unsigned long long pr = pack2(__uint_as_float(__byte_perm(even, 0x4b000000u, 0x7650 + b)),
+                                        __uint_as_float(__byte_perm(odd, 0x4b000000u, 0x7650 + b)));
+    acc = fma2_b64(add2_b64(pr, bias), xp[b], acc);
+  }
+  return acc;
+}
+
 // Bytes of a row of n elements of storage type T (16 / kPerVec bytes per element: half a byte for 4-bit codes).
 template <typename T>
 __host__ __device__ constexpr size_t row_bytes_of(size_t n) { return n * 16 / Elem<T>::kPerVec; }

@@ -633,29 +633,28 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       // 4-bit rows: the staged vector is eight times the bytes of a row.  Up to four rows are dotted side by side so
       // that every 128-byte read of it serves all of them; codes are unpacked in pairs and multiplied with packed FMAs.
       for (; rr_single < rows; rr_single += 4) {
-        float2 acc4[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc4[i] = make_float2(0.f, 0.f);
+        unsigned long long acc4[4] = {0ull, 0ull, 0ull, 0ull};  // (0.f, 0.f)
         for (int c = lane; c < nvecK; c += 32) {
-          float4 xv[8];
+          // plane q of the staged vector holds elements 4q .. 4q+3 of every chunk: two packed pairs per 16-byte read
+          ulonglong2 xv[8];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) xv[q] = reinterpret_cast<const float4*>(gvec)[q * nvecK + c];
+          for (int q = 0; q < 8; ++q) xv[q] = reinterpret_cast<const ulonglong2*>(gvec)[q * nvecK + c];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             if (rr_single + i < rows) {
-              float f[32];
-              Elem<T>::unpack(reinterpret_cast<const uint4*>(base + (size_t)(rr_single + i) * gate_row_bytes)[c], f);
+              const uint4 w = reinterpret_cast<const uint4*>(base + (size_t)(rr_single + i) * gate_row_bytes)[c];
+              const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                acc4[i] = fma2(make_float2(f[4 * q], f[4 * q + 1]), make_float2(xv[q].x, xv[q].y), acc4[i]);
-                acc4[i] = fma2(make_float2(f[4 * q + 2], f[4 * q + 3]), make_float2(xv[q].z, xv[q].w), acc4[i]);
+              for (int k = 0; k < 4; ++k) {  // word k: elements 8k .. 8k+7 = planes 2k and 2k+1
+                const unsigned long long xp[4] = {xv[2 * k].x, xv[2 * k].y, xv[2 * k + 1].x, xv[2 * k + 1].y};
+                acc4[i] = dot8_q4(ww[k], xp, acc4[i]);
               }
             }
           }
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float z = warp_sum(acc4[i].x + acc4[i].y);
+          const float z = warp_sum(sum_halves(acc4[i]));
           if (lane == rr_single + i) mine = z;
         }
       }
