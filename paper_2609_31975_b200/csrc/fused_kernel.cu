@@ -483,10 +483,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // publishes them, and collects everybody's.  All CTAs of the call become resident without waiting for this one
     // (one CTA per SM, predecessors in the stream never wait on their successors), so the bounded wait below ends as
     // soon as the slowest CTA has started and published.  The stage sits on the call's critical path, so it is made of
-    // as few dependent memory round trips as it can be: every warp takes 32-chunk segments of the CTA's rows (all
-    // loads of a warp in flight together), the segment sums are added per row in a fixed order, and the values are
-    // published with the call's number in the same 64-bit word -- a reader that finds the number has the value, no
-    // counter and no fence in between.
+    // as few dependent memory round trips as it can be: the CTA's rows of V are in shared memory by now, the warps
+    // share them, the parts of a row are added in a fixed order, and the values are published with the call's number
+    // in the same 64-bit word -- a reader that finds the number has the value, no counter and no fence in between.
     const int r = K;
     const int st = tid - kStageBase, sw = warp - kGateProducers;
     constexpr int kSW = kStageThreads / 32;
@@ -499,16 +498,21 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     float* vpart = wss + 32;
     named_bar_sync(5, kStageThreads);  // the token is staged
     mbar_wait(v_bar, 0, ctl, p.status, p.wait_cycles, 50);
-    const int nseg = (nvecD + 31) / 32, items = (vhi - vlo) * nseg;  // fits the act ring: checked on the host
-    for (int it = sw; it < items; it += kSW) {
-      const int row = it / nseg, c = (it - row * nseg) * 32 + lane;
-      const float a = warp_sum(c < nvecD ? chunk_dot<T>(vsm[(size_t)row * nvecD + c], sx, c, nvecD, 0.f) : 0.f);
-      if (lane == 0) vpart[it] = a;
+    // the warps share the CTA's rows: wpr warps per row (one when there are more rows than warps), each lane sums its
+    // chunks in a register, one warp reduction per warp and row; the parts of a row are added in a fixed order
+    const int nrows = vhi - vlo;
+    const int wpr = nrows > 0 && nrows < kSW ? kSW / nrows : 1;
+    for (int row = sw / wpr; row < nrows; row += kSW / wpr) {
+      const int part = sw % wpr;
+      float a = 0.f;
+      for (int c = part * 32 + lane; c < nvecD; c += wpr * 32) a = chunk_dot<T>(vsm[(size_t)row * nvecD + c], sx, c, nvecD, a);
+      a = warp_sum(a);
+      if (lane == 0) vpart[row * wpr + part] = a;
     }
     named_bar_sync(5, kStageThreads);
     for (int k = vlo + st; k < vhi; k += kStageThreads) {
       float v = 0.f;
-      for (int g = 0; g < nseg; ++g) v += vpart[(k - vlo) * nseg + g];
+      for (int g = 0; g < wpr; ++g) v += vpart[(k - vlo) * wpr + g];
       if (kScaled) v *= __ldg(p.s_V + k);
       asm volatile("st.global.cg.b64 [%0], %1;" ::"l"(p.vtag + k), "l"(tagged(v, ep)) : "memory");
     }
