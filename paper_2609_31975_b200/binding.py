@@ -2,6 +2,7 @@
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 
 import torch
@@ -266,7 +267,25 @@ class SparseFFN:
         self._keep = (x, gate, b_g, W_up, W_down, y)
         _check(name, fn(self._h, _ptr(x), B, ctypes.byref(g), _ptr(b_g), _ptr(W_up), _ptr(W_down),
                         ACT[act] if isinstance(act, str) else int(act), _ptr(y), self._stream(stream)))
+        self._sync_check(name, B, gate)
         return y
+
+    def status_words(self, n: int = 8):
+        """The first ``n`` 32-bit words of the device status block (synchronises): [0] status, [1] length of the
+        index list, [3] site + 256 * CTA of the last wait that gave up, [4] number of the last failed bounds check."""
+        torch.cuda.synchronize(self.device)
+        off = self._ws_ptr - self.workspace.data_ptr()
+        return self.workspace[off:off + 4 * n].view(torch.int32).cpu().tolist()
+
+    def _sync_check(self, name, B, gate):
+        """With SFFN_SYNC_CHECK=1 in the environment every call is followed by a synchronisation and a look at the
+        status word, so that the call that set it is the one that raises (diagnostics; slow)."""
+        if os.environ.get("SFFN_SYNC_CHECK") != "1":
+            return
+        w = self.status_words()
+        if w[0] != 0:
+            raise RuntimeError(f"{name} (B={B}, {'lopa' if 'V' in gate else 'standard'} gate, D={self.D}, H={self.H}): "
+                               f"device status {w[0]}, site {w[3] % 256}, CTA {w[3] // 256}, words {w}")
 
     def _call_q8(self, fn, name, x, gate, b_g, W_up, W_down, act, y, stream):
         B = 1 if x.dim() == 1 else x.shape[0]

@@ -83,6 +83,7 @@ struct FusedParams {
   int32_t* status;
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
   int act_extra;     // LoPA: act slots inside the gate ring, used once the gate is done (0 = none)
+  int act_used;      // act slots the ring protocol cycles through: n_act_slots + act_extra, or fewer (see plan())
   int v_in_smem;     // LoPA: this CTA's rows of V are copied into the (idle) act ring at the start of the call
   int gate_workers;  // warps that take gate slots, slot s going to worker s % gate_workers: the gate warps, and for
                      // the LoPA gate also act warps (a ring slot that is reused always belongs to the same worker)
@@ -165,6 +166,14 @@ __device__ __forceinline__ void raise_timeout(volatile int* ctl, int32_t* status
   ctl[kAbort] = 1;
   status[3] = site + 256 * (int)blockIdx.x;
   atomicExch(status, (int32_t)SFFN_ERR_TIMEOUT);
+}
+
+// After a wait has run out the CTA winds down.  Copies it has issued may still be in flight; they end within
+// microseconds, so a thread that leaves an aborting CTA lets that time pass first: shared memory is only given back
+// when nothing can write to it any more.
+__device__ __forceinline__ void abort_grace(volatile int* ctl) {
+  if (ctl[kAbort])
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);
 }
 
 // Bounded wait on an mbarrier phase.  try_wait parks the thread in hardware for a short,
@@ -323,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   // Act slots: NAown in the act ring, plus (short LoPA gate) p.act_extra more that lie in the gate ring and come into
   // use once every gate row has been consumed -- from then on the rows of fired neurons are all that is left to
   // fetch, and how many of them are in flight sets how fast they come.
-  const int NG = p.n_gate_slots, NAown = p.n_act_slots, NA = NAown + p.act_extra;
+  const int NG = p.n_gate_slots, NAown = p.n_act_slots, NA = p.act_used;
   const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra);
 
   unsigned char* gate_ring = smem + L.gate_ring;
@@ -425,6 +434,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
     }
     __syncwarp();
+    abort_grace(ctl);
     return;
   }
 
@@ -1033,7 +1043,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   // still carry an older call's number (bounded).  Thread (u, rg) takes two columns (one 16-byte unit) in the rows
   // rg, rg + RG, ...; the RG row groups are then added in order through shared memory.  The other CTAs leave at once
   // and their SMs take the next kernel of the stream.
-  if (warp < kFirstGateWarp) return;  // act producers (the gate producers left long ago)
+  if (warp < kFirstGateWarp) {  // act producers (the gate producers left long ago)
+    abort_grace(ctl);
+    return;
+  }
   constexpr int kTail = 32 * (kGW + kAW);
   constexpr int kRow = CPT * EPV * kGT;        // values of a stored partial
   constexpr int kUnits = kRow / 2;             // two columns each (a multiple of 32; those past D are never written)
@@ -1045,7 +1058,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const int rank = ctl[kRank];
   const int slice = rank >= 0 && rank < R ? rank : -1;
   if (rank == G - 1 && tt == 0 && !ctl[kAbort]) *p.epoch_word = ep;  // every CTA has its number: the next call tags with ep + 1
-  if (slice < 0 || ctl[kAbort]) return;
+  if (slice < 0 || ctl[kAbort]) {
+    abort_grace(ctl);
+    return;
+  }
   if (tt == 0) SFFN_GSTAMP(8);
   constexpr int kBatch = 13;
   const int32_t failed = __ldcg(p.status);  // in flight together with the partials, not after them
@@ -1111,6 +1127,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     named_bar_sync(7, kTail);
   }
   if (tt == 0) SFFN_GSTAMP(13);
+  abort_grace(ctl);
 }
 
 // ---- host side --------------------------------------------------------------------------------
@@ -1118,6 +1135,7 @@ struct Geometry {
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max, smem, cpt;
   int gate_warps, gate_workers;
   int act_extra;   // LoPA: act slots inside the gate ring (used once the gate is done)
+  int act_used;    // act slots the ring cycles through (<= n_act_slots + act_extra)
   bool v_in_smem;  // LoPA: the CTA's rows of V are copied into the idle act ring ahead of the rank-r stage
   bool ok;
 };
@@ -1187,6 +1205,23 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
     na = (ring - ng * g.gate_slot_bytes) / g.act_slot_bytes;
     if (na > 16) na = 16;
   }
+  if (lopa && slots_of_cta > ng) {
+    // The two act groups of the LoPA kernel use act slots in fours (twos below four, see further down); where the split
+    // leaves slots over, a smaller gate ring may buy the next multiple (r = 1024 at 4096 columns: 8 + 8 instead of
+    // 12 + 6 with two idle).
+    auto usable = [](int a) { return a >= 4 ? a / 4 * 4 : a >= 2 ? 2 : 0; };
+    int best_ng = ng, best = usable(na);
+    for (int t = ng - gw; t >= gw; t -= gw) {
+      int a = (ring - t * g.gate_slot_bytes) / g.act_slot_bytes;
+      a = a > 16 ? 16 : a;
+      if (usable(a) > best) { best = usable(a); best_ng = t; }
+    }
+    if (best_ng != ng) {
+      ng = best_ng;
+      na = (ring - ng * g.gate_slot_bytes) / g.act_slot_bytes;
+      if (na > 16) na = 16;
+    }
+  }
   g.n_act_slots = na;
   g.n_gate_slots = ng;
   // the rank-r stage keeps the CTA's rows of V and one sum per 32-chunk segment of them in the (then idle) act ring
@@ -1198,6 +1233,16 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   if (lopa && slots_of_cta <= ng) {
     g.act_extra = (int)((size_t)ng * g.gate_slot_bytes / g.act_slot_bytes);
     if (na + g.act_extra > 16) g.act_extra = 16 - na;
+  }
+  // Two act groups take alternate rounds.  A ring slot must always come back to the same group: a group that shared a
+  // slot with the other one could arrive for its next row there while the other group's row in between has not landed,
+  // and the barrier's parity cannot tell that phase from the one two back (seen as rare timeouts and a fault at
+  // 8192 x 28672, three act slots).  So the slots in use are a multiple of what the two groups take per lap.
+  g.act_used = na + g.act_extra;
+  if (lopa) {
+    g.act_used = g.act_used >= 4 ? g.act_used / 4 * 4 : g.act_used >= 2 ? 2 : 0;
+    if (g.act_used == 0) return g;
+    g.act_extra = g.act_used > na ? g.act_used - na : 0;
   }
   if (lopa) {
     const size_t v_max = (size_t)(K + grid - 1) / grid, sums = (v_max * ((nvecD + 31) / 32) + 32) * 4;
@@ -1318,7 +1363,7 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;
-  p.gate_warps = g.gate_warps; p.gate_workers = g.gate_workers; p.v_in_smem = g.v_in_smem ? 1 : 0; p.act_extra = g.act_extra;
+  p.gate_warps = g.gate_warps; p.gate_workers = g.gate_workers; p.v_in_smem = g.v_in_smem ? 1 : 0; p.act_extra = g.act_extra; p.act_used = g.act_used;
   p.wait_cycles = fused_test_knobs().wait_cycles;
   p.skip_arrival_cta = fused_test_knobs().skip_arrival_cta;
   p.trace = fused_test_knobs().trace;

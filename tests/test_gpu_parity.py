@@ -56,7 +56,7 @@ def run_both_paths(mod, ffn, x, gate, w, act, paths, tol=None, what=""):
         ffn.set_path(path)
         y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], act)
         torch.cuda.synchronize()
-        assert ffn.device_status() == 0
+        assert ffn.device_status() == 0, f"{what} [{path}]: status words {ffn.status_words()}"
         assert_y_close(y, ref["y"], what=f"{what} [{path}]", **kw)
         assert_active_set(ffn.last_active(), ref, what=f"{what} [{path}]")
     ffn.set_path("auto")
@@ -561,3 +561,23 @@ def test_gate_engine_setting_and_a_long_chain_of_mixed_calls(mod):
     torch.cuda.synchronize()
     assert ffn.device_status() == 0
     assert torch.equal(first, out)
+
+
+def test_lopa_act_groups_keep_their_ring_slots(mod):
+    # 16 KB rows leave the LoPA kernel few act slots; its two act groups must each keep their own (a slot that went back
+    # and forth between them let a group read the other's row when that row was late: rare timeouts, once a fault).
+    # Every call is followed by a synchronisation -- all CTAs then start at once, which is what provoked it -- and must
+    # repeat the first result bit for bit.
+    D, H, r = 8192, 4096, 1024
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=r, B_max=1)
+    lg, lw = make_lopa(mod, D, H, r, torch.bfloat16, 61, 0.8, "diag")
+    x = syn.tokens(2, D, torch.bfloat16, 61, DEV)
+    ref = run_both_paths(mod, ffn, x[0], lg, lw, "relu", ("fused",), what="lopa 8192 r=1024")
+    assert 0 < ref["n_act"][0] < H
+    ffn.set_path("fused")
+    first = [ffn.sparse_ffn_forward(x[t], lg, lw["b_g"], lw["W_up"], lw["W_down"], "relu").clone() for t in range(2)]
+    for rep in range(40):
+        y = ffn.sparse_ffn_forward(x[rep % 2], lg, lw["b_g"], lw["W_up"], lw["W_down"], "relu")
+        torch.cuda.synchronize()
+        assert ffn.device_status() == 0, f"rep {rep}: status words {ffn.status_words()}"
+        assert torch.equal(y, first[rep % 2]), f"rep {rep}"
