@@ -280,7 +280,7 @@ class SparseFFN:
     def _sync_check(self, name, B, gate):
         """With SFFN_SYNC_CHECK=1 in the environment every call is followed by a synchronisation and a look at the
         status word, so that the call that set it is the one that raises (diagnostics; slow)."""
-        if os.environ.get("SFFN_SYNC_CHECK") != "1":
+        if os.environ.get("SFFN_SYNC_CHECK") != "1" or torch.cuda.is_current_stream_capturing():
             return
         w = self.status_words()
         if w[0] != 0:
