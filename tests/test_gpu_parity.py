@@ -581,3 +581,86 @@ def test_lopa_act_groups_keep_their_ring_slots(mod):
         torch.cuda.synchronize()
         assert ffn.device_status() == 0, f"rep {rep}: status words {ffn.status_words()}"
         assert torch.equal(y, first[rep % 2]), f"rep {rep}"
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_fused_path_agrees_with_the_cuda_core_path(mod, seed):
+    # Seeded random geometries (row widths, neuron counts that leave ragged slabs, LoPA ranks, storage types, both
+    # gate engines, repeated calls): the single-token kernels against the plain CUDA-core kernels, which share none
+    # of their code; both within the usual tolerance of each other, no wait runs out, and repeats are bit for bit.
+    g = torch.Generator().manual_seed(1000 + seed)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))  # noqa: E731
+    for case in range(7):
+        dtype = (torch.bfloat16, torch.bfloat16, torch.float32)[ri(0, 2)]
+        D = 64 * ri(4, 72) if dtype == torch.bfloat16 else 64 * ri(4, 40)
+        H = ri(60, 5000)
+        lopa = ri(0, 1) == 1
+        r = 32 * ri(1, min(24, D // 64)) if lopa else 0
+        s = (0.5, 0.8, 0.9, 0.97)[ri(0, 3)]
+        act = ("relu", "sqrelu", "rsplus")[ri(0, 2)]
+        what = f"seed {seed} case {case}: D={D} H={H} r={r} {dtype} s={s} {act}"
+        ffn = mod.SparseFFN(D, H, dtype, r_max=r, B_max=1)
+        if lopa:
+            gate, w = make_lopa(mod, D, H, r, dtype, 2000 + 10 * seed + case, s, ("diag", "tiled", None)[ri(0, 2)],
+                                sign=ri(0, 1) == 1, gain=ri(0, 1) == 1, rms=ri(0, 1) == 1)
+        else:
+            gate, w = make_std(D, H, dtype, 2000 + 10 * seed + case, s)
+        x = syn.tokens(2, D, dtype, 3000 + seed, DEV)
+        ffn.set_path("general")
+        want = [ffn.sparse_ffn_forward(x[t], gate, w["b_g"], w["W_up"], w["W_down"], act).clone() for t in range(2)]
+        ffn.set_path("auto")
+        for engine in ("cuda_core", "tensor_core"):
+            ffn.set_gate_engine(engine)
+            got = []
+            for rep in range(3):
+                for t in range(2):
+                    y = ffn.sparse_ffn_forward(x[t], gate, w["b_g"], w["W_up"], w["W_down"], act)
+                    if rep == 0:
+                        got.append(y.clone())
+                        assert_y_close(y, want[t].double().cpu().numpy(), rel_l2=2e-3, max_abs=2e-3,
+                                       what=f"{what} [{engine}] token {t}")
+                    else:
+                        assert torch.equal(y, got[t]), f"{what} [{engine}] repeat {rep} token {t}"
+            torch.cuda.synchronize()
+            assert ffn.device_status() == 0, f"{what} [{engine}]: status words {ffn.status_words()}"
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_shapes_batched_paths_agree_with_the_cuda_core_path(mod, seed):
+    # The same for batches: whatever `auto` picks (the tcgen05 kernels where the shape allows) and the mma.sync kernels
+    # against the CUDA-core kernels, random batch sizes, widths, neuron counts and LoPA ranks.
+    g = torch.Generator().manual_seed(5000 + seed)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))  # noqa: E731
+    for case in range(6):
+        B = ri(2, 64)
+        D = 128 * ri(2, 32)
+        H = ri(100, 6000)
+        lopa = ri(0, 2) == 0
+        r = 64 * ri(1, min(8, D // 128)) if lopa else 0
+        s = (0.6, 0.8, 0.9, 0.97)[ri(0, 3)]
+        act = ("relu", "sqrelu", "rsplus")[ri(0, 2)]
+        what = f"seed {seed} case {case}: B={B} D={D} H={H} r={r} s={s} {act}"
+        ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=r, B_max=B)
+        if lopa:
+            gate, w = make_lopa(mod, D, H, r, torch.bfloat16, 6000 + 10 * seed + case, s, ("diag", None)[ri(0, 1)],
+                                rms=ri(0, 1) == 1)
+        else:
+            gate, w = make_std(D, H, torch.bfloat16, 6000 + 10 * seed + case, s)
+        x = syn.tokens(B, D, torch.bfloat16, 7000 + seed, DEV)
+        ffn.set_path("general")
+        want = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], act).double().cpu().numpy()
+        n_want = int(ffn.last_active().numel())
+        for path in ("auto", "mma_sync"):
+            ffn.set_path(path)
+            try:
+                y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], act)
+            except mod.SFFNError as e:            # a shape the mma.sync kernels do not take
+                assert path == "mma_sync" and e.code == 2, what
+                continue
+            # the tensor-core paths round h and the LoPA vector to bf16 pairs: a looser band than fp32 against fp32
+            assert_y_close(y, want, rel_l2=1e-2, max_abs=2e-2, what=f"{what} [{path}]")
+            assert abs(int(ffn.last_active().numel()) - n_want) <= max(4, n_want // 200), f"{what} [{path}]"
+            y2 = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], act)
+            assert torch.equal(y, y2), f"{what} [{path}] repeat"
+            torch.cuda.synchronize()
+            assert ffn.device_status() == 0, f"{what} [{path}]: status words {ffn.status_words()}"
