@@ -11,15 +11,16 @@
 //                  a_j = A(z_j), and publishes "fired" (z_j > 0) per neuron.
 //   act producers  two warps walk the published results in ascending neuron order and queue the
 //                  W_up / W_down rows of the neurons that fired into a second ring.
-//   act warps      four warps (eight for the LoPA gate, which needs only four gate warps) consume the
-//                  second ring in order: u_j = W_up[j] . x (CTA-level
-//                  reduction), h_j = a_j u_j, y_part += h_j W_down[j]; each thread keeps its own
-//                  column slice of y_part in registers and writes it out once.
+//   act warps      four warps (for the LoPA gate two groups of four on alternate rounds, and four gate warps)
+//                  consume the second ring in order: u_j = W_up[j] . x (reduction over the group),
+//                  h_j = a_j u_j, y_part += h_j W_down[j]; each thread keeps its own column slice of y_part in
+//                  registers and writes it out once.
 //
-// The last CTAs to finish sum the per-CTA partials in CTA order (deterministic, no float atomics).
-// Weights are fp32, bf16 or int8 codes with one fp32 scale per row (bf16 token).
+// The first CTAs to finish sum the per-CTA partials in CTA order (deterministic, no float atomics): every partial
+// value is stored with the call's number in the same 64-bit word, so the summing CTAs need no counter or fence.
+// Weights are fp32, bf16, int8 codes or packed 4-bit codes with one fp32 scale per row (bf16 token).
 // For the LoPA gate (Eq. 3, Sec. 3.3) the rank-r stage v = V x is spread over the CTAs of the main
-// kernel, exchanged through global memory (bounded wait on an arrival counter) and normalised (RMSNorm)
+// kernel, exchanged through global memory as tagged values (bounded re-reads) and normalised (RMSNorm)
 // into shared memory, with the U rows already sitting in the ring.
 //
 // Calls are chained with programmatic dependent launch: a kernel lets its successor start early
