@@ -37,7 +37,7 @@
  * written by device work queued immediately before a call on the same stream -- put a stream or event
  * synchronisation between an update of the weights and the next call.
  * A single-token call runs one CTA on every SM, and its CTAs wait for one another (LoPA: for the rank-r vector;
- * always: the last CTAs to finish wait for the rest before they sum the partial results; every wait is bounded).
+ * always: the first CTAs to finish stay and wait for the partial results of the rest, which they sum; every wait is bounded).
  * Calls of different handles are therefore meant to run one after another -- one stream, or streams ordered by
  * events.  Two standard-gate calls that overlap still complete; LoPA calls, or three and more calls at once, can
  * starve each other of SMs and end with SFFN_ERR_TIMEOUT in the device status instead of a result.
