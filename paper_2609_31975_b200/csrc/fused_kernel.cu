@@ -84,6 +84,7 @@ struct FusedParams {
   int32_t* status;
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
   int act_extra;     // LoPA: act slots inside the gate ring, used once the gate is done (0 = none)
+  int act_groups;    // act groups: 1, LoPA 2, or 3 when the gate warps join as a group of their own after the gate
   int act_used;      // act slots the ring protocol cycles through: n_act_slots + act_extra, or fewer (see plan())
   int v_in_smem;     // LoPA: this CTA's rows of V are copied into the (idle) act ring at the start of the call
   int gate_workers;  // warps that take gate slots, slot s going to worker s % gate_workers: the gate warps, and for
@@ -112,7 +113,7 @@ struct SmemLayout {
     sn = take(lopa ? K * 4 : 0);
     aval = take(slab_max * 4);
     slot_a = take((n_act_slots + act_extra) * 4);
-    red = take(4 * (2 * 4 + 1) * 4);  // two buffers per act group (four warps each), up to two groups
+    red = take(6 * (2 * 4 + 1) * 4);  // two buffers per act group (four warps each), up to three groups
     ctl = take(8 * 4);
     bars = take(2 * (n_gate_slots + n_act_slots + act_extra) * 8 + 8);  // + one for the CTA's rows of V (LoPA)
     row_params = take((lopa || scaled) ? (1 + (lopa ? 2 : 0) + (scaled ? 1 : 0)) * slab_max * 4 : 0);  // per-neuron gate parameters
@@ -400,7 +401,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
       mbar_init(v_bar, 1);
       for (int i = 0; i < 8; ++i) ctl[i] = 0;
-      for (int i = 0; i < 4 * (2 * 4 + 1); ++i) red[i] = 0.f;
+      for (int i = 0; i < 6 * (2 * 4 + 1); ++i) red[i] = 0.f;
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -806,7 +807,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     if (lane == 0 && ap == 0) SFFN_STAMP(7);
     if (lane == 0) {
       const int per_round = NA >= 4 ? 2 : 1;
-      const int n_end = kGroups == 1 ? n_seq + 1 : (n_seq / per_round + kGroups) * per_round;
+      const int n_end = p.act_groups == 1 ? n_seq + 1 : (n_seq / per_round + p.act_groups) * per_round;
       for (; ok && n_seq < n_end; ++n_seq) {
         if (mbar_wait<true>(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 43)) {
           if (ap == 0) slot_a[slot] = -1.f;
@@ -837,19 +838,24 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       asm volatile("bar.arrive 6, %0;" ::"r"(32 * (kGW + kAW) + 32) : "memory");
     }
     __syncwarp();
-  } else if (warp < kFAW) {
-    // ======================= gate warps ========================================================
-    for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_workers)
-      if (!gate_slot(s)) break;
-    if (lane == 0 && gw == (n_gslots - 1) % p.gate_workers) SFFN_STAMP(3);
   } else {
+    const bool gate_warp = warp < kFAW;
+    if (gate_warp) {
+      // ======================= gate warps ========================================================
+      for (int s = gw; gw < p.gate_warps && s < n_gslots; s += p.gate_workers)
+        if (!gate_slot(s)) break;
+      if (lane == 0 && gw == (n_gslots - 1) % p.gate_workers) SFFN_STAMP(3);
+    }
     // ======================= act warps =========================================================
-    const int at = tid - 32 * kFAW;
-    const int aw = warp - kFAW;
+    // (LoPA with three act groups: the four gate warps, done with the short gate, are the third group)
+    const bool third = LOPA && gate_warp && p.act_groups == 3;
+    if (!gate_warp || third) {
+    const int at = gate_warp ? kAT + tid - 32 * kFirstGateWarp : tid - 32 * kFAW;
+    const int aw = at >> 5;
     const int grp = aw / kGAW, gaw = aw % kGAW, gat = at % kGT;  // act group, warp and thread within it
     // Short gate (LoPA): the act warps have nothing to do until the first fired rows arrive, so they take gate slots
     // too -- with a dozen warps on it the whole gate is one or two slots per warp.
-    if (LOPA) {
+    if (LOPA && !gate_warp) {
       for (int s = p.gate_warps + aw; s < n_gslots; s += p.gate_workers)
         if (p.gate_warps + aw >= p.gate_workers || !gate_slot(s)) break;
       if (lane == 0 && p.gate_warps + aw == (n_gslots - 1) % p.gate_workers) SFFN_STAMP(3);
@@ -882,7 +888,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // wait ran out still joins the barrier and raises the group's stop flag, so the four warps
     // always leave the loop together.
     const bool pair = NA >= 4;  // with fewer slots, holding two at a time would stall the act producers
-    const int stride = (pair ? 2 : 1) * kGroups;  // ring slots from one round of a group to its next
+    const int stride = (pair ? 2 : 1) * p.act_groups;  // ring slots from one round of a group to its next
     int slot = (pair ? 2 : 1) * grp;
     uint32_t par = 0;
     while (slot >= NA) { slot -= NA; par ^= 1; }
@@ -999,21 +1005,24 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     }
     if (at == 0) SFFN_STAMP(4);
     if (kGroups == 2) {
-      // the second group's sums go to the first through the act ring, once both groups have left it
+      // the other groups' sums go to the first through the act ring, once every group has left it; added in group order
       float* xch = reinterpret_cast<float*>(act_ring);
-      named_bar_sync(9, kAT);
-      if (grp == 1) {
+      const int merge_threads = kGT * p.act_groups;
+      named_bar_sync(9, merge_threads);
+      if (grp > 0) {
 #pragma unroll
         for (int i = 0; i < CPT; ++i)
 #pragma unroll
-          for (int e = 0; e < EPV; ++e) xch[(i * EPV + e) * kGT + gat] = acc[i][e];
+          for (int e = 0; e < EPV; ++e) xch[(grp - 1) * (CPT * EPV * kGT) + (i * EPV + e) * kGT + gat] = acc[i][e];
       }
-      named_bar_sync(9, kAT);
+      named_bar_sync(9, merge_threads);
       if (grp == 0) {
+        for (int og = 1; og < p.act_groups; ++og) {
 #pragma unroll
-        for (int i = 0; i < CPT; ++i)
+          for (int i = 0; i < CPT; ++i)
 #pragma unroll
-          for (int e = 0; e < EPV; ++e) acc[i][e] += xch[(i * EPV + e) * kGT + gat];
+            for (int e = 0; e < EPV; ++e) acc[i][e] += xch[(og - 1) * (CPT * EPV * kGT) + (i * EPV + e) * kGT + gat];
+        }
       }
     }
     // This CTA's partial of y, every value tagged with the call's number.  Stored unit (two columns, 16 bytes)
@@ -1034,6 +1043,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     }
     if (at == 0) SFFN_STAMP(5);
     if (at == 0) SFFN_GSTAMP(12);
+    }
   }
 
   // ---- y = sum over CTAs of their partials, by the first CTAs to finish ------------------------------------------
@@ -1137,6 +1147,7 @@ struct Geometry {
   int gate_warps, gate_workers;
   int act_extra;   // LoPA: act slots inside the gate ring (used once the gate is done)
   int act_used;    // act slots the ring cycles through (<= n_act_slots + act_extra)
+  int act_groups;  // groups of four warps that take alternate rounds of the act ring (LoPA: 2 or 3)
   bool v_in_smem;  // LoPA: the CTA's rows of V are copied into the idle act ring ahead of the rank-r stage
   bool ok;
 };
@@ -1240,9 +1251,18 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   // and the barrier's parity cannot tell that phase from the one two back (seen as rare timeouts and a fault at
   // 8192 x 28672, three act slots).  So the slots in use are a multiple of what the two groups take per lap.
   g.act_used = na + g.act_extra;
+  g.act_groups = lopa ? 2 : 1;
   if (lopa) {
-    g.act_used = g.act_used >= 4 ? g.act_used / 4 * 4 : g.act_used >= 2 ? 2 : 0;
+    const int total = g.act_used;
+    g.act_used = total >= 4 ? total / 4 * 4 : total >= 2 ? 2 : 0;
     if (g.act_used == 0) return g;
+    // Three groups (the gate warps join once the short gate is done) where that costs no slots (six per lap) and the
+    // merge of three sets of sums fits the act ring.
+    if (slots_of_cta <= ng && total >= 6 && total / 6 * 6 >= g.act_used &&
+        (size_t)na * g.act_slot_bytes >= (size_t)2 * g.cpt * epv * act_threads * 4) {
+      g.act_groups = 3;
+      g.act_used = total / 6 * 6;
+    }
     g.act_extra = g.act_used > na ? g.act_used - na : 0;
   }
   if (lopa) {
@@ -1364,7 +1384,7 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;
-  p.gate_warps = g.gate_warps; p.gate_workers = g.gate_workers; p.v_in_smem = g.v_in_smem ? 1 : 0; p.act_extra = g.act_extra; p.act_used = g.act_used;
+  p.gate_warps = g.gate_warps; p.gate_workers = g.gate_workers; p.v_in_smem = g.v_in_smem ? 1 : 0; p.act_extra = g.act_extra; p.act_used = g.act_used; p.act_groups = g.act_groups;
   p.wait_cycles = fused_test_knobs().wait_cycles;
   p.skip_arrival_cta = fused_test_knobs().skip_arrival_cta;
   p.trace = fused_test_knobs().trace;
