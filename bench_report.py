@@ -52,6 +52,24 @@ def _time(calls, stream, reps=3):
     return statistics.median(best), min(best)
 
 
+def _call_intervals(calls, stream):
+    """Spacing of consecutive calls with an event recorded after every call: median and 95th percentile in
+    microseconds.  The event records keep consecutive calls from overlapping (no dependent-launch overlap across an
+    event), so these intervals are those of isolated calls, longer than the back-to-back figure."""
+    with torch.cuda.stream(stream):
+        for c in calls[: min(len(calls), 16)]:
+            c()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)]
+        ev[0].record(stream)
+        for i, c in enumerate(calls):
+            c()
+            ev[i + 1].record(stream)
+        torch.cuda.synchronize()
+    d = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(len(calls)))
+    return d[len(d) // 2], d[min(len(d) - 1, int(0.95 * len(d)))]
+
+
 def _time_graph(calls, stream, replays=5):
     """The same sequence of calls captured once in a CUDA graph and replayed: no host work between the calls."""
     with torch.cuda.stream(stream):
@@ -143,6 +161,7 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=None, a
     n_rows = statistics.mean(rows)
     us, us_min = _time_graph(sparse_calls, stream) if graph else _time(sparse_calls, stream)
     us_dense, _ = _time(dense_calls[: max(16, n_calls // 4)], stream, reps=2)
+    iv_med, iv_p95 = _call_intervals(sparse_calls, stream)
     us_lib = None
     if not _is_q8(sets[0]) and "W_g" in gate_of(sets[0]):
         us_lib, _ = _time(_library_dense_calls(sets, x, act, max(16, n_calls // 4)), stream, reps=2)
@@ -150,7 +169,8 @@ def measure(name, D, H, B, sets, gate_of, act, r=None, n_calls=200, peak=None, a
     q8 = _is_q8(sets[0])
     nbytes = _bytes(D, H, round(n_rows), 2, B, r, q8)
     row = dict(name=name, D=D, H=H, B=B, r=r, act=act, fired_rows=n_rows, fired_frac=n_rows / H,
-               us_per_call=us, us_min=us_min, tokens_per_s=B * 1e6 / us, touched_mb=nbytes / 1e6,
+               us_per_call=us, us_min=us_min, us_interval_median=iv_med, us_interval_p95=iv_p95,
+               tokens_per_s=B * 1e6 / us, touched_mb=nbytes / 1e6,
                gbs=nbytes / us / 1e3, frac_measured_peak=nbytes / us / 1e3 / peak,
                frac_nominal=nbytes / us / 1e3 / NOMINAL, dense_us=us_dense,
                dense_gbs=_bytes(D, H, H, 2, B, r, q8) / us_dense / 1e3, speedup_vs_dense=us_dense / us,
@@ -287,6 +307,8 @@ def run(out_path, quick=False, only=None, n_calls=None):
             lsets.append(lw)
         lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}
         add("lopa r=512 relu int8", D, H, 1, lsets, lg, "relu", r=512, peak=peak)
+        if not quick:
+            add("batched B=16 int8 (token by token)", D, H, 16, qsets, std, "relu", n_calls=40, peak=peak)
         del qsets, lsets
         torch.cuda.empty_cache()
     # weight-only int4 (packed 4-bit codes + one fp32 scale per row)

@@ -163,8 +163,9 @@ int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate
  * int8 codes ([H,D], [H,D], [H,D], [r,D], [H,r]); `scales` carries the row scales.  Tokens x are bf16: the handle
  * must have been created with SFFN_BF16.  Rows must be a multiple of 16 bytes (D and r multiples of 16).
  * Everything else (b_g, g_idx, g_sign, RMSNorm, act, y, the active list, double activation) is as in
- * sparse_ffn_forward / dense_ffn_forward.  One token runs in the fused kernels, batches in the CUDA-core
- * kernels (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is an offline
+ * sparse_ffn_forward / dense_ffn_forward.  One token runs in the fused kernel; a batch runs that kernel once per
+ * token (the list of fired neurons is the union over the tokens), or the CUDA-core batch kernels under
+ * SFFN_PATH_GENERAL (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is an offline
  * step outside this library. */
 typedef struct {
   const float* s_gate; /* [H]  row scales of W_g (STANDARD) or of U (LOPA) */

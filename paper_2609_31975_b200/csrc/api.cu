@@ -515,6 +515,32 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
   if (rc != SFFN_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int wkind = q8 ? (qbits == 4 ? sffn::kWQ4 : sffn::kWQ8) : h->dtype == SFFN_BF16 ? sffn::kWBF16 : sffn::kWF32;
+  // Batches of int8 / int4 rows: the single-token kernel once per token (the tensor-core batch kernels take bf16
+  // operands only, and the CUDA-core batch kernels are many times slower than B single-token calls: 1.66 ms against
+  // 0.33 ms at 4096 x 14336, B = 16).  The fired flags of the tokens are OR-ed: the list is the batch's union.
+  if (q8 && B > 1 && h->path != SFFN_PATH_GENERAL && h->path != SFFN_PATH_MMA_SYNC &&
+      sffn::fused_supported(wkind, h->D, h->H, 1, g, h->sm_count)) {
+    for (int b = 0; b < B; ++b) {
+      sffn::FusedCall c{};
+      c.wkind = wkind;
+      c.s_gate = q8->s_gate; c.s_V = q8->s_V; c.s_up = q8->s_up; c.s_down = q8->s_down;
+      c.D = h->D; c.H = h->H;
+      c.x = static_cast<const char*>(x) + (size_t)b * h->D * 2;  // bf16 tokens
+      c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up;
+      c.engine = h->gate_engine; c.y = y + (size_t)b * h->D;
+      c.dense = dense; c.flag_or = b > 0;
+      c.workspace = h->ws + h->L.fused;
+      c.r_max = h->r_max;
+      c.status = h->at<int32_t>(h->L.status);
+      c.flag = h->at<uint8_t>(h->L.flag);
+      c.sm_count = h->sm_count;
+      int launched = 0;
+      if (sffn::launch_fused(c, s, &launched) != cudaSuccess) return SFFN_ERR_CUDA;
+      h->launches += launched;
+    }
+    if (!dense) h->list_state = 2;
+    return SFFN_OK;
+  }
   const bool fused_ok = sffn::fused_supported(wkind, h->D, h->H, B, g, h->sm_count);
   if (h->path == SFFN_PATH_FUSED && !fused_ok) return SFFN_ERR_UNSUPPORTED;
   if (fused_ok && h->path != SFFN_PATH_GENERAL) {

@@ -81,6 +81,7 @@ struct FusedParams {
   unsigned long long* partial;  // [grid][row] per-CTA partials of y, each value paired with the call's number
   uint32_t* epoch_word;         // number of calls completed on this workspace
   uint8_t* flag;
+  int flag_or;       // 1 = flags are only set, never cleared (later tokens of a batch run token by token)
   int32_t* status;
   int rows_per_gate_slot, gate_slot_bytes, n_gate_slots, act_slot_bytes, n_act_slots, slab_max;
   int act_extra;     // LoPA: act slots inside the gate ring, used once the gate is done (0 = none)
@@ -710,7 +711,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     if (lane < rows) {
       const float z = kScaled ? fmaf(mine, scale, add) : mine + add;
       const bool fired = z > 0.f;
-      if (!p.dense && SFFN_IN_BOUNDS(j0 + lane < p.H && r0 + lane < p.slab_max, p.status, 3)) p.flag[j0 + lane] = fired ? 1 : 0;
+      if (!p.dense && (fired || !p.flag_or) && SFFN_IN_BOUNDS(j0 + lane < p.H && r0 + lane < p.slab_max, p.status, 3))
+        p.flag[j0 + lane] = fired ? 1 : 0;
       row_state[r0 + lane] = fired ? __float_as_uint(fmaxf(activation(p.act, z), 0.f)) : 0x80000000u;
     }
     __syncwarp();
@@ -1380,7 +1382,7 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   p.act = c.act; p.dense = c.dense ? 1 : 0;
   p.act_up = c.act_up;
   p.s_gate = c.s_gate; p.s_V = c.s_V; p.s_up = c.s_up; p.s_down = c.s_down;
-  p.flag = c.flag; p.status = c.status;
+  p.flag = c.flag; p.flag_or = c.flag_or ? 1 : 0; p.status = c.status;
   p.rows_per_gate_slot = g.rows_per_gate_slot; p.gate_slot_bytes = g.gate_slot_bytes;
   p.n_gate_slots = g.n_gate_slots; p.act_slot_bytes = g.act_slot_bytes; p.n_act_slots = g.n_act_slots;
   p.slab_max = g.slab_max;

@@ -30,6 +30,7 @@ struct FusedCall {
   void* workspace;   // fused_workspace_bytes() bytes, zeroed at handle creation
   int32_t* status;   // device status word
   uint8_t* flag;     // [H] "neuron fired" bytes (sparse calls)
+  bool flag_or;      // the bytes are only ever set (a batch run token by token: the union of the tokens' fired sets)
   int sm_count;
 };
 

@@ -83,7 +83,7 @@ def test_int4_lopa_gate_one_token(mod, r, fixed, rms):
 
 
 @pytest.mark.parametrize("B", [2, 5])
-def test_int4_batches_take_the_cuda_core_kernels(mod, B):
+def test_int4_batches_token_by_token_and_on_the_cuda_core_kernels(mod, B):
     D, H = 1024, 2049
     ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=64, B_max=B)
     gate, w = make_std(D, H, 33, 0.8)

@@ -91,12 +91,13 @@ def test_int8_lopa_gate_one_token(mod, r, fixed, sign, gain, rms):
 
 
 @pytest.mark.parametrize("B", [2, 3, 4, 7, 16])
-def test_int8_batches_take_the_cuda_core_kernels(mod, B):
+def test_int8_batches_token_by_token_and_on_the_cuda_core_kernels(mod, B):
     D, H = 1024, 2500
     ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=128, B_max=16)
     gate, w = make_std(D, H, 13, 0.9)
     x = syn.tokens(B, D, torch.bfloat16, 13, DEV)
-    ref = check(mod, ffn, x, gate, w, "relu", ("auto", "general"), f"q8 B={B}")
+    # auto / fused: the single-token kernel once per token, flags OR-ed into the union; general: the batch kernels
+    ref = check(mod, ffn, x, gate, w, "relu", ("auto", "fused", "general"), f"q8 B={B}")
     assert ref["union_mask"].sum() > ref["n_act"].max() or B == 1
     gate, w = make_lopa(mod, D, H, 128, 13, 0.9, sign=True, gain=True)
     check(mod, ffn, x, gate, w, "rsplus", ("auto",), f"q8 lopa B={B}")
