@@ -79,9 +79,12 @@ typedef enum { SFFN_F32 = 0, SFFN_BF16 = 1 } sffn_dtype;
 
 typedef enum { SFFN_GATE_STANDARD = 0, SFFN_GATE_LOPA = 1 } sffn_gate_kind;
 
-/* Which kernels serve a call.  AUTO picks the fused kernels for B = 1 when the shape allows it, the
- * tcgen05 tensor-core kernels for bf16 batches (B >= 2) and the general CUDA-core kernels otherwise;
- * the others force one family (SFFN_ERR_UNSUPPORTED if it cannot serve the call): GENERAL = CUDA-core
+/* Which kernels serve a call.  AUTO picks the fused kernels for B = 1 when the shape allows it and the
+ * tcgen05 tensor-core kernels for bf16 batches (B >= 2; more than 64 tokens run in chunks of 64, the list
+ * of fired neurons being the union over all chunks).  A batch those kernels do not take (fp32 or quantised
+ * weights, a row width they do not tile) runs the fused kernel once per token with the fired flags OR-ed,
+ * which is faster than the CUDA-core batch kernels; what is left goes to the general CUDA-core kernels.
+ * The others force one family (SFFN_ERR_UNSUPPORTED if it cannot serve the call): GENERAL = CUDA-core
  * kernels for any batch, FUSED = single-token fused kernels, MMA_SYNC = batched kernels on the
  * warp-level mma.sync tensor-core path. */
 typedef enum { SFFN_PATH_AUTO = 0, SFFN_PATH_GENERAL = 1, SFFN_PATH_FUSED = 2, SFFN_PATH_MMA_SYNC = 3 } sffn_path;
@@ -186,7 +189,8 @@ int dense_ffn_forward_q8(sffn_handle* handle, const void* x, int B, const sffn_g
  *     W[j, 2b] = s[j] * low_nibble(p[j, b]),   W[j, 2b + 1] = s[j] * high_nibble(p[j, b]).
  * The weight pointers address the packed bytes ([H, D/2], [r, D/2], [H, r/2]); `scales` as for int8.  Rows must be a
  * multiple of 16 bytes (D and r multiples of 32).  Otherwise exactly like the _q8 calls: bf16 tokens, fp32 arithmetic,
- * one token in the fused kernel (rows of up to 8192 codes there), batches and wider rows in the CUDA-core kernels. */
+ * one token in the fused kernel (rows of up to 8192 codes there), a batch once per token, wider rows in the CUDA-core
+ * kernels. */
 int sparse_ffn_forward_q4(sffn_handle* handle, const void* x, int B, const sffn_gate* gate, const float* b_g,
                           const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
                           void* stream);

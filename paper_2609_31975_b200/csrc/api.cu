@@ -25,7 +25,7 @@ constexpr int kMaxMmaTokens = 64;    // tokens per pass of the batched tensor-co
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-  size_t status, act, flag, idx, v, n, partial, xstage, ystage, fused, hmT, x2, total;
+  size_t status, act, flag, idx, v, n, partial, xstage, ystage, fused, hmT, x2, union_flag, total;
   int hm_stride;
 };
 
@@ -53,6 +53,7 @@ Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
   L.hm_stride = (H + 63) / 64 * 64 + 64;
   L.hmT = take((size_t)(B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * L.hm_stride * 2);
   L.x2 = take((size_t)2 * (B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * (r_max > 0 ? r_max : 1) * 2);
+  L.union_flag = take((size_t)H + 256);  // fired flags accumulated over the chunks of a batch of more than 64 tokens
   L.total = off;
   return L;
 }
@@ -515,17 +516,25 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
   if (rc != SFFN_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int wkind = q8 ? (qbits == 4 ? sffn::kWQ4 : sffn::kWQ8) : h->dtype == SFFN_BF16 ? sffn::kWBF16 : sffn::kWF32;
-  // Batches of int8 / int4 rows: the single-token kernel once per token (the tensor-core batch kernels take bf16
-  // operands only, and the CUDA-core batch kernels are many times slower than B single-token calls: 1.66 ms against
-  // 0.33 ms at 4096 x 14336, B = 16).  The fired flags of the tokens are OR-ed: the list is the batch's union.
-  if (q8 && B > 1 && h->path != SFFN_PATH_GENERAL && h->path != SFFN_PATH_MMA_SYNC &&
+  const bool lopa_gate = g->kind == SFFN_GATE_LOPA;
+  const int gate_k = lopa_gate ? g->r : h->D;
+  const int chunk = B < kMaxMmaTokens ? B : kMaxMmaTokens;
+  // a batch the tensor-core kernels can take (bf16 rows; more than 64 tokens: in chunks of 64)
+  const bool tensor_batch = !q8 && h->dtype == SFFN_BF16 && B >= 2 && h->path != SFFN_PATH_GENERAL &&
+                            sffn::batched_mma_supported(h->D, gate_k, lopa_gate ? 2 * chunk : chunk);
+  // Any other batch: the single-token kernel once per token, where it serves the shape.  The tensor-core batch kernels
+  // take bf16 operands only, and the CUDA-core batch kernels are slower than B single-token calls (int8, 4096 x 14336,
+  // B = 16: 1.66 ms against 0.33 ms; bf16 rows of 4000 elements: 1.03 ms against 0.46 ms; fp32: 0.86 against 0.77 ms).
+  // The fired flags of the tokens are OR-ed: the list is the batch's union.
+  if (B > 1 && !tensor_batch && h->path != SFFN_PATH_GENERAL && h->path != SFFN_PATH_MMA_SYNC &&
       sffn::fused_supported(wkind, h->D, h->H, 1, g, h->sm_count)) {
+    const size_t tok_bytes = (size_t)h->D * ((q8 || h->dtype == SFFN_BF16) ? 2 : 4);
     for (int b = 0; b < B; ++b) {
       sffn::FusedCall c{};
       c.wkind = wkind;
-      c.s_gate = q8->s_gate; c.s_V = q8->s_V; c.s_up = q8->s_up; c.s_down = q8->s_down;
+      if (q8) { c.s_gate = q8->s_gate; c.s_V = q8->s_V; c.s_up = q8->s_up; c.s_down = q8->s_down; }
       c.D = h->D; c.H = h->H;
-      c.x = static_cast<const char*>(x) + (size_t)b * h->D * 2;  // bf16 tokens
+      c.x = static_cast<const char*>(x) + (size_t)b * tok_bytes;
       c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up;
       c.engine = h->gate_engine; c.y = y + (size_t)b * h->D;
       c.dense = dense; c.flag_or = b > 0;
@@ -561,17 +570,30 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
     if (!dense) h->list_state = 2;
     return SFFN_OK;
   }
-  const int gate_k = g->kind == SFFN_GATE_LOPA ? g->r : h->D;
-  const int gate_cols = g->kind == SFFN_GATE_LOPA ? 2 * B : B;
-  if (!q8 && h->dtype == SFFN_BF16 && B >= 2 && B <= kMaxMmaTokens && h->path != SFFN_PATH_GENERAL) {
-    const bool mma_ok = sffn::batched_mma_supported(h->D, gate_k, gate_cols);
-    const bool umma_ok = mma_ok && sffn::umma_rows_supported(gate_k, gate_cols) && sffn::umma_rows_supported(h->D, B);
-    if (h->path == SFFN_PATH_MMA_SYNC && !mma_ok) return SFFN_ERR_UNSUPPORTED;
-    if (mma_ok)
-      return run_batched(h, x, B, g, b_g, W_up, W_down, act, y, dense, umma_ok && h->path != SFFN_PATH_MMA_SYNC, s);
-  } else if (h->path == SFFN_PATH_MMA_SYNC) {
-    return SFFN_ERR_UNSUPPORTED;
+  if (tensor_batch) {
+    // chunks of at most 64 tokens; with more than one chunk the fired sets are accumulated into the batch's union
+    uint8_t* uni = h->at<uint8_t>(h->L.union_flag);
+    const bool parts = B > kMaxMmaTokens;
+    if (parts && !dense) SFFN_CUDA(cudaMemsetAsync(uni, 0, h->H, s));
+    for (int b0 = 0; b0 < B; b0 += kMaxMmaTokens) {
+      const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
+      const int cols = lopa_gate ? 2 * nb : nb;
+      const bool umma_ok = sffn::umma_rows_supported(gate_k, cols) && sffn::umma_rows_supported(h->D, nb);
+      const int rc2 = run_batched(h, static_cast<const char*>(x) + (size_t)b0 * h->D * 2, nb, g, b_g, W_up, W_down, act,
+                                  y + (size_t)b0 * h->D, dense, umma_ok && h->path != SFFN_PATH_MMA_SYNC, s);
+      if (rc2 != SFFN_OK) return rc2;
+      if (parts && !dense) {
+        SFFN_CUDA(sffn::launch_mark_union(h->at<int32_t>(h->L.idx), h->at<int32_t>(h->L.status) + 1, h->H, uni, s));
+        ++h->launches;
+      }
+    }
+    if (parts && !dense) {
+      SFFN_CUDA(cudaMemcpyAsync(h->at<uint8_t>(h->L.flag), uni, h->H, cudaMemcpyDeviceToDevice, s));
+      h->list_state = 2;  // the list is compacted from the union's flags on request
+    }
+    return SFFN_OK;
   }
+  if (h->path == SFFN_PATH_MMA_SYNC) return SFFN_ERR_UNSUPPORTED;
   return run_general(h, x, B, g, b_g, W_up, W_down, act, y, dense, q8, qbits, s);
 }
 

@@ -457,6 +457,21 @@ cudaError_t launch_rmsnorm(const float* v, float* n, const float* gain, int r, i
   return launch_pdl(rmsnorm_kernel, dim3(B), dim3(256), 0, s, v, n, gain, r, stride, eps);
 }
 
+// union[idx[i]] = 1 for the listed neurons: accumulates the fired sets of the chunks of a batch that is run in parts.
+__global__ void __launch_bounds__(256) mark_union_kernel(const int32_t* idx, const int32_t* count, int H, uint8_t* u) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int n = *count;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int j = idx[i];
+    if (j >= 0 && j < H) u[j] = 1;
+  }
+}
+
+cudaError_t launch_mark_union(const int32_t* idx, const int32_t* count, int H, uint8_t* u, cudaStream_t s) {
+  return launch_pdl(mark_union_kernel, dim3(32), dim3(256), 0, s, idx, count, H, u);
+}
+
 cudaError_t launch_compact(const uint8_t* flag, int H, int32_t* idx, int32_t* count, cudaStream_t s) {
   return launch_pdl(compact_kernel, dim3(1), dim3(1024), 0, s, flag, H, idx, count);
 }

@@ -48,6 +48,7 @@ cudaError_t launch_rowdot(int wkind, bool vec_is_f32, int nb, bool gate, const R
 cudaError_t launch_rmsnorm(const float* v, float* n, const float* gain, int r, int stride, float eps,
                            int B, cudaStream_t s);
 cudaError_t launch_compact(const uint8_t* flag, int H, int32_t* idx, int32_t* count, cudaStream_t s);
+cudaError_t launch_mark_union(const int32_t* idx, const int32_t* count, int H, uint8_t* union_flags, cudaStream_t s);
 // Largest token chunk (4, 2 or 0 = unsupported D) the up/down kernel takes at this D.
 int updown_max_tokens(int wkind, int D);
 cudaError_t launch_updown(int wkind, int nb, const UpDownParams& p, int grid, cudaStream_t s);

@@ -179,6 +179,54 @@ def test_batched_lopa(mod, B, r, rms, path):
     assert_active_set(ffn.last_active(), ref, what=f"batched lopa [{path}]")
 
 
+@pytest.mark.parametrize("kind", ["standard", "lopa"])
+@pytest.mark.parametrize("B", [65, 96, 130])
+def test_batches_of_more_than_64_tokens_run_in_chunks_with_the_union_of_all(mod, kind, B):
+    D, H, r = 512, 1200, 128
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=r, B_max=130)
+    if kind == "standard":
+        gate, w = make_std(D, H, torch.bfloat16, 45, 0.9)
+    else:
+        gate, w = make_lopa(mod, D, H, r, torch.bfloat16, 45, 0.9, "diag", True, True, True)
+    p = syn.zipf_firing_profile(H, 1.1, 0.02, 0.9, seed=5)       # a union that keeps growing with the tokens
+    w["b_g"] = syn.bias_from_firing_profile(p).to(DEV)
+    x = syn.tokens(B, D, torch.bfloat16, 45, DEV)
+    ref = run_both_paths(mod, ffn, x, gate, w, "relu", ("auto", "mma_sync"), what=f"{kind} B={B}")
+    last = run_oracle(x[64 * ((B - 1) // 64):], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert last["union_mask"].sum() < ref["union_mask"].sum()    # the list is not just the last chunk's
+    yd = ffn.dense_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    dref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", route="dense")
+    assert_y_close(yd, dref["y"], what=f"dense {kind} B={B}")
+    y1 = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    y2 = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert torch.equal(y1, y2)
+
+
+@pytest.mark.parametrize("dtype,D", [(torch.float32, 512), (torch.bfloat16, 520), (torch.float32, 776)])
+@pytest.mark.parametrize("kind", ["standard", "lopa"])
+@pytest.mark.parametrize("B", [2, 5, 70])
+def test_batches_without_a_tensor_core_path_run_token_by_token(mod, dtype, D, kind, B):
+    # fp32 operands, or bf16 rows of a width the tensor-core batch kernels do not take
+    H, r = 1100, 64
+    ffn = mod.SparseFFN(D, H, dtype, r_max=r, B_max=70)
+    if kind == "standard":
+        gate, w = make_std(D, H, dtype, 46, 0.9)
+    else:
+        gate, w = make_lopa(mod, D, H, r, dtype, 46, 0.9, "diag", True, True, True)
+    x = syn.tokens(B, D, dtype, 46, DEV)
+    tol = 1e-5 if dtype == torch.float32 else None
+    ref = run_both_paths(mod, ffn, x, gate, w, "relu", ("auto", "general"), tol=tol, what=f"{kind} {dtype} B={B}")
+    launches0 = ffn.launch_count()
+    y = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert ffn.launch_count() - launches0 == B                   # one launch per token: the single-token kernel
+    for b in (0, B - 1):                                         # and bit for bit what the token gives alone
+        y1 = ffn.sparse_ffn_forward(x[b], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+        assert torch.equal(y1, y[b])
+    yd = ffn.dense_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    dref = run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", route="dense")
+    assert_y_close(yd, dref["y"], what=f"dense {kind} {dtype} B={B}", **({} if tol is None else dict(rel_l2=tol, max_abs=tol)))
+
+
 # ------------------------------------------------------------------ degenerate cases
 @pytest.mark.parametrize("path", ["general", "fused"])
 def test_full_and_zero_sparsity(mod, gate_engine, path):
