@@ -307,8 +307,11 @@ def run(out_path, quick=False, only=None, n_calls=None):
             lsets.append(lw)
         lg = lambda w: {"V": w["V"], "U": w["U"], "g_idx": gi, "use_rmsnorm": True, "rms_eps": 1e-5}
         add("lopa r=512 relu int8", D, H, 1, lsets, lg, "relu", r=512, peak=peak)
-        if not quick:
-            add("batched B=16 int8 (token by token)", D, H, 16, qsets, std, "relu", n_calls=40, peak=peak)
+        if not quick:  # batches on the tcgen05 kernels, which expand the codes to bf16 on the way to the tensor cores
+            zq = [dict(w, b_g=zb) for w in qsets]
+            for B in (4, 16, 64):
+                add(f"batched zipf B={B} int8", D, H, B, zq, std, "relu", n_calls=100, peak=peak)
+            del zq
         del qsets, lsets
         torch.cuda.empty_cache()
     # weight-only int4 (packed 4-bit codes + one fp32 scale per row)
@@ -318,6 +321,11 @@ def run(out_path, quick=False, only=None, n_calls=None):
             b = syn.gate_bias_for_sparsity(s)
             sets = [dict(w, b_g=torch.full((H,), b, device=DEV)) for w in qsets]
             add(f"decode 4096x14336 s={s} int4", D, H, 1, sets, std, "relu", peak=peak)
+        if not quick:
+            zq = [dict(w, b_g=zb) for w in qsets]
+            for B in (4, 16, 64):
+                add(f"batched zipf B={B} int4", D, H, B, zq, std, "relu", n_calls=100, peak=peak)
+            del zq
         del qsets
         torch.cuda.empty_cache()
     if not quick and (only is None or "stress" in only):

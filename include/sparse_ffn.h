@@ -80,12 +80,13 @@ typedef enum { SFFN_F32 = 0, SFFN_BF16 = 1 } sffn_dtype;
 typedef enum { SFFN_GATE_STANDARD = 0, SFFN_GATE_LOPA = 1 } sffn_gate_kind;
 
 /* Which kernels serve a call.  AUTO picks the fused kernels for B = 1 when the shape allows it and the
- * tcgen05 tensor-core kernels for bf16 batches (B >= 2; more than 64 tokens run in chunks of 64, the list
- * of fired neurons being the union over all chunks).  A batch those kernels do not take (fp32 or quantised
- * weights, a row width they do not tile) runs the fused kernel once per token with the fired flags OR-ed,
+ * tcgen05 tensor-core kernels for batches (B >= 2) of bf16 tokens with bf16, int8 or int4 rows (codes are
+ * expanded to bf16 in shared memory on their way to the tensor cores; more than 64 tokens run in chunks of 64,
+ * the list of fired neurons being the union over all chunks).  A batch those kernels do not take (fp32
+ * operands, a row width they do not tile) runs the fused kernel once per token with the fired flags OR-ed,
  * which is faster than the CUDA-core batch kernels; what is left goes to the general CUDA-core kernels.
  * The others force one family (SFFN_ERR_UNSUPPORTED if it cannot serve the call): GENERAL = CUDA-core
- * kernels for any batch, FUSED = single-token fused kernels, MMA_SYNC = batched kernels on the
+ * kernels for any batch, FUSED = single-token fused kernels (a batch: once per token), MMA_SYNC = batched kernels on the
  * warp-level mma.sync tensor-core path. */
 typedef enum { SFFN_PATH_AUTO = 0, SFFN_PATH_GENERAL = 1, SFFN_PATH_FUSED = 2, SFFN_PATH_MMA_SYNC = 3 } sffn_path;
 
@@ -166,9 +167,11 @@ int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate
  * int8 codes ([H,D], [H,D], [H,D], [r,D], [H,r]); `scales` carries the row scales.  Tokens x are bf16: the handle
  * must have been created with SFFN_BF16.  Rows must be a multiple of 16 bytes (D and r multiples of 16).
  * Everything else (b_g, g_idx, g_sign, RMSNorm, act, y, the active list, double activation) is as in
- * sparse_ffn_forward / dense_ffn_forward.  One token runs in the fused kernel; a batch runs that kernel once per
- * token (the list of fired neurons is the union over the tokens), or the CUDA-core batch kernels under
- * SFFN_PATH_GENERAL (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is an offline
+ * sparse_ffn_forward / dense_ffn_forward.  One token runs in the fused kernel; a batch runs the tcgen05 batch
+ * kernels, which expand the codes to bf16 in shared memory and apply the row scales to the accumulator rows (D and
+ * r multiples of 64, D of 256; otherwise, or under SFFN_PATH_FUSED, the fused kernel once per token; the list of
+ * fired neurons is the union over the tokens), or the CUDA-core batch kernels under SFFN_PATH_GENERAL
+ * (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is an offline
  * step outside this library. */
 typedef struct {
   const float* s_gate; /* [H]  row scales of W_g (STANDARD) or of U (LOPA) */
@@ -189,8 +192,8 @@ int dense_ffn_forward_q8(sffn_handle* handle, const void* x, int B, const sffn_g
  *     W[j, 2b] = s[j] * low_nibble(p[j, b]),   W[j, 2b + 1] = s[j] * high_nibble(p[j, b]).
  * The weight pointers address the packed bytes ([H, D/2], [r, D/2], [H, r/2]); `scales` as for int8.  Rows must be a
  * multiple of 16 bytes (D and r multiples of 32).  Otherwise exactly like the _q8 calls: bf16 tokens, fp32 arithmetic,
- * one token in the fused kernel (rows of up to 8192 codes there), a batch once per token, wider rows in the CUDA-core
- * kernels. */
+ * one token in the fused kernel (rows of up to 8192 codes there), a batch on the tcgen05 batch kernels, wider rows in
+ * the CUDA-core kernels. */
 int sparse_ffn_forward_q4(sffn_handle* handle, const void* x, int B, const sffn_gate* gate, const float* b_g,
                           const void* W_up, const void* W_down, const sffn_q8_scales* scales, int act, float* y,
                           void* stream);

@@ -250,9 +250,11 @@ thread_local int g_last_cuda_line = 0;
 // Tokens are taken kMaxMmaTokens at a time; the union (and the list) is that of the whole batch.
 int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b_g,
                 const void* W_up, const void* W_down, int act, float* y, bool dense, bool umma,
-                cudaStream_t s) {
+                const sffn_q8_scales* q8, int qbits, cudaStream_t s) {
   using namespace sffn;
   const int D = h->D, H = h->H;
+  if (q8 && !umma) return SFFN_ERR_UNSUPPORTED;  // rows of weight codes: tcgen05 kernels only
+  const int wq = q8 ? qbits : 0;
   float* actbuf = h->at<float>(h->L.act);
   uint8_t* flag = h->at<uint8_t>(h->L.flag);
   int32_t* idx = h->at<int32_t>(h->L.idx);
@@ -269,6 +271,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
       UmmaRowsParams p{};
       p.W = g->V; p.R = g->r; p.K = D;
+      p.qbits = wq; p.w_scale = q8 ? q8->s_V : nullptr;
       p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
       p.act = kUmmaActIdentity; p.a_out = vbuf + (size_t)b0 * rs; p.a_stride = rs;
       p.status = h->at<int32_t>(h->L.status);
@@ -306,6 +309,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     if (umma) {
       UmmaRowsParams p{};
       p.R = H; p.B = nb; p.b_g = b_g; p.act = act; p.status = h->at<int32_t>(h->L.status);
+      p.qbits = wq; p.w_scale = q8 ? q8->s_gate : nullptr;
       p.xtok = xtok; p.xtok_stride = D;
       p.a_out = actbuf + (size_t)b0 * H; p.a_stride = H;
       p.flag = (dense || own_list) ? nullptr : flag;
@@ -364,6 +368,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     if (umma) {
       UmmaRowsParams p{};
       p.W = W_up; p.R = H; p.K = D;
+      p.qbits = wq; p.w_scale = q8 ? q8->s_up : nullptr; p.out_scale = q8 ? q8->s_down : nullptr;
       if (own_list) {
         p.words_in = words; p.n_words = 4 * gate_tiles; p.gate_tile_rows = gate_tile_rows;
         p.gate_rows_per_word = gate_tile_rows <= 64 ? 16 : 32;
@@ -387,9 +392,10 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       SFFN_CUDA(launch_rows_mma(true, p, nb, grid_rows, s));
     }
     int nsplit = splits;
+    if (q8 && !umma_down_supported(D, nb)) return SFFN_ERR_UNSUPPORTED;
     if (umma && umma_down_supported(D, nb)) {
       UmmaDownParams d{};
-      d.W_down = W_down; d.R = H; d.D = D;
+      d.W_down = W_down; d.R = H; d.D = D; d.qbits = wq;
       d.idx = lidx; d.count = lcount;
       d.hmT = hmT; d.hm_stride = h->L.hm_stride; d.B = nb;
       d.splits = nsplit = umma_down_splits(D, h->sm_count, kMaxSplits);
@@ -520,8 +526,13 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
   const int gate_k = lopa_gate ? g->r : h->D;
   const int chunk = B < kMaxMmaTokens ? B : kMaxMmaTokens;
   // a batch the tensor-core kernels can take (bf16 rows; more than 64 tokens: in chunks of 64)
-  const bool tensor_batch = !q8 && h->dtype == SFFN_BF16 && B >= 2 && h->path != SFFN_PATH_GENERAL &&
-                            sffn::batched_mma_supported(h->D, gate_k, lopa_gate ? 2 * chunk : chunk);
+  const int gate_cols_chunk = lopa_gate ? 2 * chunk : chunk;
+  // rows of weight codes: the tcgen05 kernels only (they expand the codes to bf16 on the way to the tensor cores)
+  const bool q_tensor_ok = !q8 || (h->path != SFFN_PATH_MMA_SYNC && sffn::umma_rows_supported(gate_k, gate_cols_chunk) &&
+                                   sffn::umma_rows_supported(h->D, chunk) && sffn::umma_down_supported(h->D, chunk) &&
+                                   (!lopa_gate || sffn::umma_rows_supported(h->D, chunk)));
+  const bool tensor_batch = h->dtype == SFFN_BF16 && B >= 2 && h->path != SFFN_PATH_GENERAL && q_tensor_ok &&
+                            h->path != SFFN_PATH_FUSED && sffn::batched_mma_supported(h->D, gate_k, gate_cols_chunk);
   // Any other batch: the single-token kernel once per token, where it serves the shape.  The tensor-core batch kernels
   // take bf16 operands only, and the CUDA-core batch kernels are slower than B single-token calls (int8, 4096 x 14336,
   // B = 16: 1.66 ms against 0.33 ms; bf16 rows of 4000 elements: 1.03 ms against 0.46 ms; fp32: 0.86 against 0.77 ms).
@@ -580,7 +591,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
       const int cols = lopa_gate ? 2 * nb : nb;
       const bool umma_ok = sffn::umma_rows_supported(gate_k, cols) && sffn::umma_rows_supported(h->D, nb);
       const int rc2 = run_batched(h, static_cast<const char*>(x) + (size_t)b0 * h->D * 2, nb, g, b_g, W_up, W_down, act,
-                                  y + (size_t)b0 * h->D, dense, umma_ok && h->path != SFFN_PATH_MMA_SYNC, s);
+                                  y + (size_t)b0 * h->D, dense, umma_ok && h->path != SFFN_PATH_MMA_SYNC, q8, qbits, s);
       if (rc2 != SFFN_OK) return rc2;
       if (parts && !dense) {
         SFFN_CUDA(sffn::launch_mark_union(h->at<int32_t>(h->L.idx), h->at<int32_t>(h->L.status) + 1, h->H, uni, s));

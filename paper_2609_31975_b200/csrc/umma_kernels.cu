@@ -24,6 +24,14 @@
 // stages (up to 12) is cut out of the dynamic shared memory on the device, once the tile height is known.
 // Every kernel here is launched with programmatic dependent launch: set-up first, griddepcontrol.wait before the
 // first dependent read or global write.
+// Weight-only int8 / int4 rows (QB = 8 / 4): the copies bring the codes (and the token rows) into the ring slots;
+// four more warps (the last four of the CTA, two pairs that alternate over the stages) expand the codes to bf16 --
+// every code is an integer bf16 holds exactly -- in the swizzled layout, into a short ring of expanded blocks of
+// its own (rows kernels) or the slot's block area (down kernel), and arrive on a "ready" barrier that the MMA
+// issuers wait for instead of "full"; the row scales are applied to the accumulator rows in the epilogue (the
+// down projection's are folded into Hm).  With the weights as the A operand the tensor core takes 32 bytes of
+// bf16 per cycle and SM whatever the token count, i.e. 16 codes per cycle: quantised batches are bound by that
+// rate, not by their bytes.
 // Every wait is bounded by a cycle budget; on expiry the status word is set, all roles wind down and the TMEM
 // columns are released before the CTA exits.
 #include "umma_kernels.cuh"
@@ -46,10 +54,13 @@ constexpr int kAAtomBytes = kTileRows * 128;         // 16 KB: one [128 rows x 6
 constexpr int kThreads = 320;                        // 4 producer warps, 4 epilogue warps, 2 MMA warps
 constexpr int kThreadsRows = 384;                    // rows kernels: up to 4 MMA warps
 constexpr int kProducerWarps = 4;
-constexpr int kMaxStages = 12;
+constexpr int kMaxStages = 16;                       // barrier slots; bf16 rows use up to 12
+constexpr int kMaxStagesBf16 = 12;
+constexpr int kExpandSlots = 4;                      // quantised rows: ring of expanded bf16 blocks
 constexpr int kWalkMinTokens = 32;                   // batches from which the up kernel may walk every row
 constexpr int kWalkAllPercent = 70;                  // union share of the rows from which "every row" is walked
 constexpr int kMaxIssuers = 4;
+constexpr int kExpandWarps = 4;                      // quantised rows: warps that expand the codes to bf16
 constexpr int kScanChunks = 4;                       // in-kernel compaction: up to 4 * 384 mask words = 384 gate tiles
 constexpr int kMaxOwnTiles = 8;                      // tiles of one CTA whose rows are kept in shared memory
 constexpr int kHeaderBytes = 1024 + kMaxOwnTiles * kTileRows * 4;  // barriers + scratch, then the row lists
@@ -180,6 +191,76 @@ __device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Expands a block of weight codes to bf16: `raw` holds [rows][64] codes (QB = 8: a byte each, +-127; QB = 4: two's-
+// complement nibbles, even column in the low nibble), `dst` (1024-byte aligned) receives [rows][64] bf16 in the
+// 128-byte-swizzled K-major layout (16-byte chunk c of row i at i * 128 + ((c ^ (i & 7)) * 16)).  Thread t of nthr
+// takes the 16-code quarter t % 4 of rows t / 4, t / 4 + nthr / 4, ... (four of them in flight): a quarter warp reads two whole raw rows
+// and writes chunks of two rows that share no bank.  A code c becomes the fp32 2^23 + (c + bias) by a byte
+// permute, the bias and 2^23 are subtracted exactly, and the upper half of that fp32 is the bf16.
+template <int QB>
+__device__ __forceinline__ void expand_block(uint32_t raw, uint32_t dst, int rows, int t, int nthr) {
+  constexpr int kRawRow = 8 * QB;  // bytes of 64 codes
+  constexpr int kUnroll = 4;       // rows of one thread in flight
+  const int c = t & 3, step = nthr >> 2;
+  for (int row0 = t >> 2; row0 < rows; row0 += kUnroll * step) {
+    uint32_t w[kUnroll][4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int row = row0 + u * step;
+      const uint32_t src = raw + row * kRawRow + c * (kRawRow / 4);
+      w[u][0] = w[u][1] = w[u][2] = w[u][3] = 0;
+      if (row < rows) {
+        if (QB == 8) {
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(w[u][0]), "=r"(w[u][1]), "=r"(w[u][2]), "=r"(w[u][3])
+                       : "r"(src));
+        } else {
+          asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(w[u][0]), "=r"(w[u][1]) : "r"(src));
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int row = row0 + u * step;
+      if (row >= rows) break;
+      if (QB == 4) {
+        const uint32_t a = w[u][0] ^ 0x88888888u, b = w[u][1] ^ 0x88888888u;
+        // bytes of w[2i]: even columns of word i, of w[2i+1]: odd columns
+        w[u][0] = a & 0x0f0f0f0fu; w[u][1] = (a >> 4) & 0x0f0f0f0fu;
+        w[u][2] = b & 0x0f0f0f0fu; w[u][3] = (b >> 4) & 0x0f0f0f0fu;
+      }
+      uint32_t o[8];
+      const float off = QB == 8 ? 8388736.f : 8388616.f;  // 2^23 + 128, 2^23 + 8
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        // o[i] = codes 2i, 2i+1 of the quarter
+        uint32_t lo, hi;
+        if (QB == 8) {
+          const uint32_t v = w[u][i >> 1] ^ 0x80808080u;
+          lo = __byte_perm(v, 0x4b000000u, (i & 1) ? 0x7442 : 0x7440);
+          hi = __byte_perm(v, 0x4b000000u, (i & 1) ? 0x7443 : 0x7441);
+        } else {
+          const uint32_t sel = 0x7440 + (i & 3);
+          lo = __byte_perm(w[u][(i >> 2) * 2], 0x4b000000u, sel);
+          hi = __byte_perm(w[u][(i >> 2) * 2 + 1], 0x4b000000u, sel);
+        }
+        const float fl = __uint_as_float(lo) - off, fh = __uint_as_float(hi) - off;
+        o[i] = __byte_perm(__float_as_uint(fl), __float_as_uint(fh), 0x7632);
+      }
+      const uint32_t drow = dst + row * 128;
+      const int sw = row & 7;
+      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(drow + (((2 * c) ^ sw) << 4)), "r"(o[0]), "r"(o[1]),
+                   "r"(o[2]), "r"(o[3])
+                   : "memory");
+      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(drow + (((2 * c + 1) ^ sw) << 4)), "r"(o[4]), "r"(o[5]),
+                   "r"(o[6]), "r"(o[7])
+                   : "memory");
+    }
+  }
+}
+// Makes this thread's shared-memory stores visible to the tensor core's reads.
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // Rows per tile: 128 when there is more than one tile per CTA, otherwise the row count spread over
 // the whole grid (a multiple of 8, the swizzle period), so that every SM streams a share.
 __host__ __device__ inline int tile_rows_for(int n_rows, int grid) {
@@ -206,8 +287,8 @@ struct WalkMap<false> {
 
 enum RowsMode { kGate = 0, kUp = 1, kUpMayWalk = 2 };  // kUpMayWalk: wide batches, see walk_all below
 
-template <int MODE>
-__global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRowsParams p,
+template <int MODE, int QB>
+__global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1) umma_rows_kernel(const UmmaRowsParams p,
                                                                   const __grid_constant__ CUtensorMap map_w,
                                                                   const __grid_constant__ CUtensorMap map_x,
                                                                   const __grid_constant__ WalkMap<MODE == kUpMayWalk> map_t) {
@@ -226,6 +307,9 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   const uint32_t acc_full = smem_u32(bars + 2 * kMaxStages), acc_empty = smem_u32(bars + 2 * kMaxStages + 1);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t ready = smem_u32(bars + 2 * kMaxStages + 4);  // quantised rows: slot t of the bf16 ring is written ...
+  const uint32_t afree = ready + 8 * kExpandSlots;             // ... and has been read by its MMAs
+  constexpr int kRawRow = 8 * QB;                              // bytes of 64 codes
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int kblocks = p.K / kAtomK;
@@ -238,6 +322,11 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       mbar_init(full + 8 * s, 1);  // the producer's expect_tx arrive; the copies complete the bytes
       mbar_init(empty + 8 * s, 1);
     }
+    if (QB)
+      for (int t = 0; t < kExpandSlots; ++t) {
+        mbar_init(ready + 8 * t, kExpandWarps / 2);
+        mbar_init(afree + 8 * t, 1);
+      }
     mbar_init(acc_empty, 128);
     *abort_flag = 0;
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
@@ -267,7 +356,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
 #pragma unroll
     for (int k = 0; k < kScanChunks; ++k) {
       const int w = k * kThreadsRows + tid;
-      bits[k] = (k < nch && w < p.n_words) ? __ldcg(p.words_in + w) : 0u;
+      bits[k] = (k < nch && tid < kThreadsRows && w < p.n_words) ? __ldcg(p.words_in + w) : 0u;
     }
 #pragma unroll
     for (int k = 0; k < kScanChunks; ++k) {
@@ -279,7 +368,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
           if (lane >= d) incl += t;
         }
         first_pos[k] = incl - __popc(bits[k]);
-        if (lane == 31) scan_wt[k * (kThreadsRows / 32) + warp] = incl;
+        if (lane == 31 && warp < kThreadsRows / 32) scan_wt[k * (kThreadsRows / 32) + warp] = incl;
       }
     }
     __syncthreads();
@@ -372,15 +461,23 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   const int atoms_cap = npad <= 16 ? 4 : npad <= 32 ? 2 : 1;  // at most 8 KB of token rows per stage
   atoms = atoms > atoms_cap ? atoms_cap : atoms;
   const int a_block_bytes = tile_rows * 128, b_block_bytes = npad * 128;
-  const int b_off = atoms * a_block_bytes;                    // token rows of a stage start here
-  int stage_bytes = atoms * (a_block_bytes + b_block_bytes);
-  stage_bytes = max(stage_bytes, (atoms - 1) * a_block_bytes + mrows * 128);
+  // bytes of the bf16 weight blocks of a stage, including what the last block's MMA reads past its rows
+  const int a_bytes = (max(atoms * a_block_bytes, (atoms - 1) * a_block_bytes + mrows * 128) + 1023) & ~1023;
+  const int raw_block_bytes = tile_rows * kRawRow;
+  // bf16 rows: a slot holds the weight blocks, then the token rows.  Quantised rows: the ring slots hold what the
+  // copies bring (token rows, then the codes), and the expanded bf16 blocks have a short ring of their own (stage
+  // `it` uses slot it mod 4 of it): the codes in flight, not the expanded blocks, are what has to cover the memory
+  // latency.
+  const int b_off = QB ? 0 : atoms * a_block_bytes;           // token rows within a ring slot
+  const int w_off = QB ? atoms * b_block_bytes : 0;           // weights (as copied) within a ring slot
+  int stage_bytes = QB ? atoms * (b_block_bytes + raw_block_bytes) : max(atoms * (a_block_bytes + b_block_bytes), a_bytes);
   stage_bytes = (stage_bytes + 1023) & ~1023;
-  int S = p.ring_bytes / stage_bytes;
-  S = S > kMaxStages ? kMaxStages : S;
+  const uint32_t ring0 = stage0 + (QB ? kExpandSlots * a_bytes : 0);
+  int S = (p.ring_bytes - (QB ? kExpandSlots * a_bytes : 0)) / stage_bytes;
+  S = S > (QB ? kMaxStages : kMaxStagesBf16) ? (QB ? kMaxStages : kMaxStagesBf16) : S;
   // four issuers when the ring divides evenly among them, otherwise two (slot mod issuers = owner)
-  const int issuers = (S >= 8 && S % 4 == 0) ? 4 : 2;
-  S &= ~1;
+  const int issuers = (S >= 8 && S % 4 == 0) ? 4 : QB && S >= 4 ? 4 : 2;
+  S &= (QB && S >= 4) ? ~3 : ~1;
   const int kstages = (kblocks + atoms - 1) / atoms;
   // accumulator row that this thread's TMEM lane holds (-1: none); the same for every warp of a lane quarter
   const int row_thr = m64 ? (lane < 16 ? (warp & 3) * 16 + lane : -1) : (warp & 3) * 32 + lane;
@@ -402,7 +499,10 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   // stores the gate values, reporting whether any token fired; (union rows) scales by the gate values
   // and stores HmT.  Returns false if the wait was abandoned.
   const bool share_last = npad >= 32;  // four or more column groups: worth spreading over all warps
-  auto epilogue = [&](int tile, int tcount, int part, int nparts, bool& fired) -> bool {
+  // `shared`: all twelve warps take part.  Only the epilogue warps have followed the accumulator barrier through
+  // every earlier tile (a warp that joins for the last tile could find it still in an earlier phase, which a parity
+  // wait cannot tell from "complete"), so they wait for it and the others meet them at a named barrier.
+  auto epilogue = [&](int tile, int tcount, int part, int nparts, bool shared, bool& fired) -> bool {
     const int row_in_tile = row_thr;
     const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     const int B = p.B;
@@ -413,6 +513,8 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     // everything that does not depend on the accumulator is fetched before the wait
     if (MODE == kGate) pdl_wait();  // before the first read of a buffer an earlier kernel may write, and the first store
     float bias = 0.f, sg = 1.f;
+    const float sc = (QB && row_ok && p.w_scale) ? p.w_scale[j] : 1.f;           // scale of the weight row
+    const float osc = (QB && UP && row_ok && p.out_scale) ? p.out_scale[j] : 1.f;  // scale of the down row, folded into Hm
     int gi = -1;
     float pre[16];  // union rows: the gate values of this thread's first two column groups
     if (UP) {
@@ -429,8 +531,15 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
       sg = (row_ok && p.g_sign && p.g_sign[j] < 0) ? -1.f : 1.f;
     }
     int okw = 1;
-    if (lane == 0) okw = mbar_wait(acc_full, tcount & 1, abort_flag, p.status, p.wait_cycles) ? 1 : 0;
-    okw = __shfl_sync(0xffffffffu, okw, 0);
+    if (!shared || (warp >= 4 && warp < 8)) {
+      if (lane == 0) okw = mbar_wait(acc_full, tcount & 1, abort_flag, p.status, p.wait_cycles) ? 1 : 0;
+      okw = __shfl_sync(0xffffffffu, okw, 0);
+    }
+    if (shared) {
+      tc_fence_before();
+      named_bar_sync(3, kThreadsRows);  // reached by all twelve warps whatever happened before
+      if (*abort_flag) okw = 0;
+    }
     if (!okw) return false;
     tc_fence_after();
     if (UP) {
@@ -448,7 +557,8 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
 #pragma unroll
         for (int q = 0; q < 8; ++q)
           if (row_ok && c0 + q < B)
-            hm[(size_t)(c0 + q) * p.hm_stride] = __float2bfloat16(av[q] * activation(act_up, v[q]));
+            hm[(size_t)(c0 + q) * p.hm_stride] =
+                __float2bfloat16(QB ? av[q] * activation(act_up, v[q] * sc) * osc : av[q] * activation(act_up, v[q]));
       }
     } else {
       const int act = p.act;
@@ -462,7 +572,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
           for (int q = 0; q < 4; ++q) {
             const int b = c0 / 2 + q;
             if (row_ok && b < B) {
-              float z = v[2 * q] + v[2 * q + 1] + bias;
+              float z = QB ? (v[2 * q] + v[2 * q + 1]) * sc + bias : v[2 * q] + v[2 * q + 1] + bias;
               if (gi >= 0) z += sg * __bfloat162float(xg[(size_t)b * p.xtok_stride]);
               fired |= z > 0.f;
               arow[(size_t)b * p.a_stride] = activation(act, z);
@@ -477,7 +587,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
           for (int q = 0; q < 8; ++q) {
             const int b = c0 + q;
             if (row_ok && b < B) {
-              float z = v[q] + bias;
+              float z = QB ? v[q] * sc + bias : v[q] + bias;
               if (gi >= 0) z += sg * __bfloat162float(xg[(size_t)b * p.xtok_stride]);
               fired |= z > 0.f;
               arow[(size_t)b * p.a_stride] = activation(act, z);
@@ -511,7 +621,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
         if ((s & (kProducerWarps - 1)) != warp) continue;
         const int tile = blockIdx.x + tl * gridDim.x;
         const int na = min(atoms, kblocks - kb * atoms);
-        const uint32_t tx_bytes = (uint32_t)(na * (tile_rows + npad)) * 128;
+        const uint32_t tx_bytes = QB ? (uint32_t)(na * (tile_rows * kRawRow + npad * 128)) : (uint32_t)(na * (tile_rows + npad)) * 128;
         if (UP && !walk_all && tl != rows_of) {
           rows_of = tl;
 #pragma unroll
@@ -532,17 +642,21 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) return false;
         }
-        const uint32_t abase = stage0 + s * stage_bytes;
+        const uint32_t abase = ring0 + s * stage_bytes;
         for (int a = 0; a < na; ++a) {
           const int k0 = (kb * atoms + a) * kAtomK;
+          // where the weight block lands, the byte column it starts at, and the bytes of one landed row
+          const uint32_t wdst = abase + w_off + a * (QB ? raw_block_bytes : a_block_bytes);
+          const int wc0 = QB ? k0 * QB / 8 : k0;
+          const int wrow = QB ? kRawRow : 128;
           if (with_w && !(MODE == kGate && blockIdx.x == 0 && it == p.drop_stage)) {  // test hook: a copy that never comes
             if (UP && !walk_all) {
               if (lane * 4 < tile_rows)
-                tma_gather4(abase + a * a_block_bytes + lane * 512, &map_w, k0, r[0], r[1], r[2], r[3], full + 8 * s);
+                tma_gather4(wdst + lane * 4 * wrow, &map_w, wc0, r[0], r[1], r[2], r[3], full + 8 * s);
             } else if (UP) {
-              if (lane == 0) tma_tile_2d(abase + a * a_block_bytes, map_t.get(), k0, tile * tile_rows, full + 8 * s);
+              if (lane == 0) tma_tile_2d(wdst, map_t.get(), wc0, tile * tile_rows, full + 8 * s);
             } else if (lane == 0) {
-              tma_tile_2d(abase + a * a_block_bytes, &map_w, k0, tile * tile_rows, full + 8 * s);
+              tma_tile_2d(wdst, &map_w, wc0, tile * tile_rows, full + 8 * s);
             }
           }
           if (with_x && lane == 0) tma_tile_2d(abase + b_off + a * b_block_bytes, &map_x, k0, 0, full + 8 * s);
@@ -560,6 +674,32 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     } else {
       produce(0, total, true, true);
     }
+  } else if (QB && warp >= kThreadsRows / 32) {
+    // ======================= expanders (quantised rows): codes -> bf16 block of the slot ==========
+    // Two pairs of warps; a pair takes the slots of its parity (S is even), in the producers' order, so it meets
+    // every phase of its slots and cannot fall two phases behind; while one pair waits the other one converts.
+    const int my_tiles = (int)blockIdx.x < n_tiles ? (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int total = my_tiles * kstages;
+    const int pair = (tid - kThreadsRows) / (16 * kExpandWarps);
+    const int et = (tid - kThreadsRows) % (16 * kExpandWarps);
+    int s = 0, ph = 0, kb = 0;
+    for (int it = 0; it < total; ++it, ++s, ++kb) {
+      if (s == S) { s = 0; ph ^= 1; }
+      if (kb == kstages) kb = 0;
+      if ((s & 1) != pair) continue;
+      const int t = it % kExpandSlots;
+      // the codes have landed, and the MMAs of the stage that used the bf16 slot before are done
+      const bool ok = mbar_wait(full + 8 * s, ph, abort_flag, p.status, p.wait_cycles) &&
+                      mbar_wait(afree + 8 * t, ((it / kExpandSlots) & 1) ^ 1, abort_flag, p.status, p.wait_cycles);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const uint32_t src = ring0 + s * stage_bytes + w_off, dst = stage0 + t * a_bytes;
+      const int na = min(atoms, kblocks - kb * atoms);
+      for (int a = 0; a < na; ++a)
+        expand_block<QB ? QB : 8>(src + a * raw_block_bytes, dst + a * a_block_bytes, tile_rows, et, 16 * kExpandWarps);
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(ready + 8 * t);
+    }
   } else if (warp >= 8) {
     // ======================= MMA issuers =======================================================
     const int m = warp - 8;
@@ -576,18 +716,22 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
         for (int kb = 0; kb < kstages; ++kb, ++s) {
           if (s == S) { s = 0; ph ^= 1; }
           if ((s & (nacc - 1)) != m) continue;   // another issuer's slot
-          if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status, p.wait_cycles)) { ok = false; break; }
+          const int t = (it0 + kb) % kExpandSlots;  // quantised rows: slot of the bf16 ring
+          if (QB ? !mbar_wait(ready + 8 * t, ((it0 + kb) / kExpandSlots) & 1, abort_flag, p.status, p.wait_cycles)
+                 : !mbar_wait(full + 8 * s, ph, abort_flag, p.status, p.wait_cycles)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sbase = stage0 + s * stage_bytes;
+          const uint32_t sbase = ring0 + s * stage_bytes;
+          const uint32_t wbase = QB ? stage0 + t * a_bytes : sbase;
           const int na = min(atoms, kblocks - kb * atoms);
           for (int a = 0; a < na; ++a) {
-            const uint64_t adesc = make_desc(sbase + a * a_block_bytes);
+            const uint64_t adesc = make_desc(wbase + a * a_block_bytes);
             const uint64_t bdesc = make_desc(sbase + b_off + a * b_block_bytes);
             umma(acc, adesc, bdesc, idesc, (kb >= nacc || a > 0) ? 1u : 0u);
 #pragma unroll
             for (int k = 1; k < kAtomK / 16; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
           }
           umma_commit(empty + 8 * s);   // slot free once these MMAs have read it
+          if (QB) umma_commit(afree + 8 * t);
         }
         if (ok) umma_commit(acc_full);  // this issuer's accumulator is complete
       }
@@ -605,7 +749,7 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
     int tcount = 0;
     for (int tile = blockIdx.x; tile + (share_last ? (int)gridDim.x : 0) < n_tiles; tile += gridDim.x, ++tcount) {
       bool fired = false;
-      if (!epilogue(tile, tcount, 0, 1, fired)) break;
+      if (!epilogue(tile, tcount, 0, 1, false, fired)) break;
       const int row_in_tile = row_thr;
       const int li = tile * tile_rows + row_in_tile;
       const bool valid = row_in_tile >= 0 && row_in_tile < tile_rows && li < n_rows;
@@ -622,12 +766,12 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
   // ---- the CTA's last tile (wide batches): by now the producer and issuer warps have nothing left to do, so
   // all twelve warps share its epilogue.  A warp reads the TMEM lanes of its quarter (warp mod 4); the three warps of
   // a quarter take every third group of eight token columns.
-  if (share_last && (int)blockIdx.x < n_tiles) {
+  if (share_last && (int)blockIdx.x < n_tiles && warp < kThreadsRows / 32) {
     const int my_tiles = (n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
     const int last_tile = blockIdx.x + (my_tiles - 1) * gridDim.x;
     const int part = warp >= 8 ? 2 : warp >= 4 ? 0 : 1;
     bool fired = false;
-    const bool done = epilogue(last_tile, my_tiles - 1, part, 3, fired);
+    const bool done = epilogue(last_tile, my_tiles - 1, part, 3, true, fired);
     if (!UP && (p.flag || p.words_out)) {
       uint8_t* fired_sm = reinterpret_cast<uint8_t*>(scan_wt);  // [3][128], the scan scratch is free here
       const int row_in_tile = row_thr;
@@ -667,13 +811,16 @@ __global__ void __launch_bounds__(kThreadsRows, 1) umma_rows_kernel(const UmmaRo
 // gathered row delivers 64 contiguous d per swizzle row) and HmT[b][u] is the K-major B operand.
 // Same pipeline as above: 4 producer warps (gather4 per lane: 2 column halves x 16 row quads = one 64-row
 // stage), 2 MMA issuers with their own accumulators, 4 epilogue warps; two CTAs share an SM.
-__global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownParams p,
+template <int QB>
+__global__ void __launch_bounds__(kThreads + (QB ? 32 * kExpandWarps : 0), 2) umma_down_kernel(const UmmaDownParams p,
                                                                   const __grid_constant__ CUtensorMap map_wg,
                                                                   const __grid_constant__ CUtensorMap map_wt,
                                                                   const __grid_constant__ CUtensorMap map_hm) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int npad = p.npad;
-  const int stage_bytes = kAAtomBytes + npad * 128;
+  constexpr int kRawBytes = QB * kTileRows * kAtomK / 8;  // quantised rows: the codes of a stage's 64 rows x 128 columns
+  const int raw_off = kAAtomBytes + npad * 128;
+  const int stage_bytes = raw_off + kRawBytes;
   const int S = p.stages;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
@@ -682,6 +829,7 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
   const uint32_t acc_full = smem_u32(bars + 2 * S);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t ready = smem_u32(bars + 2 * S + 4);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int d_tiles = p.D / kTileRows;
@@ -694,6 +842,7 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
     for (int s = 0; s < S; ++s) {
       mbar_init(full + 8 * s, 1);
       mbar_init(empty + 8 * s, 1);
+      if (QB) mbar_init(ready + 8 * s, kExpandWarps / 2);
     }
     *abort_flag = 0;
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_wg) : "memory");
@@ -730,8 +879,10 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
 
   if (warp < kProducerWarps) {
     // ======================= producers (slot s belongs to warp s mod 4) =========================
-    const uint32_t tx_bytes = (uint32_t)(kAAtomBytes + npad * 128);
+    const uint32_t tx_bytes = (uint32_t)((QB ? kRawBytes : kAAtomBytes) + npad * 128);
     const int half = lane >> 4, quad = lane & 15;
+    constexpr int kHalfBytes = QB ? kRawBytes / 2 : kAAtomBytes / 2;  // landed bytes of 64 rows x 64 columns
+    constexpr int kColDiv = QB == 4 ? 2 : 1;                          // codes per byte
     int s = 0, ph = 0;
     for (int kb = 0; kb < kblocks; ++kb, ++s) {
       if (s == S) { s = 0; ph ^= 1; }
@@ -759,13 +910,33 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       const uint32_t abase = stage0 + s * stage_bytes;
+      const uint32_t wdst = QB ? abase + raw_off : abase;
       if (!walk_all) {
-        tma_gather4(abase + half * 8192 + quad * 512, &map_wg, d0 + half * kAtomK, r[0], r[1], r[2], r[3], full + 8 * s);
+        tma_gather4(wdst + half * kHalfBytes + quad * (kHalfBytes / 16), &map_wg, (d0 + half * kAtomK) / kColDiv, r[0], r[1],
+                    r[2], r[3], full + 8 * s);
       } else if (lane < 2) {
         // every row: 64 consecutive rows per column half; rows past the matrix read as zero
-        tma_tile_2d(abase + lane * 8192, &map_wt, d0 + lane * kAtomK, u0, full + 8 * s);
+        tma_tile_2d(wdst + lane * kHalfBytes, &map_wt, (d0 + lane * kAtomK) / kColDiv, u0, full + 8 * s);
       }
       if (lane == 0) tma_tile_2d(abase + kAAtomBytes, &map_hm, u0, 0, full + 8 * s);
+    }
+  } else if (QB && warp >= kThreads / 32) {
+    // ======================= expanders (quantised rows): the stage's codes -> its two bf16 blocks =
+    // two pairs of warps, each with the slots of its parity (S is even)
+    const int pair = (tid - kThreads) / (16 * kExpandWarps);
+    const int et = (tid - kThreads) % (16 * kExpandWarps);
+    int s = 0, ph = 0;
+    for (int kb = 0; kb < kblocks; ++kb, ++s) {
+      if (s == S) { s = 0; ph ^= 1; }
+      if ((s & 1) != pair) continue;
+      const bool ok = mbar_wait(full + 8 * s, ph, abort_flag, p.status, p.wait_cycles);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const uint32_t sbase = stage0 + s * stage_bytes;
+      expand_block<QB ? QB : 8>(sbase + raw_off, sbase, kAtomK, et, 16 * kExpandWarps);
+      expand_block<QB ? QB : 8>(sbase + raw_off + kRawBytes / 2, sbase + kAAtomBytes / 2, kAtomK, et, 16 * kExpandWarps);
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(ready + 8 * s);
     }
   } else if (warp >= 8) {
     // ======================= MMA issuers (slot s belongs to issuer s mod 2) =====================
@@ -778,7 +949,7 @@ __global__ void __launch_bounds__(kThreads, 2) umma_down_kernel(const UmmaDownPa
       for (int kb = 0; kb < kblocks; ++kb, ++s) {
         if (s == S) { s = 0; ph ^= 1; }
         if (nacc == 2 && (s & 1) != m) continue;
-        if (!mbar_wait(full + 8 * s, ph, abort_flag, p.status, p.wait_cycles)) { ok = false; break; }
+        if (!mbar_wait((QB ? ready : full) + 8 * s, ph, abort_flag, p.status, p.wait_cycles)) { ok = false; break; }
         tc_fence_after();
         const uint32_t sbase = stage0 + s * stage_bytes;
         const uint64_t bdesc = make_desc(sbase + kAAtomBytes);
@@ -907,6 +1078,45 @@ bool make_map(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_el
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Rows of weight codes [rows, K] (qbits 8 or 4 per code, `pitch_bytes` apart), read in boxes of 64 codes x box_rows
+// rows that land densely, without swizzle.
+bool make_map_codes(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_bytes, int box_rows, int qbits) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)K * qbits / 8, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)pitch_bytes};
+  const cuuint32_t box[2] = {(cuuint32_t)(kAtomK * qbits / 8), (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_weight_map(CUtensorMap* m, const void* base, int K, int rows, int box_rows, int qbits) {
+  return qbits ? make_map_codes(m, base, K, rows, (size_t)K * qbits / 8, box_rows, qbits)
+               : make_map(m, base, K, rows, (size_t)K, box_rows);
+}
+
+template <int MODE, typename Map>
+cudaError_t launch_rows_mode(const UmmaRowsParams& p, int grid, size_t smem, cudaStream_t s, const CUtensorMap& map_w,
+                             const CUtensorMap& map_x, const Map& map_t) {
+  static unsigned long long configured[3] = {0, 0, 0};
+  cudaError_t e;
+  if (p.qbits == 8) {
+    auto k = umma_rows_kernel<MODE, 8>;
+    if ((e = allow_dynamic_smem(k, 227 * 1024, configured[0])) != cudaSuccess) return e;
+    return launch_pdl(k, dim3(grid), dim3(kThreadsRows + 32 * kExpandWarps), smem, s, p, map_w, map_x, map_t);
+  }
+  if (p.qbits == 4) {
+    auto k = umma_rows_kernel<MODE, 4>;
+    if ((e = allow_dynamic_smem(k, 227 * 1024, configured[1])) != cudaSuccess) return e;
+    return launch_pdl(k, dim3(grid), dim3(kThreadsRows + 32 * kExpandWarps), smem, s, p, map_w, map_x, map_t);
+  }
+  auto k = umma_rows_kernel<MODE, 0>;
+  if ((e = allow_dynamic_smem(k, 227 * 1024, configured[2])) != cudaSuccess) return e;
+  return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, map_t);
+}
+
 }  // namespace
 
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s) {
@@ -918,29 +1128,20 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
   const size_t smem = 226 * 1024;
   p.ring_bytes = (int)smem - 1024 - kHeaderBytes;
   alignas(64) CUtensorMap map_w, map_x;
+  if (p.qbits != 0 && p.qbits != 8 && p.qbits != 4) return cudaErrorInvalidValue;
   // weights: all R rows; boxes of one tile's rows for the gate, single-row boxes for the gather
-  if (!make_map(&map_w, p.W, p.K, p.R, (size_t)p.K, up ? 1 : tile_rows_for(p.R, grid))) return cudaErrorNotSupported;
+  if (!make_weight_map(&map_w, p.W, p.K, p.R, up ? 1 : tile_rows_for(p.R, grid), p.qbits)) return cudaErrorNotSupported;
   // tokens: only the rows that exist; the box covers npad rows and the rest reads as zero
   if (!make_map(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)) return cudaErrorNotSupported;
-  static unsigned long long configured[3] = {0, 0, 0};
-  cudaError_t e;
-  if (!up) {
-    auto k = umma_rows_kernel<kGate>;
-    if ((e = allow_dynamic_smem(k, 227 * 1024, configured[0])) != cudaSuccess) return e;
-    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, WalkMap<false>{});
-  }
+  if (!up) return launch_rows_mode<kGate>(p, grid, smem, s, map_w, map_x, WalkMap<false>{});
   if (p.walk_all && umma_may_walk(p.B)) {
     // wide batches: the union may cover most rows; the kernel then walks every row with tiled boxes of the tile
     // height of R rows (decided on the device from the union's size, so it depends on this call's inputs only)
     WalkMap<true> map_t;
-    if (!make_map(&map_t.m, p.W, p.K, p.R, (size_t)p.K, tile_rows_for(p.R, grid))) return cudaErrorNotSupported;
-    auto k = umma_rows_kernel<kUpMayWalk>;
-    if ((e = allow_dynamic_smem(k, 227 * 1024, configured[2])) != cudaSuccess) return e;
-    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, map_t);
+    if (!make_weight_map(&map_t.m, p.W, p.K, p.R, tile_rows_for(p.R, grid), p.qbits)) return cudaErrorNotSupported;
+    return launch_rows_mode<kUpMayWalk>(p, grid, smem, s, map_w, map_x, map_t);
   }
-  auto k = umma_rows_kernel<kUp>;
-  if ((e = allow_dynamic_smem(k, 227 * 1024, configured[1])) != cudaSuccess) return e;
-  return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, WalkMap<false>{});
+  return launch_rows_mode<kUp>(p, grid, smem, s, map_w, map_x, WalkMap<false>{});
 }
 
 int umma_down_splits(int D, int sm_count, int max_splits) {
@@ -951,27 +1152,40 @@ int umma_down_splits(int D, int sm_count, int max_splits) {
 
 bool umma_down_supported(int D, int cols) { return D % kTileRows == 0 && cols >= 1 && cols <= 64; }
 
+namespace {
+template <int QB>
+cudaError_t launch_down_q(const UmmaDownParams& p, int grid, size_t smem, cudaStream_t s, const CUtensorMap& map_wg,
+                          const CUtensorMap& map_wt, const CUtensorMap& map_hm) {
+  static unsigned long long configured = 0;
+  const cudaError_t e = allow_dynamic_smem(umma_down_kernel<QB>, 113 * 1024, configured);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(umma_down_kernel<QB>, dim3(grid), dim3(kThreads + (QB ? 32 * kExpandWarps : 0)), smem, s, p, map_wg,
+                    map_wt, map_hm);
+}
+}  // namespace
+
 cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s) {
+  if (p.qbits != 0 && p.qbits != 8 && p.qbits != 4) return cudaErrorInvalidValue;
   p.npad = (p.B + 15) / 16 * 16;
   p.wait_cycles = fused_test_knobs().wait_cycles;
-  const int stage_bytes = kAAtomBytes + p.npad * 128;
+  const int stage_bytes = kAAtomBytes + p.npad * 128 + p.qbits * kTileRows * kAtomK / 8;
   int stages = (111 * 1024 - 1024 - 1024) / stage_bytes;
   if (stages > 12) stages = 12;
   stages &= ~1;
   if (stages < 2) return cudaErrorInvalidValue;
   p.stages = stages;
-  const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 2) * 8 + 64;
+  const size_t smem = 1024 + (size_t)stages * stage_bytes + (3 * stages + 4) * 8 + 64;
   const int grid = (p.D / kTileRows) * p.splits;
   alignas(64) CUtensorMap map_wg, map_wt, map_hm;
   // W_down [H, D]: inner dimension d; single-row boxes for the gather, 64-row boxes for the dense walk
-  if (!make_map(&map_wg, p.W_down, p.D, p.R, (size_t)p.D, 1)) return cudaErrorNotSupported;
-  if (!make_map(&map_wt, p.W_down, p.D, p.R, (size_t)p.D, kAtomK)) return cudaErrorNotSupported;
+  if (!make_weight_map(&map_wg, p.W_down, p.D, p.R, 1, p.qbits)) return cudaErrorNotSupported;
+  if (!make_weight_map(&map_wt, p.W_down, p.D, p.R, kAtomK, p.qbits)) return cudaErrorNotSupported;
   // HmT [B][hm_stride]: inner dimension u; token rows past B read as zero
   if (!make_map(&map_hm, p.hmT, p.hm_stride, p.B, (size_t)p.hm_stride, p.npad)) return cudaErrorNotSupported;
-  static unsigned long long configured = 0;
-  const cudaError_t e = allow_dynamic_smem(umma_down_kernel, 113 * 1024, configured);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(umma_down_kernel, dim3(grid), dim3(kThreads), smem, s, p, map_wg, map_wt, map_hm);
+  const int g = grid;
+  return p.qbits == 8   ? launch_down_q<8>(p, g, smem, s, map_wg, map_wt, map_hm)
+         : p.qbits == 4 ? launch_down_q<4>(p, g, smem, s, map_wg, map_wt, map_hm)
+                        : launch_down_q<0>(p, g, smem, s, map_wg, map_wt, map_hm);
 }
 
 cudaError_t launch_rmsnorm_split(const float* v, int B, int r, int v_stride, const float* gain, float eps,

@@ -10,8 +10,11 @@ namespace sffn {
 constexpr int kUmmaActIdentity = 3;
 
 struct UmmaRowsParams {
-  const void* W;         // [*, K] bf16, rows selected by idx (or 0..R-1)
+  const void* W;         // [*, K] bf16 (or int8 / packed int4 codes, see qbits), rows selected by idx (or 0..R-1)
   int R, K;
+  int qbits;             // 0: bf16 rows; 8 / 4: rows of weight codes, K * qbits / 8 bytes each
+  const float* w_scale;  // quantised rows: scale of row j of W (applied to its accumulator row), or null
+  const float* out_scale;  // UP, quantised rows: scale of row j of the down matrix, folded into Hm, or null
   const int32_t* idx;    // UP: list of rows, or null
   const int32_t* count;  // UP: device length of the list, or null (= R)
   const uint32_t* words_in;  // UP, instead of idx / count: the gate kernel's "fired" bit masks (n_words of
@@ -47,8 +50,9 @@ struct UmmaRowsParams {
 };
 
 struct UmmaDownParams {
-  const void* W_down;    // [R, D] bf16
+  const void* W_down;    // [R, D] bf16 (or codes, see qbits; their row scales are already folded into hmT)
   int R, D;
+  int qbits;             // 0: bf16 rows; 8 / 4: rows of weight codes
   const int32_t* idx;    // list of rows (readable up to the next multiple of 64 past its length), or null = all R rows
   const int32_t* count;  // device length of the list, or null (= R)
   const void* hmT;       // bf16 [B][hm_stride]; entries from the list's end to the next multiple of 64 are zero

@@ -302,9 +302,10 @@ def test_host_entry_and_errors(mod):
         ffn.sparse_ffn_forward(x[0], gate, w["b_g"], big[1:1 + H * D].view(H, D), w["W_down"])
     assert e.value.code == 2
     ffn.set_path("fused")
-    with pytest.raises(mod.SFFNError) as e:                           # the fused kernel is single-token
-        ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"])
-    assert e.value.code == 2
+    n0 = ffn.launch_count()                                           # the fused kernel is single-token: a batch
+    yb = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"])   # runs it once per token
+    assert ffn.launch_count() - n0 == x.shape[0]
+    assert torch.equal(yb[1], ffn.sparse_ffn_forward(x[1], gate, w["b_g"], w["W_up"], w["W_down"]))
     with pytest.raises(mod.SFFNError):                                # rows must be multiples of 16 bytes
         mod.SparseFFN(260, 64, torch.bfloat16)
 
@@ -314,6 +315,8 @@ def test_host_entry_and_errors(mod):
     (256, 50048, 4, 0.9),    # more flags than the in-kernel compaction takes: separate compaction launch
     (256, 777, 3, 0.9),      # H not a multiple of 8: ragged last tile, byte-wise flag reads
     (512, 1500, 33, 0.95),   # 33 tokens: 48 token columns, three column groups shared by all warps
+    (512, 19072, 40, 0.9),   # the same with two tiles for some CTAs: warps that join for the last tile only
+    (512, 38000, 20, 0.95),  # three tiles for some CTAs
     (256, 64, 2, 0.5),       # fewer rows than one tile of eight per CTA
 ])
 def test_batched_tcgen05_edge_shapes(mod, D, H, B, s):
