@@ -142,9 +142,18 @@ int sffn_set_gate_engine(sffn_handle* handle, int engine /* sffn_gate_engine */)
  * sparse one.  It exists as A_3 only: the gate's `act` must be one of the three sparse activations.  A neuron whose product
  * A(.) A_3(.) is zero for every token of the call contributes nothing (the "s_gated" site of the
  * paper's sparsity-sites table): the CUDA-core path (SFFN_PATH_GENERAL) then does not read its row of
- * W_down; the fused and the tensor-core paths fetch the two rows of a fired neuron together and read it.
+ * W_down; the tensor-core paths fetch the two rows of a fired neuron together and read it, and so does the
+ * single-token fused kernel unless sffn_set_gated_skip asks otherwise.
  * SFFN_ACT_NONE and SFFN_ACT_SILU are not gate activations: `act` of the forward calls stays one of the first three. */
 int sffn_set_up_activation(sffn_handle* handle, int act_up /* sffn_act */);
+
+/* The "s_gated" site on the single-token fused kernel (sparsity-sites table; Sec. 3.3 "Double activation").  on = 1:
+ * sparse calls with one token, a standard gate, bf16 or fp32 rows and an up activation set fetch the W_down row of a
+ * fired neuron only once h_j = a_j A_3(u_j) is known and is not zero: a second, dependent fetch per kept row instead of
+ * two rows fetched together.  y is bitwise the same either way; fewer bytes are read (about half of the W_down rows
+ * with A_3 = RELU), but the last rows of a call pay two round trips to memory instead of one, and on a B200 the call
+ * is not faster for it (0 to 1.5 us slower): the default is 0.  Every other kind of call ignores the setting. */
+int sffn_set_gated_skip(sffn_handle* handle, int on);
 
 /* Sparse execution of Eq. 1 (Sec. 3.1): gate in full, then only the active rows of W_up / W_down.
  * x [B,D] and all weights on the device; y [B,D] fp32 on the device, fully overwritten (zeros when

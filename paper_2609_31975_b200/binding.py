@@ -63,6 +63,7 @@ def load_library() -> ctypes.CDLL:
         lib.sffn_destroy.argtypes = [vp]
         lib.sffn_set_path.argtypes = [vp, i]
         lib.sffn_set_up_activation.argtypes = [vp, i]
+        lib.sffn_set_gated_skip.argtypes = [vp, i]
         lib.sffn_set_gate_engine.argtypes = [vp, i]
         fwd = [vp, vp, i, ctypes.POINTER(_Gate), vp, vp, vp, i, vp, vp]
         lib.sparse_ffn_forward.argtypes = fwd
@@ -212,6 +213,8 @@ class SparseFFN:
             _check("sffn_create", self.lib.sffn_create(ctypes.byref(h), D, H, r_max, B_max, self._dt,
                                                        ctypes.c_void_p(self._ws_ptr), need.value))
         self._h = h
+        if os.environ.get("SFFN_GATED_SKIP") == "1":   # lets a profiler run of bench.py take the gated variant
+            self.set_gated_skip(True)
         self._keep = None
 
     def close(self):
@@ -225,6 +228,10 @@ class SparseFFN:
         """Double activation: ``act_up`` in ACT (or None for Eq. 1) is applied to the up projection."""
         code = 3 if act_up is None else ACT_UP[act_up]
         _check("sffn_set_up_activation", self.lib.sffn_set_up_activation(self._h, code))
+
+    def set_gated_skip(self, on: bool):
+        """Single-token double-activation calls fetch W_down rows only where h != 0 (sffn_set_gated_skip; default off)."""
+        _check("sffn_set_gated_skip", self.lib.sffn_set_gated_skip(self._h, 1 if on else 0))
 
     def set_path(self, path: str):
         _check("sffn_set_path", self.lib.sffn_set_path(self._h, PATH[path]))

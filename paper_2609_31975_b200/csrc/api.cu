@@ -73,6 +73,7 @@ struct sffn_handle {
   int sm_count;
   int path;
   int act_up;  // activation on the up projection (double activation), SFFN_ACT_NONE = Eq. 1
+  int gated_skip;  // single-token fused kernel: W_down rows only where h != 0 (see sffn_set_gated_skip)
   int gate_engine = SFFN_GATE_ENGINE_AUTO;
   long long launches;
   int list_state;  // 0: no sparse call yet, 1: idx/count hold the last call's list, 2: flags hold it
@@ -131,6 +132,7 @@ int sffn_create(sffn_handle** handle, int D, int H, int r_max, int B_max, int dt
   h->sm_count = sms;
   h->path = SFFN_PATH_AUTO;
   h->act_up = SFFN_ACT_NONE;
+  h->gated_skip = 0;
   h->launches = 0;
   h->list_state = 0;
   *handle = h;
@@ -146,6 +148,12 @@ int sffn_destroy(sffn_handle* h) {
 int sffn_set_gate_engine(sffn_handle* h, int engine) {
   if (!h || engine < SFFN_GATE_ENGINE_AUTO || engine > SFFN_GATE_ENGINE_TENSOR_CORE) return SFFN_ERR_INVALID_ARG;
   h->gate_engine = engine;
+  return SFFN_OK;
+}
+
+int sffn_set_gated_skip(sffn_handle* h, int on) {
+  if (!h) return SFFN_ERR_INVALID_ARG;
+  h->gated_skip = on != 0;
   return SFFN_OK;
 }
 
@@ -547,6 +555,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
       c.D = h->D; c.H = h->H;
       c.x = static_cast<const char*>(x) + (size_t)b * tok_bytes;
       c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up;
+      c.gated_skip = h->gated_skip != 0;
       c.engine = h->gate_engine; c.y = y + (size_t)b * h->D;
       c.dense = dense; c.flag_or = b > 0;
       c.workspace = h->ws + h->L.fused;
@@ -569,6 +578,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
     if (q8) { c.s_gate = q8->s_gate; c.s_V = q8->s_V; c.s_up = q8->s_up; c.s_down = q8->s_down; }
     c.D = h->D; c.H = h->H;
     c.x = x; c.gate = g; c.b_g = b_g; c.W_up = W_up; c.W_down = W_down; c.act = act; c.act_up = h->act_up; c.engine = h->gate_engine; c.y = y;
+    c.gated_skip = h->gated_skip != 0;
     c.dense = dense;
     c.workspace = h->ws + h->L.fused;
     c.r_max = h->r_max;

@@ -99,9 +99,10 @@ struct FusedParams {
 
 // Shared-memory carve-up, identical on host and device.
 struct SmemLayout {
-  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, row_params, row_scales, slot_scales, total;
+  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, row_params, row_scales, slot_scales, gated_bars, gated_vals, total;
   __host__ __device__ SmemLayout(int D, int K, bool lopa, int n_gate_slots, int gate_slot_bytes,
-                                 int n_act_slots, int act_slot_bytes, int slab_max, bool scaled, int act_extra = 0) {
+                                 int n_act_slots, int act_slot_bytes, int slab_max, bool scaled, int act_extra = 0,
+                                 bool gated = false) {
     int off = 0;
     auto take = [&](int bytes) {
       int o = off;
@@ -120,6 +121,10 @@ struct SmemLayout {
     row_params = take((lopa || scaled) ? (1 + (lopa ? 2 : 0) + (scaled ? 1 : 0)) * slab_max * 4 : 0);  // per-neuron gate parameters
     row_scales = take(scaled ? 2 * slab_max * 4 : 0);     // int8 rows: scales of the slab's W_up / W_down rows
     slot_scales = take(scaled ? 2 * (n_act_slots + act_extra) * 4 : 0);  // the same two for the row in each act slot
+    // gated variant (W_down rows only where h != 0): the act ring is cut into single rows (2 per act slot), each with
+    // up to three barriers and three values
+    gated_bars = take(gated ? 3 * 2 * n_act_slots * 8 : 0);
+    gated_vals = take(gated ? 3 * 2 * n_act_slots * 4 : 0);
     total = off;
   }
 };
@@ -301,8 +306,16 @@ __device__ __forceinline__ long long global_ns() {
 #define SFFN_STAMP(slot) do { } while (0)
 #endif
 
-template <typename T, int CPT, bool LOPA>
+// GATED (double activation, standard gate, sparse route): the W_down row of a fired neuron is fetched only once
+// h_j = a_j A_3(u_j) is known and is not zero (the "gated" sparsity site of the paper's table of sites).  The act ring
+// is then two rings of single rows: the first act producer fills the "up" ring with W_up rows as before; the act
+// warps dot two of them per round, publish the two h and release the rows at once; the second act producer follows
+// the published h in order and copies the W_down rows that are needed into the "down" ring, which the act warps
+// consume one round behind (whatever is left after the stop marker).  Rows are added in the same order as in the
+// other variant and a skipped row would have added zeros, so y is bitwise the same.
+template <typename T, int CPT, bool LOPA, bool GATED = false>
 __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParams p) {
+  static_assert(!(GATED && LOPA), "the gated variant is built for the standard gate");
   // Warp roles: 2 gate producers, 2 act producers, then gate warps and act warps.  The standard gate needs its
   // eight gate warps to keep up with the stream; the LoPA gate is short (r elements per row), the call's time
   // is then set by the up/down rows, so eight of the twelve workers are act warps there.
@@ -336,7 +349,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   // use once every gate row has been consumed -- from then on the rows of fired neurons are all that is left to
   // fetch, and how many of them are in flight sets how fast they come.
   const int NG = p.n_gate_slots, NAown = p.n_act_slots, NA = p.act_used;
-  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra);
+  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra, GATED);
 
   unsigned char* gate_ring = smem + L.gate_ring;
   unsigned char* act_ring = smem + L.act_ring;
@@ -371,6 +384,15 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const uint32_t full_gate = bars, empty_gate = bars + 8 * NG;
   const uint32_t full_act = bars + 16 * NG, empty_act = bars + 16 * NG + 8 * NA;
   const uint32_t v_bar = bars + 16 * (NG + NA);
+  // Gated variant: NU rows of the act ring for W_up rows, ND for W_down rows (about a third: half of the fired neurons
+  // need one, and it stays for one round trip only).
+  const int NH = 2 * NAown, ND = NH / 3 < 2 ? 2 : NH / 3, NU = NH - ND;
+
+  const uint32_t full_up = smem_u32(smem + L.gated_bars), empty_up = full_up + 8 * NU, h_ready = empty_up + 8 * NU;
+  const uint32_t full_dn = h_ready + 8 * NU, empty_dn = full_dn + 8 * ND;
+  float* up_a = reinterpret_cast<float*>(smem + L.gated_vals);       // [NU] gate value of the row, < 0 = stop marker
+  volatile float* up_h = up_a + NU;                                  // [NU] h of the row, published by the act warps
+  volatile float* dn_h = up_a + 2 * NU;                              // [ND] h of the row in a down slot
 
   const int nvecD = D / EPV, nvecK = K / EPV;
   const size_t row_bytes = row_bytes_of<T>(D);
@@ -399,6 +421,17 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       for (int s = 0; s < NA; ++s) {
         mbar_init(full_act + 8 * s, kActProducers);
         mbar_init(empty_act + 8 * s, kGAW);
+      }
+      if (GATED) {
+        for (int s = 0; s < NU; ++s) {
+          mbar_init(full_up + 8 * s, 1);
+          mbar_init(empty_up + 8 * s, kGAW);
+          mbar_init(h_ready + 8 * s, 1);
+        }
+        for (int s = 0; s < ND; ++s) {
+          mbar_init(full_dn + 8 * s, 1);
+          mbar_init(empty_dn + 8 * s, kGAW);
+        }
       }
       mbar_init(v_bar, 1);
       for (int i = 0; i < 8; ++i) ctl[i] = 0;
@@ -733,12 +766,60 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     uint32_t par = 1;
     bool ok = true;
     int n_seq = 0;  // ring slots handed out so far
-    // The whole warp classifies 32 rows per step (one shared-memory read + ballots); lane 0 issues
-    // the copies of the fired ones in ascending order.  Only the leading run of finished rows is
-    // consumed, so the order never depends on which gate warp was faster.
+    // ring that this loop fills: the act slots (both producers), or, gated variant, the W_up rows (first producer)
+    const int NR = GATED ? NU : NA;
+    const uint32_t pfull = GATED ? full_up : full_act, pempty = GATED ? empty_up : empty_act;
+    float* pa = GATED ? up_a : slot_a;
 #ifdef SFFN_TRACE
     int n_issued = 0;
 #endif
+    if (GATED && ap == 1) {
+      // Gated variant, second producer: lane 0 follows the fired rows in order, waits for the h of each (published by
+      // the act warps per W_up slot) and requests the W_down row into the next slot of the down ring if it is not zero.
+      int us = 0, ds = 0;
+      uint32_t upar = 0, dpar = 1;
+      long long t_idle = 0;
+      for (int base = 0; ok && base < slab_rows;) {
+        const int row = base + lane;
+        const uint32_t st = row < slab_rows ? row_state[row] : 0x80000000u;
+        const unsigned done = __ballot_sync(0xffffffffu, st != 0xffffffffu);
+        const int prefix = done == 0xffffffffu ? 32 : __ffs(~done) - 1;
+        if (prefix == 0) {  // the next row's gate is not computed yet
+          if (t_idle == 0) t_idle = clock64();
+          __nanosleep(20);
+          if (ctl[kAbort]) ok = false;
+          else if (clock64() - t_idle > p.wait_cycles) { if (lane == 0) raise_timeout(ctl, p.status, 48); ok = false; }
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          continue;
+        }
+        t_idle = 0;
+        unsigned fired = __ballot_sync(0xffffffffu, row < slab_rows && lane < prefix && st != 0x80000000u);
+        if (lane == 0) {
+          while (fired && ok) {
+            const int r = base + __ffs(fired) - 1;
+            fired &= fired - 1;
+            ok = mbar_wait<true>(h_ready + 8 * us, upar, ctl, p.status, p.wait_cycles, 52);
+            const float hv = ok ? up_h[us] : 0.f;
+            if (++us == NU) { us = 0; upar ^= 1; }
+            if (hv == 0.f) continue;  // the row would be multiplied by zero
+            ok = mbar_wait<true>(empty_dn + 8 * ds, dpar, ctl, p.status, p.wait_cycles, 53);
+            if (!ok) break;
+            dn_h[ds] = hv;  // ordered before the act warps' read by the arrive below and the copy's completion
+            size_t j = (size_t)(slot_first_neuron(r / nr) + r % nr);
+            if (!SFFN_IN_BOUNDS(j < (size_t)p.H, p.status, 5)) j = 0;
+            mbar_expect_tx(full_dn + 8 * ds, (uint32_t)row_bytes);
+            bulk_g2s(smem_u32(act_ring) + (uint32_t)((NU + ds) * row_bytes), Wsrc + j * row_bytes, (uint32_t)row_bytes,
+                     full_dn + 8 * ds);
+            if (++ds == ND) { ds = 0; dpar ^= 1; }
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        base += prefix;
+      }
+    } else {
+    // The whole warp classifies 32 rows per step (one shared-memory read + ballots); lane 0 issues
+    // the copies of the fired ones in ascending order.  Only the leading run of finished rows is
+    // consumed, so the order never depends on which gate warp was faster.
     long long t_idle = 0;
     for (int base = 0; ok && base < slab_rows;) {
       const int row = base + lane;
@@ -761,15 +842,15 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       // is what bounds a call with a short gate).
       while (fired && ok) {
         const int place = __popc(fired & ((1u << lane) - 1u));
-        const int nb = min(__popc(fired), NA);
+        const int nb = min(__popc(fired), NR);
         const bool mine = ((fired >> lane) & 1u) != 0 && place < nb;
         bool good = true;
         if (mine) {
           int ms = slot + place;
           uint32_t mp = par;
-          if (ms >= NA) { ms -= NA; mp ^= 1; }
-          bool free_slot = mbar_wait<true>(empty_act + 8 * ms, mp, ctl, p.status, p.wait_cycles, 42);
-          if (free_slot && ms >= NAown && n_seq + place < NA) {
+          if (ms >= NR) { ms -= NR; mp ^= 1; }
+          bool free_slot = mbar_wait<true>(pempty + 8 * ms, mp, ctl, p.status, p.wait_cycles, 42);
+          if (!GATED && free_slot && ms >= NAown && n_seq + place < NA) {
             // first use of a slot inside the gate ring: not before the gate warps have read every gate row
             const long long t0 = clock64();
             while (ctl[kGateDone] < n_gslots) {
@@ -779,16 +860,17 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
             }
           }
           if (free_slot) {
-            if (ap == 0) slot_a[ms] = st == 0x80000000u ? 0.f : __uint_as_float(st);
+            if (ap == 0) pa[ms] = st == 0x80000000u ? 0.f : __uint_as_float(st);
             if (kScaled && ap == 0) {
               slot_su[ms] = row_su[row];
               slot_sd[ms] = row_sd[row];
             }
             size_t j = (size_t)(slot_first_neuron(row / nr) + row % nr);
-            if (!SFFN_IN_BOUNDS(j < (size_t)p.H && ms >= 0 && ms < NA, p.status, 2)) j = 0;
-            mbar_expect_tx(full_act + 8 * ms, (uint32_t)row_bytes);
-            bulk_g2s(smem_u32(act_slot(ms)) + (ap == 0 ? 0u : (uint32_t)row_bytes), Wsrc + j * row_bytes,
-                     (uint32_t)row_bytes, full_act + 8 * ms);
+            if (!SFFN_IN_BOUNDS(j < (size_t)p.H && ms >= 0 && ms < NR, p.status, 2)) j = 0;
+            mbar_expect_tx(pfull + 8 * ms, (uint32_t)row_bytes);
+            const uint32_t dst = GATED ? smem_u32(act_ring) + (uint32_t)(ms * row_bytes)
+                                       : smem_u32(act_slot(ms)) + (ap == 0 ? 0u : (uint32_t)row_bytes);
+            bulk_g2s(dst, Wsrc + j * row_bytes, (uint32_t)row_bytes, pfull + 8 * ms);
           } else {
             good = false;
           }
@@ -800,7 +882,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
 #endif
         slot += nb;
         n_seq += nb;
-        if (slot >= NA) { slot -= NA; par ^= 1; }
+        if (slot >= NR) { slot -= NR; par ^= 1; }
       }
       base += prefix;
     }
@@ -809,17 +891,18 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     if (lane == 0 && ap == 0) SFFN_STAMP(7);
     if (lane == 0) {
       const int per_round = NA >= 4 ? 2 : 1;
-      const int n_end = p.act_groups == 1 ? n_seq + 1 : (n_seq / per_round + p.act_groups) * per_round;
+      const int n_end = p.act_groups == 1 || GATED ? n_seq + 1 : (n_seq / per_round + p.act_groups) * per_round;
       for (; ok && n_seq < n_end; ++n_seq) {
-        if (mbar_wait<true>(empty_act + 8 * slot, par, ctl, p.status, p.wait_cycles, 43)) {
-          if (ap == 0) slot_a[slot] = -1.f;
-          mbar_arrive(full_act + 8 * slot);
+        if (mbar_wait<true>(pempty + 8 * slot, par, ctl, p.status, p.wait_cycles, 43)) {
+          if (ap == 0) pa[slot] = -1.f;
+          mbar_arrive(pfull + 8 * slot);
         } else {
           ok = false;
         }
-        if (++slot == NA) { slot = 0; par ^= 1; }
+        if (++slot == NR) { slot = 0; par ^= 1; }
       }
     }
+    }  // not the gated variant's second producer
     if (ap == 0) {
       // This CTA's place in the order of finishing (the first R sum the partials), taken now so that the round trip
       // overlaps with the act warps' last rows; -1 under the test hook that makes a CTA go missing.
@@ -889,6 +972,124 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     // arrives, so waiting for the second slot of a round cannot block for good.  A thread whose
     // wait ran out still joins the barrier and raises the group's stop flag, so the four warps
     // always leave the loop together.
+    if constexpr (GATED) {
+      // Two W_up rows per round; the W_down rows that the previous round asked for are added after this round's h
+      // have been published, whatever is left after the stop marker.
+      int us = 0, ds = 0;
+      uint32_t upar = 0, dpar = 0;
+      int pend = 0;         // W_down rows requested by the previous round
+      bool failed = false;  // a wait ran out
+      auto add_down = [&](int n) {
+        for (int k = 0; k < n && !failed; ++k) {
+          if (!mbar_wait(full_dn + 8 * ds, dpar, ctl, p.status, p.wait_cycles, 54)) { failed = true; break; }
+          const float h = dn_h[ds];
+          const uint4* wd = reinterpret_cast<const uint4*>(act_ring + (size_t)(NU + ds) * row_bytes);
+#pragma unroll
+          for (int i = 0; i < CPT; ++i) {
+            const int c = gat + i * kGT;
+            if (c < nvecD) {
+              float f[EPV];
+              Elem<T>::unpack(wd[c], f);
+#pragma unroll
+              for (int e = 0; e < EPV; e += 2) {
+                const float2 t = fma2(make_float2(h, h), make_float2(f[e], f[e + 1]), make_float2(acc[i][e], acc[i][e + 1]));
+                acc[i][e] = t.x;
+                acc[i][e + 1] = t.y;
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty_dn + 8 * ds);
+          if (++ds == ND) { ds = 0; dpar ^= 1; }
+        }
+      };
+      for (int round = 0;; ++round) {
+        float* rp = red + (round & 1) * (2 * kGAW + 1);
+        const int us1 = us + 1 == NU ? 0 : us + 1;
+        const uint32_t upar1 = us + 1 == NU ? upar ^ 1 : upar;
+        const bool got0 = mbar_wait(full_up + 8 * us, upar, ctl, p.status, p.wait_cycles, 45);
+        const float a0 = got0 ? up_a[us] : -1.f;
+        bool got1 = true;
+        float a1 = -1.f;
+        if (a0 >= 0.f) {
+          got1 = mbar_wait(full_up + 8 * us1, upar1, ctl, p.status, p.wait_cycles, 46);
+          a1 = got1 ? up_a[us1] : -1.f;
+        }
+        if (a0 >= 0.f) {
+          const uint4* wu0 = reinterpret_cast<const uint4*>(act_ring + (size_t)us * row_bytes);
+          const uint4* wu1 = reinterpret_cast<const uint4*>(act_ring + (size_t)us1 * row_bytes);
+          float part0 = 0.f, part1 = 0.f;
+          float2 pk0 = make_float2(0.f, 0.f), pk1 = pk0, pk0b = pk0, pk1b = pk0;
+#pragma unroll
+          for (int i = 0; i < CPT; ++i) {
+            const int c = gat + i * kGT;
+            if (c < nvecD) {
+              if constexpr (kXReg && EPV != 16) {
+                float f[EPV];
+                Elem<T>::unpack(wu0[c], f);
+#pragma unroll
+                for (int e = 0; e < EPV; e += 4) {
+                  pk0 = fma2(make_float2(f[e], f[e + 1]), make_float2(xr[i][e], xr[i][e + 1]), pk0);
+                  pk0b = fma2(make_float2(f[e + 2], f[e + 3]), make_float2(xr[i][e + 2], xr[i][e + 3]), pk0b);
+                }
+                if (a1 >= 0.f) {
+                  Elem<T>::unpack(wu1[c], f);
+#pragma unroll
+                  for (int e = 0; e < EPV; e += 4) {
+                    pk1 = fma2(make_float2(f[e], f[e + 1]), make_float2(xr[i][e], xr[i][e + 1]), pk1);
+                    pk1b = fma2(make_float2(f[e + 2], f[e + 3]), make_float2(xr[i][e + 2], xr[i][e + 3]), pk1b);
+                  }
+                }
+              } else {
+                part0 = chunk_dot<T>(wu0[c], sx, c, nvecD, part0);
+                if (a1 >= 0.f) part1 = chunk_dot<T>(wu1[c], sx, c, nvecD, part1);
+              }
+            }
+          }
+          if constexpr (kXReg && EPV != 16) {
+            part0 = (pk0.x + pk0.y) + (pk0b.x + pk0b.y);
+            part1 = (pk1.x + pk1.y) + (pk1b.x + pk1b.y);
+          }
+          part0 = warp_sum(part0);
+          part1 = warp_sum(part1);
+          if (lane == 0) {
+            rp[gaw] = part0;
+            rp[kGAW + gaw] = part1;
+          }
+        }
+        if (a0 < 0.f || !got1) rp[2 * kGAW] = 1.f;  // stop marker first in the round, or a failed wait
+        named_bar_sync(2, kGT);
+        const bool stop = rp[2 * kGAW] != 0.f;
+        int asked = 0;
+        if (!stop) {
+          const float u0 = (rp[0] + rp[1]) + (rp[2] + rp[3]);
+          const float u1 = (rp[kGAW] + rp[kGAW + 1]) + (rp[kGAW + 2] + rp[kGAW + 3]);
+          const float h0 = a0 * activation(p.act_up, u0), h1 = a1 >= 0.f ? a1 * activation(p.act_up, u1) : 0.f;
+          if (at == 0) {  // the arrive releases the store: the second producer reads up_h after its wait
+            up_h[us] = h0;
+            mbar_arrive(h_ready + 8 * us);
+            if (a1 >= 0.f) {
+              up_h[us1] = h1;
+              mbar_arrive(h_ready + 8 * us1);
+            }
+          }
+          __syncwarp();
+          if (lane == 0) {  // the W_up rows have been read by every thread that passed the barrier
+            mbar_arrive(empty_up + 8 * us);
+            if (a1 >= 0.f) mbar_arrive(empty_up + 8 * us1);
+          }
+          asked = (h0 != 0.f ? 1 : 0) + (h1 != 0.f ? 1 : 0);
+        }
+        add_down(pend);
+        pend = asked;
+        if (stop || a1 < 0.f || failed) {
+          add_down(pend);
+          break;
+        }
+        us += 2;
+        while (us >= NU) { us -= NU; upar ^= 1; }
+      }
+    } else {
     const bool pair = NA >= 4;  // with fewer slots, holding two at a time would stall the act producers
     const int stride = (pair ? 2 : 1) * p.act_groups;  // ring slots from one round of a group to its next
     int slot = (pair ? 2 : 1) * grp;
@@ -1004,6 +1205,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       }
       slot += stride;
       while (slot >= NA) { slot -= NA; par ^= 1; }
+    }
     }
     if (at == 0) SFFN_STAMP(4);
     if (kGroups == 2) {
@@ -1291,15 +1493,15 @@ int fused_grid(int sm_count, int H) {
   return grid > H ? H : grid;
 }
 
-template <typename T, bool LOPA>
+template <typename T, bool LOPA, bool GATED = false>
 cudaError_t launch_main(const FusedParams& p, const Geometry& g, int grid, cudaStream_t s) {
   void (*k)(const FusedParams) = nullptr;
   constexpr int kMaxCpt = 64 / Elem<T>::kPerVec < 8 && TokenOf<T>::kScaled ? 64 / Elem<T>::kPerVec : 8;  // what plan() allows
   switch (g.cpt) {
-    case 1: k = fused_ffn_kernel<T, 1, LOPA>; break;
-    case 2: k = fused_ffn_kernel<T, 2, LOPA>; break;
-    case 4: k = fused_ffn_kernel<T, (kMaxCpt >= 4 ? 4 : kMaxCpt), LOPA>; break;
-    default: k = fused_ffn_kernel<T, kMaxCpt, LOPA>; break;
+    case 1: k = fused_ffn_kernel<T, 1, LOPA, GATED>; break;
+    case 2: k = fused_ffn_kernel<T, 2, LOPA, GATED>; break;
+    case 4: k = fused_ffn_kernel<T, (kMaxCpt >= 4 ? 4 : kMaxCpt), LOPA, GATED>; break;
+    default: k = fused_ffn_kernel<T, kMaxCpt, LOPA, GATED>; break;
   }
   if (g.cpt > kMaxCpt) return cudaErrorInvalidValue;
   static unsigned long long configured[4] = {0, 0, 0, 0};  // per instantiation of this template, per row width
@@ -1362,8 +1564,17 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   const bool lopa = c.gate->kind == SFFN_GATE_LOPA;
   const int K = lopa ? c.gate->r : c.D;
   const int grid = fused_grid(c.sm_count, c.H);
-  const Geometry g = plan(c.wkind, c.D, c.H, K, lopa, grid);
+  Geometry g = plan(c.wkind, c.D, c.H, K, lopa, grid);
   if (!g.ok) return cudaErrorInvalidValue;
+  // Double activation on the sparse route of a standard gate (bf16 / fp32 rows): W_down rows only where h != 0.
+  bool gated = c.gated_skip && c.act_up != kActNone && !c.dense && !lopa &&
+               (c.wkind == kWBF16 || c.wkind == kWF32) && g.n_act_slots >= 3 && g.act_extra == 0;
+  if (gated) {
+    const SmemLayout with(c.D, K, false, g.n_gate_slots, g.gate_slot_bytes, g.n_act_slots, g.act_slot_bytes, g.slab_max,
+                          false, g.act_extra, true);
+    if (with.total <= kSmemBudget) g.smem = with.total;
+    else gated = false;
+  }
   char* ws = static_cast<char*>(c.workspace);
   int n = 0;
   cudaError_t e;
@@ -1395,9 +1606,11 @@ cudaError_t launch_fused(const FusedCall& c, cudaStream_t s, int* launched) {
   else if (c.wkind == kWQ4)
     e = lopa ? launch_main<q4_t, true>(p, g, grid, s) : launch_main<q4_t, false>(p, g, grid, s);
   else if (c.wkind == kWBF16)
-    e = lopa ? launch_main<__nv_bfloat16, true>(p, g, grid, s) : launch_main<__nv_bfloat16, false>(p, g, grid, s);
+    e = lopa ? launch_main<__nv_bfloat16, true>(p, g, grid, s)
+             : gated ? launch_main<__nv_bfloat16, false, true>(p, g, grid, s) : launch_main<__nv_bfloat16, false>(p, g, grid, s);
   else
-    e = lopa ? launch_main<float, true>(p, g, grid, s) : launch_main<float, false>(p, g, grid, s);
+    e = lopa ? launch_main<float, true>(p, g, grid, s)
+             : gated ? launch_main<float, false, true>(p, g, grid, s) : launch_main<float, false>(p, g, grid, s);
   if (e != cudaSuccess) return e;
   ++n;
   if (launched) *launched = n;

@@ -23,6 +23,7 @@ struct FusedCall {
   const void* W_down;
   int act;
   int act_up;
+  bool gated_skip;       // double activation on the sparse route: W_down rows only where h != 0
   float* y;
   bool dense;
   int engine;        // sffn_gate_engine of the handle

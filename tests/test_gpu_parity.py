@@ -418,6 +418,45 @@ def test_double_activation_all_paths(mod, gate_engine, act, act_up):
     assert ffn.device_status() == 0
 
 
+@pytest.mark.parametrize("dtype,D,H,s", [(torch.bfloat16, 512, 1000, 0.9), (torch.float32, 264, 777, 0.8),
+                                         (torch.bfloat16, 2048, 300, 0.5), (torch.bfloat16, 4096, 14336, 0.9),
+                                         (torch.float32, 4096, 2000, 0.2), (torch.bfloat16, 8192, 4000, 0.9)])
+def test_gated_skip_fetches_fewer_rows_and_changes_no_bit(mod, dtype, D, H, s):
+    """sffn_set_gated_skip: the W_down row of a fired neuron only where a_j A_3(u_j) != 0 (single token, standard gate)."""
+    gate, w = make_std(D, H, dtype, 63, s)
+    x = syn.tokens(4, D, dtype, 63, DEV)
+    ffn = mod.SparseFFN(D, H, dtype, r_max=64, B_max=4)
+    tol = dict(rel_l2=1e-5, max_abs=1e-5) if dtype == torch.float32 else {}
+    for act_up in ("relu", "silu", "rsplus", None):
+        ffn.set_up_activation(act_up)
+        for t in range(4):
+            ffn.set_gated_skip(False)
+            y0 = ffn.sparse_ffn_forward(x[t], gate, w["b_g"], w["W_up"], w["W_down"], "relu").clone()
+            ffn.set_gated_skip(True)
+            y1 = ffn.sparse_ffn_forward(x[t], gate, w["b_g"], w["W_up"], w["W_down"], "relu").clone()
+            torch.cuda.synchronize()
+            assert ffn.device_status() == 0, ffn.status_words()
+            assert torch.equal(y0, y1), f"act_up={act_up} token {t}"
+            if t == 0:
+                ref = run_oracle(x[t], gate, w["b_g"], w["W_up"], w["W_down"], "relu", act_up=act_up)
+                assert_y_close(y1, ref["y"], what=f"gated skip act_up={act_up}", **tol)
+                assert_active_set(ffn.last_active(), ref, what=f"gated skip act_up={act_up}")   # the list stays the gate's
+                if act_up == "relu" and s > 0:
+                    assert ref["n_gated"][0] < ref["n_act"][0]                   # there are rows to skip
+    # the other kinds of call ignore the setting: a batch, the dense route, a LoPA gate
+    ffn.set_up_activation("relu")
+    yb = ffn.sparse_ffn_forward(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert_y_close(yb, run_oracle(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu", act_up="relu")["y"], what="batch", **tol)
+    yd = ffn.dense_ffn_forward(x[0], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+    assert_y_close(yd, run_oracle(x[0], gate, w["b_g"], w["W_up"], w["W_down"], "relu", act_up="relu", route="dense")["y"],
+                   what="dense", **tol)
+    lg, lw = make_lopa(mod, D, H, 64, dtype, 64, 0.8, "diag")
+    yl = ffn.sparse_ffn_forward(x[1], lg, lw["b_g"], lw["W_up"], lw["W_down"], "relu")
+    assert_y_close(yl, run_oracle(x[1], lg, lw["b_g"], lw["W_up"], lw["W_down"], "relu", act_up="relu")["y"], what="lopa", **tol)
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
+
+
 # ------------------------------------------------------------------ layer loop under a CUDA graph
 @pytest.mark.parametrize("kind", ["standard", "lopa"])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
