@@ -257,3 +257,49 @@ def test_int8_full_size_decode_and_lopa(mod):
     del gate, w
     gate, w = make_lopa(mod, D, H, 512, 18, 0.9, sign=True, gain=True)
     check(mod, ffn, x[0], gate, w, "relu", ("general", "fused"), "q8 full size lopa")
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_shapes_quantised_batches_agree_with_the_single_token_kernel(mod, seed):
+    """int8 and int4 rows: the tcgen05 batch kernels (auto) against the single-token kernel run once per token (fused),
+    random batch sizes (beyond 64 too: chunks), widths, neuron counts, LoPA ranks and activations."""
+    g = torch.Generator().manual_seed(8000 + seed)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))  # noqa: E731
+    for case in range(6):
+        bits = (8, 4)[ri(0, 1)]
+        B = ri(2, 40) if ri(0, 3) else ri(65, 100)
+        D = 256 * ri(1, 16)
+        H = ri(100, 6000) if ri(0, 4) else ri(19000, 24000)
+        lopa = ri(0, 2) == 0
+        r = 64 * ri(1, min(8, D // 128)) if lopa else 0
+        s = (0.6, 0.8, 0.9, 0.97)[ri(0, 3)]
+        act = ("relu", "sqrelu", "rsplus")[ri(0, 2)]
+        what = f"seed {seed} case {case}: int{bits} B={B} D={D} H={H} r={r} s={s} {act}"
+        ffn = mod.SparseFFN(D, H, torch.bfloat16, r_max=r, B_max=B)
+        sd = 9000 + 10 * seed + case
+        if lopa:
+            w = (syn.lopa_ffn_q8 if bits == 8 else syn.lopa_ffn_q4)(D, H, r, sd, DEV, sparsity=s, with_fixed_matrix=True)
+            gate = {"V": w["V"], "U": w["U"], "use_rmsnorm": ri(0, 1) == 1, "rms_eps": 1e-5, "g_idx": mod.g_diagonal(H, D, DEV)}
+        else:
+            w = (syn.standard_ffn_q8 if bits == 8 else syn.standard_ffn_q4)(D, H, sd, DEV, sparsity=s)
+            gate = {"W_g": w["W_g"]}
+        x = syn.tokens(B, D, torch.bfloat16, sd, DEV)
+        f = ffn.sparse_ffn_forward_q8 if bits == 8 else ffn.sparse_ffn_forward_q4
+        ffn.set_path("fused")
+        try:
+            want = f(x, gate, w["b_g"], w["W_up"], w["W_down"], act).double().cpu().numpy()
+        except mod.SFFNError as e:                 # a shape the single-token kernel does not take
+            assert e.code == 2, what
+            continue
+        n_want = int(ffn.last_active().numel())
+        ffn.set_path("auto")
+        n0 = ffn.launch_count()
+        y = f(x, gate, w["b_g"], w["W_up"], w["W_down"], act)
+        assert B <= 8 or ffn.launch_count() - n0 < B, what   # the batch kernels ran, not one launch per token
+        # the tensor-core path rounds h and the LoPA vector to bf16 pairs: a looser band than fp32 against fp32
+        assert_y_close(y, want, rel_l2=1e-2, max_abs=2e-2, what=what)
+        assert abs(int(ffn.last_active().numel()) - n_want) <= max(4, n_want // 200), what
+        y2 = f(x, gate, w["b_g"], w["W_up"], w["W_down"], act)
+        assert torch.equal(y, y2), f"{what} repeat"
+        torch.cuda.synchronize()
+        assert ffn.device_status() == 0, f"{what}: status words {ffn.status_words()}"
