@@ -533,7 +533,7 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
   const bool lopa_gate = g->kind == SFFN_GATE_LOPA;
   const int gate_k = lopa_gate ? g->r : h->D;
   const int chunk = B < kMaxMmaTokens ? B : kMaxMmaTokens;
-  // a batch the tensor-core kernels can take (bf16 rows; more than 64 tokens: in chunks of 64)
+  // a batch the tensor-core kernels can take (bf16 tokens; bf16, int8 or int4 rows; more than 64 tokens: in chunks of 64)
   const int gate_cols_chunk = lopa_gate ? 2 * chunk : chunk;
   // rows of weight codes: the tcgen05 kernels only (they expand the codes to bf16 on the way to the tensor cores)
   const bool q_tensor_ok = !q8 || (h->path != SFFN_PATH_MMA_SYNC && sffn::umma_rows_supported(gate_k, gate_cols_chunk) &&
@@ -541,9 +541,10 @@ int run(sffn_handle* h, const void* x, int B, const sffn_gate* g, const float* b
                                    (!lopa_gate || sffn::umma_rows_supported(h->D, chunk)));
   const bool tensor_batch = h->dtype == SFFN_BF16 && B >= 2 && h->path != SFFN_PATH_GENERAL && q_tensor_ok &&
                             h->path != SFFN_PATH_FUSED && sffn::batched_mma_supported(h->D, gate_k, gate_cols_chunk);
-  // Any other batch: the single-token kernel once per token, where it serves the shape.  The tensor-core batch kernels
-  // take bf16 operands only, and the CUDA-core batch kernels are slower than B single-token calls (int8, 4096 x 14336,
-  // B = 16: 1.66 ms against 0.33 ms; bf16 rows of 4000 elements: 1.03 ms against 0.46 ms; fp32: 0.86 against 0.77 ms).
+  // Any other batch (fp32 operands, a row width the tensor-core kernels do not tile, SFFN_PATH_FUSED): the single-token
+  // kernel once per token, where it serves the shape.  The CUDA-core batch kernels are slower than B single-token calls
+  // (int8, 4096 x 14336, B = 16: 1.66 ms against 0.33 ms; bf16 rows of 4000 elements: 1.03 ms against 0.46 ms; fp32:
+  // 0.86 against 0.77 ms).
   // The fired flags of the tokens are OR-ed: the list is the batch's union.
   if (B > 1 && !tensor_batch && h->path != SFFN_PATH_GENERAL && h->path != SFFN_PATH_MMA_SYNC &&
       sffn::fused_supported(wkind, h->D, h->H, 1, g, h->sm_count)) {
