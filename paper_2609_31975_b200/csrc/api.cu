@@ -25,7 +25,7 @@ constexpr int kMaxMmaTokens = 64;    // tokens per pass of the batched tensor-co
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
-  size_t status, act, flag, idx, v, n, partial, xstage, ystage, fused, hmT, x2, union_flag, total;
+  size_t status, act, flag, idx, v, n, partial, xstage, ystage, fused, hmT, x2, union_flag, xlimb, nlimb, tscale, total;
   int hm_stride;
 };
 
@@ -54,6 +54,11 @@ Layout make_layout(int D, int H, int r_max, int B_max, int dtype) {
   L.hmT = take((size_t)(B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * L.hm_stride * 2);
   L.x2 = take((size_t)2 * (B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens) * (r_max > 0 ? r_max : 1) * 2);
   L.union_flag = take((size_t)H + 256);  // fired flags accumulated over the chunks of a batch of more than 64 tokens
+  // int8 rows on the tensor cores: the tokens (and the LoPA vector) as four int8 limbs each, and their scales
+  const size_t bt = B_max < kMaxMmaTokens ? B_max : kMaxMmaTokens;
+  L.xlimb = take(B_max > 1 && dtype == SFFN_BF16 ? 4 * bt * D : 0);
+  L.nlimb = take(B_max > 1 && dtype == SFFN_BF16 ? 4 * bt * (size_t)(r_max > 0 ? r_max : 1) : 0);
+  L.tscale = take(2 * kMaxMmaTokens * 4);
   L.total = off;
   return L;
 }
@@ -263,6 +268,19 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
   const int D = h->D, H = h->H;
   if (q8 && !umma) return SFFN_ERR_UNSUPPORTED;  // rows of weight codes: tcgen05 kernels only
   const int wq = q8 ? qbits : 0;
+  // int8 rows whose K blocks are whole (128 codes): multiplied as int8 against the tokens' int8 limbs, nothing to expand
+  // (the down projection keeps the expansion: its B operand, Hm, has no scale known before the whole of it exists)
+  const bool native = q8 && qbits == 8 && B <= kMaxMmaTokens && umma_rows_native_i8_supported(D, B) &&
+                      umma_rows_native_i8_supported(g->kind == SFFN_GATE_LOPA ? g->r : D, B);
+  const int wq_rows = native ? 1 : wq;
+  void* xlimb = h->ws + h->L.xlimb;
+  void* nlimb = h->ws + h->L.nlimb;
+  float* xscale = h->at<float>(h->L.tscale);
+  float* nscale = xscale + kMaxMmaTokens;
+  if (native) {
+    SFFN_CUDA(launch_token_limbs(x, B, D, D, xlimb, xscale, s));
+    ++h->launches;
+  }
   float* actbuf = h->at<float>(h->L.act);
   uint8_t* flag = h->at<uint8_t>(h->L.flag);
   int32_t* idx = h->at<int32_t>(h->L.idx);
@@ -279,11 +297,12 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
       const int nb = B - b0 < kMaxMmaTokens ? B - b0 : kMaxMmaTokens;
       UmmaRowsParams p{};
       p.W = g->V; p.R = g->r; p.K = D;
-      p.qbits = wq; p.w_scale = q8 ? q8->s_V : nullptr;
+      p.qbits = wq_rows; p.w_scale = q8 ? q8->s_V : nullptr;
       p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
+      if (native) { p.X = xlimb; p.ncols_valid = 4 * nb; p.tok_scale = xscale; }
       p.act = kUmmaActIdentity; p.a_out = vbuf + (size_t)b0 * rs; p.a_stride = rs;
       p.status = h->at<int32_t>(h->L.status);
-      SFFN_CUDA(launch_umma_rows(false, p, nb, h->sm_count, s));
+      SFFN_CUDA(launch_umma_rows(false, p, native ? 4 * nb : nb, h->sm_count, s));
       ++h->launches;
     }
   } else if (lopa) {  // v = V x on the CUDA-core row kernel (r rows only), then RMSNorm
@@ -317,13 +336,21 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     if (umma) {
       UmmaRowsParams p{};
       p.R = H; p.B = nb; p.b_g = b_g; p.act = act; p.status = h->at<int32_t>(h->L.status);
-      p.qbits = wq; p.w_scale = q8 ? q8->s_gate : nullptr;
+      p.qbits = wq_rows; p.w_scale = q8 ? q8->s_gate : nullptr;
       p.xtok = xtok; p.xtok_stride = D;
       p.a_out = actbuf + (size_t)b0 * H; p.a_stride = H;
       p.flag = (dense || own_list) ? nullptr : flag;
       p.words_out = own_list ? words : nullptr;
       int cols = nb;
-      if (lopa) {
+      if (lopa && native) {
+        // RMSNorm (or none) and the split into int8 limbs in one launch
+        SFFN_CUDA(launch_rmsnorm_limbs(vbuf + (size_t)b0 * rs, nb, g->r, rs, g->rms_gain, g->rms_eps,
+                                       g->use_rmsnorm != 0, nlimb, nscale, s));
+        ++h->launches;
+        p.W = g->U; p.K = g->r; p.X = nlimb; p.x_stride = g->r; p.tok_scale = nscale;
+        p.g_idx = g->g_idx; p.g_sign = g->g_sign;
+        cols = 4 * nb;
+      } else if (lopa) {
         // RMSNorm (or none) and the split into bf16 pairs in one launch
         SFFN_CUDA(launch_rmsnorm_split(vbuf + (size_t)b0 * rs, nb, g->r, rs, g->rms_gain, g->rms_eps,
                                        g->use_rmsnorm != 0, x2, s));
@@ -331,6 +358,9 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
         p.W = g->U; p.K = g->r; p.X = x2; p.x_stride = g->r; p.split_cols = 1;
         p.g_idx = g->g_idx; p.g_sign = g->g_sign;
         cols = 2 * nb;
+      } else if (native) {
+        p.W = g->W_g; p.K = D; p.X = xlimb; p.x_stride = D; p.tok_scale = xscale;
+        cols = 4 * nb;
       } else {
         p.W = g->W_g; p.K = D; p.X = xtok; p.x_stride = D;
       }
@@ -376,7 +406,7 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
     if (umma) {
       UmmaRowsParams p{};
       p.W = W_up; p.R = H; p.K = D;
-      p.qbits = wq; p.w_scale = q8 ? q8->s_up : nullptr; p.out_scale = q8 ? q8->s_down : nullptr;
+      p.qbits = wq_rows; p.w_scale = q8 ? q8->s_up : nullptr; p.out_scale = q8 ? q8->s_down : nullptr;
       if (own_list) {
         p.words_in = words; p.n_words = 4 * gate_tiles; p.gate_tile_rows = gate_tile_rows;
         p.gate_rows_per_word = gate_tile_rows <= 64 ? 16 : 32;
@@ -385,10 +415,11 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
         p.idx = lidx; p.count = lcount;
       }
       p.X = xb + (size_t)b0 * D * 2; p.x_stride = D; p.ncols_valid = nb; p.B = nb;
+      if (native) { p.X = xlimb; p.ncols_valid = 4 * nb; p.tok_scale = xscale; }
       p.a = actbuf + (size_t)b0 * H; p.a_stride = H;
       p.hmT = hmT; p.hm_stride = h->L.hm_stride; p.status = h->at<int32_t>(h->L.status);
       p.act_up = h->act_up;
-      SFFN_CUDA(launch_umma_rows(true, p, nb, h->sm_count, s));
+      SFFN_CUDA(launch_umma_rows(true, p, native ? 4 * nb : nb, h->sm_count, s));
     } else {
       RowsMmaParams p{};
       p.status = h->at<int32_t>(h->L.status);

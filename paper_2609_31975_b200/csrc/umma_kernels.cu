@@ -142,6 +142,18 @@ __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t b
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same for int8 operands (D int32, A and B signed 8-bit, both K-major; one MMA covers K = 32).
+__device__ __forceinline__ uint32_t make_idesc_i8(int n, int m = kTileRows) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -166,6 +178,25 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, int nacc, int stride, f
     float a = __uint_as_float(r0[i]);
     if (nacc >= 2) a += __uint_as_float(r1[i]);
     if (nacc == 4) a += __uint_as_float(r2[i]) + __uint_as_float(r3[i]);
+    v[i] = a;
+  }
+}
+
+// The same for int32 accumulators (summed exactly).
+__device__ __forceinline__ void tmem_ld8_int(uint32_t taddr, int nacc, int stride, int* v) {
+  uint32_t r0[8], r1[8], r2[8], r3[8];
+  tmem_ld8_raw(taddr, r0);
+  if (nacc >= 2) tmem_ld8_raw(taddr + stride, r1);
+  if (nacc == 4) {
+    tmem_ld8_raw(taddr + 2 * stride, r2);
+    tmem_ld8_raw(taddr + 3 * stride, r3);
+  }
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    int a = (int)r0[i];
+    if (nacc >= 2) a += (int)r1[i];
+    if (nacc == 4) a += (int)r2[i] + (int)r3[i];
     v[i] = a;
   }
 }
@@ -288,7 +319,7 @@ struct WalkMap<false> {
 enum RowsMode { kGate = 0, kUp = 1, kUpMayWalk = 2 };  // kUpMayWalk: wide batches, see walk_all below
 
 template <int MODE, int QB>
-__global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1) umma_rows_kernel(const UmmaRowsParams p,
+__global__ void __launch_bounds__(kThreadsRows + ((QB == 8 || QB == 4) ? 32 * kExpandWarps : 0), 1) umma_rows_kernel(const UmmaRowsParams p,
                                                                   const __grid_constant__ CUtensorMap map_w,
                                                                   const __grid_constant__ CUtensorMap map_x,
                                                                   const __grid_constant__ WalkMap<MODE == kUpMayWalk> map_t) {
@@ -310,19 +341,25 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
   const uint32_t ready = smem_u32(bars + 2 * kMaxStages + 4);  // quantised rows: slot t of the bf16 ring is written ...
   const uint32_t afree = ready + 8 * kExpandSlots;             // ... and has been read by its MMAs
   constexpr int kRawRow = 8 * QB;                              // bytes of 64 codes
+  // QB = 1: int8 rows and the tokens as int8 limbs (four per token, see token_limbs_kernel) go straight into
+  // kind::i8 MMAs with int32 accumulators: nothing to expand, a K block is 128 codes.  QB = 8 / 4: codes expanded
+  // to bf16 by four more warps.
+  constexpr bool kNat = QB == 1, kExp = QB == 8 || QB == 4, kQ = QB != 0;
+  constexpr int kAtomElems = kNat ? 128 : kAtomK;              // elements of one 128-byte swizzle row
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int kblocks = p.K / kAtomK;
+  const int kblocks = p.K / kAtomElems;
 
   // Set-up that needs nothing from earlier kernels runs while the predecessor in the stream finishes.
   pdl_launch_dependents();
-  const uint32_t tmem_cols = tmem_cols_for(kMaxIssuers * npad);
+  const int max_acc = npad > 128 ? 2 : kMaxIssuers;  // 512 TMEM columns: wide token blocks leave room for two accumulators
+  const uint32_t tmem_cols = tmem_cols_for(max_acc * npad);
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(full + 8 * s, 1);  // the producer's expect_tx arrive; the copies complete the bytes
       mbar_init(empty + 8 * s, 1);
     }
-    if (QB)
+    if (kExp)
       for (int t = 0; t < kExpandSlots; ++t) {
         mbar_init(ready + 8 * t, kExpandWarps / 2);
         mbar_init(afree + 8 * t, 1);
@@ -468,16 +505,17 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
   // copies bring (token rows, then the codes), and the expanded bf16 blocks have a short ring of their own (stage
   // `it` uses slot it mod 4 of it): the codes in flight, not the expanded blocks, are what has to cover the memory
   // latency.
-  const int b_off = QB ? 0 : atoms * a_block_bytes;           // token rows within a ring slot
-  const int w_off = QB ? atoms * b_block_bytes : 0;           // weights (as copied) within a ring slot
-  int stage_bytes = QB ? atoms * (b_block_bytes + raw_block_bytes) : max(atoms * (a_block_bytes + b_block_bytes), a_bytes);
+  const int b_off = kExp ? 0 : atoms * a_block_bytes;           // token rows within a ring slot
+  const int w_off = kExp ? atoms * b_block_bytes : 0;           // weights (as copied) within a ring slot
+  int stage_bytes = kExp ? atoms * (b_block_bytes + raw_block_bytes) : max(atoms * (a_block_bytes + b_block_bytes), a_bytes);
   stage_bytes = (stage_bytes + 1023) & ~1023;
-  const uint32_t ring0 = stage0 + (QB ? kExpandSlots * a_bytes : 0);
-  int S = (p.ring_bytes - (QB ? kExpandSlots * a_bytes : 0)) / stage_bytes;
-  S = S > (QB ? kMaxStages : kMaxStagesBf16) ? (QB ? kMaxStages : kMaxStagesBf16) : S;
+  const uint32_t ring0 = stage0 + (kExp ? kExpandSlots * a_bytes : 0);
+  int S = (p.ring_bytes - (kExp ? kExpandSlots * a_bytes : 0)) / stage_bytes;
+  S = S > (kExp ? kMaxStages : kMaxStagesBf16) ? (kExp ? kMaxStages : kMaxStagesBf16) : S;
   // four issuers when the ring divides evenly among them, otherwise two (slot mod issuers = owner)
-  const int issuers = (S >= 8 && S % 4 == 0) ? 4 : QB && S >= 4 ? 4 : 2;
-  S &= (QB && S >= 4) ? ~3 : ~1;
+  int issuers = (S >= 8 && S % 4 == 0) ? 4 : kExp && S >= 4 ? 4 : 2;
+  S &= (kExp && S >= 4) ? ~3 : ~1;
+  issuers = issuers > max_acc ? max_acc : issuers;
   const int kstages = (kblocks + atoms - 1) / atoms;
   // accumulator row that this thread's TMEM lane holds (-1: none); the same for every warp of a lane quarter
   const int row_thr = m64 ? (lane < 16 ? (warp & 3) * 16 + lane : -1) : (warp & 3) * 32 + lane;
@@ -513,8 +551,8 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
     // everything that does not depend on the accumulator is fetched before the wait
     if (MODE == kGate) pdl_wait();  // before the first read of a buffer an earlier kernel may write, and the first store
     float bias = 0.f, sg = 1.f;
-    const float sc = (QB && row_ok && p.w_scale) ? p.w_scale[j] : 1.f;           // scale of the weight row
-    const float osc = (QB && UP && row_ok && p.out_scale) ? p.out_scale[j] : 1.f;  // scale of the down row, folded into Hm
+    const float sc = (kQ && row_ok && p.w_scale) ? p.w_scale[j] : 1.f;           // scale of the weight row
+    const float osc = (kQ && UP && row_ok && p.out_scale) ? p.out_scale[j] : 1.f;  // scale of the down row, folded into Hm
     int gi = -1;
     float pre[16];  // union rows: the gate values of this thread's first two column groups
     if (UP) {
@@ -542,6 +580,36 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
     }
     if (!okw) return false;
     tc_fence_after();
+    if constexpr (kNat) {
+      // int32 accumulators, four columns per token (its limbs, most significant first, 7 bits apart):
+      // value = token scale * row scale * (i0 + i1 / 128 + i2 / 128^2 + i3 / 128^3)
+      __nv_bfloat16* hm = static_cast<__nv_bfloat16*>(p.hmT) + li;
+      float* arow = p.a_out + j;
+      const __nv_bfloat16* xg = static_cast<const __nv_bfloat16*>(p.xtok) + (gi >= 0 ? gi : 0);
+      for (int c0 = 8 * part; c0 < npad; c0 += 8 * nparts) {
+        int iv[8];
+        tmem_ld8_int(taddr + c0, nacc, npad, iv);
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int b = c0 / 4 + q;
+          if (row_ok && b < B) {
+            const float val = p.tok_scale[b] * sc *
+                              (((float)iv[4 * q] + (float)iv[4 * q + 1] * 0.0078125f) +
+                               ((float)iv[4 * q + 2] * 6.103515625e-05f + (float)iv[4 * q + 3] * 4.76837158203125e-07f));
+            if (UP) {
+              const float av = p.a[(size_t)b * p.a_stride + j];
+              hm[(size_t)b * p.hm_stride] = __float2bfloat16(av * activation(p.act_up, val) * osc);
+            } else {
+              float z = val + bias;
+              if (gi >= 0) z += sg * __bfloat162float(xg[(size_t)b * p.xtok_stride]);
+              fired |= z > 0.f;
+              arow[(size_t)b * p.a_stride] = activation(p.act, z);
+            }
+          }
+        }
+      }
+      return true;
+    }
     if (UP) {
       __nv_bfloat16* hm = static_cast<__nv_bfloat16*>(p.hmT) + li;
       const float* arow = p.a + j;
@@ -558,7 +626,7 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
         for (int q = 0; q < 8; ++q)
           if (row_ok && c0 + q < B)
             hm[(size_t)(c0 + q) * p.hm_stride] =
-                __float2bfloat16(QB ? av[q] * activation(act_up, v[q] * sc) * osc : av[q] * activation(act_up, v[q]));
+                __float2bfloat16(kQ ? av[q] * activation(act_up, v[q] * sc) * osc : av[q] * activation(act_up, v[q]));
       }
     } else {
       const int act = p.act;
@@ -572,7 +640,7 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
           for (int q = 0; q < 4; ++q) {
             const int b = c0 / 2 + q;
             if (row_ok && b < B) {
-              float z = QB ? (v[2 * q] + v[2 * q + 1]) * sc + bias : v[2 * q] + v[2 * q + 1] + bias;
+              float z = kQ ? (v[2 * q] + v[2 * q + 1]) * sc + bias : v[2 * q] + v[2 * q + 1] + bias;
               if (gi >= 0) z += sg * __bfloat162float(xg[(size_t)b * p.xtok_stride]);
               fired |= z > 0.f;
               arow[(size_t)b * p.a_stride] = activation(act, z);
@@ -587,7 +655,7 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
           for (int q = 0; q < 8; ++q) {
             const int b = c0 + q;
             if (row_ok && b < B) {
-              float z = QB ? v[q] * sc + bias : v[q] + bias;
+              float z = kQ ? v[q] * sc + bias : v[q] + bias;
               if (gi >= 0) z += sg * __bfloat162float(xg[(size_t)b * p.xtok_stride]);
               fired |= z > 0.f;
               arow[(size_t)b * p.a_stride] = activation(act, z);
@@ -621,7 +689,7 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
         if ((s & (kProducerWarps - 1)) != warp) continue;
         const int tile = blockIdx.x + tl * gridDim.x;
         const int na = min(atoms, kblocks - kb * atoms);
-        const uint32_t tx_bytes = QB ? (uint32_t)(na * (tile_rows * kRawRow + npad * 128)) : (uint32_t)(na * (tile_rows + npad)) * 128;
+        const uint32_t tx_bytes = kExp ? (uint32_t)(na * (tile_rows * kRawRow + npad * 128)) : (uint32_t)(na * (tile_rows + npad)) * 128;
         if (UP && !walk_all && tl != rows_of) {
           rows_of = tl;
 #pragma unroll
@@ -644,11 +712,11 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
         }
         const uint32_t abase = ring0 + s * stage_bytes;
         for (int a = 0; a < na; ++a) {
-          const int k0 = (kb * atoms + a) * kAtomK;
+          const int k0 = (kb * atoms + a) * kAtomElems;
           // where the weight block lands, the byte column it starts at, and the bytes of one landed row
-          const uint32_t wdst = abase + w_off + a * (QB ? raw_block_bytes : a_block_bytes);
-          const int wc0 = QB ? k0 * QB / 8 : k0;
-          const int wrow = QB ? kRawRow : 128;
+          const uint32_t wdst = abase + w_off + a * (kExp ? raw_block_bytes : a_block_bytes);
+          const int wc0 = kExp ? k0 * QB / 8 : k0;
+          const int wrow = kExp ? kRawRow : 128;
           if (with_w && !(MODE == kGate && blockIdx.x == 0 && it == p.drop_stage)) {  // test hook: a copy that never comes
             if (UP && !walk_all) {
               if (lane * 4 < tile_rows)
@@ -674,7 +742,7 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
     } else {
       produce(0, total, true, true);
     }
-  } else if (QB && warp >= kThreadsRows / 32) {
+  } else if (kExp && warp >= kThreadsRows / 32) {
     // ======================= expanders (quantised rows): codes -> bf16 block of the slot ==========
     // Two pairs of warps; a pair takes the slots of its parity (S is even), in the producers' order, so it meets
     // every phase of its slots and cannot fall two phases behind; while one pair waits the other one converts.
@@ -695,7 +763,7 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
       const uint32_t src = ring0 + s * stage_bytes + w_off, dst = stage0 + t * a_bytes;
       const int na = min(atoms, kblocks - kb * atoms);
       for (int a = 0; a < na; ++a)
-        expand_block<QB ? QB : 8>(src + a * raw_block_bytes, dst + a * a_block_bytes, tile_rows, et, 16 * kExpandWarps);
+        expand_block<kExp ? QB : 8>(src + a * raw_block_bytes, dst + a * a_block_bytes, tile_rows, et, 16 * kExpandWarps);
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive(ready + 8 * t);
@@ -704,7 +772,7 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
     // ======================= MMA issuers =======================================================
     const int m = warp - 8;
     if (lane == 0 && m < nacc) {
-      const uint32_t idesc = make_idesc(npad, mrows);
+      const uint32_t idesc = kNat ? make_idesc_i8(npad, mrows) : make_idesc(npad, mrows);
       const uint32_t acc = tmem_base + m * npad;
       int tcount = 0;
       bool ok = true;
@@ -717,21 +785,27 @@ __global__ void __launch_bounds__(kThreadsRows + (QB ? 32 * kExpandWarps : 0), 1
           if (s == S) { s = 0; ph ^= 1; }
           if ((s & (nacc - 1)) != m) continue;   // another issuer's slot
           const int t = (it0 + kb) % kExpandSlots;  // quantised rows: slot of the bf16 ring
-          if (QB ? !mbar_wait(ready + 8 * t, ((it0 + kb) / kExpandSlots) & 1, abort_flag, p.status, p.wait_cycles)
+          if (kExp ? !mbar_wait(ready + 8 * t, ((it0 + kb) / kExpandSlots) & 1, abort_flag, p.status, p.wait_cycles)
                  : !mbar_wait(full + 8 * s, ph, abort_flag, p.status, p.wait_cycles)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sbase = ring0 + s * stage_bytes;
-          const uint32_t wbase = QB ? stage0 + t * a_bytes : sbase;
+          const uint32_t wbase = kExp ? stage0 + t * a_bytes : sbase;
           const int na = min(atoms, kblocks - kb * atoms);
           for (int a = 0; a < na; ++a) {
             const uint64_t adesc = make_desc(wbase + a * a_block_bytes);
             const uint64_t bdesc = make_desc(sbase + b_off + a * b_block_bytes);
-            umma(acc, adesc, bdesc, idesc, (kb >= nacc || a > 0) ? 1u : 0u);
+            if (kNat) {
+              umma_i8(acc, adesc, bdesc, idesc, (kb >= nacc || a > 0) ? 1u : 0u);
 #pragma unroll
-            for (int k = 1; k < kAtomK / 16; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+              for (int k = 1; k < 4; ++k) umma_i8(acc, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+            } else {
+              umma(acc, adesc, bdesc, idesc, (kb >= nacc || a > 0) ? 1u : 0u);
+#pragma unroll
+              for (int k = 1; k < kAtomK / 16; ++k) umma(acc, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+            }
           }
           umma_commit(empty + 8 * s);   // slot free once these MMAs have read it
-          if (QB) umma_commit(afree + 8 * t);
+          if (kExp) umma_commit(afree + 8 * t);
         }
         if (ok) umma_commit(acc_full);  // this issuer's accumulator is complete
       }
@@ -1027,6 +1101,70 @@ __global__ void __launch_bounds__(256) rmsnorm_split_kernel(const float* v, int 
   }
 }
 
+// Tokens as int8 limbs for the kind::i8 MMAs: t[k] = scale * (q0 + q1 / 128 + q2 / 128^2 + q3 / 128^3) up to
+// scale * 2^-22, with scale = max |t| / 127, |q0| <= 127 and the other limbs <= 64 in magnitude.  Row 4 b + l of
+// `limbs` holds limb l of token b.  One CTA per token; `val(k)` yields the token's entries.
+template <typename F>
+__device__ __forceinline__ void write_limbs(F val, int K, int8_t* limbs, float* scale_out, float* red) {
+  float m = 0.f;
+  for (int k = threadIdx.x; k < K; k += blockDim.x) m = fmaxf(m, fabsf(val(k)));
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+  __syncthreads();  // `red` may still be read by the caller
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  float mx = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) mx = fmaxf(mx, red[w]);
+  const float scale = mx > 0.f ? mx / 127.f : 1.f;
+  if (threadIdx.x == 0) *scale_out = scale;
+  const float inv = 1.f / scale;
+  for (int k = threadIdx.x; k < K; k += blockDim.x) {
+    float t = val(k) * inv;
+    t = fminf(fmaxf(t, -127.f), 127.f);
+#pragma unroll
+    for (int l = 0; l < 4; ++l) {
+      const float q = rintf(t);
+      limbs[(size_t)l * K + k] = (int8_t)(int)q;
+      t = (t - q) * 128.f;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) token_limbs_kernel(const __nv_bfloat16* x, int K, int x_stride, int8_t* limbs,
+                                                          float* scale) {
+  __shared__ float red[8];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.x;
+  const __nv_bfloat16* xb = x + (size_t)b * x_stride;
+  write_limbs([&](int k) { return __bfloat162float(xb[k]); }, K, limbs + (size_t)4 * b * K, scale + b, red);
+}
+
+// LoPA gate with int8 rows: n = RMSNorm(v) (or v itself) as limbs.  One CTA per token.
+__global__ void __launch_bounds__(256) rmsnorm_limbs_kernel(const float* v, int r, int v_stride, const float* gain,
+                                                            float eps, int use_rms, int8_t* limbs, float* scale) {
+  __shared__ float red[8];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.x;
+  const float* vb = v + (size_t)b * v_stride;
+  float inv = 1.f;
+  if (use_rms) {
+    float ss = 0.f;
+    for (int k = threadIdx.x; k < r; k += blockDim.x) ss = fmaf(vb[k], vb[k], ss);
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    inv = rsqrtf(tot / (float)r + eps);
+  }
+  write_limbs([&](int k) { return use_rms ? (gain ? gain[k] : 1.f) * vb[k] * inv : vb[k]; }, r, limbs + (size_t)4 * b * r,
+              scale + b, red);
+}
+
 }  // namespace
 
 
@@ -1046,6 +1184,8 @@ bool umma_own_list_supported(int R, int sm_count) {
 bool umma_may_walk(int B) { return B >= kWalkMinTokens; }
 
 bool umma_rows_supported(int K, int cols) { return K % kAtomK == 0 && K >= kAtomK && cols >= 1 && cols <= 128; }
+// int8 rows multiplied as int8 (tokens as four int8 limbs each): K blocks of 128 codes, up to 64 tokens.
+bool umma_rows_native_i8_supported(int K, int tokens) { return K % 128 == 0 && K >= 128 && tokens >= 1 && tokens <= 64; }
 
 namespace {
 
@@ -1092,16 +1232,36 @@ bool make_map_codes(CUtensorMap* m, const void* base, int K, int rows, size_t pi
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// int8 matrix [rows, K] (row pitch in bytes), read in boxes of 128 codes x box_rows rows, 128-byte swizzle: the operand
+// layout of the kind::i8 MMAs.
+bool make_map_i8(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_bytes, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)pitch_bytes};
+  const cuuint32_t box[2] = {128u, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_weight_map(CUtensorMap* m, const void* base, int K, int rows, int box_rows, int qbits) {
-  return qbits ? make_map_codes(m, base, K, rows, (size_t)K * qbits / 8, box_rows, qbits)
-               : make_map(m, base, K, rows, (size_t)K, box_rows);
+  return qbits == 1 ? make_map_i8(m, base, K, rows, (size_t)K, box_rows)
+         : qbits    ? make_map_codes(m, base, K, rows, (size_t)K * qbits / 8, box_rows, qbits)
+                    : make_map(m, base, K, rows, (size_t)K, box_rows);
 }
 
 template <int MODE, typename Map>
 cudaError_t launch_rows_mode(const UmmaRowsParams& p, int grid, size_t smem, cudaStream_t s, const CUtensorMap& map_w,
                              const CUtensorMap& map_x, const Map& map_t) {
-  static unsigned long long configured[3] = {0, 0, 0};
+  static unsigned long long configured[4] = {0, 0, 0, 0};
   cudaError_t e;
+  if (p.qbits == 1) {
+    auto k = umma_rows_kernel<MODE, 1>;
+    if ((e = allow_dynamic_smem(k, 227 * 1024, configured[3])) != cudaSuccess) return e;
+    return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, map_t);
+  }
   if (p.qbits == 8) {
     auto k = umma_rows_kernel<MODE, 8>;
     if ((e = allow_dynamic_smem(k, 227 * 1024, configured[0])) != cudaSuccess) return e;
@@ -1128,11 +1288,14 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
   const size_t smem = 226 * 1024;
   p.ring_bytes = (int)smem - 1024 - kHeaderBytes;
   alignas(64) CUtensorMap map_w, map_x;
-  if (p.qbits != 0 && p.qbits != 8 && p.qbits != 4) return cudaErrorInvalidValue;
+  if (p.qbits != 0 && p.qbits != 8 && p.qbits != 4 && p.qbits != 1) return cudaErrorInvalidValue;
+  if (p.qbits == 1 && (p.K % 128 || p.npad > 256 || !p.tok_scale)) return cudaErrorInvalidValue;
   // weights: all R rows; boxes of one tile's rows for the gate, single-row boxes for the gather
   if (!make_weight_map(&map_w, p.W, p.K, p.R, up ? 1 : tile_rows_for(p.R, grid), p.qbits)) return cudaErrorNotSupported;
   // tokens: only the rows that exist; the box covers npad rows and the rest reads as zero
-  if (!make_map(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)) return cudaErrorNotSupported;
+  if (p.qbits == 1 ? !make_map_i8(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)
+                   : !make_map(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad))
+    return cudaErrorNotSupported;
   if (!up) return launch_rows_mode<kGate>(p, grid, smem, s, map_w, map_x, WalkMap<false>{});
   if (p.walk_all && umma_may_walk(p.B)) {
     // wide batches: the union may cover most rows; the kernel then walks every row with tiled boxes of the tile
@@ -1186,6 +1349,17 @@ cudaError_t launch_umma_down(UmmaDownParams p, cudaStream_t s) {
   return p.qbits == 8   ? launch_down_q<8>(p, g, smem, s, map_wg, map_wt, map_hm)
          : p.qbits == 4 ? launch_down_q<4>(p, g, smem, s, map_wg, map_wt, map_hm)
                         : launch_down_q<0>(p, g, smem, s, map_wg, map_wt, map_hm);
+}
+
+cudaError_t launch_token_limbs(const void* x, int B, int K, int x_stride, void* limbs, float* scale, cudaStream_t s) {
+  return launch_pdl(token_limbs_kernel, dim3(B), dim3(256), 0, s, static_cast<const __nv_bfloat16*>(x), K, x_stride,
+                    static_cast<int8_t*>(limbs), scale);
+}
+
+cudaError_t launch_rmsnorm_limbs(const float* v, int B, int r, int v_stride, const float* gain, float eps, bool use_rms,
+                                 void* limbs, float* scale, cudaStream_t s) {
+  return launch_pdl(rmsnorm_limbs_kernel, dim3(B), dim3(256), 0, s, v, r, v_stride, gain, eps, use_rms ? 1 : 0,
+                    static_cast<int8_t*>(limbs), scale);
 }
 
 cudaError_t launch_rmsnorm_split(const float* v, int B, int r, int v_stride, const float* gain, float eps,

@@ -12,7 +12,10 @@ constexpr int kUmmaActIdentity = 3;
 struct UmmaRowsParams {
   const void* W;         // [*, K] bf16 (or int8 / packed int4 codes, see qbits), rows selected by idx (or 0..R-1)
   int R, K;
-  int qbits;             // 0: bf16 rows; 8 / 4: rows of weight codes, K * qbits / 8 bytes each
+  int qbits;             // 0: bf16 rows; 8 / 4: rows of weight codes, K * qbits / 8 bytes each, expanded to bf16 in
+                         // shared memory; 1: int8 rows multiplied as int8 -- X then holds the tokens as int8 limbs (four
+                         // rows per token, launch_token_limbs) and tok_scale their scales
+  const float* tok_scale;  // qbits = 1: scale of each token's limbs
   const float* w_scale;  // quantised rows: scale of row j of W (applied to its accumulator row), or null
   const float* out_scale;  // UP, quantised rows: scale of row j of the down matrix, folded into Hm, or null
   const int32_t* idx;    // UP: list of rows, or null
@@ -75,6 +78,12 @@ bool umma_may_walk(int B);
 bool umma_own_list_supported(int R, int sm_count);
 void umma_gate_tiling(int R, int sm_count, int* tile_rows, int* n_tiles);
 cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, cudaStream_t s);
+bool umma_rows_native_i8_supported(int K, int tokens);
+// Tokens [B][K] bf16 as four int8 limbs each ([4 B][K], most significant first, 7 bits apart) and one scale per token.
+cudaError_t launch_token_limbs(const void* x, int B, int K, int x_stride, void* limbs, float* scale, cudaStream_t s);
+// The same for the LoPA vector n = RMSNorm(v) (or v), from fp32.
+cudaError_t launch_rmsnorm_limbs(const float* v, int B, int r, int v_stride, const float* gain, float eps, bool use_rms,
+                                 void* limbs, float* scale, cudaStream_t s);
 cudaError_t launch_rmsnorm_split(const float* v, int B, int r, int v_stride, const float* gain, float eps,
                                  bool use_rms, void* x2, cudaStream_t s);
 
