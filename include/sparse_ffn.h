@@ -80,9 +80,10 @@ typedef enum { SFFN_F32 = 0, SFFN_BF16 = 1 } sffn_dtype;
 typedef enum { SFFN_GATE_STANDARD = 0, SFFN_GATE_LOPA = 1 } sffn_gate_kind;
 
 /* Which kernels serve a call.  AUTO picks the fused kernels for B = 1 when the shape allows it and the
- * tcgen05 tensor-core kernels for batches (B >= 2) of bf16 tokens with bf16, int8 or int4 rows (codes are
- * expanded to bf16 in shared memory on their way to the tensor cores; more than 64 tokens run in chunks of 64,
- * the list of fired neurons being the union over all chunks).  A batch those kernels do not take (fp32
+ * tcgen05 tensor-core kernels for batches (B >= 2) of bf16 tokens with bf16, int8 or int4 rows (int8 rows are
+ * multiplied as int8 against the tokens split into int8 limbs, or, like int4 rows, expanded to bf16 in shared
+ * memory on their way to the tensor cores; more than 64 tokens run in chunks of 64, the list of fired neurons
+ * being the union over all chunks).  A batch those kernels do not take (fp32
  * operands, a row width they do not tile) runs the fused kernel once per token with the fired flags OR-ed,
  * which is faster than the CUDA-core batch kernels; what is left goes to the general CUDA-core kernels.
  * The others force one family (SFFN_ERR_UNSUPPORTED if it cannot serve the call): GENERAL = CUDA-core
@@ -177,11 +178,13 @@ int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate
  * must have been created with SFFN_BF16.  Rows must be a multiple of 16 bytes (D and r multiples of 16).
  * Everything else (b_g, g_idx, g_sign, RMSNorm, act, y, the active list, double activation) is as in
  * sparse_ffn_forward / dense_ffn_forward.  One token runs in the fused kernel; a batch runs the tcgen05 batch
- * kernels, which expand the codes to bf16 in shared memory and apply the row scales to the accumulator rows (D and
- * r multiples of 64, D of 256; otherwise, or under SFFN_PATH_FUSED, the fused kernel once per token; the list of
- * fired neurons is the union over the tokens), or the CUDA-core batch kernels under SFFN_PATH_GENERAL
- * (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is an offline
- * step outside this library. */
+ * kernels (D and r multiples of 64, D of 256; otherwise, or under SFFN_PATH_FUSED, the fused kernel once per token; the
+ * list of fired neurons is the union over the tokens).  There the gate and up products of int8 rows are int8 x int8
+ * with int32 accumulators, each token entering as four int8 limbs and a scale (x = s (q0 + q1/128 + q2/128^2 +
+ * q3/128^3) up to 2^-22 max|x|; D and r multiples of 128), and the down product, int4 rows and other widths expand
+ * the codes to bf16 in shared memory; row scales are applied to the accumulator rows.  The CUDA-core batch kernels
+ * serve SFFN_PATH_GENERAL (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is
+ * an offline step outside this library. */
 typedef struct {
   const float* s_gate; /* [H]  row scales of W_g (STANDARD) or of U (LOPA) */
   const float* s_V;    /* [r]  row scales of V (LOPA only; may be NULL otherwise) */
