@@ -181,8 +181,9 @@ int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate
  * kernels (D and r multiples of 64, D of 256; otherwise, or under SFFN_PATH_FUSED, the fused kernel once per token; the
  * list of fired neurons is the union over the tokens).  There the gate and up products of int8 rows are int8 x int8
  * with int32 accumulators, each token entering as four int8 limbs and a scale (x = s (q0 + q1/128 + q2/128^2 +
- * q3/128^3) up to 2^-22 max|x|; D and r multiples of 128), and the down product, int4 rows and other widths expand
- * the codes to bf16 in shared memory; row scales are applied to the accumulator rows.  The CUDA-core batch kernels
+ * q3/128^3) up to 2^-22 max|x|; D and r multiples of 128; int4 rows take the same route, their nibbles expanded to
+ * int8 in shared memory), and the down product and other widths expand the codes to bf16 in shared memory; row scales
+ * are applied to the accumulator rows.  The CUDA-core batch kernels
  * serve SFFN_PATH_GENERAL (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is
  * an offline step outside this library. */
 typedef struct {

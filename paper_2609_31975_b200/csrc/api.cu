@@ -270,9 +270,10 @@ int run_batched(sffn_handle* h, const void* x, int B, const sffn_gate* g, const 
   const int wq = q8 ? qbits : 0;
   // int8 rows whose K blocks are whole (128 codes): multiplied as int8 against the tokens' int8 limbs, nothing to expand
   // (the down projection keeps the expansion: its B operand, Hm, has no scale known before the whole of it exists)
-  const bool native = q8 && qbits == 8 && B <= kMaxMmaTokens && umma_rows_native_i8_supported(D, B) &&
+  // (int4 rows: the nibbles expanded to int8 on the way, for the same MMAs)
+  const bool native = q8 && B <= kMaxMmaTokens && umma_rows_native_i8_supported(D, B) &&
                       umma_rows_native_i8_supported(g->kind == SFFN_GATE_LOPA ? g->r : D, B);
-  const int wq_rows = native ? 1 : wq;
+  const int wq_rows = native ? (qbits == 8 ? 1 : 2) : wq;
   void* xlimb = h->ws + h->L.xlimb;
   void* nlimb = h->ws + h->L.nlimb;
   float* xscale = h->at<float>(h->L.tscale);

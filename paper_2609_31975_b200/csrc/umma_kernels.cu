@@ -289,6 +289,31 @@ __device__ __forceinline__ void expand_block(uint32_t raw, uint32_t dst, int row
     }
   }
 }
+// The same for int4 codes on their way to the int8 MMA: `raw` holds [rows][128] nibbles (64 bytes a row), `dst`
+// receives [rows][128] bytes, each 16 x its code (the nibble moved to the upper half of the byte: exact, and the factor
+// goes into the row scale), in the same swizzled layout.  Thread t takes the 32 codes of quarter t % 4 of its rows: one
+// 16-byte load, two 16-byte stores; per word of eight nibbles two masks and two byte permutes.
+__device__ __forceinline__ void expand_block_q4_i8(uint32_t raw, uint32_t dst, int rows, int t, int nthr) {
+  const int c = t & 3, step = nthr >> 2;
+  for (int row = t >> 2; row < rows; row += step) {
+    uint32_t w[4], o[8];
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(raw + row * 64 + c * 16));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t ev = (w[i] << 4) & 0xf0f0f0f0u, od = w[i] & 0xf0f0f0f0u;  // even / odd columns, times 16
+      o[2 * i] = __byte_perm(ev, od, 0x5140);
+      o[2 * i + 1] = __byte_perm(ev, od, 0x7362);
+    }
+    const uint32_t drow = dst + row * 128;
+    const int sw = row & 7;
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(drow + (((2 * c) ^ sw) << 4)), "r"(o[0]), "r"(o[1]),
+                 "r"(o[2]), "r"(o[3])
+                 : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(drow + (((2 * c + 1) ^ sw) << 4)), "r"(o[4]), "r"(o[5]),
+                 "r"(o[6]), "r"(o[7])
+                 : "memory");
+  }
+}
 // Makes this thread's shared-memory stores visible to the tensor core's reads.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -319,7 +344,7 @@ struct WalkMap<false> {
 enum RowsMode { kGate = 0, kUp = 1, kUpMayWalk = 2 };  // kUpMayWalk: wide batches, see walk_all below
 
 template <int MODE, int QB>
-__global__ void __launch_bounds__(kThreadsRows + ((QB == 8 || QB == 4) ? 32 * kExpandWarps : 0), 1) umma_rows_kernel(const UmmaRowsParams p,
+__global__ void __launch_bounds__(kThreadsRows + ((QB == 8 || QB == 4 || QB == 2) ? 32 * kExpandWarps : 0), 1) umma_rows_kernel(const UmmaRowsParams p,
                                                                   const __grid_constant__ CUtensorMap map_w,
                                                                   const __grid_constant__ CUtensorMap map_x,
                                                                   const __grid_constant__ WalkMap<MODE == kUpMayWalk> map_t) {
@@ -340,11 +365,12 @@ __global__ void __launch_bounds__(kThreadsRows + ((QB == 8 || QB == 4) ? 32 * kE
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t ready = smem_u32(bars + 2 * kMaxStages + 4);  // quantised rows: slot t of the bf16 ring is written ...
   const uint32_t afree = ready + 8 * kExpandSlots;             // ... and has been read by its MMAs
-  constexpr int kRawRow = 8 * QB;                              // bytes of 64 codes
+  constexpr int kRawRow = QB == 2 ? 64 : 8 * QB;               // bytes of the codes of one K block (as copied)
   // QB = 1: int8 rows and the tokens as int8 limbs (four per token, see token_limbs_kernel) go straight into
   // kind::i8 MMAs with int32 accumulators: nothing to expand, a K block is 128 codes.  QB = 8 / 4: codes expanded
   // to bf16 by four more warps.
-  constexpr bool kNat = QB == 1, kExp = QB == 8 || QB == 4, kQ = QB != 0;
+  // QB = 2: int4 rows expanded to int8 (16 x the code, a byte each) for the same kind::i8 MMAs.
+  constexpr bool kNat = QB == 1 || QB == 2, kExp = QB == 8 || QB == 4 || QB == 2, kQ = QB != 0;
   constexpr int kAtomElems = kNat ? 128 : kAtomK;              // elements of one 128-byte swizzle row
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -551,7 +577,7 @@ __global__ void __launch_bounds__(kThreadsRows + ((QB == 8 || QB == 4) ? 32 * kE
     // everything that does not depend on the accumulator is fetched before the wait
     if (MODE == kGate) pdl_wait();  // before the first read of a buffer an earlier kernel may write, and the first store
     float bias = 0.f, sg = 1.f;
-    const float sc = (kQ && row_ok && p.w_scale) ? p.w_scale[j] : 1.f;           // scale of the weight row
+    const float sc = ((kQ && row_ok && p.w_scale) ? p.w_scale[j] : 1.f) * (QB == 2 ? 0.0625f : 1.f);  // scale of the weight row
     const float osc = (kQ && UP && row_ok && p.out_scale) ? p.out_scale[j] : 1.f;  // scale of the down row, folded into Hm
     int gi = -1;
     float pre[16];  // union rows: the gate values of this thread's first two column groups
@@ -715,7 +741,7 @@ __global__ void __launch_bounds__(kThreadsRows + ((QB == 8 || QB == 4) ? 32 * kE
           const int k0 = (kb * atoms + a) * kAtomElems;
           // where the weight block lands, the byte column it starts at, and the bytes of one landed row
           const uint32_t wdst = abase + w_off + a * (kExp ? raw_block_bytes : a_block_bytes);
-          const int wc0 = kExp ? k0 * QB / 8 : k0;
+          const int wc0 = QB == 2 ? k0 / 2 : kExp ? k0 * QB / 8 : k0;
           const int wrow = kExp ? kRawRow : 128;
           if (with_w && !(MODE == kGate && blockIdx.x == 0 && it == p.drop_stage)) {  // test hook: a copy that never comes
             if (UP && !walk_all) {
@@ -763,7 +789,8 @@ __global__ void __launch_bounds__(kThreadsRows + ((QB == 8 || QB == 4) ? 32 * kE
       const uint32_t src = ring0 + s * stage_bytes + w_off, dst = stage0 + t * a_bytes;
       const int na = min(atoms, kblocks - kb * atoms);
       for (int a = 0; a < na; ++a)
-        expand_block<kExp ? QB : 8>(src + a * raw_block_bytes, dst + a * a_block_bytes, tile_rows, et, 16 * kExpandWarps);
+        if (QB == 2) expand_block_q4_i8(src + a * raw_block_bytes, dst + a * a_block_bytes, tile_rows, et, 16 * kExpandWarps);
+        else expand_block<(QB == 8 || QB == 4) ? QB : 8>(src + a * raw_block_bytes, dst + a * a_block_bytes, tile_rows, et, 16 * kExpandWarps);
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive(ready + 8 * t);
@@ -1220,12 +1247,13 @@ bool make_map(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_el
 
 // Rows of weight codes [rows, K] (qbits 8 or 4 per code, `pitch_bytes` apart), read in boxes of 64 codes x box_rows
 // rows that land densely, without swizzle.
-bool make_map_codes(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_bytes, int box_rows, int qbits) {
+bool make_map_codes(CUtensorMap* m, const void* base, int K, int rows, size_t pitch_bytes, int box_rows, int qbits,
+                    int box_codes = kAtomK) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)K * qbits / 8, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)pitch_bytes};
-  const cuuint32_t box[2] = {(cuuint32_t)(kAtomK * qbits / 8), (cuuint32_t)box_rows};
+  const cuuint32_t box[2] = {(cuuint32_t)(box_codes * qbits / 8), (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1248,6 +1276,7 @@ bool make_map_i8(CUtensorMap* m, const void* base, int K, int rows, size_t pitch
 
 bool make_weight_map(CUtensorMap* m, const void* base, int K, int rows, int box_rows, int qbits) {
   return qbits == 1 ? make_map_i8(m, base, K, rows, (size_t)K, box_rows)
+         : qbits == 2 ? make_map_codes(m, base, K, rows, (size_t)K / 2, box_rows, 4, 128)  // int4 rows, K blocks of 128 codes
          : qbits    ? make_map_codes(m, base, K, rows, (size_t)K * qbits / 8, box_rows, qbits)
                     : make_map(m, base, K, rows, (size_t)K, box_rows);
 }
@@ -1261,6 +1290,12 @@ cudaError_t launch_rows_mode(const UmmaRowsParams& p, int grid, size_t smem, cud
     auto k = umma_rows_kernel<MODE, 1>;
     if ((e = allow_dynamic_smem(k, 227 * 1024, configured[3])) != cudaSuccess) return e;
     return launch_pdl(k, dim3(grid), dim3(kThreadsRows), smem, s, p, map_w, map_x, map_t);
+  }
+  if (p.qbits == 2) {
+    static unsigned long long configured2 = 0;
+    auto k = umma_rows_kernel<MODE, 2>;
+    if ((e = allow_dynamic_smem(k, 227 * 1024, configured2)) != cudaSuccess) return e;
+    return launch_pdl(k, dim3(grid), dim3(kThreadsRows + 32 * kExpandWarps), smem, s, p, map_w, map_x, map_t);
   }
   if (p.qbits == 8) {
     auto k = umma_rows_kernel<MODE, 8>;
@@ -1288,12 +1323,13 @@ cudaError_t launch_umma_rows(bool up, UmmaRowsParams p, int cols, int sm_count, 
   const size_t smem = 226 * 1024;
   p.ring_bytes = (int)smem - 1024 - kHeaderBytes;
   alignas(64) CUtensorMap map_w, map_x;
-  if (p.qbits != 0 && p.qbits != 8 && p.qbits != 4 && p.qbits != 1) return cudaErrorInvalidValue;
-  if (p.qbits == 1 && (p.K % 128 || p.npad > 256 || !p.tok_scale)) return cudaErrorInvalidValue;
+  if (p.qbits != 0 && p.qbits != 8 && p.qbits != 4 && p.qbits != 1 && p.qbits != 2) return cudaErrorInvalidValue;
+  const bool i8 = p.qbits == 1 || p.qbits == 2;  // kind::i8 MMAs: X holds the tokens' int8 limbs
+  if (i8 && (p.K % 128 || p.npad > 256 || !p.tok_scale)) return cudaErrorInvalidValue;
   // weights: all R rows; boxes of one tile's rows for the gate, single-row boxes for the gather
   if (!make_weight_map(&map_w, p.W, p.K, p.R, up ? 1 : tile_rows_for(p.R, grid), p.qbits)) return cudaErrorNotSupported;
   // tokens: only the rows that exist; the box covers npad rows and the rest reads as zero
-  if (p.qbits == 1 ? !make_map_i8(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)
+  if (i8 ? !make_map_i8(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad)
                    : !make_map(&map_x, p.X, p.K, p.ncols_valid, (size_t)p.x_stride, p.npad))
     return cudaErrorNotSupported;
   if (!up) return launch_rows_mode<kGate>(p, grid, smem, s, map_w, map_x, WalkMap<false>{});

@@ -14,7 +14,8 @@ struct UmmaRowsParams {
   int R, K;
   int qbits;             // 0: bf16 rows; 8 / 4: rows of weight codes, K * qbits / 8 bytes each, expanded to bf16 in
                          // shared memory; 1: int8 rows multiplied as int8 -- X then holds the tokens as int8 limbs (four
-                         // rows per token, launch_token_limbs) and tok_scale their scales
+                         // rows per token, launch_token_limbs) and tok_scale their scales; 2: the same for int4 rows,
+                         // whose nibbles are expanded to int8 (16 x the code) in shared memory
   const float* tok_scale;  // qbits = 1: scale of each token's limbs
   const float* w_scale;  // quantised rows: scale of row j of W (applied to its accumulator row), or null
   const float* out_scale;  // UP, quantised rows: scale of row j of the down matrix, folded into Hm, or null
