@@ -99,10 +99,10 @@ struct FusedParams {
 
 // Shared-memory carve-up, identical on host and device.
 struct SmemLayout {
-  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, row_params, row_scales, slot_scales, gated_bars, gated_vals, total;
+  int gate_ring, act_ring, sx, sn, aval, slot_a, red, ctl, bars, row_params, row_scales, slot_scales, gated_bars, gated_vals, xlimb, total;
   __host__ __device__ SmemLayout(int D, int K, bool lopa, int n_gate_slots, int gate_slot_bytes,
                                  int n_act_slots, int act_slot_bytes, int slab_max, bool scaled, int act_extra = 0,
-                                 bool gated = false) {
+                                 bool gated = false, bool limbs = false) {
     int off = 0;
     auto take = [&](int bytes) {
       int o = off;
@@ -125,6 +125,9 @@ struct SmemLayout {
     // up to three barriers and three values
     gated_bars = take(gated ? 3 * 2 * n_act_slots * 8 : 0);
     gated_vals = take(gated ? 3 * 2 * n_act_slots * 4 : 0);
+    // int8 rows, standard gate: the token as three int8 limbs [3][D] for the integer dot products, after 128 bytes
+    // of scratch (the staging warps' maxima, then the limbs' scale)
+    xlimb = take(limbs ? 128 + 3 * D : 0);
     total = off;
   }
 };
@@ -349,7 +352,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   // use once every gate row has been consumed -- from then on the rows of fired neurons are all that is left to
   // fetch, and how many of them are in flight sets how fast they come.
   const int NG = p.n_gate_slots, NAown = p.n_act_slots, NA = p.act_used;
-  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra, GATED);
+  // int8 rows under a standard gate: dot products in integers (dp4a) against the token split into int8 limbs
+  constexpr bool kLimbs = EPV == 16 && !LOPA;
+  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra, GATED, kLimbs);
 
   unsigned char* gate_ring = smem + L.gate_ring;
   unsigned char* act_ring = smem + L.act_ring;
@@ -379,6 +384,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   float* slot_su = reinterpret_cast<float*>(smem + L.slot_scales);
   float* slot_sd = slot_su + NA;
   float* red = reinterpret_cast<float*>(smem + L.red);
+  float* xl_scratch = reinterpret_cast<float*>(smem + L.xlimb);          // [0..15] staging warps' max |x|, [16] limb scale
+  const uint4* xl = reinterpret_cast<const uint4*>(smem + L.xlimb + 128);  // limb l of chunk c: xl[l * nvecD + c]
   volatile int* ctl = reinterpret_cast<volatile int*>(smem + L.ctl);
   const uint32_t bars = smem_u32(smem + L.bars);
   const uint32_t full_gate = bars, empty_gate = bars + 8 * NG;
@@ -514,6 +521,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const uint32_t ep = (LOPA || warp >= kFirstGateWarp) ? __ldcg(p.epoch_word) + 1u : 0u;
   for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) row_state[i] = 0xffffffffu;
   constexpr int XEPV = Elem<X>::kPerVec;  // token elements per 16 bytes (the weights' EPV unless those are int8)
+  float xmax = 0.f;
   for (int cx = tid - kStageBase; cx < D / XEPV; cx += kStageThreads) {
     float f[XEPV];
     Elem<X>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + cx), f);
@@ -522,6 +530,47 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       const int k0 = cx * XEPV + 4 * g4;  // first of four consecutive elements: quarter (k0 % EPV) / 4 of chunk k0 / EPV
       reinterpret_cast<float4*>(sx)[((k0 % EPV) >> 2) * nvecD + k0 / EPV] =
           make_float4(f[4 * g4], f[4 * g4 + 1], f[4 * g4 + 2], f[4 * g4 + 3]);
+    }
+    if (kLimbs) {
+#pragma unroll
+      for (int e = 0; e < XEPV; ++e) xmax = fmaxf(xmax, fabsf(f[e]));
+    }
+  }
+  if (kLimbs) {
+    // The token as three int8 limbs: x[k] = s (q0 + q1 / 128 + q2 / 128^2) up to s 2^-15, s = max |x| / 127 -- an
+    // error of 2.4e-7 max |x| per entry, the size of an fp32 rounding.  Limb plane l holds q_l of every k.
+    static_assert(!kLimbs || kStageThreads / 32 <= 16, "scratch for the staging warps' maxima");
+    xmax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(xmax)));
+    if (lane == 0) xl_scratch[(tid - kStageBase) >> 5] = xmax;
+    named_bar_sync(5, kStageThreads);
+    float mx = 0.f;
+#pragma unroll
+    for (int w = 0; w < kStageThreads / 32; ++w) mx = fmaxf(mx, xl_scratch[w]);
+    const float xs = mx > 0.f ? mx / 127.f : 1.f, inv = 1.f / xs;
+    named_bar_sync(5, kStageThreads);  // every warp has read the maxima: slot 16 may be written
+    if (tid == kStageBase) xl_scratch[16] = xs;
+    int8_t* planes = reinterpret_cast<int8_t*>(smem + L.xlimb + 128);
+    for (int cx = tid - kStageBase; cx < D / XEPV; cx += kStageThreads) {
+      float f[XEPV];
+      Elem<X>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + cx), f);
+      uint32_t q[3][XEPV / 4];
+#pragma unroll
+      for (int e = 0; e < XEPV; ++e) {
+        float t = fminf(fmaxf(f[e] * inv, -127.f), 127.f);
+#pragma unroll
+        for (int l = 0; l < 3; ++l) {
+          const float r = rintf(t);
+          const uint32_t b = (uint32_t)(int)r & 0xffu;
+          if ((e & 3) == 0) q[l][e >> 2] = b;
+          else q[l][e >> 2] |= b << (8 * (e & 3));
+          t = (t - r) * 128.f;
+        }
+      }
+#pragma unroll
+      for (int l = 0; l < 3; ++l)
+#pragma unroll
+        for (int g4 = 0; g4 < XEPV / 4; ++g4)
+          *reinterpret_cast<uint32_t*>(planes + (size_t)l * D + cx * XEPV + 4 * g4) = q[l][g4];
     }
   }
   if (LOPA) {
@@ -709,7 +758,38 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         }
       }
     }
-    if (EPV == 16) {
+    if constexpr (kLimbs) {
+      // int8 rows, standard gate: integer dot products against the token's three limbs (dp4a: four products per
+      // instruction, no conversion), two rows side by side so that they share the reads of the limbs; exact int32
+      // sums (at most 2^26 per row), recombined as s (A0 + A1 / 128 + A2 / 128^2).
+      const float xs = xl_scratch[16];
+      for (; rr_single < rows; rr_single += 2) {
+        const bool two = rr_single + 1 < rows;
+        const uint4* w0 = reinterpret_cast<const uint4*>(base + (size_t)rr_single * gate_row_bytes);
+        const uint4* w1 = reinterpret_cast<const uint4*>(base + (size_t)(rr_single + (two ? 1 : 0)) * gate_row_bytes);
+        int a0[3] = {0, 0, 0}, a1[3] = {0, 0, 0};
+        for (int c = lane; c < nvecK; c += 32) {
+          const uint4 u0 = w0[c], u1 = w1[c];
+#pragma unroll
+          for (int l = 0; l < 3; ++l) {
+            const uint4 xv = xl[l * nvecK + c];
+            a0[l] = __dp4a((int)u0.x, (int)xv.x, a0[l]); a0[l] = __dp4a((int)u0.y, (int)xv.y, a0[l]);
+            a0[l] = __dp4a((int)u0.z, (int)xv.z, a0[l]); a0[l] = __dp4a((int)u0.w, (int)xv.w, a0[l]);
+            a1[l] = __dp4a((int)u1.x, (int)xv.x, a1[l]); a1[l] = __dp4a((int)u1.y, (int)xv.y, a1[l]);
+            a1[l] = __dp4a((int)u1.z, (int)xv.z, a1[l]); a1[l] = __dp4a((int)u1.w, (int)xv.w, a1[l]);
+          }
+        }
+#pragma unroll
+        for (int l = 0; l < 3; ++l) {
+          a0[l] = __reduce_add_sync(0xffffffffu, a0[l]);
+          a1[l] = __reduce_add_sync(0xffffffffu, a1[l]);
+        }
+        const float z0 = xs * (((float)a0[0] + (float)a0[1] * 0.0078125f) + (float)a0[2] * 6.103515625e-05f);
+        const float z1 = xs * (((float)a1[0] + (float)a1[1] * 0.0078125f) + (float)a1[2] * 6.103515625e-05f);
+        if (lane == rr_single) mine = z0;
+        if (two && lane == rr_single + 1) mine = z1;
+      }
+    } else if (EPV == 16) {
       // int8 rows: the staged vector is four times the bytes of a row, so two rows share every read of it
       for (; rr_single + 1 < rows; rr_single += 2) {
         const uint4* w0 = reinterpret_cast<const uint4*>(base + (size_t)rr_single * gate_row_bytes);
@@ -1111,6 +1191,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       const unsigned char* s1 = act_slot(slot1);
       float part0 = 0.f, part1 = 0.f;
       float2 pk0 = make_float2(0.f, 0.f), pk1 = pk0, pk0b = pk0, pk1b = pk0;  // packed partial sums
+      int ia0[3] = {0, 0, 0}, ia1[3] = {0, 0, 0};                             // int8 rows, standard gate: integer sums per limb
       if (a0 >= 0.f) {
         const uint4* wu0 = reinterpret_cast<const uint4*>(s0);
         const uint4* wu1 = reinterpret_cast<const uint4*>(s1);
@@ -1118,7 +1199,19 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         for (int i = 0; i < CPT; ++i) {
           const int c = gat + i * kGT;
           if (c < nvecD) {
-            if constexpr (EPV == 16) {
+            if constexpr (kLimbs) {
+              const uint4 u0 = wu0[c], u1 = wu1[c];
+#pragma unroll
+              for (int l = 0; l < 3; ++l) {
+                const uint4 xv = xl[l * nvecD + c];
+                ia0[l] = __dp4a((int)u0.x, (int)xv.x, ia0[l]); ia0[l] = __dp4a((int)u0.y, (int)xv.y, ia0[l]);
+                ia0[l] = __dp4a((int)u0.z, (int)xv.z, ia0[l]); ia0[l] = __dp4a((int)u0.w, (int)xv.w, ia0[l]);
+                if (a1 >= 0.f) {
+                  ia1[l] = __dp4a((int)u1.x, (int)xv.x, ia1[l]); ia1[l] = __dp4a((int)u1.y, (int)xv.y, ia1[l]);
+                  ia1[l] = __dp4a((int)u1.z, (int)xv.z, ia1[l]); ia1[l] = __dp4a((int)u1.w, (int)xv.w, ia1[l]);
+                }
+              }
+            } else if constexpr (EPV == 16) {
               pk0 = chunk_dot_q8(wu0[c], sx, c, nvecD, pk0);
               if (a1 >= 0.f) pk1 = chunk_dot_q8(wu1[c], sx, c, nvecD, pk1);
             } else if constexpr (kXReg) {
@@ -1144,7 +1237,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
             }
           }
         }
-        if constexpr (EPV == 16) {
+        if constexpr (kLimbs) {
+          const float xs = xl_scratch[16];
+          part0 = xs * (((float)ia0[0] + (float)ia0[1] * 0.0078125f) + (float)ia0[2] * 6.103515625e-05f);
+          part1 = xs * (((float)ia1[0] + (float)ia1[1] * 0.0078125f) + (float)ia1[2] * 6.103515625e-05f);
+        } else if constexpr (EPV == 16) {
           part0 = pk0.x + pk0.y;
           part1 = pk1.x + pk1.y;
         } else if constexpr (kXReg) {
@@ -1389,7 +1486,8 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   g.gate_slot_bytes = (nr * gate_row_bytes + 127) / 128 * 128;
   g.act_slot_bytes = (2 * row_bytes + 127) / 128 * 128;
   g.slab_max = (((H + nr - 1) / nr + grid - 1) / grid) * nr;  // most rows one CTA can own
-  const SmemLayout fixed(D, K, lopa, 0, 0, 0, 0, g.slab_max, scaled);
+  const bool limbs = wkind == kWQ8 && !lopa;
+  const SmemLayout fixed(D, K, lopa, 0, 0, 0, 0, g.slab_max, scaled, 0, false, limbs);
   // slack for what the layout sizes by slot count: gate values and scales per act slot (<= 2 x 128 B), barrier words
   // (<= 2 x (24 + 16) x 8 B)
   const int ring = kSmemBudget - fixed.total - 1024;
@@ -1482,7 +1580,7 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
     const int most = gw + 8;  // the eight act warps of the LoPA kernel
     if (slots_of_cta <= ng) g.gate_workers = slots_of_cta < gw ? gw : slots_of_cta > most ? most : slots_of_cta;
   }
-  const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max, scaled, g.act_extra);
+  const SmemLayout full(D, K, lopa, ng, g.gate_slot_bytes, na, g.act_slot_bytes, g.slab_max, scaled, g.act_extra, false, limbs);
   g.smem = full.total;
   g.ok = g.smem <= kSmemBudget;
   return g;
