@@ -354,7 +354,13 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const int NG = p.n_gate_slots, NAown = p.n_act_slots, NA = p.act_used;
   // int8 rows under a standard gate: dot products in integers (dp4a) against the token split into int8 limbs
   constexpr bool kLimbs = EPV == 16 && !LOPA;
-  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra, GATED, kLimbs);
+  // int4 rows under a standard gate: the same, with every nibble used as the byte 16 x code (the nibble moved to the
+  // upper half of a byte) and the limbs of even and odd columns stored apart, as the two masks of a word deliver them
+  constexpr bool kLimbs4 = EPV == 32 && !LOPA;
+  // The gate uses the first two limbs (dp4a is the scarce resource there: 16-odd lanes per clock and SM): an error of
+  // 3e-5 max |x| per entry, about 1e-4 of a typical |z|.  The up projection, a tenth of the work, uses all three.
+  constexpr int kGateLimbs = 2;
+  const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra, GATED, kLimbs || kLimbs4);
 
   unsigned char* gate_ring = smem + L.gate_ring;
   unsigned char* act_ring = smem + L.act_ring;
@@ -531,15 +537,15 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       reinterpret_cast<float4*>(sx)[((k0 % EPV) >> 2) * nvecD + k0 / EPV] =
           make_float4(f[4 * g4], f[4 * g4 + 1], f[4 * g4 + 2], f[4 * g4 + 3]);
     }
-    if (kLimbs) {
+    if (kLimbs || kLimbs4) {
 #pragma unroll
       for (int e = 0; e < XEPV; ++e) xmax = fmaxf(xmax, fabsf(f[e]));
     }
   }
-  if (kLimbs) {
+  if (kLimbs || kLimbs4) {
     // The token as three int8 limbs: x[k] = s (q0 + q1 / 128 + q2 / 128^2) up to s 2^-15, s = max |x| / 127 -- an
     // error of 2.4e-7 max |x| per entry, the size of an fp32 rounding.  Limb plane l holds q_l of every k.
-    static_assert(!kLimbs || kStageThreads / 32 <= 16, "scratch for the staging warps' maxima");
+    static_assert(!(kLimbs || kLimbs4) || kStageThreads / 32 <= 16, "scratch for the staging warps' maxima");
     xmax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(xmax)));
     if (lane == 0) xl_scratch[(tid - kStageBase) >> 5] = xmax;
     named_bar_sync(5, kStageThreads);
@@ -566,11 +572,21 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
           t = (t - r) * 128.f;
         }
       }
+      if (kLimbs4) {
+        // the eight entries of this thread are one word's worth of nibbles: even columns, then odd columns
+        static_assert(!kLimbs4 || XEPV == 8, "bf16 token: eight entries per 16 bytes");
 #pragma unroll
-      for (int l = 0; l < 3; ++l)
+        for (int l = 0; l < 3; ++l) {
+          const uint32_t ev = __byte_perm(q[l][0], q[l][1], 0x6420), od = __byte_perm(q[l][0], q[l][1], 0x7531);
+          *reinterpret_cast<uint2*>(planes + (size_t)l * D + cx * 8) = make_uint2(ev, od);
+        }
+      } else {
 #pragma unroll
-        for (int g4 = 0; g4 < XEPV / 4; ++g4)
-          *reinterpret_cast<uint32_t*>(planes + (size_t)l * D + cx * XEPV + 4 * g4) = q[l][g4];
+        for (int l = 0; l < 3; ++l)
+#pragma unroll
+          for (int g4 = 0; g4 < XEPV / 4; ++g4)
+            *reinterpret_cast<uint32_t*>(planes + (size_t)l * D + cx * XEPV + 4 * g4) = q[l][g4];
+      }
     }
   }
   if (LOPA) {
@@ -728,7 +744,48 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       if (lane == rr_short) mine = z;
     }
     int rr_single = rows_short;
-    if constexpr (EPV == 32) {
+    if constexpr (kLimbs4) {
+      // 4-bit rows, standard gate: integer dot products (dp4a) of the bytes 16 x code with the token's limbs; up to four
+      // rows side by side share the reads of the limbs (96 bytes per 16-byte chunk of a row).
+      const float xs = xl_scratch[16] * 0.0625f;
+      for (; rr_single < rows; rr_single += 4) {
+        int acc[4][3];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i][0] = acc[i][1] = acc[i][2] = 0;
+        for (int c = lane; c < nvecK; c += 32) {
+          uint4 xv[3][2];
+#pragma unroll
+          for (int l = 0; l < kGateLimbs; ++l) {
+            xv[l][0] = xl[(l * nvecK + c) * 2];
+            xv[l][1] = xl[(l * nvecK + c) * 2 + 1];
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (rr_single + i < rows) {
+              const uint4 w = reinterpret_cast<const uint4*>(base + (size_t)(rr_single + i) * gate_row_bytes)[c];
+              const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const int ev = (int)((ww[k] << 4) & 0xf0f0f0f0u), od = (int)(ww[k] & 0xf0f0f0f0u);
+#pragma unroll
+                for (int l = 0; l < kGateLimbs; ++l) {
+                  const uint4 h = xv[l][k >> 1];
+                  acc[i][l] = __dp4a(ev, (int)((k & 1) ? h.z : h.x), acc[i][l]);
+                  acc[i][l] = __dp4a(od, (int)((k & 1) ? h.w : h.y), acc[i][l]);
+                }
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int s0 = __reduce_add_sync(0xffffffffu, acc[i][0]), s1 = __reduce_add_sync(0xffffffffu, acc[i][1]),
+                    s2 = __reduce_add_sync(0xffffffffu, acc[i][2]);
+          const float z = xs * (((float)s0 + (float)s1 * 0.0078125f) + (float)s2 * 6.103515625e-05f);
+          if (lane == rr_single + i) mine = z;
+        }
+      }
+    } else if constexpr (EPV == 32) {
       // 4-bit rows: the staged vector is eight times the bytes of a row.  Up to four rows are dotted side by side so
       // that every 128-byte read of it serves all of them; codes are unpacked in pairs and multiplied with packed FMAs.
       for (; rr_single < rows; rr_single += 4) {
@@ -771,7 +828,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         for (int c = lane; c < nvecK; c += 32) {
           const uint4 u0 = w0[c], u1 = w1[c];
 #pragma unroll
-          for (int l = 0; l < 3; ++l) {
+          for (int l = 0; l < kGateLimbs; ++l) {
             const uint4 xv = xl[l * nvecK + c];
             a0[l] = __dp4a((int)u0.x, (int)xv.x, a0[l]); a0[l] = __dp4a((int)u0.y, (int)xv.y, a0[l]);
             a0[l] = __dp4a((int)u0.z, (int)xv.z, a0[l]); a0[l] = __dp4a((int)u0.w, (int)xv.w, a0[l]);
@@ -1199,7 +1256,24 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
         for (int i = 0; i < CPT; ++i) {
           const int c = gat + i * kGT;
           if (c < nvecD) {
-            if constexpr (kLimbs) {
+            if constexpr (kLimbs4) {
+              const uint4 u0 = wu0[c], u1 = wu1[c];
+              const uint32_t w0[4] = {u0.x, u0.y, u0.z, u0.w}, w1[4] = {u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+              for (int l = 0; l < 3; ++l) {
+                const uint4 h0 = xl[(l * nvecD + c) * 2], h1 = xl[(l * nvecD + c) * 2 + 1];
+                const uint32_t xe[4] = {h0.x, h0.z, h1.x, h1.z}, xo[4] = {h0.y, h0.w, h1.y, h1.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  ia0[l] = __dp4a((int)((w0[k] << 4) & 0xf0f0f0f0u), (int)xe[k], ia0[l]);
+                  ia0[l] = __dp4a((int)(w0[k] & 0xf0f0f0f0u), (int)xo[k], ia0[l]);
+                  if (a1 >= 0.f) {
+                    ia1[l] = __dp4a((int)((w1[k] << 4) & 0xf0f0f0f0u), (int)xe[k], ia1[l]);
+                    ia1[l] = __dp4a((int)(w1[k] & 0xf0f0f0f0u), (int)xo[k], ia1[l]);
+                  }
+                }
+              }
+            } else if constexpr (kLimbs) {
               const uint4 u0 = wu0[c], u1 = wu1[c];
 #pragma unroll
               for (int l = 0; l < 3; ++l) {
@@ -1237,8 +1311,8 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
             }
           }
         }
-        if constexpr (kLimbs) {
-          const float xs = xl_scratch[16];
+        if constexpr (kLimbs || kLimbs4) {
+          const float xs = xl_scratch[16] * (kLimbs4 ? 0.0625f : 1.f);
           part0 = xs * (((float)ia0[0] + (float)ia0[1] * 0.0078125f) + (float)ia0[2] * 6.103515625e-05f);
           part1 = xs * (((float)ia1[0] + (float)ia1[1] * 0.0078125f) + (float)ia1[2] * 6.103515625e-05f);
         } else if constexpr (EPV == 16) {
@@ -1486,7 +1560,7 @@ Geometry plan(int wkind, int D, int H, int K, bool lopa, int grid) {
   g.gate_slot_bytes = (nr * gate_row_bytes + 127) / 128 * 128;
   g.act_slot_bytes = (2 * row_bytes + 127) / 128 * 128;
   g.slab_max = (((H + nr - 1) / nr + grid - 1) / grid) * nr;  // most rows one CTA can own
-  const bool limbs = wkind == kWQ8 && !lopa;
+  const bool limbs = (wkind == kWQ8 || wkind == kWQ4) && !lopa;
   const SmemLayout fixed(D, K, lopa, 0, 0, 0, 0, g.slab_max, scaled, 0, false, limbs);
   // slack for what the layout sizes by slot count: gate values and scales per act slot (<= 2 x 128 B), barrier words
   // (<= 2 x (24 + 16) x 8 B)
