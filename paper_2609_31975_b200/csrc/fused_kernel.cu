@@ -43,6 +43,7 @@ namespace {
 constexpr int kGateProducers = 2;                          // warps 0, 1
 constexpr int kFirstActProducer = kGateProducers;          // warps 2, 3
 constexpr int kActProducers = 2;
+constexpr int kTokenLimbs = 2;      // int8 limbs of the token (quantised rows, standard gate)
 constexpr int kFirstGateWarp = kFirstActProducer + kActProducers;
 constexpr int kGateWarps = 8;
 constexpr int kFirstActWarp = kFirstGateWarp + kGateWarps;
@@ -125,9 +126,9 @@ struct SmemLayout {
     // up to three barriers and three values
     gated_bars = take(gated ? 3 * 2 * n_act_slots * 8 : 0);
     gated_vals = take(gated ? 3 * 2 * n_act_slots * 4 : 0);
-    // int8 rows, standard gate: the token as three int8 limbs [3][D] for the integer dot products, after 128 bytes
-    // of scratch (the staging warps' maxima, then the limbs' scale)
-    xlimb = take(limbs ? 128 + 3 * D : 0);
+    // quantised rows, standard gate: the token as two int8 limbs [2][D] for the integer dot products (after 128 spare
+    // bytes), then one scale per 16 entries
+    xlimb = take(limbs ? 128 + kTokenLimbs * D + D / 4 : 0);
     total = off;
   }
 };
@@ -257,6 +258,9 @@ __device__ __forceinline__ void chunk_dot2_q8(const uint4& wa, const uint4& wb, 
     acc_b = fma2(hi, make_float2(v.z, v.w), acc_b);
   }
 }
+// A small integer (|a| < 2^22) as fp32 without a conversion instruction: 1.5 x 2^23 + a is exact, and so is the
+// subtraction.
+__device__ __forceinline__ float small_int_as_float(int a) { return __int_as_float(0x4B400000 + a) - 12582912.f; }
 // One int8 chunk against the staged vector, packed.
 __device__ __forceinline__ float2 chunk_dot_q8(const uint4& w, const float* vec, int c, int nvec, float2 acc) {
   const uint32_t a[4] = {w.x, w.y, w.z, w.w};
@@ -357,9 +361,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   // int4 rows under a standard gate: the same, with every nibble used as the byte 16 x code (the nibble moved to the
   // upper half of a byte) and the limbs of even and odd columns stored apart, as the two masks of a word deliver them
   constexpr bool kLimbs4 = EPV == 32 && !LOPA;
-  // The gate uses the first two limbs (dp4a is the scarce resource there: 16-odd lanes per clock and SM): an error of
-  // 3e-5 max |x| per entry, about 1e-4 of a typical |z|.  The up projection, a tenth of the work, uses all three.
-  constexpr int kGateLimbs = 2;
+  // Two limbs (dp4a is the scarce resource: 16-odd lanes per clock and SM; a third limb cost a third more gate time):
+  // an error of 3e-5 of the chunk's largest |x| per entry, about 1e-4 of a typical |z| or |u|.
+  constexpr int kGateLimbs = kTokenLimbs;
+  constexpr int kUpLimbs = kTokenLimbs;
   const SmemLayout L(D, K, LOPA, NG, p.gate_slot_bytes, NAown, p.act_slot_bytes, p.slab_max, kScaled, p.act_extra, GATED, kLimbs || kLimbs4);
 
   unsigned char* gate_ring = smem + L.gate_ring;
@@ -390,7 +395,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   float* slot_su = reinterpret_cast<float*>(smem + L.slot_scales);
   float* slot_sd = slot_su + NA;
   float* red = reinterpret_cast<float*>(smem + L.red);
-  float* xl_scratch = reinterpret_cast<float*>(smem + L.xlimb);          // [0..15] staging warps' max |x|, [16] limb scale
+  const float* xsc = reinterpret_cast<const float*>(smem + L.xlimb + 128 + kTokenLimbs * D);  // scale of the limbs of chunk c
   const uint4* xl = reinterpret_cast<const uint4*>(smem + L.xlimb + 128);  // limb l of chunk c: xl[l * nvecD + c]
   volatile int* ctl = reinterpret_cast<volatile int*>(smem + L.ctl);
   const uint32_t bars = smem_u32(smem + L.bars);
@@ -527,44 +532,45 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
   const uint32_t ep = (LOPA || warp >= kFirstGateWarp) ? __ldcg(p.epoch_word) + 1u : 0u;
   for (int i = tid - kStageBase; i < slab_rows; i += kStageThreads) row_state[i] = 0xffffffffu;
   constexpr int XEPV = Elem<X>::kPerVec;  // token elements per 16 bytes (the weights' EPV unless those are int8)
-  float xmax = 0.f;
-  for (int cx = tid - kStageBase; cx < D / XEPV; cx += kStageThreads) {
+  // Quantised rows under a standard gate: the token is also split, 16 (int8) or 32 (int4) entries at a time -- the
+  // entries one 16-byte chunk of a row meets -- into two int8 limbs and one scale per chunk:
+  // x[k] = s_c (q0 + q1 / 128) up to 3e-5 of the chunk's largest |x| (s_c = that maximum / 127), which is two orders
+  // below the step of the codes it is multiplied with.  A chunk's scale depends on its own entries only, so an
+  // outlier costs the precision of its own chunk and no other.
+  constexpr int kGroup = EPV / XEPV;  // threads that share a chunk of the token (2 or 4; 1 where not used)
+  int8_t* planes = reinterpret_cast<int8_t*>(smem + L.xlimb + 128);
+  float* xsc_w = reinterpret_cast<float*>(smem + L.xlimb + 128 + kTokenLimbs * D);
+  for (int cx0 = warp * 32 - kStageBase; cx0 < D / XEPV; cx0 += kStageThreads) {  // warp-uniform trip count (shuffles)
+    const int cx = cx0 + lane;
+    const bool on = cx < D / XEPV;
     float f[XEPV];
-    Elem<X>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + cx), f);
-#pragma unroll
-    for (int g4 = 0; g4 < XEPV / 4; ++g4) {
-      const int k0 = cx * XEPV + 4 * g4;  // first of four consecutive elements: quarter (k0 % EPV) / 4 of chunk k0 / EPV
-      reinterpret_cast<float4*>(sx)[((k0 % EPV) >> 2) * nvecD + k0 / EPV] =
-          make_float4(f[4 * g4], f[4 * g4 + 1], f[4 * g4 + 2], f[4 * g4 + 3]);
-    }
-    if (kLimbs || kLimbs4) {
-#pragma unroll
-      for (int e = 0; e < XEPV; ++e) xmax = fmaxf(xmax, fabsf(f[e]));
-    }
-  }
-  if (kLimbs || kLimbs4) {
-    // The token as three int8 limbs: x[k] = s (q0 + q1 / 128 + q2 / 128^2) up to s 2^-15, s = max |x| / 127 -- an
-    // error of 2.4e-7 max |x| per entry, the size of an fp32 rounding.  Limb plane l holds q_l of every k.
-    static_assert(!(kLimbs || kLimbs4) || kStageThreads / 32 <= 16, "scratch for the staging warps' maxima");
-    xmax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(xmax)));
-    if (lane == 0) xl_scratch[(tid - kStageBase) >> 5] = xmax;
-    named_bar_sync(5, kStageThreads);
-    float mx = 0.f;
-#pragma unroll
-    for (int w = 0; w < kStageThreads / 32; ++w) mx = fmaxf(mx, xl_scratch[w]);
-    const float xs = mx > 0.f ? mx / 127.f : 1.f, inv = 1.f / xs;
-    named_bar_sync(5, kStageThreads);  // every warp has read the maxima: slot 16 may be written
-    if (tid == kStageBase) xl_scratch[16] = xs;
-    int8_t* planes = reinterpret_cast<int8_t*>(smem + L.xlimb + 128);
-    for (int cx = tid - kStageBase; cx < D / XEPV; cx += kStageThreads) {
-      float f[XEPV];
+    if (on) {
       Elem<X>::unpack(__ldg(reinterpret_cast<const uint4*>(p.x) + cx), f);
-      uint32_t q[3][XEPV / 4];
 #pragma unroll
-      for (int e = 0; e < XEPV; ++e) {
+      for (int g4 = 0; g4 < XEPV / 4; ++g4) {
+        const int k0 = cx * XEPV + 4 * g4;  // first of four consecutive elements: quarter (k0 % EPV) / 4 of chunk k0 / EPV
+        reinterpret_cast<float4*>(sx)[((k0 % EPV) >> 2) * nvecD + k0 / EPV] =
+            make_float4(f[4 * g4], f[4 * g4 + 1], f[4 * g4 + 2], f[4 * g4 + 3]);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < XEPV; ++e) f[e] = 0.f;
+    }
+    if constexpr (kLimbs || kLimbs4) {
+      static_assert(!(kLimbs || kLimbs4) || XEPV == 8, "bf16 token: eight entries per 16 bytes");
+      float mx = 0.f;
+#pragma unroll
+      for (int e = 0; e < XEPV; ++e) mx = fmaxf(mx, fabsf(f[e]));
+#pragma unroll
+      for (int d = 1; d < kGroup; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+      const float xs = mx > 0.f ? mx / 127.f : 1.f, inv = 1.f / xs;
+      if (on && (cx & (kGroup - 1)) == 0) xsc_w[cx / kGroup] = xs;
+      uint32_t q[kTokenLimbs][2];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
         float t = fminf(fmaxf(f[e] * inv, -127.f), 127.f);
 #pragma unroll
-        for (int l = 0; l < 3; ++l) {
+        for (int l = 0; l < kTokenLimbs; ++l) {
           const float r = rintf(t);
           const uint32_t b = (uint32_t)(int)r & 0xffu;
           if ((e & 3) == 0) q[l][e >> 2] = b;
@@ -572,20 +578,16 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
           t = (t - r) * 128.f;
         }
       }
-      if (kLimbs4) {
-        // the eight entries of this thread are one word's worth of nibbles: even columns, then odd columns
-        static_assert(!kLimbs4 || XEPV == 8, "bf16 token: eight entries per 16 bytes");
+      if (on) {
 #pragma unroll
-        for (int l = 0; l < 3; ++l) {
-          const uint32_t ev = __byte_perm(q[l][0], q[l][1], 0x6420), od = __byte_perm(q[l][0], q[l][1], 0x7531);
-          *reinterpret_cast<uint2*>(planes + (size_t)l * D + cx * 8) = make_uint2(ev, od);
+        for (int l = 0; l < kTokenLimbs; ++l) {
+          if (kLimbs4) {  // one word's worth of nibbles: even columns, then odd columns
+            const uint32_t ev = __byte_perm(q[l][0], q[l][1], 0x6420), od = __byte_perm(q[l][0], q[l][1], 0x7531);
+            *reinterpret_cast<uint2*>(planes + (size_t)l * D + cx * 8) = make_uint2(ev, od);
+          } else {
+            *reinterpret_cast<uint2*>(planes + (size_t)l * D + cx * 8) = make_uint2(q[l][0], q[l][1]);
+          }
         }
-      } else {
-#pragma unroll
-        for (int l = 0; l < 3; ++l)
-#pragma unroll
-          for (int g4 = 0; g4 < XEPV / 4; ++g4)
-            *reinterpret_cast<uint32_t*>(planes + (size_t)l * D + cx * XEPV + 4 * g4) = q[l][g4];
       }
     }
   }
@@ -747,41 +749,44 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
     if constexpr (kLimbs4) {
       // 4-bit rows, standard gate: integer dot products (dp4a) of the bytes 16 x code with the token's limbs; up to four
       // rows side by side share the reads of the limbs (96 bytes per 16-byte chunk of a row).
-      const float xs = xl_scratch[16] * 0.0625f;
+      // The integer sums of a chunk are exact and small; they are scaled by the chunk's limb scale and added in fp32.
       for (; rr_single < rows; rr_single += 4) {
-        int acc[4][3];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[i][0] = acc[i][1] = acc[i][2] = 0;
+        float facc[4] = {0.f, 0.f, 0.f, 0.f};
         for (int c = lane; c < nvecK; c += 32) {
-          uint4 xv[3][2];
+          uint4 xv[kGateLimbs][2];
 #pragma unroll
           for (int l = 0; l < kGateLimbs; ++l) {
             xv[l][0] = xl[(l * nvecK + c) * 2];
             xv[l][1] = xl[(l * nvecK + c) * 2 + 1];
           }
+          const float sc = xsc[c];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             if (rr_single + i < rows) {
               const uint4 w = reinterpret_cast<const uint4*>(base + (size_t)(rr_single + i) * gate_row_bytes)[c];
               const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+              int acc[kGateLimbs];
+#pragma unroll
+              for (int l = 0; l < kGateLimbs; ++l) acc[l] = 0;
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
                 const int ev = (int)((ww[k] << 4) & 0xf0f0f0f0u), od = (int)(ww[k] & 0xf0f0f0f0u);
 #pragma unroll
                 for (int l = 0; l < kGateLimbs; ++l) {
                   const uint4 h = xv[l][k >> 1];
-                  acc[i][l] = __dp4a(ev, (int)((k & 1) ? h.z : h.x), acc[i][l]);
-                  acc[i][l] = __dp4a(od, (int)((k & 1) ? h.w : h.y), acc[i][l]);
+                  acc[l] = __dp4a(ev, (int)((k & 1) ? h.z : h.x), acc[l]);
+                  acc[l] = __dp4a(od, (int)((k & 1) ? h.w : h.y), acc[l]);
                 }
               }
+              float v = small_int_as_float(acc[0]);
+              if (kGateLimbs > 1) v = fmaf(small_int_as_float(acc[1]), 0.0078125f, v);
+              facc[i] = fmaf(v, sc, facc[i]);
             }
           }
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int s0 = __reduce_add_sync(0xffffffffu, acc[i][0]), s1 = __reduce_add_sync(0xffffffffu, acc[i][1]),
-                    s2 = __reduce_add_sync(0xffffffffu, acc[i][2]);
-          const float z = xs * (((float)s0 + (float)s1 * 0.0078125f) + (float)s2 * 6.103515625e-05f);
+          const float z = warp_sum(facc[i]) * 0.0625f;
           if (lane == rr_single + i) mine = z;
         }
       }
@@ -819,30 +824,32 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       // int8 rows, standard gate: integer dot products against the token's three limbs (dp4a: four products per
       // instruction, no conversion), two rows side by side so that they share the reads of the limbs; exact int32
       // sums (at most 2^26 per row), recombined as s (A0 + A1 / 128 + A2 / 128^2).
-      const float xs = xl_scratch[16];
       for (; rr_single < rows; rr_single += 2) {
         const bool two = rr_single + 1 < rows;
         const uint4* w0 = reinterpret_cast<const uint4*>(base + (size_t)rr_single * gate_row_bytes);
         const uint4* w1 = reinterpret_cast<const uint4*>(base + (size_t)(rr_single + (two ? 1 : 0)) * gate_row_bytes);
-        int a0[3] = {0, 0, 0}, a1[3] = {0, 0, 0};
+        float f0 = 0.f, f1 = 0.f;
         for (int c = lane; c < nvecK; c += 32) {
           const uint4 u0 = w0[c], u1 = w1[c];
+          int a0[kGateLimbs], a1[kGateLimbs];
 #pragma unroll
           for (int l = 0; l < kGateLimbs; ++l) {
             const uint4 xv = xl[l * nvecK + c];
-            a0[l] = __dp4a((int)u0.x, (int)xv.x, a0[l]); a0[l] = __dp4a((int)u0.y, (int)xv.y, a0[l]);
+            a0[l] = __dp4a((int)u0.x, (int)xv.x, 0); a0[l] = __dp4a((int)u0.y, (int)xv.y, a0[l]);
             a0[l] = __dp4a((int)u0.z, (int)xv.z, a0[l]); a0[l] = __dp4a((int)u0.w, (int)xv.w, a0[l]);
-            a1[l] = __dp4a((int)u1.x, (int)xv.x, a1[l]); a1[l] = __dp4a((int)u1.y, (int)xv.y, a1[l]);
+            a1[l] = __dp4a((int)u1.x, (int)xv.x, 0); a1[l] = __dp4a((int)u1.y, (int)xv.y, a1[l]);
             a1[l] = __dp4a((int)u1.z, (int)xv.z, a1[l]); a1[l] = __dp4a((int)u1.w, (int)xv.w, a1[l]);
           }
+          const float sc = xsc[c];
+          float v0 = small_int_as_float(a0[0]), v1 = small_int_as_float(a1[0]);
+          if (kGateLimbs > 1) {
+            v0 = fmaf(small_int_as_float(a0[1]), 0.0078125f, v0);
+            v1 = fmaf(small_int_as_float(a1[1]), 0.0078125f, v1);
+          }
+          f0 = fmaf(v0, sc, f0);
+          f1 = fmaf(v1, sc, f1);
         }
-#pragma unroll
-        for (int l = 0; l < 3; ++l) {
-          a0[l] = __reduce_add_sync(0xffffffffu, a0[l]);
-          a1[l] = __reduce_add_sync(0xffffffffu, a1[l]);
-        }
-        const float z0 = xs * (((float)a0[0] + (float)a0[1] * 0.0078125f) + (float)a0[2] * 6.103515625e-05f);
-        const float z1 = xs * (((float)a1[0] + (float)a1[1] * 0.0078125f) + (float)a1[2] * 6.103515625e-05f);
+        const float z0 = warp_sum(f0), z1 = warp_sum(f1);
         if (lane == rr_single) mine = z0;
         if (two && lane == rr_single + 1) mine = z1;
       }
@@ -1248,7 +1255,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
       const unsigned char* s1 = act_slot(slot1);
       float part0 = 0.f, part1 = 0.f;
       float2 pk0 = make_float2(0.f, 0.f), pk1 = pk0, pk0b = pk0, pk1b = pk0;  // packed partial sums
-      int ia0[3] = {0, 0, 0}, ia1[3] = {0, 0, 0};                             // int8 rows, standard gate: integer sums per limb
+      int ia0[kTokenLimbs] = {0, 0}, ia1[kTokenLimbs] = {0, 0};                             // quantised rows, standard gate: a chunk's integer sums per limb
       if (a0 >= 0.f) {
         const uint4* wu0 = reinterpret_cast<const uint4*>(s0);
         const uint4* wu1 = reinterpret_cast<const uint4*>(s1);
@@ -1260,7 +1267,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
               const uint4 u0 = wu0[c], u1 = wu1[c];
               const uint32_t w0[4] = {u0.x, u0.y, u0.z, u0.w}, w1[4] = {u1.x, u1.y, u1.z, u1.w};
 #pragma unroll
-              for (int l = 0; l < 3; ++l) {
+              for (int l = 0; l < kUpLimbs; ++l) {
                 const uint4 h0 = xl[(l * nvecD + c) * 2], h1 = xl[(l * nvecD + c) * 2 + 1];
                 const uint32_t xe[4] = {h0.x, h0.z, h1.x, h1.z}, xo[4] = {h0.y, h0.w, h1.y, h1.w};
 #pragma unroll
@@ -1273,10 +1280,18 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
                   }
                 }
               }
+              {  // the chunk's integer sums, scaled by its limb scale, join the fp32 sums
+                const float sc = xsc[c];
+                const float v0 = fmaf(small_int_as_float(ia0[1]), 0.0078125f, small_int_as_float(ia0[0]));
+                const float v1 = fmaf(small_int_as_float(ia1[1]), 0.0078125f, small_int_as_float(ia1[0]));
+                part0 = fmaf(v0, sc, part0);
+                part1 = fmaf(v1, sc, part1);
+                ia0[0] = ia0[1] = ia1[0] = ia1[1] = 0;
+              }
             } else if constexpr (kLimbs) {
               const uint4 u0 = wu0[c], u1 = wu1[c];
 #pragma unroll
-              for (int l = 0; l < 3; ++l) {
+              for (int l = 0; l < kUpLimbs; ++l) {
                 const uint4 xv = xl[l * nvecD + c];
                 ia0[l] = __dp4a((int)u0.x, (int)xv.x, ia0[l]); ia0[l] = __dp4a((int)u0.y, (int)xv.y, ia0[l]);
                 ia0[l] = __dp4a((int)u0.z, (int)xv.z, ia0[l]); ia0[l] = __dp4a((int)u0.w, (int)xv.w, ia0[l]);
@@ -1284,6 +1299,14 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
                   ia1[l] = __dp4a((int)u1.x, (int)xv.x, ia1[l]); ia1[l] = __dp4a((int)u1.y, (int)xv.y, ia1[l]);
                   ia1[l] = __dp4a((int)u1.z, (int)xv.z, ia1[l]); ia1[l] = __dp4a((int)u1.w, (int)xv.w, ia1[l]);
                 }
+              }
+              {  // the chunk's integer sums, scaled by its limb scale, join the fp32 sums
+                const float sc = xsc[c];
+                const float v0 = fmaf(small_int_as_float(ia0[1]), 0.0078125f, small_int_as_float(ia0[0]));
+                const float v1 = fmaf(small_int_as_float(ia1[1]), 0.0078125f, small_int_as_float(ia1[0]));
+                part0 = fmaf(v0, sc, part0);
+                part1 = fmaf(v1, sc, part1);
+                ia0[0] = ia0[1] = ia1[0] = ia1[1] = 0;
               }
             } else if constexpr (EPV == 16) {
               pk0 = chunk_dot_q8(wu0[c], sx, c, nvecD, pk0);
@@ -1312,9 +1335,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_ffn_kernel(const FusedParam
           }
         }
         if constexpr (kLimbs || kLimbs4) {
-          const float xs = xl_scratch[16] * (kLimbs4 ? 0.0625f : 1.f);
-          part0 = xs * (((float)ia0[0] + (float)ia0[1] * 0.0078125f) + (float)ia0[2] * 6.103515625e-05f);
-          part1 = xs * (((float)ia1[0] + (float)ia1[1] * 0.0078125f) + (float)ia1[2] * 6.103515625e-05f);
+          if (kLimbs4) {  // the bytes were 16 x code
+            part0 *= 0.0625f;
+            part1 *= 0.0625f;
+          }
         } else if constexpr (EPV == 16) {
           part0 = pk0.x + pk0.y;
           part1 = pk1.x + pk1.y;
