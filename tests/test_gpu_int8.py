@@ -303,3 +303,39 @@ def test_random_shapes_quantised_batches_agree_with_the_single_token_kernel(mod,
         assert torch.equal(y, y2), f"{what} repeat"
         torch.cuda.synchronize()
         assert ffn.device_status() == 0, f"{what}: status words {ffn.status_words()}"
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_quantised_rows_with_outliers_in_the_token(mod, bits):
+    """The integer routes split the token into int8 limbs: per 16-byte chunk of a row in the single-token kernel, per
+    token in the batch kernels.  Entries a thousand times the rest (as activations of language models have) must not
+    cost the other entries their precision."""
+    D, H = 2048, 3000
+    w = (syn.standard_ffn_q8 if bits == 8 else syn.standard_ffn_q4)(D, H, 77, DEV, sparsity=0.8)
+    gate = {"W_g": w["W_g"]}
+    x = syn.tokens(6, D, torch.bfloat16, 77, DEV).clone()
+    x[:, 5] *= 1000.0
+    x[1, 777] *= -300.0
+    x[2, 1024:] *= 1e-3
+    ffn = mod.SparseFFN(D, H, torch.bfloat16, B_max=6)
+    oracle_ffn = oracle.ffn_q8 if bits == 8 else oracle.ffn_q4
+    f = ffn.sparse_ffn_forward_q8 if bits == 8 else ffn.sparse_ffn_forward_q4
+    ref = oracle_ffn(host(x), hq(w["W_up"]), hq(w["W_down"]), "relu", b_g=host(w["b_g"]), threads=8, W_g=hq(gate["W_g"]))
+    def same_fired_set(got_idx, z, what):
+        # the outliers scale every z by hundreds, so the dead band of the fired-set check is taken relative to max |z|
+        z = z if z.ndim == 2 else z[None, :]
+        got = np.zeros(z.shape[1], bool)
+        got[got_idx.cpu().numpy()] = True
+        diff = np.nonzero(got != (z > 0).any(axis=0))[0]
+        band = 1e-4 * np.abs(z).max()
+        assert all((np.abs(z[:, j]) < band).any() and not (z[:, j] >= band).any() for j in diff), f"{what}: {len(diff)} differ"
+
+    for t in range(3):                                           # one token: integer dot products, limbs per chunk
+        y = f(x[t], gate, w["b_g"], w["W_up"], w["W_down"], "relu")
+        assert_y_close(y, ref["y"][t], rel_l2=TOL, max_abs=TOL, what=f"int{bits} outlier token {t}")
+        same_fired_set(ffn.last_active(), ref["z"][t], f"int{bits} outlier token {t}")
+    y = f(x, gate, w["b_g"], w["W_up"], w["W_down"], "relu")     # the batch: int8 MMAs, four limbs per token
+    assert_y_close(y, ref["y"], what=f"int{bits} outlier batch")
+    same_fired_set(ffn.last_active(), ref["z"], f"int{bits} outlier batch")
+    torch.cuda.synchronize()
+    assert ffn.device_status() == 0
