@@ -177,14 +177,17 @@ int dense_ffn_forward(sffn_handle* handle, const void* x, int B, const sffn_gate
  * int8 codes ([H,D], [H,D], [H,D], [r,D], [H,r]); `scales` carries the row scales.  Tokens x are bf16: the handle
  * must have been created with SFFN_BF16.  Rows must be a multiple of 16 bytes (D and r multiples of 16).
  * Everything else (b_g, g_idx, g_sign, RMSNorm, act, y, the active list, double activation) is as in
- * sparse_ffn_forward / dense_ffn_forward.  One token runs in the fused kernel; a batch runs the tcgen05 batch
- * kernels (D and r multiples of 64, D of 256; otherwise, or under SFFN_PATH_FUSED, the fused kernel once per token; the
+ * sparse_ffn_forward / dense_ffn_forward.  One token runs in the fused kernel; under a standard gate its gate and up
+ * dot products are integer ones (dp4a) against the token split, 16 entries at a time, into two int8 limbs and a
+ * scale (x = s_c (q0 + q1/128) up to 3e-5 of the largest |x| among those 16 entries; int4: 32 entries, nibbles used
+ * as the bytes 16 x code), all sums in fp32 beyond a chunk; LoPA gates use fp32 arithmetic throughout.  A batch runs
+ * the tcgen05 batch kernels (D and r multiples of 64, D of 256; otherwise, or under SFFN_PATH_FUSED, the fused kernel once per token; the
  * list of fired neurons is the union over the tokens).  There the gate and up products of int8 rows are int8 x int8
  * with int32 accumulators, each token entering as four int8 limbs and a scale (x = s (q0 + q1/128 + q2/128^2 +
  * q3/128^3) up to 2^-22 max|x|; D and r multiples of 128; int4 rows take the same route, their nibbles expanded to
  * int8 in shared memory), and the down product and other widths expand the codes to bf16 in shared memory; row scales
- * are applied to the accumulator rows.  The CUDA-core batch kernels
- * serve SFFN_PATH_GENERAL (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is
+ * are applied to the accumulator rows.  The CUDA-core kernels (fp32 arithmetic on the decoded codes) serve
+ * SFFN_PATH_GENERAL (SFFN_PATH_MMA_SYNC: SFFN_ERR_UNSUPPORTED).  Converting a trained model to this format is
  * an offline step outside this library. */
 typedef struct {
   const float* s_gate; /* [H]  row scales of W_g (STANDARD) or of U (LOPA) */
